@@ -1,0 +1,261 @@
+"""fp64 CPU oracle for the CAAT-Net row-parallel hot path.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain definition that the
+CUDA path is checked against.  It shares no code with the CUDA path and is
+imported only by the tests, by the smoke check and by the benchmark's
+CPU-baseline leg.  Nothing in the product path may call it.
+
+Everything is numpy float64.  Inputs are expected to be already rounded to the
+run's storage type by the caller (the harness) and widened to float64, so the
+oracle and the GPU see the same values.
+
+Notation (paper's symbols in brackets):
+  t        tensor-parallel ranks               [r, M; rank index m]
+  T        tokens                              [b x t, s]
+  h        hidden size                         [h]
+  K_r      per-rank contraction width          [f / r]
+  S        shared channels = floor(h * p)      [floor(hp), Eq. A3]
+  alpha    private-channel scale, 1 or sqrt(t) [sqrt(r), Section 4 "Private channel scaling"]
+  Y[m]     rank m's input  [T, K_r]            [Y_m, H_m]
+  W[m]     rank m's weight shard stored out x in, [h, K_r]   [B~_{klm} as W[m][l][k]]
+  Zt[m]    rank m's partial output [T, h]      [Z~_{ilm}]
+  R[m]     residual entering the add           [R, R_m]
+  Hn[m]    Z[m] + R[m], the new residual stream
+  X[m]     Norm(Hn[m])                         [X_m, Eq. 9]
+
+Pins (see tests/test_oracle_pins.py): the two-device closed form of Eq. 8, a
+brute-force index-notation evaluation of Eq. A3, p=1 against an unsharded
+library matmul plus library norms, p=0 independence, rank-permutation
+invariance, the variance law of Eq. 14-15, central finite differences and the
+p=1 reduce-before-norm equivalence of Section 4 for the backward, and the
+closed forms of Appendix C for the byte counts.
+
+Parity unpinned (the paper fixes no value; these are this build's documented
+choices): eps, the norm kind per model, the default of alpha, the dtype of dW.
+The paper prints no worked numeric example of the operator, so no pin is a
+printed value; all pins are closed forms, invariants and special cases.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+RMSNORM = 0
+LAYERNORM = 1
+
+
+# --------------------------------------------------------------------------
+# F0: partition  (Section 3: the first h*p channels are shared; Eq. A3 floor(hp))
+# --------------------------------------------------------------------------
+def shared_channels(h: int, p: float) -> int:
+    """S = floor(h * p) evaluated in IEEE double, as Eq. A3 writes it."""
+    if not (0.0 <= p <= 1.0):
+        raise ValueError("p must lie in [0, 1]")
+    return int(math.floor(float(h) * float(p)))
+
+
+def private_scale(t: int, enabled: bool = True) -> float:
+    """Section 4, private channel scaling: sqrt(r) when on, 1 when off."""
+    return math.sqrt(float(t)) if enabled else 1.0
+
+
+# --------------------------------------------------------------------------
+# F1: per-rank GEMM  (Eq. A3 first line / Eq. A5 second line)
+# --------------------------------------------------------------------------
+def rank_partials(Y: np.ndarray, W: np.ndarray) -> np.ndarray:
+    """Zt[m, i, l] = sum_k Y[m, i, k] * W[m, l, k]."""
+    Y = np.asarray(Y, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    t = Y.shape[0]
+    return np.stack([Y[m] @ W[m].T for m in range(t)], axis=0)
+
+
+# --------------------------------------------------------------------------
+# F2 + F3: partial channel-reduce with private scaling  (Eq. A3 cases; Section 4)
+# --------------------------------------------------------------------------
+def partial_channel_reduce(Zt: np.ndarray, S: int, alpha: float = 1.0) -> np.ndarray:
+    """Z[m, i, l] = sum_m' Zt[m', i, l] for l < S, alpha * Zt[m, i, l] for l >= S.
+
+    The rank sum runs m' = 0 .. t-1 in that order.
+    """
+    Zt = np.asarray(Zt, dtype=np.float64)
+    t = Zt.shape[0]
+    Z = np.empty_like(Zt)
+    if S > 0:
+        Zs = np.zeros_like(Zt[0, :, :S])
+        for m in range(t):
+            Zs = Zs + Zt[m, :, :S]
+        for m in range(t):
+            Z[m, :, :S] = Zs
+    Z[:, :, S:] = alpha * Zt[:, :, S:]
+    return Z
+
+
+# --------------------------------------------------------------------------
+# F5: per-rank norm over all h channels of that rank  (Eq. 9; RMSNorm / LayerNorm)
+# --------------------------------------------------------------------------
+def norm_forward(Hn: np.ndarray, gamma: np.ndarray, beta, eps: float, norm: int):
+    """Returns X, rstd, mean (mean is None for RMSNorm). Statistics per (rank, token)."""
+    Hn = np.asarray(Hn, dtype=np.float64)
+    gamma = np.asarray(gamma, dtype=np.float64)
+    if norm == RMSNORM:
+        ms = np.mean(Hn * Hn, axis=-1)
+        rstd = 1.0 / np.sqrt(ms + eps)
+        X = Hn * rstd[..., None] * gamma
+        return X, rstd, None
+    if norm == LAYERNORM:
+        mu = np.mean(Hn, axis=-1)
+        c = Hn - mu[..., None]
+        var = np.mean(c * c, axis=-1)
+        rstd = 1.0 / np.sqrt(var + eps)
+        X = c * rstd[..., None] * gamma
+        if beta is not None:
+            X = X + np.asarray(beta, dtype=np.float64)
+        return X, rstd, mu
+    raise ValueError("unknown norm kind")
+
+
+# --------------------------------------------------------------------------
+# Forward of one row-parallel sub-layer  (F1..F5)
+# --------------------------------------------------------------------------
+def rowpar_forward(Y, W, R, gamma, beta=None, *, S: int, alpha: float = 1.0,
+                   eps: float = 1e-5, norm: int = RMSNORM) -> dict:
+    Zt = rank_partials(Y, W)                                  # F1
+    Z = partial_channel_reduce(Zt, S, alpha)                  # F2, F3
+    Hn = Z + np.asarray(R, dtype=np.float64)                  # F4 (Eq. 9 argument)
+    X, rstd, mean = norm_forward(Hn, gamma, beta, eps, norm)  # F5
+    return {"Zt": Zt, "Z": Z, "Hn": Hn, "X": X, "rstd": rstd, "mean": mean}
+
+
+# --------------------------------------------------------------------------
+# B1: norm backward (textbook) + residual gradient
+# --------------------------------------------------------------------------
+def norm_backward(dX, Hn, rstd, mean, gamma, norm: int) -> np.ndarray:
+    """Gradient of X = Norm(Hn) w.r.t. Hn contracted with dX, per (rank, token) row."""
+    dX = np.asarray(dX, dtype=np.float64)
+    Hn = np.asarray(Hn, dtype=np.float64)
+    rstd = np.asarray(rstd, dtype=np.float64)[..., None]
+    gamma = np.asarray(gamma, dtype=np.float64)
+    dxh = dX * gamma
+    if norm == RMSNORM:
+        xh = Hn * rstd
+        c = np.mean(dxh * xh, axis=-1, keepdims=True)
+        return rstd * (dxh - xh * c)
+    if norm == LAYERNORM:
+        mu = np.asarray(mean, dtype=np.float64)[..., None]
+        xh = (Hn - mu) * rstd
+        c1 = np.mean(dxh, axis=-1, keepdims=True)
+        c2 = np.mean(dxh * xh, axis=-1, keepdims=True)
+        return rstd * (dxh - c1 - xh * c2)
+    raise ValueError("unknown norm kind")
+
+
+def normalized(Hn, rstd, mean, norm: int) -> np.ndarray:
+    """x_hat, the normalised row before gain and bias."""
+    Hn = np.asarray(Hn, dtype=np.float64)
+    rstd = np.asarray(rstd, dtype=np.float64)[..., None]
+    if norm == RMSNORM:
+        return Hn * rstd
+    return (Hn - np.asarray(mean, dtype=np.float64)[..., None]) * rstd
+
+
+def residual_stream_gradient(dX, dHn, Hn, rstd, mean, gamma, norm: int) -> np.ndarray:
+    """B1/B2: g[m] = NormBwd(dX[m]) + dHn[m]; this is also dR[m] (not reduced over ranks)."""
+    g = norm_backward(dX, Hn, rstd, mean, gamma, norm)
+    if dHn is not None:
+        g = g + np.asarray(dHn, dtype=np.float64)
+    return g
+
+
+def norm_param_gradients(dX, Hn, rstd, mean, norm: int):
+    """B3: dgamma[l] = sum_m sum_i dX*x_hat ; dbeta[l] = sum_m sum_i dX (LayerNorm only).
+
+    Summed over ranks as Section 4 requires for replicated norm parameters.
+    """
+    dX = np.asarray(dX, dtype=np.float64)
+    xh = normalized(Hn, rstd, mean, norm)
+    dgamma = np.sum(dX * xh, axis=(0, 1))
+    dbeta = np.sum(dX, axis=(0, 1)) if norm == LAYERNORM else None
+    return dgamma, dbeta
+
+
+def backward_partial_channel_reduce(g, S: int, alpha: float = 1.0) -> np.ndarray:
+    """B4: the reduce placed after the norm's backward (operation 'h' of Fig. 2b).
+
+    dZt[m, i, l] = sum_m' g[m', i, l] for l < S, alpha * g[m, i, l] for l >= S.
+    It is the transpose of the forward partial channel-reduce.
+    """
+    return partial_channel_reduce(np.asarray(g, dtype=np.float64), S, alpha)
+
+
+def data_gradient(dZt, W) -> np.ndarray:
+    """B5: dY[m, i, k] = sum_l dZt[m, i, l] * W[m, l, k]."""
+    W = np.asarray(W, dtype=np.float64)
+    return np.stack([dZt[m] @ W[m] for m in range(dZt.shape[0])], axis=0)
+
+
+def weight_gradient(dZt, Y) -> np.ndarray:
+    """B6: dW[m, l, k] = sum_i dZt[m, i, l] * Y[m, i, k]."""
+    Y = np.asarray(Y, dtype=np.float64)
+    return np.stack([dZt[m].T @ Y[m] for m in range(dZt.shape[0])], axis=0)
+
+
+def rowpar_backward(dX, dHn, Y, W, Hn, rstd, mean, gamma, *, S: int, alpha: float = 1.0,
+                    norm: int = RMSNORM) -> dict:
+    """Exact gradient of rowpar_forward w.r.t. (Y, W, R, gamma, beta), contracted with
+    upstream dX (through the norm) and dHn (through the residual stream)."""
+    g = residual_stream_gradient(dX, dHn, Hn, rstd, mean, gamma, norm)   # B1
+    dgamma, dbeta = norm_param_gradients(dX, Hn, rstd, mean, norm)       # B3
+    dZt = backward_partial_channel_reduce(g, S, alpha)                   # B4
+    dY = data_gradient(dZt, W)                                           # B5
+    dW = weight_gradient(dZt, Y)                                         # B6
+    return {"g": g, "dR": g, "dZt": dZt, "dY": dY, "dW": dW, "dgamma": dgamma, "dbeta": dbeta}
+
+
+# --------------------------------------------------------------------------
+# V2: block = attention-out sub-layer then MLP-down sub-layer (two reduces per block,
+# Appendix C), chained only through the residual stream.
+# --------------------------------------------------------------------------
+def block_forward(Y_attn, W_o, Y_mlp, W_down, R0, gamma1, gamma2, beta1=None, beta2=None, *,
+                  S: int, alpha: float = 1.0, eps: float = 1e-5, norm: int = RMSNORM) -> dict:
+    f1 = rowpar_forward(Y_attn, W_o, R0, gamma1, beta1, S=S, alpha=alpha, eps=eps, norm=norm)
+    f2 = rowpar_forward(Y_mlp, W_down, f1["Hn"], gamma2, beta2, S=S, alpha=alpha, eps=eps, norm=norm)
+    return {"Hn1": f1["Hn"], "X1": f1["X"], "rstd1": f1["rstd"], "mean1": f1["mean"],
+            "Hn2": f2["Hn"], "X2": f2["X"], "rstd2": f2["rstd"], "mean2": f2["mean"]}
+
+
+def block_backward(dX1, dX2, dHn2, Y_attn, W_o, Y_mlp, W_down, Hn1, rstd1, mean1, Hn2, rstd2,
+                   mean2, gamma1, gamma2, *, S: int, alpha: float = 1.0, norm: int = RMSNORM) -> dict:
+    b2 = rowpar_backward(dX2, dHn2, Y_mlp, W_down, Hn2, rstd2, mean2, gamma2, S=S, alpha=alpha, norm=norm)
+    b1 = rowpar_backward(dX1, b2["dR"], Y_attn, W_o, Hn1, rstd1, mean1, gamma1, S=S, alpha=alpha, norm=norm)
+    return {"dY_attn": b1["dY"], "dW_o": b1["dW"], "dY_mlp": b2["dY"], "dW_down": b2["dW"],
+            "dR0": b1["dR"], "dHn1": b2["dR"], "dgamma1": b1["dgamma"], "dgamma2": b2["dgamma"],
+            "dbeta1": b1["dbeta"], "dbeta2": b2["dbeta"]}
+
+
+# --------------------------------------------------------------------------
+# V3: analytic collective bytes  (Appendix C payload P(p); Appendix D volume law)
+# --------------------------------------------------------------------------
+def allreduce_bytes(tokens: int, h: int, t: int, S: int, elem_bytes: int = 2) -> dict:
+    """Bytes a real tensor-parallel system would move for ONE partial channel-reduce.
+
+    payload_per_rank:     tokens * S * e   (each device sends and receives that many activations)
+    payload_per_rank_p1:  tokens * h * e   (the full all-reduce, p = 1)
+    ring_wire_per_rank:   2 (t-1)/t * payload  (reduce-scatter + all-gather halves)
+    """
+    payload = tokens * S * elem_bytes
+    payload_p1 = tokens * h * elem_bytes
+    ring_num = 2 * (t - 1) * payload
+    return {"payload_per_rank": payload, "payload_per_rank_p1": payload_p1,
+            "ring_wire_per_rank": ring_num // t if ring_num % t == 0 else ring_num / t,
+            "norm_grad_sync_bytes": h * 4}
+
+
+def speedup_model(h: int, s: int, r: int, C: float, p: float) -> float:
+    """Appendix C: (T(1) - T(p)) / T(1) with T = G/C' + P, written directly from
+    G = (24 s h^2 + 4 s^2 h) / r, P(p) = 2 s h p and compute/communication ratio C."""
+    G = (24.0 * s * h * h + 4.0 * s * s * h) / r
+    t1 = G / C + 2.0 * s * h * 1.0
+    tp = G / C + 2.0 * s * h * p
+    return (t1 - tp) / t1
