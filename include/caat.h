@@ -1,0 +1,203 @@
+/*
+ * caat.h - C ABI of the B200 (sm_100a) row-parallel linear layer with partial
+ * channel-reduce, residual add and per-rank norm (the hot path of CAAT-Net,
+ * "Tensor-Parallelism with Partially Synchronized Activations").
+ *
+ * The t tensor-parallel ranks are simulated as a leading batch dimension on ONE
+ * GPU ("logical devices", Section 3.2): every per-rank tensor carries a leading
+ * index m = 0..t-1 and the partial channel-reduce is a sum over that index,
+ * restricted to the shared channels.
+ *
+ * Symbols
+ *   t      tensor-parallel ranks                         (paper: r; rank index m)
+ *   T      tokens = batch x sequence                     (argument `tokens`)
+ *   h      hidden size
+ *   K      contraction width of the layer: h for the attention output projection,
+ *          ffn for the MLP down-projection;  K_r = K / t is one rank's shard
+ *   S      shared channels = floor(h * p)                (Eq. A3)
+ *   alpha  private-channel scale, sqrt(t) (default) or 1 (Section 4)
+ *
+ * Conventions (all entry points)
+ *   Layout     row-major, last index fastest, densely packed, no padding.
+ *   Pointers   every tensor argument is a DEVICE pointer, 16-byte aligned, owned by
+ *              the caller; the library keeps none of them after the call returns.
+ *              `workspace` is caller-owned device scratch of at least
+ *              caat_workspace_bytes(); its contents are undefined on return.
+ *   Streams    all work is enqueued on `cuda_stream` (a cudaStream_t cast to void*;
+ *              NULL is the default stream); calls do not synchronise.
+ *   dtype      CAAT_BF16: bf16 storage, fp32 accumulation and statistics, round to
+ *              nearest even on store.  CAAT_F32: fp32 throughout.
+ *   Errors     a caat_status is returned; argument errors are found on the host
+ *              before any launch and leave all outputs untouched.  There is no CPU
+ *              fallback: without a usable CUDA device calls return CAAT_ECUDA.
+ *   Determinism  same inputs, same device: bit-identical outputs (no floating-point
+ *              atomics; rank sums run m = 0..t-1).
+ *   Aliasing   Hn may alias R (in-place residual update); dR may alias dHn; nothing
+ *              else may overlap.
+ *   Limits     h must be a multiple of 8 (CAAT_EUNSUPPORTED otherwise); t divides
+ *              h and ffn.  The tensor-core GEMM is used for CAAT_BF16 when K_r and S
+ *              are multiples of 8; other shapes run a slower CUDA-core GEMM.
+ */
+#ifndef CAAT_H_
+#define CAAT_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct caat_ctx caat_ctx; /* opaque; immutable between set_option calls */
+
+typedef enum { CAAT_F32 = 0, CAAT_BF16 = 1 } caat_dtype;
+
+/* Which row-parallel layer: K = h (attention output projection, Eq. A5) or
+ * K = ffn (MLP down-projection, Eq. A3). */
+typedef enum { CAAT_ATTN_OUT = 0, CAAT_MLP_DOWN = 1 } caat_layer;
+
+typedef enum {
+  CAAT_OK = 0,
+  CAAT_EINVAL = 1,       /* null pointer, bad enum, value out of range          */
+  CAAT_ESHAPE = 2,       /* t does not divide h / ffn, tokens < 1, S > h        */
+  CAAT_EALIGN = 3,       /* a tensor pointer is not 16-byte aligned             */
+  CAAT_EWORKSPACE = 4,   /* workspace NULL or smaller than caat_workspace_bytes */
+  CAAT_EUNSUPPORTED = 5, /* shape outside the limits stated above               */
+  CAAT_ECUDA = 6,        /* a CUDA runtime call failed (see caat_last_cuda_error) */
+  CAAT_ETIMEOUT = 7      /* a bounded device-side wait ran out                  */
+} caat_status;
+
+typedef enum {
+  CAAT_OPT_NORM = 0,            /* 0 = RMSNorm (default), 1 = LayerNorm (Eq. 9: "Norm") */
+  CAAT_OPT_EPS = 1,             /* norm epsilon, default 1e-5                           */
+  CAAT_OPT_PRIVATE_SCALE = 2,   /* alpha; default sqrt(t); 1 switches scaling off       */
+  CAAT_OPT_SHARED_CHANNELS = 3, /* override S with an explicit integer in [0, h]        */
+  CAAT_OPT_GEMM = 4             /* 0 = automatic (default), 1 = force the CUDA-core GEMM */
+} caat_option;
+
+/* Creates a context for hidden size h, MLP width ffn, t ranks, synchronisation
+ * factor p in [0,1] (Section 3: the first h*p channels are shared; S =
+ * floor(h*p) in IEEE double, Eq. A3).  Host-only; allocates no device memory. */
+caat_status caat_create(int h, int ffn, int t, double p, caat_dtype dtype, caat_ctx **out);
+caat_status caat_set_option(caat_ctx *ctx, caat_option opt, double value);
+void caat_destroy(caat_ctx *ctx);
+
+/* S, the number of shared channels: channels [0,S) are summed over ranks and
+ * channels [S,h) stay private to each rank (Eq. A3).  -1 if ctx is NULL. */
+int caat_shared_channels(const caat_ctx *ctx);
+/* alpha currently in effect. */
+double caat_private_scale(const caat_ctx *ctx);
+
+/* Bytes of device scratch the forward (backward = 0) or backward (backward = 1)
+ * call of `layer` needs for `tokens` tokens.  For the block calls pass the larger
+ * of the two layers' figures (CAAT_MLP_DOWN's, when ffn >= h). 0 on bad arguments. */
+size_t caat_workspace_bytes(const caat_ctx *ctx, caat_layer layer, int tokens, int backward);
+
+const char *caat_strerror(caat_status s);
+/* Text of the last CUDA runtime error seen by this thread's calls ("" if none). */
+const char *caat_last_cuda_error(void);
+
+/*
+ * Forward of one row-parallel sub-layer (Eq. A3 / A5, Section 4, Eq. 9):
+ *   Zt[m,i,l] = sum_k Y[m,i,k] * W[m,l,k]                       per-rank GEMM
+ *   Z [m,i,l] = sum_m' Zt[m',i,l]        if l <  S              partial channel-reduce
+ *             = alpha * Zt[m,i,l]        if l >= S              private-channel scaling
+ *   Hn[m,i,l] = Z[m,i,l] + R[m,i,l]                             residual add
+ *   X [m,i,:] = Norm(Hn[m,i,:]) * gamma (+ beta)                per-rank norm over all h
+ * rstd (and mean for LayerNorm) are saved for the backward.
+ *
+ *   Y     [t, T, K_r] dtype  in     W    [t, h, K_r] dtype in (out x in per rank)
+ *   R     [t, T, h]   dtype  in     gamma [h] dtype in;  beta [h] dtype in or NULL
+ *   Hn    [t, T, h]   dtype  out    X    [t, T, h] dtype out
+ *   rstd  [t, T]      fp32   out    mean [t, T] fp32 out (LayerNorm) or NULL (RMSNorm)
+ */
+caat_status caat_rowpar_forward(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                const void *Y, const void *W, const void *R,
+                                const void *gamma, const void *beta,
+                                void *Hn, void *X, float *rstd, float *mean,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Backward of the same sub-layer: the exact gradient of the forward map, with the
+ * rank reduction placed AFTER the norm's backward (operation "h" of Fig. 2b,
+ * Section 4 and Appendix B), accumulated in fp32 (Section 4), and the norm
+ * parameters' gradients summed over ranks (Section 4):
+ *   g  [m,i,:] = NormBwd(dX[m,i,:]; Hn, rstd, mean, gamma) + dHn[m,i,:]
+ *   dR [m]     = g[m]                                     (per rank, NOT reduced)
+ *   dZt[m,i,l] = sum_m' g[m',i,l] if l < S, alpha * g[m,i,l] if l >= S
+ *   dY [m,i,k] = sum_l dZt[m,i,l] * W[m,l,k]
+ *   dW [m,l,k] = sum_i dZt[m,i,l] * Y[m,i,k]
+ *   dgamma[l]  = sum_m sum_i dX[m,i,l] * xhat[m,i,l];   dbeta[l] = sum_m sum_i dX[m,i,l]
+ *
+ *   dX [t,T,h] dtype in       dHn [t,T,h] dtype in or NULL (no gradient on the stream)
+ *   Y, W, gamma as in the forward; Hn, rstd, mean as the forward wrote them
+ *   dY [t,T,K_r] dtype out    dW [t,h,K_r] FP32 out       dR [t,T,h] dtype out
+ *   dgamma [h] fp32 out       dbeta [h] fp32 out (LayerNorm) or NULL
+ */
+caat_status caat_rowpar_backward(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                 const void *dX, const void *dHn,
+                                 const void *Y, const void *W, const void *Hn,
+                                 const float *rstd, const float *mean, const void *gamma,
+                                 void *dY, float *dW, void *dR, float *dgamma, float *dbeta,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Block = the attention output projection followed by the MLP down-projection, the
+ * two row-parallel layers (and the two reduces, Appendix C) of one transformer
+ * block, chained through the residual stream: R of the second layer is Hn1.
+ * Tensors as in caat_rowpar_forward with K_r = h/t for Y_attn, W_o and ffn/t for
+ * Y_mlp, W_down.  beta1/beta2/mean1/mean2 are NULL for RMSNorm.
+ */
+caat_status caat_block_forward(const caat_ctx *ctx, int tokens,
+                               const void *Y_attn, const void *W_o,
+                               const void *Y_mlp, const void *W_down, const void *R0,
+                               const void *gamma1, const void *beta1,
+                               const void *gamma2, const void *beta2,
+                               void *Hn1, void *X1, float *rstd1, float *mean1,
+                               void *Hn2, void *X2, float *rstd2, float *mean2,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Backward of the block: the MLP-down layer first (upstream dX2 through its norm,
+ * dHn2 on the outgoing residual stream), then the attention-out layer whose
+ * residual-stream gradient is the dR of the second layer (written to dHn1, an
+ * output of this call, [t,T,h] dtype).  dHn2 may be NULL.
+ */
+caat_status caat_block_backward(const caat_ctx *ctx, int tokens,
+                                const void *dX1, const void *dX2, const void *dHn2,
+                                const void *Y_attn, const void *W_o,
+                                const void *Y_mlp, const void *W_down,
+                                const void *Hn1, const float *rstd1, const float *mean1,
+                                const void *Hn2, const float *rstd2, const float *mean2,
+                                const void *gamma1, const void *gamma2,
+                                void *dY_attn, float *dW_o, void *dY_mlp, float *dW_down,
+                                void *dR0, void *dHn1,
+                                float *dgamma1, float *dbeta1, float *dgamma2, float *dbeta2,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Analytic bytes ONE partial channel-reduce would move on a real t-device system
+ * (Appendix C: each device sends and receives tokens*h*p activations per reduce;
+ * Appendix D: all-reduce = reduce-scatter + all-gather, traffic cut by 100(1-p) %).
+ * elem_bytes is 2 for 16-bit communication.  Host-only.  Outputs may be NULL.
+ *   payload_per_rank     = tokens * S * elem_bytes
+ *   payload_per_rank_p1  = tokens * h * elem_bytes          (full all-reduce)
+ *   ring_wire_per_rank   = 2 (t-1) * payload / t            (rounded down)
+ */
+caat_status caat_allreduce_bytes(const caat_ctx *ctx, int tokens, int elem_bytes,
+                                 unsigned long long *payload_per_rank,
+                                 unsigned long long *payload_per_rank_p1,
+                                 unsigned long long *ring_wire_per_rank);
+
+/* Synchronises `cuda_stream` and reports CAAT_ETIMEOUT if a kernel launched
+ * through this library gave up on a bounded wait since the last call of this
+ * function, CAAT_ECUDA if the stream is in error, else CAAT_OK. */
+caat_status caat_last_device_status(const caat_ctx *ctx, void *cuda_stream);
+
+/* Number of kernels launched through this library by the calling process since it
+ * was loaded (for benchmarks' launch accounting). */
+unsigned long long caat_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAAT_H_ */

@@ -1,0 +1,241 @@
+"""Thin ctypes binding of libcaat.so (the C ABI declared in include/caat.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  PyTorch is used for device memory (``torch.empty``), ``data_ptr()`` and the
+current CUDA stream.  There is no CPU fallback: without the built library the import
+fails, and without a CUDA device the compute calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_double, c_int, c_size_t, c_ulonglong, c_void_p
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libcaat.so")
+
+CAAT_F32, CAAT_BF16 = 0, 1
+CAAT_ATTN_OUT, CAAT_MLP_DOWN = 0, 1
+(CAAT_OK, CAAT_EINVAL, CAAT_ESHAPE, CAAT_EALIGN, CAAT_EWORKSPACE, CAAT_EUNSUPPORTED, CAAT_ECUDA,
+ CAAT_ETIMEOUT) = range(8)
+CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM = range(5)
+RMSNORM, LAYERNORM = 0, 1
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2506_19645_b200.build` "
+                      "(there is no fallback path)")
+lib = ctypes.CDLL(LIB_PATH)
+
+_P = c_void_p
+_sigs = {
+    "caat_create": (c_int, [c_int, c_int, c_int, c_double, c_int, POINTER(c_void_p)]),
+    "caat_set_option": (c_int, [_P, c_int, c_double]),
+    "caat_destroy": (None, [_P]),
+    "caat_shared_channels": (c_int, [_P]),
+    "caat_private_scale": (c_double, [_P]),
+    "caat_workspace_bytes": (c_size_t, [_P, c_int, c_int, c_int]),
+    "caat_strerror": (c_char_p, [c_int]),
+    "caat_last_cuda_error": (c_char_p, []),
+    "caat_rowpar_forward": (c_int, [_P, c_int, c_int] + [_P] * 9 + [_P, c_size_t, _P]),
+    "caat_rowpar_backward": (c_int, [_P, c_int, c_int] + [_P] * 13 + [_P, c_size_t, _P]),
+    "caat_block_forward": (c_int, [_P, c_int] + [_P] * 17 + [_P, c_size_t, _P]),
+    "caat_block_backward": (c_int, [_P, c_int] + [_P] * 25 + [_P, c_size_t, _P]),
+    "caat_allreduce_bytes": (c_int, [_P, c_int, c_int] + [POINTER(c_ulonglong)] * 3),
+    "caat_last_device_status": (c_int, [_P, _P]),
+    "caat_kernel_launches": (c_ulonglong, []),
+}
+for _name, (_res, _args) in _sigs.items():
+    _f = getattr(lib, _name)
+    _f.restype = _res
+    _f.argtypes = _args
+EXPORTED = tuple(_sigs)
+
+
+class CaatError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib.caat_strerror(status).decode()
+        if status == CAAT_ECUDA:
+            msg += ": " + lib.caat_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def _check(status: int, where: str):
+    if status != CAAT_OK:
+        raise CaatError(status, where)
+
+
+def _dtype_code(dtype) -> int:
+    if dtype == "bf16" or dtype is torch.bfloat16:
+        return CAAT_BF16
+    if dtype == "f32" or dtype is torch.float32:
+        return CAAT_F32
+    raise ValueError(f"unsupported dtype {dtype!r}")
+
+
+def _ptr(x, dtype=None, shape=None, name="tensor"):
+    """Device pointer of a contiguous CUDA tensor (None -> NULL), with shape/dtype checks."""
+    if x is None:
+        return None
+    if not isinstance(x, torch.Tensor) or not x.is_cuda:
+        raise TypeError(f"{name}: expected a CUDA tensor (the library has no host path)")
+    if not x.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous")
+    if dtype is not None and x.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {x.dtype}")
+    if shape is not None and tuple(x.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(x.shape)}")
+    return x.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Context:
+    """Owns a ``caat_ctx``.  Methods carry the names of the C entry points without the prefix."""
+
+    def __init__(self, h: int, ffn: int, t: int, p: float, dtype="bf16"):
+        self._h = c_void_p()
+        self.h, self.ffn, self.t, self.p = h, ffn, t, p
+        self.dtype_code = _dtype_code(dtype)
+        self.torch_dtype = torch.bfloat16 if self.dtype_code == CAAT_BF16 else torch.float32
+        self.norm = RMSNORM
+        _check(lib.caat_create(h, ffn, t, float(p), self.dtype_code, byref(self._h)), "caat_create")
+
+    def __del__(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib.caat_destroy(self._h)
+            self._h = c_void_p()
+
+    # ---- options / queries
+    def set_option(self, opt: int, value: float):
+        _check(lib.caat_set_option(self._h, opt, float(value)), "caat_set_option")
+        if opt == CAAT_OPT_NORM:
+            self.norm = int(value)
+        return self
+
+    @property
+    def shared_channels(self) -> int:
+        return lib.caat_shared_channels(self._h)
+
+    @property
+    def private_scale(self) -> float:
+        return lib.caat_private_scale(self._h)
+
+    def k_r(self, layer: int) -> int:
+        return (self.h if layer == CAAT_ATTN_OUT else self.ffn) // self.t
+
+    def workspace_bytes(self, layer: int, tokens: int, backward: bool) -> int:
+        return lib.caat_workspace_bytes(self._h, layer, tokens, 1 if backward else 0)
+
+    def block_workspace_bytes(self, tokens: int, backward: bool) -> int:
+        return max(self.workspace_bytes(CAAT_ATTN_OUT, tokens, backward),
+                   self.workspace_bytes(CAAT_MLP_DOWN, tokens, backward))
+
+    def allreduce_bytes(self, tokens: int, elem_bytes: int = 2) -> dict:
+        a, b, c = c_ulonglong(), c_ulonglong(), c_ulonglong()
+        _check(lib.caat_allreduce_bytes(self._h, tokens, elem_bytes, byref(a), byref(b), byref(c)),
+               "caat_allreduce_bytes")
+        return {"payload_per_rank": a.value, "payload_per_rank_p1": b.value, "ring_wire_per_rank": c.value}
+
+    def last_device_status(self) -> int:
+        return lib.caat_last_device_status(self._h, _stream())
+
+    # ---- compute: raw entry points (caller passes every buffer)
+    def rowpar_forward(self, layer, tokens, Y, W, R, gamma, beta, Hn, X, rstd, mean, workspace):
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        st = lib.caat_rowpar_forward(
+            self._h, layer, tokens,
+            _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"), _ptr(R, td, (t, tokens, h), "R"),
+            _ptr(gamma, td, (h,), "gamma"), _ptr(beta, td, (h,), "beta"),
+            _ptr(Hn, td, (t, tokens, h), "Hn"), _ptr(X, td, (t, tokens, h), "X"),
+            _ptr(rstd, torch.float32, (t, tokens), "rstd"), _ptr(mean, torch.float32, (t, tokens), "mean"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_rowpar_forward")
+
+    def rowpar_backward(self, layer, tokens, dX, dHn, Y, W, Hn, rstd, mean, gamma, dY, dW, dR, dgamma, dbeta,
+                        workspace):
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        f32 = torch.float32
+        st = lib.caat_rowpar_backward(
+            self._h, layer, tokens,
+            _ptr(dX, td, (t, tokens, h), "dX"), _ptr(dHn, td, (t, tokens, h), "dHn"),
+            _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"), _ptr(Hn, td, (t, tokens, h), "Hn"),
+            _ptr(rstd, f32, (t, tokens), "rstd"), _ptr(mean, f32, (t, tokens), "mean"), _ptr(gamma, td, (h,), "gamma"),
+            _ptr(dY, td, (t, tokens, k), "dY"), _ptr(dW, f32, (t, h, k), "dW"), _ptr(dR, td, (t, tokens, h), "dR"),
+            _ptr(dgamma, f32, (h,), "dgamma"), _ptr(dbeta, f32, (h,), "dbeta"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_rowpar_backward")
+
+    def block_forward(self, tokens, Y_attn, W_o, Y_mlp, W_down, R0, gamma1, beta1, gamma2, beta2,
+                      Hn1, X1, rstd1, mean1, Hn2, X2, rstd2, mean2, workspace):
+        td, t, h = self.torch_dtype, self.t, self.h
+        ka, km = self.k_r(CAAT_ATTN_OUT), self.k_r(CAAT_MLP_DOWN)
+        f32 = torch.float32
+        act = (t, tokens, h)
+        st = lib.caat_block_forward(
+            self._h, tokens,
+            _ptr(Y_attn, td, (t, tokens, ka), "Y_attn"), _ptr(W_o, td, (t, h, ka), "W_o"),
+            _ptr(Y_mlp, td, (t, tokens, km), "Y_mlp"), _ptr(W_down, td, (t, h, km), "W_down"),
+            _ptr(R0, td, act, "R0"), _ptr(gamma1, td, (h,), "gamma1"), _ptr(beta1, td, (h,), "beta1"),
+            _ptr(gamma2, td, (h,), "gamma2"), _ptr(beta2, td, (h,), "beta2"),
+            _ptr(Hn1, td, act, "Hn1"), _ptr(X1, td, act, "X1"), _ptr(rstd1, f32, (t, tokens), "rstd1"),
+            _ptr(mean1, f32, (t, tokens), "mean1"),
+            _ptr(Hn2, td, act, "Hn2"), _ptr(X2, td, act, "X2"), _ptr(rstd2, f32, (t, tokens), "rstd2"),
+            _ptr(mean2, f32, (t, tokens), "mean2"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_block_forward")
+
+    def block_backward(self, tokens, dX1, dX2, dHn2, Y_attn, W_o, Y_mlp, W_down, Hn1, rstd1, mean1, Hn2, rstd2,
+                       mean2, gamma1, gamma2, dY_attn, dW_o, dY_mlp, dW_down, dR0, dHn1, dgamma1, dbeta1,
+                       dgamma2, dbeta2, workspace):
+        td, t, h = self.torch_dtype, self.t, self.h
+        ka, km = self.k_r(CAAT_ATTN_OUT), self.k_r(CAAT_MLP_DOWN)
+        f32 = torch.float32
+        act = (t, tokens, h)
+        st = lib.caat_block_backward(
+            self._h, tokens,
+            _ptr(dX1, td, act, "dX1"), _ptr(dX2, td, act, "dX2"), _ptr(dHn2, td, act, "dHn2"),
+            _ptr(Y_attn, td, (t, tokens, ka), "Y_attn"), _ptr(W_o, td, (t, h, ka), "W_o"),
+            _ptr(Y_mlp, td, (t, tokens, km), "Y_mlp"), _ptr(W_down, td, (t, h, km), "W_down"),
+            _ptr(Hn1, td, act, "Hn1"), _ptr(rstd1, f32, (t, tokens), "rstd1"), _ptr(mean1, f32, (t, tokens), "mean1"),
+            _ptr(Hn2, td, act, "Hn2"), _ptr(rstd2, f32, (t, tokens), "rstd2"), _ptr(mean2, f32, (t, tokens), "mean2"),
+            _ptr(gamma1, td, (h,), "gamma1"), _ptr(gamma2, td, (h,), "gamma2"),
+            _ptr(dY_attn, td, (t, tokens, ka), "dY_attn"), _ptr(dW_o, f32, (t, h, ka), "dW_o"),
+            _ptr(dY_mlp, td, (t, tokens, km), "dY_mlp"), _ptr(dW_down, f32, (t, h, km), "dW_down"),
+            _ptr(dR0, td, act, "dR0"), _ptr(dHn1, td, act, "dHn1"),
+            _ptr(dgamma1, f32, (h,), "dgamma1"), _ptr(dbeta1, f32, (h,), "dbeta1"),
+            _ptr(dgamma2, f32, (h,), "dgamma2"), _ptr(dbeta2, f32, (h,), "dbeta2"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_block_backward")
+
+    # ---- buffer helpers (torch.empty only; no arithmetic)
+    def alloc_workspace(self, nbytes: int, device="cuda"):
+        return torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
+
+    def alloc_forward_outputs(self, tokens: int, device="cuda") -> dict:
+        td, t, h = self.torch_dtype, self.t, self.h
+        out = {"Hn": torch.empty((t, tokens, h), dtype=td, device=device),
+               "X": torch.empty((t, tokens, h), dtype=td, device=device),
+               "rstd": torch.empty((t, tokens), dtype=torch.float32, device=device),
+               "mean": torch.empty((t, tokens), dtype=torch.float32, device=device) if self.norm == LAYERNORM else None}
+        return out
+
+    def alloc_backward_outputs(self, layer: int, tokens: int, device="cuda") -> dict:
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        return {"dY": torch.empty((t, tokens, k), dtype=td, device=device),
+                "dW": torch.empty((t, h, k), dtype=torch.float32, device=device),
+                "dR": torch.empty((t, tokens, h), dtype=td, device=device),
+                "dgamma": torch.empty((h,), dtype=torch.float32, device=device),
+                "dbeta": torch.empty((h,), dtype=torch.float32, device=device) if self.norm == LAYERNORM else None}
+
+
+def kernel_launches() -> int:
+    return int(lib.caat_kernel_launches())

@@ -1,0 +1,341 @@
+// C ABI of libcaat: context, argument validation, scratch layout and the launch
+// sequences of the forward / backward of one row-parallel layer and of a block.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "caat_internal.h"
+
+namespace caat {
+
+static std::atomic<unsigned long long> g_launches{0};
+static thread_local char g_cuda_err[256] = "";
+
+__device__ unsigned int g_status_word = 0;
+
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+unsigned int* device_status_word() {
+  unsigned int* p = nullptr;
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word) != cudaSuccess) return nullptr;
+  return p;
+}
+
+static caat_status cuda_fail(cudaError_t e) {
+  std::strncpy(g_cuda_err, cudaGetErrorString(e), sizeof(g_cuda_err) - 1);
+  g_cuda_err[sizeof(g_cuda_err) - 1] = 0;
+  return CAAT_ECUDA;
+}
+
+Scratch scratch_layout(const caat_ctx* ctx, int K_r, int tokens, int backward) {
+  Scratch s{};
+  const size_t e = elem_size(ctx->dtype);
+  s.S_lo = round_down(ctx->S, kLayoutVec);
+  s.S_hi = round_up(ctx->S, kLayoutVec);
+  s.P = ctx->h - s.S_lo;
+  size_t off = 0;
+  s.zs_off = off;
+  off = align_up(off + (size_t)tokens * s.S_hi * e, 256);
+  s.zp_off = off;
+  off = align_up(off + (size_t)ctx->t * tokens * s.P * e, 256);
+  if (backward) {
+    const size_t rows = (size_t)rows_backward_partial_rows(ctx->h, tokens, ctx->dtype);
+    s.dgpart_off = off;
+    off = align_up(off + rows * ctx->h * sizeof(float), 256);
+    s.dbpart_off = off;
+    off = align_up(off + rows * ctx->h * sizeof(float), 256);
+    s.splitk_off = off;
+    s.splitk_bytes = 0;
+    if (tc_gemm_usable(ctx, K_r)) {
+      RowparShapes sh{ctx->t, tokens, ctx->h, K_r, ctx->S, s.S_lo, s.S_hi, s.P};
+      s.splitk_bytes = tc_wgrad_splitk_bytes(sh);
+    }
+    off = align_up(off + s.splitk_bytes, 256);
+  }
+  s.total = off;
+  return s;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int layer_kr(const caat_ctx* ctx, caat_layer layer) {
+  return (layer == CAAT_ATTN_OUT ? ctx->h : ctx->ffn) / ctx->t;
+}
+
+static caat_status check_common(const caat_ctx* ctx, caat_layer layer, int tokens) {
+  if (!ctx) return CAAT_EINVAL;
+  if (layer != CAAT_ATTN_OUT && layer != CAAT_MLP_DOWN) return CAAT_EINVAL;
+  if (tokens < 1) return CAAT_ESHAPE;
+  if (ctx->h % 8 != 0) return CAAT_EUNSUPPORTED;
+  const int V = ctx->dtype == CAAT_BF16 ? 8 : 4;
+  if (ctx->h / V > 512 * 4) return CAAT_EUNSUPPORTED;
+  if ((long long)ctx->t * tokens > 2000000000LL) return CAAT_EUNSUPPORTED;
+  return CAAT_OK;
+}
+
+// ---- forward of one layer ------------------------------------------------------
+static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void* Y, const void* W, const void* R,
+                                const void* gamma, const void* beta, void* Hn, void* X, float* rstd, float* mean,
+                                void* ws, cudaStream_t st) {
+  const Scratch L = scratch_layout(ctx, K_r, T, 0);
+  char* wsb = static_cast<char*>(ws);
+  void* zs = wsb + L.zs_off;
+  void* zp = wsb + L.zp_off;
+  const int t = ctx->t, h = ctx->h, S = ctx->S;
+  const size_t e = elem_size(ctx->dtype);
+  cudaError_t ce;
+
+  if (tc_gemm_usable(ctx, K_r)) {
+    RowparShapes sh{t, T, h, K_r, S, L.S_lo, L.S_hi, L.P};
+    ce = launch_tc_forward(sh, Y, W, zs, zp, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+  } else {
+    if (S > 0) {  // shared columns: one product over the whole contraction axis (all ranks)
+      GemmProblem g{};
+      g.nseg = 1;
+      g.seg[0] = GemmSeg{Y, W, 0, (long long)T * K_r, K_r, 1, 0, (long long)h * K_r, 1, K_r, t, K_r};
+      g.C = zs; g.sCb = 0; g.sCi = L.S_hi; g.M = T; g.N = S; g.batch = 1; g.c_f32 = 0;
+      ce = launch_gemm_simt(g, ctx->dtype, st);
+      if (ce != cudaSuccess) return cuda_fail(ce);
+    }
+    if (S < h) {  // private columns: one product per rank
+      GemmProblem g{};
+      g.nseg = 1;
+      g.seg[0] = GemmSeg{Y, static_cast<const char*>(W) + (size_t)S * K_r * e,
+                         (long long)T * K_r, 0, K_r, 1, (long long)h * K_r, 0, 1, K_r, 1, K_r};
+      g.C = static_cast<char*>(zp) + (size_t)(S - L.S_lo) * e;
+      g.sCb = (long long)T * L.P; g.sCi = L.P; g.M = T; g.N = h - S; g.batch = t; g.c_f32 = 0;
+      ce = launch_gemm_simt(g, ctx->dtype, st);
+      if (ce != cudaSuccess) return cuda_fail(ce);
+    }
+  }
+  RowFwdArgs a{zs, zp, R, gamma, beta, Hn, X, rstd, mean, t, T, h, S, L.S_lo, L.S_hi, L.P,
+               (float)ctx->alpha, (float)ctx->eps, ctx->norm};
+  ce = launch_rows_forward(a, ctx->dtype, st);
+  if (ce != cudaSuccess) return cuda_fail(ce);
+  return CAAT_OK;
+}
+
+// ---- backward of one layer -----------------------------------------------------
+static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void* dX, const void* dHn, const void* Y,
+                                 const void* W, const void* Hn, const float* rstd, const float* mean,
+                                 const void* gamma, void* dY, float* dW, void* dR, float* dgamma, float* dbeta,
+                                 void* ws, cudaStream_t st) {
+  const Scratch L = scratch_layout(ctx, K_r, T, 1);
+  char* wsb = static_cast<char*>(ws);
+  void* gs = wsb + L.zs_off;
+  void* zp = wsb + L.zp_off;
+  const int t = ctx->t, h = ctx->h, S = ctx->S;
+  const size_t e = elem_size(ctx->dtype);
+  cudaError_t ce;
+
+  RowBwdArgs a{dX, dHn, Hn, gamma, rstd, mean, dR, gs, zp,
+               reinterpret_cast<float*>(wsb + L.dgpart_off), reinterpret_cast<float*>(wsb + L.dbpart_off),
+               dgamma, dbeta, t, T, h, S, L.S_lo, L.S_hi, L.P, (float)ctx->alpha, ctx->norm};
+  ce = launch_rows_backward(a, ctx->dtype, st);
+  if (ce != cudaSuccess) return cuda_fail(ce);
+
+  if (tc_gemm_usable(ctx, K_r)) {
+    RowparShapes sh{t, T, h, K_r, S, L.S_lo, L.S_hi, L.P};
+    ce = launch_tc_dgrad(sh, gs, zp, W, dY, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    ce = launch_tc_wgrad(sh, gs, zp, Y, dW, wsb + L.splitk_off, L.splitk_bytes, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    return CAAT_OK;
+  }
+  const char* zp_priv = static_cast<const char*>(zp) + (size_t)(S - L.S_lo) * e;
+  {  // dY[m] = gs W[m][:S] + zp[m] W[m][S:]
+    GemmProblem g{};
+    g.nseg = 2;
+    g.seg[0] = GemmSeg{gs, W, 0, 0, L.S_hi, 1, (long long)h * K_r, 0, K_r, 1, 1, S};
+    g.seg[1] = GemmSeg{zp_priv, static_cast<const char*>(W) + (size_t)S * K_r * e,
+                       (long long)T * L.P, 0, L.P, 1, (long long)h * K_r, 0, K_r, 1, 1, h - S};
+    g.C = dY; g.sCb = (long long)T * K_r; g.sCi = K_r; g.M = T; g.N = K_r; g.batch = t; g.c_f32 = 0;
+    ce = launch_gemm_simt(g, ctx->dtype, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+  }
+  if (S > 0) {  // dW[m][:S] = gs^T Y[m]
+    GemmProblem g{};
+    g.nseg = 1;
+    g.seg[0] = GemmSeg{gs, Y, 0, 0, 1, L.S_hi, (long long)T * K_r, 0, K_r, 1, 1, T};
+    g.C = dW; g.sCb = (long long)h * K_r; g.sCi = K_r; g.M = S; g.N = K_r; g.batch = t; g.c_f32 = 1;
+    ce = launch_gemm_simt(g, ctx->dtype, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+  }
+  if (S < h) {  // dW[m][S:] = zp[m]^T Y[m]
+    GemmProblem g{};
+    g.nseg = 1;
+    g.seg[0] = GemmSeg{zp_priv, Y, (long long)T * L.P, 0, 1, L.P, (long long)T * K_r, 0, K_r, 1, 1, T};
+    g.C = dW + (size_t)S * K_r; g.sCb = (long long)h * K_r; g.sCi = K_r; g.M = h - S; g.N = K_r; g.batch = t;
+    g.c_f32 = 1;
+    ce = launch_gemm_simt(g, ctx->dtype, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+  }
+  return CAAT_OK;
+}
+
+}  // namespace caat
+
+using namespace caat;
+
+extern "C" {
+
+caat_status caat_create(int h, int ffn, int t, double p, caat_dtype dtype, caat_ctx** out) {
+  if (!out) return CAAT_EINVAL;
+  *out = nullptr;
+  if (dtype != CAAT_F32 && dtype != CAAT_BF16) return CAAT_EINVAL;
+  if (!(p >= 0.0 && p <= 1.0)) return CAAT_EINVAL;
+  if (h < 1 || ffn < 1 || t < 1) return CAAT_ESHAPE;
+  if (h % t != 0 || ffn % t != 0) return CAAT_ESHAPE;
+  caat_ctx* c = new (std::nothrow) caat_ctx();
+  if (!c) return CAAT_EINVAL;
+  c->h = h; c->ffn = ffn; c->t = t; c->p = p; c->dtype = dtype;
+  c->S = (int)std::floor((double)h * p);   // Eq. A3: l < floor(h p) is shared
+  c->alpha = std::sqrt((double)t);         // Section 4: private channels times sqrt(r)
+  c->norm = 0; c->eps = 1e-5; c->force_simt = 0;
+  *out = c;
+  return CAAT_OK;
+}
+
+caat_status caat_set_option(caat_ctx* ctx, caat_option opt, double value) {
+  if (!ctx) return CAAT_EINVAL;
+  switch (opt) {
+    case CAAT_OPT_NORM:
+      if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
+      ctx->norm = (int)value; return CAAT_OK;
+    case CAAT_OPT_EPS:
+      if (!(value >= 0.0)) return CAAT_EINVAL;
+      ctx->eps = value; return CAAT_OK;
+    case CAAT_OPT_PRIVATE_SCALE:
+      if (!std::isfinite(value)) return CAAT_EINVAL;
+      ctx->alpha = value; return CAAT_OK;
+    case CAAT_OPT_SHARED_CHANNELS:
+      if (value != std::floor(value)) return CAAT_EINVAL;
+      if (value < 0.0 || value > (double)ctx->h) return CAAT_ESHAPE;
+      ctx->S = (int)value; return CAAT_OK;
+    case CAAT_OPT_GEMM:
+      if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
+      ctx->force_simt = (int)value; return CAAT_OK;
+  }
+  return CAAT_EINVAL;
+}
+
+void caat_destroy(caat_ctx* ctx) { delete ctx; }
+
+int caat_shared_channels(const caat_ctx* ctx) { return ctx ? ctx->S : -1; }
+double caat_private_scale(const caat_ctx* ctx) { return ctx ? ctx->alpha : 0.0; }
+
+size_t caat_workspace_bytes(const caat_ctx* ctx, caat_layer layer, int tokens, int backward) {
+  if (check_common(ctx, layer, tokens) != CAAT_OK) return 0;
+  return scratch_layout(ctx, layer_kr(ctx, layer), tokens, backward ? 1 : 0).total;
+}
+
+const char* caat_strerror(caat_status s) {
+  switch (s) {
+    case CAAT_OK: return "ok";
+    case CAAT_EINVAL: return "invalid argument";
+    case CAAT_ESHAPE: return "bad shape";
+    case CAAT_EALIGN: return "pointer not 16-byte aligned";
+    case CAAT_EWORKSPACE: return "workspace missing or too small";
+    case CAAT_EUNSUPPORTED: return "shape not supported";
+    case CAAT_ECUDA: return "CUDA error";
+    case CAAT_ETIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+const char* caat_last_cuda_error(void) { return g_cuda_err; }
+
+caat_status caat_rowpar_forward(const caat_ctx* ctx, caat_layer layer, int tokens, const void* Y, const void* W,
+                                const void* R, const void* gamma, const void* beta, void* Hn, void* X, float* rstd,
+                                float* mean, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = check_common(ctx, layer, tokens);
+  if (s != CAAT_OK) return s;
+  if (!Y || !W || !R || !gamma || !Hn || !X || !rstd) return CAAT_EINVAL;
+  if (ctx->norm == 1 && !mean) return CAAT_EINVAL;
+  const void* ptrs[] = {Y, W, R, gamma, beta, Hn, X, rstd, mean, workspace};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  const int K_r = layer_kr(ctx, layer);
+  if (!workspace || workspace_bytes < scratch_layout(ctx, K_r, tokens, 0).total) return CAAT_EWORKSPACE;
+  return forward_impl(ctx, K_r, tokens, Y, W, R, gamma, beta, Hn, X, rstd, mean, workspace,
+                      static_cast<cudaStream_t>(cuda_stream));
+}
+
+caat_status caat_rowpar_backward(const caat_ctx* ctx, caat_layer layer, int tokens, const void* dX, const void* dHn,
+                                 const void* Y, const void* W, const void* Hn, const float* rstd, const float* mean,
+                                 const void* gamma, void* dY, float* dW, void* dR, float* dgamma, float* dbeta,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = check_common(ctx, layer, tokens);
+  if (s != CAAT_OK) return s;
+  if (!dX || !Y || !W || !Hn || !rstd || !gamma || !dY || !dW || !dR || !dgamma) return CAAT_EINVAL;
+  if (ctx->norm == 1 && (!mean || !dbeta)) return CAAT_EINVAL;
+  const void* ptrs[] = {dX, dHn, Y, W, Hn, rstd, mean, gamma, dY, dW, dR, dgamma, dbeta, workspace};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  const int K_r = layer_kr(ctx, layer);
+  if (!workspace || workspace_bytes < scratch_layout(ctx, K_r, tokens, 1).total) return CAAT_EWORKSPACE;
+  return backward_impl(ctx, K_r, tokens, dX, dHn, Y, W, Hn, rstd, mean, gamma, dY, dW, dR, dgamma, dbeta, workspace,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+caat_status caat_block_forward(const caat_ctx* ctx, int tokens, const void* Y_attn, const void* W_o,
+                               const void* Y_mlp, const void* W_down, const void* R0, const void* gamma1,
+                               const void* beta1, const void* gamma2, const void* beta2, void* Hn1, void* X1,
+                               float* rstd1, float* mean1, void* Hn2, void* X2, float* rstd2, float* mean2,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  // Two reduces per block (Appendix C): attention-out, then MLP-down on the new residual stream.
+  caat_status s = caat_rowpar_forward(ctx, CAAT_ATTN_OUT, tokens, Y_attn, W_o, R0, gamma1, beta1, Hn1, X1, rstd1,
+                                      mean1, workspace, workspace_bytes, cuda_stream);
+  if (s != CAAT_OK) return s;
+  return caat_rowpar_forward(ctx, CAAT_MLP_DOWN, tokens, Y_mlp, W_down, Hn1, gamma2, beta2, Hn2, X2, rstd2, mean2,
+                             workspace, workspace_bytes, cuda_stream);
+}
+
+caat_status caat_block_backward(const caat_ctx* ctx, int tokens, const void* dX1, const void* dX2, const void* dHn2,
+                                const void* Y_attn, const void* W_o, const void* Y_mlp, const void* W_down,
+                                const void* Hn1, const float* rstd1, const float* mean1, const void* Hn2,
+                                const float* rstd2, const float* mean2, const void* gamma1, const void* gamma2,
+                                void* dY_attn, float* dW_o, void* dY_mlp, float* dW_down, void* dR0, void* dHn1,
+                                float* dgamma1, float* dbeta1, float* dgamma2, float* dbeta2, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream) {
+  if (!dHn1) return CAAT_EINVAL;
+  caat_status s = caat_rowpar_backward(ctx, CAAT_MLP_DOWN, tokens, dX2, dHn2, Y_mlp, W_down, Hn2, rstd2, mean2,
+                                       gamma2, dY_mlp, dW_down, dHn1, dgamma2, dbeta2, workspace, workspace_bytes,
+                                       cuda_stream);
+  if (s != CAAT_OK) return s;
+  return caat_rowpar_backward(ctx, CAAT_ATTN_OUT, tokens, dX1, dHn1, Y_attn, W_o, Hn1, rstd1, mean1, gamma1,
+                              dY_attn, dW_o, dR0, dgamma1, dbeta1, workspace, workspace_bytes, cuda_stream);
+}
+
+caat_status caat_allreduce_bytes(const caat_ctx* ctx, int tokens, int elem_bytes, unsigned long long* payload,
+                                 unsigned long long* payload_p1, unsigned long long* ring_wire) {
+  if (!ctx || elem_bytes < 1) return CAAT_EINVAL;
+  if (tokens < 1) return CAAT_ESHAPE;
+  const unsigned long long pay = (unsigned long long)tokens * (unsigned long long)ctx->S * (unsigned long long)elem_bytes;
+  if (payload) *payload = pay;
+  if (payload_p1) *payload_p1 = (unsigned long long)tokens * (unsigned long long)ctx->h * (unsigned long long)elem_bytes;
+  if (ring_wire) *ring_wire = 2ull * (unsigned long long)(ctx->t - 1) * pay / (unsigned long long)ctx->t;
+  return CAAT_OK;
+}
+
+caat_status caat_last_device_status(const caat_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return CAAT_EINVAL;
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return cuda_fail(e);
+  unsigned int w = 0;
+  e = cudaMemcpyFromSymbol(&w, g_status_word, sizeof(w));
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (w != 0) {
+    const unsigned int zero = 0;
+    e = cudaMemcpyToSymbol(g_status_word, &zero, sizeof(zero));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CAAT_ETIMEOUT;
+  }
+  return CAAT_OK;
+}
+
+unsigned long long caat_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

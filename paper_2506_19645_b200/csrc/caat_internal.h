@@ -1,0 +1,113 @@
+// Internal declarations shared by the translation units of libcaat (CUDA side only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "caat.h"
+
+struct caat_ctx {
+  int h, ffn, t;
+  double p;
+  caat_dtype dtype;
+  int S;           // shared channels, floor(h*p) or the explicit override (Eq. A3)
+  double alpha;    // private-channel scale (Section 4)
+  int norm;        // 0 RMSNorm, 1 LayerNorm
+  double eps;
+  int force_simt;  // CAAT_OPT_GEMM
+};
+
+namespace caat {
+
+constexpr int kLayoutVec = 8;        // column granularity of the scratch layout (elements)
+constexpr int kMaxPartialRows = 1184;  // upper bound on rows of norm-gradient partials (8 x 148)
+
+inline int round_down(int x, int m) { return x / m * m; }
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Scratch layout.  The shared part of the layer output (or of its gradient) is
+// stored ONCE for all ranks, the private part per rank:
+//   zs [T, S_hi]             columns [0, S) valid, S_hi = S rounded up to 8
+//   zp [t, T, h - S_lo]      column l of the layer lives at l - S_lo, S_lo = S rounded
+//                            down to 8; columns below S - S_lo are not used
+// so that every row starts on a 16-byte boundary for any S.
+struct Scratch {
+  int S_lo, S_hi, P;       // P = h - S_lo, row length of zp
+  size_t zs_off, zp_off;   // forward: Zt shared / private.  backward: dZt shared / private
+  size_t dgpart_off, dbpart_off;  // backward: [rows, h] fp32 partial norm-parameter gradients
+  size_t splitk_off, splitk_bytes;  // backward: split-K partials of the weight gradient
+  size_t total;
+};
+
+Scratch scratch_layout(const caat_ctx* ctx, int K_r, int tokens, int backward);
+
+inline size_t elem_size(caat_dtype d) { return d == CAAT_BF16 ? 2 : 4; }
+
+// ---- generic strided batched GEMM on CUDA cores (fp32 accumulate) -------------
+//   C[b][i][j] = sum_{seg} sum_{q < Q} sum_{k < Kd} A(b,q,i,k) * B(b,q,k,j)
+// with element strides for every index; A and B have the run's dtype, C has the
+// run's dtype or fp32.
+struct GemmSeg {
+  const void* A;
+  const void* B;
+  long long sAb, sAq, sAi, sAk;
+  long long sBb, sBq, sBk, sBj;
+  int Q, Kd;
+};
+struct GemmProblem {
+  int nseg;
+  GemmSeg seg[2];
+  void* C;
+  long long sCb, sCi;  // column stride of C is 1
+  int M, N, batch;
+  int c_f32;           // 1: C is fp32 regardless of dtype
+};
+cudaError_t launch_gemm_simt(const GemmProblem& g, caat_dtype dtype, cudaStream_t st);
+
+// ---- tensor-core GEMMs (bf16, tcgen05 + TMA) -----------------------------------
+struct RowparShapes {
+  int t, T, h, K_r, S, S_lo, S_hi, P;
+};
+bool tc_gemm_usable(const caat_ctx* ctx, int K_r);
+// Zt -> (zs, zp):   zs[i,l] = sum_m sum_k Y[m,i,k] W[m,l,k] (l < S);  zp[m,i,l-S_lo] = sum_k ... (l >= S)
+cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* W, void* zs, void* zp,
+                              cudaStream_t st);
+// dY[m] = [gs | zp[m]] W[m]
+cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* zp, const void* W, void* dY,
+                            cudaStream_t st);
+// dW[m] = [gs | zp[m]]^T Y[m]   (fp32 out)
+cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* zp, const void* Y, float* dW,
+                            void* splitk, size_t splitk_bytes, cudaStream_t st);
+size_t tc_wgrad_splitk_bytes(const RowparShapes& s);
+
+// ---- row kernels ------------------------------------------------------------
+struct RowFwdArgs {
+  const void *zs, *zp, *R, *gamma, *beta;
+  void *Hn, *X;
+  float *rstd, *mean;
+  int t, T, h, S, S_lo, S_hi, P;
+  float alpha, eps;
+  int norm;
+};
+cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st);
+
+struct RowBwdArgs {
+  const void *dX, *dHn, *Hn, *gamma;
+  const float *rstd, *mean;
+  void *dR, *gs, *zp;
+  float *dgpart, *dbpart;  // [rows, h]
+  float *dgamma, *dbeta;   // [h]
+  int t, T, h, S, S_lo, S_hi, P;
+  float alpha;
+  int norm;
+};
+cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, cudaStream_t st);
+int rows_backward_partial_rows(int h, int T, caat_dtype dtype);
+
+// ---- bookkeeping ------------------------------------------------------------
+void count_launch(int n = 1);
+unsigned int* device_status_word();  // device address of the status word (per device)
+
+}  // namespace caat

@@ -1,0 +1,109 @@
+"""Host-side checks of the C ABI: the library loads, exports every declared symbol, and
+rejects bad arguments before any launch.  No GPU needed: no compute call reaches a kernel."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def caat():
+    from paper_2506_19645_b200 import build
+    build.build()
+    from paper_2506_19645_b200 import caat as m
+    return m
+
+
+def test_exports_every_declared_symbol(caat):
+    header = open(os.path.join(ROOT, "include", "caat.h")).read()
+    declared = set(re.findall(r"\b(caat_[a-z_]+)\s*\(", header))
+    assert declared, "no declarations found"
+    for name in declared:
+        assert hasattr(caat.lib, name), f"libcaat.so does not export {name}"
+    assert declared == set(caat.EXPORTED), declared ^ set(caat.EXPORTED)
+
+
+def test_create_validation_and_partition(caat):
+    h = ctypes.c_void_p()
+    assert caat.lib.caat_create(768, 3072, 4, 0.5, caat.CAAT_BF16, ctypes.byref(h)) == caat.CAAT_OK
+    assert caat.lib.caat_shared_channels(h) == 384
+    assert caat.lib.caat_private_scale(h) == pytest.approx(2.0)
+    caat.lib.caat_destroy(h)
+    assert caat.lib.caat_create(768, 3072, 5, 0.5, caat.CAAT_BF16, ctypes.byref(h)) == caat.CAAT_ESHAPE
+    assert caat.lib.caat_create(768, 3072, 4, 1.5, caat.CAAT_BF16, ctypes.byref(h)) == caat.CAAT_EINVAL
+    assert caat.lib.caat_create(768, 3072, 4, 0.5, 7, ctypes.byref(h)) == caat.CAAT_EINVAL
+    assert caat.lib.caat_create(768, 3072, 4, 0.5, caat.CAAT_BF16, None) == caat.CAAT_EINVAL
+    assert caat.lib.caat_shared_channels(None) == -1
+    for hh, p, S in [(256, 0.5, 128), (2048, 0.75, 1536), (2048, 0.25, 512), (4096, 1.0, 4096), (4096, 0.0, 0),
+                     (10, 0.35, 3), (4096, 0.703125, 2880), (4096, 0.7, 2867)]:
+        c = caat.Context(hh, 4 * hh, 2, p, "bf16")
+        assert c.shared_channels == S      # floor(h p), Eq. A3
+
+
+def test_options(caat):
+    c = caat.Context(512, 2048, 8, 0.5, "bf16")
+    assert c.private_scale == pytest.approx(8 ** 0.5)
+    c.set_option(caat.CAAT_OPT_PRIVATE_SCALE, 1.0)
+    assert c.private_scale == 1.0
+    c.set_option(caat.CAAT_OPT_SHARED_CHANNELS, 100)
+    assert c.shared_channels == 100
+    with pytest.raises(caat.CaatError) as e:
+        c.set_option(caat.CAAT_OPT_SHARED_CHANNELS, 513)
+    assert e.value.status == caat.CAAT_ESHAPE
+    with pytest.raises(caat.CaatError):
+        c.set_option(caat.CAAT_OPT_NORM, 2)
+    with pytest.raises(caat.CaatError):
+        c.set_option(99, 0)
+    assert caat.lib.caat_strerror(caat.CAAT_EWORKSPACE).decode().startswith("workspace")
+
+
+def test_workspace_and_argument_errors_before_launch(caat):
+    c = caat.Context(768, 3072, 4, 0.5, "bf16")
+    T = 64
+    need = c.workspace_bytes(caat.CAAT_MLP_DOWN, T, False)
+    assert need >= T * 384 * 2 + 4 * T * 384 * 2
+    assert c.workspace_bytes(caat.CAAT_MLP_DOWN, T, True) > need
+    assert c.workspace_bytes(caat.CAAT_MLP_DOWN, 0, False) == 0
+    fake = 0x10000  # never dereferenced: validation fails first
+    f = caat.lib.caat_rowpar_forward
+    args = [c._h, caat.CAAT_MLP_DOWN, T] + [fake] * 9
+    assert f(*args[:3], None, *args[4:], fake, need, None) == caat.CAAT_EINVAL
+    assert f(*args, fake, need - 1, None) == caat.CAAT_EWORKSPACE
+    assert f(*args, None, need, None) == caat.CAAT_EWORKSPACE
+    bad = list(args); bad[5] = fake + 2
+    assert f(*bad, fake, need, None) == caat.CAAT_EALIGN
+    assert f(c._h, 5, T, *args[3:], fake, need, None) == caat.CAAT_EINVAL
+    assert f(c._h, caat.CAAT_MLP_DOWN, 0, *args[3:], fake, need, None) == caat.CAAT_ESHAPE
+    odd = caat.Context(36, 72, 2, 0.5, "bf16")     # h not a multiple of 8
+    assert caat.lib.caat_rowpar_forward(odd._h, 0, T, *([fake] * 9), fake, 1 << 20, None) == caat.CAAT_EUNSUPPORTED
+    ln = caat.Context(768, 3072, 4, 0.5, "bf16").set_option(caat.CAAT_OPT_NORM, 1)
+    a2 = [ln._h, caat.CAAT_MLP_DOWN, T] + [fake] * 8 + [None]      # mean missing under LayerNorm
+    assert f(*a2, fake, need, None) == caat.CAAT_EINVAL
+    b = caat.lib.caat_rowpar_backward
+    bargs = [c._h, caat.CAAT_MLP_DOWN, T] + [fake] * 13
+    assert b(*bargs, fake, 16, None) == caat.CAAT_EWORKSPACE
+    bargs2 = list(bargs); bargs2[3] = None
+    assert b(*bargs2, fake, 1 << 30, None) == caat.CAAT_EINVAL
+
+
+def test_binding_refuses_host_tensors(caat):
+    import torch
+    c = caat.Context(256, 1024, 2, 0.5, "f32")
+    x = torch.zeros(2, 4, 512)
+    with pytest.raises(TypeError):
+        c.rowpar_forward(caat.CAAT_MLP_DOWN, 4, x, x, x, x, None, x, x, x, None, x)
+
+
+def test_allreduce_bytes_matches_closed_form(caat):
+    # Appendix C: tokens*h*p activations per device per reduce; Appendix D: cut by 100(1-p) %.
+    c = caat.Context(4096, 11008, 8, 0.5, "bf16")
+    a = c.allreduce_bytes(16384, 2)
+    assert a["payload_per_rank"] == 16384 * 2048 * 2 == 67108864
+    assert a["payload_per_rank_p1"] == 16384 * 4096 * 2
+    assert a["ring_wire_per_rank"] == 2 * 7 * 67108864 // 8
+    from oracle import caat_oracle as O
+    o = O.allreduce_bytes(16384, 4096, 8, 2048, 2)
+    assert o["payload_per_rank"] == a["payload_per_rank"] and o["ring_wire_per_rank"] == a["ring_wire_per_rank"]
