@@ -1,17 +1,626 @@
-// Tensor-core GEMMs (placeholder translation unit; replaced by the tcgen05 kernels).
+// bf16 tensor-core GEMMs for sm_100a: TMA -> shared-memory ring -> tcgen05.mma with the
+// fp32 accumulator in tensor memory -> tcgen05.ld epilogue.
+//
+// One persistent, warp-specialised kernel serves the three contractions of the layer:
+//   forward   Zt = Y W^T        A = Y  (K-major),  B = W (K-major)
+//   dgrad     dY = dZt W        A = dZt (K-major), B = W (N-major: K_r contiguous)
+//   wgrad     dW = dZt^T Y      A = dZt (M-major: channels contiguous), B = Y (N-major)
+// where dZt / Zt live in the split scratch layout [shared once | private per rank].
+// Shared output columns of the forward accumulate over ALL ranks in one accumulator (the
+// partial channel-reduce of Eq. A3 becomes a longer contraction), so rank partials of the
+// shared channels never exist in memory.
+//
+// Roles per CTA (192 threads): warp 0 issues TMA loads, warp 1 issues MMAs and owns the
+// tensor-memory allocation, warps 2-5 drain accumulators (tcgen05.ld) and store.  Two
+// accumulators of up to 256 columns alternate so a tile's epilogue overlaps the next
+// tile's MMAs.  Every mbarrier wait is bounded; on a timeout the kernel records a status
+// word, drains its own copies in flight, frees tensor memory and returns.
+#include <cuda.h>
+
+#include <mutex>
+
 #include "caat_internal.h"
 
 namespace caat {
-bool tc_gemm_usable(const caat_ctx*, int) { return false; }
-cudaError_t launch_tc_forward(const RowparShapes&, const void*, const void*, void*, void*, cudaStream_t) {
-  return cudaErrorNotSupported;
+namespace {
+
+constexpr int BM = 128;           // rows of an output tile (UMMA M, cta_group::1)
+constexpr int BK = 64;            // contraction elements per pipeline stage (128 bytes of bf16)
+constexpr int UMMA_K = 16;        // contraction elements per tcgen05.mma (kind::f16)
+constexpr int kThreads = 192;
+constexpr int kAccCols = 256;     // column stride between the two accumulators
+constexpr int kTmemCols = 512;
+constexpr uint32_t kSpinCap = 1u << 22;
+constexpr int kMaxStages = 8;
+
+struct Unit {            // one contraction segment of a tile
+  int mapA, mapB;        // indices into the tensor-map array
+  int ak0, am0;          // offsets added to A's K / M coordinate
+  int bk0, bn0;          // offsets added to B's K / N coordinate
+  int a_zb, a_zq;        // A's z coordinate = b * a_zb + q * a_zq
+  int b_zb, b_zq;
+  int Q;                 // rank loop (forward shared columns: all ranks, else 1)
+  int ksteps;            // stages per q = ceil(extent / BK)
+};
+
+struct Region {          // a family of output tiles with the same operand wiring
+  int nunits;
+  Unit u[2];
+  int M, N, batch;       // valid output extents per batch
+  int mtiles, ntiles;
+  void* out;             // element (b, i, j) at out + (b * ldb + i * ldc + j) elements
+  long long ldc, ldb;
+  long long split_stride;  // elements between split-K partials (0: no split-K)
+};
+
+struct Params {
+  int nregions;
+  Region r[2];
+  int BN;                // tile width (UMMA N): multiple of 16 (of 64 when B is N-major)
+  int nstages;
+  int a_mn, b_mn;        // 1: operand is MN-major in global memory
+  int out_f32;
+  int splits;            // split-K factor (only with a single unit and Q == 1)
+  int tiles_r0;          // tiles of region 0 (including splits)
+  int tiles_total;
+  unsigned int* status;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-cudaError_t launch_tc_dgrad(const RowparShapes&, const void*, const void*, const void*, void*, cudaStream_t) {
-  return cudaErrorNotSupported;
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-cudaError_t launch_tc_wgrad(const RowparShapes&, const void*, const void*, const void*, float*, void*, size_t,
-                            cudaStream_t) {
-  return cudaErrorNotSupported;
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-size_t tc_wgrad_splitk_bytes(const RowparShapes&) { return 0; }
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the cap ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kSpinCap; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+//   K-major operand : rows of 128 bytes (64 bf16 of K), 8-row groups 1024 bytes apart (SBO).
+//   MN-major operand: 64-element (128-byte) MN chunks; within a chunk K rows are 128 bytes
+//                     apart, 8-row groups 1024 bytes apart (SBO); chunks LBO bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+struct TileCoord {
+  int region, b, mt, nt, split;
+};
+
+__device__ __forceinline__ TileCoord decode_tile(const Params& p, int tile) {
+  TileCoord c;
+  c.region = (tile >= p.tiles_r0) ? 1 : 0;
+  int rem = tile - (c.region ? p.tiles_r0 : 0);
+  const Region& r = p.r[c.region];
+  c.nt = rem % r.ntiles; rem /= r.ntiles;
+  c.split = rem % p.splits; rem /= p.splits;
+  c.b = rem % r.batch; rem /= r.batch;
+  c.mt = rem;
+  return c;
+}
+
+// k-step range of a unit for a split
+__device__ __forceinline__ void split_range(const Params& p, const Unit& u, int split, int& k_begin, int& k_end) {
+  if (p.splits == 1) { k_begin = 0; k_end = u.ksteps; return; }
+  const int per = (u.ksteps + p.splits - 1) / p.splits;
+  k_begin = split * per;
+  k_end = k_begin + per < u.ksteps ? k_begin + per : u.ksteps;
+  if (k_begin > k_end) k_begin = k_end;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
+               const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map3, const Params p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // carve: [stages x (A tile | B tile)] then barriers
+  const uint32_t a_bytes = BM * BK * 2;
+  const uint32_t b_bytes = (uint32_t)p.BN * BK * 2;
+  const uint32_t stage_bytes = a_bytes + b_bytes;
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t tiles_sa = smem_u32(base);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)p.nstages * stage_bytes);
+  // bars: full[nstages], empty[nstages], tfull[2], tempty[2]
+  const uint32_t full0 = smem_u32(bars);
+  const uint32_t empty0 = full0 + 8u * p.nstages;
+  const uint32_t tfull0 = empty0 + 8u * p.nstages;
+  const uint32_t tempty0 = tfull0 + 16u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * p.nstages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const CUtensorMap* maps[4] = {&map0, &map1, &map2, &map3};
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.nstages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      long long issued = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
+        const TileCoord c = decode_tile(p, tile);
+        const Region& r = p.r[c.region];
+        const int m0 = c.mt * BM, n0 = c.nt * p.BN;
+        for (int ui = 0; ui < r.nunits && ok; ++ui) {
+          const Unit& u = r.u[ui];
+          int kb, ke;
+          split_range(p, u, c.split, kb, ke);
+          for (int q = 0; q < u.Q && ok; ++q) {
+            const int az = c.b * u.a_zb + q * u.a_zq, bz = c.b * u.b_zb + q * u.b_zq;
+            for (int kk = kb; kk < ke; ++kk) {
+              if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+              const uint32_t fb = full0 + 8u * stage;
+              const uint32_t sa = tiles_sa + (uint32_t)stage * stage_bytes, sb = sa + a_bytes;
+              mbar_expect_tx(fb, stage_bytes);
+              if (!p.a_mn) {
+                tma_load_3d(sa, maps[u.mapA], u.ak0 + kk * BK, m0, az, fb);
+              } else {
+#pragma unroll
+                for (int ch = 0; ch < BM / 64; ++ch)
+                  tma_load_3d(sa + ch * (64 * BK * 2), maps[u.mapA], u.am0 + m0 + ch * 64, u.ak0 + kk * BK, az, fb);
+              }
+              if (!p.b_mn) {
+                tma_load_3d(sb, maps[u.mapB], u.bk0 + kk * BK, u.bn0 + n0, bz, fb);
+              } else {
+                for (int ch = 0; ch < p.BN / 64; ++ch)
+                  tma_load_3d(sb + ch * (64 * BK * 2), maps[u.mapB], u.bn0 + n0 + ch * 64, u.bk0 + kk * BK, bz, fb);
+              }
+              ++issued;
+              if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+            }
+          }
+        }
+      }
+      if (!ok) {
+        // gave up: flag it, then wait (bounded) for the copies this thread still has in flight
+        *abort_flag = 1;
+        atomicExch(p.status, 1u);
+        const int pending = issued < p.nstages ? (int)issued : p.nstages;
+        int s = stage; uint32_t ph = phase;
+        for (int k = 0; k < pending; ++k) {
+          if (--s < 0) { s = p.nstages - 1; ph ^= 1u; }
+          for (uint32_t it = 0; it < (1u << 20); ++it)
+            if (mbar_try(full0 + 8u * s, ph)) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
+                             ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
+        const TileCoord c = decode_tile(p, tile);
+        const Region& r = p.r[c.region];
+        if (!mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
+        uint32_t accumulate = 0;
+        for (int ui = 0; ui < r.nunits && ok; ++ui) {
+          const Unit& u = r.u[ui];
+          int kb, ke;
+          split_range(p, u, c.split, kb, ke);
+          for (int q = 0; q < u.Q && ok; ++q) {
+            for (int kk = kb; kk < ke; ++kk) {
+              if (!mbar_wait(full0 + 8u * stage, phase, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t sa = tiles_sa + (uint32_t)stage * stage_bytes, sb = sa + a_bytes;
+#pragma unroll
+              for (int k = 0; k < BK / UMMA_K; ++k) {
+                const uint64_t ad = p.a_mn ? make_desc(sa + k * (UMMA_K * 128), 64 * BK * 2, 1024)
+                                           : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
+                const uint64_t bd = p.b_mn ? make_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024)
+                                           : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
+                umma_bf16(d_tmem, ad, bd, idesc, accumulate);
+                accumulate = 1;
+              }
+              umma_commit(empty0 + 8u * stage);   // frees the stage once these MMAs have read it
+              if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+            }
+          }
+        }
+        if (ok) umma_commit(tfull0 + 8u * acc);    // accumulator complete
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(p.status, 2u); }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter+32)
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
+      const TileCoord c = decode_tile(p, tile);
+      const Region& r = p.r[c.region];
+      // a tile whose contraction range is empty leaves the accumulator undefined: its value is 0
+      int total_k = 0;
+      for (int ui = 0; ui < r.nunits; ++ui) {
+        int kb, ke;
+        split_range(p, r.u[ui], c.split, kb, ke);
+        total_k += (ke - kb) * r.u[ui].Q;
+      }
+      if (!mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = c.mt * BM + quarter * 32 + lane;
+      const int n0 = c.nt * p.BN;
+      const bool row_ok = row < r.M;
+      const long long obase = (long long)c.split * r.split_stride + (long long)c.b * r.ldb + (long long)row * r.ldc;
+      for (int cc = 0; cc < p.BN; cc += 32) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols + cc), v);
+        tmem_ld_wait();
+        if (total_k == 0) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = 0u;
+        }
+        int ncol = r.N - (n0 + cc);         // valid columns from here, within this tile
+        if (ncol > p.BN - cc) ncol = p.BN - cc;
+        if (row_ok && ncol > 0) {
+          if (p.out_f32) {
+            float* o = static_cast<float*>(r.out) + obase + n0 + cc;
+            if (ncol >= 32 && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 4)
+                *reinterpret_cast<float4*>(o + e) = make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]),
+                                                                __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+            } else {
+              for (int e = 0; e < 32 && e < ncol; ++e) o[e] = __uint_as_float(v[e]);
+            }
+          } else {
+            __nv_bfloat16* o = static_cast<__nv_bfloat16*>(r.out) + obase + n0 + cc;
+            if (ncol >= 32 && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
+#pragma unroll
+              for (int e = 0; e < 32; e += 8) {
+                uint32_t w[4];
+#pragma unroll
+                for (int q2 = 0; q2 < 4; ++q2) {
+                  __nv_bfloat162 bb = __floats2bfloat162_rn(__uint_as_float(v[e + 2 * q2]), __uint_as_float(v[e + 2 * q2 + 1]));
+                  w[q2] = *reinterpret_cast<uint32_t*>(&bb);
+                }
+                *reinterpret_cast<uint4*>(o + e) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            } else {
+              for (int e = 0; e < 32 && e < ncol; ++e) o[e] = __float2bfloat16_rn(__uint_as_float(v[e]));
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8u * acc);
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, 3u); }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// out[i] = sum_s part[s][i], s ascending (deterministic split-K reduction)
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const float4* __restrict__ part, float4* __restrict__ out,
+                                                            long long n4, int splits) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
+    float4 s = part[i];
+    for (int k = 1; k < splits; ++k) {
+      const float4 v = part[(long long)k * n4 + i];
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    out[i] = s;
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(f);
+  });
+  return fn;
+}
+
+// bf16 tensor [d2][d1][d0] (d0 contiguous) with row pitch ld1 and plane pitch ld2 (elements);
+// box = (b0, b1, 1) with 128-byte swizzle; out-of-range elements read as zero.
+bool make_map(CUtensorMap* m, const void* base, long long d0, long long d1, long long d2, long long ld1, long long ld2,
+              int b0, int b1) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  if (d0 < 1 || d1 < 1 || d2 < 1) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)d0, (cuuint64_t)d1, (cuuint64_t)d2};
+  cuuint64_t strides[2] = {(cuuint64_t)ld1 * 2, (cuuint64_t)ld2 * 2};
+  cuuint32_t box[3] = {(cuuint32_t)b0, (cuuint32_t)b1, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int pick_bn(int n, bool multiple_of_64) {
+  // widest tile that wastes little: minimise padded width, prefer the wider tile on ties
+  const int step = multiple_of_64 ? 64 : 32;   // the epilogue drains 32 columns at a time
+  int best = 256;
+  long long best_cost = -1;
+  for (int bn = 256; bn >= 64; bn -= step) {
+    const long long tiles = (n + bn - 1) / bn;
+    const long long cost = tiles * bn * 16 + tiles * 64;  // padded columns (x16) plus a per-tile overhead
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+  }
+  return best;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+cudaError_t launch(const CUtensorMap maps[4], Params& p, cudaStream_t st) {
+  const int stage_bytes = BM * BK * 2 + p.BN * BK * 2;
+  int nst = (227 * 1024 - 2048) / stage_bytes;
+  if (nst > kMaxStages) nst = kMaxStages;
+  if (nst < 2) return cudaErrorInvalidConfiguration;
+  p.nstages = nst;
+  const size_t smem = (size_t)nst * stage_bytes + 1024 /*alignment slack*/ + (2 * nst + 4) * 8 + 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  p.status = device_status_word();
+  if (!p.status) return cudaErrorUnknown;
+  int grid = p.tiles_total < sm_count() ? p.tiles_total : sm_count();
+  if (grid < 1) return cudaSuccess;
+  tc_gemm_kernel<<<grid, kThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+void finish_tiles(Params& p) {
+  for (int g = 0; g < p.nregions; ++g) {
+    Region& r = p.r[g];
+    r.mtiles = (r.M + BM - 1) / BM;
+    r.ntiles = (r.N + p.BN - 1) / p.BN;
+  }
+  p.tiles_r0 = p.r[0].mtiles * p.r[0].ntiles * p.r[0].batch * p.splits;
+  p.tiles_total = p.tiles_r0 + (p.nregions > 1 ? p.r[1].mtiles * p.r[1].ntiles * p.r[1].batch * p.splits : 0);
+}
+
+}  // namespace
+
+bool tc_gemm_usable(const caat_ctx* ctx, int K_r) {
+  return ctx->dtype == CAAT_BF16 && !ctx->force_simt && K_r % 8 == 0 && ctx->S % 8 == 0 && ctx->h % 8 == 0;
+}
+
+// ---- forward: zs[T,S] = sum_m Y[m] W[m][:S]^T ; zp[m][T,h-S] = Y[m] W[m][S:]^T
+cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* W, void* zs, void* zp,
+                              cudaStream_t st) {
+  CUtensorMap maps[4];
+  Params p{};
+  const int n_sh = s.S, n_pr = s.h - s.S;
+  p.BN = pick_bn(n_pr > 0 && n_sh > 0 ? (n_sh < n_pr ? n_sh : n_pr) : (n_sh > 0 ? n_sh : n_pr), false);
+  if (!make_map(&maps[0], Y, s.K_r, s.T, s.t, s.K_r, (long long)s.T * s.K_r, BK, BM)) return cudaErrorInvalidValue;
+  if (!make_map(&maps[1], W, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, BK, p.BN)) return cudaErrorInvalidValue;
+  maps[2] = maps[0];
+  maps[3] = maps[1];
+  p.a_mn = 0; p.b_mn = 0; p.out_f32 = 0; p.splits = 1;
+  const int ksteps = (s.K_r + BK - 1) / BK;
+  int g = 0;
+  if (n_sh > 0) {
+    Region& r = p.r[g++];
+    r.nunits = 1;
+    r.u[0] = Unit{0, 1, 0, 0, 0, 0, /*a_zb*/ 0, /*a_zq*/ 1, /*b_zb*/ 0, /*b_zq*/ 1, s.t, ksteps};
+    r.M = s.T; r.N = n_sh; r.batch = 1;
+    r.out = zs; r.ldc = s.S_hi; r.ldb = 0; r.split_stride = 0;
+  }
+  if (n_pr > 0) {
+    Region& r = p.r[g++];
+    r.nunits = 1;
+    r.u[0] = Unit{0, 1, 0, 0, 0, s.S, 1, 0, 1, 0, 1, ksteps};
+    r.M = s.T; r.N = n_pr; r.batch = s.t;
+    r.out = static_cast<__nv_bfloat16*>(zp) + (s.S - s.S_lo); r.ldc = s.P; r.ldb = (long long)s.T * s.P;
+    r.split_stride = 0;
+  }
+  p.nregions = g;
+  finish_tiles(p);
+  return launch(maps, p, st);
+}
+
+// ---- dgrad: dY[m] = gs W[m][:S] + zp[m] W[m][S:]
+cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* zp, const void* W, void* dY,
+                            cudaStream_t st) {
+  CUtensorMap maps[4];
+  Params p{};
+  p.BN = pick_bn(s.K_r, true);
+  const int n_sh = s.S, n_pr = s.h - s.S;
+  // B = W[m] as [h rows (contraction)][K_r contiguous (N)]: N-major, boxes of 64 (N) x 64 (K)
+  if (!make_map(&maps[1], W, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, 64, BK)) return cudaErrorInvalidValue;
+  bool okA0 = n_sh > 0 ? make_map(&maps[0], gs, n_sh, s.T, 1, s.S_hi, (long long)s.T * s.S_hi, BK, BM) : true;
+  bool okA1 = n_pr > 0 ? make_map(&maps[2], zp, s.P, s.T, s.t, s.P, (long long)s.T * s.P, BK, BM) : true;
+  if (!okA0 || !okA1) return cudaErrorInvalidValue;
+  if (n_sh == 0) maps[0] = maps[2];
+  if (n_pr == 0) maps[2] = maps[0];
+  maps[3] = maps[1];
+  p.a_mn = 0; p.b_mn = 1; p.out_f32 = 0; p.splits = 1;
+  Region& r = p.r[0];
+  int nu = 0;
+  if (n_sh > 0) r.u[nu++] = Unit{0, 1, 0, 0, 0, 0, 0, 0, 1, 0, 1, (n_sh + BK - 1) / BK};
+  if (n_pr > 0) r.u[nu++] = Unit{2, 1, s.S - s.S_lo, 0, s.S, 0, 1, 0, 1, 0, 1, (n_pr + BK - 1) / BK};
+  r.nunits = nu;
+  r.M = s.T; r.N = s.K_r; r.batch = s.t;
+  r.out = dY; r.ldc = s.K_r; r.ldb = (long long)s.T * s.K_r; r.split_stride = 0;
+  p.nregions = 1;
+  finish_tiles(p);
+  return launch(maps, p, st);
+}
+
+static int wgrad_splits(const RowparShapes& s, int BN) {
+  const long long mt = ((s.S + BM - 1) / BM) + ((s.h - s.S + BM - 1) / BM);
+  const long long tiles = mt * ((s.K_r + BN - 1) / BN) * s.t;
+  const int ksteps = (s.T + BK - 1) / BK;
+  int splits = 1;
+  const int sms = 148;
+  if (tiles < sms) splits = (int)((sms + tiles - 1) / tiles);
+  if (splits > 16) splits = 16;
+  while (splits > 1 && ksteps / splits < 8) --splits;   // keep at least 8 stages per split
+  return splits;
+}
+
+size_t tc_wgrad_splitk_bytes(const RowparShapes& s) {
+  const int splits = wgrad_splits(s, pick_bn(s.K_r, true));
+  return splits > 1 ? (size_t)splits * s.t * s.h * s.K_r * sizeof(float) : 0;
+}
+
+// ---- wgrad: dW[m][:S] = gs^T Y[m] ; dW[m][S:] = zp[m]^T Y[m]      (fp32 out)
+cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* zp, const void* Y, float* dW,
+                            void* splitk, size_t splitk_bytes, cudaStream_t st) {
+  CUtensorMap maps[4];
+  Params p{};
+  p.BN = pick_bn(s.K_r, true);
+  const int n_sh = s.S, n_pr = s.h - s.S;
+  const int splits = wgrad_splits(s, p.BN);
+  const long long dw_elems = (long long)s.t * s.h * s.K_r;
+  if (splits > 1 && splitk_bytes < (size_t)splits * dw_elems * sizeof(float)) return cudaErrorInvalidValue;
+  // A = dZt as [T rows (contraction)][channels contiguous (M)]: M-major, boxes of 64 (M) x 64 (K)
+  bool okA0 = n_sh > 0 ? make_map(&maps[0], gs, n_sh, s.T, 1, s.S_hi, (long long)s.T * s.S_hi, 64, BK) : true;
+  bool okA1 = n_pr > 0 ? make_map(&maps[2], zp, s.P, s.T, s.t, s.P, (long long)s.T * s.P, 64, BK) : true;
+  // B = Y[m] as [T rows (contraction)][K_r contiguous (N)]: N-major
+  if (!okA0 || !okA1 || !make_map(&maps[1], Y, s.K_r, s.T, s.t, s.K_r, (long long)s.T * s.K_r, 64, BK))
+    return cudaErrorInvalidValue;
+  if (n_sh == 0) maps[0] = maps[2];
+  if (n_pr == 0) maps[2] = maps[0];
+  maps[3] = maps[1];
+  p.a_mn = 1; p.b_mn = 1; p.out_f32 = 1; p.splits = splits;
+  const int ksteps = (s.T + BK - 1) / BK;
+  float* out = splits > 1 ? static_cast<float*>(splitk) : dW;
+  int g = 0;
+  if (n_sh > 0) {
+    Region& r = p.r[g++];
+    r.nunits = 1;
+    r.u[0] = Unit{0, 1, 0, 0, 0, 0, 0, 0, 1, 0, 1, ksteps};
+    r.M = n_sh; r.N = s.K_r; r.batch = s.t;
+    r.out = out; r.ldc = s.K_r; r.ldb = (long long)s.h * s.K_r; r.split_stride = splits > 1 ? dw_elems : 0;
+  }
+  if (n_pr > 0) {
+    Region& r = p.r[g++];
+    r.nunits = 1;
+    r.u[0] = Unit{2, 1, 0, s.S - s.S_lo, 0, 0, 1, 0, 1, 0, 1, ksteps};
+    r.M = n_pr; r.N = s.K_r; r.batch = s.t;
+    r.out = out + (long long)s.S * s.K_r; r.ldc = s.K_r; r.ldb = (long long)s.h * s.K_r;
+    r.split_stride = splits > 1 ? dw_elems : 0;
+  }
+  p.nregions = g;
+  finish_tiles(p);
+  cudaError_t e = launch(maps, p, st);
+  if (e != cudaSuccess) return e;
+  if (splits > 1) {
+    const long long n4 = dw_elems / 4;   // K_r is a multiple of 8
+    int blocks = (int)((n4 + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    splitk_reduce_kernel<<<blocks, 256, 0, st>>>(static_cast<const float4*>(splitk), reinterpret_cast<float4*>(dW), n4,
+                                                 splits);
+    count_launch();
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
 }  // namespace caat
