@@ -1,0 +1,436 @@
+#!/usr/bin/env python
+"""Benchmark of the CAAT-Net row-parallel hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input: block forward
+(attention-out layer, then MLP-down layer: GEMM + partial channel-reduce + residual +
+norm) followed, for training workloads, by the block backward.  The t tensor-parallel
+ranks are simulated as a batch dimension on one GPU.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) every GPU
+runs an independent replica of the workload (the path has no cross-GPU exchange step):
+weak scaling, no data-path collective; time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2506_19645_b200 import synthetic  # noqa: E402
+
+DEFAULT_WORKLOAD = "block_130m"
+METRIC = "CAAT block tokens/s (sim. TP=t, sync p) on 1 B200"
+SWEEP = ["block_1p1b_p100", "block_1p1b_p075", "block_1p1b_p050", "block_1p1b_p025", "block_7b"]
+
+
+# --------------------------------------------------------------------------- peaks
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured (MEASURED_PEAKS.json; sustained bf16 figure: kernels timed inside a long step)"}
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback (earlier measurement on this pool)"}
+
+
+def recorded_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch from a committed ncu capture (profiles/traffic.json), else None."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            return json.load(f).get(workload, {}).get(kernel)
+    except Exception:
+        return None
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons while the timed region runs (read-only NVML)."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                 "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self) -> dict:
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------- algorithmic work
+def layer_work(w, k_r, backward):
+    """Algorithmic flops and bytes of ONE layer per kernel kind (inputs read once, outputs
+    written once, given the kernel's interface; e = 2 bytes)."""
+    t, T, h, S, e = w.t, w.tokens, w.h, w.S, 2
+    K = k_r * t
+    zsz = (T * S + t * T * (h - S)) * e            # split scratch: shared once, private per rank
+    out = {
+        "tc_gemm_forward": {"flops": 2.0 * T * K * h, "bytes": (T * K + K * h) * e + zsz},
+        "rows_forward": {"flops": 0.0, "bytes": zsz + 3 * t * T * h * e + t * T * 4},
+    }
+    if backward:
+        out["rows_backward"] = {"flops": 0.0, "bytes": 4 * t * T * h * e + zsz + t * T * 4}
+        out["tc_gemm_dgrad"] = {"flops": 2.0 * T * K * h, "bytes": zsz + K * h * e + T * K * e}
+        out["tc_gemm_wgrad"] = {"flops": 2.0 * T * K * h, "bytes": zsz + T * K * e + K * h * 4}
+    return out
+
+
+def step_work(w):
+    tot = {}
+    for k_r in (w.kr_attn, w.kr_mlp):
+        for kind, v in layer_work(w, k_r, w.backward).items():
+            a = tot.setdefault(kind, {"flops": 0.0, "bytes": 0.0})
+            a["flops"] += v["flops"]
+            a["bytes"] += v["bytes"]
+    return tot
+
+
+def paper_level_work(w):
+    """Whole-path algorithmic work per step (no scratch traffic): the roofline of the path."""
+    t, T, h, e = w.t, w.tokens, w.h, 2
+    fl = by = 0.0
+    for k_r in (w.kr_attn, w.kr_mlp):
+        K = k_r * t
+        fl += 2.0 * T * K * h
+        by += e * (T * K + K * h + 3 * t * T * h)
+        if w.backward:
+            fl += 4.0 * T * K * h
+            by += e * (4 * t * T * h + 2 * T * K + K * h) + 4 * K * h
+    return fl, by
+
+
+# --------------------------------------------------------------------------- the CUDA arm
+class BlockRunner:
+    def __init__(self, w, device):
+        from paper_2506_19645_b200 import caat
+        self.caat, self.w, self.dev = caat, w, device
+        self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
+        self.inp = synthetic.block_inputs(w, device=device)
+        t, T, h = w.t, w.tokens, w.h
+        td = self.ctx.torch_dtype
+        mk = lambda *s, dt=td: torch.empty(*s, dtype=dt, device=device)
+        f32 = torch.float32
+        self.out = {"Hn1": mk(t, T, h), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=f32),
+                    "Hn2": mk(t, T, h), "X2": mk(t, T, h), "rstd2": mk(t, T, dt=f32)}
+        if w.backward:
+            self.out.update({"dY_attn": mk(t, T, w.kr_attn), "dW_o": mk(t, h, w.kr_attn, dt=f32),
+                             "dY_mlp": mk(t, T, w.kr_mlp), "dW_down": mk(t, h, w.kr_mlp, dt=f32),
+                             "dR0": mk(t, T, h), "dHn1": mk(t, T, h), "dgamma1": mk(h, dt=f32), "dgamma2": mk(h, dt=f32)})
+        self.ws = self.ctx.alloc_workspace(self.ctx.block_workspace_bytes(T, w.backward), device=device)
+
+    def step(self):
+        i, o, T = self.inp, self.out, self.w.tokens
+        self.ctx.block_forward(T, i["Y_attn"], i["W_o"], i["Y_mlp"], i["W_down"], i["R0"], i["gamma1"], None,
+                               i["gamma2"], None, o["Hn1"], o["X1"], o["rstd1"], None, o["Hn2"], o["X2"], o["rstd2"],
+                               None, self.ws)
+        if self.w.backward:
+            self.ctx.block_backward(T, i["dX1"], i["dX2"], i["dHn2"], i["Y_attn"], i["W_o"], i["Y_mlp"], i["W_down"],
+                                    o["Hn1"], o["rstd1"], None, o["Hn2"], o["rstd2"], None, i["gamma1"], i["gamma2"],
+                                    o["dY_attn"], o["dW_o"], o["dY_mlp"], o["dW_down"], o["dR0"], o["dHn1"],
+                                    o["dgamma1"], None, o["dgamma2"], None, self.ws)
+
+    def touched_bytes(self):
+        n = sum(v.numel() * v.element_size() for v in self.inp.values())
+        return n + sum(v.numel() * v.element_size() for v in self.out.values())
+
+
+def time_steps(runner, steps, dist_on):
+    """Device time of exactly `steps` steps (ms), CUDA events on the launching stream."""
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        runner.step()
+    e1.record()
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    return e0.elapsed_time(e1)
+
+
+def e2e_leg(runner, steps):
+    """Same step, but every step copies its inputs from pinned host memory and reads its
+    results back to the host; all of it inside the timed region."""
+    inp_host = {k: v.cpu().pin_memory() for k, v in runner.inp.items()}
+    out_host = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in runner.out.items()}
+    h2d = sum(v.numel() * v.element_size() for v in inp_host.values())
+    d2h = sum(v.numel() * v.element_size() for v in out_host.values())
+
+    def one():
+        for k, v in inp_host.items():
+            runner.inp[k].copy_(v, non_blocking=True)
+        runner.step()
+        for k, v in runner.out.items():
+            out_host[k].copy_(v, non_blocking=True)
+
+    one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return ms, h2d, d2h
+
+
+def oracle_sample_run(w, sample_tokens):
+    """One block forward(+backward) of the fp64 oracle on `sample_tokens` tokens of the workload."""
+    from oracle import caat_oracle as O
+    ws = w.with_tokens(sample_tokens)
+    d = {k: v.to(torch.float64).numpy() for k, v in synthetic.block_inputs(ws, device="cpu").items()}
+    S, alpha = ws.S, math.sqrt(ws.t)
+    t0 = time.perf_counter()
+    f = O.block_forward(d["Y_attn"], d["W_o"], d["Y_mlp"], d["W_down"], d["R0"], d["gamma1"], d["gamma2"], S=S, alpha=alpha)
+    if w.backward:
+        O.block_backward(d["dX1"], d["dX2"], d["dHn2"], d["Y_attn"], d["W_o"], d["Y_mlp"], d["W_down"], f["Hn1"],
+                         f["rstd1"], None, f["Hn2"], f["rstd2"], None, d["gamma1"], d["gamma2"], S=S, alpha=alpha)
+    return time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return len(os.sched_getaffinity(0))
+
+
+def cpu_baseline(w, target_s=12.0):
+    probe = min(256, w.tokens)
+    tp = oracle_sample_run(w, probe)
+    tp = min(tp, oracle_sample_run(w, probe))
+    n = int(target_s / max(tp / probe, 1e-9))
+    n = max(probe, min(w.tokens, n // 256 * 256 if n >= 256 else probe))
+    ts = oracle_sample_run(w, n)
+    return {"value": n / ts, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+            "sample": f"fp64 numpy oracle, block forward{'+backward' if w.backward else ''} on {n} of {w.tokens} tokens "
+                      f"of {w.name} (all {w.t} ranks), {ts:.2f} s; host has {len(os.sched_getaffinity(0))} usable cores"}
+
+
+def run_cuda(args):
+    from paper_2506_19645_b200 import caat
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist_on = world > 1
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if dist_on:
+        torch.distributed.init_process_group("nccl", device_id=dev)
+    w = synthetic.WORKLOADS[args.workload]
+    runner = BlockRunner(w, dev)
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        runner.step()
+    torch.cuda.synchronize()
+    assert runner.ctx.last_device_status() == caat.CAAT_OK
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = caat.kernel_launches()
+    ms = time_steps(runner, args.steps, dist_on)
+    launches = caat.kernel_launches() - l0
+    # second pass of the same K steps with CUDA events around every kernel (per-kernel device times)
+    caat.profile_begin(max(1024, launches + 64))
+    ms_prof = time_steps(runner, args.steps, dist_on)
+    prof = caat.profile_end()
+    clocks = sampler.stop()
+    if dist_on:
+        tms = torch.tensor([ms], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(tms, op=torch.distributed.ReduceOp.MAX)
+        ms = float(tms.item())
+
+    ms_step = ms / args.steps
+    value = world * w.tokens * args.steps / (ms * 1e-3)
+
+    result = None
+    if rank == 0:
+        peaks = measured_peaks()
+        work = step_work(w)
+        kernels = {}
+        for kind, (kms, n) in prof.items():
+            per_step_ms = kms / args.steps
+            wk = work.get(kind)
+            ent = {"ms_per_step": per_step_ms, "launches_per_step": n / args.steps, "share": kms / sum(v[0] for v in prof.values())}
+            if wk:
+                gbs = wk["bytes"] / (per_step_ms * 1e-3) / 1e9
+                tfs = wk["flops"] / (per_step_ms * 1e-3) / 1e12
+                t_hbm, t_tc = wk["bytes"] / (peaks["hbm_gbs"] * 1e9), wk["flops"] / (peaks["bf16_tflops"] * 1e12)
+                if t_tc > t_hbm:
+                    ent.update({"bound": "tensor", "achieved": tfs, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                "frac": tfs / peaks["bf16_tflops"]})
+                else:
+                    ent.update({"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                "frac": gbs / peaks["hbm_gbs"]})
+                ent["gbs"], ent["tflops"] = gbs, tfs
+            kernels[kind] = ent
+        top = max((k for k in kernels if "frac" in kernels[k]), key=lambda k: kernels[k]["ms_per_step"])
+        roof = {k: kernels[top][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
+        roof.update({"kernel": top, "traffic": recorded_traffic(top, w.name), "peak_source": peaks["source"],
+                     "timed": f"second pass of {args.steps} steps with CUDA events around every kernel launch "
+                              f"({ms_prof / args.steps:.4f} ms/step with events)"})
+        fl, by = paper_level_work(w)
+        t_roof = max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9))
+        e2e = None
+        try:
+            ems, h2d, d2h = e2e_leg(runner, max(2, min(args.steps, 5)))
+            e2e = {"value": w.tokens / (ems * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                   "d2h_bytes_per_step": d2h, "ms_per_step": ems}
+        except Exception as ex:  # pinned-memory exhaustion on a small host
+            e2e = {"value": None, "unit": "tokens/s", "error": str(ex)[:200]}
+        ar = runner.ctx.allreduce_bytes(w.tokens, 2)
+        result = {
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p,
+                       "S": w.S, "passes": "forward+backward" if w.backward else "forward",
+                       "private_scale": "sqrt(t)", "norm": "rmsnorm", "parallelism": f"replicas x{world}",
+                       "l2": f"inputs+outputs touched per step {runner.touched_bytes() / 1e6:.0f} MB > 126 MB L2"},
+            "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "roofline": roof, "kernels": kernels,
+            "path_roofline": {"flops_per_step": fl, "bytes_per_step": by, "roofline_ms": t_roof * 1e3,
+                              "frac": t_roof * 1e3 / ms_step},
+            "collective_bytes_analytic": {"per_reduce": ar, "reduces_per_step": 4 if w.backward else 2},
+        }
+    del runner
+    torch.cuda.empty_cache()
+
+    if rank == 0 and not args.no_sweep and world == 1:
+        sweep = []
+        for name in SWEEP:
+            if name == w.name:
+                continue
+            try:
+                r = BlockRunner(synthetic.WORKLOADS[name], dev)
+                for _ in range(3):
+                    r.step()
+                k = max(3, min(args.steps, 10))
+                sms = time_steps(r, k, False) / k
+                fl, by = paper_level_work(r.w)
+                peaks = measured_peaks()
+                t_roof = max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e3
+                sweep.append({"workload": name, "p": r.w.p, "ms_per_step": sms, "tokens_per_s": r.w.tokens / (sms * 1e-3),
+                              "path_roofline_frac": t_roof / sms,
+                              "allreduce_payload_bytes": r.ctx.allreduce_bytes(r.w.tokens, 2)["payload_per_rank"]})
+                del r
+                torch.cuda.empty_cache()
+            except Exception as ex:
+                sweep.append({"workload": name, "error": str(ex)[:200]})
+        result["sweep"] = sweep
+    if rank == 0:
+        if not args.no_cpu and world == 1:
+            result["cpu_baseline"] = cpu_baseline(w)
+        else:
+            result["cpu_baseline"] = None
+        print(json.dumps(result), flush=True)
+    if dist_on:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+
+
+# --------------------------------------------------------------------------- the reference arm (oracle on host cores)
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    w = synthetic.WORKLOADS[args.workload]
+    probe = min(256, w.tokens)
+    tp = min(oracle_sample_run(w, probe), oracle_sample_run(w, probe))
+    budget = 150.0 / max(1, args.steps + args.warmup)            # seconds per step so the run ends within minutes
+    n = int(min(budget, 1.0) / max(tp / probe, 1e-9))
+    n = max(probe, min(w.tokens, n // 256 * 256 if n >= 256 else probe))
+    for _ in range(args.warmup):
+        oracle_sample_run(w, n)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_run(w, n)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = (f"fp64 numpy oracle, block forward{'+backward' if w.backward else ''}, each step a sample of {n} of "
+              f"{w.tokens} tokens of {w.name}; host has {len(os.sched_getaffinity(0))} usable cores")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p, "S": w.S,
+                   "passes": "forward+backward" if w.backward else "forward", "sample_tokens": n},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synthetic.WORKLOADS))
+    ap.add_argument("--no-sweep", action="store_true", help="skip the other workloads' tokens/s")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
+    args = ap.parse_args()
+    if args.steps < 1:
+        raise SystemExit("--steps must be >= 1")
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -197,6 +197,29 @@ caat_status caat_last_device_status(const caat_ctx *ctx, void *cuda_stream);
  * was loaded (for benchmarks' launch accounting). */
 unsigned long long caat_kernel_launches(void);
 
+/*
+ * Per-kernel timing aid for benchmarks (the paper has no counterpart).  Between
+ * caat_profile_begin and caat_profile_end every kernel launched through the library is
+ * bracketed by CUDA events on its launching stream (up to max_launches launches; later
+ * ones are counted but not timed).  caat_profile_end waits for the recorded events and
+ * returns, per kernel kind, the summed device time in milliseconds and the number of
+ * timed launches.  Process-wide, not thread-safe; event objects are kept for reuse.
+ */
+typedef enum {
+  CAAT_K_ROWS_FORWARD = 0,   /* reduce hand-off + scale + residual + norm           */
+  CAAT_K_ROWS_BACKWARD = 1,  /* norm backward + residual gradient + backward reduce */
+  CAAT_K_NORMGRAD_REDUCE = 2,/* second stage of dgamma / dbeta                      */
+  CAAT_K_GEMM_CUDA_CORE = 3, /* CUDA-core GEMM (fp32 and unaligned shapes)          */
+  CAAT_K_TC_FORWARD = 4,     /* tcgen05 GEMM, forward                               */
+  CAAT_K_TC_DGRAD = 5,       /* tcgen05 GEMM, data gradient                         */
+  CAAT_K_TC_WGRAD = 6,       /* tcgen05 GEMM, weight gradient                       */
+  CAAT_K_SPLITK_REDUCE = 7,  /* split-K reduction of the weight gradient            */
+  CAAT_K_COUNT = 8
+} caat_kernel_kind;
+caat_status caat_profile_begin(int max_launches);
+caat_status caat_profile_end(int n_kinds, double *ms_by_kind, unsigned long long *launches_by_kind);
+const char *caat_kernel_kind_name(int kind);
+
 #ifdef __cplusplus
 }
 #endif

@@ -45,6 +45,9 @@ _sigs = {
     "caat_allreduce_bytes": (c_int, [_P, c_int, c_int] + [POINTER(c_ulonglong)] * 3),
     "caat_last_device_status": (c_int, [_P, _P]),
     "caat_kernel_launches": (c_ulonglong, []),
+    "caat_profile_begin": (c_int, [c_int]),
+    "caat_profile_end": (c_int, [c_int, POINTER(c_double), POINTER(c_ulonglong)]),
+    "caat_kernel_kind_name": (c_char_p, [c_int]),
 }
 for _name, (_res, _args) in _sigs.items():
     _f = getattr(lib, _name)
@@ -239,3 +242,18 @@ class Context:
 
 def kernel_launches() -> int:
     return int(lib.caat_kernel_launches())
+
+
+CAAT_K_COUNT = 8
+
+
+def profile_begin(max_launches: int = 65536):
+    _check(lib.caat_profile_begin(max_launches), "caat_profile_begin")
+
+
+def profile_end() -> dict:
+    """{kernel kind name: (milliseconds, timed launches)} for the kinds that ran."""
+    ms = (c_double * CAAT_K_COUNT)()
+    n = (c_ulonglong * CAAT_K_COUNT)()
+    _check(lib.caat_profile_end(CAAT_K_COUNT, ms, n), "caat_profile_end")
+    return {lib.caat_kernel_kind_name(k).decode(): (ms[k], int(n[k])) for k in range(CAAT_K_COUNT) if n[k]}

@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "caat_internal.h"
 
@@ -14,7 +15,26 @@ static thread_local char g_cuda_err[256] = "";
 
 __device__ unsigned int g_status_word = 0;
 
-void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+// ---- optional per-kernel timing (benchmark aid) --------------------------------
+struct Profiler {
+  bool on = false;
+  std::vector<cudaEvent_t> ev;   // 2 per record
+  std::vector<int> kind;
+  int used = 0;
+};
+static Profiler g_prof;
+
+LaunchScope::LaunchScope(int kind, cudaStream_t s) : slot(-1), st(s) {
+  g_launches.fetch_add(1ull, std::memory_order_relaxed);
+  if (g_prof.on && g_prof.used < (int)g_prof.kind.size()) {
+    slot = g_prof.used++;
+    g_prof.kind[slot] = kind;
+    cudaEventRecord(g_prof.ev[2 * slot], st);
+  }
+}
+LaunchScope::~LaunchScope() {
+  if (slot >= 0) cudaEventRecord(g_prof.ev[2 * slot + 1], st);
+}
 
 unsigned int* device_status_word() {
   unsigned int* p = nullptr;
@@ -337,5 +357,51 @@ caat_status caat_last_device_status(const caat_ctx* ctx, void* cuda_stream) {
 }
 
 unsigned long long caat_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+caat_status caat_profile_begin(int max_launches) {
+  if (max_launches < 1 || max_launches > (1 << 20)) return CAAT_EINVAL;
+  if (g_prof.on) return CAAT_EINVAL;
+  while ((int)g_prof.ev.size() < 2 * max_launches) {
+    cudaEvent_t e;
+    cudaError_t ce = cudaEventCreate(&e);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    g_prof.ev.push_back(e);
+  }
+  g_prof.kind.assign(max_launches, -1);
+  g_prof.used = 0;
+  g_prof.on = true;
+  return CAAT_OK;
+}
+
+caat_status caat_profile_end(int n_kinds, double* ms_by_kind, unsigned long long* launches_by_kind) {
+  if (!g_prof.on) return CAAT_EINVAL;
+  g_prof.on = false;
+  if (n_kinds < 1 || !ms_by_kind || !launches_by_kind) return CAAT_EINVAL;
+  for (int k = 0; k < n_kinds; ++k) { ms_by_kind[k] = 0.0; launches_by_kind[k] = 0; }
+  for (int i = 0; i < g_prof.used; ++i) {
+    cudaError_t ce = cudaEventSynchronize(g_prof.ev[2 * i + 1]);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    float ms = 0.f;
+    ce = cudaEventElapsedTime(&ms, g_prof.ev[2 * i], g_prof.ev[2 * i + 1]);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    const int k = g_prof.kind[i];
+    if (k >= 0 && k < n_kinds) { ms_by_kind[k] += ms; launches_by_kind[k] += 1; }
+  }
+  return CAAT_OK;
+}
+
+const char* caat_kernel_kind_name(int kind) {
+  switch (kind) {
+    case CAAT_K_ROWS_FORWARD: return "rows_forward";
+    case CAAT_K_ROWS_BACKWARD: return "rows_backward";
+    case CAAT_K_NORMGRAD_REDUCE: return "normgrad_reduce";
+    case CAAT_K_GEMM_CUDA_CORE: return "gemm_cuda_core";
+    case CAAT_K_TC_FORWARD: return "tc_gemm_forward";
+    case CAAT_K_TC_DGRAD: return "tc_gemm_dgrad";
+    case CAAT_K_TC_WGRAD: return "tc_gemm_wgrad";
+    case CAAT_K_SPLITK_REDUCE: return "splitk_reduce";
+  }
+  return "";
+}
 
 }  // extern "C"

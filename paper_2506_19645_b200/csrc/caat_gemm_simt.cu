@@ -104,11 +104,11 @@ cudaError_t launch_gemm_simt(const GemmProblem& g, caat_dtype dtype, cudaStream_
   if (g.M <= 0 || g.N <= 0 || g.batch <= 0) return cudaSuccess;
   const dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
   if (grid.y > 65535 || grid.z > 65535) return cudaErrorInvalidConfiguration;
+  LaunchScope scope(CAAT_K_GEMM_CUDA_CORE, st);
   if (dtype == CAAT_BF16)
     gemm_simt_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(g);
   else
     gemm_simt_kernel<float><<<grid, 256, 0, st>>>(g);
-  count_launch();
   return cudaGetLastError();
 }
 

@@ -452,7 +452,7 @@ int sm_count() {
   return n;
 }
 
-cudaError_t launch(const CUtensorMap maps[4], Params& p, cudaStream_t st) {
+cudaError_t launch(const CUtensorMap maps[4], Params& p, int kind, cudaStream_t st) {
   const int stage_bytes = BM * BK * 2 + p.BN * BK * 2;
   int nst = (227 * 1024 - 2048) / stage_bytes;
   if (nst > kMaxStages) nst = kMaxStages;
@@ -469,8 +469,8 @@ cudaError_t launch(const CUtensorMap maps[4], Params& p, cudaStream_t st) {
   if (!p.status) return cudaErrorUnknown;
   int grid = p.tiles_total < sm_count() ? p.tiles_total : sm_count();
   if (grid < 1) return cudaSuccess;
+  LaunchScope scope(kind, st);
   tc_gemm_kernel<<<grid, kThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], p);
-  count_launch();
   return cudaGetLastError();
 }
 
@@ -521,7 +521,7 @@ cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* 
   }
   p.nregions = g;
   finish_tiles(p);
-  return launch(maps, p, st);
+  return launch(maps, p, CAAT_K_TC_FORWARD, st);
 }
 
 // ---- dgrad: dY[m] = gs W[m][:S] + zp[m] W[m][S:]
@@ -549,7 +549,7 @@ cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* z
   r.out = dY; r.ldc = s.K_r; r.ldb = (long long)s.T * s.K_r; r.split_stride = 0;
   p.nregions = 1;
   finish_tiles(p);
-  return launch(maps, p, st);
+  return launch(maps, p, CAAT_K_TC_DGRAD, st);
 }
 
 static int wgrad_splits(const RowparShapes& s, int BN) {
@@ -609,15 +609,15 @@ cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* z
   }
   p.nregions = g;
   finish_tiles(p);
-  cudaError_t e = launch(maps, p, st);
+  cudaError_t e = launch(maps, p, CAAT_K_TC_WGRAD, st);
   if (e != cudaSuccess) return e;
   if (splits > 1) {
     const long long n4 = dw_elems / 4;   // K_r is a multiple of 8
     int blocks = (int)((n4 + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
+    LaunchScope scope(CAAT_K_SPLITK_REDUCE, st);
     splitk_reduce_kernel<<<blocks, 256, 0, st>>>(static_cast<const float4*>(splitk), reinterpret_cast<float4*>(dW), n4,
                                                  splits);
-    count_launch();
     e = cudaGetLastError();
   }
   return e;

@@ -107,7 +107,14 @@ cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, cudaStre
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype);
 
 // ---- bookkeeping ------------------------------------------------------------
-void count_launch(int n = 1);
+// Brackets one kernel launch: counts it and, while profiling is on, records a CUDA event
+// before and after it on the launching stream.
+struct LaunchScope {
+  LaunchScope(int kind, cudaStream_t st);
+  ~LaunchScope();
+  int slot;
+  cudaStream_t st;
+};
 unsigned int* device_status_word();  // device address of the status word (per device)
 
 }  // namespace caat

@@ -397,13 +397,13 @@ template <typename T_>
 static cudaError_t launch_fwd_t(const RowFwdArgs& a, const RowGeom& g, cudaStream_t st) {
   const dim3 block(g.TX, g.TY);
   const dim3 grid((a.T + g.TY - 1) / g.TY);
+  LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
   switch (g.CPT) {
     case 1: rows_forward_kernel<T_, 1><<<grid, block, g.smem_fwd, st>>>(a); break;
     case 2: rows_forward_kernel<T_, 2><<<grid, block, g.smem_fwd, st>>>(a); break;
     case 4: rows_forward_kernel<T_, 4><<<grid, block, g.smem_fwd, st>>>(a); break;
     default: return cudaErrorInvalidValue;
   }
-  count_launch();
   return cudaGetLastError();
 }
 
@@ -426,13 +426,13 @@ static cudaError_t launch_bwd_t(const RowBwdArgs& a, const RowGeom& g, int rows,
     }
     if (e != cudaSuccess) return e;
   }
+  LaunchScope scope(CAAT_K_ROWS_BACKWARD, st);
   switch (g.CPT) {
     case 1: rows_backward_kernel<T_, 1><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
     case 2: rows_backward_kernel<T_, 2><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
     case 4: rows_backward_kernel<T_, 4><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
     default: return cudaErrorInvalidValue;
   }
-  count_launch();
   return cudaGetLastError();
 }
 
@@ -443,11 +443,13 @@ cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, cudaStre
   if (e != cudaSuccess) return e;
   const dim3 rb(32, 32);
   const dim3 rg((a.h + 31) / 32);
-  reduce_partials_kernel<<<rg, rb, 0, st>>>(a.dgpart, a.dgamma, rows, a.h);
-  count_launch();
+  {
+    LaunchScope scope(CAAT_K_NORMGRAD_REDUCE, st);
+    reduce_partials_kernel<<<rg, rb, 0, st>>>(a.dgpart, a.dgamma, rows, a.h);
+  }
   if (a.norm == 1 && a.dbeta && a.dbpart) {
+    LaunchScope scope(CAAT_K_NORMGRAD_REDUCE, st);
     reduce_partials_kernel<<<rg, rb, 0, st>>>(a.dbpart, a.dbeta, rows, a.h);
-    count_launch();
   }
   return cudaGetLastError();
 }
