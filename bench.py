@@ -61,7 +61,7 @@ def recorded_traffic(kernel: str, workload: str):
 class ClockSampler:
     """Samples SM clock and throttle reasons while the timed region runs (read-only NVML)."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.005):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
         self._thread = None
@@ -273,6 +273,8 @@ def run_cuda(args):
     if dist_on:
         torch.distributed.init_process_group("nccl", device_id=dev)
     w = synthetic.WORKLOADS[args.workload]
+    if args.tokens > 0:
+        w = w.with_tokens(args.tokens)
     runner = BlockRunner(w, dev)
     warm = max(args.warmup, 3)
     for _ in range(warm):
@@ -328,6 +330,8 @@ def run_cuda(args):
         t_roof = max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9))
         e2e = None
         try:
+            if args.no_e2e:
+                raise RuntimeError("skipped (--no-e2e)")
             ems, h2d, d2h = e2e_leg(runner, max(2, min(args.steps, 5)))
             e2e = {"value": w.tokens / (ems * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                    "d2h_bytes_per_step": d2h, "ms_per_step": ems}
@@ -423,6 +427,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synthetic.WORKLOADS))
     ap.add_argument("--no-sweep", action="store_true", help="skip the other workloads' tokens/s")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling on a small case)")
     args = ap.parse_args()
     if args.steps < 1:
         raise SystemExit("--steps must be >= 1")

@@ -20,7 +20,7 @@ CAAT_F32, CAAT_BF16 = 0, 1
 CAAT_ATTN_OUT, CAAT_MLP_DOWN = 0, 1
 (CAAT_OK, CAAT_EINVAL, CAAT_ESHAPE, CAAT_EALIGN, CAAT_EWORKSPACE, CAAT_EUNSUPPORTED, CAAT_ECUDA,
  CAAT_ETIMEOUT) = range(8)
-CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM = range(5)
+CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM, CAAT_OPT_ROWS = range(6)
 RMSNORM, LAYERNORM = 0, 1
 
 if not os.path.exists(LIB_PATH):

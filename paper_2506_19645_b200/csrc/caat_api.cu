@@ -132,7 +132,7 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
   }
   RowFwdArgs a{zs, zp, R, gamma, beta, Hn, X, rstd, mean, t, T, h, S, L.S_lo, L.S_hi, L.P,
                (float)ctx->alpha, (float)ctx->eps, ctx->norm};
-  ce = launch_rows_forward(a, ctx->dtype, st);
+  ce = launch_rows_forward(a, ctx->dtype, ctx->direct_rows, st);
   if (ce != cudaSuccess) return cuda_fail(ce);
   return CAAT_OK;
 }
@@ -153,7 +153,7 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
   RowBwdArgs a{dX, dHn, Hn, gamma, rstd, mean, dR, gs, zp,
                reinterpret_cast<float*>(wsb + L.dgpart_off), reinterpret_cast<float*>(wsb + L.dbpart_off),
                dgamma, dbeta, t, T, h, S, L.S_lo, L.S_hi, L.P, (float)ctx->alpha, ctx->norm};
-  ce = launch_rows_backward(a, ctx->dtype, st);
+  ce = launch_rows_backward(a, ctx->dtype, ctx->direct_rows, st);
   if (ce != cudaSuccess) return cuda_fail(ce);
 
   if (tc_gemm_usable(ctx, K_r)) {
@@ -213,7 +213,7 @@ caat_status caat_create(int h, int ffn, int t, double p, caat_dtype dtype, caat_
   c->h = h; c->ffn = ffn; c->t = t; c->p = p; c->dtype = dtype;
   c->S = (int)std::floor((double)h * p);   // Eq. A3: l < floor(h p) is shared
   c->alpha = std::sqrt((double)t);         // Section 4: private channels times sqrt(r)
-  c->norm = 0; c->eps = 1e-5; c->force_simt = 0;
+  c->norm = 0; c->eps = 1e-5; c->force_simt = 0; c->direct_rows = 0;
   *out = c;
   return CAAT_OK;
 }
@@ -237,6 +237,9 @@ caat_status caat_set_option(caat_ctx* ctx, caat_option opt, double value) {
     case CAAT_OPT_GEMM:
       if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
       ctx->force_simt = (int)value; return CAAT_OK;
+    case CAAT_OPT_ROWS:
+      if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
+      ctx->direct_rows = (int)value; return CAAT_OK;
   }
   return CAAT_EINVAL;
 }

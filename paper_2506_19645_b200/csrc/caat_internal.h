@@ -16,6 +16,7 @@ struct caat_ctx {
   int norm;        // 0 RMSNorm, 1 LayerNorm
   double eps;
   int force_simt;  // CAAT_OPT_GEMM
+  int direct_rows; // CAAT_OPT_ROWS
 };
 
 namespace caat {
@@ -91,7 +92,11 @@ struct RowFwdArgs {
   float alpha, eps;
   int norm;
 };
-cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st);
+// direct != 0 forces the plain-load kernels; otherwise the bulk-copy staged kernels run
+// whenever a ring of at least two stages fits in shared memory.
+cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
+cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st);
+bool rows_staged_usable(int h, int t, int S_lo, int S_hi, caat_dtype dtype, bool backward);
 
 struct RowBwdArgs {
   const void *dX, *dHn, *Hn, *gamma;
@@ -103,7 +108,9 @@ struct RowBwdArgs {
   float alpha;
   int norm;
 };
-cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, cudaStream_t st);
+cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
+cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,
+                                        cudaStream_t st);
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype);
 
 // ---- bookkeeping ------------------------------------------------------------

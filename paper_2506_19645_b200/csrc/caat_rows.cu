@@ -12,99 +12,21 @@
 // norm-parameter gradients are therefore thread-local and run in a fixed order.
 // Row statistics need one CTA-wide reduction per rank; the next rank's loads are issued
 // before it so that HBM requests stay in flight across the barrier.
-#include "caat_internal.h"
+//
+// These kernels move 3-5 bytes per arithmetic instruction, so the instruction count per
+// 16-byte chunk decides whether they reach HBM speed: the norm kind and the number of
+// chunks per thread are template parameters, pointers advance by one add per rank, and
+// the shared/private class of a chunk is resolved by a branch per chunk, not per element.
+#include "caat_rows_common.cuh"
 
 namespace caat {
 namespace {
 
-template <typename T_>
-struct VT;
-template <>
-struct VT<float> {
-  static constexpr int N = 4;
-  using raw = float4;
-  static __device__ __forceinline__ void unpack(const raw& r, float* f) {
-    f[0] = r.x; f[1] = r.y; f[2] = r.z; f[3] = r.w;
-  }
-  static __device__ __forceinline__ raw pack(const float* f) { return make_float4(f[0], f[1], f[2], f[3]); }
-  static __device__ __forceinline__ float round(float x) { return x; }
-};
-template <>
-struct VT<__nv_bfloat16> {
-  static constexpr int N = 8;
-  using raw = uint4;
-  static __device__ __forceinline__ void unpack(const raw& r, float* f) {
-    const unsigned w[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      f[2 * q] = __uint_as_float(w[q] << 16);
-      f[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
-    }
-  }
-  static __device__ __forceinline__ raw pack(const float* f) {
-    unsigned w[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      __nv_bfloat162 b = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
-      w[q] = *reinterpret_cast<unsigned*>(&b);
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-  }
-  static __device__ __forceinline__ float round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
-};
-
-template <typename raw>
-__device__ __forceinline__ raw ld_vec(const void* base, long long elem_off, int esz) {
-  return *reinterpret_cast<const raw*>(static_cast<const char*>(base) + elem_off * esz);
-}
-template <typename raw>
-__device__ __forceinline__ void st_vec(void* base, long long elem_off, int esz, const raw& v) {
-  *reinterpret_cast<raw*>(static_cast<char*>(base) + elem_off * esz) = v;
-}
-template <typename raw>
-__device__ __forceinline__ raw zero_raw();
-template <>
-__device__ __forceinline__ float4 zero_raw<float4>() { return make_float4(0.f, 0.f, 0.f, 0.f); }
-template <>
-__device__ __forceinline__ uint4 zero_raw<uint4>() { return make_uint4(0u, 0u, 0u, 0u); }
-
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-// Sum of NV values over the TX threads of one token row.  `red` holds
-// [2][TY][warps_x][NV] floats; `par` alternates so that one barrier per call suffices.
-template <int NV>
-__device__ __forceinline__ void row_reduce(float (&v)[NV], float* red, int& par) {
-  const int warps_x = blockDim.x >> 5;
-#pragma unroll
-  for (int q = 0; q < NV; ++q) v[q] = warp_sum(v[q]);
-  if (warps_x == 1) return;
-  float* buf = red + ((size_t)(par * blockDim.y + threadIdx.y) * warps_x) * NV;
-  if ((threadIdx.x & 31) == 0) {
-#pragma unroll
-    for (int q = 0; q < NV; ++q) buf[(threadIdx.x >> 5) * NV + q] = v[q];
-  }
-  __syncthreads();
-#pragma unroll
-  for (int q = 0; q < NV; ++q) {
-    float s = 0.f;
-    for (int w = 0; w < warps_x; ++w) s += buf[w * NV + q];
-    v[q] = s;
-  }
-  par ^= 1;
-}
-
-// column class of a chunk [col, col+V): 0 all shared, 1 all private, 2 mixed
-__device__ __forceinline__ int chunk_class(int col, int V, int S) {
-  return (col + V <= S) ? 0 : (col >= S ? 1 : 2);
-}
+using namespace rows;
 
 // ------------------------------------------------------------------ forward
-template <typename T_, int CPT>
-__global__ void __launch_bounds__(512) rows_forward_kernel(RowFwdArgs a) {
+template <typename T_, int CPT, bool LN>
+__global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_forward_kernel(const RowFwdArgs a) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
   constexpr int V = V_::N;
@@ -114,11 +36,17 @@ __global__ void __launch_bounds__(512) rows_forward_kernel(RowFwdArgs a) {
   const int TX = blockDim.x;
   const long long i = (long long)blockIdx.x * blockDim.y + threadIdx.y;
   const bool valid = i < a.T;
-  const bool ln = a.norm == 1;
+  const float inv_h = 1.0f / (float)a.h;
+  const long long rank_h = (long long)a.T * a.h * ES;   // byte stride between ranks
+  const long long rank_p = (long long)a.T * a.P * ES;
 
   int col[CPT], cls[CPT];
   bool act[CPT];
   float gam[CPT][V], bet[CPT][V], zs[CPT][V];
+  const char* pR[CPT];
+  const char* pZ[CPT];
+  char* pHn[CPT];
+  char* pX[CPT];
 #pragma unroll
   for (int j = 0; j < CPT; ++j) {
     col[j] = (threadIdx.x + j * TX) * V;
@@ -126,32 +54,37 @@ __global__ void __launch_bounds__(512) rows_forward_kernel(RowFwdArgs a) {
     cls[j] = chunk_class(col[j], V, a.S);
 #pragma unroll
     for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; bet[j][e] = 0.f; zs[j][e] = 0.f; }
+    const long long off_h = (i * a.h + col[j]) * ES;
+    pR[j] = static_cast<const char*>(a.R) + off_h;
+    pHn[j] = static_cast<char*>(a.Hn) + off_h;
+    pX[j] = static_cast<char*>(a.X) + off_h;
+    pZ[j] = static_cast<const char*>(a.zp) + (i * a.P + (col[j] - a.S_lo)) * ES;
     if (act[j]) {
-      V_::unpack(ld_vec<raw>(a.gamma, col[j], ES), gam[j]);
-      if (ln && a.beta) V_::unpack(ld_vec<raw>(a.beta, col[j], ES), bet[j]);
-      if (cls[j] != 1) V_::unpack(ld_vec<raw>(a.zs, i * a.S_hi + col[j], ES), zs[j]);
+      V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+      if (LN && a.beta) V_::unpack(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
+      if (cls[j] != 1) V_::unpack(ldg<raw>(static_cast<const char*>(a.zs) + (i * a.S_hi + col[j]) * ES), zs[j]);
     }
   }
 
   raw rR[CPT], rZ[CPT];
-  auto issue = [&](int m, raw(&R_)[CPT], raw(&Z_)[CPT]) {
 #pragma unroll
-    for (int j = 0; j < CPT; ++j) {
-      R_[j] = zero_raw<raw>();
-      Z_[j] = zero_raw<raw>();
-      if (act[j]) {
-        const long long row = (long long)m * a.T + i;
-        R_[j] = ld_vec<raw>(a.R, row * a.h + col[j], ES);
-        if (cls[j] != 0) Z_[j] = ld_vec<raw>(a.zp, row * a.P + (col[j] - a.S_lo), ES);
-      }
-    }
-  };
-  issue(0, rR, rZ);
+  for (int j = 0; j < CPT; ++j) {
+    rR[j] = act[j] ? ldg<raw>(pR[j]) : zero_raw<raw>();
+    rZ[j] = (act[j] && cls[j] != 0) ? ldg<raw>(pZ[j]) : zero_raw<raw>();
+  }
+  float* rstd_p = a.rstd + i;
+  float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
 
   for (int m = 0; m < a.t; ++m) {
     raw nR[CPT], nZ[CPT];
-    if (m + 1 < a.t) issue(m + 1, nR, nZ);
-    const long long row = (long long)m * a.T + i;
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) {   // next rank's loads go out before this rank's barrier
+      pR[j] += rank_h;
+      pZ[j] += rank_p;
+      const bool more = act[j] && (m + 1 < a.t);
+      nR[j] = more ? ldg<raw>(pR[j]) : zero_raw<raw>();
+      nZ[j] = (more && cls[j] != 0) ? ldg<raw>(pZ[j]) : zero_raw<raw>();
+    }
 
     float hn[CPT][V];
     float st[1] = {0.f};
@@ -159,53 +92,65 @@ __global__ void __launch_bounds__(512) rows_forward_kernel(RowFwdArgs a) {
     for (int j = 0; j < CPT; ++j) {
       float r[V], zp[V];
       V_::unpack(rR[j], r);
-      V_::unpack(rZ[j], zp);
+      if (cls[j] == 0) {
 #pragma unroll
-      for (int e = 0; e < V; ++e) {
-        const float z = (cls[j] == 0 || (cls[j] == 2 && col[j] + e < a.S)) ? zs[j][e] : a.alpha * zp[e];
-        hn[j][e] = act[j] ? z + r[e] : 0.f;
+        for (int e = 0; e < V; ++e) hn[j][e] = zs[j][e] + r[e];
+      } else if (cls[j] == 1) {
+        V_::unpack(rZ[j], zp);
+#pragma unroll
+        for (int e = 0; e < V; ++e) hn[j][e] = fmaf(a.alpha, zp[e], r[e]);
+      } else {
+        V_::unpack(rZ[j], zp);
+#pragma unroll
+        for (int e = 0; e < V; ++e) hn[j][e] = (col[j] + e < a.S ? zs[j][e] : a.alpha * zp[e]) + r[e];
       }
-      if (act[j]) st_vec<raw>(a.Hn, row * a.h + col[j], ES, V_::pack(hn[j]));
+      if (act[j]) stg<raw>(pHn[j], V_::pack(hn[j]));
+      pHn[j] += rank_h;
 #pragma unroll
-      for (int e = 0; e < V; ++e) st[0] += ln ? hn[j][e] : hn[j][e] * hn[j][e];
+      for (int e = 0; e < V; ++e) st[0] = LN ? st[0] + hn[j][e] : fmaf(hn[j][e], hn[j][e], st[0]);
     }
     row_reduce<1>(st, red, par);
     float mu = 0.f, rs;
-    if (ln) {
-      mu = st[0] / (float)a.h;
+    if (LN) {
+      mu = st[0] * inv_h;
       float sq[1] = {0.f};
 #pragma unroll
       for (int j = 0; j < CPT; ++j)
 #pragma unroll
         for (int e = 0; e < V; ++e) {
           const float d = act[j] ? hn[j][e] - mu : 0.f;
-          sq[0] += d * d;
+          sq[0] = fmaf(d, d, sq[0]);
         }
       row_reduce<1>(sq, red, par);
-      rs = 1.0f / sqrtf(sq[0] / (float)a.h + a.eps);
+      rs = rsqrtf(fmaf(sq[0], inv_h, a.eps));
     } else {
-      rs = 1.0f / sqrtf(st[0] / (float)a.h + a.eps);
+      rs = rsqrtf(fmaf(st[0], inv_h, a.eps));
     }
 #pragma unroll
     for (int j = 0; j < CPT; ++j) {
-      if (!act[j]) continue;
       float x[V];
 #pragma unroll
-      for (int e = 0; e < V; ++e) x[e] = (hn[j][e] - mu) * rs * gam[j][e] + bet[j][e];
-      st_vec<raw>(a.X, row * a.h + col[j], ES, V_::pack(x));
+      for (int e = 0; e < V; ++e) {
+        if (LN) x[e] = fmaf(hn[j][e] - mu, rs * gam[j][e], bet[j][e]);
+        else x[e] = hn[j][e] * (rs * gam[j][e]);
+      }
+      if (act[j]) stg<raw>(pX[j], V_::pack(x));
+      pX[j] += rank_h;
     }
     if (valid && threadIdx.x == 0) {
-      a.rstd[row] = rs;
-      if (ln && a.mean) a.mean[row] = mu;
+      *rstd_p = rs;
+      if (LN && mean_p) *mean_p = mu;
     }
+    rstd_p += a.T;
+    if (LN && mean_p) mean_p += a.T;
 #pragma unroll
     for (int j = 0; j < CPT; ++j) { rR[j] = nR[j]; rZ[j] = nZ[j]; }
   }
 }
 
 // ------------------------------------------------------------------ backward
-template <typename T_, int CPT>
-__global__ void __launch_bounds__(512) rows_backward_kernel(RowBwdArgs a, int ngroups) {
+template <typename T_, int CPT, bool LN>
+__global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(const RowBwdArgs a, int ngroups) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
   constexpr int V = V_::N;
@@ -213,46 +158,51 @@ __global__ void __launch_bounds__(512) rows_backward_kernel(RowBwdArgs a, int ng
   extern __shared__ float red[];
   int par = 0;
   const int TX = blockDim.x;
-  const bool ln = a.norm == 1;
   const float inv_h = 1.0f / (float)a.h;
+  const long long rank_h = (long long)a.T * a.h * ES;
+  const long long rank_p = (long long)a.T * a.P * ES;
+  const bool has_dh = a.dHn != nullptr;
 
   int col[CPT], cls[CPT];
   bool colok[CPT];
-  float gam[CPT][V], dgacc[CPT][V], dbacc[CPT][V];
+  float gam[CPT][V], dgacc[CPT][V], dbacc[LN ? CPT : 1][V];
 #pragma unroll
   for (int j = 0; j < CPT; ++j) {
     col[j] = (threadIdx.x + j * TX) * V;
     colok[j] = col[j] < a.h;
     cls[j] = chunk_class(col[j], V, a.S);
 #pragma unroll
-    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; dgacc[j][e] = 0.f; dbacc[j][e] = 0.f; }
-    if (colok[j]) V_::unpack(ld_vec<raw>(a.gamma, col[j], ES), gam[j]);
+    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; dgacc[j][e] = 0.f; if constexpr (LN) dbacc[j][e] = 0.f; }
+    if (colok[j]) V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
   }
 
   for (int grp = blockIdx.x; grp < ngroups; grp += gridDim.x) {
     const long long i = (long long)grp * blockDim.y + threadIdx.y;
     const bool valid = i < a.T;
     bool act[CPT];
-#pragma unroll
-    for (int j = 0; j < CPT; ++j) act[j] = valid && colok[j];
-
+    const char* pdX[CPT];
+    const char* pHn[CPT];
+    const char* pdH[CPT];
+    char* pdR[CPT];
+    char* pZ[CPT];
     raw rdX[CPT], rHn[CPT], rdH[CPT];
-    float rs_c, mu_c;
-    auto issue = [&](int m, raw(&dX_)[CPT], raw(&Hn_)[CPT], raw(&dH_)[CPT], float& rs, float& mu) {
-      const long long row = (long long)m * a.T + i;
-      rs = valid ? a.rstd[row] : 0.f;
-      mu = (valid && ln) ? a.mean[row] : 0.f;
 #pragma unroll
-      for (int j = 0; j < CPT; ++j) {
-        dX_[j] = zero_raw<raw>(); Hn_[j] = zero_raw<raw>(); dH_[j] = zero_raw<raw>();
-        if (act[j]) {
-          dX_[j] = ld_vec<raw>(a.dX, row * a.h + col[j], ES);
-          Hn_[j] = ld_vec<raw>(a.Hn, row * a.h + col[j], ES);
-          if (a.dHn) dH_[j] = ld_vec<raw>(a.dHn, row * a.h + col[j], ES);
-        }
-      }
-    };
-    issue(0, rdX, rHn, rdH, rs_c, mu_c);
+    for (int j = 0; j < CPT; ++j) {
+      act[j] = valid && colok[j];
+      const long long off_h = (i * a.h + col[j]) * ES;
+      pdX[j] = static_cast<const char*>(a.dX) + off_h;
+      pHn[j] = static_cast<const char*>(a.Hn) + off_h;
+      pdH[j] = static_cast<const char*>(a.dHn) + off_h;
+      pdR[j] = static_cast<char*>(a.dR) + off_h;
+      pZ[j] = static_cast<char*>(a.zp) + (i * a.P + (col[j] - a.S_lo)) * ES;
+      rdX[j] = act[j] ? ldg<raw>(pdX[j]) : zero_raw<raw>();
+      rHn[j] = act[j] ? ldg<raw>(pHn[j]) : zero_raw<raw>();
+      rdH[j] = (act[j] && has_dh) ? ldg<raw>(pdH[j]) : zero_raw<raw>();
+    }
+    const float* rstd_p = a.rstd + i;
+    const float* mean_p = LN ? a.mean + i : nullptr;
+    float rs_c = valid ? *rstd_p : 0.f;
+    float mu_c = (LN && valid) ? *mean_p : 0.f;
 
     float gsum[CPT][V];
 #pragma unroll
@@ -262,12 +212,24 @@ __global__ void __launch_bounds__(512) rows_backward_kernel(RowBwdArgs a, int ng
 
     for (int m = 0; m < a.t; ++m) {
       raw ndX[CPT], nHn[CPT], ndH[CPT];
-      float rs_n = 0.f, mu_n = 0.f;
-      if (m + 1 < a.t) issue(m + 1, ndX, nHn, ndH, rs_n, mu_n);
-      const long long row = (long long)m * a.T + i;
+      const bool more_rank = m + 1 < a.t;
+      rstd_p += a.T;
+      if (LN) mean_p += a.T;
+      const float rs_n = (valid && more_rank) ? *rstd_p : 0.f;
+      const float mu_n = (LN && valid && more_rank) ? *mean_p : 0.f;
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        pdX[j] += rank_h; pHn[j] += rank_h; pdH[j] += rank_h;
+        const bool more = act[j] && more_rank;
+        ndX[j] = more ? ldg<raw>(pdX[j]) : zero_raw<raw>();
+        nHn[j] = more ? ldg<raw>(pHn[j]) : zero_raw<raw>();
+        ndH[j] = (more && has_dh) ? ldg<raw>(pdH[j]) : zero_raw<raw>();
+      }
 
       float xh[CPT][V], dxh[CPT][V];
-      float s[2] = {0.f, 0.f};
+      float s[LN ? 2 : 1];
+#pragma unroll
+      for (int q = 0; q < (LN ? 2 : 1); ++q) s[q] = 0.f;
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
         float dx[V], hn[V];
@@ -275,31 +237,48 @@ __global__ void __launch_bounds__(512) rows_backward_kernel(RowBwdArgs a, int ng
         V_::unpack(rHn[j], hn);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
-          xh[j][e] = act[j] ? (hn[e] - mu_c) * rs_c : 0.f;
+          xh[j][e] = LN ? (act[j] ? (hn[e] - mu_c) * rs_c : 0.f) : hn[e] * rs_c;
           dxh[j][e] = dx[e] * gam[j][e];
-          s[0] += dxh[j][e];
-          s[1] += dxh[j][e] * xh[j][e];
-          dgacc[j][e] += dx[e] * xh[j][e];
-          dbacc[j][e] += dx[e];
+          if (LN) { s[0] += dxh[j][e]; s[1] = fmaf(dxh[j][e], xh[j][e], s[1]); }
+          else s[0] = fmaf(dxh[j][e], xh[j][e], s[0]);
+          dgacc[j][e] = fmaf(dx[e], xh[j][e], dgacc[j][e]);
+          if constexpr (LN) dbacc[j][e] += dx[e];
         }
       }
-      row_reduce<2>(s, red, par);
-      const float c1 = ln ? s[0] * inv_h : 0.f;
-      const float c2 = s[1] * inv_h;
+      row_reduce<LN ? 2 : 1>(s, red, par);
+      const float c1 = LN ? s[0] * inv_h : 0.f;
+      const float c2 = (LN ? s[1] : s[0]) * inv_h;
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
-        if (!act[j]) continue;
-        float dh[V], g[V], zp[V];
+        float dh[V], g[V];
         V_::unpack(rdH[j], dh);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
-          g[e] = rs_c * (dxh[j][e] - c1 - xh[j][e] * c2) + dh[e];
-          const bool shared = cls[j] == 0 || (cls[j] == 2 && col[j] + e < a.S);
-          gsum[j][e] += shared ? g[e] : 0.f;       // fp32 rank sum, m ascending
-          zp[e] = shared ? 0.f : a.alpha * g[e];   // private gradient carries alpha
+          float tt = fmaf(-xh[j][e], c2, dxh[j][e]);
+          if (LN) tt -= c1;
+          g[e] = fmaf(rs_c, tt, dh[e]);
         }
-        st_vec<raw>(a.dR, row * a.h + col[j], ES, V_::pack(g));
-        if (cls[j] != 0) st_vec<raw>(a.zp, row * a.P + (col[j] - a.S_lo), ES, V_::pack(zp));
+        if (act[j]) stg<raw>(pdR[j], V_::pack(g));
+        pdR[j] += rank_h;
+        if (cls[j] == 0) {
+#pragma unroll
+          for (int e = 0; e < V; ++e) gsum[j][e] += g[e];          // fp32 rank sum, m ascending
+        } else {
+          float zp[V];
+          if (cls[j] == 1) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) zp[e] = a.alpha * g[e];    // private gradient carries alpha
+          } else {
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              const bool shared = col[j] + e < a.S;
+              gsum[j][e] += shared ? g[e] : 0.f;
+              zp[e] = shared ? 0.f : a.alpha * g[e];
+            }
+          }
+          if (act[j]) stg<raw>(pZ[j], V_::pack(zp));
+        }
+        pZ[j] += rank_p;
       }
 #pragma unroll
       for (int j = 0; j < CPT; ++j) { rdX[j] = ndX[j]; rHn[j] = nHn[j]; rdH[j] = ndH[j]; }
@@ -307,22 +286,36 @@ __global__ void __launch_bounds__(512) rows_backward_kernel(RowBwdArgs a, int ng
     }
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
-      if (act[j] && cls[j] != 1) st_vec<raw>(a.gs, i * a.S_hi + col[j], ES, V_::pack(gsum[j]));
+      if (act[j] && cls[j] != 1)
+        stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, V_::pack(gsum[j]));
   }
 
-  // Partial norm-parameter gradients of this CTA: sum the TY token rows in order, then
-  // one row of [h] per CTA.
-  __syncthreads();
-  float* acc = red;  // reuse: [TY][TX*CPT*V]
-  const int per_row = TX * CPT * V;
-  for (int which = 0; which < (ln ? 2 : 1); ++which) {
+  // Partial norm-parameter gradients of this CTA: one row of [h] per CTA.  With several
+  // token rows per CTA (TY > 1) they are first summed through shared memory, in order.
+  for (int which = 0; which < (LN ? 2 : 1); ++which) {
     float* out = which == 0 ? a.dgpart : a.dbpart;
     if (out == nullptr) continue;
+    if (blockDim.y == 1) {
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        if (!colok[j]) continue;
+        const float* src = (which == 0 || !LN) ? dgacc[j] : dbacc[LN ? j : 0];
+#pragma unroll
+        for (int e = 0; e < V; e += 4)
+          *reinterpret_cast<float4*>(out + (size_t)blockIdx.x * a.h + col[j] + e) =
+              make_float4(src[e], src[e + 1], src[e + 2], src[e + 3]);
+      }
+      continue;
+    }
+    __syncthreads();
+    float* acc = red;  // reuse: [TY][TX*CPT*V]
+    const int per_row = TX * CPT * V;
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
 #pragma unroll
       for (int e = 0; e < V; ++e)
-        acc[(size_t)threadIdx.y * per_row + (j * TX + threadIdx.x) * V + e] = which == 0 ? dgacc[j][e] : dbacc[j][e];
+        acc[(size_t)threadIdx.y * per_row + (j * TX + threadIdx.x) * V + e] =
+            (which == 0 || !LN) ? dgacc[j][e] : dbacc[LN ? j : 0][e];
     __syncthreads();
     if (threadIdx.y == 0) {
 #pragma unroll
@@ -340,7 +333,6 @@ __global__ void __launch_bounds__(512) rows_backward_kernel(RowBwdArgs a, int ng
               make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
       }
     }
-    __syncthreads();
   }
 }
 
@@ -361,28 +353,33 @@ __global__ void __launch_bounds__(1024) reduce_partials_kernel(const float* __re
   }
 }
 
-struct RowGeom {
-  int TX, TY, CPT;
-  size_t smem_fwd, smem_bwd;
-};
-
-RowGeom row_geometry(int h, caat_dtype dtype) {
-  const int V = dtype == CAAT_BF16 ? 8 : 4;
-  const int chunks = h / V;
-  RowGeom g;
-  int tx = round_up(chunks, 32);
-  g.CPT = 1;
-  while (tx > 512) {
-    g.CPT *= 2;
-    tx = round_up((chunks + g.CPT - 1) / g.CPT, 32);
+template <typename T_, bool LN>
+cudaError_t launch_fwd_t(const RowFwdArgs& a, const RowGeom& g, cudaStream_t st) {
+  const dim3 block(g.TX, g.TY);
+  const dim3 grid((a.T + g.TY - 1) / g.TY);
+  LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
+  switch (g.CPT) {
+    case 1: rows_forward_kernel<T_, 1, LN><<<grid, block, g.smem_fwd, st>>>(a); break;
+    case 2: rows_forward_kernel<T_, 2, LN><<<grid, block, g.smem_fwd, st>>>(a); break;
+    case 4: rows_forward_kernel<T_, 4, LN><<<grid, block, g.smem_fwd, st>>>(a); break;
+    default: return cudaErrorInvalidValue;
   }
-  g.TX = tx;
-  g.TY = tx >= 256 ? 1 : 256 / tx;
-  const size_t red = (size_t)2 * g.TY * (g.TX / 32) * 2 * sizeof(float);
-  g.smem_fwd = red;
-  const size_t acc = (size_t)g.TY * g.TX * g.CPT * V * sizeof(float);
-  g.smem_bwd = red > acc ? red : acc;
-  return g;
+  return cudaGetLastError();
+}
+
+template <typename T_, bool LN>
+cudaError_t launch_bwd_t(const RowBwdArgs& a, const RowGeom& g, int rows, cudaStream_t st) {
+  const dim3 block(g.TX, g.TY);
+  const int ngroups = (a.T + g.TY - 1) / g.TY;
+  const dim3 grid(rows);
+  LaunchScope scope(CAAT_K_ROWS_BACKWARD, st);
+  switch (g.CPT) {
+    case 1: rows_backward_kernel<T_, 1, LN><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
+    case 2: rows_backward_kernel<T_, 2, LN><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
+    case 4: rows_backward_kernel<T_, 4, LN><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
+    default: return cudaErrorInvalidValue;
+  }
+  return cudaGetLastError();
 }
 
 }  // namespace
@@ -393,53 +390,24 @@ int rows_backward_partial_rows(int h, int T, caat_dtype dtype) {
   return ngroups < kMaxPartialRows ? ngroups : kMaxPartialRows;
 }
 
-template <typename T_>
-static cudaError_t launch_fwd_t(const RowFwdArgs& a, const RowGeom& g, cudaStream_t st) {
-  const dim3 block(g.TX, g.TY);
-  const dim3 grid((a.T + g.TY - 1) / g.TY);
-  LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
-  switch (g.CPT) {
-    case 1: rows_forward_kernel<T_, 1><<<grid, block, g.smem_fwd, st>>>(a); break;
-    case 2: rows_forward_kernel<T_, 2><<<grid, block, g.smem_fwd, st>>>(a); break;
-    case 4: rows_forward_kernel<T_, 4><<<grid, block, g.smem_fwd, st>>>(a); break;
-    default: return cudaErrorInvalidValue;
-  }
-  return cudaGetLastError();
-}
-
-cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st) {
+cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st) {
+  if (!direct && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, false)) return launch_rows_forward_staged(a, dtype, st);
   const RowGeom g = row_geometry(a.h, dtype);
-  return dtype == CAAT_BF16 ? launch_fwd_t<__nv_bfloat16>(a, g, st) : launch_fwd_t<float>(a, g, st);
+  if (dtype == CAAT_BF16)
+    return a.norm == 1 ? launch_fwd_t<__nv_bfloat16, true>(a, g, st) : launch_fwd_t<__nv_bfloat16, false>(a, g, st);
+  return a.norm == 1 ? launch_fwd_t<float, true>(a, g, st) : launch_fwd_t<float, false>(a, g, st);
 }
 
-template <typename T_>
-static cudaError_t launch_bwd_t(const RowBwdArgs& a, const RowGeom& g, int rows, cudaStream_t st) {
-  const dim3 block(g.TX, g.TY);
-  const int ngroups = (a.T + g.TY - 1) / g.TY;
-  const dim3 grid(rows);
-  if (g.smem_bwd > 48 * 1024) {
-    cudaError_t e = cudaSuccess;
-    switch (g.CPT) {
-      case 1: e = cudaFuncSetAttribute(rows_backward_kernel<T_, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bwd); break;
-      case 2: e = cudaFuncSetAttribute(rows_backward_kernel<T_, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bwd); break;
-      case 4: e = cudaFuncSetAttribute(rows_backward_kernel<T_, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bwd); break;
-    }
-    if (e != cudaSuccess) return e;
-  }
-  LaunchScope scope(CAAT_K_ROWS_BACKWARD, st);
-  switch (g.CPT) {
-    case 1: rows_backward_kernel<T_, 1><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
-    case 2: rows_backward_kernel<T_, 2><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
-    case 4: rows_backward_kernel<T_, 4><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
-    default: return cudaErrorInvalidValue;
-  }
-  return cudaGetLastError();
-}
-
-cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, cudaStream_t st) {
+cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st) {
   const RowGeom g = row_geometry(a.h, dtype);
-  const int rows = rows_backward_partial_rows(a.h, a.T, dtype);
-  cudaError_t e = dtype == CAAT_BF16 ? launch_bwd_t<__nv_bfloat16>(a, g, rows, st) : launch_bwd_t<float>(a, g, rows, st);
+  int rows = rows_backward_partial_rows(a.h, a.T, dtype);
+  cudaError_t e;
+  if (!direct && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, true))
+    e = launch_rows_backward_staged(a, dtype, rows, &rows, st);
+  else if (dtype == CAAT_BF16)
+    e = a.norm == 1 ? launch_bwd_t<__nv_bfloat16, true>(a, g, rows, st) : launch_bwd_t<__nv_bfloat16, false>(a, g, rows, st);
+  else
+    e = a.norm == 1 ? launch_bwd_t<float, true>(a, g, rows, st) : launch_bwd_t<float, false>(a, g, rows, st);
   if (e != cudaSuccess) return e;
   const dim3 rb(32, 32);
   const dim3 rg((a.h + 31) / 32);

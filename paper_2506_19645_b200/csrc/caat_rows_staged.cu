@@ -1,0 +1,679 @@
+// Row kernels, bulk-copy staged variant (the default).
+//
+// The row work is pure streaming: what limits it is how many bytes a CTA keeps in flight.
+// With plain loads that is bounded by registers (threads x loads per thread); here the
+// inputs of one (token group, rank) - a few contiguous rows - are fetched by ONE thread
+// with cp.async.bulk into a shared-memory ring, several ranks (and token groups) ahead,
+// completion signalled on an mbarrier per stage.  Consumer threads keep the mapping of
+// the direct kernels (a thread owns the same 16-byte column chunk of every rank of its
+// token; rank sums are thread-local and run m = 0..t-1), read their chunk from shared
+// memory and write results with 128-bit stores.  The CTA-wide barrier of the row
+// reduction doubles as the "stage is free" signal, so there are no empty-barriers.
+//
+// CTAs are persistent (token groups strided by the grid).  Every mbarrier wait is bounded:
+// on a timeout the CTA sets the library's status word, drains its copies in flight and
+// returns.
+#include "caat_rows_common.cuh"
+
+namespace caat {
+namespace {
+
+using namespace rows;
+
+constexpr uint32_t kSpinCap = 1u << 22;
+constexpr int kMaxStages = 8;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpinCap; ++it)
+    if (mbar_try(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+template <typename raw>
+__device__ __forceinline__ raw lds(const uint8_t* p) { return *reinterpret_cast<const raw*>(p); }
+
+struct StageGeom {
+  int nstages;
+  uint32_t off_a, off_b, off_c;  // byte offsets of the three row buffers inside a stage
+  uint32_t stage_bytes;
+  uint32_t ring_off, bar_off, red_off, stat_off, acc_off;
+  size_t smem;
+};
+
+// ------------------------------------------------------------------ forward
+// stage buffers: a = R rows [TY, h], b = zp rows [TY, P], c = zs rows [TY, S_hi] (rank 0 only)
+template <typename T_, int CPT, bool LN>
+__global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1)
+rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
+  using V_ = VT<T_>;
+  using raw = typename V_::raw;
+  constexpr int V = V_::N;
+  constexpr int ES = sizeof(T_);
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* ring = smem + sg.ring_off;
+  const uint32_t bar0 = smem_u32(smem + sg.bar_off);
+  float* red = reinterpret_cast<float*>(smem + sg.red_off);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + sg.bar_off + 8 * kMaxStages);
+  int par = 0;
+  const int TX = blockDim.x, TY = blockDim.y;
+  const bool leader = threadIdx.x == 0 && threadIdx.y == 0;
+  const float inv_h = 1.0f / (float)a.h;
+  const int NS = sg.nstages;
+  const bool has_priv = a.P > 0 && a.S < a.h;
+  const bool has_shared = a.S > 0;
+
+  // sequence k = n * t + m over this CTA's (token group n, rank m) pairs
+  const int my_groups = blockIdx.x < ngroups ? (ngroups - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const long long total = (long long)my_groups * a.t;
+
+  // leader only: fetch the inputs of (its token group nn, rank mm) into stage ss
+  int nn = 0, mm = 0, ss = 0;
+  auto issue = [&]() {
+    if (nn >= my_groups) return;
+    const int n = nn, m = mm, s = ss;
+    if (++mm == a.t) { mm = 0; ++nn; }
+    if (++ss == NS) ss = 0;
+    const long long g = blockIdx.x + (long long)n * gridDim.x;
+    const long long i0 = g * TY;
+    const int rowsN = (int)((a.T - i0) < TY ? (a.T - i0) : TY);
+    const uint32_t bar = bar0 + 8u * s;
+    const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
+    const uint32_t bR = (uint32_t)rowsN * a.h * ES;
+    const uint32_t bP = has_priv ? (uint32_t)rowsN * a.P * ES : 0u;
+    const uint32_t bS = (m == 0 && has_shared) ? (uint32_t)rowsN * a.S_hi * ES : 0u;
+    mbar_expect_tx(bar, bR + bP + bS);
+    const long long row = (long long)m * a.T + i0;
+    bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * a.h * ES, bR, bar);
+    if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
+    if (bS) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.zs) + i0 * a.S_hi * ES, bS, bar);
+  };
+
+  if (leader) {
+    for (int s = 0; s < NS; ++s) mbar_init(bar0 + 8u * s, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  long long issued = 0;
+  if (leader) {
+    for (; issued < NS && issued < total; ++issued) issue();
+  }
+
+  int col[CPT], cls[CPT];
+  bool colok[CPT];
+  float gam[CPT][V], bet[CPT][V];
+#pragma unroll
+  for (int j = 0; j < CPT; ++j) {
+    col[j] = (threadIdx.x + j * TX) * V;
+    colok[j] = col[j] < a.h;
+    cls[j] = chunk_class(col[j], V, a.S);
+#pragma unroll
+    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; bet[j][e] = 0.f; }
+    if (colok[j]) {
+      V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+      if (LN && a.beta) V_::unpack(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
+    }
+  }
+
+  long long k = 0;
+  int cs = 0;            // consumer's stage and its phase parity
+  uint32_t cph = 0;
+  bool dead = false;
+  for (int n = 0; n < my_groups && !dead; ++n) {
+    const long long g = blockIdx.x + (long long)n * gridDim.x;
+    const long long i = g * TY + threadIdx.y;
+    const bool valid = i < a.T;
+    bool act[CPT];
+    float zs[CPT][V];
+    char* pHn[CPT];
+    char* pX[CPT];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) {
+      act[j] = valid && colok[j];
+      const long long off_h = (i * a.h + col[j]) * ES;
+      pHn[j] = static_cast<char*>(a.Hn) + off_h;
+      pX[j] = static_cast<char*>(a.X) + off_h;
+#pragma unroll
+      for (int e = 0; e < V; ++e) zs[j][e] = 0.f;
+    }
+    float* rstd_p = a.rstd + i;
+    float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
+    const long long rank_h = (long long)a.T * a.h * ES;
+
+    for (int m = 0; m < a.t; ++m, ++k) {
+      const uint8_t* stage = ring + (size_t)cs * sg.stage_bytes;
+      if (!mbar_wait(bar0 + 8u * cs, cph)) *abort_flag = 1;
+      if (++cs == NS) { cs = 0; cph ^= 1u; }
+
+      float hn[CPT][V];
+      float st[1] = {0.f};
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        float r[V], zp[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) { r[e] = 0.f; zp[e] = 0.f; }
+        if (act[j]) {
+          V_::unpack(lds<raw>(stage + sg.off_a + ((size_t)threadIdx.y * a.h + col[j]) * ES), r);
+          if (cls[j] != 0) V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)threadIdx.y * a.P + (col[j] - a.S_lo)) * ES), zp);
+          if (m == 0 && cls[j] != 1) V_::unpack(lds<raw>(stage + sg.off_c + ((size_t)threadIdx.y * a.S_hi + col[j]) * ES), zs[j]);
+        }
+        if (cls[j] == 0) {
+#pragma unroll
+          for (int e = 0; e < V; ++e) hn[j][e] = zs[j][e] + r[e];
+        } else if (cls[j] == 1) {
+#pragma unroll
+          for (int e = 0; e < V; ++e) hn[j][e] = fmaf(a.alpha, zp[e], r[e]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < V; ++e) hn[j][e] = (col[j] + e < a.S ? zs[j][e] : a.alpha * zp[e]) + r[e];
+        }
+        if (act[j]) stg<raw>(pHn[j], V_::pack(hn[j]));
+        pHn[j] += rank_h;
+#pragma unroll
+        for (int e = 0; e < V; ++e) st[0] = LN ? st[0] + hn[j][e] : fmaf(hn[j][e], hn[j][e], st[0]);
+      }
+      row_reduce_sync<1>(st, red, par);      // CTA barrier: every thread is done reading this stage
+      if (*abort_flag) { dead = true; break; }
+      if (leader && issued < total) { issue(); ++issued; }
+      float mu = 0.f, rs;
+      if (LN) {
+        mu = st[0] * inv_h;
+        float sq[1] = {0.f};
+#pragma unroll
+        for (int j = 0; j < CPT; ++j)
+#pragma unroll
+          for (int e = 0; e < V; ++e) {
+            const float d = act[j] ? hn[j][e] - mu : 0.f;
+            sq[0] = fmaf(d, d, sq[0]);
+          }
+        row_reduce_sync<1>(sq, red, par);
+        rs = rsqrtf(fmaf(sq[0], inv_h, a.eps));
+      } else {
+        rs = rsqrtf(fmaf(st[0], inv_h, a.eps));
+      }
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        float x[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          if (LN) x[e] = fmaf(hn[j][e] - mu, rs * gam[j][e], bet[j][e]);
+          else x[e] = hn[j][e] * (rs * gam[j][e]);
+        }
+        if (act[j]) stg<raw>(pX[j], V_::pack(x));
+        pX[j] += rank_h;
+      }
+      if (valid && threadIdx.x == 0) {
+        *rstd_p = rs;
+        if (LN && mean_p) *mean_p = mu;
+      }
+      rstd_p += a.T;
+      if (LN && mean_p) mean_p += a.T;
+    }
+  }
+  if (dead && leader) {
+    atomicExch(status, 4u);
+    // wait (bounded) for this CTA's copies still in flight before its shared memory goes away
+    for (long long q = k + 1; q < issued; ++q)
+      for (uint32_t it = 0; it < (1u << 20); ++it)
+        if (mbar_try(bar0 + 8u * (uint32_t)(q % NS), (uint32_t)((q / NS) & 1))) break;
+  }
+}
+
+// ------------------------------------------------------------------ backward
+// stage buffers: a = dX rows, b = Hn rows, c = dHn rows (when given)
+template <typename T_, int CPT, bool LN>
+__global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1)
+rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
+  using V_ = VT<T_>;
+  using raw = typename V_::raw;
+  constexpr int V = V_::N;
+  constexpr int ES = sizeof(T_);
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* ring = smem + sg.ring_off;
+  const uint32_t bar0 = smem_u32(smem + sg.bar_off);
+  float* red = reinterpret_cast<float*>(smem + sg.red_off);
+  float* stat = reinterpret_cast<float*>(smem + sg.stat_off);   // [2 buffers][2 (rstd, mean)][t * TY]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + sg.bar_off + 8 * kMaxStages);
+  int par = 0;
+  const int TX = blockDim.x, TY = blockDim.y;
+  const int tid = threadIdx.y * TX + threadIdx.x, nthr = TX * TY;
+  const bool leader = tid == 0;
+  const float inv_h = 1.0f / (float)a.h;
+  const int NS = sg.nstages;
+  const bool has_dh = a.dHn != nullptr;
+  const int nstat = a.t * TY;
+
+  const int my_groups = blockIdx.x < ngroups ? (ngroups - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  const long long total = (long long)my_groups * a.t;
+
+  int nn = 0, mm = 0, ss = 0;
+  auto issue = [&]() {   // leader only: fetch (its token group nn, rank mm) into stage ss
+    if (nn >= my_groups) return;
+    const int n = nn, m = mm, s = ss;
+    if (++mm == a.t) { mm = 0; ++nn; }
+    if (++ss == NS) ss = 0;
+    const long long g = blockIdx.x + (long long)n * gridDim.x;
+    const long long i0 = g * TY;
+    const int rowsN = (int)((a.T - i0) < TY ? (a.T - i0) : TY);
+    const uint32_t bar = bar0 + 8u * s;
+    const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
+    const uint32_t b = (uint32_t)rowsN * a.h * ES;
+    mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
+    const long long off = ((long long)m * a.T + i0) * a.h * ES;
+    bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
+    bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
+    if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
+  };
+  // row statistics of token group n: element (m, ty) of rstd / mean
+  auto load_stats = [&](int n, float* dst) {
+    const long long g = blockIdx.x + (long long)n * gridDim.x;
+    for (int q = tid; q < nstat; q += nthr) {
+      const int m = q / TY, ty = q % TY;
+      const long long i = g * TY + ty;
+      const bool ok = n < my_groups && i < a.T;
+      dst[q] = ok ? a.rstd[(long long)m * a.T + i] : 0.f;
+      if (LN) dst[nstat + q] = ok ? a.mean[(long long)m * a.T + i] : 0.f;
+    }
+  };
+
+  if (leader) {
+    for (int s = 0; s < NS; ++s) mbar_init(bar0 + 8u * s, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  long long issued = 0;
+  if (leader) {
+    for (; issued < NS && issued < total; ++issued) issue();
+  }
+  load_stats(0, stat);
+
+  int col[CPT], cls[CPT];
+  bool colok[CPT];
+  float gam[CPT][V], dgacc[CPT][V], dbacc[LN ? CPT : 1][V];
+#pragma unroll
+  for (int j = 0; j < CPT; ++j) {
+    col[j] = (threadIdx.x + j * TX) * V;
+    colok[j] = col[j] < a.h;
+    cls[j] = chunk_class(col[j], V, a.S);
+#pragma unroll
+    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; dgacc[j][e] = 0.f; if constexpr (LN) dbacc[j][e] = 0.f; }
+    if (colok[j]) V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+  }
+  __syncthreads();   // stats of group 0 visible
+
+  long long k = 0;
+  int cs = 0;            // consumer's stage and its phase parity
+  uint32_t cph = 0;
+  bool dead = false;
+  for (int n = 0; n < my_groups && !dead; ++n) {
+    const long long g = blockIdx.x + (long long)n * gridDim.x;
+    const long long i = g * TY + threadIdx.y;
+    const bool valid = i < a.T;
+    const float* st_cur = stat + (size_t)(n & 1) * 2 * nstat;
+    float* st_nxt = stat + (size_t)((n + 1) & 1) * 2 * nstat;
+    // prefetch the next group's row statistics into registers; they are parked in shared
+    // memory at the end of this group (a whole group of work hides the latency)
+    float pre_r[2] = {0.f, 0.f}, pre_m[2] = {0.f, 0.f};
+    {
+      const long long g2 = blockIdx.x + (long long)(n + 1) * gridDim.x;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int q = tid + u * nthr;
+        if (q < nstat && n + 1 < my_groups) {
+          const int m2 = q / TY, ty2 = q % TY;
+          const long long i2 = g2 * TY + ty2;
+          if (i2 < a.T) {
+            pre_r[u] = a.rstd[(long long)m2 * a.T + i2];
+            if (LN) pre_m[u] = a.mean[(long long)m2 * a.T + i2];
+          }
+        }
+      }
+    }
+    bool act[CPT];
+    char* pdR[CPT];
+    char* pZ[CPT];
+    float gsum[CPT][V];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) {
+      act[j] = valid && colok[j];
+      pdR[j] = static_cast<char*>(a.dR) + (i * a.h + col[j]) * ES;
+      pZ[j] = static_cast<char*>(a.zp) + (i * a.P + (col[j] - a.S_lo)) * ES;
+#pragma unroll
+      for (int e = 0; e < V; ++e) gsum[j][e] = 0.f;
+    }
+    const long long rank_h = (long long)a.T * a.h * ES;
+    const long long rank_p = (long long)a.T * a.P * ES;
+
+    for (int m = 0; m < a.t; ++m, ++k) {
+      const uint8_t* stage = ring + (size_t)cs * sg.stage_bytes;
+      if (!mbar_wait(bar0 + 8u * cs, cph)) *abort_flag = 1;
+      if (++cs == NS) { cs = 0; cph ^= 1u; }
+      const float rs_c = st_cur[m * TY + threadIdx.y];
+      const float mu_c = LN ? st_cur[nstat + m * TY + threadIdx.y] : 0.f;
+
+      float xh[CPT][V], dxh[CPT][V], dh[CPT][V];
+      float sacc[LN ? 2 : 1];
+#pragma unroll
+      for (int q = 0; q < (LN ? 2 : 1); ++q) sacc[q] = 0.f;
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        float dx[V], hn[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) { dx[e] = 0.f; hn[e] = 0.f; dh[j][e] = 0.f; }
+        if (act[j]) {
+          const size_t o = ((size_t)threadIdx.y * a.h + col[j]) * ES;
+          V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
+          V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
+          if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + o), dh[j]);
+        }
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          xh[j][e] = LN ? (act[j] ? (hn[e] - mu_c) * rs_c : 0.f) : hn[e] * rs_c;
+          dxh[j][e] = dx[e] * gam[j][e];
+          if (LN) { sacc[0] += dxh[j][e]; sacc[1] = fmaf(dxh[j][e], xh[j][e], sacc[1]); }
+          else sacc[0] = fmaf(dxh[j][e], xh[j][e], sacc[0]);
+          dgacc[j][e] = fmaf(dx[e], xh[j][e], dgacc[j][e]);
+          if constexpr (LN) dbacc[j][e] += dx[e];
+        }
+      }
+      row_reduce_sync<LN ? 2 : 1>(sacc, red, par);   // CTA barrier: stage fully read
+      if (*abort_flag) { dead = true; break; }
+      if (leader && issued < total) { issue(); ++issued; }
+      const float c1 = LN ? sacc[0] * inv_h : 0.f;
+      const float c2 = (LN ? sacc[1] : sacc[0]) * inv_h;
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        float gg[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          float tt = fmaf(-xh[j][e], c2, dxh[j][e]);
+          if (LN) tt -= c1;
+          gg[e] = fmaf(rs_c, tt, dh[j][e]);
+        }
+        if (act[j]) stg<raw>(pdR[j], V_::pack(gg));
+        pdR[j] += rank_h;
+        if (cls[j] == 0) {
+#pragma unroll
+          for (int e = 0; e < V; ++e) gsum[j][e] += gg[e];          // fp32 rank sum, m ascending
+        } else {
+          float zp[V];
+          if (cls[j] == 1) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) zp[e] = a.alpha * gg[e];    // private gradient carries alpha
+          } else {
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              const bool shared = col[j] + e < a.S;
+              gsum[j][e] += shared ? gg[e] : 0.f;
+              zp[e] = shared ? 0.f : a.alpha * gg[e];
+            }
+          }
+          if (act[j]) stg<raw>(pZ[j], V_::pack(zp));
+        }
+        pZ[j] += rank_p;
+      }
+    }
+    if (dead) break;
+#pragma unroll
+    for (int j = 0; j < CPT; ++j)
+      if (act[j] && cls[j] != 1)
+        stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, V_::pack(gsum[j]));
+    // park the next group's statistics; the last barrier of this group separates these writes
+    // from the reads of group n-1's buffer, the barrier below from the reads of group n+1
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int q = tid + u * nthr;
+      if (q < nstat) { st_nxt[q] = pre_r[u]; if (LN) st_nxt[nstat + q] = pre_m[u]; }
+    }
+    for (int q = tid + 2 * nthr; q < nstat && n + 1 < my_groups; q += nthr) {   // t * TY > 2 * threads: rare
+      const int m2 = q / TY, ty2 = q % TY;
+      const long long i2 = (blockIdx.x + (long long)(n + 1) * gridDim.x) * TY + ty2;
+      st_nxt[q] = i2 < a.T ? a.rstd[(long long)m2 * a.T + i2] : 0.f;
+      if (LN) st_nxt[nstat + q] = i2 < a.T ? a.mean[(long long)m2 * a.T + i2] : 0.f;
+    }
+    __syncthreads();
+  }
+  if (dead) {
+    if (leader) {
+      atomicExch(status, 5u);
+      for (long long q = k + 1; q < issued; ++q)
+        for (uint32_t it = 0; it < (1u << 20); ++it)
+          if (mbar_try(bar0 + 8u * (uint32_t)(q % NS), (uint32_t)((q / NS) & 1))) break;
+    }
+    return;
+  }
+
+  // Partial norm-parameter gradients of this CTA: one row of [h] per CTA, token rows of the
+  // CTA summed in order through shared memory when TY > 1.
+  for (int which = 0; which < (LN ? 2 : 1); ++which) {
+    float* out = which == 0 ? a.dgpart : a.dbpart;
+    if (out == nullptr) continue;
+    if (TY == 1) {
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        if (!colok[j]) continue;
+        const float* src = (which == 0 || !LN) ? dgacc[j] : dbacc[LN ? j : 0];
+#pragma unroll
+        for (int e = 0; e < V; e += 4)
+          *reinterpret_cast<float4*>(out + (size_t)blockIdx.x * a.h + col[j] + e) =
+              make_float4(src[e], src[e + 1], src[e + 2], src[e + 3]);
+      }
+      continue;
+    }
+    __syncthreads();
+    float* acc = reinterpret_cast<float*>(smem + sg.acc_off);   // [TY][TX*CPT*V], overlays the ring
+    const int per_row = TX * CPT * V;
+#pragma unroll
+    for (int j = 0; j < CPT; ++j)
+#pragma unroll
+      for (int e = 0; e < V; ++e)
+        acc[(size_t)threadIdx.y * per_row + (j * TX + threadIdx.x) * V + e] =
+            (which == 0 || !LN) ? dgacc[j][e] : dbacc[LN ? j : 0][e];
+    __syncthreads();
+    if (threadIdx.y == 0) {
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        if (!colok[j]) continue;
+        float sum[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) sum[e] = 0.f;
+        for (int y = 0; y < TY; ++y)
+#pragma unroll
+          for (int e = 0; e < V; ++e) sum[e] += acc[(size_t)y * per_row + (j * TX + threadIdx.x) * V + e];
+#pragma unroll
+        for (int e = 0; e < V; e += 4)
+          *reinterpret_cast<float4*>(out + (size_t)blockIdx.x * a.h + col[j] + e) =
+              make_float4(sum[e], sum[e + 1], sum[e + 2], sum[e + 3]);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------ host side
+StageGeom stage_geometry(const RowGeom& g, int h, int P, int S_hi, int t, int ES, bool backward, bool has_c,
+                         size_t budget) {
+  StageGeom sg{};
+  const uint32_t rowA = (uint32_t)g.TY * h * ES;
+  if (backward) {
+    sg.off_a = 0; sg.off_b = rowA; sg.off_c = 2 * rowA;
+    sg.stage_bytes = (has_c ? 3 : 2) * rowA;
+  } else {
+    const uint32_t rowB = (uint32_t)g.TY * P * ES, rowC = (uint32_t)g.TY * S_hi * ES;
+    sg.off_a = 0; sg.off_b = rowA; sg.off_c = rowA + rowB;
+    sg.stage_bytes = rowA + rowB + rowC;
+  }
+  sg.stage_bytes = (sg.stage_bytes + 127u) & ~127u;
+  // fixed part: barriers + abort flag, reduction scratch, row statistics
+  size_t off = 0;
+  sg.bar_off = (uint32_t)off; off += 8 * kMaxStages + 16;
+  off = align_up(off, 16);
+  sg.red_off = (uint32_t)off; off += (size_t)2 * g.TY * 16 * 2 * sizeof(float);
+  sg.stat_off = (uint32_t)off; off += backward ? (size_t)2 * 2 * t * g.TY * sizeof(float) : 0;
+  off = align_up(off, 128);
+  sg.ring_off = (uint32_t)off;
+  sg.acc_off = sg.ring_off;
+  const size_t acc = (backward && g.TY > 1) ? (size_t)g.TY * g.TX * g.CPT * (16 / ES) * sizeof(float) : 0;
+  int ns = (int)((budget - off) / sg.stage_bytes);
+  if (ns > kMaxStages) ns = kMaxStages;
+  sg.nstages = ns;
+  size_t ring = (size_t)(ns > 0 ? ns : 0) * sg.stage_bytes;
+  if (ring < acc) ring = acc;
+  sg.smem = off + ring;
+  return sg;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <typename K>
+cudaError_t set_smem(K kernel, size_t bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+template <typename T_, bool LN>
+cudaError_t launch_fwd_staged_t(const RowFwdArgs& a, const RowGeom& g, const StageGeom& sg, int grid, int ngroups,
+                                unsigned int* status, cudaStream_t st) {
+  const dim3 block(g.TX, g.TY);
+  cudaError_t e = cudaSuccess;
+  LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
+  switch (g.CPT) {
+    case 1:
+      e = set_smem(rows_forward_staged<T_, 1, LN>, sg.smem);
+      if (e == cudaSuccess) rows_forward_staged<T_, 1, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
+      break;
+    case 2:
+      e = set_smem(rows_forward_staged<T_, 2, LN>, sg.smem);
+      if (e == cudaSuccess) rows_forward_staged<T_, 2, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
+      break;
+    case 4:
+      e = set_smem(rows_forward_staged<T_, 4, LN>, sg.smem);
+      if (e == cudaSuccess) rows_forward_staged<T_, 4, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
+      break;
+    default: return cudaErrorInvalidValue;
+  }
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+template <typename T_, bool LN>
+cudaError_t launch_bwd_staged_t(const RowBwdArgs& a, const RowGeom& g, const StageGeom& sg, int grid, int ngroups,
+                                unsigned int* status, cudaStream_t st) {
+  const dim3 block(g.TX, g.TY);
+  cudaError_t e = cudaSuccess;
+  LaunchScope scope(CAAT_K_ROWS_BACKWARD, st);
+  switch (g.CPT) {
+    case 1:
+      e = set_smem(rows_backward_staged<T_, 1, LN>, sg.smem);
+      if (e == cudaSuccess) rows_backward_staged<T_, 1, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
+      break;
+    case 2:
+      e = set_smem(rows_backward_staged<T_, 2, LN>, sg.smem);
+      if (e == cudaSuccess) rows_backward_staged<T_, 2, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
+      break;
+    case 4:
+      e = set_smem(rows_backward_staged<T_, 4, LN>, sg.smem);
+      if (e == cudaSuccess) rows_backward_staged<T_, 4, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
+      break;
+    default: return cudaErrorInvalidValue;
+  }
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+constexpr size_t kSmemPerSm = 227 * 1024;
+
+// resident CTAs per SM the register budget allows (64 registers per thread when CPT == 1)
+int ctas_per_sm(const RowGeom& g) {
+  if (g.CPT != 1) return 1;
+  int n = 1024 / (g.TX * g.TY);
+  return n < 1 ? 1 : (n > 8 ? 8 : n);
+}
+
+}  // namespace
+
+bool rows_staged_usable(int h, int t, int S_lo, int S_hi, caat_dtype dtype, bool backward) {
+  const RowGeom g = row_geometry(h, dtype);
+  const int ES = (int)elem_size(dtype);
+  const StageGeom sg = stage_geometry(g, h, h - S_lo, S_hi, t, ES, backward, true, kSmemPerSm - 1024);
+  return sg.nstages >= 2;
+}
+
+cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st) {
+  const RowGeom g = row_geometry(a.h, dtype);
+  const int ES = (int)elem_size(dtype);
+  int per_sm = ctas_per_sm(g);
+  StageGeom sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, kSmemPerSm / per_sm - 1024);
+  while (sg.nstages < 3 && per_sm > 1) {   // rows too long: fewer CTAs per SM, each with a larger ring
+    --per_sm;
+    sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, kSmemPerSm / per_sm - 1024);
+  }
+  if (sg.nstages < 2) return cudaErrorInvalidConfiguration;
+  const int ngroups = (a.T + g.TY - 1) / g.TY;
+  int grid = sm_count() * per_sm;
+  if (grid > ngroups) grid = ngroups;
+  unsigned int* status = device_status_word();
+  if (!status) return cudaErrorUnknown;
+  if (dtype == CAAT_BF16)
+    return a.norm == 1 ? launch_fwd_staged_t<__nv_bfloat16, true>(a, g, sg, grid, ngroups, status, st)
+                       : launch_fwd_staged_t<__nv_bfloat16, false>(a, g, sg, grid, ngroups, status, st);
+  return a.norm == 1 ? launch_fwd_staged_t<float, true>(a, g, sg, grid, ngroups, status, st)
+                     : launch_fwd_staged_t<float, false>(a, g, sg, grid, ngroups, status, st);
+}
+
+// The grid (= rows of norm-gradient partials) must not exceed what the scratch layout reserves.
+cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,
+                                        cudaStream_t st) {
+  const RowGeom g = row_geometry(a.h, dtype);
+  const int ES = (int)elem_size(dtype);
+  const bool has_c = a.dHn != nullptr;
+  int per_sm = ctas_per_sm(g);
+  StageGeom sg = stage_geometry(g, a.h, 0, 0, a.t, ES, true, has_c, kSmemPerSm / per_sm - 1024);
+  while (sg.nstages < 3 && per_sm > 1) {
+    --per_sm;
+    sg = stage_geometry(g, a.h, 0, 0, a.t, ES, true, has_c, kSmemPerSm / per_sm - 1024);
+  }
+  if (sg.nstages < 2) return cudaErrorInvalidConfiguration;
+  const int ngroups = (a.T + g.TY - 1) / g.TY;
+  int grid = sm_count() * per_sm;
+  if (grid > ngroups) grid = ngroups;
+  if (grid > max_rows) grid = max_rows;
+  *rows_used = grid;
+  unsigned int* status = device_status_word();
+  if (!status) return cudaErrorUnknown;
+  if (dtype == CAAT_BF16)
+    return a.norm == 1 ? launch_bwd_staged_t<__nv_bfloat16, true>(a, g, sg, grid, ngroups, status, st)
+                       : launch_bwd_staged_t<__nv_bfloat16, false>(a, g, sg, grid, ngroups, status, st);
+  return a.norm == 1 ? launch_bwd_staged_t<float, true>(a, g, sg, grid, ngroups, status, st)
+                     : launch_bwd_staged_t<float, false>(a, g, sg, grid, ngroups, status, st);
+}
+
+}  // namespace caat

@@ -102,6 +102,19 @@ def test_both_gemm_paths_agree_with_oracle(force_simt):
     _check_backward(ctx, caat.CAAT_MLP_DOWN, d, "bf16")
 
 
+@pytest.mark.parametrize("direct_rows", [False, True])
+@pytest.mark.parametrize("t,T,h,ffn,S,norm,dtype", [
+    (8, 77, 4096, 11008, 2048, 0, "bf16"), (4, 301, 768, 3072, 380, 1, "bf16"), (2, 131, 256, 1024, 100, 1, "f32"),
+    (8, 1500, 2048, 5632, 2048, 0, "bf16"), (3, 45, 9216, 9216, 4608, 0, "bf16")])
+def test_both_row_kernel_variants(direct_rows, t, T, h, ffn, S, norm, dtype):
+    # the bulk-copy staged kernels (default) and the plain-load kernels compute the same thing;
+    # T = 1500 makes persistent CTAs walk several token groups, h = 9216 takes two chunks per thread
+    ctx = G.make_ctx(t, h, ffn, dtype, S=S, norm=norm, direct_rows=direct_rows)
+    d = _layer_case(t, T, h, ctx.k_r(caat.CAAT_ATTN_OUT), dtype, S, seed=T, backward=True)
+    _check_forward(ctx, caat.CAAT_ATTN_OUT, d, dtype)
+    _check_backward(ctx, caat.CAAT_ATTN_OUT, d, dtype)
+
+
 # ------------------------------------------------------------------ partition: bit-exact
 @pytest.mark.parametrize("S", [0, 1, 7, 8, 9, 127, 128, 129, 255, 256, 257, 504, 511, 512])
 def test_partition_bit_exact_integer_inputs(S):
