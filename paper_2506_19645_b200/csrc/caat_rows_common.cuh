@@ -113,8 +113,11 @@ inline RowGeom row_geometry(int h, caat_dtype dtype) {
   const int V = dtype == CAAT_BF16 ? 8 : 4;
   const int chunks = h / V;
   RowGeom g;
-  int tx = round_up(chunks, 32);
-  g.CPT = 1;
+  // Two chunks per thread whenever the row is long enough: the per-rank overhead (barrier
+  // wait, row reduction, pointer updates) is paid once per thread, and 256 threads with up
+  // to 128 registers leave room for two CTAs per SM without spills.
+  g.CPT = chunks < 64 ? 1 : 2;
+  int tx = round_up((chunks + g.CPT - 1) / g.CPT, 32);
   while (tx > 512) {
     g.CPT *= 2;
     tx = round_up((chunks + g.CPT - 1) / g.CPT, 32);

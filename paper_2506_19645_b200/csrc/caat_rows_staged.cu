@@ -20,7 +20,8 @@ namespace {
 
 using namespace rows;
 
-constexpr uint32_t kSpinCap = 1u << 22;
+constexpr uint32_t kSpinCap = 1u << 18;
+constexpr uint32_t kSuspendHintNs = 20000u;   // the waiting warp sleeps in hardware instead of spinning
 constexpr int kMaxStages = 8;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -33,9 +34,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok != 0;
 }
@@ -63,8 +64,8 @@ struct StageGeom {
 
 // ------------------------------------------------------------------ forward
 // stage buffers: a = R rows [TY, h], b = zp rows [TY, P], c = zs rows [TY, S_hi] (rank 0 only)
-template <typename T_, int CPT, bool LN>
-__global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1)
+template <typename T_, int CPT, bool LN, int MAXT>
+__global__ void __launch_bounds__(MAXT, (CPT == 1 || MAXT <= 256) ? 2 : 1)
 rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
@@ -243,8 +244,8 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
 
 // ------------------------------------------------------------------ backward
 // stage buffers: a = dX rows, b = Hn rows, c = dHn rows (when given)
-template <typename T_, int CPT, bool LN>
-__global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1)
+template <typename T_, int CPT, bool LN, int MAXT>
+__global__ void __launch_bounds__(MAXT, (CPT == 1 || MAXT <= 256) ? 2 : 1)
 rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
@@ -567,21 +568,18 @@ cudaError_t launch_fwd_staged_t(const RowFwdArgs& a, const RowGeom& g, const Sta
   const dim3 block(g.TX, g.TY);
   cudaError_t e = cudaSuccess;
   LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
-  switch (g.CPT) {
-    case 1:
-      e = set_smem(rows_forward_staged<T_, 1, LN>, sg.smem);
-      if (e == cudaSuccess) rows_forward_staged<T_, 1, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
-      break;
-    case 2:
-      e = set_smem(rows_forward_staged<T_, 2, LN>, sg.smem);
-      if (e == cudaSuccess) rows_forward_staged<T_, 2, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
-      break;
-    case 4:
-      e = set_smem(rows_forward_staged<T_, 4, LN>, sg.smem);
-      if (e == cudaSuccess) rows_forward_staged<T_, 4, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
-      break;
-    default: return cudaErrorInvalidValue;
-  }
+  const int threads = g.TX * g.TY;
+#define CAAT_LAUNCH(CPT_, MAXT_)                                                                   \
+  do {                                                                                             \
+    e = set_smem(rows_forward_staged<T_, CPT_, LN, MAXT_>, sg.smem);                                            \
+    if (e == cudaSuccess) rows_forward_staged<T_, CPT_, LN, MAXT_><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);       \
+  } while (0)
+  if (g.CPT == 1) CAAT_LAUNCH(1, 512);
+  else if (g.CPT == 2 && threads <= 256) CAAT_LAUNCH(2, 256);
+  else if (g.CPT == 2) CAAT_LAUNCH(2, 512);
+  else if (g.CPT == 4) CAAT_LAUNCH(4, 512);
+  else return cudaErrorInvalidValue;
+#undef CAAT_LAUNCH
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -591,21 +589,18 @@ cudaError_t launch_bwd_staged_t(const RowBwdArgs& a, const RowGeom& g, const Sta
   const dim3 block(g.TX, g.TY);
   cudaError_t e = cudaSuccess;
   LaunchScope scope(CAAT_K_ROWS_BACKWARD, st);
-  switch (g.CPT) {
-    case 1:
-      e = set_smem(rows_backward_staged<T_, 1, LN>, sg.smem);
-      if (e == cudaSuccess) rows_backward_staged<T_, 1, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
-      break;
-    case 2:
-      e = set_smem(rows_backward_staged<T_, 2, LN>, sg.smem);
-      if (e == cudaSuccess) rows_backward_staged<T_, 2, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
-      break;
-    case 4:
-      e = set_smem(rows_backward_staged<T_, 4, LN>, sg.smem);
-      if (e == cudaSuccess) rows_backward_staged<T_, 4, LN><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);
-      break;
-    default: return cudaErrorInvalidValue;
-  }
+  const int threads = g.TX * g.TY;
+#define CAAT_LAUNCH(CPT_, MAXT_)                                                                   \
+  do {                                                                                             \
+    e = set_smem(rows_backward_staged<T_, CPT_, LN, MAXT_>, sg.smem);                                            \
+    if (e == cudaSuccess) rows_backward_staged<T_, CPT_, LN, MAXT_><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);       \
+  } while (0)
+  if (g.CPT == 1) CAAT_LAUNCH(1, 512);
+  else if (g.CPT == 2 && threads <= 256) CAAT_LAUNCH(2, 256);
+  else if (g.CPT == 2) CAAT_LAUNCH(2, 512);
+  else if (g.CPT == 4) CAAT_LAUNCH(4, 512);
+  else return cudaErrorInvalidValue;
+#undef CAAT_LAUNCH
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -613,8 +608,9 @@ constexpr size_t kSmemPerSm = 227 * 1024;
 
 // resident CTAs per SM the register budget allows (64 registers per thread when CPT == 1)
 int ctas_per_sm(const RowGeom& g) {
-  if (g.CPT != 1) return 1;
-  int n = 1024 / (g.TX * g.TY);
+  const int threads = g.TX * g.TY;
+  if (g.CPT != 1) return threads <= 256 ? 2 : 1;   // 128 registers per thread
+  int n = 1024 / threads;                           // 64 registers per thread
   return n < 1 ? 1 : (n > 8 ? 8 : n);
 }
 
