@@ -32,6 +32,7 @@ constexpr int kAccCols = 256;     // column stride between the two accumulators
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSpinCap = 1u << 22;
 constexpr int kMaxStages = 8;
+constexpr int kCBuf = 128 * 64;   // one output staging buffer: 128 rows x 64 bytes (32 bf16 / 16 fp32 columns)
 
 struct Unit {            // one contraction segment of a tile
   int mapA, mapB;        // indices into the tensor-map array
@@ -47,11 +48,8 @@ struct Region {          // a family of output tiles with the same operand wirin
   int nunits;
   Unit u[2];
   int M, N, batch;       // valid output extents per batch
-  int mtiles, ntiles;
-  void* out;             // element (b, i, j) at out + (b * ldb + i * ldc + j) elements
-  long long ldc, ldb;
-  long long split_stride;  // elements between split-K partials (0: no split-K)
-};
+  int mtiles, ntiles;    // the output goes through the region's own tensor map (TMA store);
+};                       // its z coordinate is split * batch + b
 
 struct Params {
   int nregions;
@@ -128,6 +126,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, int x, int y, int z, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+               ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
@@ -171,7 +190,8 @@ __device__ __forceinline__ void split_range(const Params& p, const Unit& u, int 
 
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
-               const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map3, const Params p) {
+               const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map3,
+               const __grid_constant__ CUtensorMap cmap0, const __grid_constant__ CUtensorMap cmap1, const Params p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // carve: [stages x (A tile | B tile)] then barriers
   const uint32_t a_bytes = BM * BK * 2;
@@ -179,7 +199,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   const uint32_t stage_bytes = a_bytes + b_bytes;
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t tiles_sa = smem_u32(base);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)p.nstages * stage_bytes);
+  uint8_t* cstage = base + (size_t)p.nstages * stage_bytes;   // 3 output staging buffers of kCBuf bytes
+  uint64_t* bars = reinterpret_cast<uint64_t*>(cstage + 3 * kCBuf);
   // bars: full[nstages], empty[nstages], tfull[2], tempty[2]
   const uint32_t full0 = smem_u32(bars);
   const uint32_t empty0 = full0 + 8u * p.nstages;
@@ -190,6 +211,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const CUtensorMap* maps[4] = {&map0, &map1, &map2, &map3};
+  const CUtensorMap* cmaps[2] = {&cmap0, &cmap1};
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.nstages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
@@ -307,6 +329,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter+32)
     int acc = 0; uint32_t acc_phase = 0;
+    uint32_t slab = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
       const TileCoord c = decode_tile(p, tile);
@@ -320,49 +343,50 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       }
       if (!mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int row = c.mt * BM + quarter * 32 + lane;
+      // Drain 64-byte-wide column slabs (32 bf16 / 16 fp32 columns): TMEM -> registers ->
+      // swizzled staging buffer -> TMA store (coalesced; rows and columns outside the region's
+      // extents are clipped by the tensor map).  Three buffers, one 128-thread barrier per slab.
       const int n0 = c.nt * p.BN;
-      const bool row_ok = row < r.M;
-      const long long obase = (long long)c.split * r.split_stride + (long long)c.b * r.ldb + (long long)row * r.ldc;
-      for (int cc = 0; cc < p.BN; cc += 32) {
+      const int m0 = c.mt * BM;
+      const int zc = c.split * r.batch + c.b;
+      const int sub = p.out_f32 ? 16 : 32;
+      const int rr = quarter * 32 + lane;                 // row of the tile this thread holds
+      const uint32_t sw = (uint32_t)((rr >> 1) & 3);      // 64-byte swizzle: chunk ^= (row / 2) % 4
+      for (int cc = 0; cc < p.BN && n0 + cc < r.N; cc += sub) {
         uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols + cc), v);
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols + cc);
+        if (p.out_f32) tmem_ld16(taddr, v); else tmem_ld32(taddr, v);
         tmem_ld_wait();
         if (total_k == 0) {
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = 0u;
         }
-        int ncol = r.N - (n0 + cc);         // valid columns from here, within this tile
-        if (ncol > p.BN - cc) ncol = p.BN - cc;
-        if (row_ok && ncol > 0) {
-          if (p.out_f32) {
-            float* o = static_cast<float*>(r.out) + obase + n0 + cc;
-            if (ncol >= 32 && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
+        const uint32_t buf = smem_u32(cstage + (size_t)(slab % 3) * kCBuf);
+        const uint32_t rowaddr = buf + (uint32_t)rr * 64u;
+        if (p.out_f32) {
 #pragma unroll
-              for (int e = 0; e < 32; e += 4)
-                *reinterpret_cast<float4*>(o + e) = make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]),
-                                                                __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-            } else {
-              for (int e = 0; e < 32 && e < ncol; ++e) o[e] = __uint_as_float(v[e]);
+          for (int q4 = 0; q4 < 4; ++q4)
+            sts128(rowaddr + (((uint32_t)q4 ^ sw) << 4), v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+        } else {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint32_t w[4];
+#pragma unroll
+            for (int q2 = 0; q2 < 4; ++q2) {
+              __nv_bfloat162 bb = __floats2bfloat162_rn(__uint_as_float(v[8 * q4 + 2 * q2]), __uint_as_float(v[8 * q4 + 2 * q2 + 1]));
+              w[q2] = *reinterpret_cast<uint32_t*>(&bb);
             }
-          } else {
-            __nv_bfloat16* o = static_cast<__nv_bfloat16*>(r.out) + obase + n0 + cc;
-            if (ncol >= 32 && ((reinterpret_cast<uintptr_t>(o) & 15u) == 0)) {
-#pragma unroll
-              for (int e = 0; e < 32; e += 8) {
-                uint32_t w[4];
-#pragma unroll
-                for (int q2 = 0; q2 < 4; ++q2) {
-                  __nv_bfloat162 bb = __floats2bfloat162_rn(__uint_as_float(v[e + 2 * q2]), __uint_as_float(v[e + 2 * q2 + 1]));
-                  w[q2] = *reinterpret_cast<uint32_t*>(&bb);
-                }
-                *reinterpret_cast<uint4*>(o + e) = make_uint4(w[0], w[1], w[2], w[3]);
-              }
-            } else {
-              for (int e = 0; e < 32 && e < ncol; ++e) o[e] = __float2bfloat16_rn(__uint_as_float(v[e]));
-            }
+            sts128(rowaddr + (((uint32_t)q4 ^ sw) << 4), w[0], w[1], w[2], w[3]);
           }
         }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        epi_barrier();
+        if (warp == 2 && lane == 0) {
+          tma_store_3d(cmaps[c.region], n0 + cc, m0, zc, buf);
+          bulk_commit();
+          bulk_wait_read1();     // the store before this one has finished reading its buffer
+        }
+        ++slab;
       }
       tc_fence_before();
       __syncwarp();
@@ -370,6 +394,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
+    if (warp == 2 && lane == 0) bulk_wait_all();   // all output stores of this CTA are complete
     if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, 3u); }
   }
 
@@ -412,31 +437,39 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 tensor [d2][d1][d0] (d0 contiguous) with row pitch ld1 and plane pitch ld2 (elements);
-// box = (b0, b1, 1) with 128-byte swizzle; out-of-range elements read as zero.
+// Tensor [d2][d1][d0] (d0 contiguous) with row pitch ld1 and plane pitch ld2 (elements);
+// box = (b0, b1, 1); out-of-range elements read as zero and are not written.
 bool make_map(CUtensorMap* m, const void* base, long long d0, long long d1, long long d2, long long ld1, long long ld2,
-              int b0, int b1) {
+              int b0, int b1, bool f32 = false, CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_128B) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   if (d0 < 1 || d1 < 1 || d2 < 1) return false;
+  const cuuint64_t es_bytes = f32 ? 4 : 2;
   cuuint64_t dims[3] = {(cuuint64_t)d0, (cuuint64_t)d1, (cuuint64_t)d2};
-  cuuint64_t strides[2] = {(cuuint64_t)ld1 * 2, (cuuint64_t)ld2 * 2};
+  cuuint64_t strides[2] = {(cuuint64_t)ld1 * es_bytes, (cuuint64_t)ld2 * es_bytes};
   cuuint32_t box[3] = {(cuuint32_t)b0, (cuuint32_t)b1, 1};
   cuuint32_t es[3] = {1, 1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                  const_cast<void*>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
+// Output map: slabs of 64 bytes x 128 rows, 64-byte swizzle (matches the epilogue's staging layout).
+bool make_cmap(CUtensorMap* m, const void* base, long long d0, long long d1, long long d2, long long ld1,
+               long long ld2, bool f32) {
+  return make_map(m, base, d0, d1, d2, ld1, ld2, f32 ? 16 : 32, BM, f32, CU_TENSOR_MAP_SWIZZLE_64B);
+}
+
 int pick_bn(int n, bool multiple_of_64) {
-  // widest tile that wastes little: minimise padded width, prefer the wider tile on ties
+  // Operand traffic per tile and k-step is proportional to (BM + BN): minimise tiles * (BM + BN),
+  // preferring the wider tile on ties.
   const int step = multiple_of_64 ? 64 : 32;   // the epilogue drains 32 columns at a time
   int best = 256;
   long long best_cost = -1;
   for (int bn = 256; bn >= 64; bn -= step) {
     const long long tiles = (n + bn - 1) / bn;
-    const long long cost = tiles * bn * 16 + tiles * 64;  // padded columns (x16) plus a per-tile overhead
+    const long long cost = tiles * (BM + bn);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
   }
   return best;
@@ -452,13 +485,13 @@ int sm_count() {
   return n;
 }
 
-cudaError_t launch(const CUtensorMap maps[4], Params& p, int kind, cudaStream_t st) {
+cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params& p, int kind, cudaStream_t st) {
   const int stage_bytes = BM * BK * 2 + p.BN * BK * 2;
-  int nst = (227 * 1024 - 2048) / stage_bytes;
+  int nst = (227 * 1024 - 2048 - 3 * kCBuf) / stage_bytes;
   if (nst > kMaxStages) nst = kMaxStages;
   if (nst < 2) return cudaErrorInvalidConfiguration;
   p.nstages = nst;
-  const size_t smem = (size_t)nst * stage_bytes + 1024 /*alignment slack*/ + (2 * nst + 4) * 8 + 16;
+  const size_t smem = (size_t)nst * stage_bytes + 3 * kCBuf + 1024 /*alignment slack*/ + (2 * nst + 4) * 8 + 16;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -470,7 +503,7 @@ cudaError_t launch(const CUtensorMap maps[4], Params& p, int kind, cudaStream_t 
   int grid = p.tiles_total < sm_count() ? p.tiles_total : sm_count();
   if (grid < 1) return cudaSuccess;
   LaunchScope scope(kind, st);
-  tc_gemm_kernel<<<grid, kThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  tc_gemm_kernel<<<grid, kThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], p);
   return cudaGetLastError();
 }
 
@@ -493,7 +526,7 @@ bool tc_gemm_usable(const caat_ctx* ctx, int K_r) {
 // ---- forward: zs[T,S] = sum_m Y[m] W[m][:S]^T ; zp[m][T,h-S] = Y[m] W[m][S:]^T
 cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* W, void* zs, void* zp,
                               cudaStream_t st) {
-  CUtensorMap maps[4];
+  CUtensorMap maps[4], cmaps[2];
   Params p{};
   const int n_sh = s.S, n_pr = s.h - s.S;
   p.BN = pick_bn(n_pr > 0 && n_sh > 0 ? (n_sh < n_pr ? n_sh : n_pr) : (n_sh > 0 ? n_sh : n_pr), false);
@@ -509,25 +542,27 @@ cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* 
     r.nunits = 1;
     r.u[0] = Unit{0, 1, 0, 0, 0, 0, /*a_zb*/ 0, /*a_zq*/ 1, /*b_zb*/ 0, /*b_zq*/ 1, s.t, ksteps};
     r.M = s.T; r.N = n_sh; r.batch = 1;
-    r.out = zs; r.ldc = s.S_hi; r.ldb = 0; r.split_stride = 0;
+    if (!make_cmap(&cmaps[g - 1], zs, n_sh, s.T, 1, s.S_hi, (long long)s.T * s.S_hi, false)) return cudaErrorInvalidValue;
   }
   if (n_pr > 0) {
     Region& r = p.r[g++];
     r.nunits = 1;
     r.u[0] = Unit{0, 1, 0, 0, 0, s.S, 1, 0, 1, 0, 1, ksteps};
     r.M = s.T; r.N = n_pr; r.batch = s.t;
-    r.out = static_cast<__nv_bfloat16*>(zp) + (s.S - s.S_lo); r.ldc = s.P; r.ldb = (long long)s.T * s.P;
-    r.split_stride = 0;
+    if (!make_cmap(&cmaps[g - 1], static_cast<__nv_bfloat16*>(zp) + (s.S - s.S_lo), n_pr, s.T, s.t, s.P,
+                   (long long)s.T * s.P, false))
+      return cudaErrorInvalidValue;
   }
+  if (g == 1) cmaps[1] = cmaps[0];
   p.nregions = g;
   finish_tiles(p);
-  return launch(maps, p, CAAT_K_TC_FORWARD, st);
+  return launch(maps, cmaps, p, CAAT_K_TC_FORWARD, st);
 }
 
 // ---- dgrad: dY[m] = gs W[m][:S] + zp[m] W[m][S:]
 cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* zp, const void* W, void* dY,
                             cudaStream_t st) {
-  CUtensorMap maps[4];
+  CUtensorMap maps[4], cmaps[2];
   Params p{};
   p.BN = pick_bn(s.K_r, true);
   const int n_sh = s.S, n_pr = s.h - s.S;
@@ -546,10 +581,11 @@ cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* z
   if (n_pr > 0) r.u[nu++] = Unit{2, 1, s.S - s.S_lo, 0, s.S, 0, 1, 0, 1, 0, 1, (n_pr + BK - 1) / BK};
   r.nunits = nu;
   r.M = s.T; r.N = s.K_r; r.batch = s.t;
-  r.out = dY; r.ldc = s.K_r; r.ldb = (long long)s.T * s.K_r; r.split_stride = 0;
+  if (!make_cmap(&cmaps[0], dY, s.K_r, s.T, s.t, s.K_r, (long long)s.T * s.K_r, false)) return cudaErrorInvalidValue;
+  cmaps[1] = cmaps[0];
   p.nregions = 1;
   finish_tiles(p);
-  return launch(maps, p, CAAT_K_TC_DGRAD, st);
+  return launch(maps, cmaps, p, CAAT_K_TC_DGRAD, st);
 }
 
 static int wgrad_splits(const RowparShapes& s, int BN) {
@@ -572,7 +608,7 @@ size_t tc_wgrad_splitk_bytes(const RowparShapes& s) {
 // ---- wgrad: dW[m][:S] = gs^T Y[m] ; dW[m][S:] = zp[m]^T Y[m]      (fp32 out)
 cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* zp, const void* Y, float* dW,
                             void* splitk, size_t splitk_bytes, cudaStream_t st) {
-  CUtensorMap maps[4];
+  CUtensorMap maps[4], cmaps[2];
   Params p{};
   p.BN = pick_bn(s.K_r, true);
   const int n_sh = s.S, n_pr = s.h - s.S;
@@ -597,19 +633,22 @@ cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* z
     r.nunits = 1;
     r.u[0] = Unit{0, 1, 0, 0, 0, 0, 0, 0, 1, 0, 1, ksteps};
     r.M = n_sh; r.N = s.K_r; r.batch = s.t;
-    r.out = out; r.ldc = s.K_r; r.ldb = (long long)s.h * s.K_r; r.split_stride = splits > 1 ? dw_elems : 0;
+    if (!make_cmap(&cmaps[g - 1], out, s.K_r, n_sh, (long long)s.t * splits, s.K_r, (long long)s.h * s.K_r, true))
+      return cudaErrorInvalidValue;
   }
   if (n_pr > 0) {
     Region& r = p.r[g++];
     r.nunits = 1;
     r.u[0] = Unit{2, 1, 0, s.S - s.S_lo, 0, 0, 1, 0, 1, 0, 1, ksteps};
     r.M = n_pr; r.N = s.K_r; r.batch = s.t;
-    r.out = out + (long long)s.S * s.K_r; r.ldc = s.K_r; r.ldb = (long long)s.h * s.K_r;
-    r.split_stride = splits > 1 ? dw_elems : 0;
+    if (!make_cmap(&cmaps[g - 1], out + (long long)s.S * s.K_r, s.K_r, n_pr, (long long)s.t * splits, s.K_r,
+                   (long long)s.h * s.K_r, true))
+      return cudaErrorInvalidValue;
   }
+  if (g == 1) cmaps[1] = cmaps[0];
   p.nregions = g;
   finish_tiles(p);
-  cudaError_t e = launch(maps, p, CAAT_K_TC_WGRAD, st);
+  cudaError_t e = launch(maps, cmaps, p, CAAT_K_TC_WGRAD, st);
   if (e != cudaSuccess) return e;
   if (splits > 1) {
     const long long n4 = dw_elems / 4;   // K_r is a multiple of 8
