@@ -63,7 +63,9 @@ typedef enum {
   CAAT_EWORKSPACE = 4,   /* workspace NULL or smaller than caat_workspace_bytes */
   CAAT_EUNSUPPORTED = 5, /* shape outside the limits stated above               */
   CAAT_ECUDA = 6,        /* a CUDA runtime call failed (see caat_last_cuda_error) */
-  CAAT_ETIMEOUT = 7      /* a bounded device-side wait ran out                  */
+  CAAT_ETIMEOUT = 7,     /* a bounded device-side wait ran out                  */
+  CAAT_ELIMIT = 8        /* the call needs more than the built-in scratch of
+                            caat_rowpar_forward_noalloc (CAAT_NOALLOC_SCRATCH_BYTES) */
 } caat_status;
 
 typedef enum {
@@ -117,6 +119,42 @@ caat_status caat_rowpar_forward(const caat_ctx *ctx, caat_layer layer, int token
                                 const void *gamma, const void *beta,
                                 void *Hn, void *X, float *rstd, float *mean,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * caat_rowpar_forward for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the forward above, same arithmetic, same
+ * kernels, same results.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits when the layer is invoked -
+ * inside a serving loop whose memory pool is frozen after start-up, under a framework that
+ * forbids allocation on its compute stream, or in a process whose device memory is handed
+ * out by another component - and that therefore has no workspace buffer to pass.  Instead
+ * of a caller-owned workspace the call uses a fixed scratch array of
+ * CAAT_NOALLOC_SCRATCH_BYTES that is part of the library's device image; every GPU that
+ * loads the library holds those bytes until the process exits.
+ *
+ * Arguments and outputs are those of caat_rowpar_forward without workspace/workspace_bytes;
+ * the caller still owns and passes every input and output tensor.
+ *   Limit      the call is rejected with CAAT_ELIMIT, before any launch, when
+ *              caat_workspace_bytes(ctx, layer, tokens, 0) exceeds CAAT_NOALLOC_SCRATCH_BYTES
+ *              (e.g. 130M shapes, t=4, h=768, p=0.5: up to 8738 tokens per call).
+ *   Set-up     the first call on each device looks up the scratch array's device address
+ *              (once per device, with that device current).  Make that first call before
+ *              starting any CUDA stream capture on the device.
+ *   Allocation the call itself performs no cudaMalloc / cudaFree and calls no allocating
+ *              library routine.
+ *   Sharing    all calls on a device use the same array, which keeps whatever the last call
+ *              left in it.  Nothing in it needs to start at zero (every element that is read
+ *              is written earlier in the same call).  Two calls that overlap on the GPU
+ *              (different streams, or different host threads without ordering) race on it:
+ *              order such calls on one stream or with events.
+ */
+#define CAAT_NOALLOC_SCRATCH_BYTES (32u * 1024u * 1024u)
+caat_status caat_rowpar_forward_noalloc(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                        const void *Y, const void *W, const void *R,
+                                        const void *gamma, const void *beta,
+                                        void *Hn, void *X, float *rstd, float *mean,
+                                        void *cuda_stream);
 
 /*
  * Backward of the same sub-layer: the exact gradient of the forward map, with the

@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_PKG, "libcaat.so")
 CAAT_F32, CAAT_BF16 = 0, 1
 CAAT_ATTN_OUT, CAAT_MLP_DOWN = 0, 1
 (CAAT_OK, CAAT_EINVAL, CAAT_ESHAPE, CAAT_EALIGN, CAAT_EWORKSPACE, CAAT_EUNSUPPORTED, CAAT_ECUDA,
- CAAT_ETIMEOUT) = range(8)
+ CAAT_ETIMEOUT, CAAT_ELIMIT) = range(9)
+CAAT_NOALLOC_SCRATCH_BYTES = 32 * 1024 * 1024
 CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM, CAAT_OPT_ROWS = range(6)
 RMSNORM, LAYERNORM = 0, 1
 
@@ -39,6 +40,7 @@ _sigs = {
     "caat_strerror": (c_char_p, [c_int]),
     "caat_last_cuda_error": (c_char_p, []),
     "caat_rowpar_forward": (c_int, [_P, c_int, c_int] + [_P] * 9 + [_P, c_size_t, _P]),
+    "caat_rowpar_forward_noalloc": (c_int, [_P, c_int, c_int] + [_P] * 9 + [_P]),
     "caat_rowpar_backward": (c_int, [_P, c_int, c_int] + [_P] * 13 + [_P, c_size_t, _P]),
     "caat_block_forward": (c_int, [_P, c_int] + [_P] * 17 + [_P, c_size_t, _P]),
     "caat_block_backward": (c_int, [_P, c_int] + [_P] * 25 + [_P, c_size_t, _P]),
@@ -159,6 +161,20 @@ class Context:
             _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
             _stream())
         _check(st, "caat_rowpar_forward")
+
+    def rowpar_forward_noalloc(self, layer, tokens, Y, W, R, gamma, beta, Hn, X, rstd, mean):
+        """caat_rowpar_forward without a caller workspace: for callers that cannot allocate device
+        memory when the layer runs.  Scratch is the library's built-in array (32 MiB); larger
+        problems raise CaatError(CAAT_ELIMIT).  Calls on one device must not overlap on the GPU."""
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        st = lib.caat_rowpar_forward_noalloc(
+            self._h, layer, tokens,
+            _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"), _ptr(R, td, (t, tokens, h), "R"),
+            _ptr(gamma, td, (h,), "gamma"), _ptr(beta, td, (h,), "beta"),
+            _ptr(Hn, td, (t, tokens, h), "Hn"), _ptr(X, td, (t, tokens, h), "X"),
+            _ptr(rstd, torch.float32, (t, tokens), "rstd"), _ptr(mean, torch.float32, (t, tokens), "mean"),
+            _stream())
+        _check(st, "caat_rowpar_forward_noalloc")
 
     def rowpar_backward(self, layer, tokens, dX, dHn, Y, W, Hn, rstd, mean, gamma, dY, dW, dR, dgamma, dbeta,
                         workspace):

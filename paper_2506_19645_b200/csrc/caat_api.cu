@@ -264,6 +264,7 @@ const char* caat_strerror(caat_status s) {
     case CAAT_EUNSUPPORTED: return "shape not supported";
     case CAAT_ECUDA: return "CUDA error";
     case CAAT_ETIMEOUT: return "device-side wait timed out";
+    case CAAT_ELIMIT: return "needs more than the built-in scratch of the no-allocation entry point";
   }
   return "unknown status";
 }
