@@ -1,0 +1,141 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times (block
+forward + backward through the C ABI on the full token count).
+
+The fp64 oracle cannot hold a full-size problem at once, so it walks the tokens in chunks
+(tokens are independent rows in everything except dW and dgamma, which are sums over tokens
+and are accumulated across chunks).  Compared: every forward/backward activation output on a
+seeded sample of tokens (whole rows, all ranks), dgamma in full, and dW on a seeded sample of
+(rank, channel, input) entries, each a full sum over all tokens.  Saved tensors handed to the
+GPU backward are the oracle's forward results rounded to their storage types, never GPU
+outputs."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import caat_oracle as O
+from paper_2506_19645_b200 import caat, synthetic
+from tests.helpers import assert_close, f64
+
+pytestmark = pytest.mark.gpu
+
+CHUNK = 1024
+
+
+def _chunks(T):
+    for a in range(0, T, CHUNK):
+        yield a, min(T, a + CHUNK)
+
+
+def _check_block_full(name, n_tok=48, n_dw=512, seed=123):
+    w = synthetic.WORKLOADS[name]
+    t, T, h, S = w.t, w.tokens, w.h, w.S
+    alpha = math.sqrt(t)
+    ka, km = w.kr_attn, w.kr_mlp
+    dev = synthetic.block_inputs(w, device="cuda")
+    host = {k: v.cpu() for k, v in dev.items()}
+    rng = np.random.default_rng(seed)
+    tok = np.sort(rng.choice(T, size=min(n_tok, T), replace=False))
+    dws = {"attn": (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, ka, n_dw)),
+           "mlp": (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, km, n_dw))}
+    Wd = {"attn": f64(host["W_o"]), "mlp": f64(host["W_down"])}
+    g1, g2 = f64(host["gamma1"]), f64(host["gamma2"])
+
+    # ---------------- oracle forward, chunked; keep saved tensors (rounded) and sampled rows
+    sHn1 = torch.empty((t, T, h), dtype=torch.bfloat16); sHn2 = torch.empty_like(sHn1)
+    sr1 = torch.empty((t, T), dtype=torch.float32); sr2 = torch.empty_like(sr1)
+    fwd_s = {k: [] for k in ("Hn1", "X1", "rstd1", "Hn2", "X2", "rstd2")}
+    for a, b in _chunks(T):
+        sl = slice(a, b)
+        o = O.block_forward(f64(host["Y_attn"][:, sl]), Wd["attn"], f64(host["Y_mlp"][:, sl]), Wd["mlp"],
+                            f64(host["R0"][:, sl]), g1, g2, S=S, alpha=alpha)
+        sHn1[:, sl] = torch.from_numpy(o["Hn1"]).to(torch.bfloat16); sHn2[:, sl] = torch.from_numpy(o["Hn2"]).to(torch.bfloat16)
+        sr1[:, sl] = torch.from_numpy(o["rstd1"]).float(); sr2[:, sl] = torch.from_numpy(o["rstd2"]).float()
+        loc = tok[(tok >= a) & (tok < b)] - a
+        for k in fwd_s:
+            fwd_s[k].append(o[k][:, loc])
+    fwd_s = {k: np.concatenate(v, axis=1) for k, v in fwd_s.items()}
+
+    # ---------------- GPU: the bench's launch configuration (block forward, then block backward)
+    ctx = caat.Context(w.h, w.ffn, t, w.p, "bf16")
+    assert ctx.shared_channels == S
+    mk = lambda *s, dt=torch.bfloat16: torch.empty(*s, dtype=dt, device="cuda")
+    f32 = torch.float32
+    out = {"Hn1": mk(t, T, h), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=f32), "Hn2": mk(t, T, h), "X2": mk(t, T, h),
+           "rstd2": mk(t, T, dt=f32)}
+    ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, True))
+    ctx.block_forward(T, dev["Y_attn"], dev["W_o"], dev["Y_mlp"], dev["W_down"], dev["R0"], dev["gamma1"], None,
+                      dev["gamma2"], None, out["Hn1"], out["X1"], out["rstd1"], None, out["Hn2"], out["X2"],
+                      out["rstd2"], None, ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+    tk = torch.from_numpy(tok).cuda()
+    for k in fwd_s:
+        assert_close(out[k].index_select(1, tk), fwd_s[k], "bf16", f"{name}:{k}")
+    if not w.backward:
+        return
+    del out
+    bo = {"dY_attn": mk(t, T, ka), "dW_o": mk(t, h, ka, dt=f32), "dY_mlp": mk(t, T, km), "dW_down": mk(t, h, km, dt=f32),
+          "dR0": mk(t, T, h), "dHn1": mk(t, T, h), "dgamma1": mk(h, dt=f32), "dgamma2": mk(h, dt=f32)}
+    ctx.block_backward(T, dev["dX1"], dev["dX2"], dev["dHn2"], dev["Y_attn"], dev["W_o"], dev["Y_mlp"], dev["W_down"],
+                       sHn1.cuda(), sr1.cuda(), None, sHn2.cuda(), sr2.cuda(), None, dev["gamma1"], dev["gamma2"],
+                       bo["dY_attn"], bo["dW_o"], bo["dY_mlp"], bo["dW_down"], bo["dR0"], bo["dHn1"], bo["dgamma1"], None,
+                       bo["dgamma2"], None, ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+
+    # ---------------- oracle backward, chunked (MLP-down first, then attention-out on its dR)
+    acc = {"dgamma1": np.zeros(h), "dgamma2": np.zeros(h), "dW_attn": np.zeros(n_dw), "dW_mlp": np.zeros(n_dw)}
+    bwd_s = {k: [] for k in ("dY_attn", "dY_mlp", "dR0", "dHn1")}
+    for a, b in _chunks(T):
+        sl = slice(a, b)
+        loc = tok[(tok >= a) & (tok < b)] - a
+        Hn2, r2 = f64(sHn2[:, sl]), f64(sr2[:, sl])
+        gm = O.residual_stream_gradient(f64(host["dX2"][:, sl]), f64(host["dHn2"][:, sl]), Hn2, r2, None, g2, O.RMSNORM)
+        acc["dgamma2"] += O.norm_param_gradients(f64(host["dX2"][:, sl]), Hn2, r2, None, O.RMSNORM)[0]
+        dZ2 = O.backward_partial_channel_reduce(gm, S, alpha)
+        Hn1, r1 = f64(sHn1[:, sl]), f64(sr1[:, sl])
+        ga = O.residual_stream_gradient(f64(host["dX1"][:, sl]), gm, Hn1, r1, None, g1, O.RMSNORM)
+        acc["dgamma1"] += O.norm_param_gradients(f64(host["dX1"][:, sl]), Hn1, r1, None, O.RMSNORM)[0]
+        dZ1 = O.backward_partial_channel_reduce(ga, S, alpha)
+        bwd_s["dY_mlp"].append(O.data_gradient(dZ2[:, loc], Wd["mlp"]))
+        bwd_s["dY_attn"].append(O.data_gradient(dZ1[:, loc], Wd["attn"]))
+        bwd_s["dHn1"].append(gm[:, loc]); bwd_s["dR0"].append(ga[:, loc])
+        for key, dZ, Yk in (("attn", dZ1, "Y_attn"), ("mlp", dZ2, "Y_mlp")):
+            m_, l_, k_ = dws[key]
+            Y = f64(host[Yk][:, sl])
+            acc["dW_" + key] += np.einsum("ni,ni->n", dZ[m_, :, l_], Y[m_, :, k_])   # dW[m,l,k] = sum_i dZt[m,i,l] Y[m,i,k]
+    bwd_s = {k: np.concatenate(v, axis=1) for k, v in bwd_s.items()}
+
+    for k in bwd_s:
+        assert_close(bo[k].index_select(1, tk), bwd_s[k], "bf16", f"{name}:{k}")
+    assert_close(bo["dgamma1"], acc["dgamma1"], "bf16", f"{name}:dgamma1")
+    assert_close(bo["dgamma2"], acc["dgamma2"], "bf16", f"{name}:dgamma2")
+    for key, gk in (("attn", "dW_o"), ("mlp", "dW_down")):
+        m_, l_, k_ = (torch.from_numpy(x).cuda() for x in dws[key])
+        assert_close(bo[gk][m_, l_, k_], acc["dW_" + key], "bf16", f"{name}:{gk}")
+
+
+def test_full_size_block_130m():
+    _check_block_full("block_130m", n_tok=96)
+
+
+@pytest.mark.parametrize("name", ["block_1p1b_p100", "block_1p1b_p050", "block_1p1b_p025"])
+def test_full_size_block_1p1b(name):
+    _check_block_full(name)
+
+
+def test_full_size_block_1p1b_p075_forward_sample():
+    # p = 0.75 at full size: forward only (the backward reduce at this S is covered at reduced T)
+    w = synthetic.WORKLOADS["block_1p1b_p075"]
+    fw = synthetic.Workload("block_1p1b_p075_fwd", w.t, w.tokens, w.h, w.ffn, w.p, w.dtype, w.kind, False, w.seed)
+    synthetic.WORKLOADS[fw.name] = fw
+    try:
+        _check_block_full(fw.name)
+    finally:
+        del synthetic.WORKLOADS[fw.name]
+
+
+def test_full_size_block_7b():
+    _check_block_full("block_7b", n_tok=32, n_dw=384)
