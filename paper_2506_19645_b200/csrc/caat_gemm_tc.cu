@@ -17,6 +17,8 @@
 // word, drains its own copies in flight, frees tensor memory and returns.
 #include <cuda.h>
 
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "caat_internal.h"
@@ -49,7 +51,9 @@ struct Region {          // a family of output tiles with the same operand wirin
   Unit u[2];
   int M, N, batch;       // valid output extents per batch
   int mtiles, ntiles;    // the output goes through the region's own tensor map (TMA store);
-};                       // its z coordinate is split * batch + b
+                         // its z coordinate is split * batch + b
+  int b_slowest;         // tile order: 1 = rank index slowest (a rank's weights / activations stay
+};                       // hot in L2 while its row tiles stream), 0 = row tile slowest
 
 struct Params {
   int nregions;
@@ -58,10 +62,12 @@ struct Params {
   int nstages;
   int a_mn, b_mn;        // 1: operand is MN-major in global memory
   int out_f32;
+  int cg;                // CTAs per tile: 1, or 2 (tcgen05 cta_group::2, clusters of two)
   int splits;            // split-K factor (only with a single unit and Q == 1)
   int tiles_r0;          // tiles of region 0 (including splits)
   int tiles_total;
   unsigned int* status;
+  int debug;             // measurement aid: 1 = producer skips the loads, 2 = epilogue skips the stores
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -174,8 +180,13 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& p, int tile) {
   const Region& r = p.r[c.region];
   c.nt = rem % r.ntiles; rem /= r.ntiles;
   c.split = rem % p.splits; rem /= p.splits;
-  c.b = rem % r.batch; rem /= r.batch;
-  c.mt = rem;
+  if (r.b_slowest) {
+    c.mt = rem % r.mtiles; rem /= r.mtiles;
+    c.b = rem;
+  } else {
+    c.b = rem % r.batch; rem /= r.batch;
+    c.mt = rem;
+  }
   return c;
 }
 
@@ -188,14 +199,61 @@ __device__ __forceinline__ void split_range(const Params& p, const Unit& u, int 
   if (k_begin > k_end) k_begin = k_end;
 }
 
+// ---- cluster helpers (CG == 2: a CTA pair works on one 256-row tile) -------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t saddr, uint32_t rank) {   // same offset in CTA `rank`
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion may be signalled on the peer CTA's mbarrier (no multicast)
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {   // arrives on `bar` in BOTH CTAs of the pair
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((unsigned short)3)
+      : "memory");
+}
+
+// CG = 1: one CTA per 128-row tile.  CG = 2: a cluster of two CTAs per 256-row tile
+// (tcgen05 cta_group::2): each CTA stages its own 128 rows of A and HALF of the B tile, the
+// leader (cluster rank 0) issues the MMAs for both and the tensor cores read B from both CTAs'
+// shared memory, so the operand bytes a CTA pulls from L2 per flop drop by a third.
+template <int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
                const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map3,
                const __grid_constant__ CUtensorMap cmap0, const __grid_constant__ CUtensorMap cmap1, const Params p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  // carve: [stages x (A tile | B tile)] then barriers
+  constexpr int BMT = BM * CG;                     // rows of a tile (of the pair's tile)
+  const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;
+  const int worker = blockIdx.x / CG, nworkers = gridDim.x / CG;
+  // carve: [stages x (A tile | this CTA's part of the B tile)], output staging, barriers
+  const uint32_t bn_cta = (uint32_t)p.BN / CG;
   const uint32_t a_bytes = BM * BK * 2;
-  const uint32_t b_bytes = (uint32_t)p.BN * BK * 2;
+  const uint32_t b_bytes = bn_cta * BK * 2;
   const uint32_t stage_bytes = a_bytes + b_bytes;
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t tiles_sa = smem_u32(base);
@@ -215,16 +273,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.nstages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8u * a, 1); mbar_init(tempty0 + 8u * a, 4 * CG); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CG == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync();      // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -234,10 +298,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       int stage = 0; uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
+      for (int tile = worker; tile < p.tiles_total && ok; tile += nworkers) {
         const TileCoord c = decode_tile(p, tile);
         const Region& r = p.r[c.region];
-        const int m0 = c.mt * BM, n0 = c.nt * p.BN;
+        const int m0 = c.mt * BMT + (int)rank * BM, n0 = c.nt * p.BN + (int)(rank * bn_cta);
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
           int kb, ke;
@@ -246,21 +310,34 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
             const int az = c.b * u.a_zb + q * u.a_zq, bz = c.b * u.b_zb + q * u.b_zq;
             for (int kk = kb; kk < ke; ++kk) {
               if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-              const uint32_t fb = full0 + 8u * stage;
+              const uint32_t fb_local = full0 + 8u * stage;
+              // completion is signalled on the LEADER's barrier; the leader expects both CTAs' bytes
+              const uint32_t fb = CG == 2 ? mapa_rank(fb_local, 0) : fb_local;
               const uint32_t sa = tiles_sa + (uint32_t)stage * stage_bytes, sb = sa + a_bytes;
-              mbar_expect_tx(fb, stage_bytes);
-              if (!p.a_mn) {
-                tma_load_3d(sa, maps[u.mapA], u.ak0 + kk * BK, m0, az, fb);
+              if (p.debug & 1) {
+                if (rank == 0) mbar_arrive(fb_local);
+                ++issued; if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+                continue;
+              }
+              if (rank == 0)
+                mbar_expect_tx(fb_local, (uint32_t)CG * (((p.debug & 4) ? 0u : a_bytes) + ((p.debug & 8) ? 0u : b_bytes)));
+              auto load = [&](uint32_t dst, const CUtensorMap* m, int x, int y, int z) {
+                if (CG == 2) tma_load_3d_pair(dst, m, x, y, z, fb); else tma_load_3d(dst, m, x, y, z, fb);
+              };
+              if (p.debug & 4) {
+              } else if (!p.a_mn) {
+                load(sa, maps[u.mapA], u.ak0 + kk * BK, m0, az);
               } else {
 #pragma unroll
                 for (int ch = 0; ch < BM / 64; ++ch)
-                  tma_load_3d(sa + ch * (64 * BK * 2), maps[u.mapA], u.am0 + m0 + ch * 64, u.ak0 + kk * BK, az, fb);
+                  load(sa + ch * (64 * BK * 2), maps[u.mapA], u.am0 + m0 + ch * 64, u.ak0 + kk * BK, az);
               }
-              if (!p.b_mn) {
-                tma_load_3d(sb, maps[u.mapB], u.bk0 + kk * BK, u.bn0 + n0, bz, fb);
+              if (p.debug & 8) {
+              } else if (!p.b_mn) {
+                load(sb, maps[u.mapB], u.bk0 + kk * BK, u.bn0 + n0, bz);
               } else {
-                for (int ch = 0; ch < p.BN / 64; ++ch)
-                  tma_load_3d(sb + ch * (64 * BK * 2), maps[u.mapB], u.bn0 + n0 + ch * 64, u.bk0 + kk * BK, bz, fb);
+                for (int ch = 0; ch < (int)bn_cta / 64; ++ch)
+                  load(sb + ch * (64 * BK * 2), maps[u.mapB], u.bn0 + n0 + ch * 64, u.bk0 + kk * BK, bz);
               }
               ++issued;
               if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
@@ -270,6 +347,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       }
       if (!ok) {
         // gave up: flag it, then wait (bounded) for the copies this thread still has in flight
+        // (the pair's copies complete on the leader's barriers; the peer just gives them time)
         *abort_flag = 1;
         atomicExch(p.status, 1u);
         const int pending = issued < p.nstages ? (int)issued : p.nstages;
@@ -277,19 +355,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         for (int k = 0; k < pending; ++k) {
           if (--s < 0) { s = p.nstages - 1; ph ^= 1u; }
           for (uint32_t it = 0; it < (1u << 20); ++it)
-            if (mbar_try(full0 + 8u * s, ph)) break;
+            if (rank == 0 && mbar_try(full0 + 8u * s, ph)) break;
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only when CG == 2)
+    if (lane == 0 && rank == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-                             ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                             ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BMT >> 4) << 24);
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
+      for (int tile = worker; tile < p.tiles_total && ok; tile += nworkers) {
         const TileCoord c = decode_tile(p, tile);
         const Region& r = p.r[c.region];
         if (!mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -311,15 +389,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
                                            : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
                 const uint64_t bd = p.b_mn ? make_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024)
                                            : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
-                umma_bf16(d_tmem, ad, bd, idesc, accumulate);
+                if (CG == 2) umma_bf16_pair(d_tmem, ad, bd, idesc, accumulate);
+                else umma_bf16(d_tmem, ad, bd, idesc, accumulate);
                 accumulate = 1;
               }
-              umma_commit(empty0 + 8u * stage);   // frees the stage once these MMAs have read it
+              // frees the stage (in both CTAs) once these MMAs have read it
+              if (CG == 2) umma_commit_pair(empty0 + 8u * stage); else umma_commit(empty0 + 8u * stage);
               if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
             }
           }
         }
-        if (ok) umma_commit(tfull0 + 8u * acc);    // accumulator complete
+        if (ok) {                                   // accumulator complete (in both CTAs)
+          if (CG == 2) umma_commit_pair(tfull0 + 8u * acc); else umma_commit(tfull0 + 8u * acc);
+        }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -331,7 +413,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     int acc = 0; uint32_t acc_phase = 0;
     uint32_t slab = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
+    for (int tile = worker; tile < p.tiles_total && ok; tile += nworkers) {
       const TileCoord c = decode_tile(p, tile);
       const Region& r = p.r[c.region];
       // a tile whose contraction range is empty leaves the accumulator undefined: its value is 0
@@ -347,12 +429,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       // swizzled staging buffer -> TMA store (coalesced; rows and columns outside the region's
       // extents are clipped by the tensor map).  Three buffers, one 128-thread barrier per slab.
       const int n0 = c.nt * p.BN;
-      const int m0 = c.mt * BM;
+      const int m0 = c.mt * BMT + (int)rank * BM;
       const int zc = c.split * r.batch + c.b;
       const int sub = p.out_f32 ? 16 : 32;
       const int rr = quarter * 32 + lane;                 // row of the tile this thread holds
       const uint32_t sw = (uint32_t)((rr >> 1) & 3);      // 64-byte swizzle: chunk ^= (row / 2) % 4
-      for (int cc = 0; cc < p.BN && n0 + cc < r.N; cc += sub) {
+      for (int cc = 0; cc < p.BN && n0 + cc < r.N && !(p.debug & 2); cc += sub) {
         uint32_t v[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols + cc);
         if (p.out_f32) tmem_ld16(taddr, v); else tmem_ld32(taddr, v);
@@ -390,7 +472,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8u * acc);
+      if (lane == 0) {           // this CTA's part of the accumulator is drained: tell the MMA issuer
+        if (CG == 2) mbar_arrive_cluster(mapa_rank(tempty0 + 8u * acc, 0)); else mbar_arrive(tempty0 + 8u * acc);
+      }
       acc ^= 1;
       if (acc == 0) acc_phase ^= 1u;
     }
@@ -400,9 +484,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
 
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync();   // the leader's MMAs read the peer's shared memory: leave together
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    if (CG == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -461,16 +549,60 @@ bool make_cmap(CUtensorMap* m, const void* base, long long d0, long long d1, lon
   return make_map(m, base, d0, d1, d2, ld1, ld2, f32 ? 16 : 32, BM, f32, CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
-int pick_bn(int n, bool multiple_of_64) {
-  // Operand traffic per tile and k-step is proportional to (BM + BN): minimise tiles * (BM + BN),
-  // preferring the wider tile on ties.
-  const int step = multiple_of_64 ? 64 : 32;   // the epilogue drains 32 columns at a time
-  int best = 256;
-  long long best_cost = -1;
-  for (int bn = 256; bn >= 64; bn -= step) {
-    const long long tiles = (n + bn - 1) / bn;
-    const long long cost = tiles * (BM + bn);
-    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+// ---- tile configuration ------------------------------------------------------------------
+// A small cost model picks the tile width BN, the CTA-pair mode cg and (weight gradient) the
+// split-K factor.  Unit of time: one 128 x 256 x 64 MMA step at full tensor rate (~0.2 us).
+//  * a k-step of a 128 x BN (x cg) tile costs BN/256, stretched when the operand bytes a CTA
+//    pulls from L2 per flop, proportional to (128 + BN/cg) / BN, exceed what L2 delivers
+//    (measured: 128 x 256 tiles with cg = 1 run at ~0.73 of the tensor rate);
+//  * the epilogue of a tile (~10 units at BN = 256) overlaps the next tile's main loop, so a
+//    tile costs max(main loop, epilogue) plus a fixed hand-off (larger across a CTA pair);
+//  * tiles are dealt round-robin to 148 / cg workers: few tiles cost whole waves;
+//  * split-K partials are written and read back once (fp32).
+struct RegionShape { int M, N, batch, ksteps; };
+struct TileCfg { int bn, cg, splits; double cost; };
+
+double estimate_cost(const RegionShape* r, int nr, int bn, int cg, int splits, double out_bytes) {
+  const double workers = 148.0 / cg;
+  const double step = (bn / 256.0) * fmax(1.0, 0.92 * (128.0 + (double)bn / cg) / bn);
+  const double epi = 10.0 * bn / 256.0;
+  double total = 0, ntiles = 0;
+  for (int i = 0; i < nr; ++i) {
+    if (r[i].M <= 0 || r[i].N <= 0) continue;
+    const double tiles = (double)((r[i].M + 128 * cg - 1) / (128 * cg)) * ((r[i].N + bn - 1) / bn) * r[i].batch * splits;
+    const double ks = (double)((r[i].ksteps + splits - 1) / splits);
+    total += tiles * (fmax(ks * step, epi) + (cg == 2 ? 3.5 : 2.0));
+    ntiles += tiles;
+  }
+  if (ntiles == 0) return 0;
+  double t = fmax(total / workers, ceil(ntiles / workers) * (total / ntiles));
+  if (splits > 1) t += 2.0 * splits * out_bytes / 6.4e12 / 0.2e-6;
+  return t;
+}
+
+TileCfg pick_tile(const RegionShape* r, int nr, bool b_n_major, int max_splits, double out_bytes) {
+  static const int max_cg = [] { const char* e = getenv("CAAT_TC_CG"); return e && atoi(e) == 1 ? 1 : 2; }();
+  TileCfg best{256, 1, 1, -1.0};
+  int min_ksteps = 1 << 30;
+  for (int i = 0; i < nr; ++i)
+    if (r[i].M > 0 && r[i].N > 0 && r[i].ksteps < min_ksteps) min_ksteps = r[i].ksteps;
+  for (int cg = 1; cg <= max_cg; ++cg) {
+    bool ok = true;
+    int nmin = 1 << 30;
+    for (int i = 0; i < nr; ++i) {
+      if (r[i].M <= 0 || r[i].N <= 0) continue;
+      if (cg == 2 && r[i].M < 256) ok = false;          // a pair needs two row blocks
+      if (r[i].N < nmin) nmin = r[i].N;
+    }
+    if (!ok) continue;
+    const int step = b_n_major ? 64 * cg : 32 * cg;    // N-major B: whole 64-column chunks per CTA
+    for (int bn = 256; bn >= 64 * cg; bn -= step) {
+      for (int splits = 1; splits <= max_splits; ++splits) {
+        if (splits > 1 && min_ksteps / splits < 8) break;
+        const double c = estimate_cost(r, nr, bn, cg, splits, out_bytes);
+        if (best.cost < 0 || c < best.cost * 0.995) best = TileCfg{bn, cg, splits, c};
+      }
+    }
   }
   return best;
 }
@@ -486,7 +618,7 @@ int sm_count() {
 }
 
 cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params& p, int kind, cudaStream_t st) {
-  const int stage_bytes = BM * BK * 2 + p.BN * BK * 2;
+  const int stage_bytes = BM * BK * 2 + (p.BN / p.cg) * BK * 2;
   int nst = (227 * 1024 - 2048 - 3 * kCBuf) / stage_bytes;
   if (nst > kMaxStages) nst = kMaxStages;
   if (nst < 2) return cudaErrorInvalidConfiguration;
@@ -494,23 +626,44 @@ cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params
   const size_t smem = (size_t)nst * stage_bytes + 3 * kCBuf + 1024 /*alignment slack*/ + (2 * nst + 4) * 8 + 16;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   p.status = device_status_word();
   if (!p.status) return cudaErrorUnknown;
-  int grid = p.tiles_total < sm_count() ? p.tiles_total : sm_count();
-  if (grid < 1) return cudaSuccess;
+  static const int dbg = [] { const char* e = getenv("CAAT_TC_DEBUG"); return e ? atoi(e) : 0; }();
+  p.debug = dbg;
+  static const bool verbose = getenv("CAAT_TC_VERBOSE") != nullptr;
+  if (verbose)
+    fprintf(stderr, "[caat tc] kind=%d BN=%d cg=%d splits=%d stages=%d tiles=%d (r0 M=%d N=%d b=%d)\n", kind, p.BN, p.cg,
+            p.splits, nst, p.tiles_total, p.r[0].M, p.r[0].N, p.r[0].batch);
+  const int workers_max = sm_count() / p.cg;
+  const int workers = p.tiles_total < workers_max ? p.tiles_total : workers_max;
+  if (workers < 1) return cudaSuccess;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(workers * p.cg));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = (unsigned)p.cg;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
   LaunchScope scope(kind, st);
-  tc_gemm_kernel<<<grid, kThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], p);
-  return cudaGetLastError();
+  if (p.cg == 2)
+    return cudaLaunchKernelEx(&cfg, tc_gemm_kernel<2>, maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], p);
+  return cudaLaunchKernelEx(&cfg, tc_gemm_kernel<1>, maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], p);
 }
 
 void finish_tiles(Params& p) {
   for (int g = 0; g < p.nregions; ++g) {
     Region& r = p.r[g];
-    r.mtiles = (r.M + BM - 1) / BM;
+    r.mtiles = (r.M + BM * p.cg - 1) / (BM * p.cg);
     r.ntiles = (r.N + p.BN - 1) / p.BN;
   }
   p.tiles_r0 = p.r[0].mtiles * p.r[0].ntiles * p.r[0].batch * p.splits;
@@ -529,26 +682,30 @@ cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* 
   CUtensorMap maps[4], cmaps[2];
   Params p{};
   const int n_sh = s.S, n_pr = s.h - s.S;
-  p.BN = pick_bn(n_pr > 0 && n_sh > 0 ? (n_sh < n_pr ? n_sh : n_pr) : (n_sh > 0 ? n_sh : n_pr), false);
+  const int ksteps = (s.K_r + BK - 1) / BK;
+  {
+    const RegionShape rs[2] = {{s.T, n_sh, 1, ksteps * s.t}, {s.T, n_pr, s.t, ksteps}};
+    const TileCfg c = pick_tile(rs, 2, false, 1, 0.0);
+    p.BN = c.bn; p.cg = c.cg;
+  }
   if (!make_map(&maps[0], Y, s.K_r, s.T, s.t, s.K_r, (long long)s.T * s.K_r, BK, BM)) return cudaErrorInvalidValue;
-  if (!make_map(&maps[1], W, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, BK, p.BN)) return cudaErrorInvalidValue;
+  if (!make_map(&maps[1], W, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, BK, p.BN / p.cg)) return cudaErrorInvalidValue;
   maps[2] = maps[0];
   maps[3] = maps[1];
   p.a_mn = 0; p.b_mn = 0; p.out_f32 = 0; p.splits = 1;
-  const int ksteps = (s.K_r + BK - 1) / BK;
   int g = 0;
   if (n_sh > 0) {
     Region& r = p.r[g++];
     r.nunits = 1;
     r.u[0] = Unit{0, 1, 0, 0, 0, 0, /*a_zb*/ 0, /*a_zq*/ 1, /*b_zb*/ 0, /*b_zq*/ 1, s.t, ksteps};
-    r.M = s.T; r.N = n_sh; r.batch = 1;
+    r.M = s.T; r.N = n_sh; r.batch = 1; r.b_slowest = 0;
     if (!make_cmap(&cmaps[g - 1], zs, n_sh, s.T, 1, s.S_hi, (long long)s.T * s.S_hi, false)) return cudaErrorInvalidValue;
   }
   if (n_pr > 0) {
     Region& r = p.r[g++];
     r.nunits = 1;
     r.u[0] = Unit{0, 1, 0, 0, 0, s.S, 1, 0, 1, 0, 1, ksteps};
-    r.M = s.T; r.N = n_pr; r.batch = s.t;
+    r.M = s.T; r.N = n_pr; r.batch = s.t; r.b_slowest = 1;
     if (!make_cmap(&cmaps[g - 1], static_cast<__nv_bfloat16*>(zp) + (s.S - s.S_lo), n_pr, s.T, s.t, s.P,
                    (long long)s.T * s.P, false))
       return cudaErrorInvalidValue;
@@ -564,7 +721,11 @@ cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* z
                             cudaStream_t st) {
   CUtensorMap maps[4], cmaps[2];
   Params p{};
-  p.BN = pick_bn(s.K_r, true);
+  {
+    const RegionShape rs[1] = {{s.T, s.K_r, s.t, (s.S + BK - 1) / BK + (s.h - s.S + BK - 1) / BK}};
+    const TileCfg c = pick_tile(rs, 1, true, 1, 0.0);
+    p.BN = c.bn; p.cg = c.cg;
+  }
   const int n_sh = s.S, n_pr = s.h - s.S;
   // B = W[m] as [h rows (contraction)][K_r contiguous (N)]: N-major, boxes of 64 (N) x 64 (K)
   if (!make_map(&maps[1], W, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, 64, BK)) return cudaErrorInvalidValue;
@@ -580,7 +741,7 @@ cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* z
   if (n_sh > 0) r.u[nu++] = Unit{0, 1, 0, 0, 0, 0, 0, 0, 1, 0, 1, (n_sh + BK - 1) / BK};
   if (n_pr > 0) r.u[nu++] = Unit{2, 1, s.S - s.S_lo, 0, s.S, 0, 1, 0, 1, 0, 1, (n_pr + BK - 1) / BK};
   r.nunits = nu;
-  r.M = s.T; r.N = s.K_r; r.batch = s.t;
+  r.M = s.T; r.N = s.K_r; r.batch = s.t; r.b_slowest = 1;
   if (!make_cmap(&cmaps[0], dY, s.K_r, s.T, s.t, s.K_r, (long long)s.T * s.K_r, false)) return cudaErrorInvalidValue;
   cmaps[1] = cmaps[0];
   p.nregions = 1;
@@ -588,20 +749,14 @@ cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* z
   return launch(maps, cmaps, p, CAAT_K_TC_DGRAD, st);
 }
 
-static int wgrad_splits(const RowparShapes& s, int BN) {
-  const long long mt = ((s.S + BM - 1) / BM) + ((s.h - s.S + BM - 1) / BM);
-  const long long tiles = mt * ((s.K_r + BN - 1) / BN) * s.t;
+static TileCfg wgrad_cfg(const RowparShapes& s) {
   const int ksteps = (s.T + BK - 1) / BK;
-  int splits = 1;
-  const int sms = 148;
-  if (tiles < sms) splits = (int)((sms + tiles - 1) / tiles);
-  if (splits > 16) splits = 16;
-  while (splits > 1 && ksteps / splits < 8) --splits;   // keep at least 8 stages per split
-  return splits;
+  const RegionShape rs[2] = {{s.S, s.K_r, s.t, ksteps}, {s.h - s.S, s.K_r, s.t, ksteps}};
+  return pick_tile(rs, 2, true, 16, (double)s.t * s.h * s.K_r * sizeof(float));
 }
 
 size_t tc_wgrad_splitk_bytes(const RowparShapes& s) {
-  const int splits = wgrad_splits(s, pick_bn(s.K_r, true));
+  const int splits = wgrad_cfg(s).splits;
   return splits > 1 ? (size_t)splits * s.t * s.h * s.K_r * sizeof(float) : 0;
 }
 
@@ -610,9 +765,10 @@ cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* z
                             void* splitk, size_t splitk_bytes, cudaStream_t st) {
   CUtensorMap maps[4], cmaps[2];
   Params p{};
-  p.BN = pick_bn(s.K_r, true);
+  const TileCfg wc = wgrad_cfg(s);
+  p.BN = wc.bn; p.cg = wc.cg;
   const int n_sh = s.S, n_pr = s.h - s.S;
-  const int splits = wgrad_splits(s, p.BN);
+  const int splits = wc.splits;
   const long long dw_elems = (long long)s.t * s.h * s.K_r;
   if (splits > 1 && splitk_bytes < (size_t)splits * dw_elems * sizeof(float)) return cudaErrorInvalidValue;
   // A = dZt as [T rows (contraction)][channels contiguous (M)]: M-major, boxes of 64 (M) x 64 (K)
@@ -632,7 +788,7 @@ cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* z
     Region& r = p.r[g++];
     r.nunits = 1;
     r.u[0] = Unit{0, 1, 0, 0, 0, 0, 0, 0, 1, 0, 1, ksteps};
-    r.M = n_sh; r.N = s.K_r; r.batch = s.t;
+    r.M = n_sh; r.N = s.K_r; r.batch = s.t; r.b_slowest = 0;   // the shared gradient panel serves all ranks at once
     if (!make_cmap(&cmaps[g - 1], out, s.K_r, n_sh, (long long)s.t * splits, s.K_r, (long long)s.h * s.K_r, true))
       return cudaErrorInvalidValue;
   }
@@ -640,7 +796,7 @@ cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* z
     Region& r = p.r[g++];
     r.nunits = 1;
     r.u[0] = Unit{2, 1, 0, s.S - s.S_lo, 0, 0, 1, 0, 1, 0, 1, ksteps};
-    r.M = n_pr; r.N = s.K_r; r.batch = s.t;
+    r.M = n_pr; r.N = s.K_r; r.batch = s.t; r.b_slowest = 1;
     if (!make_cmap(&cmaps[g - 1], out + (long long)s.S * s.K_r, s.K_r, n_pr, (long long)s.t * splits, s.K_r,
                    (long long)s.h * s.K_r, true))
       return cudaErrorInvalidValue;
