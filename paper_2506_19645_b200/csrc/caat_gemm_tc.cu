@@ -190,6 +190,16 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& p, int tile) {
   return c;
 }
 
+// Columns of B a tile really needs: the last tile of a ragged N (N-major B only) is narrowed to
+// whole 64-column chunks per CTA, so no padded columns are loaded or multiplied.
+__device__ __forceinline__ int tile_cols(const Params& p, const Region& r, int nt, int cg) {
+  if (!p.b_mn || (p.debug & 16)) return p.BN;
+  const int left = r.N - nt * p.BN;
+  if (left >= p.BN) return p.BN;
+  const int q = 64 * cg;
+  return (left + q - 1) / q * q;
+}
+
 // k-step range of a unit for a split
 __device__ __forceinline__ void split_range(const Params& p, const Unit& u, int split, int& k_begin, int& k_end) {
   if (p.splits == 1) { k_begin = 0; k_end = u.ksteps; return; }
@@ -301,7 +311,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       for (int tile = worker; tile < p.tiles_total && ok; tile += nworkers) {
         const TileCoord c = decode_tile(p, tile);
         const Region& r = p.r[c.region];
-        const int m0 = c.mt * BMT + (int)rank * BM, n0 = c.nt * p.BN + (int)(rank * bn_cta);
+        const uint32_t cols_cta = (uint32_t)tile_cols(p, r, c.nt, CG) / CG;    // B columns this CTA stages
+        const uint32_t b_tile_bytes = cols_cta * BK * 2;
+        const int m0 = c.mt * BMT + (int)rank * BM, n0 = c.nt * p.BN + (int)(rank * cols_cta);
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
           int kb, ke;
@@ -320,7 +332,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
                 continue;
               }
               if (rank == 0)
-                mbar_expect_tx(fb_local, (uint32_t)CG * (((p.debug & 4) ? 0u : a_bytes) + ((p.debug & 8) ? 0u : b_bytes)));
+                mbar_expect_tx(fb_local, (uint32_t)CG * (((p.debug & 4) ? 0u : a_bytes) + ((p.debug & 8) ? 0u : b_tile_bytes)));
               auto load = [&](uint32_t dst, const CUtensorMap* m, int x, int y, int z) {
                 if (CG == 2) tma_load_3d_pair(dst, m, x, y, z, fb); else tma_load_3d(dst, m, x, y, z, fb);
               };
@@ -336,7 +348,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
               } else if (!p.b_mn) {
                 load(sb, maps[u.mapB], u.bk0 + kk * BK, u.bn0 + n0, bz);
               } else {
-                for (int ch = 0; ch < (int)bn_cta / 64; ++ch)
+                for (int ch = 0; ch < (int)cols_cta / 64; ++ch)
                   load(sb + ch * (64 * BK * 2), maps[u.mapB], u.bn0 + n0 + ch * 64, u.bk0 + kk * BK, bz);
               }
               ++issued;
@@ -362,8 +374,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only when CG == 2)
     if (lane == 0 && rank == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-                             ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(BMT >> 4) << 24);
+      const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
+                              ((uint32_t)(BMT >> 4) << 24);
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
@@ -373,6 +385,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         if (!mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
+        const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(p, r, c.nt, CG) >> 3) << 17);
         uint32_t accumulate = 0;
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
@@ -562,17 +575,24 @@ bool make_cmap(CUtensorMap* m, const void* base, long long d0, long long d1, lon
 struct RegionShape { int M, N, batch, ksteps; };
 struct TileCfg { int bn, cg, splits; double cost; };
 
-double estimate_cost(const RegionShape* r, int nr, int bn, int cg, int splits, double out_bytes) {
+double estimate_cost(const RegionShape* r, int nr, int bn, int cg, int splits, double out_bytes, bool b_n_major) {
   const double workers = 148.0 / cg;
   const double step = (bn / 256.0) * fmax(1.0, 0.92 * (128.0 + (double)bn / cg) / bn);
   const double epi = 10.0 * bn / 256.0;
+  const double handoff = cg == 2 ? 3.5 : 2.0;
   double total = 0, ntiles = 0;
   for (int i = 0; i < nr; ++i) {
     if (r[i].M <= 0 || r[i].N <= 0) continue;
-    const double tiles = (double)((r[i].M + 128 * cg - 1) / (128 * cg)) * ((r[i].N + bn - 1) / bn) * r[i].batch * splits;
+    const double rows = (double)((r[i].M + 128 * cg - 1) / (128 * cg)) * r[i].batch * splits;
     const double ks = (double)((r[i].ksteps + splits - 1) / splits);
-    total += tiles * (fmax(ks * step, epi) + (cg == 2 ? 3.5 : 2.0));
-    ntiles += tiles;
+    const int full = r[i].N / bn, rest = r[i].N % bn;
+    total += rows * full * (fmax(ks * step, epi) + handoff);
+    ntiles += rows * full;
+    if (rest) {   // the last, ragged tile: an N-major B operand is narrowed to whole 64-column chunks
+      const double w = b_n_major ? (double)((rest + 64 * cg - 1) / (64 * cg) * (64 * cg)) / bn : 1.0;
+      total += rows * (fmax(ks * step * w, epi * w) + handoff);
+      ntiles += rows;
+    }
   }
   if (ntiles == 0) return 0;
   double t = fmax(total / workers, ceil(ntiles / workers) * (total / ntiles));
@@ -599,7 +619,7 @@ TileCfg pick_tile(const RegionShape* r, int nr, bool b_n_major, int max_splits, 
     for (int bn = 256; bn >= 64 * cg; bn -= step) {
       for (int splits = 1; splits <= max_splits; ++splits) {
         if (splits > 1 && min_ksteps / splits < 8) break;
-        const double c = estimate_cost(r, nr, bn, cg, splits, out_bytes);
+        const double c = estimate_cost(r, nr, bn, cg, splits, out_bytes, b_n_major);
         if (best.cost < 0 || c < best.cost * 0.995) best = TileCfg{bn, cg, splits, c};
       }
     }

@@ -64,8 +64,13 @@ struct StageGeom {
 
 // ------------------------------------------------------------------ forward
 // stage buffers: a = R rows [TY, h], b = zp rows [TY, P], c = zs rows [TY, S_hi] (rank 0 only)
+// resident CTAs per SM the launch bounds ask for: one chunk per thread in small CTAs leaves ~85
+// registers per thread at three CTAs, two chunks per thread 128 registers at two CTAs
+template <int CPT, int MAXT>
+struct MinBlocks { static constexpr int value = MAXT <= 256 ? (CPT == 1 ? 3 : 2) : (CPT == 1 ? 2 : 1); };
+
 template <typename T_, int CPT, bool LN, int MAXT>
-__global__ void __launch_bounds__(MAXT, (CPT == 1 || MAXT <= 256) ? 2 : 1)
+__global__ void __launch_bounds__(MAXT, MinBlocks<CPT, MAXT>::value)
 rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
@@ -245,7 +250,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
 // ------------------------------------------------------------------ backward
 // stage buffers: a = dX rows, b = Hn rows, c = dHn rows (when given)
 template <typename T_, int CPT, bool LN, int MAXT>
-__global__ void __launch_bounds__(MAXT, (CPT == 1 || MAXT <= 256) ? 2 : 1)
+__global__ void __launch_bounds__(MAXT, MinBlocks<CPT, MAXT>::value)
 rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
@@ -574,7 +579,8 @@ cudaError_t launch_fwd_staged_t(const RowFwdArgs& a, const RowGeom& g, const Sta
     e = set_smem(rows_forward_staged<T_, CPT_, LN, MAXT_>, sg.smem);                                            \
     if (e == cudaSuccess) rows_forward_staged<T_, CPT_, LN, MAXT_><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);       \
   } while (0)
-  if (g.CPT == 1) CAAT_LAUNCH(1, 512);
+  if (g.CPT == 1 && threads <= 256) CAAT_LAUNCH(1, 256);
+  else if (g.CPT == 1) CAAT_LAUNCH(1, 512);
   else if (g.CPT == 2 && threads <= 256) CAAT_LAUNCH(2, 256);
   else if (g.CPT == 2) CAAT_LAUNCH(2, 512);
   else if (g.CPT == 4) CAAT_LAUNCH(4, 512);
@@ -595,7 +601,8 @@ cudaError_t launch_bwd_staged_t(const RowBwdArgs& a, const RowGeom& g, const Sta
     e = set_smem(rows_backward_staged<T_, CPT_, LN, MAXT_>, sg.smem);                                            \
     if (e == cudaSuccess) rows_backward_staged<T_, CPT_, LN, MAXT_><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);       \
   } while (0)
-  if (g.CPT == 1) CAAT_LAUNCH(1, 512);
+  if (g.CPT == 1 && threads <= 256) CAAT_LAUNCH(1, 256);
+  else if (g.CPT == 1) CAAT_LAUNCH(1, 512);
   else if (g.CPT == 2 && threads <= 256) CAAT_LAUNCH(2, 256);
   else if (g.CPT == 2) CAAT_LAUNCH(2, 512);
   else if (g.CPT == 4) CAAT_LAUNCH(4, 512);
@@ -610,8 +617,9 @@ constexpr size_t kSmemPerSm = 227 * 1024;
 int ctas_per_sm(const RowGeom& g) {
   const int threads = g.TX * g.TY;
   if (g.CPT != 1) return threads <= 256 ? 2 : 1;   // 128 registers per thread
-  int n = 1024 / threads;                           // 64 registers per thread
-  return n < 1 ? 1 : (n > 8 ? 8 : n);
+  if (threads > 256) return 2;                      // 64 registers per thread
+  int n = 65536 / (threads * 80);                   // 80 registers per thread
+  return n < 1 ? 1 : (n > 6 ? 6 : n);
 }
 
 }  // namespace
