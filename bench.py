@@ -182,7 +182,31 @@ class BlockRunner:
         return n + sum(v.numel() * v.element_size() for v in self.out.values())
 
 
-def time_steps(runner, steps, dist_on):
+def capture_step(runner):
+    """One step captured into a CUDA graph (launch-bound workloads: a decode step is tens of
+    microseconds).  Returns (graph, kernels per step) or (None, 0) when capture is not possible."""
+    from paper_2506_19645_b200 import caat
+    try:
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            runner.step()                      # warm the side stream
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        l0 = caat.kernel_launches()
+        with torch.cuda.graph(g, stream=side):
+            runner.step()
+        per_step = caat.kernel_launches() - l0
+        g.replay()
+        torch.cuda.synchronize()
+        return g, int(per_step)
+    except Exception as ex:  # noqa: BLE001
+        sys.stderr.write(f"bench: CUDA graph capture failed ({ex}); timing eager launches\n")
+        return None, 0
+
+
+def time_steps(runner, steps, dist_on, graph=None):
     """Device time of exactly `steps` steps (ms), CUDA events on the launching stream."""
     torch.cuda.synchronize()
     if dist_on:
@@ -190,7 +214,10 @@ def time_steps(runner, steps, dist_on):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
-        runner.step()
+        if graph is not None:
+            graph.replay()
+        else:
+            runner.step()
     e1.record()
     torch.cuda.synchronize()
     if dist_on:
@@ -282,11 +309,16 @@ def run_cuda(args):
     torch.cuda.synchronize()
     assert runner.ctx.last_device_status() == caat.CAAT_OK
 
+    # launch-bound steps (decode: tens of microseconds) are replayed from a CUDA graph
+    graph, per_step = (None, 0)
+    probe = time_steps(runner, 5, False) / 5
+    if probe < 0.25 and not args.no_graph:
+        graph, per_step = capture_step(runner)
     sampler = ClockSampler(local)
     sampler.start()
     l0 = caat.kernel_launches()
-    ms = time_steps(runner, args.steps, dist_on)
-    launches = caat.kernel_launches() - l0
+    ms = time_steps(runner, args.steps, dist_on, graph)
+    launches = per_step * args.steps if graph is not None else caat.kernel_launches() - l0
     # second pass of the same K steps with CUDA events around every kernel (per-kernel device times)
     caat.profile_begin(max(1024, launches + 64))
     ms_prof = time_steps(runner, args.steps, dist_on)
@@ -345,6 +377,7 @@ def run_cuda(args):
             "config": {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p,
                        "S": w.S, "passes": "forward+backward" if w.backward else "forward",
                        "private_scale": "sqrt(t)", "norm": "rmsnorm", "parallelism": f"replicas x{world}",
+                       "launch": "cuda graph replay" if graph is not None else "eager",
                        "l2": f"inputs+outputs touched per step {runner.touched_bytes() / 1e6:.0f} MB > 126 MB L2"},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "roofline": roof, "kernels": kernels,
             "path_roofline": {"flops_per_step": fl, "bytes_per_step": by, "roofline_ms": t_roof * 1e3,
@@ -428,6 +461,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the other workloads' tokens/s")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-graph", action="store_true", help="never replay launch-bound steps from a CUDA graph")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling on a small case)")
     args = ap.parse_args()
     if args.steps < 1:

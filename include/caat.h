@@ -74,8 +74,11 @@ typedef enum {
   CAAT_OPT_PRIVATE_SCALE = 2,   /* alpha; default sqrt(t); 1 switches scaling off       */
   CAAT_OPT_SHARED_CHANNELS = 3, /* override S with an explicit integer in [0, h]        */
   CAAT_OPT_GEMM = 4,            /* 0 = automatic (default), 1 = force the CUDA-core GEMM */
-  CAAT_OPT_ROWS = 5             /* 0 = automatic (default: bulk-copy staged row kernels),
+  CAAT_OPT_ROWS = 5,            /* 0 = automatic (default: bulk-copy staged row kernels),
                                    1 = force the plain-load row kernels                  */
+  CAAT_OPT_DECODE = 6           /* 0 = automatic (default: forward calls with at most 64 tokens
+                                   stream the weights with swapped GEMM operands),
+                                   1 = always use the large-batch forward                */
 } caat_option;
 
 /* Creates a context for hidden size h, MLP width ffn, t ranks, synchronisation

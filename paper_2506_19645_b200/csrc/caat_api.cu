@@ -37,15 +37,27 @@ LaunchScope::~LaunchScope() {
 }
 
 unsigned int* device_status_word() {
-  unsigned int* p = nullptr;
-  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word) != cudaSuccess) return nullptr;
-  return p;
+  // looked up once per device (the lookup is not a stream operation; caching it keeps launches
+  // free of runtime queries, which also matters inside a stream capture)
+  static unsigned int* cache[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (cache[dev] == nullptr) {
+    unsigned int* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word) != cudaSuccess) return nullptr;
+    cache[dev] = p;
+  }
+  return cache[dev];
 }
 
 static caat_status cuda_fail(cudaError_t e) {
   std::strncpy(g_cuda_err, cudaGetErrorString(e), sizeof(g_cuda_err) - 1);
   g_cuda_err[sizeof(g_cuda_err) - 1] = 0;
   return CAAT_ECUDA;
+}
+
+static size_t decode_planes_bytes(const caat_ctx* ctx, int tokens) {
+  return align_up((size_t)kDecodeMaxSplits * ctx->t * tokens * ctx->h * sizeof(float), 256);
 }
 
 Scratch scratch_layout(const caat_ctx* ctx, int K_r, int tokens, int backward) {
@@ -59,6 +71,9 @@ Scratch scratch_layout(const caat_ctx* ctx, int K_r, int tokens, int backward) {
   off = align_up(off + (size_t)tokens * s.S_hi * e, 256);
   s.zp_off = off;
   off = align_up(off + (size_t)ctx->t * tokens * s.P * e, 256);
+  s.zt_off = off;
+  if (!backward && tokens <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r))   // two layers' planes
+    off = align_up(off + 2 * decode_planes_bytes(ctx, tokens), 256);
   if (backward) {
     const size_t rows = (size_t)rows_backward_partial_rows(ctx->h, tokens, ctx->dtype);
     s.dgpart_off = off;
@@ -106,6 +121,22 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
   const size_t e = elem_size(ctx->dtype);
   cudaError_t ce;
 
+  if (T <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r)) {
+    // few tokens (decode): the weights dominate the traffic; stream them with swapped operands and
+    // let the row kernel form the rank sum from fp32 per-rank partials
+    float* zt = reinterpret_cast<float*>(wsb + L.zt_off);
+    const int splits = tc_decode_splits(K_r, K_r, T);
+    const DecodeProblem pr{K_r, Y, W, zt, splits};
+    ce = launch_tc_forward_decode(t, T, h, &pr, 1, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    RowPartArgs a{};
+    a.L[0] = PartialLayer{zt, splits, gamma, beta, Hn, X, rstd, mean};
+    a.nlayers = 1; a.R = R; a.t = t; a.T = T; a.h = h; a.S = S;
+    a.alpha = (float)ctx->alpha; a.eps = (float)ctx->eps; a.norm = ctx->norm;
+    ce = launch_rows_forward_partials(a, ctx->dtype, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    return CAAT_OK;
+  }
   if (tc_gemm_usable(ctx, K_r)) {
     RowparShapes sh{t, T, h, K_r, S, L.S_lo, L.S_hi, L.P};
     ce = launch_tc_forward(sh, Y, W, zs, zp, st);
@@ -213,7 +244,7 @@ caat_status caat_create(int h, int ffn, int t, double p, caat_dtype dtype, caat_
   c->h = h; c->ffn = ffn; c->t = t; c->p = p; c->dtype = dtype;
   c->S = (int)std::floor((double)h * p);   // Eq. A3: l < floor(h p) is shared
   c->alpha = std::sqrt((double)t);         // Section 4: private channels times sqrt(r)
-  c->norm = 0; c->eps = 1e-5; c->force_simt = 0; c->direct_rows = 0;
+  c->norm = 0; c->eps = 1e-5; c->force_simt = 0; c->direct_rows = 0; c->no_decode = 0;
   *out = c;
   return CAAT_OK;
 }
@@ -237,6 +268,9 @@ caat_status caat_set_option(caat_ctx* ctx, caat_option opt, double value) {
     case CAAT_OPT_GEMM:
       if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
       ctx->force_simt = (int)value; return CAAT_OK;
+    case CAAT_OPT_DECODE:
+      if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
+      ctx->no_decode = (int)value; return CAAT_OK;
     case CAAT_OPT_ROWS:
       if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
       ctx->direct_rows = (int)value; return CAAT_OK;
@@ -310,6 +344,39 @@ caat_status caat_block_forward(const caat_ctx* ctx, int tokens, const void* Y_at
                                float* rstd1, float* mean1, void* Hn2, void* X2, float* rstd2, float* mean2,
                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
   // Two reduces per block (Appendix C): attention-out, then MLP-down on the new residual stream.
+  if (ctx && tokens >= 1 && tokens <= kDecodeMaxTokens && !ctx->no_decode &&
+      tc_gemm_usable(ctx, ctx->h / ctx->t) && tc_gemm_usable(ctx, ctx->ffn / ctx->t)) {
+    // few tokens: the two layers' GEMMs do not depend on each other, so both weight streams run in
+    // ONE launch, and one row kernel walks both layers of a (token, rank) row
+    caat_status s = check_common(ctx, CAAT_MLP_DOWN, tokens);
+    if (s != CAAT_OK) return s;
+    if (!Y_attn || !W_o || !Y_mlp || !W_down || !R0 || !gamma1 || !gamma2 || !Hn1 || !X1 || !rstd1 || !Hn2 || !X2 || !rstd2)
+      return CAAT_EINVAL;
+    if (ctx->norm == 1 && (!mean1 || !mean2)) return CAAT_EINVAL;
+    const void* ptrs[] = {Y_attn, W_o, Y_mlp, W_down, R0, gamma1, beta1, gamma2, beta2, Hn1, X1, rstd1, mean1,
+                          Hn2, X2, rstd2, mean2, workspace};
+    for (const void* p : ptrs)
+      if (p && !aligned16(p)) return CAAT_EALIGN;
+    const int ka = ctx->h / ctx->t, km = ctx->ffn / ctx->t;
+    const Scratch L = scratch_layout(ctx, km, tokens, 0);
+    if (!workspace || workspace_bytes < L.total) return CAAT_EWORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    float* zt1 = reinterpret_cast<float*>(static_cast<char*>(workspace) + L.zt_off);
+    float* zt2 = reinterpret_cast<float*>(static_cast<char*>(workspace) + L.zt_off + decode_planes_bytes(ctx, tokens));
+    const int kmin = ka < km ? ka : km;
+    const int sp1 = tc_decode_splits(ka, kmin, tokens), sp2 = tc_decode_splits(km, kmin, tokens);
+    const DecodeProblem pr[2] = {{ka, Y_attn, W_o, zt1, sp1}, {km, Y_mlp, W_down, zt2, sp2}};
+    cudaError_t ce = launch_tc_forward_decode(ctx->t, tokens, ctx->h, pr, 2, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    RowPartArgs a{};
+    a.L[0] = PartialLayer{zt1, sp1, gamma1, beta1, Hn1, X1, rstd1, mean1};
+    a.L[1] = PartialLayer{zt2, sp2, gamma2, beta2, Hn2, X2, rstd2, mean2};
+    a.nlayers = 2; a.R = R0; a.t = ctx->t; a.T = tokens; a.h = ctx->h; a.S = ctx->S;
+    a.alpha = (float)ctx->alpha; a.eps = (float)ctx->eps; a.norm = ctx->norm;
+    ce = launch_rows_forward_partials(a, ctx->dtype, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    return CAAT_OK;
+  }
   caat_status s = caat_rowpar_forward(ctx, CAAT_ATTN_OUT, tokens, Y_attn, W_o, R0, gamma1, beta1, Hn1, X1, rstd1,
                                       mean1, workspace, workspace_bytes, cuda_stream);
   if (s != CAAT_OK) return s;

@@ -52,6 +52,8 @@ struct Region {          // a family of output tiles with the same operand wirin
   int M, N, batch;       // valid output extents per batch
   int mtiles, ntiles;    // the output goes through the region's own tensor map (TMA store);
                          // its z coordinate is split * batch + b
+  float* out_t;          // transposed direct-store output (decode), else unused
+  int splits;            // split-K factor of this region's tiles (set by finish_tiles from Params::splits when 0)
   int b_slowest;         // tile order: 1 = rank index slowest (a rank's weights / activations stay
 };                       // hot in L2 while its row tiles stream), 0 = row tile slowest
 
@@ -62,6 +64,8 @@ struct Params {
   int nstages;
   int a_mn, b_mn;        // 1: operand is MN-major in global memory
   int out_f32;
+  int out_transposed;    // 1: D is [channels x tokens]; store fp32 straight to the region's out_t[z][token][channel]
+  long long out_t_ld;    // channels per token row of out_t
   int cg;                // CTAs per tile: 1, or 2 (tcgen05 cta_group::2, clusters of two)
   int splits;            // split-K factor (only with a single unit and Q == 1)
   int tiles_r0;          // tiles of region 0 (including splits)
@@ -179,7 +183,7 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& p, int tile) {
   int rem = tile - (c.region ? p.tiles_r0 : 0);
   const Region& r = p.r[c.region];
   c.nt = rem % r.ntiles; rem /= r.ntiles;
-  c.split = rem % p.splits; rem /= p.splits;
+  c.split = rem % r.splits; rem /= r.splits;
   if (r.b_slowest) {
     c.mt = rem % r.mtiles; rem /= r.mtiles;
     c.b = rem;
@@ -201,9 +205,9 @@ __device__ __forceinline__ int tile_cols(const Params& p, const Region& r, int n
 }
 
 // k-step range of a unit for a split
-__device__ __forceinline__ void split_range(const Params& p, const Unit& u, int split, int& k_begin, int& k_end) {
-  if (p.splits == 1) { k_begin = 0; k_end = u.ksteps; return; }
-  const int per = (u.ksteps + p.splits - 1) / p.splits;
+__device__ __forceinline__ void split_range(int splits, const Unit& u, int split, int& k_begin, int& k_end) {
+  if (splits == 1) { k_begin = 0; k_end = u.ksteps; return; }
+  const int per = (u.ksteps + splits - 1) / splits;
   k_begin = split * per;
   k_end = k_begin + per < u.ksteps ? k_begin + per : u.ksteps;
   if (k_begin > k_end) k_begin = k_end;
@@ -317,7 +321,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
           int kb, ke;
-          split_range(p, u, c.split, kb, ke);
+          split_range(r.splits, u, c.split, kb, ke);
           for (int q = 0; q < u.Q && ok; ++q) {
             const int az = c.b * u.a_zb + q * u.a_zq, bz = c.b * u.b_zb + q * u.b_zq;
             for (int kk = kb; kk < ke; ++kk) {
@@ -390,7 +394,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
           int kb, ke;
-          split_range(p, u, c.split, kb, ke);
+          split_range(r.splits, u, c.split, kb, ke);
           for (int q = 0; q < u.Q && ok; ++q) {
             for (int kk = kb; kk < ke; ++kk) {
               if (!mbar_wait(full0 + 8u * stage, phase, abort_flag)) { ok = false; break; }
@@ -433,7 +437,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       int total_k = 0;
       for (int ui = 0; ui < r.nunits; ++ui) {
         int kb, ke;
-        split_range(p, r.u[ui], c.split, kb, ke);
+        split_range(r.splits, r.u[ui], c.split, kb, ke);
         total_k += (ke - kb) * r.u[ui].Q;
       }
       if (!mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag)) { ok = false; break; }
@@ -447,6 +451,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       const int sub = p.out_f32 ? 16 : 32;
       const int rr = quarter * 32 + lane;                 // row of the tile this thread holds
       const uint32_t sw = (uint32_t)((rr >> 1) & 3);      // 64-byte swizzle: chunk ^= (row / 2) % 4
+      if (p.out_transposed) {
+        // swap-AB (decode): TMEM lane = output channel, column = token.  For a fixed token the 32
+        // lanes of a warp hold 32 consecutive channels: plain 128-byte coalesced stores.
+        const long long chan = (long long)m0 + rr;
+        for (int cc = 0; cc < p.BN && n0 + cc < r.N; cc += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols + cc), v);
+          tmem_ld_wait();
+          if (chan < r.M) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int tok = n0 + cc + e;
+              if (tok < r.N) r.out_t[((long long)zc * r.N + tok) * p.out_t_ld + chan] = total_k == 0 ? 0.f : __uint_as_float(v[e]);
+            }
+          }
+        }
+      } else
       for (int cc = 0; cc < p.BN && n0 + cc < r.N && !(p.debug & 2); cc += sub) {
         uint32_t v[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols + cc);
@@ -685,9 +706,10 @@ void finish_tiles(Params& p) {
     Region& r = p.r[g];
     r.mtiles = (r.M + BM * p.cg - 1) / (BM * p.cg);
     r.ntiles = (r.N + p.BN - 1) / p.BN;
+    if (r.splits < 1) r.splits = p.splits < 1 ? 1 : p.splits;
   }
-  p.tiles_r0 = p.r[0].mtiles * p.r[0].ntiles * p.r[0].batch * p.splits;
-  p.tiles_total = p.tiles_r0 + (p.nregions > 1 ? p.r[1].mtiles * p.r[1].ntiles * p.r[1].batch * p.splits : 0);
+  p.tiles_r0 = p.r[0].mtiles * p.r[0].ntiles * p.r[0].batch * p.r[0].splits;
+  p.tiles_total = p.tiles_r0 + (p.nregions > 1 ? p.r[1].mtiles * p.r[1].ntiles * p.r[1].batch * p.r[1].splits : 0);
 }
 
 }  // namespace
@@ -732,6 +754,54 @@ cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* 
   }
   if (g == 1) cmaps[1] = cmaps[0];
   p.nregions = g;
+  finish_tiles(p);
+  return launch(maps, cmaps, p, CAAT_K_TC_FORWARD, st);
+}
+
+// ---- decode forward (few tokens): zt[m][i][l] = sum_k W[m][l][k] Y[m][i][k], fp32, for ALL channels.
+// The operands are swapped (weights on the 128-row side, tokens on the narrow side) so that a tile
+// streams 128 x K_r weights however few tokens there are; every (rank, 128-channel block) is a tile,
+// which spreads the weight stream over all SMs.  The rank sum of the shared channels is left to the
+// row kernel (the partials are tiny at these token counts).
+int tc_decode_splits(int K_r, int K_r_min, int T) {
+  // Work items are (rank, 128-channel block, split).  Splitting the longer layer's contraction until its
+  // items are about as long as the shorter layer's makes the round-robin deal even; the fp32 partial
+  // planes this adds (t * splits * T * h * 4 bytes) are kept near a tenth of the layer's weight bytes.
+  const int ks = (K_r + BK - 1) / BK, ks_min = (K_r_min + BK - 1) / BK;
+  int sp = (ks + ks_min / 2) / (ks_min > 0 ? ks_min : 1);
+  const int cap_traffic = K_r / (20 * T);
+  if (sp > cap_traffic) sp = cap_traffic;
+  if (sp > kDecodeMaxSplits) sp = kDecodeMaxSplits;
+  if (sp > ks / 2) sp = ks / 2;
+  return sp < 1 ? 1 : sp;
+}
+
+cudaError_t launch_tc_forward_decode(int t, int T, int h, const DecodeProblem* pr, int n, cudaStream_t st) {
+  if (n < 1 || n > 2) return cudaErrorInvalidValue;
+  CUtensorMap maps[4], cmaps[2];
+  Params p{};
+  p.BN = (T + 31) / 32 * 32;
+  if (p.BN > 256) return cudaErrorInvalidValue;
+  p.cg = 1;
+  p.a_mn = 0; p.b_mn = 0; p.out_f32 = 1; p.splits = 1;
+  p.out_transposed = 1; p.out_t_ld = h;
+  // longer contraction first: round-robin dealing then fills the tail with the short items
+  int order[2] = {0, 1};
+  if (n == 2 && pr[1].K_r > pr[0].K_r) { order[0] = 1; order[1] = 0; }
+  for (int g = 0; g < n; ++g) {
+    const DecodeProblem& q = pr[order[g]];
+    if (!make_map(&maps[2 * g], q.W, q.K_r, h, t, q.K_r, (long long)h * q.K_r, BK, BM)) return cudaErrorInvalidValue;
+    if (!make_map(&maps[2 * g + 1], q.Y, q.K_r, T, t, q.K_r, (long long)T * q.K_r, BK, p.BN)) return cudaErrorInvalidValue;
+    Region& r = p.r[g];
+    r.nunits = 1;
+    r.u[0] = Unit{2 * g, 2 * g + 1, 0, 0, 0, 0, 1, 0, 1, 0, 1, (q.K_r + BK - 1) / BK};
+    r.M = h; r.N = T; r.batch = t; r.b_slowest = 1;
+    r.out_t = q.zt;
+    r.splits = q.splits;
+  }
+  if (n == 1) { maps[2] = maps[0]; maps[3] = maps[1]; }
+  cmaps[0] = maps[0]; cmaps[1] = maps[0];          // unused: the epilogue stores directly
+  p.nregions = n;
   finish_tiles(p);
   return launch(maps, cmaps, p, CAAT_K_TC_FORWARD, st);
 }

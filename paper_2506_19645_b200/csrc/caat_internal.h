@@ -17,6 +17,7 @@ struct caat_ctx {
   double eps;
   int force_simt;  // CAAT_OPT_GEMM
   int direct_rows; // CAAT_OPT_ROWS
+  int no_decode;   // CAAT_OPT_DECODE
 };
 
 namespace caat {
@@ -39,6 +40,7 @@ struct Scratch {
   size_t zs_off, zp_off;   // forward: Zt shared / private.  backward: dZt shared / private
   size_t dgpart_off, dbpart_off;  // backward: [rows, h] fp32 partial norm-parameter gradients
   size_t splitk_off, splitk_bytes;  // backward: split-K partials of the weight gradient
+  size_t zt_off;           // forward, few tokens: fp32 per-rank partials [t, T, h]
   size_t total;
 };
 
@@ -82,6 +84,13 @@ cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* z
 cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* zp, const void* Y, float* dW,
                             void* splitk, size_t splitk_bytes, cudaStream_t st);
 size_t tc_wgrad_splitk_bytes(const RowparShapes& s);
+// decode (few tokens): per-rank fp32 partials for all channels, zt[t, T, h]
+constexpr int kDecodeMaxTokens = 64;
+// zt[split * t + m][i][l] = partial of sum_k W[m][l][k] Y[m][i][k]; one or two layers in one launch
+struct DecodeProblem { int K_r; const void* Y; const void* W; float* zt; int splits; };
+int tc_decode_splits(int K_r, int K_r_min, int T);
+constexpr int kDecodeMaxSplits = 4;
+cudaError_t launch_tc_forward_decode(int t, int T, int h, const DecodeProblem* pr, int n, cudaStream_t st);
 
 // ---- row kernels ------------------------------------------------------------
 struct RowFwdArgs {
@@ -96,6 +105,18 @@ struct RowFwdArgs {
 // whenever a ring of at least two stages fits in shared memory.
 cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
 cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st);
+// forward row work from fp32 partial planes (decode); with two layers the second layer's residual is
+// the first layer's new residual stream (as stored), both layers in one launch
+struct PartialLayer { const float* zt; int splits; const void* gamma; const void* beta; void* Hn; void* X; float* rstd; float* mean; };
+struct RowPartArgs {
+  PartialLayer L[2];
+  int nlayers;
+  const void* R;
+  int t, T, h, S;
+  float alpha, eps;
+  int norm;
+};
+cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype, cudaStream_t st);
 bool rows_staged_usable(int h, int t, int S_lo, int S_hi, caat_dtype dtype, bool backward);
 
 struct RowBwdArgs {

@@ -336,6 +336,93 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
   }
 }
 
+// ------------------------------------------------------------------ forward from fp32 partial planes (decode)
+// One CTA per (token, rank).  zt holds fp32 partial outputs [splits * t, T, h] for ALL channels (plane
+// z = split * t + rank).  Shared channels: sum of every plane, z ascending; private channels: sum over
+// the splits of this rank's planes, times alpha.  Every rank's CTA forms the shared sum for itself (a few
+// kilobytes, L2 hits), so no CTA waits for another.  With two layers the second one's residual is the
+// first one's new residual stream as stored (rounded to the storage type).
+template <typename T_, bool LN>
+__global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPartArgs a) {
+  using V_ = VT<T_>;
+  using raw = typename V_::raw;
+  constexpr int V = V_::N;
+  constexpr int ES = sizeof(T_);
+  extern __shared__ float sm[];
+  float* hrow = sm;                       // [h] the new residual stream of this row, fp32
+  float* red = sm + a.h;                  // reduction scratch
+  int par = 0;
+  const int i = blockIdx.x, m = blockIdx.y;
+  const long long row = (long long)m * a.T + i;
+  const long long plane = (long long)a.T * a.h;
+  const float inv_h = 1.0f / (float)a.h;
+  for (int layer = 0; layer < a.nlayers; ++layer) {
+    const PartialLayer& L = a.L[layer];
+    const int nplanes = L.splits * a.t;
+    float st[1] = {0.f};
+    for (int c = threadIdx.x * V; c < a.h; c += blockDim.x * V) {
+      float r[V], z[V], hn[V];
+      if (layer == 0) {
+        V_::unpack(ldg<raw>(static_cast<const char*>(a.R) + (row * a.h + c) * ES), r);
+      } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) r[e] = V_::round(hrow[c + e]);
+      }
+#pragma unroll
+      for (int e = 0; e < V; ++e) z[e] = 0.f;
+      const float* base = L.zt + (long long)i * a.h + c;
+      const bool shared_chunk = c + V <= a.S;          // the partition is a multiple of 8 on this path
+      const int z0 = shared_chunk ? 0 : m, zstep = shared_chunk ? 1 : a.t;
+      const int nz = shared_chunk ? nplanes : L.splits;
+#pragma unroll 8
+      for (int q = 0; q < nz; ++q) {
+        const float* pz = base + (long long)(z0 + q * zstep) * plane;
+#pragma unroll
+        for (int e = 0; e < V; e += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(pz + e);
+          z[e] += v.x; z[e + 1] += v.y; z[e + 2] += v.z; z[e + 3] += v.w;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < V; ++e) {
+        hn[e] = (shared_chunk ? z[e] : a.alpha * z[e]) + r[e];
+        st[0] = LN ? st[0] + hn[e] : fmaf(hn[e], hn[e], st[0]);
+      }
+      if (layer > 0) __syncwarp();
+#pragma unroll
+      for (int e = 0; e < V; ++e) hrow[c + e] = hn[e];
+      stg<raw>(static_cast<char*>(L.Hn) + (row * a.h + c) * ES, V_::pack(hn));
+    }
+    row_reduce_sync<1>(st, red, par);
+    float mu = 0.f, rs;
+    if (LN) {
+      mu = st[0] * inv_h;
+      float sq[1] = {0.f};
+      for (int c = threadIdx.x * V; c < a.h; c += blockDim.x * V)
+#pragma unroll
+        for (int e = 0; e < V; ++e) { const float d = hrow[c + e] - mu; sq[0] = fmaf(d, d, sq[0]); }
+      row_reduce_sync<1>(sq, red, par);
+      rs = rsqrtf(fmaf(sq[0], inv_h, a.eps));
+    } else {
+      rs = rsqrtf(fmaf(st[0], inv_h, a.eps));
+    }
+    for (int c = threadIdx.x * V; c < a.h; c += blockDim.x * V) {
+      float g[V], b[V], x[V];
+      V_::unpack(ldg<raw>(static_cast<const char*>(L.gamma) + (long long)c * ES), g);
+#pragma unroll
+      for (int e = 0; e < V; ++e) b[e] = 0.f;
+      if (LN && L.beta) V_::unpack(ldg<raw>(static_cast<const char*>(L.beta) + (long long)c * ES), b);
+#pragma unroll
+      for (int e = 0; e < V; ++e) x[e] = LN ? fmaf(hrow[c + e] - mu, rs * g[e], b[e]) : hrow[c + e] * (rs * g[e]);
+      stg<raw>(static_cast<char*>(L.X) + (row * a.h + c) * ES, V_::pack(x));
+    }
+    if (threadIdx.x == 0) {
+      L.rstd[row] = rs;
+      if (LN && L.mean) L.mean[row] = mu;
+    }
+  }
+}
+
 // out[l] = sum over `rows` partial rows, fixed order: 32 row lanes then a serial combine.
 __global__ void __launch_bounds__(1024) reduce_partials_kernel(const float* __restrict__ part, float* __restrict__ out,
                                                                int rows, int h) {
@@ -383,6 +470,24 @@ cudaError_t launch_bwd_t(const RowBwdArgs& a, const RowGeom& g, int rows, cudaSt
 }
 
 }  // namespace
+
+cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype, cudaStream_t st) {
+  const int V = dtype == CAAT_BF16 ? 8 : 4;
+  int threads = round_up(a.h / V, 32);               // one chunk per thread when the row allows
+  if (threads > 512) threads = 512;
+  if (threads < 32) threads = 32;
+  const dim3 grid(a.T, a.t);
+  const size_t smem = (size_t)a.h * sizeof(float) + 2 * 16 * 2 * sizeof(float);
+  LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
+  if (dtype == CAAT_BF16) {
+    if (a.norm == 1) rows_forward_partials_kernel<__nv_bfloat16, true><<<grid, threads, smem, st>>>(a);
+    else rows_forward_partials_kernel<__nv_bfloat16, false><<<grid, threads, smem, st>>>(a);
+  } else {
+    if (a.norm == 1) rows_forward_partials_kernel<float, true><<<grid, threads, smem, st>>>(a);
+    else rows_forward_partials_kernel<float, false><<<grid, threads, smem, st>>>(a);
+  }
+  return cudaGetLastError();
+}
 
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype) {
   const RowGeom g = row_geometry(h, dtype);

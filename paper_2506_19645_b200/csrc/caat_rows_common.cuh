@@ -18,6 +18,7 @@ struct VT<float> {
     f[0] = r.x; f[1] = r.y; f[2] = r.z; f[3] = r.w;
   }
   static __device__ __forceinline__ raw pack(const float* f) { return make_float4(f[0], f[1], f[2], f[3]); }
+  static __device__ __forceinline__ float round(float x) { return x; }
 };
 template <>
 struct VT<__nv_bfloat16> {
@@ -40,6 +41,7 @@ struct VT<__nv_bfloat16> {
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
   }
+  static __device__ __forceinline__ float round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 };
 
 template <typename raw>

@@ -15,7 +15,7 @@ from tests.helpers import f64, to_dtype
 GUARD = 64  # canary elements after every output buffer
 
 
-def make_ctx(t, h, ffn, dtype, S=None, p=0.5, alpha=None, norm=0, eps=None, force_simt=False, direct_rows=False):
+def make_ctx(t, h, ffn, dtype, S=None, p=0.5, alpha=None, norm=0, eps=None, force_simt=False, direct_rows=False, no_decode=False):
     ctx = caat.Context(h, ffn, t, p, dtype)
     if S is not None:
         ctx.set_option(caat.CAAT_OPT_SHARED_CHANNELS, S)
@@ -31,6 +31,8 @@ def make_ctx(t, h, ffn, dtype, S=None, p=0.5, alpha=None, norm=0, eps=None, forc
         ctx.set_option(caat.CAAT_OPT_GEMM, 1)
     if direct_rows:
         ctx.set_option(caat.CAAT_OPT_ROWS, 1)
+    if no_decode:
+        ctx.set_option(caat.CAAT_OPT_DECODE, 1)
     return ctx
 
 

@@ -246,6 +246,44 @@ def test_block_forward_backward_small():
         assert_close(g, ob[name], "bf16", name)
 
 
+@pytest.mark.parametrize("no_decode", [False, True])
+@pytest.mark.parametrize("t,T,h,ffn,S,norm", [(8, 64, 4096, 11008, 2048, 0), (4, 37, 768, 3072, 384, 1),
+                                             (8, 1, 2048, 5632, 2048, 0), (2, 5, 256, 1024, 0, 0)])
+def test_few_token_forward_both_paths(no_decode, t, T, h, ffn, S, norm):
+    # forward calls with at most 64 tokens take the weight-streaming path (swapped GEMM operands,
+    # rank sum in the row kernel); CAAT_OPT_DECODE = 1 sends them down the large-batch path
+    ctx = G.make_ctx(t, h, ffn, "bf16", S=S, norm=norm, no_decode=no_decode)
+    for layer in (caat.CAAT_ATTN_OUT, caat.CAAT_MLP_DOWN):
+        d = _layer_case(t, T, h, ctx.k_r(layer), "bf16", S, seed=T + layer)
+        g = torch.Generator().manual_seed(6)
+        d["gamma"] = (1 + 0.1 * torch.randn(h, generator=g)).bfloat16()
+        d["beta"] = (0.1 * torch.randn(h, generator=g)).bfloat16()
+        _check_forward(ctx, layer, d, "bf16")
+
+
+@pytest.mark.parametrize("T,p,no_decode", [(1, 1.0, False), (8, 0.5, False), (64, 0.5, False), (64, 0.5, True), (33, 0.25, False)])
+def test_block_forward_few_tokens(T, p, no_decode):
+    # block forward at decode sizes: one GEMM launch for both layers + one row kernel for both
+    from oracle import caat_oracle as O
+    w = synthetic.Workload("blk_dec", 8, T, 4096, 11008, p, "bf16", "block", False, 3)
+    d = synthetic.block_inputs(w)
+    ctx = G.make_ctx(w.t, w.h, w.ffn, "bf16", p=w.p, no_decode=no_decode)
+    t, h = w.t, w.h
+    dev = {k: v.cuda() for k, v in d.items()}
+    mk = lambda *s, dt=torch.bfloat16: torch.empty(*s, dtype=dt, device="cuda")
+    Hn1, X1, Hn2, X2 = (mk(t, T, h) for _ in range(4))
+    rstd1, rstd2 = mk(t, T, dt=torch.float32), mk(t, T, dt=torch.float32)
+    ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, False))
+    ctx.block_forward(T, dev["Y_attn"], dev["W_o"], dev["Y_mlp"], dev["W_down"], dev["R0"], dev["gamma1"], None,
+                      dev["gamma2"], None, Hn1, X1, rstd1, None, Hn2, X2, rstd2, None, ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+    fo = O.block_forward(f64(d["Y_attn"]), f64(d["W_o"]), f64(d["Y_mlp"]), f64(d["W_down"]), f64(d["R0"]),
+                         f64(d["gamma1"]), f64(d["gamma2"]), S=ctx.shared_channels, alpha=ctx.private_scale)
+    for name, g in (("Hn1", Hn1), ("X1", X1), ("Hn2", Hn2), ("X2", X2), ("rstd1", rstd1), ("rstd2", rstd2)):
+        assert_close(g, fo[name], "bf16", name)
+
+
 # ------------------------------------------------------------------ decode shapes (forward only)
 @pytest.mark.parametrize("T", [1, 8, 64])
 @pytest.mark.parametrize("p", [1.0, 0.5])
