@@ -74,8 +74,9 @@ typedef enum {
   CAAT_OPT_PRIVATE_SCALE = 2,   /* alpha; default sqrt(t); 1 switches scaling off       */
   CAAT_OPT_SHARED_CHANNELS = 3, /* override S with an explicit integer in [0, h]        */
   CAAT_OPT_GEMM = 4,            /* 0 = automatic (default), 1 = force the CUDA-core GEMM */
-  CAAT_OPT_ROWS = 5,            /* 0 = automatic (default: bulk-copy staged row kernels),
-                                   1 = force the plain-load row kernels                  */
+  CAAT_OPT_ROWS = 5,            /* row kernels: 0 = automatic (default: warp-per-token kernels for
+                                   rows of at most 1024 bf16 channels, bulk-copy staged kernels
+                                   otherwise), 1 = plain-load kernels, 2 = staged kernels always */
   CAAT_OPT_DECODE = 6           /* 0 = automatic (default: forward calls with at most 64 tokens
                                    stream the weights with swapped GEMM operands),
                                    1 = always use the large-batch forward                */

@@ -272,7 +272,7 @@ caat_status caat_set_option(caat_ctx* ctx, caat_option opt, double value) {
       if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
       ctx->no_decode = (int)value; return CAAT_OK;
     case CAAT_OPT_ROWS:
-      if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
+      if (value != 0.0 && value != 1.0 && value != 2.0) return CAAT_EINVAL;
       ctx->direct_rows = (int)value; return CAAT_OK;
   }
   return CAAT_EINVAL;

@@ -101,8 +101,9 @@ struct RowFwdArgs {
   float alpha, eps;
   int norm;
 };
-// direct != 0 forces the plain-load kernels; otherwise the bulk-copy staged kernels run
-// whenever a ring of at least two stages fits in shared memory.
+// direct: 0 = automatic (warp-per-token kernels for short rows, else the bulk-copy staged kernels
+// whenever a ring of at least two stages fits in shared memory), 1 = plain-load kernels,
+// 2 = staged kernels even for short rows.
 cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
 cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st);
 // forward row work from fp32 partial planes (decode); with two layers the second layer's residual is
@@ -117,6 +118,9 @@ struct RowPartArgs {
   int norm;
 };
 cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype, cudaStream_t st);
+// warp-per-token kernels for short rows (h <= 1024 in bf16); rows_warp_cpt == 0: not applicable
+int rows_warp_cpt(int h, int t, caat_dtype dtype);
+cudaError_t launch_rows_forward_warp(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st);
 bool rows_staged_usable(int h, int t, int S_lo, int S_hi, caat_dtype dtype, bool backward);
 
 struct RowBwdArgs {
@@ -132,6 +136,8 @@ struct RowBwdArgs {
 cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
 cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,
                                         cudaStream_t st);
+cudaError_t launch_rows_backward_warp(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,
+                                      cudaStream_t st);
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype);
 
 // ---- bookkeeping ------------------------------------------------------------

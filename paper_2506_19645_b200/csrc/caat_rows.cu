@@ -495,8 +495,15 @@ int rows_backward_partial_rows(int h, int T, caat_dtype dtype) {
   return ngroups < kMaxPartialRows ? ngroups : kMaxPartialRows;
 }
 
+static int rows_mode_override(int direct) {   // CAAT_ROWS_MODE = 0/1/2 overrides the context option (experiments)
+  static const int env = [] { const char* e = getenv("CAAT_ROWS_MODE"); return e ? atoi(e) : -1; }();
+  return env >= 0 ? env : direct;
+}
+
 cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st) {
-  if (!direct && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, false)) return launch_rows_forward_staged(a, dtype, st);
+  direct = rows_mode_override(direct);
+  if (direct == 0 && rows_warp_cpt(a.h, a.t, dtype) > 0) return launch_rows_forward_warp(a, dtype, st);
+  if (direct != 1 && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, false)) return launch_rows_forward_staged(a, dtype, st);
   const RowGeom g = row_geometry(a.h, dtype);
   if (dtype == CAAT_BF16)
     return a.norm == 1 ? launch_fwd_t<__nv_bfloat16, true>(a, g, st) : launch_fwd_t<__nv_bfloat16, false>(a, g, st);
@@ -504,10 +511,13 @@ cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direc
 }
 
 cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st) {
+  direct = rows_mode_override(direct);
   const RowGeom g = row_geometry(a.h, dtype);
   int rows = rows_backward_partial_rows(a.h, a.T, dtype);
   cudaError_t e;
-  if (!direct && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, true))
+  if (direct == 0 && rows_warp_cpt(a.h, a.t, dtype) > 0)
+    e = launch_rows_backward_warp(a, dtype, rows, &rows, st);
+  else if (direct != 1 && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, true))
     e = launch_rows_backward_staged(a, dtype, rows, &rows, st);
   else if (dtype == CAAT_BF16)
     e = a.norm == 1 ? launch_bwd_t<__nv_bfloat16, true>(a, g, rows, st) : launch_bwd_t<__nv_bfloat16, false>(a, g, rows, st);

@@ -1,0 +1,564 @@
+// Row kernels for SHORT rows (at most four 16-byte chunks per lane: h <= 1024 in bf16).
+//
+// With short rows the CTA-wide reduction and barrier per rank of the general kernels cost more
+// than the arithmetic.  Here ONE WARP owns a token: its lanes cover the row's chunks (lane, lane+32,
+// ...), it walks the ranks m = 0..t-1, row statistics are plain warp shuffles and the rank sum of
+// the shared channels is lane-local.  Warps never wait for each other: a dedicated producer warp
+// keeps a shared-memory ring of (token group, rank) stages filled with cp.async.bulk, consumers
+// signal "stage read" on an mbarrier per stage, and the only CTA-wide step is the final fold of
+// the warps' partial norm-parameter gradients.  All waits are bounded (status word on timeout).
+#include "caat_rows_common.cuh"
+
+namespace caat {
+namespace {
+
+using namespace rows;
+
+constexpr int kW = 4;                    // consumer warps = tokens per group
+constexpr int kThreads = (kW + 1) * 32;  // + one producer warp
+constexpr int kMaxStages = 8;
+constexpr uint32_t kSpinCap = 1u << 18;
+constexpr uint32_t kSuspendHintNs = 20000u;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kSpinCap; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+template <typename raw>
+__device__ __forceinline__ raw lds(const uint8_t* p) { return *reinterpret_cast<const raw*>(p); }
+
+struct WarpGeom {
+  int nstages;
+  uint32_t off_a, off_b, off_c, stage_bytes;
+  uint32_t bar_off, ring_off;
+  size_t smem;
+};
+
+// ------------------------------------------------------------------ forward
+// stage: a = R rows [kW, h], b = zp rows [kW, P], c = zs rows [kW, S_hi] (rank 0 only)
+template <typename T_, int CPT, bool LN>
+__global__ void __launch_bounds__(kThreads, 3)
+rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned int* status) {
+  using V_ = VT<T_>;
+  using raw = typename V_::raw;
+  constexpr int V = V_::N;
+  constexpr int ES = sizeof(T_);
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* ring = smem + sg.ring_off;
+  const uint32_t full0 = smem_u32(smem + sg.bar_off), empty0 = full0 + 8u * kMaxStages;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + sg.bar_off + 16 * kMaxStages);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int NS = sg.nstages;
+  const bool has_priv = a.P > 0 && a.S < a.h, has_shared = a.S > 0;
+  const int my_groups = blockIdx.x < ngroups ? (ngroups - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NS; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, kW); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == kW) {
+    // ---------------------------------------------------------- producer
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      long long issued = 0;
+      bool ok = true;
+      for (int n = 0; n < my_groups && ok; ++n) {
+        const long long i0 = (blockIdx.x + (long long)n * gridDim.x) * kW;
+        const int rowsN = (int)((a.T - i0) < kW ? (a.T - i0) : kW);
+        for (int m = 0; m < a.t; ++m) {
+          if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t bar = full0 + 8u * s;
+          const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
+          const uint32_t bR = (uint32_t)rowsN * a.h * ES;
+          const uint32_t bP = has_priv ? (uint32_t)rowsN * a.P * ES : 0u;
+          const uint32_t bS = (m == 0 && has_shared) ? (uint32_t)rowsN * a.S_hi * ES : 0u;
+          mbar_expect_tx(bar, bR + bP + bS);
+          const long long row = (long long)m * a.T + i0;
+          bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * a.h * ES, bR, bar);
+          if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
+          if (bS) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.zs) + i0 * a.S_hi * ES, bS, bar);
+          ++issued;
+          if (++s == NS) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicExch(status, 6u);
+        const int pending = issued < NS ? (int)issued : NS;
+        for (int k = 0; k < pending; ++k) {        // let this CTA's copies in flight land
+          if (--s < 0) { s = NS - 1; ph ^= 1u; }
+          for (uint32_t it = 0; it < (1u << 12); ++it)
+            if (mbar_try(full0 + 8u * s, ph)) break;
+        }
+      }
+    }
+    return;
+  }
+
+  // ------------------------------------------------------------ consumers: warp w owns token i0 + w
+  int col[CPT], cls[CPT];
+  bool colok[CPT];
+  float gam[CPT][V], bet[CPT][V];
+#pragma unroll
+  for (int j = 0; j < CPT; ++j) {
+    col[j] = (lane + 32 * j) * V;
+    colok[j] = col[j] < a.h;
+    cls[j] = chunk_class(col[j], V, a.S);
+#pragma unroll
+    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; bet[j][e] = 0.f; }
+    if (colok[j]) {
+      V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+      if (LN && a.beta) V_::unpack(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
+    }
+  }
+  const float inv_h = 1.0f / (float)a.h;
+  const long long rank_h = (long long)a.T * a.h * ES;
+  int s = 0; uint32_t ph = 0;
+  bool dead = false;
+  for (int n = 0; n < my_groups && !dead; ++n) {
+    const long long i = (blockIdx.x + (long long)n * gridDim.x) * kW + warp;
+    const bool valid = i < a.T;
+    float zs[CPT][V];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j)
+#pragma unroll
+      for (int e = 0; e < V; ++e) zs[j][e] = 0.f;
+    char* pHn = static_cast<char*>(a.Hn) + i * a.h * ES;
+    char* pX = static_cast<char*>(a.X) + i * a.h * ES;
+    float* rstd_p = a.rstd + i;
+    float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
+    for (int m = 0; m < a.t; ++m) {
+      if (!mbar_wait(full0 + 8u * s, ph, abort_flag)) { dead = true; break; }
+      const uint8_t* stage = ring + (size_t)s * sg.stage_bytes;
+      float hn[CPT][V];
+      float st = 0.f;
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        float r[V], zp[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) { r[e] = 0.f; zp[e] = 0.f; }
+        const bool act = valid && colok[j];
+        if (act) {
+          V_::unpack(lds<raw>(stage + sg.off_a + ((size_t)warp * a.h + col[j]) * ES), r);
+          if (cls[j] != 0) V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES), zp);
+          if (m == 0 && cls[j] != 1) V_::unpack(lds<raw>(stage + sg.off_c + ((size_t)warp * a.S_hi + col[j]) * ES), zs[j]);
+        }
+        if (cls[j] == 0) {
+#pragma unroll
+          for (int e = 0; e < V; ++e) hn[j][e] = zs[j][e] + r[e];
+        } else if (cls[j] == 1) {
+#pragma unroll
+          for (int e = 0; e < V; ++e) hn[j][e] = fmaf(a.alpha, zp[e], r[e]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < V; ++e) hn[j][e] = (col[j] + e < a.S ? zs[j][e] : a.alpha * zp[e]) + r[e];
+        }
+        if (act) stg<raw>(pHn + (long long)col[j] * ES, V_::pack(hn[j]));
+#pragma unroll
+        for (int e = 0; e < V; ++e) st = LN ? st + hn[j][e] : fmaf(hn[j][e], hn[j][e], st);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8u * s);      // this warp is done with the stage
+      if (++s == NS) { s = 0; ph ^= 1u; }
+      st = warp_sum(st);
+      float mu = 0.f, rs;
+      if (LN) {
+        mu = st * inv_h;
+        float sq = 0.f;
+#pragma unroll
+        for (int j = 0; j < CPT; ++j)
+#pragma unroll
+          for (int e = 0; e < V; ++e) {
+            const float d = (valid && colok[j]) ? hn[j][e] - mu : 0.f;
+            sq = fmaf(d, d, sq);
+          }
+        rs = rsqrtf(fmaf(warp_sum(sq), inv_h, a.eps));
+      } else {
+        rs = rsqrtf(fmaf(st, inv_h, a.eps));
+      }
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) {
+        float x[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          if (LN) x[e] = fmaf(hn[j][e] - mu, rs * gam[j][e], bet[j][e]);
+          else x[e] = hn[j][e] * (rs * gam[j][e]);
+        }
+        if (valid && colok[j]) stg<raw>(pX + (long long)col[j] * ES, V_::pack(x));
+      }
+      if (valid && lane == 0) {
+        *rstd_p = rs;
+        if (LN && mean_p) *mean_p = mu;
+      }
+      pHn += rank_h; pX += rank_h; rstd_p += a.T;
+      if (LN && mean_p) mean_p += a.T;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ backward
+// stage: a = dX rows, b = Hn rows, c = dHn rows (when given), kW tokens each
+template <typename T_, int CPT, bool LN>
+__global__ void __launch_bounds__(kThreads, 3)
+rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned int* status) {
+  using V_ = VT<T_>;
+  using raw = typename V_::raw;
+  constexpr int V = V_::N;
+  constexpr int ES = sizeof(T_);
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* ring = smem + sg.ring_off;
+  const uint32_t full0 = smem_u32(smem + sg.bar_off), empty0 = full0 + 8u * kMaxStages;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + sg.bar_off + 16 * kMaxStages);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int NS = sg.nstages;
+  const bool has_dh = a.dHn != nullptr;
+  const int my_groups = blockIdx.x < ngroups ? (ngroups - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NS; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, kW); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  int col[CPT], cls[CPT];
+  bool colok[CPT];
+  float gam[CPT][V], dgacc[CPT][V], dbacc[LN ? CPT : 1][V];
+#pragma unroll
+  for (int j = 0; j < CPT; ++j) {
+    col[j] = (lane + 32 * j) * V;
+    colok[j] = col[j] < a.h;
+    cls[j] = chunk_class(col[j], V, a.S);
+#pragma unroll
+    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; dgacc[j][e] = 0.f; if constexpr (LN) dbacc[j][e] = 0.f; }
+  }
+
+  if (warp == kW) {
+    // ---------------------------------------------------------- producer
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      long long issued = 0;
+      bool ok = true;
+      for (int n = 0; n < my_groups && ok; ++n) {
+        const long long i0 = (blockIdx.x + (long long)n * gridDim.x) * kW;
+        const int rowsN = (int)((a.T - i0) < kW ? (a.T - i0) : kW);
+        const uint32_t b = (uint32_t)rowsN * a.h * ES;
+        for (int m = 0; m < a.t; ++m) {
+          if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t bar = full0 + 8u * s;
+          const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
+          mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
+          const long long off = ((long long)m * a.T + i0) * a.h * ES;
+          bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
+          bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
+          if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
+          ++issued;
+          if (++s == NS) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicExch(status, 7u);
+        const int pending = issued < NS ? (int)issued : NS;
+        for (int k = 0; k < pending; ++k) {
+          if (--s < 0) { s = NS - 1; ph ^= 1u; }
+          for (uint32_t it = 0; it < (1u << 12); ++it)
+            if (mbar_try(full0 + 8u * s, ph)) break;
+        }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------- consumers
+#pragma unroll
+    for (int j = 0; j < CPT; ++j)
+      if (colok[j]) V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+    const float inv_h = 1.0f / (float)a.h;
+    const long long rank_h = (long long)a.T * a.h * ES, rank_p = (long long)a.T * a.P * ES;
+    int s = 0; uint32_t ph = 0;
+    bool dead = false;
+    // lane m holds rstd (mean) of rank m for the current token; the next token's are fetched a group ahead
+    auto load_stat = [&](const float* base, int n) -> float {
+      const long long i = (blockIdx.x + (long long)n * gridDim.x) * kW + warp;
+      return (base != nullptr && n < my_groups && i < a.T && lane < a.t) ? base[(long long)lane * a.T + i] : 0.f;
+    };
+    float rs_next = load_stat(a.rstd, 0), mu_next = LN ? load_stat(a.mean, 0) : 0.f;
+    for (int n = 0; n < my_groups && !dead; ++n) {
+      const long long i = (blockIdx.x + (long long)n * gridDim.x) * kW + warp;
+      const bool valid = i < a.T;
+      const float rs_lane = rs_next, mu_lane = mu_next;
+      rs_next = load_stat(a.rstd, n + 1);
+      if (LN) mu_next = load_stat(a.mean, n + 1);
+      float gsum[CPT][V];
+#pragma unroll
+      for (int j = 0; j < CPT; ++j)
+#pragma unroll
+        for (int e = 0; e < V; ++e) gsum[j][e] = 0.f;
+      char* pdR = static_cast<char*>(a.dR) + i * a.h * ES;
+      char* pZ = static_cast<char*>(a.zp) + (i * a.P - a.S_lo) * ES;
+      for (int m = 0; m < a.t; ++m) {
+        if (!mbar_wait(full0 + 8u * s, ph, abort_flag)) { dead = true; break; }
+        const uint8_t* stage = ring + (size_t)s * sg.stage_bytes;
+        const float rs = __shfl_sync(0xffffffffu, rs_lane, m);
+        const float mu = LN ? __shfl_sync(0xffffffffu, mu_lane, m) : 0.f;
+        // pass 1: row statistics and norm-parameter gradients
+        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) {
+          if (!(valid && colok[j])) continue;
+          float dx[V], hn[V];
+          const size_t o = ((size_t)warp * a.h + col[j]) * ES;
+          V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
+          V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
+#pragma unroll
+          for (int e = 0; e < V; ++e) {
+            const float xh = (hn[e] - mu) * rs;
+            const float dxh = dx[e] * gam[j][e];
+            if (LN) s1 += dxh;
+            s2 = fmaf(dxh, xh, s2);
+            dgacc[j][e] = fmaf(dx[e], xh, dgacc[j][e]);
+            if constexpr (LN) dbacc[j][e] += dx[e];
+          }
+        }
+        const float c1 = LN ? warp_sum(s1) * inv_h : 0.f;
+        const float c2 = warp_sum(s2) * inv_h;
+        // pass 2: gradients (the stage is re-read: cheaper than keeping the row in registers)
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) {
+          if (!(valid && colok[j])) continue;
+          float dx[V], hn[V], dh[V], gg[V];
+          const size_t o = ((size_t)warp * a.h + col[j]) * ES;
+          V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
+          V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
+#pragma unroll
+          for (int e = 0; e < V; ++e) dh[e] = 0.f;
+          if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + o), dh);
+#pragma unroll
+          for (int e = 0; e < V; ++e) {
+            const float xh = (hn[e] - mu) * rs;
+            float tt = fmaf(-xh, c2, dx[e] * gam[j][e]);
+            if (LN) tt -= c1;
+            gg[e] = fmaf(rs, tt, dh[e]);
+          }
+          stg<raw>(pdR + (long long)col[j] * ES, V_::pack(gg));
+          if (cls[j] == 0) {
+#pragma unroll
+            for (int e = 0; e < V; ++e) gsum[j][e] += gg[e];          // fp32 rank sum, m ascending
+          } else {
+            float zp[V];
+            if (cls[j] == 1) {
+#pragma unroll
+              for (int e = 0; e < V; ++e) zp[e] = a.alpha * gg[e];    // private gradient carries alpha
+            } else {
+#pragma unroll
+              for (int e = 0; e < V; ++e) {
+                const bool shared = col[j] + e < a.S;
+                gsum[j][e] += shared ? gg[e] : 0.f;
+                zp[e] = shared ? 0.f : a.alpha * gg[e];
+              }
+            }
+            stg<raw>(pZ + (long long)col[j] * ES, V_::pack(zp));
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8u * s);
+        if (++s == NS) { s = 0; ph ^= 1u; }
+        pdR += rank_h; pZ += rank_p;
+      }
+      if (dead) break;
+#pragma unroll
+      for (int j = 0; j < CPT; ++j)
+        if (valid && colok[j] && cls[j] != 1)
+          stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, V_::pack(gsum[j]));
+    }
+  }
+
+  // fold the warps' partial norm-parameter gradients: one row of [h] per CTA (the ring is free by now:
+  // every copy that was issued has been consumed, or the kernel gave up and the values do not matter)
+  __syncthreads();
+  float* acc = reinterpret_cast<float*>(ring);        // [kW][h]
+  for (int which = 0; which < (LN ? 2 : 1); ++which) {
+    float* out = which == 0 ? a.dgpart : a.dbpart;
+    if (out == nullptr) continue;
+    if (warp < kW) {
+#pragma unroll
+      for (int j = 0; j < CPT; ++j)
+        if (colok[j])
+#pragma unroll
+          for (int e = 0; e < V; ++e)
+            acc[(size_t)warp * a.h + col[j] + e] = (which == 0 || !LN) ? dgacc[j][e] : dbacc[LN ? j : 0][e];
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < a.h; c += blockDim.x) {
+      float sum = 0.f;
+#pragma unroll
+      for (int w = 0; w < kW; ++w) sum += acc[(size_t)w * a.h + c];
+      out[(size_t)blockIdx.x * a.h + c] = sum;
+    }
+    __syncthreads();
+  }
+}
+
+WarpGeom warp_geometry(int h, int P, int S_hi, int ES, bool backward, bool has_c, size_t budget) {
+  WarpGeom g{};
+  const uint32_t rowA = (uint32_t)kW * h * ES;
+  if (backward) {
+    g.off_a = 0; g.off_b = rowA; g.off_c = 2 * rowA;
+    g.stage_bytes = (has_c ? 3 : 2) * rowA;
+  } else {
+    const uint32_t rowB = (uint32_t)kW * P * ES, rowC = (uint32_t)kW * S_hi * ES;
+    g.off_a = 0; g.off_b = rowA; g.off_c = rowA + rowB;
+    g.stage_bytes = rowA + rowB + rowC;
+  }
+  g.stage_bytes = (g.stage_bytes + 127u) & ~127u;
+  g.bar_off = 0;
+  g.ring_off = (uint32_t)align_up(16 * kMaxStages + 16, 128);
+  int ns = (int)((budget - g.ring_off) / g.stage_bytes);
+  if (ns > kMaxStages) ns = kMaxStages;
+  g.nstages = ns;
+  size_t ring = (size_t)(ns > 0 ? ns : 0) * g.stage_bytes;
+  const size_t acc = backward ? (size_t)kW * h * sizeof(float) : 0;
+  if (ring < acc) ring = acc;
+  g.smem = g.ring_off + ring;
+  return g;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+constexpr size_t kSmemPerSm = 227 * 1024;
+constexpr int kCtasPerSm = 3;
+
+template <typename K>
+cudaError_t set_smem(K kernel, size_t bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+template <typename T_, bool LN>
+cudaError_t launch_fwd_warp_t(const RowFwdArgs& a, int cpt, const WarpGeom& g, int grid, int ngroups,
+                              unsigned int* status, cudaStream_t st) {
+  cudaError_t e = cudaSuccess;
+  LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
+#define CAAT_LAUNCH(CPT_)                                                                      \
+  do {                                                                                         \
+    e = set_smem(rows_forward_warp<T_, CPT_, LN>, g.smem);                                     \
+    if (e == cudaSuccess) rows_forward_warp<T_, CPT_, LN><<<grid, kThreads, g.smem, st>>>(a, g, ngroups, status); \
+  } while (0)
+  switch (cpt) {
+    case 1: CAAT_LAUNCH(1); break;
+    case 2: CAAT_LAUNCH(2); break;
+    case 3: CAAT_LAUNCH(3); break;
+    case 4: CAAT_LAUNCH(4); break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef CAAT_LAUNCH
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+template <typename T_, bool LN>
+cudaError_t launch_bwd_warp_t(const RowBwdArgs& a, int cpt, const WarpGeom& g, int grid, int ngroups,
+                              unsigned int* status, cudaStream_t st) {
+  cudaError_t e = cudaSuccess;
+  LaunchScope scope(CAAT_K_ROWS_BACKWARD, st);
+#define CAAT_LAUNCH(CPT_)                                                                       \
+  do {                                                                                          \
+    e = set_smem(rows_backward_warp<T_, CPT_, LN>, g.smem);                                     \
+    if (e == cudaSuccess) rows_backward_warp<T_, CPT_, LN><<<grid, kThreads, g.smem, st>>>(a, g, ngroups, status); \
+  } while (0)
+  switch (cpt) {
+    case 1: CAAT_LAUNCH(1); break;
+    case 2: CAAT_LAUNCH(2); break;
+    case 3: CAAT_LAUNCH(3); break;
+    case 4: CAAT_LAUNCH(4); break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef CAAT_LAUNCH
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+}  // namespace
+
+// chunks per lane of the warp-per-token kernels, 0 when the row is too long for them
+int rows_warp_cpt(int h, int t, caat_dtype dtype) {
+  const int V = dtype == CAAT_BF16 ? 8 : 4;
+  const int chunks = h / V;
+  const int cpt = (chunks + 31) / 32;
+  return (cpt >= 1 && cpt <= 4 && t <= 32) ? cpt : 0;
+}
+
+cudaError_t launch_rows_forward_warp(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st) {
+  const int cpt = rows_warp_cpt(a.h, a.t, dtype);
+  const int ES = (int)elem_size(dtype);
+  const WarpGeom g = warp_geometry(a.h, a.P, a.S_hi, ES, false, true, kSmemPerSm / kCtasPerSm - 1024);
+  if (cpt == 0 || g.nstages < 2) return cudaErrorInvalidConfiguration;
+  const int ngroups = (a.T + kW - 1) / kW;
+  int grid = sm_count() * kCtasPerSm;
+  if (grid > ngroups) grid = ngroups;
+  unsigned int* status = device_status_word();
+  if (!status) return cudaErrorUnknown;
+  if (dtype == CAAT_BF16)
+    return a.norm == 1 ? launch_fwd_warp_t<__nv_bfloat16, true>(a, cpt, g, grid, ngroups, status, st)
+                       : launch_fwd_warp_t<__nv_bfloat16, false>(a, cpt, g, grid, ngroups, status, st);
+  return a.norm == 1 ? launch_fwd_warp_t<float, true>(a, cpt, g, grid, ngroups, status, st)
+                     : launch_fwd_warp_t<float, false>(a, cpt, g, grid, ngroups, status, st);
+}
+
+cudaError_t launch_rows_backward_warp(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,
+                                      cudaStream_t st) {
+  const int cpt = rows_warp_cpt(a.h, a.t, dtype);
+  const int ES = (int)elem_size(dtype);
+  const WarpGeom g = warp_geometry(a.h, 0, 0, ES, true, a.dHn != nullptr, kSmemPerSm / kCtasPerSm - 1024);
+  if (cpt == 0 || g.nstages < 2) return cudaErrorInvalidConfiguration;
+  const int ngroups = (a.T + kW - 1) / kW;
+  int grid = sm_count() * kCtasPerSm;
+  if (grid > ngroups) grid = ngroups;
+  if (grid > max_rows) grid = max_rows;
+  *rows_used = grid;
+  unsigned int* status = device_status_word();
+  if (!status) return cudaErrorUnknown;
+  if (dtype == CAAT_BF16)
+    return a.norm == 1 ? launch_bwd_warp_t<__nv_bfloat16, true>(a, cpt, g, grid, ngroups, status, st)
+                       : launch_bwd_warp_t<__nv_bfloat16, false>(a, cpt, g, grid, ngroups, status, st);
+  return a.norm == 1 ? launch_bwd_warp_t<float, true>(a, cpt, g, grid, ngroups, status, st)
+                     : launch_bwd_warp_t<float, false>(a, cpt, g, grid, ngroups, status, st);
+}
+
+}  // namespace caat

@@ -30,7 +30,7 @@ def make_ctx(t, h, ffn, dtype, S=None, p=0.5, alpha=None, norm=0, eps=None, forc
     if force_simt:
         ctx.set_option(caat.CAAT_OPT_GEMM, 1)
     if direct_rows:
-        ctx.set_option(caat.CAAT_OPT_ROWS, 1)
+        ctx.set_option(caat.CAAT_OPT_ROWS, int(direct_rows))
     if no_decode:
         ctx.set_option(caat.CAAT_OPT_DECODE, 1)
     return ctx

@@ -102,13 +102,15 @@ def test_both_gemm_paths_agree_with_oracle(force_simt):
     _check_backward(ctx, caat.CAAT_MLP_DOWN, d, "bf16")
 
 
-@pytest.mark.parametrize("direct_rows", [False, True])
+@pytest.mark.parametrize("direct_rows", [0, 1, 2])
 @pytest.mark.parametrize("t,T,h,ffn,S,norm,dtype", [
     (8, 77, 4096, 11008, 2048, 0, "bf16"), (4, 301, 768, 3072, 380, 1, "bf16"), (2, 131, 256, 1024, 100, 1, "f32"),
-    (8, 1500, 2048, 5632, 2048, 0, "bf16"), (3, 45, 9216, 9216, 4608, 0, "bf16")])
+    (8, 1500, 2048, 5632, 2048, 0, "bf16"), (3, 45, 9216, 9216, 4608, 0, "bf16"),
+    (4, 2003, 768, 3072, 384, 0, "bf16"), (8, 1, 1024, 4096, 100, 1, "bf16"), (16, 70, 512, 2048, 512, 0, "f32")])
 def test_both_row_kernel_variants(direct_rows, t, T, h, ffn, S, norm, dtype):
-    # the bulk-copy staged kernels (default) and the plain-load kernels compute the same thing;
-    # T = 1500 makes persistent CTAs walk several token groups, h = 9216 takes two chunks per thread
+    # the three row-kernel families compute the same thing: automatic choice (warp-per-token for
+    # short rows, bulk-copy staged otherwise), plain loads (1), staged always (2);
+    # T = 1500 makes persistent CTAs walk several token groups, h = 9216 takes four chunks per thread
     ctx = G.make_ctx(t, h, ffn, dtype, S=S, norm=norm, direct_rows=direct_rows)
     d = _layer_case(t, T, h, ctx.k_r(caat.CAAT_ATTN_OUT), dtype, S, seed=T, backward=True)
     _check_forward(ctx, caat.CAAT_ATTN_OUT, d, dtype)
