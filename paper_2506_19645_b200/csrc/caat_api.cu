@@ -87,6 +87,9 @@ Scratch scratch_layout(const caat_ctx* ctx, int K_r, int tokens, int backward) {
       s.splitk_bytes = tc_wgrad_splitk_bytes(sh);
     }
     off = align_up(off + s.splitk_bytes, 256);
+    s.wt_off = off;
+    if (tc_gemm_usable(ctx, K_r) && tc_dgrad_wants_wt(tokens))
+      off = align_up(off + (size_t)ctx->t * ctx->h * K_r * e, 256);
   }
   s.total = off;
   return s;
@@ -189,7 +192,7 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
 
   if (tc_gemm_usable(ctx, K_r)) {
     RowparShapes sh{t, T, h, K_r, S, L.S_lo, L.S_hi, L.P};
-    ce = launch_tc_dgrad(sh, gs, zp, W, dY, st);
+    ce = launch_tc_dgrad(sh, gs, zp, W, dY, tc_dgrad_wants_wt(T) ? wsb + L.wt_off : nullptr, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
     ce = launch_tc_wgrad(sh, gs, zp, Y, dW, wsb + L.splitk_off, L.splitk_bytes, st);
     if (ce != cudaSuccess) return cuda_fail(ce);

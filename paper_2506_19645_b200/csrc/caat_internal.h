@@ -40,6 +40,7 @@ struct Scratch {
   size_t zs_off, zp_off;   // forward: Zt shared / private.  backward: dZt shared / private
   size_t dgpart_off, dbpart_off;  // backward: [rows, h] fp32 partial norm-parameter gradients
   size_t splitk_off, splitk_bytes;  // backward: split-K partials of the weight gradient
+  size_t wt_off;           // backward: transposed weights [t, K_r, h] (when the data gradient asks for them)
   size_t zt_off;           // forward, few tokens: fp32 per-rank partials [t, T, h]
   size_t total;
 };
@@ -78,8 +79,11 @@ bool tc_gemm_usable(const caat_ctx* ctx, int K_r);
 cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* W, void* zs, void* zp,
                               cudaStream_t st);
 // dY[m] = [gs | zp[m]] W[m]
+// wt_scratch: optional [t, K_r, h] bf16 scratch; when given, W is transposed into it first and the
+// GEMM reads a K-major B operand
 cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* zp, const void* W, void* dY,
-                            cudaStream_t st);
+                            void* wt_scratch, cudaStream_t st);
+bool tc_dgrad_wants_wt(int tokens);
 // dW[m] = [gs | zp[m]]^T Y[m]   (fp32 out)
 cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* zp, const void* Y, float* dW,
                             void* splitk, size_t splitk_bytes, cudaStream_t st);
