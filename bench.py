@@ -29,7 +29,7 @@ sys.path.insert(0, ROOT)
 
 import torch  # noqa: E402
 
-from paper_2506_19645_b200 import synthetic  # noqa: E402
+from paper_2506_19645_b200 import replicas, synthetic  # noqa: E402
 
 DEFAULT_WORKLOAD = "block_130m"
 METRIC = "CAAT block tokens/s (sim. TP=t, sync p) on 1 B200"
@@ -289,9 +289,7 @@ def cpu_baseline(w, target_s=12.0):
 
 def run_cuda(args):
     from paper_2506_19645_b200 import caat
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = replicas.rank_env()
     dist_on = world > 1
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device (there is no CPU path)")
@@ -324,13 +322,10 @@ def run_cuda(args):
     ms_prof = time_steps(runner, args.steps, dist_on)
     prof = caat.profile_end()
     clocks = sampler.stop()
-    if dist_on:
-        tms = torch.tensor([ms], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(tms, op=torch.distributed.ReduceOp.MAX)
-        ms = float(tms.item())
+    ms = replicas.max_over_ranks(ms, dev)
 
     ms_step = ms / args.steps
-    value = world * w.tokens * args.steps / (ms * 1e-3)
+    value = replicas.whole_job_rate(w.tokens, args.steps, world, ms)
 
     result = None
     if rank == 0:

@@ -71,7 +71,8 @@ struct Params {
   int tiles_r0;          // tiles of region 0 (including splits)
   int tiles_total;
   unsigned int* status;
-  int debug;             // measurement aid: 1 = producer skips the loads, 2 = epilogue skips the stores
+  int debug;             // measurement aid (env CAAT_TC_DEBUG; results are then wrong): 1 = no operand loads,
+                         // 2 = no output stores, 4 = no A loads, 8 = no B loads
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -197,7 +198,7 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& p, int tile) {
 // Columns of B a tile really needs: the last tile of a ragged N (N-major B only) is narrowed to
 // whole 64-column chunks per CTA, so no padded columns are loaded or multiplied.
 __device__ __forceinline__ int tile_cols(const Params& p, const Region& r, int nt, int cg) {
-  if (!p.b_mn || (p.debug & 16)) return p.BN;
+  if (!p.b_mn) return p.BN;
   const int left = r.N - nt * p.BN;
   if (left >= p.BN) return p.BN;
   const int q = 64 * cg;

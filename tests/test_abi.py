@@ -62,7 +62,7 @@ def test_options(caat):
 
 def test_workspace_and_argument_errors_before_launch(caat):
     c = caat.Context(768, 3072, 4, 0.5, "bf16")
-    T = 64
+    T = 256        # above the few-token (decode) threshold, whose forward scratch holds fp32 planes
     need = c.workspace_bytes(caat.CAAT_MLP_DOWN, T, False)
     assert need >= T * 384 * 2 + 4 * T * 384 * 2
     assert c.workspace_bytes(caat.CAAT_MLP_DOWN, T, True) > need
