@@ -10,8 +10,11 @@
 // partial channel-reduce of Eq. A3 becomes a longer contraction), so rank partials of the
 // shared channels never exist in memory.
 //
-// Roles per CTA (192 threads): warp 0 issues TMA loads, warp 1 issues MMAs and owns the
-// tensor-memory allocation, warps 2-5 drain accumulators (tcgen05.ld) and store.  Two
+// Roles per CTA (224 threads): warp 0 issues the TMA loads of the A operand and warp 6 those
+// of the B operand (one thread issuing every box of a stage was the limiter when a stage is
+// four boxes; two instruction streams walk the same schedule independently), warp 1 issues
+// MMAs and owns the tensor-memory allocation, warps 2-5 drain accumulators (tcgen05.ld) and
+// store.  Two
 // accumulators of up to 256 columns alternate so a tile's epilogue overlaps the next
 // tile's MMAs.  Every mbarrier wait is bounded; on a timeout the kernel records a status
 // word, drains its own copies in flight, frees tensor memory and returns.
@@ -29,7 +32,8 @@ namespace {
 constexpr int BM = 128;           // rows of an output tile (UMMA M, cta_group::1)
 constexpr int BK = 64;            // contraction elements per pipeline stage (128 bytes of bf16)
 constexpr int UMMA_K = 16;        // contraction elements per tcgen05.mma (kind::f16)
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;     // warps: 0 = A producer, 1 = MMA issuer, 2..5 = epilogue, 6 = B producer
+constexpr int kProducerB = 6;
 constexpr int kAccCols = 256;     // column stride between the two accumulators
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSpinCap = 1u << 22;
@@ -307,9 +311,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
+  if (warp == 0 || warp == kProducerB) {
+    // ------------------------------------------------------------ TMA producers
+    // Two single-thread producers run the same schedule: warp 0 issues the A boxes (and, in the
+    // leader CTA, posts the stage's expected bytes), warp kProducerB the B boxes.  Issuing a
+    // stage's boxes from one thread was the bottleneck of the operand pipeline (up to four boxes
+    // per stage for M-/N-major operands); two independent instruction streams halve it.
     if (lane == 0) {
+      const bool isA = warp == 0;
       int stage = 0; uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
@@ -319,42 +328,43 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         const uint32_t cols_cta = (uint32_t)tile_cols(p, r, c.nt, CG) / CG;    // B columns this CTA stages
         const uint32_t b_tile_bytes = cols_cta * BK * 2;
         const int m0 = c.mt * BMT + (int)rank * BM, n0 = c.nt * p.BN + (int)(rank * cols_cta);
+        const uint32_t tx = (uint32_t)CG * (((p.debug & 4) ? 0u : a_bytes) + ((p.debug & 8) ? 0u : b_tile_bytes));
+        const bool skip = isA ? (p.debug & 4) != 0 : (p.debug & 8) != 0;
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
+          const CUtensorMap* map = maps[isA ? u.mapA : u.mapB];
           int kb, ke;
           split_range(r.splits, u, c.split, kb, ke);
           for (int q = 0; q < u.Q && ok; ++q) {
-            const int az = c.b * u.a_zb + q * u.a_zq, bz = c.b * u.b_zb + q * u.b_zq;
+            const int z = isA ? c.b * u.a_zb + q * u.a_zq : c.b * u.b_zb + q * u.b_zq;
             for (int kk = kb; kk < ke; ++kk) {
               if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
               const uint32_t fb_local = full0 + 8u * stage;
               // completion is signalled on the LEADER's barrier; the leader expects both CTAs' bytes
               const uint32_t fb = CG == 2 ? mapa_rank(fb_local, 0) : fb_local;
               const uint32_t sa = tiles_sa + (uint32_t)stage * stage_bytes, sb = sa + a_bytes;
-              if (p.debug & 1) {
-                if (rank == 0) mbar_arrive(fb_local);
-                ++issued; if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
-                continue;
+              if (isA && rank == 0) {
+                if (p.debug & 1) mbar_arrive(fb_local); else mbar_expect_tx(fb_local, tx);
               }
-              if (rank == 0)
-                mbar_expect_tx(fb_local, (uint32_t)CG * (((p.debug & 4) ? 0u : a_bytes) + ((p.debug & 8) ? 0u : b_tile_bytes)));
-              auto load = [&](uint32_t dst, const CUtensorMap* m, int x, int y, int z) {
-                if (CG == 2) tma_load_3d_pair(dst, m, x, y, z, fb); else tma_load_3d(dst, m, x, y, z, fb);
-              };
-              if (p.debug & 4) {
-              } else if (!p.a_mn) {
-                load(sa, maps[u.mapA], u.ak0 + kk * BK, m0, az);
-              } else {
+              if (!(p.debug & 1) && !skip) {
+                auto load = [&](uint32_t dst, int x, int y) {
+                  if (CG == 2) tma_load_3d_pair(dst, map, x, y, z, fb); else tma_load_3d(dst, map, x, y, z, fb);
+                };
+                if (isA) {
+                  if (!p.a_mn) {
+                    load(sa, u.ak0 + kk * BK, m0);
+                  } else {
 #pragma unroll
-                for (int ch = 0; ch < BM / 64; ++ch)
-                  load(sa + ch * (64 * BK * 2), maps[u.mapA], u.am0 + m0 + ch * 64, u.ak0 + kk * BK, az);
-              }
-              if (p.debug & 8) {
-              } else if (!p.b_mn) {
-                load(sb, maps[u.mapB], u.bk0 + kk * BK, u.bn0 + n0, bz);
-              } else {
-                for (int ch = 0; ch < (int)cols_cta / 64; ++ch)
-                  load(sb + ch * (64 * BK * 2), maps[u.mapB], u.bn0 + n0 + ch * 64, u.bk0 + kk * BK, bz);
+                    for (int ch = 0; ch < BM / 64; ++ch) load(sa + ch * (64 * BK * 2), u.am0 + m0 + ch * 64, u.ak0 + kk * BK);
+                  }
+                } else {
+                  if (!p.b_mn) {
+                    load(sb, u.bk0 + kk * BK, u.bn0 + n0);
+                  } else {
+                    for (int ch = 0; ch < (int)cols_cta / 64; ++ch)
+                      load(sb + ch * (64 * BK * 2), u.bn0 + n0 + ch * 64, u.bk0 + kk * BK);
+                  }
+                }
               }
               ++issued;
               if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
@@ -363,7 +373,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         }
       }
       if (!ok) {
-        // gave up: flag it, then wait (bounded) for the copies this thread still has in flight
+        // gave up: flag it, then wait (bounded) for the copies still in flight
         // (the pair's copies complete on the leader's barriers; the peer just gives them time)
         *abort_flag = 1;
         atomicExch(p.status, 1u);
@@ -425,7 +435,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       }
       if (!ok) { *abort_flag = 1; atomicExch(p.status, 2u); }
     }
-  } else {
+  } else if (warp <= 5) {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter+32)
     int acc = 0; uint32_t acc_phase = 0;
