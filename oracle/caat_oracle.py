@@ -28,7 +28,10 @@ brute-force index-notation evaluation of Eq. A3, p=1 against an unsharded
 library matmul plus library norms, p=0 independence, rank-permutation
 invariance, the variance law of Eq. 14-15, central finite differences and the
 p=1 reduce-before-norm equivalence of Section 4 for the backward, and the
-closed forms of Appendix C for the byte counts.
+closed forms of Appendix C for the byte counts.  The compact-layout functions
+(shared part of the residual stream stored once) are pinned by their own finite
+differences, by equality with the per-rank forward on a tied residual, and by the
+rank-sum relation between a tied variable's gradient and its copies' gradients.
 
 Parity unpinned (the paper fixes no value; these are this build's documented
 choices): eps, the norm kind per model, the default of alpha, the dtype of dW.
@@ -232,6 +235,93 @@ def block_backward(dX1, dX2, dHn2, Y_attn, W_o, Y_mlp, W_down, Hn1, rstd1, mean1
     return {"dY_attn": b1["dY"], "dW_o": b1["dW"], "dY_mlp": b2["dY"], "dW_down": b2["dW"],
             "dR0": b1["dR"], "dHn1": b2["dR"], "dgamma1": b1["dgamma"], "dgamma2": b2["dgamma"],
             "dbeta1": b1["dbeta"], "dbeta2": b2["dbeta"]}
+
+
+# --------------------------------------------------------------------------
+# Compact ("logical devices on one GPU", Section 3.2) residual layout.  When every rank holds
+# the same values on the shared channels of the residual stream - which the partial
+# channel-reduce guarantees from the first layer on, if the stream entering the network is
+# tied - those channels are ONE variable stored once:
+#     Rs [T, S]  shared part          Rp [t, T, h - S]  private part of every rank
+# The forward is the same map as rowpar_forward applied to R[m] = [Rs | Rp[m]]; the backward
+# below is the gradient of that map with Rs (and Hns) treated as single variables, written
+# out on its own (it does not go through rowpar_backward).
+# --------------------------------------------------------------------------
+def rowpar_forward_compact(Y, W, Rs, Rp, gamma, beta=None, *, S: int, alpha: float = 1.0,
+                           eps: float = 1e-5, norm: int = RMSNORM) -> dict:
+    Zt = rank_partials(Y, W)                                       # F1
+    t, T, h = Zt.shape
+    Zs = np.zeros((T, S))                                          # F2: rank sum, m ascending
+    for m in range(t):
+        Zs = Zs + Zt[m, :, :S]
+    Hns = Zs + np.asarray(Rs, dtype=np.float64)                    # F4 on the shared channels, once
+    Hnp = alpha * Zt[:, :, S:] + np.asarray(Rp, dtype=np.float64)  # F3 + F4 on the private channels
+    X = np.empty((t, T, h))
+    rstd = np.empty((t, T))
+    mean = np.empty((t, T)) if norm == LAYERNORM else None
+    for m in range(t):                                             # F5: statistics over all h channels of rank m
+        row = np.concatenate([Hns, Hnp[m]], axis=1)
+        X[m], rstd[m], mu = norm_forward(row, gamma, beta, eps, norm)
+        if norm == LAYERNORM:
+            mean[m] = mu
+    return {"Hns": Hns, "Hnp": Hnp, "X": X, "rstd": rstd, "mean": mean}
+
+
+def rowpar_backward_compact(dX, dHns, dHnp, Y, W, Hns, Hnp, rstd, mean, gamma, *, S: int,
+                            alpha: float = 1.0, norm: int = RMSNORM) -> dict:
+    """Gradient of rowpar_forward_compact contracted with dX (through every rank's norm), dHns
+    (on the shared part of the outgoing stream, one variable) and dHnp (private parts).
+
+    Hns feeds the norm of EVERY rank, so its gradient collects all ranks' norm backward: that
+    rank sum is the backward partial channel-reduce (operation 'h' of Fig. 2b, after the norm
+    backward).  Because Hns = sum_m Zt[m][:, :S] + Rs, the same tensor is the gradient of Rs
+    and of the shared columns of every rank's Zt.
+    """
+    dX = np.asarray(dX, dtype=np.float64)
+    Hns = np.asarray(Hns, dtype=np.float64)
+    Hnp = np.asarray(Hnp, dtype=np.float64)
+    t, T, h = dX.shape
+    gs = np.zeros((T, S)) if dHns is None else np.asarray(dHns, dtype=np.float64).copy()
+    gp = np.empty((t, T, h - S))
+    dgamma = np.zeros(h)
+    dbeta = np.zeros(h) if norm == LAYERNORM else None
+    for m in range(t):
+        row = np.concatenate([Hns, Hnp[m]], axis=1)
+        mu = None if mean is None else np.asarray(mean, dtype=np.float64)[m]
+        n_m = norm_backward(dX[m], row, np.asarray(rstd, dtype=np.float64)[m], mu, gamma, norm)   # B1
+        gs = gs + n_m[:, :S]                                   # B4, m ascending, in full precision
+        gp[m] = n_m[:, S:]
+        dgamma += np.sum(dX[m] * normalized(row, np.asarray(rstd, dtype=np.float64)[m], mu, norm), axis=0)   # B3
+        if norm == LAYERNORM:
+            dbeta += np.sum(dX[m], axis=0)
+    if dHnp is not None:
+        gp = gp + np.asarray(dHnp, dtype=np.float64)
+    dZt = np.empty((t, T, h))
+    for m in range(t):
+        dZt[m, :, :S] = gs
+        dZt[m, :, S:] = alpha * gp[m]                          # private channels carry alpha
+    return {"dRs": gs, "dRp": gp, "dZt": dZt, "dY": data_gradient(dZt, W), "dW": weight_gradient(dZt, Y),
+            "dgamma": dgamma, "dbeta": dbeta}
+
+
+def block_forward_compact(Y_attn, W_o, Y_mlp, W_down, R0s, R0p, gamma1, gamma2, beta1=None, beta2=None, *,
+                          S: int, alpha: float = 1.0, eps: float = 1e-5, norm: int = RMSNORM) -> dict:
+    f1 = rowpar_forward_compact(Y_attn, W_o, R0s, R0p, gamma1, beta1, S=S, alpha=alpha, eps=eps, norm=norm)
+    f2 = rowpar_forward_compact(Y_mlp, W_down, f1["Hns"], f1["Hnp"], gamma2, beta2, S=S, alpha=alpha, eps=eps, norm=norm)
+    return {"Hn1s": f1["Hns"], "Hn1p": f1["Hnp"], "X1": f1["X"], "rstd1": f1["rstd"], "mean1": f1["mean"],
+            "Hn2s": f2["Hns"], "Hn2p": f2["Hnp"], "X2": f2["X"], "rstd2": f2["rstd"], "mean2": f2["mean"]}
+
+
+def block_backward_compact(dX1, dX2, dHn2s, dHn2p, Y_attn, W_o, Y_mlp, W_down, Hn1s, Hn1p, rstd1, mean1,
+                           Hn2s, Hn2p, rstd2, mean2, gamma1, gamma2, *, S: int, alpha: float = 1.0,
+                           norm: int = RMSNORM) -> dict:
+    b2 = rowpar_backward_compact(dX2, dHn2s, dHn2p, Y_mlp, W_down, Hn2s, Hn2p, rstd2, mean2, gamma2,
+                                 S=S, alpha=alpha, norm=norm)
+    b1 = rowpar_backward_compact(dX1, b2["dRs"], b2["dRp"], Y_attn, W_o, Hn1s, Hn1p, rstd1, mean1, gamma1,
+                                 S=S, alpha=alpha, norm=norm)
+    return {"dY_attn": b1["dY"], "dW_o": b1["dW"], "dY_mlp": b2["dY"], "dW_down": b2["dW"],
+            "dR0s": b1["dRs"], "dR0p": b1["dRp"], "dHn1s": b2["dRs"], "dHn1p": b2["dRp"],
+            "dgamma1": b1["dgamma"], "dgamma2": b2["dgamma"], "dbeta1": b1["dbeta"], "dbeta2": b2["dbeta"]}
 
 
 # --------------------------------------------------------------------------

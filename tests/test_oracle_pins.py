@@ -335,6 +335,122 @@ def test_block_chains_through_residual_and_matches_finite_differences():
         assert np.abs(num - b[gname]).max() / max(1.0, np.abs(num).max()) < 2e-7, name
 
 
+# ---------------------------------------------------------------- compact residual layout
+def _rand_compact(rng, t, T, h, K_r, S):
+    return {"Y": rng.standard_normal((t, T, K_r)), "W": rng.standard_normal((t, h, K_r)) * 0.3,
+            "Rs": rng.standard_normal((T, S)), "Rp": rng.standard_normal((t, T, h - S)),
+            "gamma": 1.0 + 0.2 * rng.standard_normal(h), "beta": 0.1 * rng.standard_normal(h)}
+
+
+@pytest.mark.parametrize("norm", [O.RMSNORM, O.LAYERNORM])
+def test_compact_forward_is_per_rank_forward_on_tied_residual(norm):
+    # the compact form is the per-rank map evaluated on R[m] = [Rs | Rp[m]]
+    rng = _rng(21)
+    t, T, h, K_r, S, alpha = 3, 5, 12, 4, 8, math.sqrt(3.0)
+    d = _rand_compact(rng, t, T, h, K_r, S)
+    R = np.concatenate([np.broadcast_to(d["Rs"], (t, T, S)), d["Rp"]], axis=2)
+    ref = O.rowpar_forward(d["Y"], d["W"], R, d["gamma"], d["beta"], S=S, alpha=alpha, norm=norm)
+    out = O.rowpar_forward_compact(d["Y"], d["W"], d["Rs"], d["Rp"], d["gamma"], d["beta"], S=S, alpha=alpha, norm=norm)
+    for m in range(t):
+        np.testing.assert_allclose(out["Hns"], ref["Hn"][m, :, :S], rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(out["Hnp"], ref["Hn"][:, :, S:], rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(out["X"], ref["X"], rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(out["rstd"], ref["rstd"], rtol=1e-13)
+
+
+@pytest.mark.parametrize("norm", [O.RMSNORM, O.LAYERNORM])
+@pytest.mark.parametrize("S,alpha", [(0, 2.0), (4, 1.0), (4, math.sqrt(3.0)), (6, 1.7)])
+def test_compact_backward_matches_finite_differences(norm, S, alpha):
+    rng = _rng(22)
+    t, T, h, K_r = 3, 2, 6, 4
+    d = _rand_compact(rng, t, T, h, K_r, S)
+    Gx, Gs, Gp = rng.standard_normal((t, T, h)), rng.standard_normal((T, S)), rng.standard_normal((t, T, h - S))
+
+    def loss():
+        o = O.rowpar_forward_compact(d["Y"], d["W"], d["Rs"], d["Rp"], d["gamma"], d["beta"], S=S, alpha=alpha, norm=norm)
+        return float(np.sum(Gx * o["X"]) + np.sum(Gs * o["Hns"]) + np.sum(Gp * o["Hnp"]))
+
+    f = O.rowpar_forward_compact(d["Y"], d["W"], d["Rs"], d["Rp"], d["gamma"], d["beta"], S=S, alpha=alpha, norm=norm)
+    b = O.rowpar_backward_compact(Gx, Gs, Gp, d["Y"], d["W"], f["Hns"], f["Hnp"], f["rstd"], f["mean"], d["gamma"],
+                                  S=S, alpha=alpha, norm=norm)
+    checks = [("Y", b["dY"]), ("W", b["dW"]), ("Rs", b["dRs"]), ("Rp", b["dRp"]), ("gamma", b["dgamma"])]
+    if norm == O.LAYERNORM:
+        checks.append(("beta", b["dbeta"]))
+    step = 1e-6
+    for name, grad in checks:
+        if d[name].size == 0:
+            assert grad.size == 0
+            continue
+        num = np.zeros_like(d[name])
+        it = np.nditer(d[name], flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = d[name][idx]
+            d[name][idx] = keep + step; lp = loss()
+            d[name][idx] = keep - step; lm = loss()
+            d[name][idx] = keep
+            num[idx] = (lp - lm) / (2 * step)
+        assert np.abs(num - grad).max() / max(1.0, np.abs(num).max()) < 2e-7, name
+
+
+def test_compact_backward_is_rank_sum_of_per_rank_backward():
+    # per-rank copies of a tied variable: the gradient of the single variable is the sum of the
+    # copies' gradients, for ANY split of the upstream dHns over the copies
+    rng = _rng(23)
+    t, T, h, K_r, S, alpha = 4, 3, 16, 5, 8, 2.0
+    d = _rand_compact(rng, t, T, h, K_r, S)
+    Gx, Gs, Gp = rng.standard_normal((t, T, h)), rng.standard_normal((T, S)), rng.standard_normal((t, T, h - S))
+    f = O.rowpar_forward_compact(d["Y"], d["W"], d["Rs"], d["Rp"], d["gamma"], None, S=S, alpha=alpha)
+    b = O.rowpar_backward_compact(Gx, Gs, Gp, d["Y"], d["W"], f["Hns"], f["Hnp"], f["rstd"], None, d["gamma"], S=S, alpha=alpha)
+    split = rng.standard_normal((t, 1, 1)); split = split / split.sum()
+    dHn = np.concatenate([split * Gs[None], Gp], axis=2)
+    Hn = np.concatenate([np.broadcast_to(f["Hns"], (t, T, S)), f["Hnp"]], axis=2)
+    ref = O.rowpar_backward(Gx, dHn, d["Y"], d["W"], Hn, f["rstd"], None, d["gamma"], S=S, alpha=alpha)
+    np.testing.assert_allclose(b["dRs"], ref["dR"][:, :, :S].sum(0), rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(b["dRp"], ref["dR"][:, :, S:], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(b["dY"], ref["dY"], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(b["dW"], ref["dW"], rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(b["dgamma"], ref["dgamma"], rtol=1e-11, atol=1e-12)
+
+
+def test_compact_block_matches_finite_differences():
+    rng = _rng(24)
+    t, T, h, ka, km, S, alpha = 2, 2, 4, 2, 3, 2, math.sqrt(2.0)
+    inp = {"Y_attn": rng.standard_normal((t, T, ka)), "W_o": rng.standard_normal((t, h, ka)) * 0.4,
+           "Y_mlp": rng.standard_normal((t, T, km)), "W_down": rng.standard_normal((t, h, km)) * 0.4,
+           "R0s": rng.standard_normal((T, S)), "R0p": rng.standard_normal((t, T, h - S)),
+           "gamma1": 1 + 0.1 * rng.standard_normal(h), "gamma2": 1 + 0.1 * rng.standard_normal(h)}
+    G1, G2 = rng.standard_normal((t, T, h)), rng.standard_normal((t, T, h))
+    Gs, Gp = rng.standard_normal((T, S)), rng.standard_normal((t, T, h - S))
+
+    def fwd():
+        return O.block_forward_compact(inp["Y_attn"], inp["W_o"], inp["Y_mlp"], inp["W_down"], inp["R0s"], inp["R0p"],
+                                       inp["gamma1"], inp["gamma2"], S=S, alpha=alpha)
+
+    def loss():
+        o = fwd()
+        return float(np.sum(G1 * o["X1"]) + np.sum(G2 * o["X2"]) + np.sum(Gs * o["Hn2s"]) + np.sum(Gp * o["Hn2p"]))
+
+    o = fwd()
+    b = O.block_backward_compact(G1, G2, Gs, Gp, inp["Y_attn"], inp["W_o"], inp["Y_mlp"], inp["W_down"], o["Hn1s"],
+                                 o["Hn1p"], o["rstd1"], None, o["Hn2s"], o["Hn2p"], o["rstd2"], None, inp["gamma1"],
+                                 inp["gamma2"], S=S, alpha=alpha)
+    pairs = [("Y_attn", "dY_attn"), ("W_o", "dW_o"), ("Y_mlp", "dY_mlp"), ("W_down", "dW_down"),
+             ("R0s", "dR0s"), ("R0p", "dR0p"), ("gamma1", "dgamma1"), ("gamma2", "dgamma2")]
+    step = 1e-6
+    for name, gname in pairs:
+        num = np.zeros_like(inp[name])
+        it = np.nditer(inp[name], flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = inp[name][idx]
+            inp[name][idx] = keep + step; lp = loss()
+            inp[name][idx] = keep - step; lm = loss()
+            inp[name][idx] = keep
+            num[idx] = (lp - lm) / (2 * step)
+        assert np.abs(num - b[gname]).max() / max(1.0, np.abs(num).max()) < 2e-7, name
+
+
 # ---------------------------------------------------------------- analytic bytes
 def test_allreduce_bytes_closed_forms():
     # Appendix C: per block forward the payload is P(p) = 2 s h p activations per device (two reduces).
