@@ -219,6 +219,70 @@ caat_status caat_block_backward(const caat_ctx *ctx, int tokens,
                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Compact residual layout ("logical devices" on one GPU, Section 3.2).
+ *
+ * The partial channel-reduce makes the first S channels of the layer output identical on
+ * every rank (Eq. A3, l < S), so when the residual entering the first layer is tied on those
+ * channels the shared part of the residual stream is ONE tensor for the whole network.  These
+ * entry points store it once:
+ *     shared part   [T, S]          dtype   (Rs, Hns, dHns, dRs)
+ *     private part  [t, T, h - S]   dtype   (Rp, Hnp, dHnp, dRp), column l of rank m at l - S
+ * Same arithmetic as caat_rowpar_forward / _backward applied to R[m] = [Rs | Rp[m]]; X, rstd,
+ * mean stay per rank ([t, T, h], [t, T]): the statistics of rank m cover its private
+ * channels too, so X differs between ranks on the shared channels as well.
+ *
+ * Backward: Hns is read by every rank's norm, so its gradient collects all ranks' norm
+ * backward plus the gradient arriving on the single shared stream,
+ *     gs[i,l]   = dHns[i,l] + sum_m NormBwd(dX[m])[i,l]      (l <  S; fp32 sum, m ascending)
+ *     gp[m,i,l] = dHnp[m,i,l] + NormBwd(dX[m])[i,l]          (l >= S)
+ *     dRs = gs,  dRp = gp,  dZt[m] = [gs | alpha * gp[m]],  dY, dW, dgamma, dbeta as above.
+ * gs is the backward partial channel-reduce (operation "h" of Fig. 2b) and the shared
+ * residual gradient at once.  dHns and dHnp are both given or both NULL.
+ *
+ * Requires S % 8 == 0 (CAAT_EUNSUPPORTED otherwise).  A part that is empty (S = 0 or S = h)
+ * may be passed as NULL.  Workspace sizes are those of the per-rank entry points.
+ */
+caat_status caat_rowpar_forward_compact(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                        const void *Y, const void *W,
+                                        const void *Rs, const void *Rp,
+                                        const void *gamma, const void *beta,
+                                        void *Hns, void *Hnp, void *X, float *rstd, float *mean,
+                                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+caat_status caat_rowpar_backward_compact(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                         const void *dX, const void *dHns, const void *dHnp,
+                                         const void *Y, const void *W,
+                                         const void *Hns, const void *Hnp,
+                                         const float *rstd, const float *mean, const void *gamma,
+                                         void *dY, float *dW, void *dRs, void *dRp,
+                                         float *dgamma, float *dbeta,
+                                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+/* Block (attention-out then MLP-down) on the compact stream; dHn1s / dHn1p are outputs
+ * (the residual gradient between the two layers), as dHn1 in caat_block_backward. */
+caat_status caat_block_forward_compact(const caat_ctx *ctx, int tokens,
+                                       const void *Y_attn, const void *W_o,
+                                       const void *Y_mlp, const void *W_down,
+                                       const void *R0s, const void *R0p,
+                                       const void *gamma1, const void *beta1,
+                                       const void *gamma2, const void *beta2,
+                                       void *Hn1s, void *Hn1p, void *X1, float *rstd1, float *mean1,
+                                       void *Hn2s, void *Hn2p, void *X2, float *rstd2, float *mean2,
+                                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+caat_status caat_block_backward_compact(const caat_ctx *ctx, int tokens,
+                                        const void *dX1, const void *dX2,
+                                        const void *dHn2s, const void *dHn2p,
+                                        const void *Y_attn, const void *W_o,
+                                        const void *Y_mlp, const void *W_down,
+                                        const void *Hn1s, const void *Hn1p,
+                                        const float *rstd1, const float *mean1,
+                                        const void *Hn2s, const void *Hn2p,
+                                        const float *rstd2, const float *mean2,
+                                        const void *gamma1, const void *gamma2,
+                                        void *dY_attn, float *dW_o, void *dY_mlp, float *dW_down,
+                                        void *dR0s, void *dR0p, void *dHn1s, void *dHn1p,
+                                        float *dgamma1, float *dbeta1, float *dgamma2, float *dbeta2,
+                                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Analytic bytes ONE partial channel-reduce would move on a real t-device system
  * (Appendix C: each device sends and receives tokens*h*p activations per reduce;
  * Appendix D: all-reduce = reduce-scatter + all-gather, traffic cut by 100(1-p) %).

@@ -44,6 +44,10 @@ _sigs = {
     "caat_rowpar_backward": (c_int, [_P, c_int, c_int] + [_P] * 13 + [_P, c_size_t, _P]),
     "caat_block_forward": (c_int, [_P, c_int] + [_P] * 17 + [_P, c_size_t, _P]),
     "caat_block_backward": (c_int, [_P, c_int] + [_P] * 25 + [_P, c_size_t, _P]),
+    "caat_rowpar_forward_compact": (c_int, [_P, c_int, c_int] + [_P] * 11 + [_P, c_size_t, _P]),
+    "caat_rowpar_backward_compact": (c_int, [_P, c_int, c_int] + [_P] * 16 + [_P, c_size_t, _P]),
+    "caat_block_forward_compact": (c_int, [_P, c_int] + [_P] * 20 + [_P, c_size_t, _P]),
+    "caat_block_backward_compact": (c_int, [_P, c_int] + [_P] * 30 + [_P, c_size_t, _P]),
     "caat_allreduce_bytes": (c_int, [_P, c_int, c_int] + [POINTER(c_ulonglong)] * 3),
     "caat_last_device_status": (c_int, [_P, _P]),
     "caat_kernel_launches": (c_ulonglong, []),
@@ -92,6 +96,8 @@ def _ptr(x, dtype=None, shape=None, name="tensor"):
         raise TypeError(f"{name}: expected {dtype}, got {x.dtype}")
     if shape is not None and tuple(x.shape) != tuple(shape):
         raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(x.shape)}")
+    if x.numel() == 0:
+        return None
     return x.data_ptr()
 
 
@@ -234,6 +240,80 @@ class Context:
             _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
             _stream())
         _check(st, "caat_block_backward")
+
+    # ---- compact residual layout: shared part [T, S] once, private parts [t, T, h - S]
+    def rowpar_forward_compact(self, layer, tokens, Y, W, Rs, Rp, gamma, beta, Hns, Hnp, X, rstd, mean, workspace):
+        td, t, h, k, S = self.torch_dtype, self.t, self.h, self.k_r(layer), self.shared_channels
+        sh, pr, f32 = (tokens, S), (t, tokens, h - S), torch.float32
+        st = lib.caat_rowpar_forward_compact(
+            self._h, layer, tokens,
+            _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"), _ptr(Rs, td, sh, "Rs"), _ptr(Rp, td, pr, "Rp"),
+            _ptr(gamma, td, (h,), "gamma"), _ptr(beta, td, (h,), "beta"),
+            _ptr(Hns, td, sh, "Hns"), _ptr(Hnp, td, pr, "Hnp"), _ptr(X, td, (t, tokens, h), "X"),
+            _ptr(rstd, f32, (t, tokens), "rstd"), _ptr(mean, f32, (t, tokens), "mean"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_rowpar_forward_compact")
+
+    def rowpar_backward_compact(self, layer, tokens, dX, dHns, dHnp, Y, W, Hns, Hnp, rstd, mean, gamma, dY, dW,
+                                dRs, dRp, dgamma, dbeta, workspace):
+        td, t, h, k, S = self.torch_dtype, self.t, self.h, self.k_r(layer), self.shared_channels
+        sh, pr, f32 = (tokens, S), (t, tokens, h - S), torch.float32
+        st = lib.caat_rowpar_backward_compact(
+            self._h, layer, tokens,
+            _ptr(dX, td, (t, tokens, h), "dX"), _ptr(dHns, td, sh, "dHns"), _ptr(dHnp, td, pr, "dHnp"),
+            _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"),
+            _ptr(Hns, td, sh, "Hns"), _ptr(Hnp, td, pr, "Hnp"),
+            _ptr(rstd, f32, (t, tokens), "rstd"), _ptr(mean, f32, (t, tokens), "mean"), _ptr(gamma, td, (h,), "gamma"),
+            _ptr(dY, td, (t, tokens, k), "dY"), _ptr(dW, f32, (t, h, k), "dW"),
+            _ptr(dRs, td, sh, "dRs"), _ptr(dRp, td, pr, "dRp"),
+            _ptr(dgamma, f32, (h,), "dgamma"), _ptr(dbeta, f32, (h,), "dbeta"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_rowpar_backward_compact")
+
+    def block_forward_compact(self, tokens, Y_attn, W_o, Y_mlp, W_down, R0s, R0p, gamma1, beta1, gamma2, beta2,
+                              Hn1s, Hn1p, X1, rstd1, mean1, Hn2s, Hn2p, X2, rstd2, mean2, workspace):
+        td, t, h, S = self.torch_dtype, self.t, self.h, self.shared_channels
+        ka, km = self.k_r(CAAT_ATTN_OUT), self.k_r(CAAT_MLP_DOWN)
+        sh, pr, act, st2, f32 = (tokens, S), (t, tokens, h - S), (t, tokens, h), (t, tokens), torch.float32
+        st = lib.caat_block_forward_compact(
+            self._h, tokens,
+            _ptr(Y_attn, td, (t, tokens, ka), "Y_attn"), _ptr(W_o, td, (t, h, ka), "W_o"),
+            _ptr(Y_mlp, td, (t, tokens, km), "Y_mlp"), _ptr(W_down, td, (t, h, km), "W_down"),
+            _ptr(R0s, td, sh, "R0s"), _ptr(R0p, td, pr, "R0p"),
+            _ptr(gamma1, td, (h,), "gamma1"), _ptr(beta1, td, (h,), "beta1"),
+            _ptr(gamma2, td, (h,), "gamma2"), _ptr(beta2, td, (h,), "beta2"),
+            _ptr(Hn1s, td, sh, "Hn1s"), _ptr(Hn1p, td, pr, "Hn1p"), _ptr(X1, td, act, "X1"),
+            _ptr(rstd1, f32, st2, "rstd1"), _ptr(mean1, f32, st2, "mean1"),
+            _ptr(Hn2s, td, sh, "Hn2s"), _ptr(Hn2p, td, pr, "Hn2p"), _ptr(X2, td, act, "X2"),
+            _ptr(rstd2, f32, st2, "rstd2"), _ptr(mean2, f32, st2, "mean2"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_block_forward_compact")
+
+    def block_backward_compact(self, tokens, dX1, dX2, dHn2s, dHn2p, Y_attn, W_o, Y_mlp, W_down, Hn1s, Hn1p, rstd1,
+                               mean1, Hn2s, Hn2p, rstd2, mean2, gamma1, gamma2, dY_attn, dW_o, dY_mlp, dW_down,
+                               dR0s, dR0p, dHn1s, dHn1p, dgamma1, dbeta1, dgamma2, dbeta2, workspace):
+        td, t, h, S = self.torch_dtype, self.t, self.h, self.shared_channels
+        ka, km = self.k_r(CAAT_ATTN_OUT), self.k_r(CAAT_MLP_DOWN)
+        sh, pr, act, st2, f32 = (tokens, S), (t, tokens, h - S), (t, tokens, h), (t, tokens), torch.float32
+        st = lib.caat_block_backward_compact(
+            self._h, tokens,
+            _ptr(dX1, td, act, "dX1"), _ptr(dX2, td, act, "dX2"), _ptr(dHn2s, td, sh, "dHn2s"), _ptr(dHn2p, td, pr, "dHn2p"),
+            _ptr(Y_attn, td, (t, tokens, ka), "Y_attn"), _ptr(W_o, td, (t, h, ka), "W_o"),
+            _ptr(Y_mlp, td, (t, tokens, km), "Y_mlp"), _ptr(W_down, td, (t, h, km), "W_down"),
+            _ptr(Hn1s, td, sh, "Hn1s"), _ptr(Hn1p, td, pr, "Hn1p"), _ptr(rstd1, f32, st2, "rstd1"), _ptr(mean1, f32, st2, "mean1"),
+            _ptr(Hn2s, td, sh, "Hn2s"), _ptr(Hn2p, td, pr, "Hn2p"), _ptr(rstd2, f32, st2, "rstd2"), _ptr(mean2, f32, st2, "mean2"),
+            _ptr(gamma1, td, (h,), "gamma1"), _ptr(gamma2, td, (h,), "gamma2"),
+            _ptr(dY_attn, td, (t, tokens, ka), "dY_attn"), _ptr(dW_o, f32, (t, h, ka), "dW_o"),
+            _ptr(dY_mlp, td, (t, tokens, km), "dY_mlp"), _ptr(dW_down, f32, (t, h, km), "dW_down"),
+            _ptr(dR0s, td, sh, "dR0s"), _ptr(dR0p, td, pr, "dR0p"), _ptr(dHn1s, td, sh, "dHn1s"), _ptr(dHn1p, td, pr, "dHn1p"),
+            _ptr(dgamma1, f32, (h,), "dgamma1"), _ptr(dbeta1, f32, (h,), "dbeta1"),
+            _ptr(dgamma2, f32, (h,), "dgamma2"), _ptr(dbeta2, f32, (h,), "dbeta2"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_block_backward_compact")
 
     # ---- buffer helpers (torch.empty only; no arithmetic)
     def alloc_workspace(self, nbytes: int, device="cuda"):

@@ -115,7 +115,9 @@ static caat_status check_common(const caat_ctx* ctx, caat_layer layer, int token
 // ---- forward of one layer ------------------------------------------------------
 static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void* Y, const void* W, const void* R,
                                 const void* gamma, const void* beta, void* Hn, void* X, float* rstd, float* mean,
-                                void* ws, cudaStream_t st) {
+                                void* ws, cudaStream_t st, int compact = 0, const void* Rs = nullptr,
+                                void* Hns = nullptr) {
+  // compact: R / Hn are the private parts [t, T, h - S], Rs / Hns the shared part [T, S] stored once
   const Scratch L = scratch_layout(ctx, K_r, T, 0);
   char* wsb = static_cast<char*>(ws);
   void* zs = wsb + L.zs_off;
@@ -124,7 +126,7 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
   const size_t e = elem_size(ctx->dtype);
   cudaError_t ce;
 
-  if (T <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r)) {
+  if (!compact && T <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r)) {
     // few tokens (decode): the weights dominate the traffic; stream them with swapped operands and
     // let the row kernel form the rank sum from fp32 per-rank partials
     float* zt = reinterpret_cast<float*>(wsb + L.zt_off);
@@ -166,6 +168,7 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
   }
   RowFwdArgs a{zs, zp, R, gamma, beta, Hn, X, rstd, mean, t, T, h, S, L.S_lo, L.S_hi, L.P,
                (float)ctx->alpha, (float)ctx->eps, ctx->norm};
+  a.compact = compact; a.Rs = Rs; a.Hns = Hns;
   ce = launch_rows_forward(a, ctx->dtype, ctx->direct_rows, st);
   if (ce != cudaSuccess) return cuda_fail(ce);
   return CAAT_OK;
@@ -175,10 +178,13 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
 static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void* dX, const void* dHn, const void* Y,
                                  const void* W, const void* Hn, const float* rstd, const float* mean,
                                  const void* gamma, void* dY, float* dW, void* dR, float* dgamma, float* dbeta,
-                                 void* ws, cudaStream_t st) {
+                                 void* ws, cudaStream_t st, int compact = 0, const void* Hns = nullptr,
+                                 const void* dHns = nullptr, void* dRs = nullptr) {
+  // compact: Hn / dHn / dR are the private parts; the shared residual gradient dRs [T, S] is at the
+  // same time the shared part of dZt, so the GEMMs read it where the caller wants it
   const Scratch L = scratch_layout(ctx, K_r, T, 1);
   char* wsb = static_cast<char*>(ws);
-  void* gs = wsb + L.zs_off;
+  void* gs = compact ? dRs : wsb + L.zs_off;
   void* zp = wsb + L.zp_off;
   const int t = ctx->t, h = ctx->h, S = ctx->S;
   const size_t e = elem_size(ctx->dtype);
@@ -187,6 +193,7 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
   RowBwdArgs a{dX, dHn, Hn, gamma, rstd, mean, dR, gs, zp,
                reinterpret_cast<float*>(wsb + L.dgpart_off), reinterpret_cast<float*>(wsb + L.dbpart_off),
                dgamma, dbeta, t, T, h, S, L.S_lo, L.S_hi, L.P, (float)ctx->alpha, ctx->norm};
+  a.compact = compact; a.Hns = Hns; a.dHns = dHns;
   ce = launch_rows_backward(a, ctx->dtype, ctx->direct_rows, st);
   if (ce != cudaSuccess) return cuda_fail(ce);
 
@@ -401,6 +408,90 @@ caat_status caat_block_backward(const caat_ctx* ctx, int tokens, const void* dX1
   if (s != CAAT_OK) return s;
   return caat_rowpar_backward(ctx, CAAT_ATTN_OUT, tokens, dX1, dHn1, Y_attn, W_o, Hn1, rstd1, mean1, gamma1,
                               dY_attn, dW_o, dR0, dgamma1, dbeta1, workspace, workspace_bytes, cuda_stream);
+}
+
+// ---- compact residual layout ---------------------------------------------------
+static caat_status check_compact(const caat_ctx* ctx, caat_layer layer, int tokens) {
+  caat_status s = check_common(ctx, layer, tokens);
+  if (s != CAAT_OK) return s;
+  if (ctx->S % kLayoutVec != 0) return CAAT_EUNSUPPORTED;   // rows of both parts must start on 16 bytes
+  return CAAT_OK;
+}
+
+caat_status caat_rowpar_forward_compact(const caat_ctx* ctx, caat_layer layer, int tokens, const void* Y,
+                                        const void* W, const void* Rs, const void* Rp, const void* gamma,
+                                        const void* beta, void* Hns, void* Hnp, void* X, float* rstd, float* mean,
+                                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = check_compact(ctx, layer, tokens);
+  if (s != CAAT_OK) return s;
+  const bool has_s = ctx->S > 0, has_p = ctx->S < ctx->h;
+  if (!Y || !W || !gamma || !X || !rstd) return CAAT_EINVAL;
+  if ((has_s && (!Rs || !Hns)) || (has_p && (!Rp || !Hnp))) return CAAT_EINVAL;
+  if (ctx->norm == 1 && !mean) return CAAT_EINVAL;
+  const void* ptrs[] = {Y, W, Rs, Rp, gamma, beta, Hns, Hnp, X, rstd, mean, workspace};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  const int K_r = layer_kr(ctx, layer);
+  if (!workspace || workspace_bytes < scratch_layout(ctx, K_r, tokens, 0).total) return CAAT_EWORKSPACE;
+  return forward_impl(ctx, K_r, tokens, Y, W, Rp, gamma, beta, Hnp, X, rstd, mean, workspace,
+                      static_cast<cudaStream_t>(cuda_stream), 1, Rs, Hns);
+}
+
+caat_status caat_rowpar_backward_compact(const caat_ctx* ctx, caat_layer layer, int tokens, const void* dX,
+                                         const void* dHns, const void* dHnp, const void* Y, const void* W,
+                                         const void* Hns, const void* Hnp, const float* rstd, const float* mean,
+                                         const void* gamma, void* dY, float* dW, void* dRs, void* dRp, float* dgamma,
+                                         float* dbeta, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = check_compact(ctx, layer, tokens);
+  if (s != CAAT_OK) return s;
+  const bool has_s = ctx->S > 0, has_p = ctx->S < ctx->h;
+  if (!dX || !Y || !W || !rstd || !gamma || !dY || !dW || !dgamma) return CAAT_EINVAL;
+  if ((has_s && (!Hns || !dRs)) || (has_p && (!Hnp || !dRp))) return CAAT_EINVAL;
+  // the gradient on the outgoing stream is given for both parts or for neither
+  const bool any_dh = (has_s && dHns) || (has_p && dHnp);
+  if (any_dh && ((has_s && !dHns) || (has_p && !dHnp))) return CAAT_EINVAL;
+  if (ctx->norm == 1 && (!mean || !dbeta)) return CAAT_EINVAL;
+  const void* ptrs[] = {dX, dHns, dHnp, Y, W, Hns, Hnp, rstd, mean, gamma, dY, dW, dRs, dRp, dgamma, dbeta, workspace};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  const int K_r = layer_kr(ctx, layer);
+  if (!workspace || workspace_bytes < scratch_layout(ctx, K_r, tokens, 1).total) return CAAT_EWORKSPACE;
+  // "a gradient is given" is one flag inside the kernels: an absent (empty) part borrows the other pointer
+  const void* dh_p = any_dh ? (has_p ? dHnp : dHns) : nullptr;
+  const void* dh_s = any_dh ? (has_s ? dHns : dHnp) : nullptr;
+  return backward_impl(ctx, K_r, tokens, dX, dh_p, Y, W, Hnp, rstd, mean, gamma, dY, dW, dRp, dgamma, dbeta, workspace,
+                       static_cast<cudaStream_t>(cuda_stream), 1, Hns, dh_s, dRs);
+}
+
+caat_status caat_block_forward_compact(const caat_ctx* ctx, int tokens, const void* Y_attn, const void* W_o,
+                                       const void* Y_mlp, const void* W_down, const void* R0s, const void* R0p,
+                                       const void* gamma1, const void* beta1, const void* gamma2, const void* beta2,
+                                       void* Hn1s, void* Hn1p, void* X1, float* rstd1, float* mean1, void* Hn2s,
+                                       void* Hn2p, void* X2, float* rstd2, float* mean2, void* workspace,
+                                       size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = caat_rowpar_forward_compact(ctx, CAAT_ATTN_OUT, tokens, Y_attn, W_o, R0s, R0p, gamma1, beta1, Hn1s,
+                                              Hn1p, X1, rstd1, mean1, workspace, workspace_bytes, cuda_stream);
+  if (s != CAAT_OK) return s;
+  return caat_rowpar_forward_compact(ctx, CAAT_MLP_DOWN, tokens, Y_mlp, W_down, Hn1s, Hn1p, gamma2, beta2, Hn2s, Hn2p,
+                                     X2, rstd2, mean2, workspace, workspace_bytes, cuda_stream);
+}
+
+caat_status caat_block_backward_compact(const caat_ctx* ctx, int tokens, const void* dX1, const void* dX2,
+                                        const void* dHn2s, const void* dHn2p, const void* Y_attn, const void* W_o,
+                                        const void* Y_mlp, const void* W_down, const void* Hn1s, const void* Hn1p,
+                                        const float* rstd1, const float* mean1, const void* Hn2s, const void* Hn2p,
+                                        const float* rstd2, const float* mean2, const void* gamma1,
+                                        const void* gamma2, void* dY_attn, float* dW_o, void* dY_mlp, float* dW_down,
+                                        void* dR0s, void* dR0p, void* dHn1s, void* dHn1p, float* dgamma1,
+                                        float* dbeta1, float* dgamma2, float* dbeta2, void* workspace,
+                                        size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = caat_rowpar_backward_compact(ctx, CAAT_MLP_DOWN, tokens, dX2, dHn2s, dHn2p, Y_mlp, W_down, Hn2s, Hn2p,
+                                               rstd2, mean2, gamma2, dY_mlp, dW_down, dHn1s, dHn1p, dgamma2, dbeta2,
+                                               workspace, workspace_bytes, cuda_stream);
+  if (s != CAAT_OK) return s;
+  return caat_rowpar_backward_compact(ctx, CAAT_ATTN_OUT, tokens, dX1, dHn1s, dHn1p, Y_attn, W_o, Hn1s, Hn1p, rstd1,
+                                      mean1, gamma1, dY_attn, dW_o, dR0s, dR0p, dgamma1, dbeta1, workspace,
+                                      workspace_bytes, cuda_stream);
 }
 
 caat_status caat_allreduce_bytes(const caat_ctx* ctx, int tokens, int elem_bytes, unsigned long long* payload,

@@ -104,6 +104,11 @@ struct RowFwdArgs {
   int t, T, h, S, S_lo, S_hi, P;
   float alpha, eps;
   int norm;
+  // compact residual layout (S a multiple of 8, so S_lo = S_hi = S): the shared channels of the
+  // stream exist once, Rs / Hns [T, S]; R / Hn then hold the private parts [t, T, P]
+  int compact;
+  const void* Rs;
+  void* Hns;
 };
 // direct: 0 = automatic (warp-per-token kernels for short rows, else the bulk-copy staged kernels
 // whenever a ring of at least two stages fits in shared memory), 1 = plain-load kernels,
@@ -136,6 +141,10 @@ struct RowBwdArgs {
   int t, T, h, S, S_lo, S_hi, P;
   float alpha;
   int norm;
+  // compact residual layout: Hns / dHns [T, S] exist once; Hn, dHn, dR hold the private parts
+  // [t, T, P]; the shared residual gradient is gs itself (dRs = dZt on the shared channels)
+  int compact;
+  const void *Hns, *dHns;
 };
 cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
 cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,

@@ -25,7 +25,8 @@ namespace {
 using namespace rows;
 
 // ------------------------------------------------------------------ forward
-template <typename T_, int CPT, bool LN>
+// CL: compact residual layout (shared part of R / Hn stored once, [T, S]; private parts [t, T, P])
+template <typename T_, int CPT, bool LN, bool CL>
 __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_forward_kernel(const RowFwdArgs a) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
@@ -55,10 +56,17 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_forward_kernel(con
 #pragma unroll
     for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; bet[j][e] = 0.f; zs[j][e] = 0.f; }
     const long long off_h = (i * a.h + col[j]) * ES;
-    pR[j] = static_cast<const char*>(a.R) + off_h;
-    pHn[j] = static_cast<char*>(a.Hn) + off_h;
+    const long long off_p = (i * a.P + (col[j] - a.S_lo)) * ES;
+    if (CL) {
+      const long long off_s = (i * a.S_hi + col[j]) * ES;
+      pR[j] = cls[j] == 0 ? static_cast<const char*>(a.Rs) + off_s : static_cast<const char*>(a.R) + off_p;
+      pHn[j] = cls[j] == 0 ? static_cast<char*>(a.Hns) + off_s : static_cast<char*>(a.Hn) + off_p;
+    } else {
+      pR[j] = static_cast<const char*>(a.R) + off_h;
+      pHn[j] = static_cast<char*>(a.Hn) + off_h;
+    }
     pX[j] = static_cast<char*>(a.X) + off_h;
-    pZ[j] = static_cast<const char*>(a.zp) + (i * a.P + (col[j] - a.S_lo)) * ES;
+    pZ[j] = static_cast<const char*>(a.zp) + off_p;
     if (act[j]) {
       V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
       if (LN && a.beta) V_::unpack(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
@@ -79,10 +87,11 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_forward_kernel(con
     raw nR[CPT], nZ[CPT];
 #pragma unroll
     for (int j = 0; j < CPT; ++j) {   // next rank's loads go out before this rank's barrier
-      pR[j] += rank_h;
+      pR[j] += CL ? rank_p : rank_h;      // (compact, shared chunk: the pointer is not used again)
       pZ[j] += rank_p;
       const bool more = act[j] && (m + 1 < a.t);
-      nR[j] = more ? ldg<raw>(pR[j]) : zero_raw<raw>();
+      if (CL && cls[j] == 0) nR[j] = rR[j];   // the shared residual is the same for every rank
+      else nR[j] = more ? ldg<raw>(pR[j]) : zero_raw<raw>();
       nZ[j] = (more && cls[j] != 0) ? ldg<raw>(pZ[j]) : zero_raw<raw>();
     }
 
@@ -104,8 +113,8 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_forward_kernel(con
 #pragma unroll
         for (int e = 0; e < V; ++e) hn[j][e] = (col[j] + e < a.S ? zs[j][e] : a.alpha * zp[e]) + r[e];
       }
-      if (act[j]) stg<raw>(pHn[j], V_::pack(hn[j]));
-      pHn[j] += rank_h;
+      if (act[j] && !(CL && cls[j] == 0 && m > 0)) stg<raw>(pHn[j], V_::pack(hn[j]));
+      pHn[j] += CL ? rank_p : rank_h;
 #pragma unroll
       for (int e = 0; e < V; ++e) st[0] = LN ? st[0] + hn[j][e] : fmaf(hn[j][e], hn[j][e], st[0]);
     }
@@ -149,7 +158,7 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_forward_kernel(con
 }
 
 // ------------------------------------------------------------------ backward
-template <typename T_, int CPT, bool LN>
+template <typename T_, int CPT, bool LN, bool CL>
 __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(const RowBwdArgs a, int ngroups) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
@@ -190,11 +199,19 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
     for (int j = 0; j < CPT; ++j) {
       act[j] = valid && colok[j];
       const long long off_h = (i * a.h + col[j]) * ES;
+      const long long off_p = (i * a.P + (col[j] - a.S_lo)) * ES;
       pdX[j] = static_cast<const char*>(a.dX) + off_h;
-      pHn[j] = static_cast<const char*>(a.Hn) + off_h;
-      pdH[j] = static_cast<const char*>(a.dHn) + off_h;
-      pdR[j] = static_cast<char*>(a.dR) + off_h;
-      pZ[j] = static_cast<char*>(a.zp) + (i * a.P + (col[j] - a.S_lo)) * ES;
+      if (CL) {
+        const long long off_s = (i * a.S_hi + col[j]) * ES;
+        pHn[j] = cls[j] == 0 ? static_cast<const char*>(a.Hns) + off_s : static_cast<const char*>(a.Hn) + off_p;
+        pdH[j] = cls[j] == 0 ? static_cast<const char*>(a.dHns) + off_s : static_cast<const char*>(a.dHn) + off_p;
+        pdR[j] = static_cast<char*>(a.dR) + off_p;
+      } else {
+        pHn[j] = static_cast<const char*>(a.Hn) + off_h;
+        pdH[j] = static_cast<const char*>(a.dHn) + off_h;
+        pdR[j] = static_cast<char*>(a.dR) + off_h;
+      }
+      pZ[j] = static_cast<char*>(a.zp) + off_p;
       rdX[j] = act[j] ? ldg<raw>(pdX[j]) : zero_raw<raw>();
       rHn[j] = act[j] ? ldg<raw>(pHn[j]) : zero_raw<raw>();
       rdH[j] = (act[j] && has_dh) ? ldg<raw>(pdH[j]) : zero_raw<raw>();
@@ -206,9 +223,14 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
 
     float gsum[CPT][V];
 #pragma unroll
-    for (int j = 0; j < CPT; ++j)
+    for (int j = 0; j < CPT; ++j) {
 #pragma unroll
       for (int e = 0; e < V; ++e) gsum[j][e] = 0.f;
+      if (CL && cls[j] == 0) {   // the gradient on the single shared stream enters the rank sum once
+        V_::unpack(rdH[j], gsum[j]);
+        rdH[j] = zero_raw<raw>();
+      }
+    }
 
     for (int m = 0; m < a.t; ++m) {
       raw ndX[CPT], nHn[CPT], ndH[CPT];
@@ -219,11 +241,16 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
       const float mu_n = (LN && valid && more_rank) ? *mean_p : 0.f;
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
-        pdX[j] += rank_h; pHn[j] += rank_h; pdH[j] += rank_h;
+        pdX[j] += rank_h; pHn[j] += CL ? rank_p : rank_h; pdH[j] += CL ? rank_p : rank_h;
         const bool more = act[j] && more_rank;
         ndX[j] = more ? ldg<raw>(pdX[j]) : zero_raw<raw>();
-        nHn[j] = more ? ldg<raw>(pHn[j]) : zero_raw<raw>();
-        ndH[j] = (more && has_dh) ? ldg<raw>(pdH[j]) : zero_raw<raw>();
+        if (CL && cls[j] == 0) {
+          nHn[j] = rHn[j];                  // one shared row for every rank
+          ndH[j] = zero_raw<raw>();
+        } else {
+          nHn[j] = more ? ldg<raw>(pHn[j]) : zero_raw<raw>();
+          ndH[j] = (more && has_dh) ? ldg<raw>(pdH[j]) : zero_raw<raw>();
+        }
       }
 
       float xh[CPT][V], dxh[CPT][V];
@@ -258,8 +285,8 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
           if (LN) tt -= c1;
           g[e] = fmaf(rs_c, tt, dh[e]);
         }
-        if (act[j]) stg<raw>(pdR[j], V_::pack(g));
-        pdR[j] += rank_h;
+        if (act[j] && !(CL && cls[j] == 0)) stg<raw>(pdR[j], V_::pack(g));
+        pdR[j] += CL ? rank_p : rank_h;
         if (cls[j] == 0) {
 #pragma unroll
           for (int e = 0; e < V; ++e) gsum[j][e] += g[e];          // fp32 rank sum, m ascending
@@ -440,30 +467,30 @@ __global__ void __launch_bounds__(1024) reduce_partials_kernel(const float* __re
   }
 }
 
-template <typename T_, bool LN>
+template <typename T_, bool LN, bool CL>
 cudaError_t launch_fwd_t(const RowFwdArgs& a, const RowGeom& g, cudaStream_t st) {
   const dim3 block(g.TX, g.TY);
   const dim3 grid((a.T + g.TY - 1) / g.TY);
   LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
   switch (g.CPT) {
-    case 1: rows_forward_kernel<T_, 1, LN><<<grid, block, g.smem_fwd, st>>>(a); break;
-    case 2: rows_forward_kernel<T_, 2, LN><<<grid, block, g.smem_fwd, st>>>(a); break;
-    case 4: rows_forward_kernel<T_, 4, LN><<<grid, block, g.smem_fwd, st>>>(a); break;
+    case 1: rows_forward_kernel<T_, 1, LN, CL><<<grid, block, g.smem_fwd, st>>>(a); break;
+    case 2: rows_forward_kernel<T_, 2, LN, CL><<<grid, block, g.smem_fwd, st>>>(a); break;
+    case 4: rows_forward_kernel<T_, 4, LN, CL><<<grid, block, g.smem_fwd, st>>>(a); break;
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
 }
 
-template <typename T_, bool LN>
+template <typename T_, bool LN, bool CL>
 cudaError_t launch_bwd_t(const RowBwdArgs& a, const RowGeom& g, int rows, cudaStream_t st) {
   const dim3 block(g.TX, g.TY);
   const int ngroups = (a.T + g.TY - 1) / g.TY;
   const dim3 grid(rows);
   LaunchScope scope(CAAT_K_ROWS_BACKWARD, st);
   switch (g.CPT) {
-    case 1: rows_backward_kernel<T_, 1, LN><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
-    case 2: rows_backward_kernel<T_, 2, LN><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
-    case 4: rows_backward_kernel<T_, 4, LN><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
+    case 1: rows_backward_kernel<T_, 1, LN, CL><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
+    case 2: rows_backward_kernel<T_, 2, LN, CL><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
+    case 4: rows_backward_kernel<T_, 4, LN, CL><<<grid, block, g.smem_bwd, st>>>(a, ngroups); break;
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
@@ -502,12 +529,18 @@ static int rows_mode_override(int direct) {   // CAAT_ROWS_MODE = 0/1/2 override
 
 cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st) {
   direct = rows_mode_override(direct);
+  if (a.compact) direct = 1;
   if (direct == 0 && rows_warp_cpt(a.h, a.t, dtype) > 0) return launch_rows_forward_warp(a, dtype, st);
   if (direct != 1 && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, false)) return launch_rows_forward_staged(a, dtype, st);
   const RowGeom g = row_geometry(a.h, dtype);
+  if (a.compact) {
+    if (dtype == CAAT_BF16)
+      return a.norm == 1 ? launch_fwd_t<__nv_bfloat16, true, true>(a, g, st) : launch_fwd_t<__nv_bfloat16, false, true>(a, g, st);
+    return a.norm == 1 ? launch_fwd_t<float, true, true>(a, g, st) : launch_fwd_t<float, false, true>(a, g, st);
+  }
   if (dtype == CAAT_BF16)
-    return a.norm == 1 ? launch_fwd_t<__nv_bfloat16, true>(a, g, st) : launch_fwd_t<__nv_bfloat16, false>(a, g, st);
-  return a.norm == 1 ? launch_fwd_t<float, true>(a, g, st) : launch_fwd_t<float, false>(a, g, st);
+    return a.norm == 1 ? launch_fwd_t<__nv_bfloat16, true, false>(a, g, st) : launch_fwd_t<__nv_bfloat16, false, false>(a, g, st);
+  return a.norm == 1 ? launch_fwd_t<float, true, false>(a, g, st) : launch_fwd_t<float, false, false>(a, g, st);
 }
 
 cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st) {
@@ -515,14 +548,19 @@ cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int dire
   const RowGeom g = row_geometry(a.h, dtype);
   int rows = rows_backward_partial_rows(a.h, a.T, dtype);
   cudaError_t e;
+  if (a.compact) direct = 1;
   if (direct == 0 && rows_warp_cpt(a.h, a.t, dtype) > 0)
     e = launch_rows_backward_warp(a, dtype, rows, &rows, st);
   else if (direct != 1 && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, true))
     e = launch_rows_backward_staged(a, dtype, rows, &rows, st);
+  else if (a.compact && dtype == CAAT_BF16)
+    e = a.norm == 1 ? launch_bwd_t<__nv_bfloat16, true, true>(a, g, rows, st) : launch_bwd_t<__nv_bfloat16, false, true>(a, g, rows, st);
+  else if (a.compact)
+    e = a.norm == 1 ? launch_bwd_t<float, true, true>(a, g, rows, st) : launch_bwd_t<float, false, true>(a, g, rows, st);
   else if (dtype == CAAT_BF16)
-    e = a.norm == 1 ? launch_bwd_t<__nv_bfloat16, true>(a, g, rows, st) : launch_bwd_t<__nv_bfloat16, false>(a, g, rows, st);
+    e = a.norm == 1 ? launch_bwd_t<__nv_bfloat16, true, false>(a, g, rows, st) : launch_bwd_t<__nv_bfloat16, false, false>(a, g, rows, st);
   else
-    e = a.norm == 1 ? launch_bwd_t<float, true>(a, g, rows, st) : launch_bwd_t<float, false>(a, g, rows, st);
+    e = a.norm == 1 ? launch_bwd_t<float, true, false>(a, g, rows, st) : launch_bwd_t<float, false, false>(a, g, rows, st);
   if (e != cudaSuccess) return e;
   const dim3 rb(32, 32);
   const dim3 rg((a.h + 31) / 32);

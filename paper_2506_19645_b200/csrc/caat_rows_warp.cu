@@ -56,14 +56,15 @@ __device__ __forceinline__ raw lds(const uint8_t* p) { return *reinterpret_cast<
 
 struct WarpGeom {
   int nstages;
-  uint32_t off_a, off_b, off_c, stage_bytes;
+  uint32_t off_a, off_b, off_c, off_d, off_e, stage_bytes;   // d, e: compact layout only
   uint32_t bar_off, ring_off;
   size_t smem;
 };
 
 // ------------------------------------------------------------------ forward
 // stage: a = R rows [kW, h], b = zp rows [kW, P], c = zs rows [kW, S_hi] (rank 0 only)
-template <typename T_, int CPT, bool LN>
+// compact layout (CL): a = private residual rows [kW, P], d = shared residual rows [kW, S] (rank 0 only)
+template <typename T_, int CPT, bool LN, bool CL>
 __global__ void __launch_bounds__(kThreads, 3)
 rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
@@ -100,14 +101,15 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
           if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t bar = full0 + 8u * s;
           const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
-          const uint32_t bR = (uint32_t)rowsN * a.h * ES;
           const uint32_t bP = has_priv ? (uint32_t)rowsN * a.P * ES : 0u;
+          const uint32_t bR = CL ? bP : (uint32_t)rowsN * a.h * ES;
           const uint32_t bS = (m == 0 && has_shared) ? (uint32_t)rowsN * a.S_hi * ES : 0u;
-          mbar_expect_tx(bar, bR + bP + bS);
+          mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS));
           const long long row = (long long)m * a.T + i0;
-          bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * a.h * ES, bR, bar);
+          if (bR) bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * (CL ? a.P : a.h) * ES, bR, bar);
           if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
           if (bS) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.zs) + i0 * a.S_hi * ES, bS, bar);
+          if (CL && bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Rs) + i0 * a.S_hi * ES, bS, bar);
           ++issued;
           if (++s == NS) { s = 0; ph ^= 1u; }
         }
@@ -144,6 +146,7 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
   }
   const float inv_h = 1.0f / (float)a.h;
   const long long rank_h = (long long)a.T * a.h * ES;
+  const long long rank_hn = CL ? (long long)a.T * a.P * ES : rank_h;   // rank stride of the stream's (private) rows
   int s = 0; uint32_t ph = 0;
   bool dead = false;
   for (int n = 0; n < my_groups && !dead; ++n) {
@@ -154,7 +157,8 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
     for (int j = 0; j < CPT; ++j)
 #pragma unroll
       for (int e = 0; e < V; ++e) zs[j][e] = 0.f;
-    char* pHn = static_cast<char*>(a.Hn) + i * a.h * ES;
+    // compact: column l of the private rows sits at l - S
+    char* pHn = CL ? static_cast<char*>(a.Hn) + (i * a.P - a.S_lo) * ES : static_cast<char*>(a.Hn) + i * a.h * ES;
     char* pX = static_cast<char*>(a.X) + i * a.h * ES;
     float* rstd_p = a.rstd + i;
     float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
@@ -170,9 +174,24 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
         for (int e = 0; e < V; ++e) { r[e] = 0.f; zp[e] = 0.f; }
         const bool act = valid && colok[j];
         if (act) {
-          V_::unpack(lds<raw>(stage + sg.off_a + ((size_t)warp * a.h + col[j]) * ES), r);
-          if (cls[j] != 0) V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES), zp);
-          if (m == 0 && cls[j] != 1) V_::unpack(lds<raw>(stage + sg.off_c + ((size_t)warp * a.S_hi + col[j]) * ES), zs[j]);
+          if constexpr (CL) {
+            if (cls[j] != 0) {
+              const size_t op = ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES;
+              V_::unpack(lds<raw>(stage + sg.off_a + op), r);
+              V_::unpack(lds<raw>(stage + sg.off_b + op), zp);
+            } else if (m == 0) {      // the shared part of the new stream, formed once: zs + Rs
+              float rs0[V];
+              const size_t os = ((size_t)warp * a.S_hi + col[j]) * ES;
+              V_::unpack(lds<raw>(stage + sg.off_c + os), zs[j]);
+              V_::unpack(lds<raw>(stage + sg.off_d + os), rs0);
+#pragma unroll
+              for (int e = 0; e < V; ++e) zs[j][e] += rs0[e];
+            }
+          } else {
+            V_::unpack(lds<raw>(stage + sg.off_a + ((size_t)warp * a.h + col[j]) * ES), r);
+            if (cls[j] != 0) V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES), zp);
+            if (m == 0 && cls[j] != 1) V_::unpack(lds<raw>(stage + sg.off_c + ((size_t)warp * a.S_hi + col[j]) * ES), zs[j]);
+          }
         }
         if (cls[j] == 0) {
 #pragma unroll
@@ -184,7 +203,12 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
 #pragma unroll
           for (int e = 0; e < V; ++e) hn[j][e] = (col[j] + e < a.S ? zs[j][e] : a.alpha * zp[e]) + r[e];
         }
-        if (act) stg<raw>(pHn + (long long)col[j] * ES, V_::pack(hn[j]));
+        if constexpr (CL) {
+          if (act && cls[j] != 0) stg<raw>(pHn + (long long)col[j] * ES, V_::pack(hn[j]));
+          else if (act && m == 0) stg<raw>(static_cast<char*>(a.Hns) + (i * a.S_hi + col[j]) * ES, V_::pack(hn[j]));
+        } else {
+          if (act) stg<raw>(pHn + (long long)col[j] * ES, V_::pack(hn[j]));
+        }
 #pragma unroll
         for (int e = 0; e < V; ++e) st = LN ? st + hn[j][e] : fmaf(hn[j][e], hn[j][e], st);
       }
@@ -221,7 +245,7 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
         *rstd_p = rs;
         if (LN && mean_p) *mean_p = mu;
       }
-      pHn += rank_h; pX += rank_h; rstd_p += a.T;
+      pHn += rank_hn; pX += rank_h; rstd_p += a.T;
       if (LN && mean_p) mean_p += a.T;
     }
   }
@@ -229,7 +253,9 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
 
 // ------------------------------------------------------------------ backward
 // stage: a = dX rows, b = Hn rows, c = dHn rows (when given), kW tokens each
-template <typename T_, int CPT, bool LN>
+// compact layout (CL): b, c = private rows [kW, P]; d = shared stream rows, e = shared stream-gradient rows
+// [kW, S] (rank 0 only); a lane keeps its shared chunks of the stream in registers across the ranks
+template <typename T_, int CPT, bool LN, bool CL>
 __global__ void __launch_bounds__(kThreads, 3)
 rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
@@ -279,11 +305,23 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
           if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t bar = full0 + 8u * s;
           const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
-          mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
           const long long off = ((long long)m * a.T + i0) * a.h * ES;
-          bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
-          bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
-          if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
+          if constexpr (CL) {
+            const uint32_t bP = (uint32_t)rowsN * a.P * ES;                       // 0 when there is no private part
+            const uint32_t bS = m == 0 ? (uint32_t)rowsN * a.S_hi * ES : 0u;      // 0 when there is no shared part
+            mbar_expect_tx(bar, b + (has_dh ? 2 : 1) * (bP + bS));
+            const long long offp = ((long long)m * a.T + i0) * a.P * ES, offs = i0 * a.S_hi * ES;
+            bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
+            if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + offp, bP, bar);
+            if (bP && has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + offp, bP, bar);
+            if (bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Hns) + offs, bS, bar);
+            if (bS && has_dh) bulk_g2s(dst + sg.off_e, static_cast<const char*>(a.dHns) + offs, bS, bar);
+          } else {
+            mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
+            bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
+            bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
+            if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
+          }
           ++issued;
           if (++s == NS) { s = 0; ph ^= 1u; }
         }
@@ -325,13 +363,27 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
       for (int j = 0; j < CPT; ++j)
 #pragma unroll
         for (int e = 0; e < V; ++e) gsum[j][e] = 0.f;
-      char* pdR = static_cast<char*>(a.dR) + i * a.h * ES;
+      char* pdR = CL ? static_cast<char*>(a.dR) + (i * a.P - a.S_lo) * ES : static_cast<char*>(a.dR) + i * a.h * ES;
       char* pZ = static_cast<char*>(a.zp) + (i * a.P - a.S_lo) * ES;
+      raw hs[CL ? CPT : 1];      // compact: this lane's shared chunks of the stream, kept for every rank
       for (int m = 0; m < a.t; ++m) {
         if (!mbar_wait(full0 + 8u * s, ph, abort_flag)) { dead = true; break; }
         const uint8_t* stage = ring + (size_t)s * sg.stage_bytes;
         const float rs = __shfl_sync(0xffffffffu, rs_lane, m);
         const float mu = LN ? __shfl_sync(0xffffffffu, mu_lane, m) : 0.f;
+        if constexpr (CL) {
+          if (m == 0) {
+#pragma unroll
+            for (int j = 0; j < CPT; ++j) {
+              hs[j] = zero_raw<raw>();
+              if (valid && colok[j] && cls[j] == 0) {
+                const size_t os = ((size_t)warp * a.S_hi + col[j]) * ES;
+                hs[j] = lds<raw>(stage + sg.off_d + os);
+                if (has_dh) V_::unpack(lds<raw>(stage + sg.off_e + os), gsum[j]);   // enters the rank sum once
+              }
+            }
+          }
+        }
         // pass 1: row statistics and norm-parameter gradients
         float s1 = 0.f, s2 = 0.f;
 #pragma unroll
@@ -340,7 +392,12 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
           float dx[V], hn[V];
           const size_t o = ((size_t)warp * a.h + col[j]) * ES;
           V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
-          V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
+          if constexpr (CL) {
+            if (cls[j] == 0) V_::unpack(hs[j], hn);
+            else V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES), hn);
+          } else {
+            V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
+          }
 #pragma unroll
           for (int e = 0; e < V; ++e) {
             const float xh = (hn[e] - mu) * rs;
@@ -360,10 +417,20 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
           float dx[V], hn[V], dh[V], gg[V];
           const size_t o = ((size_t)warp * a.h + col[j]) * ES;
           V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
-          V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
 #pragma unroll
           for (int e = 0; e < V; ++e) dh[e] = 0.f;
-          if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + o), dh);
+          if constexpr (CL) {
+            if (cls[j] == 0) {
+              V_::unpack(hs[j], hn);
+            } else {
+              const size_t op = ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES;
+              V_::unpack(lds<raw>(stage + sg.off_b + op), hn);
+              if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + op), dh);
+            }
+          } else {
+            V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
+            if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + o), dh);
+          }
 #pragma unroll
           for (int e = 0; e < V; ++e) {
             const float xh = (hn[e] - mu) * rs;
@@ -371,7 +438,7 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
             if (LN) tt -= c1;
             gg[e] = fmaf(rs, tt, dh[e]);
           }
-          stg<raw>(pdR + (long long)col[j] * ES, V_::pack(gg));
+          if (!(CL && cls[j] == 0)) stg<raw>(pdR + (long long)col[j] * ES, V_::pack(gg));
           if (cls[j] == 0) {
 #pragma unroll
             for (int e = 0; e < V; ++e) gsum[j][e] += gg[e];          // fp32 rank sum, m ascending
@@ -394,7 +461,7 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * s);
         if (++s == NS) { s = 0; ph ^= 1u; }
-        pdR += rank_h; pZ += rank_p;
+        pdR += CL ? rank_p : rank_h; pZ += rank_p;
       }
       if (dead) break;
 #pragma unroll
@@ -430,16 +497,24 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
   }
 }
 
-WarpGeom warp_geometry(int h, int P, int S_hi, int ES, bool backward, bool has_c, size_t budget) {
+WarpGeom warp_geometry(int h, int P, int S_hi, int ES, bool backward, bool has_c, bool compact, size_t budget) {
   WarpGeom g{};
   const uint32_t rowA = (uint32_t)kW * h * ES;
-  if (backward) {
+  const uint32_t rowP = (uint32_t)kW * P * ES, rowS = (uint32_t)kW * S_hi * ES;
+  if (backward && compact) {          // dX | Hnp | dHnp | Hns | dHns   (P + S_hi = h)
+    g.off_a = 0; g.off_b = rowA; g.off_c = rowA + rowP;
+    g.off_d = has_c ? rowA + 2 * rowP : rowA + rowP;
+    g.off_e = g.off_d + rowS;
+    g.stage_bytes = g.off_d + (has_c ? 2 : 1) * rowS;
+  } else if (backward) {
     g.off_a = 0; g.off_b = rowA; g.off_c = 2 * rowA;
     g.stage_bytes = (has_c ? 3 : 2) * rowA;
+  } else if (compact) {               // Rp | zp | zs | Rs
+    g.off_a = 0; g.off_b = rowP; g.off_c = 2 * rowP; g.off_d = 2 * rowP + rowS;
+    g.stage_bytes = 2 * rowP + 2 * rowS;
   } else {
-    const uint32_t rowB = (uint32_t)kW * P * ES, rowC = (uint32_t)kW * S_hi * ES;
-    g.off_a = 0; g.off_b = rowA; g.off_c = rowA + rowB;
-    g.stage_bytes = rowA + rowB + rowC;
+    g.off_a = 0; g.off_b = rowA; g.off_c = rowA + rowP;
+    g.stage_bytes = rowA + rowP + rowS;
   }
   g.stage_bytes = (g.stage_bytes + 127u) & ~127u;
   g.bar_off = 0;
@@ -472,15 +547,15 @@ cudaError_t set_smem(K kernel, size_t bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
-template <typename T_, bool LN>
+template <typename T_, bool LN, bool CL>
 cudaError_t launch_fwd_warp_t(const RowFwdArgs& a, int cpt, const WarpGeom& g, int grid, int ngroups,
                               unsigned int* status, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
   LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
 #define CAAT_LAUNCH(CPT_)                                                                      \
   do {                                                                                         \
-    e = set_smem(rows_forward_warp<T_, CPT_, LN>, g.smem);                                     \
-    if (e == cudaSuccess) rows_forward_warp<T_, CPT_, LN><<<grid, kThreads, g.smem, st>>>(a, g, ngroups, status); \
+    e = set_smem(rows_forward_warp<T_, CPT_, LN, CL>, g.smem);                                 \
+    if (e == cudaSuccess) rows_forward_warp<T_, CPT_, LN, CL><<<grid, kThreads, g.smem, st>>>(a, g, ngroups, status); \
   } while (0)
   switch (cpt) {
     case 1: CAAT_LAUNCH(1); break;
@@ -493,15 +568,15 @@ cudaError_t launch_fwd_warp_t(const RowFwdArgs& a, int cpt, const WarpGeom& g, i
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-template <typename T_, bool LN>
+template <typename T_, bool LN, bool CL>
 cudaError_t launch_bwd_warp_t(const RowBwdArgs& a, int cpt, const WarpGeom& g, int grid, int ngroups,
                               unsigned int* status, cudaStream_t st) {
   cudaError_t e = cudaSuccess;
   LaunchScope scope(CAAT_K_ROWS_BACKWARD, st);
 #define CAAT_LAUNCH(CPT_)                                                                       \
   do {                                                                                          \
-    e = set_smem(rows_backward_warp<T_, CPT_, LN>, g.smem);                                     \
-    if (e == cudaSuccess) rows_backward_warp<T_, CPT_, LN><<<grid, kThreads, g.smem, st>>>(a, g, ngroups, status); \
+    e = set_smem(rows_backward_warp<T_, CPT_, LN, CL>, g.smem);                                 \
+    if (e == cudaSuccess) rows_backward_warp<T_, CPT_, LN, CL><<<grid, kThreads, g.smem, st>>>(a, g, ngroups, status); \
   } while (0)
   switch (cpt) {
     case 1: CAAT_LAUNCH(1); break;
@@ -527,25 +602,32 @@ int rows_warp_cpt(int h, int t, caat_dtype dtype) {
 cudaError_t launch_rows_forward_warp(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st) {
   const int cpt = rows_warp_cpt(a.h, a.t, dtype);
   const int ES = (int)elem_size(dtype);
-  const WarpGeom g = warp_geometry(a.h, a.P, a.S_hi, ES, false, true, kSmemPerSm / kCtasPerSm - 1024);
+  const WarpGeom g = warp_geometry(a.h, a.P, a.S_hi, ES, false, true, a.compact != 0, kSmemPerSm / kCtasPerSm - 1024);
   if (cpt == 0 || g.nstages < 2) return cudaErrorInvalidConfiguration;
   const int ngroups = (a.T + kW - 1) / kW;
   int grid = sm_count() * kCtasPerSm;
   if (grid > ngroups) grid = ngroups;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
+  if (a.compact) {
+    if (dtype == CAAT_BF16)
+      return a.norm == 1 ? launch_fwd_warp_t<__nv_bfloat16, true, true>(a, cpt, g, grid, ngroups, status, st)
+                         : launch_fwd_warp_t<__nv_bfloat16, false, true>(a, cpt, g, grid, ngroups, status, st);
+    return a.norm == 1 ? launch_fwd_warp_t<float, true, true>(a, cpt, g, grid, ngroups, status, st)
+                       : launch_fwd_warp_t<float, false, true>(a, cpt, g, grid, ngroups, status, st);
+  }
   if (dtype == CAAT_BF16)
-    return a.norm == 1 ? launch_fwd_warp_t<__nv_bfloat16, true>(a, cpt, g, grid, ngroups, status, st)
-                       : launch_fwd_warp_t<__nv_bfloat16, false>(a, cpt, g, grid, ngroups, status, st);
-  return a.norm == 1 ? launch_fwd_warp_t<float, true>(a, cpt, g, grid, ngroups, status, st)
-                     : launch_fwd_warp_t<float, false>(a, cpt, g, grid, ngroups, status, st);
+    return a.norm == 1 ? launch_fwd_warp_t<__nv_bfloat16, true, false>(a, cpt, g, grid, ngroups, status, st)
+                       : launch_fwd_warp_t<__nv_bfloat16, false, false>(a, cpt, g, grid, ngroups, status, st);
+  return a.norm == 1 ? launch_fwd_warp_t<float, true, false>(a, cpt, g, grid, ngroups, status, st)
+                     : launch_fwd_warp_t<float, false, false>(a, cpt, g, grid, ngroups, status, st);
 }
 
 cudaError_t launch_rows_backward_warp(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,
                                       cudaStream_t st) {
   const int cpt = rows_warp_cpt(a.h, a.t, dtype);
   const int ES = (int)elem_size(dtype);
-  const WarpGeom g = warp_geometry(a.h, 0, 0, ES, true, a.dHn != nullptr, kSmemPerSm / kCtasPerSm - 1024);
+  const WarpGeom g = warp_geometry(a.h, a.P, a.S_hi, ES, true, a.dHn != nullptr, a.compact != 0, kSmemPerSm / kCtasPerSm - 1024);
   if (cpt == 0 || g.nstages < 2) return cudaErrorInvalidConfiguration;
   const int ngroups = (a.T + kW - 1) / kW;
   int grid = sm_count() * kCtasPerSm;
@@ -554,11 +636,18 @@ cudaError_t launch_rows_backward_warp(const RowBwdArgs& a, caat_dtype dtype, int
   *rows_used = grid;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
+  if (a.compact) {
+    if (dtype == CAAT_BF16)
+      return a.norm == 1 ? launch_bwd_warp_t<__nv_bfloat16, true, true>(a, cpt, g, grid, ngroups, status, st)
+                         : launch_bwd_warp_t<__nv_bfloat16, false, true>(a, cpt, g, grid, ngroups, status, st);
+    return a.norm == 1 ? launch_bwd_warp_t<float, true, true>(a, cpt, g, grid, ngroups, status, st)
+                       : launch_bwd_warp_t<float, false, true>(a, cpt, g, grid, ngroups, status, st);
+  }
   if (dtype == CAAT_BF16)
-    return a.norm == 1 ? launch_bwd_warp_t<__nv_bfloat16, true>(a, cpt, g, grid, ngroups, status, st)
-                       : launch_bwd_warp_t<__nv_bfloat16, false>(a, cpt, g, grid, ngroups, status, st);
-  return a.norm == 1 ? launch_bwd_warp_t<float, true>(a, cpt, g, grid, ngroups, status, st)
-                     : launch_bwd_warp_t<float, false>(a, cpt, g, grid, ngroups, status, st);
+    return a.norm == 1 ? launch_bwd_warp_t<__nv_bfloat16, true, false>(a, cpt, g, grid, ngroups, status, st)
+                       : launch_bwd_warp_t<__nv_bfloat16, false, false>(a, cpt, g, grid, ngroups, status, st);
+  return a.norm == 1 ? launch_bwd_warp_t<float, true, false>(a, cpt, g, grid, ngroups, status, st)
+                     : launch_bwd_warp_t<float, false, false>(a, cpt, g, grid, ngroups, status, st);
 }
 
 }  // namespace caat
