@@ -529,7 +529,6 @@ static int rows_mode_override(int direct) {   // CAAT_ROWS_MODE = 0/1/2 override
 
 cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st) {
   direct = rows_mode_override(direct);
-  if (a.compact) direct = 1;
   if (direct == 0 && rows_warp_cpt(a.h, a.t, dtype) > 0) return launch_rows_forward_warp(a, dtype, st);
   if (direct != 1 && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, false)) return launch_rows_forward_staged(a, dtype, st);
   const RowGeom g = row_geometry(a.h, dtype);
@@ -548,7 +547,6 @@ cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int dire
   const RowGeom g = row_geometry(a.h, dtype);
   int rows = rows_backward_partial_rows(a.h, a.T, dtype);
   cudaError_t e;
-  if (a.compact) direct = 1;
   if (direct == 0 && rows_warp_cpt(a.h, a.t, dtype) > 0)
     e = launch_rows_backward_warp(a, dtype, rows, &rows, st);
   else if (direct != 1 && rows_staged_usable(a.h, a.t, a.S_lo, a.S_hi, dtype, true))

@@ -57,6 +57,7 @@ __device__ __forceinline__ raw lds(const uint8_t* p) { return *reinterpret_cast<
 struct StageGeom {
   int nstages;
   uint32_t off_a, off_b, off_c;  // byte offsets of the three row buffers inside a stage
+  uint32_t off_d, off_e;         // compact layout: the shared rows of the stream (and of its gradient)
   uint32_t stage_bytes;
   uint32_t ring_off, bar_off, red_off, stat_off, acc_off;
   size_t smem;
@@ -69,7 +70,8 @@ struct StageGeom {
 template <int CPT, int MAXT>
 struct MinBlocks { static constexpr int value = MAXT <= 256 ? (CPT == 1 ? 3 : 2) : (CPT == 1 ? 2 : 1); };
 
-template <typename T_, int CPT, bool LN, int MAXT>
+// compact layout (CL): a = private residual rows [TY, P], d = shared residual rows [TY, S] (rank 0 only)
+template <typename T_, int CPT, bool LN, int MAXT, bool CL>
 __global__ void __launch_bounds__(MAXT, MinBlocks<CPT, MAXT>::value)
 rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
@@ -105,14 +107,15 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     const int rowsN = (int)((a.T - i0) < TY ? (a.T - i0) : TY);
     const uint32_t bar = bar0 + 8u * s;
     const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
-    const uint32_t bR = (uint32_t)rowsN * a.h * ES;
     const uint32_t bP = has_priv ? (uint32_t)rowsN * a.P * ES : 0u;
+    const uint32_t bR = CL ? bP : (uint32_t)rowsN * a.h * ES;
     const uint32_t bS = (m == 0 && has_shared) ? (uint32_t)rowsN * a.S_hi * ES : 0u;
-    mbar_expect_tx(bar, bR + bP + bS);
+    mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS));
     const long long row = (long long)m * a.T + i0;
-    bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * a.h * ES, bR, bar);
+    if (bR) bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * (CL ? a.P : a.h) * ES, bR, bar);
     if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
     if (bS) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.zs) + i0 * a.S_hi * ES, bS, bar);
+    if (CL && bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Rs) + i0 * a.S_hi * ES, bS, bar);
   };
 
   if (leader) {
@@ -159,7 +162,9 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     for (int j = 0; j < CPT; ++j) {
       act[j] = valid && colok[j];
       const long long off_h = (i * a.h + col[j]) * ES;
-      pHn[j] = static_cast<char*>(a.Hn) + off_h;
+      if (CL) pHn[j] = cls[j] == 0 ? static_cast<char*>(a.Hns) + (i * a.S_hi + col[j]) * ES
+                                   : static_cast<char*>(a.Hn) + (i * a.P + (col[j] - a.S_lo)) * ES;
+      else pHn[j] = static_cast<char*>(a.Hn) + off_h;
       pX[j] = static_cast<char*>(a.X) + off_h;
 #pragma unroll
       for (int e = 0; e < V; ++e) zs[j][e] = 0.f;
@@ -167,6 +172,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     float* rstd_p = a.rstd + i;
     float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
     const long long rank_h = (long long)a.T * a.h * ES;
+    const long long rank_hn = CL ? (long long)a.T * a.P * ES : rank_h;
 
     for (int m = 0; m < a.t; ++m, ++k) {
       const uint8_t* stage = ring + (size_t)cs * sg.stage_bytes;
@@ -181,9 +187,24 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
 #pragma unroll
         for (int e = 0; e < V; ++e) { r[e] = 0.f; zp[e] = 0.f; }
         if (act[j]) {
-          V_::unpack(lds<raw>(stage + sg.off_a + ((size_t)threadIdx.y * a.h + col[j]) * ES), r);
-          if (cls[j] != 0) V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)threadIdx.y * a.P + (col[j] - a.S_lo)) * ES), zp);
-          if (m == 0 && cls[j] != 1) V_::unpack(lds<raw>(stage + sg.off_c + ((size_t)threadIdx.y * a.S_hi + col[j]) * ES), zs[j]);
+          if constexpr (CL) {
+            if (cls[j] != 0) {
+              const size_t op = ((size_t)threadIdx.y * a.P + (col[j] - a.S_lo)) * ES;
+              V_::unpack(lds<raw>(stage + sg.off_a + op), r);
+              V_::unpack(lds<raw>(stage + sg.off_b + op), zp);
+            } else if (m == 0) {      // the shared part of the new stream, formed once: zs + Rs
+              float rs0[V];
+              const size_t os = ((size_t)threadIdx.y * a.S_hi + col[j]) * ES;
+              V_::unpack(lds<raw>(stage + sg.off_c + os), zs[j]);
+              V_::unpack(lds<raw>(stage + sg.off_d + os), rs0);
+#pragma unroll
+              for (int e = 0; e < V; ++e) zs[j][e] += rs0[e];
+            }
+          } else {
+            V_::unpack(lds<raw>(stage + sg.off_a + ((size_t)threadIdx.y * a.h + col[j]) * ES), r);
+            if (cls[j] != 0) V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)threadIdx.y * a.P + (col[j] - a.S_lo)) * ES), zp);
+            if (m == 0 && cls[j] != 1) V_::unpack(lds<raw>(stage + sg.off_c + ((size_t)threadIdx.y * a.S_hi + col[j]) * ES), zs[j]);
+          }
         }
         if (cls[j] == 0) {
 #pragma unroll
@@ -195,8 +216,8 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
 #pragma unroll
           for (int e = 0; e < V; ++e) hn[j][e] = (col[j] + e < a.S ? zs[j][e] : a.alpha * zp[e]) + r[e];
         }
-        if (act[j]) stg<raw>(pHn[j], V_::pack(hn[j]));
-        pHn[j] += rank_h;
+        if (act[j] && !(CL && cls[j] == 0 && m > 0)) stg<raw>(pHn[j], V_::pack(hn[j]));
+        pHn[j] += rank_hn;
 #pragma unroll
         for (int e = 0; e < V; ++e) st[0] = LN ? st[0] + hn[j][e] : fmaf(hn[j][e], hn[j][e], st[0]);
       }
@@ -249,7 +270,9 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
 
 // ------------------------------------------------------------------ backward
 // stage buffers: a = dX rows, b = Hn rows, c = dHn rows (when given)
-template <typename T_, int CPT, bool LN, int MAXT>
+// compact layout (CL): b, c = private rows [TY, P]; d = shared stream rows, e = shared stream-gradient
+// rows [TY, S] (rank 0 only); a thread keeps its shared chunks of the stream in registers across ranks
+template <typename T_, int CPT, bool LN, int MAXT, bool CL>
 __global__ void __launch_bounds__(MAXT, MinBlocks<CPT, MAXT>::value)
 rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
@@ -286,11 +309,23 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
     const uint32_t bar = bar0 + 8u * s;
     const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
     const uint32_t b = (uint32_t)rowsN * a.h * ES;
-    mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
     const long long off = ((long long)m * a.T + i0) * a.h * ES;
-    bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
-    bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
-    if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
+    if constexpr (CL) {
+      const uint32_t bP = (uint32_t)rowsN * a.P * ES;                       // 0 when there is no private part
+      const uint32_t bS = m == 0 ? (uint32_t)rowsN * a.S_hi * ES : 0u;      // 0 when there is no shared part
+      mbar_expect_tx(bar, b + (has_dh ? 2 : 1) * (bP + bS));
+      const long long offp = ((long long)m * a.T + i0) * a.P * ES, offs = i0 * a.S_hi * ES;
+      bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
+      if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + offp, bP, bar);
+      if (bP && has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + offp, bP, bar);
+      if (bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Hns) + offs, bS, bar);
+      if (bS && has_dh) bulk_g2s(dst + sg.off_e, static_cast<const char*>(a.dHns) + offs, bS, bar);
+    } else {
+      mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
+      bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
+      bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
+      if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
+    }
   };
   // row statistics of token group n: element (m, ty) of rstd / mean
   auto load_stats = [&](int n, float* dst) {
@@ -366,13 +401,15 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
 #pragma unroll
     for (int j = 0; j < CPT; ++j) {
       act[j] = valid && colok[j];
-      pdR[j] = static_cast<char*>(a.dR) + (i * a.h + col[j]) * ES;
       pZ[j] = static_cast<char*>(a.zp) + (i * a.P + (col[j] - a.S_lo)) * ES;
+      pdR[j] = CL ? static_cast<char*>(a.dR) + (i * a.P + (col[j] - a.S_lo)) * ES
+                  : static_cast<char*>(a.dR) + (i * a.h + col[j]) * ES;
 #pragma unroll
       for (int e = 0; e < V; ++e) gsum[j][e] = 0.f;
     }
     const long long rank_h = (long long)a.T * a.h * ES;
     const long long rank_p = (long long)a.T * a.P * ES;
+    raw hs[CL ? CPT : 1];      // compact: this thread's shared chunks of the stream, kept for every rank
 
     for (int m = 0; m < a.t; ++m, ++k) {
       const uint8_t* stage = ring + (size_t)cs * sg.stage_bytes;
@@ -393,8 +430,23 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
         if (act[j]) {
           const size_t o = ((size_t)threadIdx.y * a.h + col[j]) * ES;
           V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
-          V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
-          if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + o), dh[j]);
+          if constexpr (CL) {
+            if (cls[j] == 0) {
+              if (m == 0) {
+                const size_t os = ((size_t)threadIdx.y * a.S_hi + col[j]) * ES;
+                hs[j] = lds<raw>(stage + sg.off_d + os);
+                if (has_dh) V_::unpack(lds<raw>(stage + sg.off_e + os), gsum[j]);   // enters the rank sum once
+              }
+              V_::unpack(hs[j], hn);
+            } else {
+              const size_t op = ((size_t)threadIdx.y * a.P + (col[j] - a.S_lo)) * ES;
+              V_::unpack(lds<raw>(stage + sg.off_b + op), hn);
+              if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + op), dh[j]);
+            }
+          } else {
+            V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
+            if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + o), dh[j]);
+          }
         }
 #pragma unroll
         for (int e = 0; e < V; ++e) {
@@ -420,8 +472,8 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
           if (LN) tt -= c1;
           gg[e] = fmaf(rs_c, tt, dh[j][e]);
         }
-        if (act[j]) stg<raw>(pdR[j], V_::pack(gg));
-        pdR[j] += rank_h;
+        if (act[j] && !(CL && cls[j] == 0)) stg<raw>(pdR[j], V_::pack(gg));
+        pdR[j] += CL ? rank_p : rank_h;
         if (cls[j] == 0) {
 #pragma unroll
           for (int e = 0; e < V; ++e) gsum[j][e] += gg[e];          // fp32 rank sum, m ascending
@@ -521,16 +573,24 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
 
 // ------------------------------------------------------------------ host side
 StageGeom stage_geometry(const RowGeom& g, int h, int P, int S_hi, int t, int ES, bool backward, bool has_c,
-                         size_t budget) {
+                         bool compact, size_t budget) {
   StageGeom sg{};
   const uint32_t rowA = (uint32_t)g.TY * h * ES;
-  if (backward) {
+  const uint32_t rowP = (uint32_t)g.TY * P * ES, rowS = (uint32_t)g.TY * S_hi * ES;
+  if (backward && compact) {          // dX | Hnp | dHnp | Hns | dHns   (P + S_hi = h)
+    sg.off_a = 0; sg.off_b = rowA; sg.off_c = rowA + rowP;
+    sg.off_d = has_c ? rowA + 2 * rowP : rowA + rowP;
+    sg.off_e = sg.off_d + rowS;
+    sg.stage_bytes = sg.off_d + (has_c ? 2 : 1) * rowS;
+  } else if (backward) {
     sg.off_a = 0; sg.off_b = rowA; sg.off_c = 2 * rowA;
     sg.stage_bytes = (has_c ? 3 : 2) * rowA;
+  } else if (compact) {               // Rp | zp | zs | Rs
+    sg.off_a = 0; sg.off_b = rowP; sg.off_c = 2 * rowP; sg.off_d = 2 * rowP + rowS;
+    sg.stage_bytes = 2 * rowP + 2 * rowS;
   } else {
-    const uint32_t rowB = (uint32_t)g.TY * P * ES, rowC = (uint32_t)g.TY * S_hi * ES;
-    sg.off_a = 0; sg.off_b = rowA; sg.off_c = rowA + rowB;
-    sg.stage_bytes = rowA + rowB + rowC;
+    sg.off_a = 0; sg.off_b = rowA; sg.off_c = rowA + rowP;
+    sg.stage_bytes = rowA + rowP + rowS;
   }
   sg.stage_bytes = (sg.stage_bytes + 127u) & ~127u;
   // fixed part: barriers + abort flag, reduction scratch, row statistics
@@ -567,7 +627,7 @@ cudaError_t set_smem(K kernel, size_t bytes) {
   return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
-template <typename T_, bool LN>
+template <typename T_, bool LN, bool CL>
 cudaError_t launch_fwd_staged_t(const RowFwdArgs& a, const RowGeom& g, const StageGeom& sg, int grid, int ngroups,
                                 unsigned int* status, cudaStream_t st) {
   const dim3 block(g.TX, g.TY);
@@ -576,8 +636,8 @@ cudaError_t launch_fwd_staged_t(const RowFwdArgs& a, const RowGeom& g, const Sta
   const int threads = g.TX * g.TY;
 #define CAAT_LAUNCH(CPT_, MAXT_)                                                                   \
   do {                                                                                             \
-    e = set_smem(rows_forward_staged<T_, CPT_, LN, MAXT_>, sg.smem);                                            \
-    if (e == cudaSuccess) rows_forward_staged<T_, CPT_, LN, MAXT_><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);       \
+    e = set_smem(rows_forward_staged<T_, CPT_, LN, MAXT_, CL>, sg.smem);                                        \
+    if (e == cudaSuccess) rows_forward_staged<T_, CPT_, LN, MAXT_, CL><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);   \
   } while (0)
   if (g.CPT == 1 && threads <= 256) CAAT_LAUNCH(1, 256);
   else if (g.CPT == 1) CAAT_LAUNCH(1, 512);
@@ -589,7 +649,7 @@ cudaError_t launch_fwd_staged_t(const RowFwdArgs& a, const RowGeom& g, const Sta
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-template <typename T_, bool LN>
+template <typename T_, bool LN, bool CL>
 cudaError_t launch_bwd_staged_t(const RowBwdArgs& a, const RowGeom& g, const StageGeom& sg, int grid, int ngroups,
                                 unsigned int* status, cudaStream_t st) {
   const dim3 block(g.TX, g.TY);
@@ -598,8 +658,8 @@ cudaError_t launch_bwd_staged_t(const RowBwdArgs& a, const RowGeom& g, const Sta
   const int threads = g.TX * g.TY;
 #define CAAT_LAUNCH(CPT_, MAXT_)                                                                   \
   do {                                                                                             \
-    e = set_smem(rows_backward_staged<T_, CPT_, LN, MAXT_>, sg.smem);                                            \
-    if (e == cudaSuccess) rows_backward_staged<T_, CPT_, LN, MAXT_><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);       \
+    e = set_smem(rows_backward_staged<T_, CPT_, LN, MAXT_, CL>, sg.smem);                                        \
+    if (e == cudaSuccess) rows_backward_staged<T_, CPT_, LN, MAXT_, CL><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);   \
   } while (0)
   if (g.CPT == 1 && threads <= 256) CAAT_LAUNCH(1, 256);
   else if (g.CPT == 1) CAAT_LAUNCH(1, 512);
@@ -627,7 +687,7 @@ int ctas_per_sm(const RowGeom& g) {
 bool rows_staged_usable(int h, int t, int S_lo, int S_hi, caat_dtype dtype, bool backward) {
   const RowGeom g = row_geometry(h, dtype);
   const int ES = (int)elem_size(dtype);
-  const StageGeom sg = stage_geometry(g, h, h - S_lo, S_hi, t, ES, backward, true, kSmemPerSm - 1024);
+  const StageGeom sg = stage_geometry(g, h, h - S_lo, S_hi, t, ES, backward, true, false, kSmemPerSm - 1024);
   return sg.nstages >= 2;
 }
 
@@ -635,10 +695,11 @@ cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cu
   const RowGeom g = row_geometry(a.h, dtype);
   const int ES = (int)elem_size(dtype);
   int per_sm = ctas_per_sm(g);
-  StageGeom sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, kSmemPerSm / per_sm - 1024);
+  const bool cl = a.compact != 0;
+  StageGeom sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, cl, kSmemPerSm / per_sm - 1024);
   while (sg.nstages < 3 && per_sm > 1) {   // rows too long: fewer CTAs per SM, each with a larger ring
     --per_sm;
-    sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, kSmemPerSm / per_sm - 1024);
+    sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, cl, kSmemPerSm / per_sm - 1024);
   }
   if (sg.nstages < 2) return cudaErrorInvalidConfiguration;
   const int ngroups = (a.T + g.TY - 1) / g.TY;
@@ -646,11 +707,18 @@ cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cu
   if (grid > ngroups) grid = ngroups;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
+  if (cl) {
+    if (dtype == CAAT_BF16)
+      return a.norm == 1 ? launch_fwd_staged_t<__nv_bfloat16, true, true>(a, g, sg, grid, ngroups, status, st)
+                         : launch_fwd_staged_t<__nv_bfloat16, false, true>(a, g, sg, grid, ngroups, status, st);
+    return a.norm == 1 ? launch_fwd_staged_t<float, true, true>(a, g, sg, grid, ngroups, status, st)
+                       : launch_fwd_staged_t<float, false, true>(a, g, sg, grid, ngroups, status, st);
+  }
   if (dtype == CAAT_BF16)
-    return a.norm == 1 ? launch_fwd_staged_t<__nv_bfloat16, true>(a, g, sg, grid, ngroups, status, st)
-                       : launch_fwd_staged_t<__nv_bfloat16, false>(a, g, sg, grid, ngroups, status, st);
-  return a.norm == 1 ? launch_fwd_staged_t<float, true>(a, g, sg, grid, ngroups, status, st)
-                     : launch_fwd_staged_t<float, false>(a, g, sg, grid, ngroups, status, st);
+    return a.norm == 1 ? launch_fwd_staged_t<__nv_bfloat16, true, false>(a, g, sg, grid, ngroups, status, st)
+                       : launch_fwd_staged_t<__nv_bfloat16, false, false>(a, g, sg, grid, ngroups, status, st);
+  return a.norm == 1 ? launch_fwd_staged_t<float, true, false>(a, g, sg, grid, ngroups, status, st)
+                     : launch_fwd_staged_t<float, false, false>(a, g, sg, grid, ngroups, status, st);
 }
 
 // The grid (= rows of norm-gradient partials) must not exceed what the scratch layout reserves.
@@ -660,10 +728,11 @@ cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, i
   const int ES = (int)elem_size(dtype);
   const bool has_c = a.dHn != nullptr;
   int per_sm = ctas_per_sm(g);
-  StageGeom sg = stage_geometry(g, a.h, 0, 0, a.t, ES, true, has_c, kSmemPerSm / per_sm - 1024);
+  const bool cl = a.compact != 0;
+  StageGeom sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, true, has_c, cl, kSmemPerSm / per_sm - 1024);
   while (sg.nstages < 3 && per_sm > 1) {
     --per_sm;
-    sg = stage_geometry(g, a.h, 0, 0, a.t, ES, true, has_c, kSmemPerSm / per_sm - 1024);
+    sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, true, has_c, cl, kSmemPerSm / per_sm - 1024);
   }
   if (sg.nstages < 2) return cudaErrorInvalidConfiguration;
   const int ngroups = (a.T + g.TY - 1) / g.TY;
@@ -673,11 +742,18 @@ cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, i
   *rows_used = grid;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
+  if (cl) {
+    if (dtype == CAAT_BF16)
+      return a.norm == 1 ? launch_bwd_staged_t<__nv_bfloat16, true, true>(a, g, sg, grid, ngroups, status, st)
+                         : launch_bwd_staged_t<__nv_bfloat16, false, true>(a, g, sg, grid, ngroups, status, st);
+    return a.norm == 1 ? launch_bwd_staged_t<float, true, true>(a, g, sg, grid, ngroups, status, st)
+                       : launch_bwd_staged_t<float, false, true>(a, g, sg, grid, ngroups, status, st);
+  }
   if (dtype == CAAT_BF16)
-    return a.norm == 1 ? launch_bwd_staged_t<__nv_bfloat16, true>(a, g, sg, grid, ngroups, status, st)
-                       : launch_bwd_staged_t<__nv_bfloat16, false>(a, g, sg, grid, ngroups, status, st);
-  return a.norm == 1 ? launch_bwd_staged_t<float, true>(a, g, sg, grid, ngroups, status, st)
-                     : launch_bwd_staged_t<float, false>(a, g, sg, grid, ngroups, status, st);
+    return a.norm == 1 ? launch_bwd_staged_t<__nv_bfloat16, true, false>(a, g, sg, grid, ngroups, status, st)
+                       : launch_bwd_staged_t<__nv_bfloat16, false, false>(a, g, sg, grid, ngroups, status, st);
+  return a.norm == 1 ? launch_bwd_staged_t<float, true, false>(a, g, sg, grid, ngroups, status, st)
+                     : launch_bwd_staged_t<float, false, false>(a, g, sg, grid, ngroups, status, st);
 }
 
 }  // namespace caat
