@@ -106,58 +106,87 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- algorithmic work
-def layer_work(w, k_r, backward):
+def layer_work(w, k_r, backward, compact=False):
     """Algorithmic flops and bytes of ONE layer per kernel kind (inputs read once, outputs
-    written once, given the kernel's interface; e = 2 bytes)."""
+    written once, given the kernel's interface; e = 2 bytes).  compact: the residual stream and
+    its gradient are stored shared-once + private-per-rank, like the scratch."""
     t, T, h, S, e = w.t, w.tokens, w.h, w.S, 2
     K = k_r * t
     zsz = (T * S + t * T * (h - S)) * e            # split scratch: shared once, private per rank
+    full = t * T * h * e
+    stream = zsz if compact else full              # one tensor of the residual stream
     out = {
         "tc_gemm_forward": {"flops": 2.0 * T * K * h, "bytes": (T * K + K * h) * e + zsz},
-        "rows_forward": {"flops": 0.0, "bytes": zsz + 3 * t * T * h * e + t * T * 4},
+        "rows_forward": {"flops": 0.0, "bytes": zsz + 2 * stream + full + t * T * 4},
     }
     if backward:
-        out["rows_backward"] = {"flops": 0.0, "bytes": 4 * t * T * h * e + zsz + t * T * 4}
+        # reads dX, Hn, dHn; writes dR and the scratch (compact: dRs is the scratch's shared part)
+        bwd_out = stream + t * T * (h - S) * e if compact else stream + zsz
+        out["rows_backward"] = {"flops": 0.0, "bytes": full + 2 * stream + bwd_out + t * T * 4}
         out["tc_gemm_dgrad"] = {"flops": 2.0 * T * K * h, "bytes": zsz + K * h * e + T * K * e}
         out["tc_gemm_wgrad"] = {"flops": 2.0 * T * K * h, "bytes": zsz + T * K * e + K * h * 4}
     return out
 
 
-def step_work(w):
+def step_work(w, compact=False):
     tot = {}
     for k_r in (w.kr_attn, w.kr_mlp):
-        for kind, v in layer_work(w, k_r, w.backward).items():
+        for kind, v in layer_work(w, k_r, w.backward, compact).items():
             a = tot.setdefault(kind, {"flops": 0.0, "bytes": 0.0})
             a["flops"] += v["flops"]
             a["bytes"] += v["bytes"]
     return tot
 
 
-def paper_level_work(w):
+def paper_level_work(w, compact=False):
     """Whole-path algorithmic work per step (no scratch traffic): the roofline of the path."""
     t, T, h, e = w.t, w.tokens, w.h, 2
+    full = t * T * h
+    stream = T * w.S + t * T * (h - w.S) if compact else full
     fl = by = 0.0
     for k_r in (w.kr_attn, w.kr_mlp):
         K = k_r * t
         fl += 2.0 * T * K * h
-        by += e * (T * K + K * h + 3 * t * T * h)
+        by += e * (T * K + K * h + 2 * stream + full)
         if w.backward:
             fl += 4.0 * T * K * h
-            by += e * (4 * t * T * h + 2 * T * K + K * h) + 4 * K * h
+            by += e * (full + 3 * stream + 2 * T * K + K * h) + 4 * K * h
     return fl, by
+
+
+def r_w_compact_ok(w):
+    """The compact-layout entry points need a partition on a 16-byte boundary and more than a few tokens."""
+    return w.S % 8 == 0 and w.tokens > 64
 
 
 # --------------------------------------------------------------------------- the CUDA arm
 class BlockRunner:
-    def __init__(self, w, device):
+    def __init__(self, w, device, compact=False):
         from paper_2506_19645_b200 import caat
-        self.caat, self.w, self.dev = caat, w, device
+        self.caat, self.w, self.dev, self.compact = caat, w, device, compact
         self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
         self.inp = synthetic.block_inputs(w, device=device)
         t, T, h = w.t, w.tokens, w.h
         td = self.ctx.torch_dtype
         mk = lambda *s, dt=td: torch.empty(*s, dtype=dt, device=device)
         f32 = torch.float32
+        if compact:
+            # same synthetic block, with the (tied) shared channels of the stream kept once
+            S, i = w.S, self.inp
+            for name in ("R0", "dHn2"):
+                if name in i:
+                    x = i.pop(name)
+                    i[name + "s"], i[name + "p"] = x[0, :, :S].contiguous(), x[:, :, S:].contiguous()
+            sh, pr = (T, S), (t, T, h - S)
+            self.out = {"Hn1s": mk(*sh), "Hn1p": mk(*pr), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=f32),
+                        "Hn2s": mk(*sh), "Hn2p": mk(*pr), "X2": mk(t, T, h), "rstd2": mk(t, T, dt=f32)}
+            if w.backward:
+                self.out.update({"dY_attn": mk(t, T, w.kr_attn), "dW_o": mk(t, h, w.kr_attn, dt=f32),
+                                 "dY_mlp": mk(t, T, w.kr_mlp), "dW_down": mk(t, h, w.kr_mlp, dt=f32),
+                                 "dR0s": mk(*sh), "dR0p": mk(*pr), "dHn1s": mk(*sh), "dHn1p": mk(*pr),
+                                 "dgamma1": mk(h, dt=f32), "dgamma2": mk(h, dt=f32)})
+            self.ws = self.ctx.alloc_workspace(self.ctx.block_workspace_bytes(T, w.backward), device=device)
+            return
         self.out = {"Hn1": mk(t, T, h), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=f32),
                     "Hn2": mk(t, T, h), "X2": mk(t, T, h), "rstd2": mk(t, T, dt=f32)}
         if w.backward:
@@ -168,6 +197,18 @@ class BlockRunner:
 
     def step(self):
         i, o, T = self.inp, self.out, self.w.tokens
+        if self.compact:
+            self.ctx.block_forward_compact(T, i["Y_attn"], i["W_o"], i["Y_mlp"], i["W_down"], i["R0s"], i["R0p"],
+                                           i["gamma1"], None, i["gamma2"], None, o["Hn1s"], o["Hn1p"], o["X1"],
+                                           o["rstd1"], None, o["Hn2s"], o["Hn2p"], o["X2"], o["rstd2"], None, self.ws)
+            if self.w.backward:
+                self.ctx.block_backward_compact(T, i["dX1"], i["dX2"], i["dHn2s"], i["dHn2p"], i["Y_attn"], i["W_o"],
+                                                i["Y_mlp"], i["W_down"], o["Hn1s"], o["Hn1p"], o["rstd1"], None,
+                                                o["Hn2s"], o["Hn2p"], o["rstd2"], None, i["gamma1"], i["gamma2"],
+                                                o["dY_attn"], o["dW_o"], o["dY_mlp"], o["dW_down"], o["dR0s"],
+                                                o["dR0p"], o["dHn1s"], o["dHn1p"], o["dgamma1"], None, o["dgamma2"],
+                                                None, self.ws)
+            return
         self.ctx.block_forward(T, i["Y_attn"], i["W_o"], i["Y_mlp"], i["W_down"], i["R0"], i["gamma1"], None,
                                i["gamma2"], None, o["Hn1"], o["X1"], o["rstd1"], None, o["Hn2"], o["X2"], o["rstd2"],
                                None, self.ws)
@@ -300,7 +341,8 @@ def run_cuda(args):
     w = synthetic.WORKLOADS[args.workload]
     if args.tokens > 0:
         w = w.with_tokens(args.tokens)
-    runner = BlockRunner(w, dev)
+    compact = args.layout == "compact"
+    runner = BlockRunner(w, dev, compact)
     warm = max(args.warmup, 3)
     for _ in range(warm):
         runner.step()
@@ -330,7 +372,7 @@ def run_cuda(args):
     result = None
     if rank == 0:
         peaks = measured_peaks()
-        work = step_work(w)
+        work = step_work(w, compact)
         kernels = {}
         for kind, (kms, n) in prof.items():
             per_step_ms = kms / args.steps
@@ -350,10 +392,10 @@ def run_cuda(args):
             kernels[kind] = ent
         top = max((k for k in kernels if "frac" in kernels[k]), key=lambda k: kernels[k]["ms_per_step"])
         roof = {k: kernels[top][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
-        roof.update({"kernel": top, "traffic": recorded_traffic(top, w.name), "peak_source": peaks["source"],
+        roof.update({"kernel": top, "traffic": recorded_traffic(top, w.name + ("@compact" if compact else "")), "peak_source": peaks["source"],
                      "timed": f"second pass of {args.steps} steps with CUDA events around every kernel launch "
                               f"({ms_prof / args.steps:.4f} ms/step with events)"})
-        fl, by = paper_level_work(w)
+        fl, by = paper_level_work(w, compact)
         t_roof = max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9))
         e2e = None
         try:
@@ -372,6 +414,7 @@ def run_cuda(args):
             "config": {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p,
                        "S": w.S, "passes": "forward+backward" if w.backward else "forward",
                        "private_scale": "sqrt(t)", "norm": "rmsnorm", "parallelism": f"replicas x{world}",
+                       "residual_layout": "compact (shared channels of the stream stored once)" if compact else "per rank [t,T,h]",
                        "launch": "cuda graph replay" if graph is not None else "eager",
                        "l2": f"inputs+outputs touched per step {runner.touched_bytes() / 1e6:.0f} MB > 126 MB L2"},
             "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "roofline": roof, "kernels": kernels,
@@ -401,6 +444,16 @@ def run_cuda(args):
                               "allreduce_payload_bytes": r.ctx.allreduce_bytes(r.w.tokens, 2)["payload_per_rank"]})
                 del r
                 torch.cuda.empty_cache()
+                if r_w_compact_ok(synthetic.WORKLOADS[name]):
+                    # the same block on the compact residual layout (shared channels of the stream stored once)
+                    r = BlockRunner(synthetic.WORKLOADS[name], dev, True)
+                    for _ in range(3):
+                        r.step()
+                    cms = time_steps(r, k, False) / k
+                    sweep[-1]["compact_layout_ms_per_step"] = cms
+                    sweep[-1]["compact_layout_tokens_per_s"] = r.w.tokens / (cms * 1e-3)
+                    del r
+                    torch.cuda.empty_cache()
             except Exception as ex:
                 sweep.append({"workload": name, "error": str(ex)[:200]})
         result["sweep"] = sweep
@@ -457,6 +510,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-graph", action="store_true", help="never replay launch-bound steps from a CUDA graph")
+    ap.add_argument("--layout", default="per_rank", choices=["per_rank", "compact"],
+                    help="residual-stream layout: per rank [t,T,h] (the benchmark's configuration) or compact")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling on a small case)")
     args = ap.parse_args()
     if args.steps < 1:

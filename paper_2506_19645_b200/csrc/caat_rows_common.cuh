@@ -44,6 +44,42 @@ struct VT<__nv_bfloat16> {
   static __device__ __forceinline__ float round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 };
 
+// ---- packed fp32 pairs (sm_100 executes fma / add / mul on two fp32 lanes per instruction; each lane
+// is the IEEE single-precision result of the scalar operation)
+__device__ __forceinline__ float2 f2(float x) { return make_float2(x, x); }
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+
+// 16-byte chunk <-> V/2 pairs of fp32
+__device__ __forceinline__ void unpack2(const uint4& r, float2 (&f)[4]) {
+  const unsigned w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) f[q] = make_float2(__uint_as_float(w[q] << 16), __uint_as_float(w[q] & 0xffff0000u));
+}
+__device__ __forceinline__ void unpack2(const float4& r, float2 (&f)[2]) {
+  f[0] = make_float2(r.x, r.y);
+  f[1] = make_float2(r.z, r.w);
+}
+__device__ __forceinline__ uint4 pack2(const float2 (&f)[4]) {
+  unsigned w[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    __nv_bfloat162 b = __floats2bfloat162_rn(f[q].x, f[q].y);
+    w[q] = *reinterpret_cast<unsigned*>(&b);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+__device__ __forceinline__ float4 pack2(const float2 (&f)[2]) { return make_float4(f[0].x, f[0].y, f[1].x, f[1].y); }
+
+// 16-byte shared-memory load through a 32-bit shared address (volatile: stays behind the barrier waits)
+template <typename raw>
+__device__ __forceinline__ raw lds32(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return *reinterpret_cast<raw*>(&v);
+}
+
 template <typename raw>
 __device__ __forceinline__ raw zero_raw();
 template <>

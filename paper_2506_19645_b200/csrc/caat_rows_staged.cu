@@ -60,6 +60,8 @@ struct StageGeom {
   uint32_t off_d, off_e;         // compact layout: the shared rows of the stream (and of its gradient)
   uint32_t stage_bytes;
   uint32_t ring_off, bar_off, red_off, stat_off, acc_off;
+  uint32_t zero_off;             // 16 zero bytes inside every stage (read by chunks past the row end)
+  uint32_t keep_off;             // compact backward: [TY, S] shared rows of the stream, kept for all ranks of a token group
   size_t smem;
 };
 
@@ -95,13 +97,19 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
   const int my_groups = blockIdx.x < ngroups ? (ngroups - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const long long total = (long long)my_groups * a.t;
 
-  // leader only: fetch the inputs of (its token group nn, rank mm) into stage ss
+  // Fetch the inputs of (token group nn, rank mm) into stage ss.  Every thread calls it (all keep the
+  // counters); the copies of a stage are issued by lane 0 of DIFFERENT warps, so that no warp carries
+  // more than one copy's issue latency into the next CTA barrier.  Warp 0 posts the expected bytes with
+  // its arrival; a copy landing before that only drives the byte count negative for a moment, the phase
+  // cannot complete before the arrival.
   int nn = 0, mm = 0, ss = 0;
+  const int issuer = ((threadIdx.y * TX + threadIdx.x) & 31) == 0 ? (int)(threadIdx.y * TX + threadIdx.x) >> 5 : 99;
   auto issue = [&]() {
     if (nn >= my_groups) return;
     const int n = nn, m = mm, s = ss;
     if (++mm == a.t) { mm = 0; ++nn; }
     if (++ss == NS) ss = 0;
+    if (issuer > 3) return;
     const long long g = blockIdx.x + (long long)n * gridDim.x;
     const long long i0 = g * TY;
     const int rowsN = (int)((a.T - i0) < TY ? (a.T - i0) : TY);
@@ -110,12 +118,17 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     const uint32_t bP = has_priv ? (uint32_t)rowsN * a.P * ES : 0u;
     const uint32_t bR = CL ? bP : (uint32_t)rowsN * a.h * ES;
     const uint32_t bS = (m == 0 && has_shared) ? (uint32_t)rowsN * a.S_hi * ES : 0u;
-    mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS));
     const long long row = (long long)m * a.T + i0;
-    if (bR) bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * (CL ? a.P : a.h) * ES, bR, bar);
-    if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
-    if (bS) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.zs) + i0 * a.S_hi * ES, bS, bar);
-    if (CL && bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Rs) + i0 * a.S_hi * ES, bS, bar);
+    if (issuer == 0) {
+      mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS));
+      if (bR) bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * (CL ? a.P : a.h) * ES, bR, bar);
+    } else if (issuer == 1) {
+      if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
+    } else if (issuer == 2) {
+      if (bS) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.zs) + i0 * a.S_hi * ES, bS, bar);
+    } else {
+      if (CL && bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Rs) + i0 * a.S_hi * ES, bS, bar);
+    }
   };
 
   if (leader) {
@@ -124,30 +137,47 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if ((int)(threadIdx.y * TX + threadIdx.x) < NS)   // the zero slot of every stage (no copy ever lands there)
+    *reinterpret_cast<uint4*>(ring + (size_t)(threadIdx.y * TX + threadIdx.x) * sg.stage_bytes + sg.zero_off) =
+        make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
-  long long issued = 0;
-  if (leader) {
-    for (; issued < NS && issued < total; ++issued) issue();
-  }
+  for (int q = 0; q < NS; ++q) issue();
 
+  // Per-thread constants of the hot loop: the chunk's class and its byte offsets inside a stage.  Chunks
+  // past the row end read a zeroed slot that every stage carries, so the loop needs no bounds predicates
+  // on its loads.
+  constexpr int H2 = V / 2;
+  const uint32_t ring32 = smem_u32(ring);
   int col[CPT], cls[CPT];
   bool colok[CPT];
-  float gam[CPT][V], bet[CPT][V];
+  uint32_t oA[CPT], oB[CPT];
+  float2 gam[CPT][H2], bet[LN ? CPT : 1][H2];
 #pragma unroll
   for (int j = 0; j < CPT; ++j) {
     col[j] = (threadIdx.x + j * TX) * V;
     colok[j] = col[j] < a.h;
     cls[j] = chunk_class(col[j], V, a.S);
 #pragma unroll
-    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; bet[j][e] = 0.f; }
+    for (int q = 0; q < H2; ++q) { gam[j][q] = f2(0.f); if constexpr (LN) bet[j][q] = f2(0.f); }
+    oA[j] = oB[j] = sg.zero_off;
     if (colok[j]) {
-      V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
-      if (LN && a.beta) V_::unpack(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
+      unpack2(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+      if constexpr (LN) {
+        if (a.beta) unpack2(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
+      }
+      const uint32_t priv = ((uint32_t)threadIdx.y * a.P + (uint32_t)(col[j] - a.S_lo)) * ES;
+      if (cls[j] != 0) oB[j] = sg.off_b + priv;
+      if (CL) { if (cls[j] != 0) oA[j] = sg.off_a + priv; }
+      else oA[j] = sg.off_a + ((uint32_t)threadIdx.y * a.h + col[j]) * ES;
     }
   }
+  const float2 alpha2 = f2(a.alpha);
+  const long long rank_h = (long long)a.T * a.h * ES;
+  const long long rank_hn = CL ? (long long)a.T * a.P * ES : rank_h;
 
   long long k = 0;
-  int cs = 0;            // consumer's stage and its phase parity
+  uint32_t sb = ring32;   // consumer's stage (shared address), its index and phase parity
+  int cs = 0;
   uint32_t cph = 0;
   bool dead = false;
   for (int n = 0; n < my_groups && !dead; ++n) {
@@ -155,7 +185,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     const long long i = g * TY + threadIdx.y;
     const bool valid = i < a.T;
     bool act[CPT];
-    float zs[CPT][V];
+    float2 zs[CPT][H2];     // shared part of the layer output (compact: of the new stream), formed once per token
     char* pHn[CPT];
     char* pX[CPT];
 #pragma unroll
@@ -167,88 +197,94 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
       else pHn[j] = static_cast<char*>(a.Hn) + off_h;
       pX[j] = static_cast<char*>(a.X) + off_h;
 #pragma unroll
-      for (int e = 0; e < V; ++e) zs[j][e] = 0.f;
+      for (int q = 0; q < H2; ++q) zs[j][q] = f2(0.f);
     }
     float* rstd_p = a.rstd + i;
     float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
-    const long long rank_h = (long long)a.T * a.h * ES;
-    const long long rank_hn = CL ? (long long)a.T * a.P * ES : rank_h;
 
     for (int m = 0; m < a.t; ++m, ++k) {
-      const uint8_t* stage = ring + (size_t)cs * sg.stage_bytes;
       if (!mbar_wait(bar0 + 8u * cs, cph)) *abort_flag = 1;
-      if (++cs == NS) { cs = 0; cph ^= 1u; }
 
-      float hn[CPT][V];
-      float st[1] = {0.f};
+      float2 hn[CPT][H2];
+      float2 acc = f2(0.f);
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
-        float r[V], zp[V];
+        if (m == 0 && cls[j] != 1 && colok[j]) {
+          const uint32_t os = ((uint32_t)threadIdx.y * a.S_hi + col[j]) * ES;
+          unpack2(lds32<raw>(sb + sg.off_c + os), zs[j]);
+          if constexpr (CL) {       // the shared part of the new stream: zs + Rs
+            float2 r0[H2];
+            unpack2(lds32<raw>(sb + sg.off_d + os), r0);
 #pragma unroll
-        for (int e = 0; e < V; ++e) { r[e] = 0.f; zp[e] = 0.f; }
-        if (act[j]) {
-          if constexpr (CL) {
-            if (cls[j] != 0) {
-              const size_t op = ((size_t)threadIdx.y * a.P + (col[j] - a.S_lo)) * ES;
-              V_::unpack(lds<raw>(stage + sg.off_a + op), r);
-              V_::unpack(lds<raw>(stage + sg.off_b + op), zp);
-            } else if (m == 0) {      // the shared part of the new stream, formed once: zs + Rs
-              float rs0[V];
-              const size_t os = ((size_t)threadIdx.y * a.S_hi + col[j]) * ES;
-              V_::unpack(lds<raw>(stage + sg.off_c + os), zs[j]);
-              V_::unpack(lds<raw>(stage + sg.off_d + os), rs0);
-#pragma unroll
-              for (int e = 0; e < V; ++e) zs[j][e] += rs0[e];
-            }
-          } else {
-            V_::unpack(lds<raw>(stage + sg.off_a + ((size_t)threadIdx.y * a.h + col[j]) * ES), r);
-            if (cls[j] != 0) V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)threadIdx.y * a.P + (col[j] - a.S_lo)) * ES), zp);
-            if (m == 0 && cls[j] != 1) V_::unpack(lds<raw>(stage + sg.off_c + ((size_t)threadIdx.y * a.S_hi + col[j]) * ES), zs[j]);
+            for (int q = 0; q < H2; ++q) zs[j][q] = add2(zs[j][q], r0[q]);
           }
         }
         if (cls[j] == 0) {
+          if constexpr (CL) {
 #pragma unroll
-          for (int e = 0; e < V; ++e) hn[j][e] = zs[j][e] + r[e];
-        } else if (cls[j] == 1) {
+            for (int q = 0; q < H2; ++q) hn[j][q] = zs[j][q];
+          } else {
+            float2 r[H2];
+            unpack2(lds32<raw>(sb + oA[j]), r);
 #pragma unroll
-          for (int e = 0; e < V; ++e) hn[j][e] = fmaf(a.alpha, zp[e], r[e]);
+            for (int q = 0; q < H2; ++q) hn[j][q] = add2(zs[j][q], r[q]);
+          }
         } else {
+          float2 r[H2], zp[H2];
+          unpack2(lds32<raw>(sb + oA[j]), r);
+          unpack2(lds32<raw>(sb + oB[j]), zp);
+          if (cls[j] == 1) {
 #pragma unroll
-          for (int e = 0; e < V; ++e) hn[j][e] = (col[j] + e < a.S ? zs[j][e] : a.alpha * zp[e]) + r[e];
+            for (int q = 0; q < H2; ++q) hn[j][q] = fma2(alpha2, zp[q], r[q]);
+          } else {   // the one chunk that straddles the partition
+#pragma unroll
+            for (int q = 0; q < H2; ++q) {
+              hn[j][q].x = (col[j] + 2 * q < a.S ? zs[j][q].x : a.alpha * zp[q].x) + r[q].x;
+              hn[j][q].y = (col[j] + 2 * q + 1 < a.S ? zs[j][q].y : a.alpha * zp[q].y) + r[q].y;
+            }
+          }
         }
-        if (act[j] && !(CL && cls[j] == 0 && m > 0)) stg<raw>(pHn[j], V_::pack(hn[j]));
+        if (act[j] && !(CL && cls[j] == 0 && m > 0)) stg<raw>(pHn[j], pack2(hn[j]));
         pHn[j] += rank_hn;
 #pragma unroll
-        for (int e = 0; e < V; ++e) st[0] = LN ? st[0] + hn[j][e] : fmaf(hn[j][e], hn[j][e], st[0]);
+        for (int q = 0; q < H2; ++q) acc = LN ? add2(acc, hn[j][q]) : fma2(hn[j][q], hn[j][q], acc);
       }
+      float st[1] = {acc.x + acc.y};
       row_reduce_sync<1>(st, red, par);      // CTA barrier: every thread is done reading this stage
       if (*abort_flag) { dead = true; break; }
-      if (leader && issued < total) { issue(); ++issued; }
+      issue();
+      sb += sg.stage_bytes;
+      if (++cs == NS) { cs = 0; cph ^= 1u; sb = ring32; }
       float mu = 0.f, rs;
       if (LN) {
         mu = st[0] * inv_h;
-        float sq[1] = {0.f};
+        float2 sq2 = f2(0.f);
 #pragma unroll
-        for (int j = 0; j < CPT; ++j)
+        for (int j = 0; j < CPT; ++j) {
+          if (!colok[j]) continue;
 #pragma unroll
-          for (int e = 0; e < V; ++e) {
-            const float d = act[j] ? hn[j][e] - mu : 0.f;
-            sq[0] = fmaf(d, d, sq[0]);
+          for (int q = 0; q < H2; ++q) {
+            const float2 d = add2(hn[j][q], f2(-mu));
+            sq2 = fma2(d, d, sq2);
           }
+        }
+        float sq[1] = {sq2.x + sq2.y};
         row_reduce_sync<1>(sq, red, par);
         rs = rsqrtf(fmaf(sq[0], inv_h, a.eps));
       } else {
         rs = rsqrtf(fmaf(st[0], inv_h, a.eps));
       }
+      const float2 rs2 = f2(rs);
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
-        float x[V];
+        float2 x[H2];
 #pragma unroll
-        for (int e = 0; e < V; ++e) {
-          if (LN) x[e] = fmaf(hn[j][e] - mu, rs * gam[j][e], bet[j][e]);
-          else x[e] = hn[j][e] * (rs * gam[j][e]);
+        for (int q = 0; q < H2; ++q) {
+          const float2 sc = mul2(rs2, gam[j][q]);
+          if constexpr (LN) x[q] = fma2(add2(hn[j][q], f2(-mu)), sc, bet[j][q]);
+          else x[q] = mul2(hn[j][q], sc);
         }
-        if (act[j]) stg<raw>(pX[j], V_::pack(x));
+        if (act[j]) stg<raw>(pX[j], pack2(x));
         pX[j] += rank_h;
       }
       if (valid && threadIdx.x == 0) {
@@ -262,6 +298,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
   if (dead && leader) {
     atomicExch(status, 4u);
     // wait (bounded) for this CTA's copies still in flight before its shared memory goes away
+    const long long issued = (k + NS) < total ? (k + NS) : total;
     for (long long q = k + 1; q < issued; ++q)
       for (uint32_t it = 0; it < (1u << 20); ++it)
         if (mbar_try(bar0 + 8u * (uint32_t)(q % NS), (uint32_t)((q / NS) & 1))) break;
@@ -297,12 +334,16 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
   const int my_groups = blockIdx.x < ngroups ? (ngroups - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const long long total = (long long)my_groups * a.t;
 
+  // fetch (token group nn, rank mm) into stage ss: called by every thread, one copy per issuing warp
+  // (see the forward kernel)
   int nn = 0, mm = 0, ss = 0;
-  auto issue = [&]() {   // leader only: fetch (its token group nn, rank mm) into stage ss
+  const int issuer = (tid & 31) == 0 ? tid >> 5 : 99;
+  auto issue = [&]() {
     if (nn >= my_groups) return;
     const int n = nn, m = mm, s = ss;
     if (++mm == a.t) { mm = 0; ++nn; }
     if (++ss == NS) ss = 0;
+    if (issuer > 4) return;
     const long long g = blockIdx.x + (long long)n * gridDim.x;
     const long long i0 = g * TY;
     const int rowsN = (int)((a.T - i0) < TY ? (a.T - i0) : TY);
@@ -313,18 +354,28 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
     if constexpr (CL) {
       const uint32_t bP = (uint32_t)rowsN * a.P * ES;                       // 0 when there is no private part
       const uint32_t bS = m == 0 ? (uint32_t)rowsN * a.S_hi * ES : 0u;      // 0 when there is no shared part
-      mbar_expect_tx(bar, b + (has_dh ? 2 : 1) * (bP + bS));
       const long long offp = ((long long)m * a.T + i0) * a.P * ES, offs = i0 * a.S_hi * ES;
-      bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
-      if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + offp, bP, bar);
-      if (bP && has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + offp, bP, bar);
-      if (bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Hns) + offs, bS, bar);
-      if (bS && has_dh) bulk_g2s(dst + sg.off_e, static_cast<const char*>(a.dHns) + offs, bS, bar);
+      if (issuer == 0) {
+        mbar_expect_tx(bar, b + (has_dh ? 2 : 1) * (bP + bS));
+        bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
+      } else if (issuer == 1) {
+        if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + offp, bP, bar);
+      } else if (issuer == 2) {
+        if (bP && has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + offp, bP, bar);
+      } else if (issuer == 3) {
+        if (bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Hns) + offs, bS, bar);
+      } else {
+        if (bS && has_dh) bulk_g2s(dst + sg.off_e, static_cast<const char*>(a.dHns) + offs, bS, bar);
+      }
     } else {
-      mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
-      bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
-      bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
-      if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
+      if (issuer == 0) {
+        mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
+        bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
+      } else if (issuer == 1) {
+        bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
+      } else if (issuer == 2) {
+        if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
+      }
     }
   };
   // row statistics of token group n: element (m, ty) of rstd / mean
@@ -345,29 +396,39 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (tid < NS)   // the zero slot of every stage (no copy ever lands there)
+    *reinterpret_cast<uint4*>(ring + (size_t)tid * sg.stage_bytes + sg.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
-  long long issued = 0;
-  if (leader) {
-    for (; issued < NS && issued < total; ++issued) issue();
-  }
+  for (int q = 0; q < NS; ++q) issue();
   load_stats(0, stat);
 
+  // Per-thread constants of the hot loop: chunk class and byte offsets inside a stage.  Chunks past the
+  // row end, and every chunk of a token past T, read the zeroed slot each stage carries: they then add
+  // exact zeros to the sums, and the loop needs no predicates on its loads.
+  constexpr int H2 = V / 2;
+  const uint32_t ring32 = smem_u32(ring);
+  const uint32_t keep32 = smem_u32(smem + sg.keep_off);
   int col[CPT], cls[CPT];
   bool colok[CPT];
-  float gam[CPT][V], dgacc[CPT][V], dbacc[LN ? CPT : 1][V];
+  float2 gam[CPT][H2], dgacc[CPT][H2], dbacc[LN ? CPT : 1][H2];
 #pragma unroll
   for (int j = 0; j < CPT; ++j) {
     col[j] = (threadIdx.x + j * TX) * V;
     colok[j] = col[j] < a.h;
     cls[j] = chunk_class(col[j], V, a.S);
 #pragma unroll
-    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; dgacc[j][e] = 0.f; if constexpr (LN) dbacc[j][e] = 0.f; }
-    if (colok[j]) V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+    for (int q = 0; q < H2; ++q) { gam[j][q] = f2(0.f); dgacc[j][q] = f2(0.f); if constexpr (LN) dbacc[j][q] = f2(0.f); }
+    if (colok[j]) unpack2(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
   }
+  const uint32_t off_hc = sg.off_c - sg.off_b;   // from a chunk of the stream to the same chunk of its gradient
+  const float2 alpha2 = f2(a.alpha);
+  const long long rank_h = (long long)a.T * a.h * ES;
+  const long long rank_p = (long long)a.T * a.P * ES;
   __syncthreads();   // stats of group 0 visible
 
   long long k = 0;
-  int cs = 0;            // consumer's stage and its phase parity
+  uint32_t sb = ring32;  // consumer's stage (shared address), its index and phase parity
+  int cs = 0;
   uint32_t cph = 0;
   bool dead = false;
   for (int n = 0; n < my_groups && !dead; ++n) {
@@ -395,111 +456,121 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
       }
     }
     bool act[CPT];
-    char* pdR[CPT];
-    char* pZ[CPT];
-    float gsum[CPT][V];
+    // this group's stage-relative addresses of the dX chunk and of the stream chunk (its gradient sits at
+    // the same place in its own buffer); the zero slot when the chunk is inactive.  Compact: private
+    // chunks sit at l - S in rows of P, shared chunks come from the kept row.
+    uint32_t aX[CPT], aH[CPT];
+    // outputs: byte offset of the chunk in dR (per-rank layout) and in zp / compact dR, advanced per rank
+    long long qR[CL ? 1 : CPT], qZ[CPT];
+    float2 gsum[CPT][H2];
 #pragma unroll
     for (int j = 0; j < CPT; ++j) {
       act[j] = valid && colok[j];
-      pZ[j] = static_cast<char*>(a.zp) + (i * a.P + (col[j] - a.S_lo)) * ES;
-      pdR[j] = CL ? static_cast<char*>(a.dR) + (i * a.P + (col[j] - a.S_lo)) * ES
-                  : static_cast<char*>(a.dR) + (i * a.h + col[j]) * ES;
+      const uint32_t oX = ((uint32_t)threadIdx.y * a.h + col[j]) * ES;
+      const uint32_t oH = (CL && cls[j] != 0) ? ((uint32_t)threadIdx.y * a.P + (uint32_t)(col[j] - a.S_lo)) * ES : oX;
+      aX[j] = act[j] ? sg.off_a + oX : sg.zero_off;
+      aH[j] = act[j] ? sg.off_b + oH : sg.zero_off;
+      qZ[j] = (i * a.P + (col[j] - a.S_lo)) * ES;
+      if constexpr (!CL) qR[j] = (i * a.h + col[j]) * ES;
 #pragma unroll
-      for (int e = 0; e < V; ++e) gsum[j][e] = 0.f;
+      for (int q = 0; q < H2; ++q) gsum[j][q] = f2(0.f);
     }
-    const long long rank_h = (long long)a.T * a.h * ES;
-    const long long rank_p = (long long)a.T * a.P * ES;
-    raw hs[CL ? CPT : 1];      // compact: this thread's shared chunks of the stream, kept for every rank
 
     for (int m = 0; m < a.t; ++m, ++k) {
-      const uint8_t* stage = ring + (size_t)cs * sg.stage_bytes;
       if (!mbar_wait(bar0 + 8u * cs, cph)) *abort_flag = 1;
-      if (++cs == NS) { cs = 0; cph ^= 1u; }
       const float rs_c = st_cur[m * TY + threadIdx.y];
       const float mu_c = LN ? st_cur[nstat + m * TY + threadIdx.y] : 0.f;
+      const float2 rs2 = f2(rs_c);
 
-      float xh[CPT][V], dxh[CPT][V], dh[CPT][V];
-      float sacc[LN ? 2 : 1];
-#pragma unroll
-      for (int q = 0; q < (LN ? 2 : 1); ++q) sacc[q] = 0.f;
+      float2 xh[CPT][H2], dxh[CPT][H2];
+      raw rdh[CPT];     // stream-gradient chunk, kept packed across the barrier (it is needed only after it)
+      float2 s1 = f2(0.f), s2 = f2(0.f);
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
-        float dx[V], hn[V];
-#pragma unroll
-        for (int e = 0; e < V; ++e) { dx[e] = 0.f; hn[e] = 0.f; dh[j][e] = 0.f; }
-        if (act[j]) {
-          const size_t o = ((size_t)threadIdx.y * a.h + col[j]) * ES;
-          V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
-          if constexpr (CL) {
-            if (cls[j] == 0) {
-              if (m == 0) {
-                const size_t os = ((size_t)threadIdx.y * a.S_hi + col[j]) * ES;
-                hs[j] = lds<raw>(stage + sg.off_d + os);
-                if (has_dh) V_::unpack(lds<raw>(stage + sg.off_e + os), gsum[j]);   // enters the rank sum once
-              }
-              V_::unpack(hs[j], hn);
-            } else {
-              const size_t op = ((size_t)threadIdx.y * a.P + (col[j] - a.S_lo)) * ES;
-              V_::unpack(lds<raw>(stage + sg.off_b + op), hn);
-              if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + op), dh[j]);
-            }
-          } else {
-            V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
-            if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + o), dh[j]);
+        float2 dx[H2], hn[H2];
+        unpack2(lds32<raw>(sb + aX[j]), dx);
+        if (CL && cls[j] == 0) {
+          // compact: the shared chunk of the stream (and of its gradient) arrives with rank 0 only; the
+          // thread parks it in a shared-memory row of its own (written and read by this thread alone)
+          const uint32_t os = ((uint32_t)threadIdx.y * a.S_hi + col[j]) * ES;
+          if (m == 0 && act[j]) {
+            const raw h0 = lds32<raw>(sb + sg.off_d + os);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(keep32 + os), "r"(reinterpret_cast<const uint4&>(h0).x),
+                         "r"(reinterpret_cast<const uint4&>(h0).y), "r"(reinterpret_cast<const uint4&>(h0).z),
+                         "r"(reinterpret_cast<const uint4&>(h0).w) : "memory");
+            if (has_dh) unpack2(lds32<raw>(sb + sg.off_e + os), gsum[j]);   // enters the rank sum once
           }
+          unpack2(lds32<raw>(act[j] ? keep32 + os : sb + sg.zero_off), hn);
+          rdh[j] = zero_raw<raw>();
+        } else {
+          unpack2(lds32<raw>(sb + aH[j]), hn);
+          rdh[j] = has_dh ? lds32<raw>(sb + aH[j] + (act[j] ? off_hc : 0u)) : zero_raw<raw>();
         }
 #pragma unroll
-        for (int e = 0; e < V; ++e) {
-          xh[j][e] = LN ? (act[j] ? (hn[e] - mu_c) * rs_c : 0.f) : hn[e] * rs_c;
-          dxh[j][e] = dx[e] * gam[j][e];
-          if (LN) { sacc[0] += dxh[j][e]; sacc[1] = fmaf(dxh[j][e], xh[j][e], sacc[1]); }
-          else sacc[0] = fmaf(dxh[j][e], xh[j][e], sacc[0]);
-          dgacc[j][e] = fmaf(dx[e], xh[j][e], dgacc[j][e]);
-          if constexpr (LN) dbacc[j][e] += dx[e];
+        for (int q = 0; q < H2; ++q) {
+          xh[j][q] = LN ? mul2(add2(hn[q], f2(-mu_c)), rs2) : mul2(hn[q], rs2);
+          dxh[j][q] = mul2(dx[q], gam[j][q]);
+          if (LN) s1 = add2(s1, dxh[j][q]);
+          s2 = fma2(dxh[j][q], xh[j][q], s2);
+          dgacc[j][q] = fma2(dx[q], xh[j][q], dgacc[j][q]);
+          if constexpr (LN) dbacc[j][q] = add2(dbacc[j][q], dx[q]);
         }
       }
+      float sacc[LN ? 2 : 1];
+      if (LN) { sacc[0] = s1.x + s1.y; sacc[LN ? 1 : 0] = s2.x + s2.y; }
+      else sacc[0] = s2.x + s2.y;
       row_reduce_sync<LN ? 2 : 1>(sacc, red, par);   // CTA barrier: stage fully read
       if (*abort_flag) { dead = true; break; }
-      if (leader && issued < total) { issue(); ++issued; }
+      issue();
+      sb += sg.stage_bytes;
+      if (++cs == NS) { cs = 0; cph ^= 1u; sb = ring32; }
       const float c1 = LN ? sacc[0] * inv_h : 0.f;
-      const float c2 = (LN ? sacc[1] : sacc[0]) * inv_h;
+      const float c2 = (LN ? sacc[LN ? 1 : 0] : sacc[0]) * inv_h;
+      const float2 nc2 = f2(-c2), nc1 = f2(-c1);
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
-        float gg[V];
+        float2 gg[H2], dh[H2];
+        unpack2(rdh[j], dh);
 #pragma unroll
-        for (int e = 0; e < V; ++e) {
-          float tt = fmaf(-xh[j][e], c2, dxh[j][e]);
-          if (LN) tt -= c1;
-          gg[e] = fmaf(rs_c, tt, dh[j][e]);
+        for (int q = 0; q < H2; ++q) {
+          float2 tt = fma2(xh[j][q], nc2, dxh[j][q]);
+          if (LN) tt = add2(tt, nc1);
+          gg[q] = fma2(rs2, tt, dh[q]);
         }
-        if (act[j] && !(CL && cls[j] == 0)) stg<raw>(pdR[j], V_::pack(gg));
-        pdR[j] += CL ? rank_p : rank_h;
+        if constexpr (CL) {
+          if (act[j] && cls[j] != 0) stg<raw>(static_cast<char*>(a.dR) + qZ[j], pack2(gg));
+        } else {
+          if (act[j]) stg<raw>(static_cast<char*>(a.dR) + qR[j], pack2(gg));
+          qR[j] += rank_h;
+        }
         if (cls[j] == 0) {
 #pragma unroll
-          for (int e = 0; e < V; ++e) gsum[j][e] += gg[e];          // fp32 rank sum, m ascending
+          for (int q = 0; q < H2; ++q) gsum[j][q] = add2(gsum[j][q], gg[q]);   // fp32 rank sum, m ascending
         } else {
-          float zp[V];
+          float2 zp[H2];
           if (cls[j] == 1) {
 #pragma unroll
-            for (int e = 0; e < V; ++e) zp[e] = a.alpha * gg[e];    // private gradient carries alpha
+            for (int q = 0; q < H2; ++q) zp[q] = mul2(alpha2, gg[q]);         // private gradient carries alpha
           } else {
 #pragma unroll
-            for (int e = 0; e < V; ++e) {
-              const bool shared = col[j] + e < a.S;
-              gsum[j][e] += shared ? gg[e] : 0.f;
-              zp[e] = shared ? 0.f : a.alpha * gg[e];
+            for (int q = 0; q < H2; ++q) {
+              const bool sx = col[j] + 2 * q < a.S, sy = col[j] + 2 * q + 1 < a.S;
+              gsum[j][q].x += sx ? gg[q].x : 0.f;
+              gsum[j][q].y += sy ? gg[q].y : 0.f;
+              zp[q].x = sx ? 0.f : a.alpha * gg[q].x;
+              zp[q].y = sy ? 0.f : a.alpha * gg[q].y;
             }
           }
-          if (act[j]) stg<raw>(pZ[j], V_::pack(zp));
+          if (act[j]) stg<raw>(static_cast<char*>(a.zp) + qZ[j], pack2(zp));
         }
-        pZ[j] += rank_p;
+        qZ[j] += rank_p;
       }
     }
     if (dead) break;
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
       if (act[j] && cls[j] != 1)
-        stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, V_::pack(gsum[j]));
+        stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, pack2(gsum[j]));
     // park the next group's statistics; the last barrier of this group separates these writes
     // from the reads of group n-1's buffer, the barrier below from the reads of group n+1
 #pragma unroll
@@ -518,6 +589,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
   if (dead) {
     if (leader) {
       atomicExch(status, 5u);
+      const long long issued = (k + NS) < total ? (k + NS) : total;
       for (long long q = k + 1; q < issued; ++q)
         for (uint32_t it = 0; it < (1u << 20); ++it)
           if (mbar_try(bar0 + 8u * (uint32_t)(q % NS), (uint32_t)((q / NS) & 1))) break;
@@ -534,11 +606,11 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
         if (!colok[j]) continue;
-        const float* src = (which == 0 || !LN) ? dgacc[j] : dbacc[LN ? j : 0];
+        const float2* src = (which == 0 || !LN) ? dgacc[j] : dbacc[LN ? j : 0];
 #pragma unroll
-        for (int e = 0; e < V; e += 4)
-          *reinterpret_cast<float4*>(out + (size_t)blockIdx.x * a.h + col[j] + e) =
-              make_float4(src[e], src[e + 1], src[e + 2], src[e + 3]);
+        for (int q = 0; q < H2; q += 2)
+          *reinterpret_cast<float4*>(out + (size_t)blockIdx.x * a.h + col[j] + 2 * q) =
+              make_float4(src[q].x, src[q].y, src[q + 1].x, src[q + 1].y);
       }
       continue;
     }
@@ -548,9 +620,11 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
 #pragma unroll
-      for (int e = 0; e < V; ++e)
-        acc[(size_t)threadIdx.y * per_row + (j * TX + threadIdx.x) * V + e] =
-            (which == 0 || !LN) ? dgacc[j][e] : dbacc[LN ? j : 0][e];
+      for (int q = 0; q < H2; ++q) {
+        const float2 v = (which == 0 || !LN) ? dgacc[j][q] : dbacc[LN ? j : 0][q];
+        acc[(size_t)threadIdx.y * per_row + (j * TX + threadIdx.x) * V + 2 * q] = v.x;
+        acc[(size_t)threadIdx.y * per_row + (j * TX + threadIdx.x) * V + 2 * q + 1] = v.y;
+      }
     __syncthreads();
     if (threadIdx.y == 0) {
 #pragma unroll
@@ -592,13 +666,16 @@ StageGeom stage_geometry(const RowGeom& g, int h, int P, int S_hi, int t, int ES
     sg.off_a = 0; sg.off_b = rowA; sg.off_c = rowA + rowP;
     sg.stage_bytes = rowA + rowP + rowS;
   }
-  sg.stage_bytes = (sg.stage_bytes + 127u) & ~127u;
+  sg.zero_off = sg.stage_bytes;
+  sg.stage_bytes = (sg.stage_bytes + 16u + 127u) & ~127u;
   // fixed part: barriers + abort flag, reduction scratch, row statistics
   size_t off = 0;
   sg.bar_off = (uint32_t)off; off += 8 * kMaxStages + 16;
   off = align_up(off, 16);
   sg.red_off = (uint32_t)off; off += (size_t)2 * g.TY * 16 * 2 * sizeof(float);
   sg.stat_off = (uint32_t)off; off += backward ? (size_t)2 * 2 * t * g.TY * sizeof(float) : 0;
+  off = align_up(off, 128);
+  sg.keep_off = (uint32_t)off; off += (backward && compact) ? (size_t)rowS : 0;
   off = align_up(off, 128);
   sg.ring_off = (uint32_t)off;
   sg.acc_off = sg.ring_off;
