@@ -57,6 +57,8 @@ __device__ __forceinline__ raw lds(const uint8_t* p) { return *reinterpret_cast<
 struct WarpGeom {
   int nstages;
   uint32_t off_a, off_b, off_c, off_d, off_e, stage_bytes;   // d, e: compact layout only
+  uint32_t zero_off;   // 16 zero bytes inside every stage (read by chunks past the row end)
+  uint32_t keep_off;   // compact backward: [kW, S] shared rows of the stream, parked for all ranks of a token
   uint32_t bar_off, ring_off;
   size_t smem;
 };
@@ -86,6 +88,8 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if ((int)threadIdx.x < NS)   // the zero slot of every stage (no copy ever lands there)
+    *reinterpret_cast<uint4*>(ring + (size_t)threadIdx.x * sg.stage_bytes + sg.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
 
   if (warp == kW) {
@@ -129,34 +133,47 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
   }
 
   // ------------------------------------------------------------ consumers: warp w owns token i0 + w
+  // per-lane constants: chunk class and byte offsets inside a stage (the zero slot for chunks past the row end)
+  constexpr int H2 = V / 2;
+  const uint32_t ring32 = smem_u32(ring);
   int col[CPT], cls[CPT];
   bool colok[CPT];
-  float gam[CPT][V], bet[CPT][V];
+  uint32_t oA[CPT], oB[CPT];
+  float2 gam[CPT][H2], bet[LN ? CPT : 1][H2];
 #pragma unroll
   for (int j = 0; j < CPT; ++j) {
     col[j] = (lane + 32 * j) * V;
     colok[j] = col[j] < a.h;
     cls[j] = chunk_class(col[j], V, a.S);
 #pragma unroll
-    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; bet[j][e] = 0.f; }
+    for (int q = 0; q < H2; ++q) { gam[j][q] = f2(0.f); if constexpr (LN) bet[j][q] = f2(0.f); }
+    oA[j] = oB[j] = sg.zero_off;
     if (colok[j]) {
-      V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
-      if (LN && a.beta) V_::unpack(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
+      unpack2(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+      if constexpr (LN) {
+        if (a.beta) unpack2(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
+      }
+      const uint32_t priv = ((uint32_t)warp * a.P + (uint32_t)(col[j] - a.S_lo)) * ES;
+      if (cls[j] != 0) oB[j] = sg.off_b + priv;
+      if (CL) { if (cls[j] != 0) oA[j] = sg.off_a + priv; }
+      else oA[j] = sg.off_a + ((uint32_t)warp * a.h + col[j]) * ES;
     }
   }
   const float inv_h = 1.0f / (float)a.h;
+  const float2 alpha2 = f2(a.alpha);
   const long long rank_h = (long long)a.T * a.h * ES;
   const long long rank_hn = CL ? (long long)a.T * a.P * ES : rank_h;   // rank stride of the stream's (private) rows
   int s = 0; uint32_t ph = 0;
+  uint32_t sb = ring32;
   bool dead = false;
   for (int n = 0; n < my_groups && !dead; ++n) {
     const long long i = (blockIdx.x + (long long)n * gridDim.x) * kW + warp;
     const bool valid = i < a.T;
-    float zs[CPT][V];
+    float2 zs[CPT][H2];
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
 #pragma unroll
-      for (int e = 0; e < V; ++e) zs[j][e] = 0.f;
+      for (int q = 0; q < H2; ++q) zs[j][q] = f2(0.f);
     // compact: column l of the private rows sits at l - S
     char* pHn = CL ? static_cast<char*>(a.Hn) + (i * a.P - a.S_lo) * ES : static_cast<char*>(a.Hn) + i * a.h * ES;
     char* pX = static_cast<char*>(a.X) + i * a.h * ES;
@@ -164,82 +181,88 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
     float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
     for (int m = 0; m < a.t; ++m) {
       if (!mbar_wait(full0 + 8u * s, ph, abort_flag)) { dead = true; break; }
-      const uint8_t* stage = ring + (size_t)s * sg.stage_bytes;
-      float hn[CPT][V];
-      float st = 0.f;
+      float2 hn[CPT][H2];
+      float2 acc = f2(0.f);
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
-        float r[V], zp[V];
-#pragma unroll
-        for (int e = 0; e < V; ++e) { r[e] = 0.f; zp[e] = 0.f; }
         const bool act = valid && colok[j];
-        if (act) {
-          if constexpr (CL) {
-            if (cls[j] != 0) {
-              const size_t op = ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES;
-              V_::unpack(lds<raw>(stage + sg.off_a + op), r);
-              V_::unpack(lds<raw>(stage + sg.off_b + op), zp);
-            } else if (m == 0) {      // the shared part of the new stream, formed once: zs + Rs
-              float rs0[V];
-              const size_t os = ((size_t)warp * a.S_hi + col[j]) * ES;
-              V_::unpack(lds<raw>(stage + sg.off_c + os), zs[j]);
-              V_::unpack(lds<raw>(stage + sg.off_d + os), rs0);
+        if (m == 0 && cls[j] != 1 && colok[j]) {
+          const uint32_t os = ((uint32_t)warp * a.S_hi + col[j]) * ES;
+          unpack2(lds32<raw>(sb + sg.off_c + os), zs[j]);
+          if constexpr (CL) {       // the shared part of the new stream, formed once: zs + Rs
+            float2 r0[H2];
+            unpack2(lds32<raw>(sb + sg.off_d + os), r0);
 #pragma unroll
-              for (int e = 0; e < V; ++e) zs[j][e] += rs0[e];
-            }
-          } else {
-            V_::unpack(lds<raw>(stage + sg.off_a + ((size_t)warp * a.h + col[j]) * ES), r);
-            if (cls[j] != 0) V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES), zp);
-            if (m == 0 && cls[j] != 1) V_::unpack(lds<raw>(stage + sg.off_c + ((size_t)warp * a.S_hi + col[j]) * ES), zs[j]);
+            for (int q = 0; q < H2; ++q) zs[j][q] = add2(zs[j][q], r0[q]);
           }
         }
         if (cls[j] == 0) {
+          if constexpr (CL) {
 #pragma unroll
-          for (int e = 0; e < V; ++e) hn[j][e] = zs[j][e] + r[e];
-        } else if (cls[j] == 1) {
+            for (int q = 0; q < H2; ++q) hn[j][q] = zs[j][q];
+          } else {
+            float2 r[H2];
+            unpack2(lds32<raw>(sb + oA[j]), r);
 #pragma unroll
-          for (int e = 0; e < V; ++e) hn[j][e] = fmaf(a.alpha, zp[e], r[e]);
+            for (int q = 0; q < H2; ++q) hn[j][q] = add2(zs[j][q], r[q]);
+          }
         } else {
+          float2 r[H2], zp[H2];
+          unpack2(lds32<raw>(sb + oA[j]), r);
+          unpack2(lds32<raw>(sb + oB[j]), zp);
+          if (cls[j] == 1) {
 #pragma unroll
-          for (int e = 0; e < V; ++e) hn[j][e] = (col[j] + e < a.S ? zs[j][e] : a.alpha * zp[e]) + r[e];
+            for (int q = 0; q < H2; ++q) hn[j][q] = fma2(alpha2, zp[q], r[q]);
+          } else {   // the one chunk that straddles the partition
+#pragma unroll
+            for (int q = 0; q < H2; ++q) {
+              hn[j][q].x = (col[j] + 2 * q < a.S ? zs[j][q].x : a.alpha * zp[q].x) + r[q].x;
+              hn[j][q].y = (col[j] + 2 * q + 1 < a.S ? zs[j][q].y : a.alpha * zp[q].y) + r[q].y;
+            }
+          }
         }
         if constexpr (CL) {
-          if (act && cls[j] != 0) stg<raw>(pHn + (long long)col[j] * ES, V_::pack(hn[j]));
-          else if (act && m == 0) stg<raw>(static_cast<char*>(a.Hns) + (i * a.S_hi + col[j]) * ES, V_::pack(hn[j]));
+          if (act && cls[j] != 0) stg<raw>(pHn + (long long)col[j] * ES, pack2(hn[j]));
+          else if (act && m == 0) stg<raw>(static_cast<char*>(a.Hns) + (i * a.S_hi + col[j]) * ES, pack2(hn[j]));
         } else {
-          if (act) stg<raw>(pHn + (long long)col[j] * ES, V_::pack(hn[j]));
+          if (act) stg<raw>(pHn + (long long)col[j] * ES, pack2(hn[j]));
         }
 #pragma unroll
-        for (int e = 0; e < V; ++e) st = LN ? st + hn[j][e] : fmaf(hn[j][e], hn[j][e], st);
+        for (int q = 0; q < H2; ++q) acc = LN ? add2(acc, hn[j][q]) : fma2(hn[j][q], hn[j][q], acc);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8u * s);      // this warp is done with the stage
-      if (++s == NS) { s = 0; ph ^= 1u; }
-      st = warp_sum(st);
+      sb += sg.stage_bytes;
+      if (++s == NS) { s = 0; ph ^= 1u; sb = ring32; }
+      const float st = warp_sum(acc.x + acc.y);
       float mu = 0.f, rs;
       if (LN) {
         mu = st * inv_h;
-        float sq = 0.f;
+        float2 sq2 = f2(0.f);
 #pragma unroll
-        for (int j = 0; j < CPT; ++j)
+        for (int j = 0; j < CPT; ++j) {
+          if (!colok[j]) continue;
 #pragma unroll
-          for (int e = 0; e < V; ++e) {
-            const float d = (valid && colok[j]) ? hn[j][e] - mu : 0.f;
-            sq = fmaf(d, d, sq);
+          for (int q = 0; q < H2; ++q) {
+            const float2 d = add2(hn[j][q], f2(-mu));
+            sq2 = fma2(d, d, sq2);
           }
-        rs = rsqrtf(fmaf(warp_sum(sq), inv_h, a.eps));
+        }
+        rs = rsqrtf(fmaf(warp_sum(sq2.x + sq2.y), inv_h, a.eps));
       } else {
         rs = rsqrtf(fmaf(st, inv_h, a.eps));
       }
+      const float2 rs2 = f2(rs);
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
-        float x[V];
+        float2 x[H2];
 #pragma unroll
-        for (int e = 0; e < V; ++e) {
-          if (LN) x[e] = fmaf(hn[j][e] - mu, rs * gam[j][e], bet[j][e]);
-          else x[e] = hn[j][e] * (rs * gam[j][e]);
+        for (int q = 0; q < H2; ++q) {
+          const float2 sc = mul2(rs2, gam[j][q]);
+          if constexpr (LN) x[q] = fma2(add2(hn[j][q], f2(-mu)), sc, bet[j][q]);
+          else x[q] = mul2(hn[j][q], sc);
         }
-        if (valid && colok[j]) stg<raw>(pX + (long long)col[j] * ES, V_::pack(x));
+        if (valid && colok[j]) stg<raw>(pX + (long long)col[j] * ES, pack2(x));
       }
       if (valid && lane == 0) {
         *rstd_p = rs;
@@ -277,18 +300,21 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if ((int)threadIdx.x < NS)   // the zero slot of every stage (no copy ever lands there)
+    *reinterpret_cast<uint4*>(ring + (size_t)threadIdx.x * sg.stage_bytes + sg.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
 
+  constexpr int H2 = V / 2;
   int col[CPT], cls[CPT];
   bool colok[CPT];
-  float gam[CPT][V], dgacc[CPT][V], dbacc[LN ? CPT : 1][V];
+  float2 gam[CPT][H2], dgacc[CPT][H2], dbacc[LN ? CPT : 1][H2];
 #pragma unroll
   for (int j = 0; j < CPT; ++j) {
     col[j] = (lane + 32 * j) * V;
     colok[j] = col[j] < a.h;
     cls[j] = chunk_class(col[j], V, a.S);
 #pragma unroll
-    for (int e = 0; e < V; ++e) { gam[j][e] = 0.f; dgacc[j][e] = 0.f; if constexpr (LN) dbacc[j][e] = 0.f; }
+    for (int q = 0; q < H2; ++q) { gam[j][q] = f2(0.f); dgacc[j][q] = f2(0.f); if constexpr (LN) dbacc[j][q] = f2(0.f); }
   }
 
   if (warp == kW) {
@@ -339,12 +365,19 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
     }
   } else {
     // ---------------------------------------------------------- consumers
+    // Inactive chunks (past the row end, or a token past T) read the zero slot every stage carries, so
+    // they add exact zeros to the sums and the loads need no predicates.
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
-      if (colok[j]) V_::unpack(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+      if (colok[j]) unpack2(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
+    const uint32_t ring32 = smem_u32(ring);
+    const uint32_t keep32 = smem_u32(smem + sg.keep_off);
+    const uint32_t off_hc = sg.off_c - sg.off_b;   // from a chunk of the stream to the same chunk of its gradient
     const float inv_h = 1.0f / (float)a.h;
+    const float2 alpha2 = f2(a.alpha);
     const long long rank_h = (long long)a.T * a.h * ES, rank_p = (long long)a.T * a.P * ES;
     int s = 0; uint32_t ph = 0;
+    uint32_t sb = ring32;
     bool dead = false;
     // lane m holds rstd (mean) of rank m for the current token; the next token's are fetched a group ahead
     auto load_stat = [&](const float* base, int n) -> float {
@@ -358,116 +391,123 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
       const float rs_lane = rs_next, mu_lane = mu_next;
       rs_next = load_stat(a.rstd, n + 1);
       if (LN) mu_next = load_stat(a.mean, n + 1);
-      float gsum[CPT][V];
+      float2 gsum[CPT][H2];
+      // stage-relative addresses of this token's dX chunk and stream chunk; compact: private chunks sit at
+      // l - S in rows of P, shared chunks come from a row the warp parks in shared memory for all ranks
+      uint32_t aX[CPT], aH[CPT];
 #pragma unroll
-      for (int j = 0; j < CPT; ++j)
+      for (int j = 0; j < CPT; ++j) {
+        const bool act = valid && colok[j];
+        const uint32_t oX = ((uint32_t)warp * a.h + col[j]) * ES;
+        const uint32_t oH = (CL && cls[j] != 0) ? ((uint32_t)warp * a.P + (uint32_t)(col[j] - a.S_lo)) * ES : oX;
+        aX[j] = act ? sg.off_a + oX : sg.zero_off;
+        aH[j] = act ? sg.off_b + oH : sg.zero_off;
 #pragma unroll
-        for (int e = 0; e < V; ++e) gsum[j][e] = 0.f;
+        for (int q = 0; q < H2; ++q) gsum[j][q] = f2(0.f);
+      }
       char* pdR = CL ? static_cast<char*>(a.dR) + (i * a.P - a.S_lo) * ES : static_cast<char*>(a.dR) + i * a.h * ES;
       char* pZ = static_cast<char*>(a.zp) + (i * a.P - a.S_lo) * ES;
-      raw hs[CL ? CPT : 1];      // compact: this lane's shared chunks of the stream, kept for every rank
       for (int m = 0; m < a.t; ++m) {
         if (!mbar_wait(full0 + 8u * s, ph, abort_flag)) { dead = true; break; }
-        const uint8_t* stage = ring + (size_t)s * sg.stage_bytes;
         const float rs = __shfl_sync(0xffffffffu, rs_lane, m);
         const float mu = LN ? __shfl_sync(0xffffffffu, mu_lane, m) : 0.f;
+        const float2 rs2 = f2(rs);
         if constexpr (CL) {
           if (m == 0) {
 #pragma unroll
             for (int j = 0; j < CPT; ++j) {
-              hs[j] = zero_raw<raw>();
               if (valid && colok[j] && cls[j] == 0) {
-                const size_t os = ((size_t)warp * a.S_hi + col[j]) * ES;
-                hs[j] = lds<raw>(stage + sg.off_d + os);
-                if (has_dh) V_::unpack(lds<raw>(stage + sg.off_e + os), gsum[j]);   // enters the rank sum once
+                const uint32_t os = ((uint32_t)warp * a.S_hi + col[j]) * ES;
+                const raw h0 = lds32<raw>(sb + sg.off_d + os);
+                const uint4& u = reinterpret_cast<const uint4&>(h0);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(keep32 + os), "r"(u.x), "r"(u.y), "r"(u.z), "r"(u.w)
+                             : "memory");
+                if (has_dh) unpack2(lds32<raw>(sb + sg.off_e + os), gsum[j]);   // enters the rank sum once
               }
             }
           }
         }
         // pass 1: row statistics and norm-parameter gradients
-        float s1 = 0.f, s2 = 0.f;
+        float2 s1 = f2(0.f), s2 = f2(0.f);
 #pragma unroll
         for (int j = 0; j < CPT; ++j) {
-          if (!(valid && colok[j])) continue;
-          float dx[V], hn[V];
-          const size_t o = ((size_t)warp * a.h + col[j]) * ES;
-          V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
-          if constexpr (CL) {
-            if (cls[j] == 0) V_::unpack(hs[j], hn);
-            else V_::unpack(lds<raw>(stage + sg.off_b + ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES), hn);
-          } else {
-            V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
-          }
+          float2 dx[H2], hn[H2];
+          unpack2(lds32<raw>(sb + aX[j]), dx);
+          uint32_t hsrc = sb + aH[j];
+          if (CL && cls[j] == 0) hsrc = (valid && colok[j]) ? keep32 + ((uint32_t)warp * a.S_hi + col[j]) * ES : sb + sg.zero_off;
+          unpack2(lds32<raw>(hsrc), hn);
 #pragma unroll
-          for (int e = 0; e < V; ++e) {
-            const float xh = (hn[e] - mu) * rs;
-            const float dxh = dx[e] * gam[j][e];
-            if (LN) s1 += dxh;
-            s2 = fmaf(dxh, xh, s2);
-            dgacc[j][e] = fmaf(dx[e], xh, dgacc[j][e]);
-            if constexpr (LN) dbacc[j][e] += dx[e];
+          for (int q = 0; q < H2; ++q) {
+            const float2 xh = LN ? mul2(add2(hn[q], f2(-mu)), rs2) : mul2(hn[q], rs2);
+            const float2 dxh = mul2(dx[q], gam[j][q]);
+            if (LN) s1 = add2(s1, dxh);
+            s2 = fma2(dxh, xh, s2);
+            dgacc[j][q] = fma2(dx[q], xh, dgacc[j][q]);
+            if constexpr (LN) dbacc[j][q] = add2(dbacc[j][q], dx[q]);
           }
         }
-        const float c1 = LN ? warp_sum(s1) * inv_h : 0.f;
-        const float c2 = warp_sum(s2) * inv_h;
+        const float c1 = LN ? warp_sum(s1.x + s1.y) * inv_h : 0.f;
+        const float c2 = warp_sum(s2.x + s2.y) * inv_h;
+        const float2 nc1 = f2(-c1), nc2 = f2(-c2);
         // pass 2: gradients (the stage is re-read: cheaper than keeping the row in registers)
 #pragma unroll
         for (int j = 0; j < CPT; ++j) {
           if (!(valid && colok[j])) continue;
-          float dx[V], hn[V], dh[V], gg[V];
-          const size_t o = ((size_t)warp * a.h + col[j]) * ES;
-          V_::unpack(lds<raw>(stage + sg.off_a + o), dx);
+          float2 dx[H2], hn[H2], dh[H2], gg[H2];
+          unpack2(lds32<raw>(sb + aX[j]), dx);
+          if (CL && cls[j] == 0) {
+            unpack2(lds32<raw>(keep32 + ((uint32_t)warp * a.S_hi + col[j]) * ES), hn);
 #pragma unroll
-          for (int e = 0; e < V; ++e) dh[e] = 0.f;
-          if constexpr (CL) {
-            if (cls[j] == 0) {
-              V_::unpack(hs[j], hn);
-            } else {
-              const size_t op = ((size_t)warp * a.P + (col[j] - a.S_lo)) * ES;
-              V_::unpack(lds<raw>(stage + sg.off_b + op), hn);
-              if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + op), dh);
-            }
+            for (int q = 0; q < H2; ++q) dh[q] = f2(0.f);
           } else {
-            V_::unpack(lds<raw>(stage + sg.off_b + o), hn);
-            if (has_dh) V_::unpack(lds<raw>(stage + sg.off_c + o), dh);
+            unpack2(lds32<raw>(sb + aH[j]), hn);
+            if (has_dh) {
+              unpack2(lds32<raw>(sb + aH[j] + off_hc), dh);
+            } else {
+#pragma unroll
+              for (int q = 0; q < H2; ++q) dh[q] = f2(0.f);
+            }
           }
 #pragma unroll
-          for (int e = 0; e < V; ++e) {
-            const float xh = (hn[e] - mu) * rs;
-            float tt = fmaf(-xh, c2, dx[e] * gam[j][e]);
-            if (LN) tt -= c1;
-            gg[e] = fmaf(rs, tt, dh[e]);
+          for (int q = 0; q < H2; ++q) {
+            const float2 xh = LN ? mul2(add2(hn[q], f2(-mu)), rs2) : mul2(hn[q], rs2);
+            float2 tt = fma2(xh, nc2, mul2(dx[q], gam[j][q]));
+            if (LN) tt = add2(tt, nc1);
+            gg[q] = fma2(rs2, tt, dh[q]);
           }
-          if (!(CL && cls[j] == 0)) stg<raw>(pdR + (long long)col[j] * ES, V_::pack(gg));
+          if (!(CL && cls[j] == 0)) stg<raw>(pdR + (long long)col[j] * ES, pack2(gg));
           if (cls[j] == 0) {
 #pragma unroll
-            for (int e = 0; e < V; ++e) gsum[j][e] += gg[e];          // fp32 rank sum, m ascending
+            for (int q = 0; q < H2; ++q) gsum[j][q] = add2(gsum[j][q], gg[q]);   // fp32 rank sum, m ascending
           } else {
-            float zp[V];
+            float2 zp[H2];
             if (cls[j] == 1) {
 #pragma unroll
-              for (int e = 0; e < V; ++e) zp[e] = a.alpha * gg[e];    // private gradient carries alpha
+              for (int q = 0; q < H2; ++q) zp[q] = mul2(alpha2, gg[q]);         // private gradient carries alpha
             } else {
 #pragma unroll
-              for (int e = 0; e < V; ++e) {
-                const bool shared = col[j] + e < a.S;
-                gsum[j][e] += shared ? gg[e] : 0.f;
-                zp[e] = shared ? 0.f : a.alpha * gg[e];
+              for (int q = 0; q < H2; ++q) {
+                const bool sx = col[j] + 2 * q < a.S, sy = col[j] + 2 * q + 1 < a.S;
+                gsum[j][q].x += sx ? gg[q].x : 0.f;
+                gsum[j][q].y += sy ? gg[q].y : 0.f;
+                zp[q].x = sx ? 0.f : a.alpha * gg[q].x;
+                zp[q].y = sy ? 0.f : a.alpha * gg[q].y;
               }
             }
-            stg<raw>(pZ + (long long)col[j] * ES, V_::pack(zp));
+            stg<raw>(pZ + (long long)col[j] * ES, pack2(zp));
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * s);
-        if (++s == NS) { s = 0; ph ^= 1u; }
+        sb += sg.stage_bytes;
+        if (++s == NS) { s = 0; ph ^= 1u; sb = ring32; }
         pdR += CL ? rank_p : rank_h; pZ += rank_p;
       }
       if (dead) break;
 #pragma unroll
       for (int j = 0; j < CPT; ++j)
         if (valid && colok[j] && cls[j] != 1)
-          stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, V_::pack(gsum[j]));
+          stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, pack2(gsum[j]));
     }
   }
 
@@ -483,8 +523,11 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
       for (int j = 0; j < CPT; ++j)
         if (colok[j])
 #pragma unroll
-          for (int e = 0; e < V; ++e)
-            acc[(size_t)warp * a.h + col[j] + e] = (which == 0 || !LN) ? dgacc[j][e] : dbacc[LN ? j : 0][e];
+          for (int q = 0; q < H2; ++q) {
+            const float2 v = (which == 0 || !LN) ? dgacc[j][q] : dbacc[LN ? j : 0][q];
+            acc[(size_t)warp * a.h + col[j] + 2 * q] = v.x;
+            acc[(size_t)warp * a.h + col[j] + 2 * q + 1] = v.y;
+          }
     }
     __syncthreads();
     for (int c = threadIdx.x; c < a.h; c += blockDim.x) {
@@ -516,9 +559,11 @@ WarpGeom warp_geometry(int h, int P, int S_hi, int ES, bool backward, bool has_c
     g.off_a = 0; g.off_b = rowA; g.off_c = rowA + rowP;
     g.stage_bytes = rowA + rowP + rowS;
   }
-  g.stage_bytes = (g.stage_bytes + 127u) & ~127u;
+  g.zero_off = g.stage_bytes;
+  g.stage_bytes = (g.stage_bytes + 16u + 127u) & ~127u;
   g.bar_off = 0;
-  g.ring_off = (uint32_t)align_up(16 * kMaxStages + 16, 128);
+  g.keep_off = (uint32_t)align_up(16 * kMaxStages + 16, 128);
+  g.ring_off = (uint32_t)align_up(g.keep_off + ((backward && compact) ? rowS : 0u), 128);
   int ns = (int)((budget - g.ring_off) / g.stage_bytes);
   if (ns > kMaxStages) ns = kMaxStages;
   g.nstages = ns;
