@@ -77,9 +77,17 @@ typedef enum {
   CAAT_OPT_ROWS = 5,            /* row kernels: 0 = automatic (default: warp-per-token kernels for
                                    rows of at most 1024 bf16 channels, bulk-copy staged kernels
                                    otherwise), 1 = plain-load kernels, 2 = staged kernels always */
-  CAAT_OPT_DECODE = 6           /* 0 = automatic (default: forward calls with at most 64 tokens
+  CAAT_OPT_DECODE = 6,          /* 0 = automatic (default: forward calls with at most 64 tokens
                                    stream the weights with swapped GEMM operands),
                                    1 = always use the large-batch forward                */
+  CAAT_OPT_BACKWARD_REDUCE = 7  /* precision of the backward rank sum on the shared channels
+                                   (Section 4, "fp32 accumulation"); a numerics-study switch:
+                                   0 = the ranks' gradients are summed in fp32 as computed (default);
+                                   1 = each rank's gradient is first rounded to the run dtype (what
+                                       a 16-bit all-reduce carries), the sum runs in fp32;
+                                   2 = rounded, and the running sum is rounded to the run dtype
+                                       after every addition (accumulation in 16 bit).
+                                   1 and 2 run on the plain-load row kernels.              */
 } caat_option;
 
 /* Creates a context for hidden size h, MLP width ffn, t ranks, synchronisation

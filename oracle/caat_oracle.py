@@ -183,13 +183,42 @@ def norm_param_gradients(dX, Hn, rstd, mean, norm: int):
     return dgamma, dbeta
 
 
-def backward_partial_channel_reduce(g, S: int, alpha: float = 1.0) -> np.ndarray:
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """Round to bfloat16 (8 significand bits, round to nearest even) and widen back to float64.
+    Written on the bit pattern of the float32 value: add 0x7FFF plus the last kept bit, drop 16 bits."""
+    f = np.asarray(x, dtype=np.float64).astype(np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16) << 16
+    out = (r & 0xFFFFFFFF).astype(np.uint32).view(np.float32).astype(np.float64)
+    return np.where(np.isfinite(f), out, f.astype(np.float64))
+
+
+def backward_partial_channel_reduce(g, S: int, alpha: float = 1.0, reduce_mode: int = 0) -> np.ndarray:
     """B4: the reduce placed after the norm's backward (operation 'h' of Fig. 2b).
 
     dZt[m, i, l] = sum_m' g[m', i, l] for l < S, alpha * g[m, i, l] for l >= S.
     It is the transpose of the forward partial channel-reduce.
+
+    reduce_mode models the precision of the rank sum that Section 4 discusses (16-bit runs only):
+      0  exact sum of the ranks' gradients (what fp32 accumulation approximates),
+      1  every rank's term rounded to bfloat16 first (a 16-bit all-reduce payload), summed exactly,
+      2  terms rounded to bfloat16 and the running sum rounded to bfloat16 after every addition,
+         m ascending (accumulation in 16 bit).
     """
-    return partial_channel_reduce(np.asarray(g, dtype=np.float64), S, alpha)
+    g = np.asarray(g, dtype=np.float64)
+    if reduce_mode == 0:
+        return partial_channel_reduce(g, S, alpha)
+    t = g.shape[0]
+    dZt = np.empty_like(g)
+    acc = np.zeros_like(g[0, :, :S])
+    for m in range(t):
+        acc = acc + round_bf16(g[m, :, :S])
+        if reduce_mode == 2:
+            acc = round_bf16(acc)
+    for m in range(t):
+        dZt[m, :, :S] = acc
+    dZt[:, :, S:] = alpha * g[:, :, S:]
+    return dZt
 
 
 def data_gradient(dZt, W) -> np.ndarray:
@@ -205,12 +234,12 @@ def weight_gradient(dZt, Y) -> np.ndarray:
 
 
 def rowpar_backward(dX, dHn, Y, W, Hn, rstd, mean, gamma, *, S: int, alpha: float = 1.0,
-                    norm: int = RMSNORM) -> dict:
+                    norm: int = RMSNORM, reduce_mode: int = 0) -> dict:
     """Exact gradient of rowpar_forward w.r.t. (Y, W, R, gamma, beta), contracted with
     upstream dX (through the norm) and dHn (through the residual stream)."""
     g = residual_stream_gradient(dX, dHn, Hn, rstd, mean, gamma, norm)   # B1
     dgamma, dbeta = norm_param_gradients(dX, Hn, rstd, mean, norm)       # B3
-    dZt = backward_partial_channel_reduce(g, S, alpha)                   # B4
+    dZt = backward_partial_channel_reduce(g, S, alpha, reduce_mode)      # B4
     dY = data_gradient(dZt, W)                                           # B5
     dW = weight_gradient(dZt, Y)                                         # B6
     return {"g": g, "dR": g, "dZt": dZt, "dY": dY, "dW": dW, "dgamma": dgamma, "dbeta": dbeta}

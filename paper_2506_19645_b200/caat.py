@@ -21,7 +21,8 @@ CAAT_ATTN_OUT, CAAT_MLP_DOWN = 0, 1
 (CAAT_OK, CAAT_EINVAL, CAAT_ESHAPE, CAAT_EALIGN, CAAT_EWORKSPACE, CAAT_EUNSUPPORTED, CAAT_ECUDA,
  CAAT_ETIMEOUT, CAAT_ELIMIT) = range(9)
 CAAT_NOALLOC_SCRATCH_BYTES = 32 * 1024 * 1024
-CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM, CAAT_OPT_ROWS, CAAT_OPT_DECODE = range(7)
+(CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM, CAAT_OPT_ROWS,
+ CAAT_OPT_DECODE, CAAT_OPT_BACKWARD_REDUCE) = range(8)
 RMSNORM, LAYERNORM = 0, 1
 
 if not os.path.exists(LIB_PATH):

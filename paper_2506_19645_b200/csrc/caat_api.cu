@@ -194,7 +194,8 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
                reinterpret_cast<float*>(wsb + L.dgpart_off), reinterpret_cast<float*>(wsb + L.dbpart_off),
                dgamma, dbeta, t, T, h, S, L.S_lo, L.S_hi, L.P, (float)ctx->alpha, ctx->norm};
   a.compact = compact; a.Hns = Hns; a.dHns = dHns;
-  ce = launch_rows_backward(a, ctx->dtype, ctx->direct_rows, st);
+  a.reduce_mode = ctx->bwd_reduce;
+  ce = launch_rows_backward(a, ctx->dtype, ctx->bwd_reduce ? 1 : ctx->direct_rows, st);
   if (ce != cudaSuccess) return cuda_fail(ce);
 
   if (tc_gemm_usable(ctx, K_r)) {
@@ -254,7 +255,7 @@ caat_status caat_create(int h, int ffn, int t, double p, caat_dtype dtype, caat_
   c->h = h; c->ffn = ffn; c->t = t; c->p = p; c->dtype = dtype;
   c->S = (int)std::floor((double)h * p);   // Eq. A3: l < floor(h p) is shared
   c->alpha = std::sqrt((double)t);         // Section 4: private channels times sqrt(r)
-  c->norm = 0; c->eps = 1e-5; c->force_simt = 0; c->direct_rows = 0; c->no_decode = 0;
+  c->norm = 0; c->eps = 1e-5; c->force_simt = 0; c->direct_rows = 0; c->no_decode = 0; c->bwd_reduce = 0;
   *out = c;
   return CAAT_OK;
 }
@@ -284,6 +285,9 @@ caat_status caat_set_option(caat_ctx* ctx, caat_option opt, double value) {
     case CAAT_OPT_ROWS:
       if (value != 0.0 && value != 1.0 && value != 2.0) return CAAT_EINVAL;
       ctx->direct_rows = (int)value; return CAAT_OK;
+    case CAAT_OPT_BACKWARD_REDUCE:
+      if (value != 0.0 && value != 1.0 && value != 2.0) return CAAT_EINVAL;
+      ctx->bwd_reduce = (int)value; return CAAT_OK;
   }
   return CAAT_EINVAL;
 }

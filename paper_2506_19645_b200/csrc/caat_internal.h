@@ -18,6 +18,7 @@ struct caat_ctx {
   int force_simt;  // CAAT_OPT_GEMM
   int direct_rows; // CAAT_OPT_ROWS
   int no_decode;   // CAAT_OPT_DECODE
+  int bwd_reduce;  // CAAT_OPT_BACKWARD_REDUCE
 };
 
 namespace caat {
@@ -145,6 +146,7 @@ struct RowBwdArgs {
   // [t, T, P]; the shared residual gradient is gs itself (dRs = dZt on the shared channels)
   int compact;
   const void *Hns, *dHns;
+  int reduce_mode;   // CAAT_OPT_BACKWARD_REDUCE (plain-load kernels only)
 };
 cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
 cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,

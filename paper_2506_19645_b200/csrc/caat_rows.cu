@@ -288,8 +288,16 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
         if (act[j] && !(CL && cls[j] == 0)) stg<raw>(pdR[j], V_::pack(g));
         pdR[j] += CL ? rank_p : rank_h;
         if (cls[j] == 0) {
+          if (a.reduce_mode == 0) {
 #pragma unroll
-          for (int e = 0; e < V; ++e) gsum[j][e] += g[e];          // fp32 rank sum, m ascending
+            for (int e = 0; e < V; ++e) gsum[j][e] += g[e];          // fp32 rank sum, m ascending
+          } else {   // numerics study: the rank's term as a 16-bit wire carries it; optionally a 16-bit running sum
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              const float sum = gsum[j][e] + V_::round(g[e]);
+              gsum[j][e] = a.reduce_mode == 2 ? V_::round(sum) : sum;
+            }
+          }
         } else {
           float zp[V];
           if (cls[j] == 1) {
@@ -299,7 +307,8 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
 #pragma unroll
             for (int e = 0; e < V; ++e) {
               const bool shared = col[j] + e < a.S;
-              gsum[j][e] += shared ? g[e] : 0.f;
+              const float term = shared ? (a.reduce_mode ? V_::round(g[e]) : g[e]) : 0.f;
+              gsum[j][e] = a.reduce_mode == 2 ? V_::round(gsum[j][e] + term) : gsum[j][e] + term;
               zp[e] = shared ? 0.f : a.alpha * g[e];
             }
           }

@@ -15,7 +15,8 @@ from tests.helpers import f64, to_dtype
 GUARD = 64  # canary elements after every output buffer
 
 
-def make_ctx(t, h, ffn, dtype, S=None, p=0.5, alpha=None, norm=0, eps=None, force_simt=False, direct_rows=False, no_decode=False):
+def make_ctx(t, h, ffn, dtype, S=None, p=0.5, alpha=None, norm=0, eps=None, force_simt=False, direct_rows=False, no_decode=False,
+             bwd_reduce=0):
     ctx = caat.Context(h, ffn, t, p, dtype)
     if S is not None:
         ctx.set_option(caat.CAAT_OPT_SHARED_CHANNELS, S)
@@ -33,6 +34,9 @@ def make_ctx(t, h, ffn, dtype, S=None, p=0.5, alpha=None, norm=0, eps=None, forc
         ctx.set_option(caat.CAAT_OPT_ROWS, int(direct_rows))
     if no_decode:
         ctx.set_option(caat.CAAT_OPT_DECODE, 1)
+    if bwd_reduce:
+        ctx.set_option(caat.CAAT_OPT_BACKWARD_REDUCE, bwd_reduce)
+    ctx._bwd_reduce = bwd_reduce
     return ctx
 
 
@@ -111,4 +115,5 @@ def gpu_backward(ctx, layer, d, Hn, rstd, mean, with_dHn=True):
 def oracle_backward(ctx, d, Hn, rstd, mean, with_dHn=True):
     return O.rowpar_backward(f64(d["dX"]), f64(d["dHn"]) if with_dHn else None, f64(d["Y"]), f64(d["W"]),
                              f64(Hn), f64(rstd), f64(mean) if mean is not None else None, f64(d["gamma"]),
-                             S=ctx.shared_channels, alpha=ctx.private_scale, norm=ctx.norm)
+                             S=ctx.shared_channels, alpha=ctx.private_scale, norm=ctx.norm,
+                             reduce_mode=getattr(ctx, "_bwd_reduce", 0))

@@ -335,6 +335,42 @@ def test_block_chains_through_residual_and_matches_finite_differences():
         assert np.abs(num - b[gname]).max() / max(1.0, np.abs(num).max()) < 2e-7, name
 
 
+# ---------------------------------------------------------------- precision models of the backward reduce
+def test_round_bf16_matches_library_cast():
+    rng = _rng(31)
+    x = np.concatenate([rng.standard_normal(4096) * 10.0 ** rng.integers(-6, 6, 4096),
+                        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895313892515355e38, 1e-40])])
+    ref = torch.tensor(x, dtype=torch.float64).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(O.round_bf16(x), ref)
+    # ties go to the even significand: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert O.round_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert O.round_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+
+
+def test_reduce_precision_models():
+    rng = _rng(32)
+    t, T, h, S = 16, 64, 32, 16
+    g = rng.standard_normal((t, T, h))
+    exact = O.backward_partial_channel_reduce(g, S, 2.0)
+    wire = O.backward_partial_channel_reduce(g, S, 2.0, reduce_mode=1)
+    acc16 = O.backward_partial_channel_reduce(g, S, 2.0, reduce_mode=2)
+    # private channels are untouched by the model; shared ones are identical on every rank
+    for r in (wire, acc16):
+        np.testing.assert_array_equal(r[:, :, S:], exact[:, :, S:])
+        assert all(np.array_equal(r[0, :, :S], r[m, :, :S]) for m in range(t))
+    # mode 1 is the exact sum of rounded terms; mode 2 stays on the bfloat16 grid
+    np.testing.assert_allclose(wire[0, :, :S], O.round_bf16(g[:, :, :S]).sum(0), rtol=0, atol=1e-12)
+    np.testing.assert_array_equal(acc16[0, :, :S], O.round_bf16(acc16[0, :, :S]))
+    # error bounds: each rounding is at most half a unit in the last place (2^-9 relative)
+    e1 = np.abs(wire - exact)[0, :, :S]
+    assert e1.max() <= 2.0 ** -9 * np.abs(g[:, :, :S]).sum(0).max() * 1.0001
+    e2 = np.abs(acc16 - exact)[0, :, :S]
+    assert e1.mean() < e2.mean()          # accumulating in 16 bit loses more than a 16-bit payload
+    # a value already on the grid, one rank: both models are exact
+    one = O.round_bf16(rng.standard_normal((1, 4, 8)))
+    np.testing.assert_array_equal(O.backward_partial_channel_reduce(one, 8, 1.0, reduce_mode=2), one)
+
+
 # ---------------------------------------------------------------- compact residual layout
 def _rand_compact(rng, t, T, h, K_r, S):
     return {"Y": rng.standard_normal((t, T, K_r)), "W": rng.standard_normal((t, h, K_r)) * 0.3,
