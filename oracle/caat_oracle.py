@@ -32,6 +32,9 @@ closed forms of Appendix C for the byte counts.  The compact-layout functions
 (shared part of the residual stream stored once) are pinned by their own finite
 differences, by equality with the per-rank forward on a tied residual, and by the
 rank-sum relation between a tied variable's gradient and its copies' gradients.
+The column-parallel half (colpar_*, mlp_*) is pinned by library silu / autograd, by
+finite differences, and by the textbook identity that with identical inputs on every
+rank the concatenated shards equal the unsharded layer (Section 3, Eq. 2-3).
 
 Parity unpinned (the paper fixes no value; these are this build's documented
 choices): eps, the norm kind per model, the default of alpha, the dtype of dW.
@@ -351,6 +354,81 @@ def block_backward_compact(dX1, dX2, dHn2s, dHn2p, Y_attn, W_o, Y_mlp, W_down, H
     return {"dY_attn": b1["dY"], "dW_o": b1["dW"], "dY_mlp": b2["dY"], "dW_down": b2["dW"],
             "dR0s": b1["dRs"], "dR0p": b1["dRp"], "dHn1s": b2["dRs"], "dHn1p": b2["dRp"],
             "dgamma1": b1["dgamma"], "dgamma2": b2["dgamma"], "dbeta1": b1["dbeta"], "dbeta2": b2["dbeta"]}
+
+
+# --------------------------------------------------------------------------
+# Column-parallel half in front of the row-parallel layer (Section 3, "Y_m = sigma(X_m A_m)";
+# Eq. A3, inner sum).  With partially synchronised activations every rank has its OWN input X_m
+# (the per-rank norm output), so the layer is a batch of t independent products.
+#   A[m]   rank m's weight shard stored out x in, [N, h]        [A~_{jkm} as A[m][k][j]]
+#   NONE     out = X_m A_m^T                       (QKV projection: N = 3 h / t)
+#   SILU     Y   = silu(X_m A_m^T)                 (an elementwise sigma, as Eq. A3 writes it)
+#   SWIGLU   Y   = silu(G) * U,  [G | U] = X_m A_m^T,  N = 2 F  (the gated MLP of the Llama models
+#            the paper trains; rows [0, F) of A_m are the gate, rows [F, 2F) the up projection)
+# --------------------------------------------------------------------------
+ACT_NONE = 0
+ACT_SILU = 1
+ACT_SWIGLU = 2
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    x = np.asarray(x, dtype=np.float64)
+    return x / (1.0 + np.exp(-x))
+
+
+def silu_grad(x: np.ndarray) -> np.ndarray:
+    """d silu / dx = s (1 + x (1 - s)), s = logistic(x)."""
+    x = np.asarray(x, dtype=np.float64)
+    sg = 1.0 / (1.0 + np.exp(-x))
+    return sg * (1.0 + x * (1.0 - sg))
+
+
+def colpar_forward(X, A, act: int = ACT_NONE) -> dict:
+    """pre[m] = X[m] A[m]^T; Y = act(pre).  Returns pre (saved for the backward) and Y."""
+    pre = rank_partials(X, A)                    # the same batched product as F1, other operands
+    if act == ACT_NONE:
+        return {"pre": pre, "Y": pre}
+    if act == ACT_SILU:
+        return {"pre": pre, "Y": silu(pre)}
+    if act == ACT_SWIGLU:
+        F = pre.shape[2] // 2
+        return {"pre": pre, "Y": silu(pre[:, :, :F]) * pre[:, :, F:]}
+    raise ValueError("unknown activation")
+
+
+def colpar_backward(dY, X, A, pre, act: int = ACT_NONE) -> dict:
+    """Gradient of colpar_forward contracted with dY: dpre (through the activation), then
+    dX[m] = dpre[m] A[m] and dA[m] = dpre[m]^T X[m], rank by rank (no cross-rank term:
+    each rank's X_m is its own variable)."""
+    dY = np.asarray(dY, dtype=np.float64)
+    pre = np.asarray(pre, dtype=np.float64)
+    if act == ACT_NONE:
+        dpre = dY
+    elif act == ACT_SILU:
+        dpre = dY * silu_grad(pre)
+    elif act == ACT_SWIGLU:
+        F = pre.shape[2] // 2
+        G, U = pre[:, :, :F], pre[:, :, F:]
+        dpre = np.concatenate([dY * U * silu_grad(G), dY * silu(G)], axis=2)
+    else:
+        raise ValueError("unknown activation")
+    return {"dpre": dpre, "dX": data_gradient(dpre, A), "dA": weight_gradient(dpre, X)}
+
+
+def mlp_forward(X, A, B, R, gamma, beta=None, *, act: int = ACT_SWIGLU, S: int, alpha: float = 1.0,
+                eps: float = 1e-5, norm: int = RMSNORM) -> dict:
+    """A whole tensor-parallel MLP with partial channel-reduce (Eq. A3): column-parallel half on the
+    per-rank inputs, then the row-parallel half with reduce, scaling, residual and norm."""
+    c = colpar_forward(X, A, act)
+    r = rowpar_forward(c["Y"], B, R, gamma, beta, S=S, alpha=alpha, eps=eps, norm=norm)
+    return {"pre": c["pre"], "Y": c["Y"], "Hn": r["Hn"], "X": r["X"], "rstd": r["rstd"], "mean": r["mean"]}
+
+
+def mlp_backward(dXout, dHn, X, A, B, pre, Y, Hn, rstd, mean, gamma, *, act: int = ACT_SWIGLU, S: int,
+                 alpha: float = 1.0, norm: int = RMSNORM) -> dict:
+    r = rowpar_backward(dXout, dHn, Y, B, Hn, rstd, mean, gamma, S=S, alpha=alpha, norm=norm)
+    c = colpar_backward(r["dY"], X, A, pre, act)
+    return {"dX": c["dX"], "dA": c["dA"], "dB": r["dW"], "dR": r["dR"], "dgamma": r["dgamma"], "dbeta": r["dbeta"]}
 
 
 # --------------------------------------------------------------------------

@@ -335,6 +335,90 @@ def test_block_chains_through_residual_and_matches_finite_differences():
         assert np.abs(num - b[gname]).max() / max(1.0, np.abs(num).max()) < 2e-7, name
 
 
+# ---------------------------------------------------------------- column-parallel half
+def test_silu_and_its_derivative_match_the_library():
+    x = np.linspace(-12, 12, 4001)
+    xt = torch.tensor(x, requires_grad=True)
+    y = F.silu(xt)
+    y.sum().backward()
+    np.testing.assert_allclose(O.silu(x), y.detach().numpy(), rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(O.silu_grad(x), xt.grad.numpy(), rtol=1e-12, atol=1e-14)
+
+
+@pytest.mark.parametrize("act", [O.ACT_NONE, O.ACT_SILU, O.ACT_SWIGLU])
+def test_colpar_shards_concatenate_to_the_unsharded_layer(act):
+    # Section 3 (standard tensor parallelism): with the SAME input on every rank, the column shards'
+    # outputs side by side are the unsharded sigma(X A)
+    rng = _rng(41)
+    t, T, h, N = 4, 7, 10, 6
+    Xs = rng.standard_normal((T, h))
+    A = rng.standard_normal((t, N, h)) * 0.5
+    out = O.colpar_forward(np.broadcast_to(Xs, (t, T, h)), A, act)["Y"]
+    if act == O.ACT_SWIGLU:
+        Fh = N // 2
+        gate = np.concatenate([A[m, :Fh] for m in range(t)], 0)       # [t Fh, h]
+        up = np.concatenate([A[m, Fh:] for m in range(t)], 0)
+        ref = F.silu(torch.tensor(Xs @ gate.T)).numpy() * (Xs @ up.T)
+    else:
+        full = np.concatenate([A[m] for m in range(t)], 0)
+        pre = Xs @ full.T
+        ref = pre if act == O.ACT_NONE else F.silu(torch.tensor(pre)).numpy()
+    np.testing.assert_allclose(np.concatenate([out[m] for m in range(t)], 1), ref, rtol=1e-12, atol=1e-12)
+
+
+@pytest.mark.parametrize("act", [O.ACT_NONE, O.ACT_SILU, O.ACT_SWIGLU])
+def test_colpar_backward_matches_autograd(act):
+    rng = _rng(42)
+    t, T, h, N = 3, 5, 8, 6
+    X, A = rng.standard_normal((t, T, h)), rng.standard_normal((t, N, h)) * 0.5
+    dY = rng.standard_normal((t, T, N // 2 if act == O.ACT_SWIGLU else N))
+    Xt, At = torch.tensor(X, requires_grad=True), torch.tensor(A, requires_grad=True)
+    pre = torch.einsum("mik,mlk->mil", Xt, At)
+    if act == O.ACT_NONE:
+        Y = pre
+    elif act == O.ACT_SILU:
+        Y = F.silu(pre)
+    else:
+        Y = F.silu(pre[:, :, :N // 2]) * pre[:, :, N // 2:]
+    (Y * torch.tensor(dY)).sum().backward()
+    f = O.colpar_forward(X, A, act)
+    np.testing.assert_allclose(f["Y"], Y.detach().numpy(), rtol=1e-12, atol=1e-13)
+    b = O.colpar_backward(dY, X, A, f["pre"], act)
+    np.testing.assert_allclose(b["dX"], Xt.grad.numpy(), rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(b["dA"], At.grad.numpy(), rtol=1e-11, atol=1e-12)
+
+
+def test_mlp_backward_matches_finite_differences():
+    rng = _rng(43)
+    t, T, h, Fh, S, alpha = 2, 2, 4, 3, 2, math.sqrt(2.0)
+    d = {"X": rng.standard_normal((t, T, h)), "A": rng.standard_normal((t, 2 * Fh, h)) * 0.5,
+         "B": rng.standard_normal((t, h, Fh)) * 0.5, "R": rng.standard_normal((t, T, h)),
+         "gamma": 1 + 0.1 * rng.standard_normal(h)}
+    Gx, Gh = rng.standard_normal((t, T, h)), rng.standard_normal((t, T, h))
+
+    def fwd():
+        return O.mlp_forward(d["X"], d["A"], d["B"], d["R"], d["gamma"], S=S, alpha=alpha)
+
+    def loss():
+        o = fwd()
+        return float(np.sum(Gx * o["X"]) + np.sum(Gh * o["Hn"]))
+
+    o = fwd()
+    b = O.mlp_backward(Gx, Gh, d["X"], d["A"], d["B"], o["pre"], o["Y"], o["Hn"], o["rstd"], None, d["gamma"], S=S, alpha=alpha)
+    step = 1e-6
+    for name, gname in (("X", "dX"), ("A", "dA"), ("B", "dB"), ("R", "dR"), ("gamma", "dgamma")):
+        num = np.zeros_like(d[name])
+        it = np.nditer(d[name], flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = d[name][idx]
+            d[name][idx] = keep + step; lp = loss()
+            d[name][idx] = keep - step; lm = loss()
+            d[name][idx] = keep
+            num[idx] = (lp - lm) / (2 * step)
+        assert np.abs(num - b[gname]).max() / max(1.0, np.abs(num).max()) < 2e-7, name
+
+
 # ---------------------------------------------------------------- precision models of the backward reduce
 def test_round_bf16_matches_library_cast():
     rng = _rng(31)
