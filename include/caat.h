@@ -291,6 +291,36 @@ caat_status caat_block_backward_compact(const caat_ctx *ctx, int tokens,
                                         void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Column-parallel half in front of a row-parallel layer (Section 3: Y_m = sigma(X_m A_m); the
+ * inner sum of Eq. A3; the QKV projection in front of attention, Eq. A5).  With partially
+ * synchronised activations every rank has its OWN input X_m (the per-rank norm output X of the
+ * previous layer), so the layer is t independent products, no reduce:
+ *   pre[m,i,n] = sum_j X[m,i,j] * A[m,n,j]                         n < n_out
+ *   CAAT_ACT_NONE    Y = pre                        (QKV projection: n_out = 3 h / t)
+ *   CAAT_ACT_SILU    Y[m,i,n] = silu(pre[m,i,n])    (an elementwise sigma)
+ *   CAAT_ACT_SWIGLU  Y[m,i,n] = silu(pre[m,i,n]) * pre[m,i,F+n],  n < F = n_out / 2
+ *                    (gated MLP of the Llama models: rows [0,F) of A_m are the gate, rows
+ *                    [F,2F) the up projection; Y is the row-parallel layer's input, F = ffn/t)
+ *
+ *   X   [t, T, h]      dtype in      A  [t, n_out, h] dtype in (out x in per rank)
+ *   pre [t, T, n_out]  dtype out (kept for the backward)
+ *   Y   [t, T, n_out or n_out/2] dtype out; NULL for CAAT_ACT_NONE (pre is the result)
+ * Backward, given dY (the gradient on Y; on pre for CAAT_ACT_NONE):
+ *   dpre = dY through the activation,  dX[m] = dpre[m] A[m],  dA[m] = dpre[m]^T X[m]
+ *   dX [t, T, h] dtype out (the upstream gradient dX of the previous row-parallel layer's norm)
+ *   dA [t, n_out, h] FP32 out
+ * n_out must be a multiple of 8 (16 for CAAT_ACT_SWIGLU).  The forward needs no workspace.
+ */
+typedef enum { CAAT_ACT_NONE = 0, CAAT_ACT_SILU = 1, CAAT_ACT_SWIGLU = 2 } caat_activation;
+size_t caat_colpar_workspace_bytes(const caat_ctx *ctx, caat_activation act, int n_out, int tokens);
+caat_status caat_colpar_forward(const caat_ctx *ctx, caat_activation act, int n_out, int tokens,
+                                const void *X, const void *A, void *pre, void *Y, void *cuda_stream);
+caat_status caat_colpar_backward(const caat_ctx *ctx, caat_activation act, int n_out, int tokens,
+                                 const void *dY, const void *X, const void *A, const void *pre,
+                                 void *dX, float *dA,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Analytic bytes ONE partial channel-reduce would move on a real t-device system
  * (Appendix C: each device sends and receives tokens*h*p activations per reduce;
  * Appendix D: all-reduce = reduce-scatter + all-gather, traffic cut by 100(1-p) %).
@@ -330,7 +360,8 @@ typedef enum {
   CAAT_K_TC_DGRAD = 5,       /* tcgen05 GEMM, data gradient                         */
   CAAT_K_TC_WGRAD = 6,       /* tcgen05 GEMM, weight gradient                       */
   CAAT_K_SPLITK_REDUCE = 7,  /* split-K reduction of the weight gradient            */
-  CAAT_K_COUNT = 8
+  CAAT_K_ACTIVATION = 8,     /* activation of the column-parallel half / its derivative */
+  CAAT_K_COUNT = 9
 } caat_kernel_kind;
 caat_status caat_profile_begin(int max_launches);
 caat_status caat_profile_end(int n_kinds, double *ms_by_kind, unsigned long long *launches_by_kind);

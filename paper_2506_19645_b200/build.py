@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcaat.so")
-SOURCES = ["caat_api.cu", "caat_rows.cu", "caat_rows_staged.cu", "caat_rows_warp.cu", "caat_gemm_simt.cu", "caat_gemm_tc.cu", "caat_static.cu"]
+SOURCES = ["caat_api.cu", "caat_rows.cu", "caat_rows_staged.cu", "caat_rows_warp.cu", "caat_gemm_simt.cu", "caat_gemm_tc.cu", "caat_static.cu", "caat_colpar.cu"]
 
 
 def _newest_source_mtime() -> float:

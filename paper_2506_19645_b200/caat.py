@@ -24,6 +24,7 @@ CAAT_NOALLOC_SCRATCH_BYTES = 32 * 1024 * 1024
 (CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM, CAAT_OPT_ROWS,
  CAAT_OPT_DECODE, CAAT_OPT_BACKWARD_REDUCE) = range(8)
 RMSNORM, LAYERNORM = 0, 1
+CAAT_ACT_NONE, CAAT_ACT_SILU, CAAT_ACT_SWIGLU = 0, 1, 2
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2506_19645_b200.build` "
@@ -49,6 +50,9 @@ _sigs = {
     "caat_rowpar_backward_compact": (c_int, [_P, c_int, c_int] + [_P] * 16 + [_P, c_size_t, _P]),
     "caat_block_forward_compact": (c_int, [_P, c_int] + [_P] * 20 + [_P, c_size_t, _P]),
     "caat_block_backward_compact": (c_int, [_P, c_int] + [_P] * 30 + [_P, c_size_t, _P]),
+    "caat_colpar_workspace_bytes": (c_size_t, [_P, c_int, c_int, c_int]),
+    "caat_colpar_forward": (c_int, [_P, c_int, c_int, c_int] + [_P] * 4 + [_P]),
+    "caat_colpar_backward": (c_int, [_P, c_int, c_int, c_int] + [_P] * 6 + [_P, c_size_t, _P]),
     "caat_allreduce_bytes": (c_int, [_P, c_int, c_int] + [POINTER(c_ulonglong)] * 3),
     "caat_last_device_status": (c_int, [_P, _P]),
     "caat_kernel_launches": (c_ulonglong, []),
@@ -316,6 +320,31 @@ class Context:
             _stream())
         _check(st, "caat_block_backward_compact")
 
+    # ---- column-parallel half: pre = X A^T per rank, Y = act(pre)
+    def colpar_workspace_bytes(self, act: int, n_out: int, tokens: int) -> int:
+        return int(lib.caat_colpar_workspace_bytes(self._h, act, n_out, tokens))
+
+    def colpar_forward(self, act, n_out, tokens, X, A, pre, Y):
+        td, t, h = self.torch_dtype, self.t, self.h
+        wy = n_out // 2 if act == CAAT_ACT_SWIGLU else n_out
+        st = lib.caat_colpar_forward(
+            self._h, act, n_out, tokens,
+            _ptr(X, td, (t, tokens, h), "X"), _ptr(A, td, (t, n_out, h), "A"), _ptr(pre, td, (t, tokens, n_out), "pre"),
+            _ptr(Y, td, (t, tokens, wy), "Y"), _stream())
+        _check(st, "caat_colpar_forward")
+
+    def colpar_backward(self, act, n_out, tokens, dY, X, A, pre, dX, dA, workspace):
+        td, t, h = self.torch_dtype, self.t, self.h
+        wy = n_out // 2 if act == CAAT_ACT_SWIGLU else n_out
+        st = lib.caat_colpar_backward(
+            self._h, act, n_out, tokens,
+            _ptr(dY, td, (t, tokens, wy), "dY"), _ptr(X, td, (t, tokens, h), "X"), _ptr(A, td, (t, n_out, h), "A"),
+            _ptr(pre, td, (t, tokens, n_out), "pre"), _ptr(dX, td, (t, tokens, h), "dX"),
+            _ptr(dA, torch.float32, (t, n_out, h), "dA"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
+            _stream())
+        _check(st, "caat_colpar_backward")
+
     # ---- buffer helpers (torch.empty only; no arithmetic)
     def alloc_workspace(self, nbytes: int, device="cuda"):
         return torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
@@ -341,7 +370,7 @@ def kernel_launches() -> int:
     return int(lib.caat_kernel_launches())
 
 
-CAAT_K_COUNT = 8
+CAAT_K_COUNT = 9
 
 
 def profile_begin(max_launches: int = 65536):

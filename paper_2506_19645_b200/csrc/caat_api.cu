@@ -498,6 +498,129 @@ caat_status caat_block_backward_compact(const caat_ctx* ctx, int tokens, const v
                                       workspace_bytes, cuda_stream);
 }
 
+// ---- column-parallel half ------------------------------------------------------
+namespace {
+struct ColScratch { size_t dpre_off, splitk_off, splitk_bytes, wt_off, total; };
+
+bool col_tc_usable(const caat_ctx* ctx, int n_out) {
+  return ctx->dtype == CAAT_BF16 && !ctx->force_simt && ctx->h % 8 == 0 && n_out % 8 == 0;
+}
+
+RowparShapes col_shapes(const caat_ctx* ctx, int n_out, int T) {
+  // the row-parallel GEMM wiring with no shared columns: "h" is the output width, "K_r" the input width
+  return RowparShapes{ctx->t, T, n_out, ctx->h, 0, 0, 0, n_out};
+}
+
+ColScratch col_scratch(const caat_ctx* ctx, caat_activation act, int n_out, int T) {
+  ColScratch s{};
+  const size_t e = elem_size(ctx->dtype);
+  size_t off = 0;
+  s.dpre_off = off;
+  if (act != CAAT_ACT_NONE) off = align_up(off + (size_t)ctx->t * T * n_out * e, 256);
+  s.splitk_off = off;
+  if (col_tc_usable(ctx, n_out)) {
+    s.splitk_bytes = tc_wgrad_splitk_bytes(col_shapes(ctx, n_out, T));
+    off = align_up(off + s.splitk_bytes, 256);
+    s.wt_off = off;
+    if (tc_dgrad_wants_wt(T)) off = align_up(off + (size_t)ctx->t * ctx->h * n_out * e, 256);
+  }
+  s.total = off > 16 ? off : 16;
+  return s;
+}
+
+caat_status check_col(const caat_ctx* ctx, caat_activation act, int n_out, int tokens) {
+  if (!ctx) return CAAT_EINVAL;
+  if (act != CAAT_ACT_NONE && act != CAAT_ACT_SILU && act != CAAT_ACT_SWIGLU) return CAAT_EINVAL;
+  if (tokens < 1 || n_out < 1) return CAAT_ESHAPE;
+  if (ctx->h % 8 != 0 || n_out % (act == CAAT_ACT_SWIGLU ? 16 : 8) != 0) return CAAT_EUNSUPPORTED;
+  if ((long long)ctx->t * tokens > 2000000000LL) return CAAT_EUNSUPPORTED;
+  return CAAT_OK;
+}
+}  // namespace
+
+size_t caat_colpar_workspace_bytes(const caat_ctx* ctx, caat_activation act, int n_out, int tokens) {
+  if (check_col(ctx, act, n_out, tokens) != CAAT_OK) return 0;
+  return col_scratch(ctx, act, n_out, tokens).total;
+}
+
+caat_status caat_colpar_forward(const caat_ctx* ctx, caat_activation act, int n_out, int tokens, const void* X,
+                                const void* A, void* pre, void* Y, void* cuda_stream) {
+  caat_status s = check_col(ctx, act, n_out, tokens);
+  if (s != CAAT_OK) return s;
+  if (!X || !A || !pre || (act != CAAT_ACT_NONE && !Y)) return CAAT_EINVAL;
+  const void* ptrs[] = {X, A, pre, Y};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int t = ctx->t, T = tokens, h = ctx->h;
+  cudaError_t ce;
+  if (col_tc_usable(ctx, n_out)) {
+    ce = launch_tc_forward(col_shapes(ctx, n_out, T), X, A, nullptr, pre, st);
+  } else {
+    GemmProblem g{};
+    g.nseg = 1;
+    g.seg[0] = GemmSeg{X, A, (long long)T * h, 0, h, 1, (long long)n_out * h, 0, 1, h, 1, h};
+    g.C = pre; g.sCb = (long long)T * n_out; g.sCi = n_out; g.M = T; g.N = n_out; g.batch = t; g.c_f32 = 0;
+    ce = launch_gemm_simt(g, ctx->dtype, st);
+  }
+  if (ce != cudaSuccess) return cuda_fail(ce);
+  if (act != CAAT_ACT_NONE) {
+    const int gated = act == CAAT_ACT_SWIGLU;
+    ce = launch_act_forward(ctx->dtype, gated, pre, Y, (long long)t * T, gated ? n_out / 2 : n_out, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+  }
+  return CAAT_OK;
+}
+
+caat_status caat_colpar_backward(const caat_ctx* ctx, caat_activation act, int n_out, int tokens, const void* dY,
+                                 const void* X, const void* A, const void* pre, void* dX, float* dA, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = check_col(ctx, act, n_out, tokens);
+  if (s != CAAT_OK) return s;
+  if (!dY || !X || !A || !dX || !dA || (act != CAAT_ACT_NONE && !pre)) return CAAT_EINVAL;
+  const void* ptrs[] = {dY, X, A, pre, dX, dA, workspace};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  const ColScratch L = col_scratch(ctx, act, n_out, tokens);
+  if (!workspace || workspace_bytes < L.total) return CAAT_EWORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* wsb = static_cast<char*>(workspace);
+  const int t = ctx->t, T = tokens, h = ctx->h;
+  cudaError_t ce;
+  const void* dpre = dY;
+  if (act != CAAT_ACT_NONE) {
+    const int gated = act == CAAT_ACT_SWIGLU;
+    ce = launch_act_backward(ctx->dtype, gated, dY, pre, wsb + L.dpre_off, (long long)t * T, gated ? n_out / 2 : n_out, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    dpre = wsb + L.dpre_off;
+  }
+  if (col_tc_usable(ctx, n_out)) {
+    const RowparShapes sh = col_shapes(ctx, n_out, T);
+    ce = launch_tc_dgrad(sh, nullptr, dpre, A, dX, tc_dgrad_wants_wt(T) ? wsb + L.wt_off : nullptr, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    ce = launch_tc_wgrad(sh, nullptr, dpre, X, dA, wsb + L.splitk_off, L.splitk_bytes, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+    return CAAT_OK;
+  }
+  {  // dX[m] = dpre[m] A[m]
+    GemmProblem g{};
+    g.nseg = 1;
+    g.seg[0] = GemmSeg{dpre, A, (long long)T * n_out, 0, n_out, 1, (long long)n_out * h, 0, h, 1, 1, n_out};
+    g.C = dX; g.sCb = (long long)T * h; g.sCi = h; g.M = T; g.N = h; g.batch = t; g.c_f32 = 0;
+    ce = launch_gemm_simt(g, ctx->dtype, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+  }
+  {  // dA[m] = dpre[m]^T X[m]
+    GemmProblem g{};
+    g.nseg = 1;
+    g.seg[0] = GemmSeg{dpre, X, (long long)T * n_out, 0, 1, n_out, (long long)T * h, 0, h, 1, 1, T};
+    g.C = dA; g.sCb = (long long)n_out * h; g.sCi = h; g.M = n_out; g.N = h; g.batch = t; g.c_f32 = 1;
+    ce = launch_gemm_simt(g, ctx->dtype, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+  }
+  return CAAT_OK;
+}
+
 caat_status caat_allreduce_bytes(const caat_ctx* ctx, int tokens, int elem_bytes, unsigned long long* payload,
                                  unsigned long long* payload_p1, unsigned long long* ring_wire) {
   if (!ctx || elem_bytes < 1) return CAAT_EINVAL;
@@ -569,6 +692,7 @@ const char* caat_kernel_kind_name(int kind) {
     case CAAT_K_TC_DGRAD: return "tc_gemm_dgrad";
     case CAAT_K_TC_WGRAD: return "tc_gemm_wgrad";
     case CAAT_K_SPLITK_REDUCE: return "splitk_reduce";
+    case CAAT_K_ACTIVATION: return "activation";
   }
   return "";
 }

@@ -155,6 +155,13 @@ cudaError_t launch_rows_backward_warp(const RowBwdArgs& a, caat_dtype dtype, int
                                       cudaStream_t st);
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype);
 
+// ---- activation of the column-parallel half (streaming kernels) ---------------
+// gated: pre has 2 * width_out columns [gate | up], Y = silu(gate) * up; else Y = silu(pre)
+cudaError_t launch_act_forward(caat_dtype dtype, int gated, const void* pre, void* Y, long long rows, int width_out,
+                               cudaStream_t st);
+cudaError_t launch_act_backward(caat_dtype dtype, int gated, const void* dY, const void* pre, void* dpre,
+                                long long rows, int width_out, cudaStream_t st);
+
 // ---- bookkeeping ------------------------------------------------------------
 // Brackets one kernel launch: counts it and, while profiling is on, records a CUDA event
 // before and after it on the launching stream.
