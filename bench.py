@@ -33,7 +33,12 @@ from paper_2506_19645_b200 import replicas, synthetic  # noqa: E402
 
 DEFAULT_WORKLOAD = "block_130m"
 METRIC = "CAAT block tokens/s (sim. TP=t, sync p) on 1 B200"
-SWEEP = ["block_1p1b_p100", "block_1p1b_p075", "block_1p1b_p050", "block_1p1b_p025", "block_7b"]
+
+
+def metric_name(w):
+    return METRIC.replace("block", "MLP (column- + row-parallel half)") if w.kind == "mlp" else METRIC
+SWEEP = ["block_1p1b_p100", "block_1p1b_p075", "block_1p1b_p050", "block_1p1b_p025", "block_7b",
+         "mlp_130m", "mlp_1p1b_p050", "mlp_7b"]
 
 
 # --------------------------------------------------------------------------- peaks
@@ -128,10 +133,26 @@ def layer_work(w, k_r, backward, compact=False):
     return out
 
 
+def colpar_work(w):
+    """Algorithmic work of the column-parallel MLP half (gate|up GEMM per rank + SwiGLU), e = 2 bytes."""
+    t, T, h, F, e = w.t, w.tokens, w.h, w.kr_mlp, 2
+    fl = 2.0 * t * T * h * 2 * F
+    out = {"tc_gemm_forward": {"flops": fl, "bytes": (t * T * h + t * 2 * F * h + t * T * 2 * F) * e},
+           "activation": {"flops": 0.0, "bytes": t * T * 3 * F * e}}
+    if w.backward:
+        out["activation"]["bytes"] += t * T * 5 * F * e
+        out["tc_gemm_dgrad"] = {"flops": fl, "bytes": (t * T * 2 * F + t * 2 * F * h + t * T * h) * e}
+        out["tc_gemm_wgrad"] = {"flops": fl, "bytes": (t * T * 2 * F + t * T * h) * e + t * 2 * F * h * 4}
+    return out
+
+
 def step_work(w, compact=False):
     tot = {}
-    for k_r in (w.kr_attn, w.kr_mlp):
-        for kind, v in layer_work(w, k_r, w.backward, compact).items():
+    parts = [layer_work(w, k_r, w.backward, compact) for k_r in ((w.kr_mlp,) if w.kind == "mlp" else (w.kr_attn, w.kr_mlp))]
+    if w.kind == "mlp":
+        parts.append(colpar_work(w))
+    for part in parts:
+        for kind, v in part.items():
             a = tot.setdefault(kind, {"flops": 0.0, "bytes": 0.0})
             a["flops"] += v["flops"]
             a["bytes"] += v["bytes"]
@@ -144,7 +165,11 @@ def paper_level_work(w, compact=False):
     full = t * T * h
     stream = T * w.S + t * T * (h - w.S) if compact else full
     fl = by = 0.0
-    for k_r in (w.kr_attn, w.kr_mlp):
+    if w.kind == "mlp":   # column-parallel half: X, A in; pre kept for the backward; dX, dA out
+        F = w.kr_mlp
+        fl += 2.0 * t * T * h * 2 * F * (3 if w.backward else 1)
+        by += e * (full + t * 2 * F * h + t * T * 2 * F) + (e * (t * T * 2 * F + full) + 4 * t * 2 * F * h if w.backward else 0)
+    for k_r in ((w.kr_mlp,) if w.kind == "mlp" else (w.kr_attn, w.kr_mlp)):
         K = k_r * t
         fl += 2.0 * T * K * h
         by += e * (T * K + K * h + 2 * stream + full)
@@ -223,6 +248,46 @@ class BlockRunner:
         return n + sum(v.numel() * v.element_size() for v in self.out.values())
 
 
+class MlpRunner:
+    """The whole tensor-parallel MLP: column-parallel gate|up + SwiGLU, then the MLP-down layer with partial
+    channel-reduce (and the gradient of both), as two library calls per direction."""
+
+    def __init__(self, w, device, compact=False):
+        from paper_2506_19645_b200 import caat
+        assert not compact
+        self.caat, self.w, self.dev, self.compact = caat, w, device, False
+        self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
+        self.inp = synthetic.mlp_inputs(w, device=device)
+        t, T, h, F = w.t, w.tokens, w.h, w.kr_mlp
+        td, f32 = self.ctx.torch_dtype, torch.float32
+        mk = lambda *s, dt=td: torch.empty(*s, dtype=dt, device=device)
+        self.out = {"pre": mk(t, T, 2 * F), "Y": mk(t, T, F), "Hn": mk(t, T, h), "Xout": mk(t, T, h), "rstd": mk(t, T, dt=f32)}
+        if w.backward:
+            self.out.update({"dY": mk(t, T, F), "dB": mk(t, h, F, dt=f32), "dR": mk(t, T, h), "dgamma": mk(h, dt=f32),
+                             "dX": mk(t, T, h), "dA": mk(t, 2 * F, h, dt=f32)})
+        nbytes = max(self.ctx.workspace_bytes(caat.CAAT_MLP_DOWN, T, w.backward),
+                     self.ctx.colpar_workspace_bytes(caat.CAAT_ACT_SWIGLU, 2 * F, T))
+        self.ws = self.ctx.alloc_workspace(nbytes, device=device)
+
+    def step(self):
+        c, i, o, T, F = self.caat, self.inp, self.out, self.w.tokens, self.w.kr_mlp
+        self.ctx.colpar_forward(c.CAAT_ACT_SWIGLU, 2 * F, T, i["X"], i["A"], o["pre"], o["Y"])
+        self.ctx.rowpar_forward(c.CAAT_MLP_DOWN, T, o["Y"], i["B"], i["R"], i["gamma"], None, o["Hn"], o["Xout"], o["rstd"],
+                                None, self.ws)
+        if self.w.backward:
+            self.ctx.rowpar_backward(c.CAAT_MLP_DOWN, T, i["dXout"], i["dHn"], o["Y"], i["B"], o["Hn"], o["rstd"], None,
+                                     i["gamma"], o["dY"], o["dB"], o["dR"], o["dgamma"], None, self.ws)
+            self.ctx.colpar_backward(c.CAAT_ACT_SWIGLU, 2 * F, T, o["dY"], i["X"], i["A"], o["pre"], o["dX"], o["dA"], self.ws)
+
+    def touched_bytes(self):
+        n = sum(v.numel() * v.element_size() for v in self.inp.values())
+        return n + sum(v.numel() * v.element_size() for v in self.out.values())
+
+
+def make_runner(w, device, compact=False):
+    return MlpRunner(w, device, compact) if w.kind == "mlp" else BlockRunner(w, device, compact)
+
+
 def capture_step(runner):
     """One step captured into a CUDA graph (launch-bound workloads: a decode step is tens of
     microseconds).  Returns (graph, kernels per step) or (None, 0) when capture is not possible."""
@@ -271,7 +336,7 @@ def e2e_leg(runner, steps):
     host memory and reads its results back to the host, all inside the timed region.  The three
     phases run on three streams over two sets of device buffers, so the copy of step s+1, the
     kernels of step s and the read-back of step s-1 overlap (PCIe moves both ways at once)."""
-    runners = [runner, BlockRunner(runner.w, runner.dev, runner.compact)]
+    runners = [runner, make_runner(runner.w, runner.dev, runner.compact)]
     inp_host = {k: v.cpu().pin_memory() for k, v in runner.inp.items()}
     out_host = [{k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in runner.out.items()} for _ in range(2)]
     h2d = sum(v.numel() * v.element_size() for v in inp_host.values())
@@ -322,8 +387,16 @@ def oracle_sample_run(w, sample_tokens):
     """One block forward(+backward) of the fp64 oracle on `sample_tokens` tokens of the workload."""
     from oracle import caat_oracle as O
     ws = w.with_tokens(sample_tokens)
-    d = {k: v.to(torch.float64).numpy() for k, v in synthetic.block_inputs(ws, device="cpu").items()}
     S, alpha = ws.S, math.sqrt(ws.t)
+    if w.kind == "mlp":
+        d = {k: v.to(torch.float64).numpy() for k, v in synthetic.mlp_inputs(ws, device="cpu").items()}
+        t0 = time.perf_counter()
+        f = O.mlp_forward(d["X"], d["A"], d["B"], d["R"], d["gamma"], S=S, alpha=alpha)
+        if w.backward:
+            O.mlp_backward(d["dXout"], d["dHn"], d["X"], d["A"], d["B"], f["pre"], f["Y"], f["Hn"], f["rstd"], None,
+                           d["gamma"], S=S, alpha=alpha)
+        return time.perf_counter() - t0
+    d = {k: v.to(torch.float64).numpy() for k, v in synthetic.block_inputs(ws, device="cpu").items()}
     t0 = time.perf_counter()
     f = O.block_forward(d["Y_attn"], d["W_o"], d["Y_mlp"], d["W_down"], d["R0"], d["gamma1"], d["gamma2"], S=S, alpha=alpha)
     if w.backward:
@@ -367,7 +440,7 @@ def run_cuda(args):
     if args.tokens > 0:
         w = w.with_tokens(args.tokens)
     compact = args.layout == "compact"
-    runner = BlockRunner(w, dev, compact)
+    runner = make_runner(w, dev, compact)
     warm = max(args.warmup, 3)
     for _ in range(warm):
         runner.step()
@@ -434,7 +507,7 @@ def run_cuda(args):
             e2e = {"value": None, "unit": "tokens/s", "error": str(ex)[:200]}
         ar = runner.ctx.allreduce_bytes(w.tokens, 2)
         result = {
-            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
+            "metric": metric_name(w), "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p,
@@ -457,7 +530,7 @@ def run_cuda(args):
             if name == w.name:
                 continue
             try:
-                r = BlockRunner(synthetic.WORKLOADS[name], dev)
+                r = make_runner(synthetic.WORKLOADS[name], dev)
                 for _ in range(3):
                     r.step()
                 k = max(3, min(args.steps, 10))
@@ -470,7 +543,7 @@ def run_cuda(args):
                               "allreduce_payload_bytes": r.ctx.allreduce_bytes(r.w.tokens, 2)["payload_per_rank"]})
                 del r
                 torch.cuda.empty_cache()
-                if r_w_compact_ok(synthetic.WORKLOADS[name]):
+                if r_w_compact_ok(synthetic.WORKLOADS[name]) and synthetic.WORKLOADS[name].kind == "block":
                     # the same block on the compact residual layout (shared channels of the stream stored once)
                     r = BlockRunner(synthetic.WORKLOADS[name], dev, True)
                     for _ in range(3):
@@ -514,7 +587,7 @@ def run_reference(args):
     sample = (f"fp64 numpy oracle, block forward{'+backward' if w.backward else ''}, each step a sample of {n} of "
               f"{w.tokens} tokens of {w.name}; host has {len(os.sched_getaffinity(0))} usable cores")
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s",
+        "impl": "reference", "metric": metric_name(w), "value": value, "unit": "tokens/s",
         "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",

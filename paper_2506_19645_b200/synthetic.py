@@ -30,7 +30,8 @@ class Workload:
     ffn: int        # MLP inner width (total, over all ranks)
     p: float        # synchronisation factor
     dtype: str      # "f32" | "bf16"  (storage type; accumulation is fp32)
-    kind: str       # "layer" (one MLP-down-like layer) | "block" (attention-out + MLP-down)
+    kind: str       # "layer" (one MLP-down-like layer) | "block" (attention-out + MLP-down) |
+                    # "mlp" (column-parallel gate/up + SwiGLU, then the MLP-down layer)
     backward: bool
     seed: int = 0
 
@@ -66,6 +67,11 @@ WORKLOADS = {
     ] + [
         _w(f"decode_7b_T{T}_p{int(p * 100):03d}", 8, T, 4096, 11008, p, "bf16", "block", False)
         for T in (1, 8, 64) for p in (1.0, 0.5)
+    ] + [
+        # the whole tensor-parallel MLP of the same models: column-parallel half + row-parallel half
+        _w("mlp_130m", 4, 8 * 2048, 768, 3072, 0.5, "bf16", "mlp", True),
+        _w("mlp_1p1b_p050", 8, 8 * 2048, 2048, 5632, 0.5, "bf16", "mlp", True),
+        _w("mlp_7b", 8, 4 * 4096, 4096, 11008, 0.5, "bf16", "mlp", True),
     ]
 }
 
@@ -107,6 +113,28 @@ def layer_inputs(t, tokens, h, k_r, dtype="bf16", seed=0, S=0, backward=False,
     if backward:
         out["dX"] = _randn(gen, (t, tokens, h), 1.0, td, device)
         out["dHn"] = _randn(gen, (t, tokens, h), 1.0, td, device)
+    return out
+
+
+def mlp_inputs(w: Workload, tied_residual=True, device="cpu", weight_std=0.02) -> dict:
+    """Inputs of a whole MLP: per-rank normalised input X [t,T,h], gate|up weights A [t, 2 ffn/t, h],
+    down weights B [t, h, ffn/t], residual R, gain, and the upstream gradients of the backward."""
+    td = torch_dtype(w.dtype)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(w.seed)
+    t, T, h, F = w.t, w.tokens, w.h, w.kr_mlp
+    out = {
+        "X": _randn(gen, (t, T, h), 1.0, td, device),
+        "A": _randn(gen, (t, 2 * F, h), weight_std, td, device),
+        "B": _randn(gen, (t, h, F), weight_std, td, device),
+        "R": _randn(gen, (t, T, h), 1.0, td, device),
+        "gamma": torch.ones(h, dtype=td, device=device),
+    }
+    if tied_residual:
+        tie_shared_channels(out["R"], w.S)
+    if w.backward:
+        out["dXout"] = _randn(gen, (t, T, h), 1.0, td, device)
+        out["dHn"] = _randn(gen, (t, T, h), 1.0, td, device)
     return out
 
 
