@@ -139,3 +139,88 @@ def test_full_size_block_1p1b_p075_forward_sample():
 
 def test_full_size_block_7b():
     _check_block_full("block_7b", n_tok=32, n_dw=384)
+
+
+def _check_mlp_full(name, n_tok=32, n_dw=384, seed=321):
+    """Whole MLP (column-parallel gate|up + SwiGLU, then MLP-down with partial channel-reduce) at the bench's
+    size and launch sequence; the oracle walks the tokens in chunks and accumulates the token sums."""
+    w = synthetic.WORKLOADS[name]
+    t, T, h, S, F = w.t, w.tokens, w.h, w.S, w.kr_mlp
+    alpha = math.sqrt(t)
+    dev = synthetic.mlp_inputs(w, device="cuda")
+    host = {k: v.cpu() for k, v in dev.items()}
+    rng = np.random.default_rng(seed)
+    tok = np.sort(rng.choice(T, size=min(n_tok, T), replace=False))
+    iA = (rng.integers(0, t, n_dw), rng.integers(0, 2 * F, n_dw), rng.integers(0, h, n_dw))
+    iB = (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, F, n_dw))
+    A, B, g = f64(host["A"]), f64(host["B"]), f64(host["gamma"])
+    bf, f32 = torch.bfloat16, torch.float32
+
+    spre = torch.empty((t, T, 2 * F), dtype=bf); sY = torch.empty((t, T, F), dtype=bf)
+    sHn = torch.empty((t, T, h), dtype=bf); sr = torch.empty((t, T), dtype=f32)
+    fwd_s = {k: [] for k in ("pre", "Y", "Hn", "X", "rstd")}
+    for a, b in _chunks(T):
+        sl = slice(a, b)
+        o = O.mlp_forward(f64(host["X"][:, sl]), A, B, f64(host["R"][:, sl]), g, S=S, alpha=alpha)
+        spre[:, sl] = torch.from_numpy(o["pre"]).to(bf); sY[:, sl] = torch.from_numpy(o["Y"]).to(bf)
+        sHn[:, sl] = torch.from_numpy(o["Hn"]).to(bf); sr[:, sl] = torch.from_numpy(o["rstd"]).float()
+        loc = tok[(tok >= a) & (tok < b)] - a
+        for k in fwd_s:
+            fwd_s[k].append(o[k][:, loc])
+    fwd_s = {k: np.concatenate(v, axis=1) for k, v in fwd_s.items()}
+
+    ctx = caat.Context(w.h, w.ffn, t, w.p, "bf16")
+    mk = lambda *s, dt=bf: torch.empty(*s, dtype=dt, device="cuda")
+    out = {"pre": mk(t, T, 2 * F), "Y": mk(t, T, F), "Hn": mk(t, T, h), "X": mk(t, T, h), "rstd": mk(t, T, dt=f32)}
+    ws = ctx.alloc_workspace(max(ctx.workspace_bytes(caat.CAAT_MLP_DOWN, T, True),
+                                 ctx.colpar_workspace_bytes(caat.CAAT_ACT_SWIGLU, 2 * F, T)))
+    ctx.colpar_forward(caat.CAAT_ACT_SWIGLU, 2 * F, T, dev["X"], dev["A"], out["pre"], out["Y"])
+    ctx.rowpar_forward(caat.CAAT_MLP_DOWN, T, out["Y"], dev["B"], dev["R"], dev["gamma"], None, out["Hn"], out["X"],
+                       out["rstd"], None, ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+    tk = torch.from_numpy(tok).cuda()
+    for k in fwd_s:
+        assert_close(out[k].index_select(1, tk), fwd_s[k], "bf16", f"{name}:{k}")
+    del out
+
+    bo = {"dY": mk(t, T, F), "dB": mk(t, h, F, dt=f32), "dR": mk(t, T, h), "dgamma": mk(h, dt=f32), "dX": mk(t, T, h),
+          "dA": mk(t, 2 * F, h, dt=f32)}
+    dY_saved = torch.empty((t, T, F), dtype=bf)
+    acc = {"dgamma": np.zeros(h), "dA": np.zeros(n_dw), "dB": np.zeros(n_dw)}
+    bwd_s = {k: [] for k in ("dX", "dR", "dY")}
+    for a, b in _chunks(T):
+        sl = slice(a, b)
+        loc = tok[(tok >= a) & (tok < b)] - a
+        Hn, r = f64(sHn[:, sl]), f64(sr[:, sl])
+        gm = O.residual_stream_gradient(f64(host["dXout"][:, sl]), f64(host["dHn"][:, sl]), Hn, r, None, g, O.RMSNORM)
+        acc["dgamma"] += O.norm_param_gradients(f64(host["dXout"][:, sl]), Hn, r, None, O.RMSNORM)[0]
+        dZ = O.backward_partial_channel_reduce(gm, S, alpha)
+        Y = f64(sY[:, sl])
+        dY = O.data_gradient(dZ, B)
+        dY_saved[:, sl] = torch.from_numpy(dY).to(bf)
+        m_, l_, k_ = iB
+        acc["dB"] += np.einsum("ni,ni->n", dZ[m_, :, l_], Y[m_, :, k_])
+        cb = O.colpar_backward(f64(dY_saved[:, sl]), f64(host["X"][:, sl]), A, f64(spre[:, sl]), O.ACT_SWIGLU)
+        m_, n_, j_ = iA
+        acc["dA"] += np.einsum("ni,ni->n", cb["dpre"][m_, :, n_], f64(host["X"][:, sl])[m_, :, j_])
+        bwd_s["dX"].append(cb["dX"][:, loc]); bwd_s["dR"].append(gm[:, loc]); bwd_s["dY"].append(dY[:, loc])
+    bwd_s = {k: np.concatenate(v, axis=1) for k, v in bwd_s.items()}
+    ctx.rowpar_backward(caat.CAAT_MLP_DOWN, T, dev["dXout"], dev["dHn"], sY.cuda(), dev["B"], sHn.cuda(), sr.cuda(), None,
+                        dev["gamma"], bo["dY"], bo["dB"], bo["dR"], bo["dgamma"], None, ws)
+    # the column-parallel backward runs on the oracle's dY (rounded), so the two halves are checked independently
+    ctx.colpar_backward(caat.CAAT_ACT_SWIGLU, 2 * F, T, dY_saved.cuda(), dev["X"], dev["A"], spre.cuda(), bo["dX"], bo["dA"], ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+    for k in bwd_s:
+        assert_close(bo[k].index_select(1, tk), bwd_s[k], "bf16", f"{name}:{k}")
+    assert_close(bo["dgamma"], acc["dgamma"], "bf16", f"{name}:dgamma")
+    m_, l_, k_ = (torch.from_numpy(x).cuda() for x in iB)
+    assert_close(bo["dB"][m_, l_, k_], acc["dB"], "bf16", f"{name}:dB")
+    m_, n_, j_ = (torch.from_numpy(x).cuda() for x in iA)
+    assert_close(bo["dA"][m_, n_, j_], acc["dA"], "bf16", f"{name}:dA")
+
+
+@pytest.mark.parametrize("name", ["mlp_130m", "mlp_7b"])
+def test_full_size_mlp(name):
+    _check_mlp_full(name)
