@@ -842,7 +842,10 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16
 bool tc_dgrad_wants_wt(int tokens) {
   static const int env = [] { const char* e = getenv("CAAT_TC_WT"); return e ? atoi(e) : -1; }();
   if (env >= 0) return env == 1;
-  return tokens >= 4096;
+  // Off by default: with the B operand's boxes issued by a producer warp of their own, reading W in
+  // place (N-major) beats transposing it first at every size measured (7B dgrad 1.86 vs 2.01 ms).
+  (void)tokens;
+  return false;
 }
 
 // ---- dgrad: dY[m] = gs W[m][:S] + zp[m] W[m][S:]

@@ -55,7 +55,7 @@ def _colpar_gpu(ctx, act, n_out, d, pre_saved=None):
     (8, 130, 4096, 1536, "bf16", False),    # 7B QKV width 3 h / t
     (2, 70, 256, 1024, "f32", False),       # fp32 runs on the CUDA-core GEMM
     (3, 45, 264, 176, "bf16", True),        # forced CUDA-core GEMM in bf16
-    (8, 5000, 1024, 512, "bf16", False),    # many tokens: the data gradient reads transposed weights
+    (8, 5000, 1024, 512, "bf16", False),    # many tokens, persistent CTAs walk many tiles
 ])
 def test_colpar_forward_backward(act, t, T, h, n_out, dtype, simt):
     ctx = G.make_ctx(t, h, 4 * h, dtype, force_simt=simt)
