@@ -634,6 +634,9 @@ double estimate_cost(const RegionShape* r, int nr, int bn, int cg, int splits, d
 
 TileCfg pick_tile(const RegionShape* r, int nr, bool b_n_major, int max_splits, double out_bytes) {
   static const int max_cg = [] { const char* e = getenv("CAAT_TC_CG"); return e && atoi(e) == 1 ? 1 : 2; }();
+  // measurement aids: CAAT_TC_BN / CAAT_TC_CGF pin the tile width / the pair mode instead of the model's choice
+  static const int force_bn = [] { const char* e = getenv("CAAT_TC_BN"); return e ? atoi(e) : 0; }();
+  static const int force_cg = [] { const char* e = getenv("CAAT_TC_CGF"); return e ? atoi(e) : 0; }();
   TileCfg best{256, 1, 1, -1.0};
   int min_ksteps = 1 << 30;
   for (int i = 0; i < nr; ++i)
@@ -647,8 +650,10 @@ TileCfg pick_tile(const RegionShape* r, int nr, bool b_n_major, int max_splits, 
       if (r[i].N < nmin) nmin = r[i].N;
     }
     if (!ok) continue;
+    if (force_cg && cg != force_cg && !(force_cg == 2 && cg == 1 && max_cg == 2)) continue;
     const int step = b_n_major ? 64 * cg : 32 * cg;    // N-major B: whole 64-column chunks per CTA
     for (int bn = 256; bn >= 64 * cg; bn -= step) {
+      if (force_bn && bn != force_bn && force_bn % step == 0 && force_bn >= 64 * cg) continue;
       for (int splits = 1; splits <= max_splits; ++splits) {
         if (splits > 1 && min_ksteps / splits < 8) break;
         const double c = estimate_cost(r, nr, bn, cg, splits, out_bytes, b_n_major);
