@@ -2,6 +2,7 @@
 // sequences of the forward / backward of one row-parallel layer and of a block.
 #include <atomic>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -34,6 +35,11 @@ LaunchScope::LaunchScope(int kind, cudaStream_t s) : slot(-1), st(s) {
 }
 LaunchScope::~LaunchScope() {
   if (slot >= 0) cudaEventRecord(g_prof.ev[2 * slot + 1], st);
+}
+
+bool pdl_enabled() {
+  static const bool on = [] { const char* e = getenv("CAAT_PDL"); return !(e && e[0] == '0'); }();
+  return on;
 }
 
 unsigned int* device_status_word() {

@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(256) act_forward_kernel(const void* __restrict
   const int chunks = width_out / V;
   const int ld_pre = GATED ? 2 * width_out : width_out;
   const long long total = rows * chunks;
+  pdl_wait();
   for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < total; q += (long long)gridDim.x * blockDim.x) {
     const long long r = q / chunks;
     const int c = (int)(q - r * chunks) * V;
@@ -64,6 +65,7 @@ __global__ void __launch_bounds__(256) act_backward_kernel(const void* __restric
   const int chunks = width_out / V;
   const int ld_pre = GATED ? 2 * width_out : width_out;
   const long long total = rows * chunks;
+  pdl_wait();
   for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < total; q += (long long)gridDim.x * blockDim.x) {
     const long long r = q / chunks;
     const int c = (int)(q - r * chunks) * V;
@@ -118,11 +120,11 @@ cudaError_t launch_act_forward(caat_dtype dtype, int gated, const void* pre, voi
   const int grid = act_grid(rows, width_out, V);
   LaunchScope scope(CAAT_K_ACTIVATION, st);
   if (dtype == CAAT_BF16) {
-    if (gated) act_forward_kernel<__nv_bfloat16, true><<<grid, 256, 0, st>>>(pre, Y, rows, width_out);
-    else act_forward_kernel<__nv_bfloat16, false><<<grid, 256, 0, st>>>(pre, Y, rows, width_out);
+    if (gated) return launch_pdl(act_forward_kernel<__nv_bfloat16, true>, dim3(grid), dim3(256), 0, st, pre, Y, rows, width_out);
+    else return launch_pdl(act_forward_kernel<__nv_bfloat16, false>, dim3(grid), dim3(256), 0, st, pre, Y, rows, width_out);
   } else {
-    if (gated) act_forward_kernel<float, true><<<grid, 256, 0, st>>>(pre, Y, rows, width_out);
-    else act_forward_kernel<float, false><<<grid, 256, 0, st>>>(pre, Y, rows, width_out);
+    if (gated) return launch_pdl(act_forward_kernel<float, true>, dim3(grid), dim3(256), 0, st, pre, Y, rows, width_out);
+    else return launch_pdl(act_forward_kernel<float, false>, dim3(grid), dim3(256), 0, st, pre, Y, rows, width_out);
   }
   return cudaGetLastError();
 }
@@ -133,11 +135,11 @@ cudaError_t launch_act_backward(caat_dtype dtype, int gated, const void* dY, con
   const int grid = act_grid(rows, width_out, V);
   LaunchScope scope(CAAT_K_ACTIVATION, st);
   if (dtype == CAAT_BF16) {
-    if (gated) act_backward_kernel<__nv_bfloat16, true><<<grid, 256, 0, st>>>(dY, pre, dpre, rows, width_out);
-    else act_backward_kernel<__nv_bfloat16, false><<<grid, 256, 0, st>>>(dY, pre, dpre, rows, width_out);
+    if (gated) return launch_pdl(act_backward_kernel<__nv_bfloat16, true>, dim3(grid), dim3(256), 0, st, dY, pre, dpre, rows, width_out);
+    else return launch_pdl(act_backward_kernel<__nv_bfloat16, false>, dim3(grid), dim3(256), 0, st, dY, pre, dpre, rows, width_out);
   } else {
-    if (gated) act_backward_kernel<float, true><<<grid, 256, 0, st>>>(dY, pre, dpre, rows, width_out);
-    else act_backward_kernel<float, false><<<grid, 256, 0, st>>>(dY, pre, dpre, rows, width_out);
+    if (gated) return launch_pdl(act_backward_kernel<float, true>, dim3(grid), dim3(256), 0, st, dY, pre, dpre, rows, width_out);
+    else return launch_pdl(act_backward_kernel<float, false>, dim3(grid), dim3(256), 0, st, dY, pre, dpre, rows, width_out);
   }
   return cudaGetLastError();
 }

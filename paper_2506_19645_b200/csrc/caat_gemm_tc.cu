@@ -310,6 +310,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
   if (CG == 2) cluster_sync();      // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();   // set-up done; operands and outputs may still be in use by the previous kernel until here
 
   if (warp == 0 || warp == kProducerB) {
     // ------------------------------------------------------------ TMA producers
@@ -542,6 +543,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
 // out[i] = sum_s part[s][i], s ascending (deterministic split-K reduction)
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float4* __restrict__ part, float4* __restrict__ out,
                                                             long long n4, int splits) {
+  pdl_wait();
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (long long)gridDim.x * blockDim.x) {
     float4 s = part[i];
     for (int k = 1; k < splits; ++k) {
@@ -704,13 +706,15 @@ cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr{};
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = (unsigned)p.cg;
-  attr.val.clusterDim.y = 1;
-  attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
+  cudaLaunchAttribute attr[2] = {};
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)p.cg;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
   LaunchScope scope(kind, st);
   if (p.cg == 2)
     return cudaLaunchKernelEx(&cfg, tc_gemm_kernel<2>, maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], p);
@@ -958,9 +962,8 @@ cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* z
     int blocks = (int)((n4 + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
     LaunchScope scope(CAAT_K_SPLITK_REDUCE, st);
-    splitk_reduce_kernel<<<blocks, 256, 0, st>>>(static_cast<const float4*>(splitk), reinterpret_cast<float4*>(dW), n4,
-                                                 splits);
-    e = cudaGetLastError();
+    e = launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, st, static_cast<const float4*>(splitk),
+                   reinterpret_cast<float4*>(dW), n4, splits);
   }
   return e;
 }

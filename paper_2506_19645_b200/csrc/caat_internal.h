@@ -162,6 +162,34 @@ cudaError_t launch_act_forward(caat_dtype dtype, int gated, const void* pre, voi
 cudaError_t launch_act_backward(caat_dtype dtype, int gated, const void* dY, const void* pre, void* dpre,
                                 long long rows, int width_out, cudaStream_t st);
 
+// ---- programmatic dependent launch --------------------------------------------
+// Kernels launched through launch_pdl may be scheduled while their predecessor in the stream is still
+// draining: their CTAs set up shared memory, barriers and tensor memory, then call pdl_wait(), which
+// returns once the predecessor has completed and its writes are visible.  Nothing that reads or writes
+// global memory may precede pdl_wait().  (Without the launch attribute the instruction returns at once.)
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+bool pdl_enabled();   // CAAT_PDL=0 in the environment switches the launch attribute off (measurements)
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- bookkeeping ------------------------------------------------------------
 // Brackets one kernel launch: counts it and, while profiling is on, records a CUDA event
 // before and after it on the launching stream.

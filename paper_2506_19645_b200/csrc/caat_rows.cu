@@ -385,6 +385,7 @@ __global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPar
   constexpr int V = V_::N;
   constexpr int ES = sizeof(T_);
   extern __shared__ float sm[];
+  pdl_wait();
   float* hrow = sm;                       // [h] the new residual stream of this row, fp32
   float* red = sm + a.h;                  // reduction scratch
   int par = 0;
@@ -463,6 +464,7 @@ __global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPar
 __global__ void __launch_bounds__(1024) reduce_partials_kernel(const float* __restrict__ part, float* __restrict__ out,
                                                                int rows, int h) {
   __shared__ float sm[32][33];
+  pdl_wait();
   const int c = blockIdx.x * 32 + threadIdx.x;
   float s = 0.f;
   if (c < h)
@@ -516,13 +518,11 @@ cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype,
   const size_t smem = (size_t)a.h * sizeof(float) + 2 * 16 * 2 * sizeof(float);
   LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
   if (dtype == CAAT_BF16) {
-    if (a.norm == 1) rows_forward_partials_kernel<__nv_bfloat16, true><<<grid, threads, smem, st>>>(a);
-    else rows_forward_partials_kernel<__nv_bfloat16, false><<<grid, threads, smem, st>>>(a);
-  } else {
-    if (a.norm == 1) rows_forward_partials_kernel<float, true><<<grid, threads, smem, st>>>(a);
-    else rows_forward_partials_kernel<float, false><<<grid, threads, smem, st>>>(a);
+    if (a.norm == 1) return launch_pdl(rows_forward_partials_kernel<__nv_bfloat16, true>, grid, dim3(threads), smem, st, a);
+    return launch_pdl(rows_forward_partials_kernel<__nv_bfloat16, false>, grid, dim3(threads), smem, st, a);
   }
-  return cudaGetLastError();
+  if (a.norm == 1) return launch_pdl(rows_forward_partials_kernel<float, true>, grid, dim3(threads), smem, st, a);
+  return launch_pdl(rows_forward_partials_kernel<float, false>, grid, dim3(threads), smem, st, a);
 }
 
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype) {
@@ -573,11 +573,13 @@ cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int dire
   const dim3 rg((a.h + 31) / 32);
   {
     LaunchScope scope(CAAT_K_NORMGRAD_REDUCE, st);
-    reduce_partials_kernel<<<rg, rb, 0, st>>>(a.dgpart, a.dgamma, rows, a.h);
+    e = launch_pdl(reduce_partials_kernel, rg, rb, 0, st, (const float*)a.dgpart, a.dgamma, rows, a.h);
+    if (e != cudaSuccess) return e;
   }
   if (a.norm == 1 && a.dbeta && a.dbpart) {
     LaunchScope scope(CAAT_K_NORMGRAD_REDUCE, st);
-    reduce_partials_kernel<<<rg, rb, 0, st>>>(a.dbpart, a.dbeta, rows, a.h);
+    e = launch_pdl(reduce_partials_kernel, rg, rb, 0, st, (const float*)a.dbpart, a.dbeta, rows, a.h);
+    if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();
 }

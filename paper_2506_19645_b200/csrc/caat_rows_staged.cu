@@ -141,6 +141,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     *reinterpret_cast<uint4*>(ring + (size_t)(threadIdx.y * TX + threadIdx.x) * sg.stage_bytes + sg.zero_off) =
         make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
+  pdl_wait();   // from here on global memory is touched
   for (int q = 0; q < NS; ++q) issue();
 
   // Per-thread constants of the hot loop: the chunk's class and its byte offsets inside a stage.  Chunks
@@ -399,6 +400,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
   if (tid < NS)   // the zero slot of every stage (no copy ever lands there)
     *reinterpret_cast<uint4*>(ring + (size_t)tid * sg.stage_bytes + sg.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
+  pdl_wait();   // from here on global memory is touched
   for (int q = 0; q < NS; ++q) issue();
   load_stats(0, stat);
 
@@ -714,7 +716,7 @@ cudaError_t launch_fwd_staged_t(const RowFwdArgs& a, const RowGeom& g, const Sta
 #define CAAT_LAUNCH(CPT_, MAXT_)                                                                   \
   do {                                                                                             \
     e = set_smem(rows_forward_staged<T_, CPT_, LN, MAXT_, CL>, sg.smem);                                        \
-    if (e == cudaSuccess) rows_forward_staged<T_, CPT_, LN, MAXT_, CL><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);   \
+    if (e == cudaSuccess) e = launch_pdl(rows_forward_staged<T_, CPT_, LN, MAXT_, CL>, dim3(grid), block, sg.smem, st, a, sg, ngroups, status);   \
   } while (0)
   if (g.CPT == 1 && threads <= 256) CAAT_LAUNCH(1, 256);
   else if (g.CPT == 1) CAAT_LAUNCH(1, 512);
@@ -736,7 +738,7 @@ cudaError_t launch_bwd_staged_t(const RowBwdArgs& a, const RowGeom& g, const Sta
 #define CAAT_LAUNCH(CPT_, MAXT_)                                                                   \
   do {                                                                                             \
     e = set_smem(rows_backward_staged<T_, CPT_, LN, MAXT_, CL>, sg.smem);                                        \
-    if (e == cudaSuccess) rows_backward_staged<T_, CPT_, LN, MAXT_, CL><<<grid, block, sg.smem, st>>>(a, sg, ngroups, status);   \
+    if (e == cudaSuccess) e = launch_pdl(rows_backward_staged<T_, CPT_, LN, MAXT_, CL>, dim3(grid), block, sg.smem, st, a, sg, ngroups, status);   \
   } while (0)
   if (g.CPT == 1 && threads <= 256) CAAT_LAUNCH(1, 256);
   else if (g.CPT == 1) CAAT_LAUNCH(1, 512);

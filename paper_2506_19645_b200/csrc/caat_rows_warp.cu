@@ -91,6 +91,7 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
   if ((int)threadIdx.x < NS)   // the zero slot of every stage (no copy ever lands there)
     *reinterpret_cast<uint4*>(ring + (size_t)threadIdx.x * sg.stage_bytes + sg.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
+  pdl_wait();   // from here on global memory is touched
 
   if (warp == kW) {
     // ---------------------------------------------------------- producer
@@ -303,6 +304,7 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
   if ((int)threadIdx.x < NS)   // the zero slot of every stage (no copy ever lands there)
     *reinterpret_cast<uint4*>(ring + (size_t)threadIdx.x * sg.stage_bytes + sg.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
+  pdl_wait();   // from here on global memory is touched
 
   constexpr int H2 = V / 2;
   int col[CPT], cls[CPT];
@@ -600,7 +602,7 @@ cudaError_t launch_fwd_warp_t(const RowFwdArgs& a, int cpt, const WarpGeom& g, i
 #define CAAT_LAUNCH(CPT_)                                                                      \
   do {                                                                                         \
     e = set_smem(rows_forward_warp<T_, CPT_, LN, CL>, g.smem);                                 \
-    if (e == cudaSuccess) rows_forward_warp<T_, CPT_, LN, CL><<<grid, kThreads, g.smem, st>>>(a, g, ngroups, status); \
+    if (e == cudaSuccess) e = launch_pdl(rows_forward_warp<T_, CPT_, LN, CL>, dim3(grid), dim3(kThreads), g.smem, st, a, g, ngroups, status); \
   } while (0)
   switch (cpt) {
     case 1: CAAT_LAUNCH(1); break;
@@ -621,7 +623,7 @@ cudaError_t launch_bwd_warp_t(const RowBwdArgs& a, int cpt, const WarpGeom& g, i
 #define CAAT_LAUNCH(CPT_)                                                                       \
   do {                                                                                          \
     e = set_smem(rows_backward_warp<T_, CPT_, LN, CL>, g.smem);                                 \
-    if (e == cudaSuccess) rows_backward_warp<T_, CPT_, LN, CL><<<grid, kThreads, g.smem, st>>>(a, g, ngroups, status); \
+    if (e == cudaSuccess) e = launch_pdl(rows_backward_warp<T_, CPT_, LN, CL>, dim3(grid), dim3(kThreads), g.smem, st, a, g, ngroups, status); \
   } while (0)
   switch (cpt) {
     case 1: CAAT_LAUNCH(1); break;
