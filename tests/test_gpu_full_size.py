@@ -224,3 +224,101 @@ def _check_mlp_full(name, n_tok=32, n_dw=384, seed=321):
 @pytest.mark.parametrize("name", ["mlp_130m", "mlp_7b"])
 def test_full_size_mlp(name):
     _check_mlp_full(name)
+
+
+def _check_block_full_compact(name, n_tok=32, n_dw=384, seed=456):
+    """The block on the compact residual stream (shared channels stored once) at the bench's size and launch
+    sequence: chunked oracle, sampled tokens for per-token outputs, token sums accumulated over chunks."""
+    w = synthetic.WORKLOADS[name]
+    t, T, h, S = w.t, w.tokens, w.h, w.S
+    alpha = math.sqrt(t)
+    ka, km = w.kr_attn, w.kr_mlp
+    dev = synthetic.block_inputs(w, device="cuda")
+    host = {k: v.cpu() for k, v in dev.items()}
+    split = lambda x: (x[0, :, :S].contiguous(), x[:, :, S:].contiguous())
+    R0s, R0p = split(host["R0"]); dH2s, dH2p = split(host["dHn2"])
+    rng = np.random.default_rng(seed)
+    tok = np.sort(rng.choice(T, size=min(n_tok, T), replace=False))
+    dws = {"attn": (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, ka, n_dw)),
+           "mlp": (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, km, n_dw))}
+    Wd = {"attn": f64(host["W_o"]), "mlp": f64(host["W_down"])}
+    g1, g2 = f64(host["gamma1"]), f64(host["gamma2"])
+    bf, f32 = torch.bfloat16, torch.float32
+
+    sv = {"Hn1s": torch.empty((T, S), dtype=bf), "Hn1p": torch.empty((t, T, h - S), dtype=bf), "rstd1": torch.empty((t, T), dtype=f32),
+          "Hn2s": torch.empty((T, S), dtype=bf), "Hn2p": torch.empty((t, T, h - S), dtype=bf), "rstd2": torch.empty((t, T), dtype=f32)}
+    keys = ("Hn1s", "Hn1p", "X1", "rstd1", "Hn2s", "Hn2p", "X2", "rstd2")
+    fwd_s = {k: [] for k in keys}
+    tdim = lambda k: 0 if k.endswith("s") else 1           # token axis of a tensor: shared parts are [T, S]
+    for a, b in _chunks(T):
+        sl = slice(a, b)
+        o = O.block_forward_compact(f64(host["Y_attn"][:, sl]), Wd["attn"], f64(host["Y_mlp"][:, sl]), Wd["mlp"],
+                                    f64(R0s[sl]), f64(R0p[:, sl]), g1, g2, S=S, alpha=alpha)
+        for k in sv:
+            if tdim(k) == 0:
+                sv[k][sl] = torch.from_numpy(o[k]).to(sv[k].dtype)
+            else:
+                sv[k][:, sl] = torch.from_numpy(o[k]).to(sv[k].dtype)
+        loc = tok[(tok >= a) & (tok < b)] - a
+        for k in keys:
+            fwd_s[k].append(np.take(o[k], loc, axis=tdim(k)))
+    fwd_s = {k: np.concatenate(v, axis=tdim(k)) for k, v in fwd_s.items()}
+
+    ctx = caat.Context(w.h, w.ffn, t, w.p, "bf16")
+    mk = lambda *s, dt=bf: torch.empty(*s, dtype=dt, device="cuda")
+    out = {"Hn1s": mk(T, S), "Hn1p": mk(t, T, h - S), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=f32),
+           "Hn2s": mk(T, S), "Hn2p": mk(t, T, h - S), "X2": mk(t, T, h), "rstd2": mk(t, T, dt=f32)}
+    ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, True))
+    ctx.block_forward_compact(T, dev["Y_attn"], dev["W_o"], dev["Y_mlp"], dev["W_down"], R0s.cuda(), R0p.cuda(), dev["gamma1"],
+                              None, dev["gamma2"], None, out["Hn1s"], out["Hn1p"], out["X1"], out["rstd1"], None,
+                              out["Hn2s"], out["Hn2p"], out["X2"], out["rstd2"], None, ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+    tk = torch.from_numpy(tok).cuda()
+    for k in keys:
+        assert_close(out[k].index_select(tdim(k), tk), fwd_s[k], "bf16", f"{name}:{k}")
+    del out
+
+    bo = {"dY_attn": mk(t, T, ka), "dW_o": mk(t, h, ka, dt=f32), "dY_mlp": mk(t, T, km), "dW_down": mk(t, h, km, dt=f32),
+          "dR0s": mk(T, S), "dR0p": mk(t, T, h - S), "dHn1s": mk(T, S), "dHn1p": mk(t, T, h - S),
+          "dgamma1": mk(h, dt=f32), "dgamma2": mk(h, dt=f32)}
+    ctx.block_backward_compact(T, dev["dX1"], dev["dX2"], dH2s.cuda(), dH2p.cuda(), dev["Y_attn"], dev["W_o"], dev["Y_mlp"],
+                               dev["W_down"], sv["Hn1s"].cuda(), sv["Hn1p"].cuda(), sv["rstd1"].cuda(), None,
+                               sv["Hn2s"].cuda(), sv["Hn2p"].cuda(), sv["rstd2"].cuda(), None, dev["gamma1"], dev["gamma2"],
+                               bo["dY_attn"], bo["dW_o"], bo["dY_mlp"], bo["dW_down"], bo["dR0s"], bo["dR0p"], bo["dHn1s"],
+                               bo["dHn1p"], bo["dgamma1"], None, bo["dgamma2"], None, ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+
+    acc = {"dgamma1": np.zeros(h), "dgamma2": np.zeros(h), "dW_attn": np.zeros(n_dw), "dW_mlp": np.zeros(n_dw)}
+    bkeys = ("dY_attn", "dY_mlp", "dR0s", "dR0p", "dHn1s", "dHn1p")
+    bwd_s = {k: [] for k in bkeys}
+    for a, b in _chunks(T):
+        sl = slice(a, b)
+        loc = tok[(tok >= a) & (tok < b)] - a
+        b2 = O.rowpar_backward_compact(f64(host["dX2"][:, sl]), f64(dH2s[sl]), f64(dH2p[:, sl]), f64(host["Y_mlp"][:, sl]),
+                                       Wd["mlp"], f64(sv["Hn2s"][sl]), f64(sv["Hn2p"][:, sl]), f64(sv["rstd2"][:, sl]), None, g2,
+                                       S=S, alpha=alpha)
+        b1 = O.rowpar_backward_compact(f64(host["dX1"][:, sl]), b2["dRs"], b2["dRp"], f64(host["Y_attn"][:, sl]), Wd["attn"],
+                                       f64(sv["Hn1s"][sl]), f64(sv["Hn1p"][:, sl]), f64(sv["rstd1"][:, sl]), None, g1,
+                                       S=S, alpha=alpha)
+        acc["dgamma2"] += b2["dgamma"]; acc["dgamma1"] += b1["dgamma"]
+        for key, bb in (("attn", b1), ("mlp", b2)):
+            m_, l_, k_ = dws[key]
+            acc["dW_" + key] += bb["dW"][m_, l_, k_]
+        for k, v in (("dY_attn", b1["dY"]), ("dY_mlp", b2["dY"]), ("dR0s", b1["dRs"]), ("dR0p", b1["dRp"]),
+                     ("dHn1s", b2["dRs"]), ("dHn1p", b2["dRp"])):
+            bwd_s[k].append(np.take(v, loc, axis=tdim(k) if k.startswith("dR") or k.startswith("dHn") else 1))
+    for k in bkeys:
+        ax = tdim(k) if k.startswith("dR") or k.startswith("dHn") else 1
+        assert_close(bo[k].index_select(ax, tk), np.concatenate(bwd_s[k], axis=ax), "bf16", f"{name}:{k}")
+    assert_close(bo["dgamma1"], acc["dgamma1"], "bf16", f"{name}:dgamma1")
+    assert_close(bo["dgamma2"], acc["dgamma2"], "bf16", f"{name}:dgamma2")
+    for key, gk in (("attn", "dW_o"), ("mlp", "dW_down")):
+        m_, l_, k_ = (torch.from_numpy(x).cuda() for x in dws[key])
+        assert_close(bo[gk][m_, l_, k_], acc["dW_" + key], "bf16", f"{name}:{gk}")
+
+
+@pytest.mark.parametrize("name", ["block_130m", "block_7b"])
+def test_full_size_block_compact(name):
+    _check_block_full_compact(name)
