@@ -125,8 +125,9 @@ def layer_work(w, k_r, backward, compact=False):
         "rows_forward": {"flops": 0.0, "bytes": zsz + 2 * stream + full + t * T * 4},
     }
     if backward:
-        # reads dX, Hn, dHn; writes dR and the scratch (compact: dRs is the scratch's shared part)
-        bwd_out = stream + t * T * (h - S) * e if compact else stream + zsz
+        # reads dX, Hn, dHn; writes dR and the reduced shared gradient gs [T, S] (compact: gs is dRs, part of dR).
+        # The GEMMs read the private gradient from dR itself: no scaled copy is written.
+        bwd_out = stream if compact else stream + T * S * e
         out["rows_backward"] = {"flops": 0.0, "bytes": full + 2 * stream + bwd_out + t * T * 4}
         out["tc_gemm_dgrad"] = {"flops": 2.0 * T * K * h, "bytes": zsz + K * h * e + T * K * e}
         out["tc_gemm_wgrad"] = {"flops": 2.0 * T * K * h, "bytes": zsz + T * K * e + K * h * 4}

@@ -94,7 +94,7 @@ Scratch scratch_layout(const caat_ctx* ctx, int K_r, int tokens, int backward) {
     }
     off = align_up(off + s.splitk_bytes, 256);
     s.wt_off = off;
-    if (tc_gemm_usable(ctx, K_r) && tc_dgrad_wants_wt(tokens))
+    if (tc_gemm_usable(ctx, K_r) && ctx->alpha != 1.0 && ctx->S < ctx->h)
       off = align_up(off + (size_t)ctx->t * ctx->h * K_r * e, 256);
   }
   s.total = off;
@@ -196,19 +196,27 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
   const size_t e = elem_size(ctx->dtype);
   cudaError_t ce;
 
+  // Tensor-core path: the GEMMs take the private gradient straight from dR (alpha rides on the weights'
+  // private rows in the data gradient and on the epilogue in the weight gradient), so the row kernel writes
+  // no scaled copy of it.
+  const bool tc = tc_gemm_usable(ctx, K_r);
+  if (tc) zp = nullptr;
   RowBwdArgs a{dX, dHn, Hn, gamma, rstd, mean, dR, gs, zp,
                reinterpret_cast<float*>(wsb + L.dgpart_off), reinterpret_cast<float*>(wsb + L.dbpart_off),
                dgamma, dbeta, t, T, h, S, L.S_lo, L.S_hi, L.P, (float)ctx->alpha, ctx->norm};
   a.compact = compact; a.Hns = Hns; a.dHns = dHns;
   a.reduce_mode = ctx->bwd_reduce;
+  const bool prescale = tc && ctx->alpha != 1.0 && S < h;
+  if (prescale) { a.w_src = W; a.w_dst = wsb + L.wt_off; a.w_Kr = K_r; }
   ce = launch_rows_backward(a, ctx->dtype, ctx->bwd_reduce ? 1 : ctx->direct_rows, st);
   if (ce != cudaSuccess) return cuda_fail(ce);
 
-  if (tc_gemm_usable(ctx, K_r)) {
+  if (tc) {
     RowparShapes sh{t, T, h, K_r, S, L.S_lo, L.S_hi, L.P};
-    ce = launch_tc_dgrad(sh, gs, zp, W, dY, tc_dgrad_wants_wt(T) ? wsb + L.wt_off : nullptr, st);
+    const PrivOperand pv = compact ? PrivOperand{dR, L.P, 0, (float)ctx->alpha} : PrivOperand{dR, h, S, (float)ctx->alpha};
+    ce = launch_tc_dgrad(sh, gs, pv, W, dY, wsb + L.wt_off, prescale, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
-    ce = launch_tc_wgrad(sh, gs, zp, Y, dW, wsb + L.splitk_off, L.splitk_bytes, st);
+    ce = launch_tc_wgrad(sh, gs, pv, Y, dW, wsb + L.splitk_off, L.splitk_bytes, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
     return CAAT_OK;
   }
@@ -528,7 +536,6 @@ ColScratch col_scratch(const caat_ctx* ctx, caat_activation act, int n_out, int 
     s.splitk_bytes = tc_wgrad_splitk_bytes(col_shapes(ctx, n_out, T));
     off = align_up(off + s.splitk_bytes, 256);
     s.wt_off = off;
-    if (tc_dgrad_wants_wt(T)) off = align_up(off + (size_t)ctx->t * ctx->h * n_out * e, 256);
   }
   s.total = off > 16 ? off : 16;
   return s;
@@ -602,9 +609,10 @@ caat_status caat_colpar_backward(const caat_ctx* ctx, caat_activation act, int n
   }
   if (col_tc_usable(ctx, n_out)) {
     const RowparShapes sh = col_shapes(ctx, n_out, T);
-    ce = launch_tc_dgrad(sh, nullptr, dpre, A, dX, tc_dgrad_wants_wt(T) ? wsb + L.wt_off : nullptr, st);
+    const PrivOperand pv{dpre, n_out, 0, 1.0f};
+    ce = launch_tc_dgrad(sh, nullptr, pv, A, dX, nullptr, false, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
-    ce = launch_tc_wgrad(sh, nullptr, dpre, X, dA, wsb + L.splitk_off, L.splitk_bytes, st);
+    ce = launch_tc_wgrad(sh, nullptr, pv, X, dA, wsb + L.splitk_off, L.splitk_bytes, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
     return CAAT_OK;
   }

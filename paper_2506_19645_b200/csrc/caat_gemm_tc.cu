@@ -59,7 +59,9 @@ struct Region {          // a family of output tiles with the same operand wirin
   float* out_t;          // transposed direct-store output (decode), else unused
   int splits;            // split-K factor of this region's tiles (set by finish_tiles from Params::splits when 0)
   int b_slowest;         // tile order: 1 = rank index slowest (a rank's weights / activations stay
-};                       // hot in L2 while its row tiles stream), 0 = row tile slowest
+                         // hot in L2 while its row tiles stream), 0 = row tile slowest
+  float scale;           // fp32 outputs are multiplied by it in the epilogue (0 means 1)
+};
 
 struct Params {
   int nregions;
@@ -489,6 +491,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = 0u;
         }
+        if (p.out_f32 && r.scale != 0.f && r.scale != 1.f) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * r.scale);
+        }
         const uint32_t buf = smem_u32(cstage + (size_t)(slab % 3) * kCBuf);
         const uint32_t rowaddr = buf + (uint32_t)rr * 64u;
         if (p.out_f32) {
@@ -826,73 +832,70 @@ cudaError_t launch_tc_forward_decode(int t, int T, int h, const DecodeProblem* p
   return launch(maps, cmaps, p, CAAT_K_TC_FORWARD, st);
 }
 
-// out[b][c][r] = in[b][r][c]  (bf16, per-rank weight shard [rows = h][cols = K_r] -> [K_r][h])
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in,
-                                                             __nv_bfloat16* __restrict__ out, int rows, int cols) {
-  __shared__ __nv_bfloat16 tile[64][66];
-  const long long plane = (long long)rows * cols;
-  const __nv_bfloat16* src = in + blockIdx.z * plane;
-  __nv_bfloat16* dst = out + blockIdx.z * plane;
-  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
-  for (int i = threadIdx.y; i < 64; i += 4) {
-    const int r = r0 + i, c = c0 + threadIdx.x;
-    if (r < rows && c < cols) tile[i][threadIdx.x] = src[(long long)r * cols + c];
-  }
-  __syncthreads();
-  for (int i = threadIdx.y; i < 64; i += 4) {
-    const int c = c0 + i, r = r0 + threadIdx.x;
-    if (r < rows && c < cols) dst[(long long)c * rows + r] = tile[threadIdx.x][i];
+// out[b][l][:] = alpha * W[b][l][:] for the private rows l in [S, h) of every rank's weight shard (bf16,
+// 16 bytes per thread).  The data gradient then takes the private gradient g as stored in dR instead of
+// a scaled copy of it: sum_l (alpha g[l]) W[l][k] = sum_l g[l] (alpha W[l][k]); the weights are the
+// small operand.
+__global__ void __launch_bounds__(256) scale_private_rows_kernel(const uint4* __restrict__ W, uint4* __restrict__ out,
+                                                                 int h, int K_r, int S, float alpha) {
+  pdl_wait();
+  const int row_chunks = K_r / 8;
+  const long long per_rank = (long long)(h - S) * row_chunks;
+  const long long base = ((long long)blockIdx.y * h + S) * row_chunks;
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < per_rank; q += (long long)gridDim.x * blockDim.x) {
+    const uint4 v = W[base + q];
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+    unsigned o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 bb = __floats2bfloat162_rn(alpha * __uint_as_float(w[i] << 16), alpha * __uint_as_float(w[i] & 0xffff0000u));
+      o[i] = *reinterpret_cast<unsigned*>(&bb);
+    }
+    out[base + q] = make_uint4(o[0], o[1], o[2], o[3]);
   }
 }
 
-// The data gradient reads its B operand (the weights) fastest when the contraction index is
-// contiguous (measured: the N-major form costs about 10 % of the kernel).  Transposing the weights
-// costs 4 * K * h bytes of traffic, which pays off once there are a few thousand tokens.
-bool tc_dgrad_wants_wt(int tokens) {
-  static const int env = [] { const char* e = getenv("CAAT_TC_WT"); return e ? atoi(e) : -1; }();
-  if (env >= 0) return env == 1;
-  // Off by default: with the B operand's boxes issued by a producer warp of their own, reading W in
-  // place (N-major) beats transposing it first at every size measured (7B dgrad 1.86 vs 2.01 ms).
-  (void)tokens;
-  return false;
-}
-
-// ---- dgrad: dY[m] = gs W[m][:S] + zp[m] W[m][S:]
-cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* zp, const void* W, void* dY,
-                            void* wt_scratch, cudaStream_t st) {
+// ---- dgrad: dY[m] = gs W[m][:S] + (alpha gp[m]) W[m][S:]
+// pv describes where the private gradient lives and what still multiplies it (see PrivOperand); when
+// pv.alpha != 1 the private rows of W are scaled into w_scaled ([t, h, K_r], only rows >= S are written).
+cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const PrivOperand& pv, const void* W, void* dY,
+                            void* w_scaled, bool w_scaled_ready, cudaStream_t st) {
   CUtensorMap maps[4], cmaps[2];
   Params p{};
-  const bool use_wt = wt_scratch != nullptr && s.h % 8 == 0;
   {
     const RegionShape rs[1] = {{s.T, s.K_r, s.t, (s.S + BK - 1) / BK + (s.h - s.S + BK - 1) / BK}};
-    const TileCfg c = pick_tile(rs, 1, !use_wt, 1, 0.0);
+    const TileCfg c = pick_tile(rs, 1, true, 1, 0.0);
     p.BN = c.bn; p.cg = c.cg;
   }
   const int n_sh = s.S, n_pr = s.h - s.S;
-  if (use_wt) {
-    // B = W[m]^T as [K_r rows (N)][h contiguous (contraction)]: K-major, like the forward's B
-    const dim3 tb(64, 4), tg((s.K_r + 63) / 64, (s.h + 63) / 64, s.t);
-    {
-      LaunchScope scope(CAAT_K_TC_DGRAD, st);
-      transpose_bf16_kernel<<<tg, tb, 0, st>>>(static_cast<const __nv_bfloat16*>(W), static_cast<__nv_bfloat16*>(wt_scratch), s.h, s.K_r);
-    }
-    if (!make_map(&maps[1], wt_scratch, s.h, s.K_r, s.t, s.h, (long long)s.h * s.K_r, BK, p.BN / p.cg)) return cudaErrorInvalidValue;
-  } else
   // B = W[m] as [h rows (contraction)][K_r contiguous (N)]: N-major, boxes of 64 (N) x 64 (K)
   if (!make_map(&maps[1], W, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, 64, BK)) return cudaErrorInvalidValue;
+  maps[3] = maps[1];
+  if (n_pr > 0 && pv.alpha != 1.0f) {
+    if (!w_scaled) return cudaErrorInvalidValue;
+    if (!w_scaled_ready) {
+      LaunchScope scope(CAAT_K_TC_DGRAD, st);
+      const long long per_rank = (long long)n_pr * (s.K_r / 8);
+      int blocks = (int)((per_rank + 255) / 256);
+      if (blocks > 148 * 4) blocks = 148 * 4;
+      cudaError_t e = launch_pdl(scale_private_rows_kernel, dim3(blocks, s.t), dim3(256), 0, st, static_cast<const uint4*>(W),
+                                 static_cast<uint4*>(w_scaled), s.h, s.K_r, s.S, pv.alpha);
+      if (e != cudaSuccess) return e;
+    }
+    if (!make_map(&maps[3], w_scaled, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, 64, BK)) return cudaErrorInvalidValue;
+  }
   bool okA0 = n_sh > 0 ? make_map(&maps[0], gs, n_sh, s.T, 1, s.S_hi, (long long)s.T * s.S_hi, BK, BM) : true;
-  bool okA1 = n_pr > 0 ? make_map(&maps[2], zp, s.P, s.T, s.t, s.P, (long long)s.T * s.P, BK, BM) : true;
+  bool okA1 = n_pr > 0 ? make_map(&maps[2], pv.ptr, pv.ld, s.T, s.t, pv.ld, (long long)s.T * pv.ld, BK, BM) : true;
   if (!okA0 || !okA1) return cudaErrorInvalidValue;
   if (n_sh == 0) maps[0] = maps[2];
   if (n_pr == 0) maps[2] = maps[0];
-  maps[3] = maps[1];
-  p.a_mn = 0; p.b_mn = use_wt ? 0 : 1; p.out_f32 = 0; p.splits = 1;
+  p.a_mn = 0; p.b_mn = 1; p.out_f32 = 0; p.splits = 1;
   Region& r = p.r[0];
   int nu = 0;
   if (n_sh > 0) r.u[nu++] = Unit{0, 1, 0, 0, 0, 0, 0, 0, 1, 0, 1, (n_sh + BK - 1) / BK};
-  if (n_pr > 0) r.u[nu++] = Unit{2, 1, s.S - s.S_lo, 0, s.S, 0, 1, 0, 1, 0, 1, (n_pr + BK - 1) / BK};
+  if (n_pr > 0) r.u[nu++] = Unit{2, 3, pv.col0, 0, s.S, 0, 1, 0, 1, 0, 1, (n_pr + BK - 1) / BK};
   r.nunits = nu;
-  r.M = s.T; r.N = s.K_r; r.batch = s.t; r.b_slowest = 1;
+  r.M = s.T; r.N = s.K_r; r.batch = s.t; r.b_slowest = 1; r.scale = 1.0f;
   if (!make_cmap(&cmaps[0], dY, s.K_r, s.T, s.t, s.K_r, (long long)s.T * s.K_r, false)) return cudaErrorInvalidValue;
   cmaps[1] = cmaps[0];
   p.nregions = 1;
@@ -911,8 +914,8 @@ size_t tc_wgrad_splitk_bytes(const RowparShapes& s) {
   return splits > 1 ? (size_t)splits * s.t * s.h * s.K_r * sizeof(float) : 0;
 }
 
-// ---- wgrad: dW[m][:S] = gs^T Y[m] ; dW[m][S:] = zp[m]^T Y[m]      (fp32 out)
-cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* zp, const void* Y, float* dW,
+// ---- wgrad: dW[m][:S] = gs^T Y[m] ; dW[m][S:] = alpha gp[m]^T Y[m]      (fp32 out; alpha in the epilogue)
+cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const PrivOperand& pv, const void* Y, float* dW,
                             void* splitk, size_t splitk_bytes, cudaStream_t st) {
   CUtensorMap maps[4], cmaps[2];
   Params p{};
@@ -924,7 +927,7 @@ cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* z
   if (splits > 1 && splitk_bytes < (size_t)splits * dw_elems * sizeof(float)) return cudaErrorInvalidValue;
   // A = dZt as [T rows (contraction)][channels contiguous (M)]: M-major, boxes of 64 (M) x 64 (K)
   bool okA0 = n_sh > 0 ? make_map(&maps[0], gs, n_sh, s.T, 1, s.S_hi, (long long)s.T * s.S_hi, 64, BK) : true;
-  bool okA1 = n_pr > 0 ? make_map(&maps[2], zp, s.P, s.T, s.t, s.P, (long long)s.T * s.P, 64, BK) : true;
+  bool okA1 = n_pr > 0 ? make_map(&maps[2], pv.ptr, pv.ld, s.T, s.t, pv.ld, (long long)s.T * pv.ld, 64, BK) : true;
   // B = Y[m] as [T rows (contraction)][K_r contiguous (N)]: N-major
   if (!okA0 || !okA1 || !make_map(&maps[1], Y, s.K_r, s.T, s.t, s.K_r, (long long)s.T * s.K_r, 64, BK))
     return cudaErrorInvalidValue;
@@ -940,14 +943,16 @@ cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* z
     r.nunits = 1;
     r.u[0] = Unit{0, 1, 0, 0, 0, 0, 0, 0, 1, 0, 1, ksteps};
     r.M = n_sh; r.N = s.K_r; r.batch = s.t; r.b_slowest = 0;   // the shared gradient panel serves all ranks at once
+    r.scale = 1.0f;
     if (!make_cmap(&cmaps[g - 1], out, s.K_r, n_sh, (long long)s.t * splits, s.K_r, (long long)s.h * s.K_r, true))
       return cudaErrorInvalidValue;
   }
   if (n_pr > 0) {
     Region& r = p.r[g++];
     r.nunits = 1;
-    r.u[0] = Unit{2, 1, 0, s.S - s.S_lo, 0, 0, 1, 0, 1, 0, 1, ksteps};
+    r.u[0] = Unit{2, 1, 0, pv.col0, 0, 0, 1, 0, 1, 0, 1, ksteps};
     r.M = n_pr; r.N = s.K_r; r.batch = s.t; r.b_slowest = 1;
+    r.scale = pv.alpha;
     if (!make_cmap(&cmaps[g - 1], out + (long long)s.S * s.K_r, s.K_r, n_pr, (long long)s.t * splits, s.K_r,
                    (long long)s.h * s.K_r, true))
       return cudaErrorInvalidValue;

@@ -41,7 +41,7 @@ struct Scratch {
   size_t zs_off, zp_off;   // forward: Zt shared / private.  backward: dZt shared / private
   size_t dgpart_off, dbpart_off;  // backward: [rows, h] fp32 partial norm-parameter gradients
   size_t splitk_off, splitk_bytes;  // backward: split-K partials of the weight gradient
-  size_t wt_off;           // backward: transposed weights [t, K_r, h] (when the data gradient asks for them)
+  size_t wt_off;           // backward: the private rows of W times alpha, [t, h, K_r] (tensor-core path, alpha != 1)
   size_t zt_off;           // forward, few tokens: fp32 per-rank partials [t, T, h]
   size_t total;
 };
@@ -79,14 +79,18 @@ bool tc_gemm_usable(const caat_ctx* ctx, int K_r);
 // Zt -> (zs, zp):   zs[i,l] = sum_m sum_k Y[m,i,k] W[m,l,k] (l < S);  zp[m,i,l-S_lo] = sum_k ... (l >= S)
 cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* W, void* zs, void* zp,
                               cudaStream_t st);
-// dY[m] = [gs | zp[m]] W[m]
-// wt_scratch: optional [t, K_r, h] bf16 scratch; when given, W is transposed into it first and the
-// GEMM reads a K-major B operand
-cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const void* zp, const void* W, void* dY,
-                            void* wt_scratch, cudaStream_t st);
-bool tc_dgrad_wants_wt(int tokens);
-// dW[m] = [gs | zp[m]]^T Y[m]   (fp32 out)
-cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const void* zp, const void* Y, float* dW,
+// The private part of dZt as the backward GEMMs read it: element (m, i, l) for l >= S sits at
+// ptr[(m * T + i) * ld + col0 + (l - S)], and the gradient is alpha times the stored value.
+//   scratch copy written by the row kernel:   {zp, P, S - S_lo, 1}
+//   the residual gradient itself (per rank):  {dR, h, S, alpha}      (no scaled copy is written at all)
+//   compact stream:                           {dRp, P, 0, alpha}
+struct PrivOperand { const void* ptr; int ld; int col0; float alpha; };
+// dY[m] = [gs | alpha gp[m]] W[m];  w_scaled: [t, h, K_r] scratch for the alpha-scaled private rows of W
+// w_scaled_ready: the scaled rows are already in w_scaled (written by the row kernels' reduction launch)
+cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const PrivOperand& pv, const void* W, void* dY,
+                            void* w_scaled, bool w_scaled_ready, cudaStream_t st);
+// dW[m] = [gs | alpha gp[m]]^T Y[m]   (fp32 out)
+cudaError_t launch_tc_wgrad(const RowparShapes& s, const void* gs, const PrivOperand& pv, const void* Y, float* dW,
                             void* splitk, size_t splitk_bytes, cudaStream_t st);
 size_t tc_wgrad_splitk_bytes(const RowparShapes& s);
 // decode (few tokens): per-rank fp32 partials for all channels, zt[t, T, h]
@@ -136,7 +140,7 @@ bool rows_staged_usable(int h, int t, int S_lo, int S_hi, caat_dtype dtype, bool
 struct RowBwdArgs {
   const void *dX, *dHn, *Hn, *gamma;
   const float *rstd, *mean;
-  void *dR, *gs, *zp;
+  void *dR, *gs, *zp;      // zp may be NULL: the scaled private copy is then not written (the GEMMs read dR)
   float *dgpart, *dbpart;  // [rows, h]
   float *dgamma, *dbeta;   // [h]
   int t, T, h, S, S_lo, S_hi, P;
@@ -147,6 +151,11 @@ struct RowBwdArgs {
   int compact;
   const void *Hns, *dHns;
   int reduce_mode;   // CAAT_OPT_BACKWARD_REDUCE (plain-load kernels only)
+  // optional side job of the norm-gradient reduction launch: w_dst[m][l][:] = alpha * w_src[m][l][:] for the
+  // private rows l >= S of the layer's weights [t, h, w_Kr] (bf16), which the data gradient reads next
+  const void* w_src;
+  void* w_dst;
+  int w_Kr;
 };
 cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
 cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,

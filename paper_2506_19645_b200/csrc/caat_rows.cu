@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
               zp[e] = shared ? 0.f : a.alpha * g[e];
             }
           }
-          if (act[j]) stg<raw>(pZ[j], V_::pack(zp));
+          if (act[j] && a.zp) stg<raw>(pZ[j], V_::pack(zp));
         }
         pZ[j] += rank_p;
       }
@@ -461,10 +461,34 @@ __global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPar
 }
 
 // out[l] = sum over `rows` partial rows, fixed order: 32 row lanes then a serial combine.
+// Blocks past the first `nreduce` run an unrelated small job that has to happen between the row kernel and the
+// data gradient anyway and would otherwise cost a launch of its own: scaling the private rows of the weights.
+struct ScaleJob { const uint4* src; uint4* dst; int t, h, K_r, S; float alpha; };
+
 __global__ void __launch_bounds__(1024) reduce_partials_kernel(const float* __restrict__ part, float* __restrict__ out,
-                                                               int rows, int h) {
+                                                               int rows, int h, int nreduce, ScaleJob job) {
   __shared__ float sm[32][33];
   pdl_wait();
+  if ((int)blockIdx.x >= nreduce) {
+    const int row_chunks = job.K_r / 8;
+    const long long per_rank = (long long)(job.h - job.S) * row_chunks, total = per_rank * job.t;
+    const long long nthreads = (long long)(gridDim.x - nreduce) * 1024;
+    for (long long q = (long long)(blockIdx.x - nreduce) * 1024 + threadIdx.y * 32 + threadIdx.x; q < total; q += nthreads) {
+      const long long m = q / per_rank, r = q - m * per_rank;
+      const long long idx = (m * job.h + job.S) * row_chunks + r;
+      const uint4 v = job.src[idx];
+      const unsigned w[4] = {v.x, v.y, v.z, v.w};
+      unsigned o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 bb = __floats2bfloat162_rn(job.alpha * __uint_as_float(w[i] << 16),
+                                                  job.alpha * __uint_as_float(w[i] & 0xffff0000u));
+        o[i] = *reinterpret_cast<unsigned*>(&bb);
+      }
+      job.dst[idx] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    return;
+  }
   const int c = blockIdx.x * 32 + threadIdx.x;
   float s = 0.f;
   if (c < h)
@@ -570,15 +594,26 @@ cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int dire
     e = a.norm == 1 ? launch_bwd_t<float, true, false>(a, g, rows, st) : launch_bwd_t<float, false, false>(a, g, rows, st);
   if (e != cudaSuccess) return e;
   const dim3 rb(32, 32);
-  const dim3 rg((a.h + 31) / 32);
+  const int nreduce = (a.h + 31) / 32;
+  ScaleJob job{};
+  int nscale = 0;
+  if (a.w_dst && a.w_src && a.S < a.h) {
+    job = ScaleJob{static_cast<const uint4*>(a.w_src), static_cast<uint4*>(a.w_dst), a.t, a.h, a.w_Kr, a.S, a.alpha};
+    const long long total = (long long)a.t * (a.h - a.S) * (a.w_Kr / 8);
+    nscale = (int)((total + 4 * 1024 - 1) / (4 * 1024));          // four 16-byte chunks per thread
+    if (nscale > 148) nscale = 148;
+    if (nscale < 1) nscale = 1;
+  }
   {
     LaunchScope scope(CAAT_K_NORMGRAD_REDUCE, st);
-    e = launch_pdl(reduce_partials_kernel, rg, rb, 0, st, (const float*)a.dgpart, a.dgamma, rows, a.h);
+    e = launch_pdl(reduce_partials_kernel, dim3(nreduce + nscale), rb, 0, st, (const float*)a.dgpart, a.dgamma, rows, a.h,
+                   nreduce, job);
     if (e != cudaSuccess) return e;
   }
   if (a.norm == 1 && a.dbeta && a.dbpart) {
     LaunchScope scope(CAAT_K_NORMGRAD_REDUCE, st);
-    e = launch_pdl(reduce_partials_kernel, rg, rb, 0, st, (const float*)a.dbpart, a.dbeta, rows, a.h);
+    e = launch_pdl(reduce_partials_kernel, dim3(nreduce), rb, 0, st, (const float*)a.dbpart, a.dbeta, rows, a.h, nreduce,
+                   ScaleJob{});
     if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();

@@ -563,7 +563,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
               zp[q].y = sy ? 0.f : a.alpha * gg[q].y;
             }
           }
-          if (act[j]) stg<raw>(static_cast<char*>(a.zp) + qZ[j], pack2(zp));
+          if (act[j] && a.zp) stg<raw>(static_cast<char*>(a.zp) + qZ[j], pack2(zp));
         }
         qZ[j] += rank_p;
       }

@@ -496,7 +496,7 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
                 zp[q].y = sy ? 0.f : a.alpha * gg[q].y;
               }
             }
-            stg<raw>(pZ + (long long)col[j] * ES, pack2(zp));
+            if (a.zp) stg<raw>(pZ + (long long)col[j] * ES, pack2(zp));
           }
         }
         __syncwarp();
