@@ -832,32 +832,9 @@ cudaError_t launch_tc_forward_decode(int t, int T, int h, const DecodeProblem* p
   return launch(maps, cmaps, p, CAAT_K_TC_FORWARD, st);
 }
 
-// out[b][l][:] = alpha * W[b][l][:] for the private rows l in [S, h) of every rank's weight shard (bf16,
-// 16 bytes per thread).  The data gradient then takes the private gradient g as stored in dR instead of
-// a scaled copy of it: sum_l (alpha g[l]) W[l][k] = sum_l g[l] (alpha W[l][k]); the weights are the
-// small operand.
-__global__ void __launch_bounds__(256) scale_private_rows_kernel(const uint4* __restrict__ W, uint4* __restrict__ out,
-                                                                 int h, int K_r, int S, float alpha) {
-  pdl_wait();
-  const int row_chunks = K_r / 8;
-  const long long per_rank = (long long)(h - S) * row_chunks;
-  const long long base = ((long long)blockIdx.y * h + S) * row_chunks;
-  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < per_rank; q += (long long)gridDim.x * blockDim.x) {
-    const uint4 v = W[base + q];
-    const unsigned w[4] = {v.x, v.y, v.z, v.w};
-    unsigned o[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      __nv_bfloat162 bb = __floats2bfloat162_rn(alpha * __uint_as_float(w[i] << 16), alpha * __uint_as_float(w[i] & 0xffff0000u));
-      o[i] = *reinterpret_cast<unsigned*>(&bb);
-    }
-    out[base + q] = make_uint4(o[0], o[1], o[2], o[3]);
-  }
-}
-
 // ---- dgrad: dY[m] = gs W[m][:S] + (alpha gp[m]) W[m][S:]
 // pv describes where the private gradient lives and what still multiplies it (see PrivOperand); when
-// pv.alpha != 1 the private rows of W are scaled into w_scaled ([t, h, K_r], only rows >= S are written).
+// pv.alpha != 1, w_scaled ([t, h, K_r], only rows >= S are used) must hold alpha times the private rows of W.
 cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const PrivOperand& pv, const void* W, void* dY,
                             void* w_scaled, bool w_scaled_ready, cudaStream_t st) {
   CUtensorMap maps[4], cmaps[2];
@@ -872,16 +849,9 @@ cudaError_t launch_tc_dgrad(const RowparShapes& s, const void* gs, const PrivOpe
   if (!make_map(&maps[1], W, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, 64, BK)) return cudaErrorInvalidValue;
   maps[3] = maps[1];
   if (n_pr > 0 && pv.alpha != 1.0f) {
-    if (!w_scaled) return cudaErrorInvalidValue;
-    if (!w_scaled_ready) {
-      LaunchScope scope(CAAT_K_TC_DGRAD, st);
-      const long long per_rank = (long long)n_pr * (s.K_r / 8);
-      int blocks = (int)((per_rank + 255) / 256);
-      if (blocks > 148 * 4) blocks = 148 * 4;
-      cudaError_t e = launch_pdl(scale_private_rows_kernel, dim3(blocks, s.t), dim3(256), 0, st, static_cast<const uint4*>(W),
-                                 static_cast<uint4*>(w_scaled), s.h, s.K_r, s.S, pv.alpha);
-      if (e != cudaSuccess) return e;
-    }
+    // sum_l (alpha g[l]) W[l][k] = sum_l g[l] (alpha W[l][k]): the private gradient is read as stored in dR,
+    // the weights' private rows (the small operand) carry alpha; they were scaled by the launch before this one
+    if (!w_scaled || !w_scaled_ready) return cudaErrorInvalidValue;
     if (!make_map(&maps[3], w_scaled, s.K_r, s.h, s.t, s.K_r, (long long)s.h * s.K_r, 64, BK)) return cudaErrorInvalidValue;
   }
   bool okA0 = n_sh > 0 ? make_map(&maps[0], gs, n_sh, s.T, 1, s.S_hi, (long long)s.T * s.S_hi, BK, BM) : true;
