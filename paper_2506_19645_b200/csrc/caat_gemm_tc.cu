@@ -78,7 +78,9 @@ struct Params {
   int tiles_total;
   unsigned int* status;
   int debug;             // measurement aid (env CAAT_TC_DEBUG; results are then wrong): 1 = no operand loads,
-                         // 2 = no output stores, 4 = no A loads, 8 = no B loads
+                         // 2 = no epilogue work at all, 4 = no A loads, 8 = no B loads; epilogue stops after the
+                         // tensor-memory load (32) / after the staging stores (16); 64 = no slab barrier,
+                         // 128 = no TMA store
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -497,6 +499,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         }
         const uint32_t buf = smem_u32(cstage + (size_t)(slab % 3) * kCBuf);
         const uint32_t rowaddr = buf + (uint32_t)rr * 64u;
+        if (p.debug & 32) { ++slab; continue; }
         if (p.out_f32) {
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
@@ -513,9 +516,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
             sts128(rowaddr + (((uint32_t)q4 ^ sw) << 4), w[0], w[1], w[2], w[3]);
           }
         }
+        if (p.debug & 16) { ++slab; continue; }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        epi_barrier();
-        if (warp == 2 && lane == 0) {
+        if (!(p.debug & 64)) epi_barrier();
+        if (warp == 2 && lane == 0 && !(p.debug & 128)) {
           tma_store_3d(cmaps[c.region], n0 + cc, m0, zc, buf);
           bulk_commit();
           bulk_wait_read1();     // the store before this one has finished reading its buffer
