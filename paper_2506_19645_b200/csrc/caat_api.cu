@@ -76,7 +76,8 @@ Scratch scratch_layout(const caat_ctx* ctx, int K_r, int tokens, int backward) {
   s.zs_off = off;
   off = align_up(off + (size_t)tokens * s.S_hi * e, 256);
   s.zp_off = off;
-  off = align_up(off + (size_t)ctx->t * tokens * s.P * e, 256);
+  if (!(backward && tc_gemm_usable(ctx, K_r)))   // the tensor-core backward reads the private gradient from dR
+    off = align_up(off + (size_t)ctx->t * tokens * s.P * e, 256);
   s.zt_off = off;
   if (!backward && tokens <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r))   // two layers' planes
     off = align_up(off + 2 * decode_planes_bytes(ctx, tokens), 256);
