@@ -103,9 +103,11 @@ int caat_shared_channels(const caat_ctx *ctx);
 /* alpha currently in effect. */
 double caat_private_scale(const caat_ctx *ctx);
 
-/* Bytes of device scratch the forward (backward = 0) or backward (backward = 1)
- * call of `layer` needs for `tokens` tokens.  For the block calls pass the larger
- * of the two layers' figures (CAAT_MLP_DOWN's, when ffn >= h). 0 on bad arguments. */
+/* Bytes of device scratch for `tokens` tokens of `layer`: backward = 0, what the forward
+ * call needs; backward = 1, enough for the forward AND the backward call (a training step
+ * runs both on one buffer; neither keeps anything in it between calls).  For the block
+ * calls pass the larger of the two layers' figures (CAAT_MLP_DOWN's, when ffn >= h).
+ * 0 on bad arguments. */
 size_t caat_workspace_bytes(const caat_ctx *ctx, caat_layer layer, int tokens, int backward);
 
 const char *caat_strerror(caat_status s);

@@ -314,7 +314,10 @@ double caat_private_scale(const caat_ctx* ctx) { return ctx ? ctx->alpha : 0.0; 
 
 size_t caat_workspace_bytes(const caat_ctx* ctx, caat_layer layer, int tokens, int backward) {
   if (check_common(ctx, layer, tokens) != CAAT_OK) return 0;
-  return scratch_layout(ctx, layer_kr(ctx, layer), tokens, backward ? 1 : 0).total;
+  const size_t fwd = scratch_layout(ctx, layer_kr(ctx, layer), tokens, 0).total;
+  if (!backward) return fwd;
+  const size_t bwd = scratch_layout(ctx, layer_kr(ctx, layer), tokens, 1).total;
+  return bwd > fwd ? bwd : fwd;   // a training step runs both calls on one buffer
 }
 
 const char* caat_strerror(caat_status s) {
