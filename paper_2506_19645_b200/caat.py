@@ -122,7 +122,8 @@ class Context:
         _check(lib.caat_create(h, ffn, t, float(p), self.dtype_code, byref(self._h)), "caat_create")
 
     def __del__(self):
-        if getattr(self, "_h", None) is not None and self._h.value:
+        # at interpreter shutdown the module globals may already be gone
+        if getattr(self, "_h", None) is not None and self._h.value and lib is not None:
             lib.caat_destroy(self._h)
             self._h = c_void_p()
 
