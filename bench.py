@@ -492,6 +492,24 @@ def run_cuda(args):
     ms_step = ms / args.steps
     value = replicas.whole_job_rate(w.tokens, args.steps, world, ms)
 
+    # end-to-end leg: every rank runs it at the same time (each GPU has its own host link); the job's figure is
+    # all replicas' tokens over the slowest rank's time
+    e2e = None
+    try:
+        if args.no_e2e:
+            raise RuntimeError("skipped (--no-e2e)")
+        if dist_on:
+            torch.distributed.barrier()
+        ems, h2d, d2h = e2e_leg(runner, max(4, min(args.steps, 8)))
+        ems = replicas.max_over_ranks(ems, dev)
+        e2e = {"value": world * w.tokens / (ems * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d * world,
+               "d2h_bytes_per_step": d2h * world, "ms_per_step": ems,
+               "overlap": "copy-in, kernels and read-back of consecutive steps on three streams, two buffer sets"}
+    except Exception as ex:  # pinned-memory exhaustion on a small host
+        if dist_on:
+            replicas.max_over_ranks(0.0, dev)     # keep the ranks' collectives matched
+        e2e = {"value": None, "unit": "tokens/s", "error": str(ex)[:200]}
+
     result = None
     if rank == 0:
         peaks = measured_peaks()
@@ -520,16 +538,6 @@ def run_cuda(args):
                               f"({ms_prof / args.steps:.4f} ms/step with events)"})
         fl, by = paper_level_work(w, compact)
         t_roof = max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9))
-        e2e = None
-        try:
-            if args.no_e2e:
-                raise RuntimeError("skipped (--no-e2e)")
-            ems, h2d, d2h = e2e_leg(runner, max(4, min(args.steps, 8)))
-            e2e = {"value": w.tokens / (ems * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-                   "d2h_bytes_per_step": d2h, "ms_per_step": ems,
-                   "overlap": "copy-in, kernels and read-back of consecutive steps on three streams, two buffer sets"}
-        except Exception as ex:  # pinned-memory exhaustion on a small host
-            e2e = {"value": None, "unit": "tokens/s", "error": str(ex)[:200]}
         ar = runner.ctx.allreduce_bytes(w.tokens, 2)
         result = {
             "metric": metric_name(w), "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
