@@ -181,8 +181,8 @@ def paper_level_work(w, compact=False):
 
 
 def r_w_compact_ok(w):
-    """The compact-layout entry points need a partition on a 16-byte boundary and more than a few tokens."""
-    return w.S % 8 == 0 and w.tokens > 64
+    """The compact-layout entry points need a partition on a 16-byte boundary."""
+    return w.S % 8 == 0
 
 
 # --------------------------------------------------------------------------- the CUDA arm

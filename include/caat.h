@@ -250,7 +250,9 @@ caat_status caat_block_backward(const caat_ctx *ctx, int tokens,
  * residual gradient at once.  dHns and dHnp are both given or both NULL.
  *
  * Requires S % 8 == 0 (CAAT_EUNSUPPORTED otherwise).  A part that is empty (S = 0 or S = h)
- * may be passed as NULL.  Workspace sizes are those of the per-rank entry points.
+ * may be passed as NULL.  Workspace sizes are those of the per-rank entry points.  Forward
+ * calls with at most 64 tokens stream the weights with swapped GEMM operands here too
+ * (CAAT_OPT_DECODE); this is the single-device serving arrangement of Section 3.2.
  */
 caat_status caat_rowpar_forward_compact(const caat_ctx *ctx, caat_layer layer, int tokens,
                                         const void *Y, const void *W,

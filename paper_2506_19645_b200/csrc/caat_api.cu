@@ -133,7 +133,7 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
   const size_t e = elem_size(ctx->dtype);
   cudaError_t ce;
 
-  if (!compact && T <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r)) {
+  if (T <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r)) {
     // few tokens (decode): the weights dominate the traffic; stream them with swapped operands and
     // let the row kernel form the rank sum from fp32 per-rank partials
     float* zt = reinterpret_cast<float*>(wsb + L.zt_off);
@@ -142,8 +142,8 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
     ce = launch_tc_forward_decode(t, T, h, &pr, 1, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
     RowPartArgs a{};
-    a.L[0] = PartialLayer{zt, splits, gamma, beta, Hn, X, rstd, mean};
-    a.nlayers = 1; a.R = R; a.t = t; a.T = T; a.h = h; a.S = S;
+    a.L[0] = PartialLayer{zt, splits, gamma, beta, Hn, X, rstd, mean, Hns};
+    a.nlayers = 1; a.R = R; a.t = t; a.T = T; a.h = h; a.S = S; a.compact = compact; a.Rs = Rs;
     a.alpha = (float)ctx->alpha; a.eps = (float)ctx->eps; a.norm = ctx->norm;
     ce = launch_rows_forward_partials(a, ctx->dtype, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
@@ -249,6 +249,57 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
     ce = launch_gemm_simt(g, ctx->dtype, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
   }
+  return CAAT_OK;
+}
+
+// ---- block forward with few tokens (decode) --------------------------------------
+// The two layers' GEMMs do not depend on each other, so both weight streams run in ONE launch, and one
+// row kernel walks both layers of a (token, rank) row.  compact: R0 / Hn1 / Hn2 are the private parts
+// [t, T, h - S] and R0s / Hn1s / Hn2s the shared part [T, S] of the stream.
+static bool block_decode_applies(const caat_ctx* ctx, int tokens) {
+  return ctx && tokens >= 1 && tokens <= kDecodeMaxTokens && !ctx->no_decode &&
+         tc_gemm_usable(ctx, ctx->h / ctx->t) && tc_gemm_usable(ctx, ctx->ffn / ctx->t);
+}
+
+static caat_status block_decode(const caat_ctx* ctx, int tokens, const void* Y_attn, const void* W_o, const void* Y_mlp,
+                                const void* W_down, const void* R0, const void* gamma1, const void* beta1,
+                                const void* gamma2, const void* beta2, void* Hn1, void* X1, float* rstd1, float* mean1,
+                                void* Hn2, void* X2, float* rstd2, float* mean2, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream, int compact, const void* R0s, void* Hn1s, void* Hn2s) {
+  caat_status s = check_common(ctx, CAAT_MLP_DOWN, tokens);
+  if (s != CAAT_OK) return s;
+  const bool has_s = ctx->S > 0, has_p = ctx->S < ctx->h;
+  if (!Y_attn || !W_o || !Y_mlp || !W_down || !gamma1 || !gamma2 || !X1 || !rstd1 || !X2 || !rstd2) return CAAT_EINVAL;
+  if (compact) {
+    if (ctx->S % kLayoutVec != 0) return CAAT_EUNSUPPORTED;
+    if ((has_s && (!R0s || !Hn1s || !Hn2s)) || (has_p && (!R0 || !Hn1 || !Hn2))) return CAAT_EINVAL;
+  } else if (!R0 || !Hn1 || !Hn2) {
+    return CAAT_EINVAL;
+  }
+  if (ctx->norm == 1 && (!mean1 || !mean2)) return CAAT_EINVAL;
+  const void* ptrs[] = {Y_attn, W_o, Y_mlp, W_down, R0, R0s, gamma1, beta1, gamma2, beta2, Hn1, Hn1s, X1, rstd1, mean1,
+                        Hn2, Hn2s, X2, rstd2, mean2, workspace};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  const int ka = ctx->h / ctx->t, km = ctx->ffn / ctx->t;
+  const Scratch L = scratch_layout(ctx, km, tokens, 0);
+  if (!workspace || workspace_bytes < L.total) return CAAT_EWORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  float* zt1 = reinterpret_cast<float*>(static_cast<char*>(workspace) + L.zt_off);
+  float* zt2 = reinterpret_cast<float*>(static_cast<char*>(workspace) + L.zt_off + decode_planes_bytes(ctx, tokens));
+  const int kmin = ka < km ? ka : km;
+  const int sp1 = tc_decode_splits(ka, kmin, tokens), sp2 = tc_decode_splits(km, kmin, tokens);
+  const DecodeProblem pr[2] = {{ka, Y_attn, W_o, zt1, sp1}, {km, Y_mlp, W_down, zt2, sp2}};
+  cudaError_t ce = launch_tc_forward_decode(ctx->t, tokens, ctx->h, pr, 2, st);
+  if (ce != cudaSuccess) return cuda_fail(ce);
+  RowPartArgs a{};
+  a.L[0] = PartialLayer{zt1, sp1, gamma1, beta1, Hn1, X1, rstd1, mean1, Hn1s};
+  a.L[1] = PartialLayer{zt2, sp2, gamma2, beta2, Hn2, X2, rstd2, mean2, Hn2s};
+  a.nlayers = 2; a.R = R0; a.t = ctx->t; a.T = tokens; a.h = ctx->h; a.S = ctx->S;
+  a.alpha = (float)ctx->alpha; a.eps = (float)ctx->eps; a.norm = ctx->norm;
+  a.compact = compact; a.Rs = R0s;
+  ce = launch_rows_forward_partials(a, ctx->dtype, st);
+  if (ce != cudaSuccess) return cuda_fail(ce);
   return CAAT_OK;
 }
 
@@ -376,39 +427,9 @@ caat_status caat_block_forward(const caat_ctx* ctx, int tokens, const void* Y_at
                                float* rstd1, float* mean1, void* Hn2, void* X2, float* rstd2, float* mean2,
                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
   // Two reduces per block (Appendix C): attention-out, then MLP-down on the new residual stream.
-  if (ctx && tokens >= 1 && tokens <= kDecodeMaxTokens && !ctx->no_decode &&
-      tc_gemm_usable(ctx, ctx->h / ctx->t) && tc_gemm_usable(ctx, ctx->ffn / ctx->t)) {
-    // few tokens: the two layers' GEMMs do not depend on each other, so both weight streams run in
-    // ONE launch, and one row kernel walks both layers of a (token, rank) row
-    caat_status s = check_common(ctx, CAAT_MLP_DOWN, tokens);
-    if (s != CAAT_OK) return s;
-    if (!Y_attn || !W_o || !Y_mlp || !W_down || !R0 || !gamma1 || !gamma2 || !Hn1 || !X1 || !rstd1 || !Hn2 || !X2 || !rstd2)
-      return CAAT_EINVAL;
-    if (ctx->norm == 1 && (!mean1 || !mean2)) return CAAT_EINVAL;
-    const void* ptrs[] = {Y_attn, W_o, Y_mlp, W_down, R0, gamma1, beta1, gamma2, beta2, Hn1, X1, rstd1, mean1,
-                          Hn2, X2, rstd2, mean2, workspace};
-    for (const void* p : ptrs)
-      if (p && !aligned16(p)) return CAAT_EALIGN;
-    const int ka = ctx->h / ctx->t, km = ctx->ffn / ctx->t;
-    const Scratch L = scratch_layout(ctx, km, tokens, 0);
-    if (!workspace || workspace_bytes < L.total) return CAAT_EWORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    float* zt1 = reinterpret_cast<float*>(static_cast<char*>(workspace) + L.zt_off);
-    float* zt2 = reinterpret_cast<float*>(static_cast<char*>(workspace) + L.zt_off + decode_planes_bytes(ctx, tokens));
-    const int kmin = ka < km ? ka : km;
-    const int sp1 = tc_decode_splits(ka, kmin, tokens), sp2 = tc_decode_splits(km, kmin, tokens);
-    const DecodeProblem pr[2] = {{ka, Y_attn, W_o, zt1, sp1}, {km, Y_mlp, W_down, zt2, sp2}};
-    cudaError_t ce = launch_tc_forward_decode(ctx->t, tokens, ctx->h, pr, 2, st);
-    if (ce != cudaSuccess) return cuda_fail(ce);
-    RowPartArgs a{};
-    a.L[0] = PartialLayer{zt1, sp1, gamma1, beta1, Hn1, X1, rstd1, mean1};
-    a.L[1] = PartialLayer{zt2, sp2, gamma2, beta2, Hn2, X2, rstd2, mean2};
-    a.nlayers = 2; a.R = R0; a.t = ctx->t; a.T = tokens; a.h = ctx->h; a.S = ctx->S;
-    a.alpha = (float)ctx->alpha; a.eps = (float)ctx->eps; a.norm = ctx->norm;
-    ce = launch_rows_forward_partials(a, ctx->dtype, st);
-    if (ce != cudaSuccess) return cuda_fail(ce);
-    return CAAT_OK;
-  }
+  if (block_decode_applies(ctx, tokens))
+    return block_decode(ctx, tokens, Y_attn, W_o, Y_mlp, W_down, R0, gamma1, beta1, gamma2, beta2, Hn1, X1, rstd1, mean1,
+                        Hn2, X2, rstd2, mean2, workspace, workspace_bytes, cuda_stream, 0, nullptr, nullptr, nullptr);
   caat_status s = caat_rowpar_forward(ctx, CAAT_ATTN_OUT, tokens, Y_attn, W_o, R0, gamma1, beta1, Hn1, X1, rstd1,
                                       mean1, workspace, workspace_bytes, cuda_stream);
   if (s != CAAT_OK) return s;
@@ -491,6 +512,9 @@ caat_status caat_block_forward_compact(const caat_ctx* ctx, int tokens, const vo
                                        void* Hn1s, void* Hn1p, void* X1, float* rstd1, float* mean1, void* Hn2s,
                                        void* Hn2p, void* X2, float* rstd2, float* mean2, void* workspace,
                                        size_t workspace_bytes, void* cuda_stream) {
+  if (block_decode_applies(ctx, tokens))
+    return block_decode(ctx, tokens, Y_attn, W_o, Y_mlp, W_down, R0p, gamma1, beta1, gamma2, beta2, Hn1p, X1, rstd1, mean1,
+                        Hn2p, X2, rstd2, mean2, workspace, workspace_bytes, cuda_stream, 1, R0s, Hn1s, Hn2s);
   caat_status s = caat_rowpar_forward_compact(ctx, CAAT_ATTN_OUT, tokens, Y_attn, W_o, R0s, R0p, gamma1, beta1, Hn1s,
                                               Hn1p, X1, rstd1, mean1, workspace, workspace_bytes, cuda_stream);
   if (s != CAAT_OK) return s;

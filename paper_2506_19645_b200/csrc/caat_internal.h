@@ -122,7 +122,10 @@ cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direc
 cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st);
 // forward row work from fp32 partial planes (decode); with two layers the second layer's residual is
 // the first layer's new residual stream (as stored), both layers in one launch
-struct PartialLayer { const float* zt; int splits; const void* gamma; const void* beta; void* Hn; void* X; float* rstd; float* mean; };
+struct PartialLayer {
+  const float* zt; int splits; const void* gamma; const void* beta; void* Hn; void* X; float* rstd; float* mean;
+  void* Hns;   // compact layout: the shared part of this layer's new stream, [T, S]; Hn then holds the private parts
+};
 struct RowPartArgs {
   PartialLayer L[2];
   int nlayers;
@@ -130,6 +133,8 @@ struct RowPartArgs {
   int t, T, h, S;
   float alpha, eps;
   int norm;
+  int compact;      // R / Hn are [t, T, h - S] private parts, Rs / Hns [T, S] the shared part stored once
+  const void* Rs;
 };
 cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype, cudaStream_t st);
 // warp-per-token kernels for short rows (h <= 1024 in bf16); rows_warp_cpt == 0: not applicable

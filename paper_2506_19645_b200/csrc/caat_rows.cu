@@ -399,8 +399,12 @@ __global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPar
     float st[1] = {0.f};
     for (int c = threadIdx.x * V; c < a.h; c += blockDim.x * V) {
       float r[V], z[V], hn[V];
+      const bool shared_chunk = c + V <= a.S;          // the partition is a multiple of 8 on this path
+      // compact layout: where this chunk of the stream lives (shared part once, private part per rank)
+      const long long coff = shared_chunk ? ((long long)i * a.S + c) * ES : (row * (a.h - a.S) + (c - a.S)) * ES;
       if (layer == 0) {
-        V_::unpack(ldg<raw>(static_cast<const char*>(a.R) + (row * a.h + c) * ES), r);
+        if (a.compact) V_::unpack(ldg<raw>(static_cast<const char*>(shared_chunk ? a.Rs : a.R) + coff), r);
+        else V_::unpack(ldg<raw>(static_cast<const char*>(a.R) + (row * a.h + c) * ES), r);
       } else {
 #pragma unroll
         for (int e = 0; e < V; ++e) r[e] = V_::round(hrow[c + e]);
@@ -408,7 +412,6 @@ __global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPar
 #pragma unroll
       for (int e = 0; e < V; ++e) z[e] = 0.f;
       const float* base = L.zt + (long long)i * a.h + c;
-      const bool shared_chunk = c + V <= a.S;          // the partition is a multiple of 8 on this path
       const int z0 = shared_chunk ? 0 : m, zstep = shared_chunk ? 1 : a.t;
       const int nz = shared_chunk ? nplanes : L.splits;
 #pragma unroll 8
@@ -428,7 +431,11 @@ __global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPar
       if (layer > 0) __syncwarp();
 #pragma unroll
       for (int e = 0; e < V; ++e) hrow[c + e] = hn[e];
-      stg<raw>(static_cast<char*>(L.Hn) + (row * a.h + c) * ES, V_::pack(hn));
+      if (a.compact) {      // every rank's CTA forms the same shared values; rank 0's writes them
+        if (!shared_chunk || m == 0) stg<raw>(static_cast<char*>(shared_chunk ? L.Hns : L.Hn) + coff, V_::pack(hn));
+      } else {
+        stg<raw>(static_cast<char*>(L.Hn) + (row * a.h + c) * ES, V_::pack(hn));
+      }
     }
     row_reduce_sync<1>(st, red, par);
     float mu = 0.f, rs;

@@ -179,3 +179,32 @@ def test_compact_block_matches_oracle():
     # the difference is one storage rounding, inside the tolerance
     for k in bo:
         assert_close(bo[k].cpu(), ob[k], "bf16", k)
+
+
+@pytest.mark.parametrize("no_decode", [False, True])
+@pytest.mark.parametrize("T,t,h,ffn,S", [(1, 8, 4096, 11008, 2048), (8, 8, 4096, 11008, 4096), (64, 8, 4096, 11008, 2048),
+                                         (33, 4, 768, 3072, 384), (64, 2, 256, 1024, 0)])
+def test_compact_block_few_tokens(no_decode, T, t, h, ffn, S):
+    # few tokens: both layers' weights stream through one swapped-operand GEMM and one row kernel walks both layers of
+    # a row, here on the compact stream; the large-batch path (no_decode) must give the same block
+    w = synthetic.Workload("compact_decode_case", t, T, h, ffn, S / h, "bf16", "block", False, 7 + T)
+    d = synthetic.block_inputs(w)
+    ctx = G.make_ctx(t, h, ffn, "bf16", S=S, no_decode=no_decode)
+    td, f32, alpha = torch.bfloat16, torch.float32, ctx.private_scale
+    R0s, R0p = _split(d["R0"], S)
+    fo = O.block_forward_compact(f64(d["Y_attn"]), f64(d["W_o"]), f64(d["Y_mlp"]), f64(d["W_down"]), f64(R0s), f64(R0p),
+                                 f64(d["gamma1"]), f64(d["gamma2"]), S=S, alpha=alpha)
+    out = {"Hn1s": G.Guarded((T, S), td), "Hn1p": G.Guarded((t, T, h - S), td), "X1": G.Guarded((t, T, h), td),
+           "rstd1": G.Guarded((t, T), f32), "Hn2s": G.Guarded((T, S), td), "Hn2p": G.Guarded((t, T, h - S), td),
+           "X2": G.Guarded((t, T, h), td), "rstd2": G.Guarded((t, T), f32)}
+    ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, False))
+    c = {k: v.cuda() for k, v in d.items()}
+    ctx.block_forward_compact(T, c["Y_attn"], c["W_o"], c["Y_mlp"], c["W_down"], R0s.cuda(), R0p.cuda(), c["gamma1"], None,
+                              c["gamma2"], None, out["Hn1s"].view, out["Hn1p"].view, out["X1"].view, out["rstd1"].view, None,
+                              out["Hn2s"].view, out["Hn2p"].view, out["X2"].view, out["rstd2"].view, None, ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+    for k, g in out.items():
+        g.check(k)
+        if fo[k].size:
+            assert_close(g.view.cpu(), fo[k], "bf16", k)
