@@ -94,20 +94,10 @@ __global__ void __launch_bounds__(256) act_backward_kernel(const void* __restric
   }
 }
 
-int sm_count_() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
-
 int act_grid(long long rows, int width_out, int V) {
   const long long total = rows * (width_out / V);
   long long blocks = (total + 255) / 256;
-  const long long cap = (long long)sm_count_() * 8;     // eight resident CTAs of 256 threads per SM
+  const long long cap = (long long)sm_count() * 8;     // eight resident CTAs of 256 threads per SM
   if (blocks > cap) blocks = cap;
   return (int)(blocks < 1 ? 1 : blocks);
 }

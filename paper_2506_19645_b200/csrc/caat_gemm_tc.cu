@@ -676,16 +676,6 @@ TileCfg pick_tile(const RegionShape* r, int nr, bool b_n_major, int max_splits, 
   return best;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
-
 cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params& p, int kind, cudaStream_t st) {
   const int stage_bytes = BM * BK * 2 + (p.BN / p.cg) * BK * 2;
   int nst = (227 * 1024 - 2048 - 3 * kCBuf) / stage_bytes;
@@ -693,12 +683,14 @@ cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params
   if (nst < 2) return cudaErrorInvalidConfiguration;
   p.nstages = nst;
   const size_t smem = (size_t)nst * stage_bytes + 3 * kCBuf + 1024 /*alignment slack*/ + (2 * nst + 4) * 8 + 16;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[64] = {};      // the attribute belongs to the device's copy of the kernel: once per device
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!attr_set[dev]) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   p.status = device_status_word();
   if (!p.status) return cudaErrorUnknown;

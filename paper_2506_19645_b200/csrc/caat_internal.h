@@ -214,5 +214,6 @@ struct LaunchScope {
   cudaStream_t st;
 };
 unsigned int* device_status_word();  // device address of the status word (per device)
+int sm_count();                       // multiprocessors of the current device (grids are sized in multiples of it)
 
 }  // namespace caat

@@ -576,16 +576,6 @@ WarpGeom warp_geometry(int h, int P, int S_hi, int ES, bool backward, bool has_c
   return g;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
-
 constexpr size_t kSmemPerSm = 227 * 1024;
 constexpr int kCtasPerSm = 3;
 
