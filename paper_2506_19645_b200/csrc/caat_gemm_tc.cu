@@ -399,6 +399,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
+      // Descriptors differ from stage to stage and from MMA to MMA only in their 14-bit address field:
+      // the constant part is built once and the loop adds 16-byte units to the low word.  The issuing
+      // thread's instruction count per k-step is what bounds short contractions.
+      const uint64_t a_const = p.a_mn ? make_desc(0, 64 * BK * 2, 1024) : make_desc(0, 16, 1024);
+      const uint64_t b_const = p.b_mn ? make_desc(0, 64 * BK * 2, 1024) : make_desc(0, 16, 1024);
+      const uint32_t a_hi = (uint32_t)(a_const >> 32), b_hi = (uint32_t)(b_const >> 32);
+      const uint32_t a_k16 = (p.a_mn ? UMMA_K * 128 : UMMA_K * 2) >> 4, b_k16 = (p.b_mn ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+      const uint32_t stage16 = stage_bytes >> 4;
+      const uint32_t a_lo0 = (uint32_t)a_const + (tiles_sa >> 4), b_lo0 = (uint32_t)b_const + ((tiles_sa + a_bytes) >> 4);
+      uint32_t a_lo = a_lo0, b_lo = b_lo0;
+      uint32_t full_bar = full0, empty_bar = empty0;
       for (int tile = worker; tile < p.tiles_total && ok; tile += nworkers) {
         const TileCoord c = decode_tile(p, tile);
         const Region& r = p.r[c.region];
@@ -413,22 +424,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           split_range(r.splits, u, c.split, kb, ke);
           for (int q = 0; q < u.Q && ok; ++q) {
             for (int kk = kb; kk < ke; ++kk) {
-              if (!mbar_wait(full0 + 8u * stage, phase, abort_flag)) { ok = false; break; }
+              if (!mbar_wait(full_bar, phase, abort_flag)) { ok = false; break; }
               tc_fence_after();
-              const uint32_t sa = tiles_sa + (uint32_t)stage * stage_bytes, sb = sa + a_bytes;
 #pragma unroll
               for (int k = 0; k < BK / UMMA_K; ++k) {
-                const uint64_t ad = p.a_mn ? make_desc(sa + k * (UMMA_K * 128), 64 * BK * 2, 1024)
-                                           : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
-                const uint64_t bd = p.b_mn ? make_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024)
-                                           : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
+                const uint64_t ad = ((uint64_t)a_hi << 32) | (a_lo + (uint32_t)k * a_k16);
+                const uint64_t bd = ((uint64_t)b_hi << 32) | (b_lo + (uint32_t)k * b_k16);
                 if (CG == 2) umma_bf16_pair(d_tmem, ad, bd, idesc, accumulate);
                 else umma_bf16(d_tmem, ad, bd, idesc, accumulate);
                 accumulate = 1;
               }
               // frees the stage (in both CTAs) once these MMAs have read it
-              if (CG == 2) umma_commit_pair(empty0 + 8u * stage); else umma_commit(empty0 + 8u * stage);
-              if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+              if (CG == 2) umma_commit_pair(empty_bar); else umma_commit(empty_bar);
+              a_lo += stage16; b_lo += stage16; full_bar += 8u; empty_bar += 8u;
+              if (++stage == p.nstages) {
+                stage = 0; phase ^= 1u;
+                a_lo = a_lo0; b_lo = b_lo0; full_bar = full0; empty_bar = empty0;
+              }
             }
           }
         }
