@@ -17,6 +17,8 @@
 // 16-byte chunk decides whether they reach HBM speed: the norm kind and the number of
 // chunks per thread are template parameters, pointers advance by one add per rank, and
 // the shared/private class of a chunk is resolved by a branch per chunk, not per element.
+#include <cooperative_groups.h>
+
 #include "caat_rows_common.cuh"
 
 namespace caat {
@@ -467,6 +469,212 @@ __global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPar
   }
 }
 
+
+// ---- the same step for very few rows: a cluster of t CTAs per token ------------------------------
+// With a handful of tokens the kernel above is one long dependency chain per CTA: every rank's CTA
+// sums all splits * t planes of the shared channels, eight loads at a time, layer after layer.  Here
+// the t CTAs of a token form a thread-block cluster and divide that work: CTA m fetches, with
+// asynchronous 16-byte copies that are all in flight at once (both layers), a 1/t slice of the shared
+// channels of every plane plus its own rank's private channels; it sums its slice (planes ascending,
+// the order of the kernel above, so the results are bit-identical) and stores the sums into every peer's
+// shared memory; one cluster barrier later each CTA holds the complete rank sum.  A thread owns one
+// 16-byte chunk of the row for both layers (rows of up to 512 chunks), so the new residual stream stays
+// in registers between the statistics, the normalisation and the second layer.
+namespace cgx = cooperative_groups;
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+               ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// float4 slots of the staging area a CTA needs (the widest shared slice is ceil(S/4 / t) chunks)
+inline size_t cluster_partials_smem(const RowPartArgs& a) {
+  const int S4 = a.S / 4, P4 = (a.h - a.S) / 4;
+  const int ns_max = (S4 + a.t - 1) / a.t;
+  size_t f4 = (size_t)a.nlayers * S4 + 16;            // rank sums of the shared channels, reduction scratch
+  for (int l = 0; l < a.nlayers; ++l) f4 += (size_t)a.L[l].splits * ((size_t)a.t * ns_max + P4);
+  return f4 * sizeof(float4);
+}
+
+template <typename T_, bool LN>
+__global__ void __launch_bounds__(512, 1) rows_forward_partials_cluster_kernel(const RowPartArgs a) {
+  using V_ = VT<T_>;
+  using raw = typename V_::raw;
+  constexpr int V = V_::N;
+  constexpr int ES = sizeof(T_);
+  extern __shared__ float4 sm4[];
+  cgx::cluster_group cluster = cgx::this_cluster();
+  const int i = blockIdx.x, m = blockIdx.y;             // the cluster spans the ranks of token i: cluster rank == m
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  const int S4 = a.S / 4, P4 = (a.h - a.S) / 4;
+  const int cs0 = (int)((long long)S4 * m / a.t);       // this CTA's slice of the shared channels, in float4 units
+  const int ns = (int)((long long)S4 * (m + 1) / a.t) - cs0;
+  float4* zs = sm4;                                     // [nlayers][S4]: complete after the cluster barrier
+  float* red = reinterpret_cast<float*>(sm4 + a.nlayers * S4);
+  float4* stage = sm4 + a.nlayers * S4 + 16;
+  const long long row = (long long)m * a.T + i;
+  const long long plane = (long long)a.T * a.h;
+  int par = 0;
+  // a peer's shared memory may be written only once that CTA runs: arrive now, wait before the first remote store
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+  pdl_wait();
+
+  // ---- every partial this CTA needs, both layers, in flight at once
+  int sh_off[2] = {0, 0}, pr_off[2] = {0, 0};
+  {
+    int off = 0;
+#pragma unroll
+    for (int l = 0; l < 2; ++l) {
+      if (l >= a.nlayers) break;
+      const int splits = a.L[l].splits, nplanes = splits * a.t;
+      const float* zt = a.L[l].zt + (long long)i * a.h;
+      sh_off[l] = off;
+      for (int idx = tid; idx < nplanes * ns; idx += nthr) {
+        const int z = idx / ns, c = idx - z * ns;
+        cp_async16(stage + off + idx, zt + z * plane + 4 * (cs0 + c));
+      }
+      off += nplanes * ns;
+      pr_off[l] = off;
+      for (int idx = tid; idx < splits * P4; idx += nthr) {
+        const int q = idx / P4, c = idx - q * P4;
+        cp_async16(stage + off + idx, zt + (long long)(m + q * a.t) * plane + a.S + 4 * c);
+      }
+      off += splits * P4;
+    }
+  }
+  // ---- this thread's chunk of the row: residual and norm parameters, fetched behind the copies
+  const int c = tid * V;
+  const bool active = c < a.h;
+  const bool shared_chunk = c + V <= a.S;               // the partition is a multiple of 8 on this path
+  const long long coff = shared_chunk ? ((long long)i * a.S + c) * ES : (row * (a.h - a.S) + (c - a.S)) * ES;
+  float r[V], g[2][V], b[2][V];
+#pragma unroll
+  for (int e = 0; e < V; ++e) { r[e] = 0.f; g[0][e] = g[1][e] = 0.f; b[0][e] = b[1][e] = 0.f; }
+  if (active) {
+    if (a.compact) V_::unpack(ldg<raw>(static_cast<const char*>(shared_chunk ? a.Rs : a.R) + coff), r);
+    else V_::unpack(ldg<raw>(static_cast<const char*>(a.R) + (row * a.h + c) * ES), r);
+#pragma unroll
+    for (int l = 0; l < 2; ++l) {
+      if (l >= a.nlayers) break;
+      V_::unpack(ldg<raw>(static_cast<const char*>(a.L[l].gamma) + (long long)c * ES), g[l]);
+      if (LN && a.L[l].beta) V_::unpack(ldg<raw>(static_cast<const char*>(a.L[l].beta) + (long long)c * ES), b[l]);
+    }
+  }
+  cp_async_wait_all();
+  __syncthreads();
+  asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+
+  // ---- sums: planes ascending.  Shared slice -> every CTA of the cluster; private -> in place (split 0's slot)
+#pragma unroll
+  for (int l = 0; l < 2; ++l) {
+      if (l >= a.nlayers) break;
+    const int splits = a.L[l].splits, nplanes = splits * a.t;
+    for (int q = tid; q < ns; q += nthr) {
+      const float4* src = stage + sh_off[l] + q;
+      float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int z = 0; z < nplanes; ++z) {
+        const float4 v = src[(size_t)z * ns];
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+      }
+      for (int peer = 0; peer < a.t; ++peer) cluster.map_shared_rank(zs, peer)[l * S4 + cs0 + q] = s;
+    }
+    for (int q = tid; q < P4; q += nthr) {
+      float4* src = stage + pr_off[l] + q;
+      float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int k = 0; k < splits; ++k) {
+        const float4 v = src[(size_t)k * P4];
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+      }
+      *src = s;
+    }
+  }
+  cluster.sync();     // every slice has arrived (and this CTA's own private sums are visible to all its threads)
+
+  const float inv_h = 1.0f / (float)a.h;
+  float hn[V];
+#pragma unroll
+  for (int e = 0; e < V; ++e) hn[e] = 0.f;
+#pragma unroll
+  for (int l = 0; l < 2; ++l) {
+      if (l >= a.nlayers) break;
+    const PartialLayer& L = a.L[l];
+    float st[1] = {0.f};
+    if (active) {
+      float z[V];
+      const float4* src = shared_chunk ? zs + l * S4 + c / 4 : stage + pr_off[l] + (c - a.S) / 4;
+#pragma unroll
+      for (int e = 0; e < V; e += 4) {
+        const float4 v = src[e / 4];
+        z[e] = v.x; z[e + 1] = v.y; z[e + 2] = v.z; z[e + 3] = v.w;
+      }
+#pragma unroll
+      for (int e = 0; e < V; ++e) {
+        const float res = l == 0 ? r[e] : V_::round(hn[e]);    // the second layer's residual is the first one's stream as stored
+        hn[e] = (shared_chunk ? z[e] : a.alpha * z[e]) + res;
+        st[0] = LN ? st[0] + hn[e] : fmaf(hn[e], hn[e], st[0]);
+      }
+      if (a.compact) {      // every rank's CTA forms the same shared values; rank 0's writes them
+        if (!shared_chunk || m == 0) stg<raw>(static_cast<char*>(shared_chunk ? L.Hns : L.Hn) + coff, V_::pack(hn));
+      } else {
+        stg<raw>(static_cast<char*>(L.Hn) + (row * a.h + c) * ES, V_::pack(hn));
+      }
+    }
+    row_reduce_sync<1>(st, red, par);
+    float mu = 0.f, rs;
+    if (LN) {
+      mu = st[0] * inv_h;
+      float sq[1] = {0.f};
+      if (active) {
+#pragma unroll
+        for (int e = 0; e < V; ++e) { const float d = hn[e] - mu; sq[0] = fmaf(d, d, sq[0]); }
+      }
+      row_reduce_sync<1>(sq, red, par);
+      rs = rsqrtf(fmaf(sq[0], inv_h, a.eps));
+    } else {
+      rs = rsqrtf(fmaf(st[0], inv_h, a.eps));
+    }
+    if (active) {
+      float x[V];
+#pragma unroll
+      for (int e = 0; e < V; ++e) x[e] = LN ? fmaf(hn[e] - mu, rs * g[l][e], b[l][e]) : hn[e] * (rs * g[l][e]);
+      stg<raw>(static_cast<char*>(L.X) + (row * a.h + c) * ES, V_::pack(x));
+    }
+    if (tid == 0) {
+      L.rstd[row] = rs;
+      if (LN && L.mean) L.mean[row] = mu;
+    }
+  }
+}
+
+template <typename T_, bool LN>
+cudaError_t launch_partials_cluster(const RowPartArgs& a, int threads, size_t smem, cudaStream_t st) {
+  static bool attr_set[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!attr_set[dev]) {
+    const cudaError_t e = cudaFuncSetAttribute(rows_forward_partials_cluster_kernel<T_, LN>,
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set[dev] = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.T, a.t);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2] = {};
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1;
+  attr[0].val.clusterDim.y = (unsigned)a.t;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, rows_forward_partials_cluster_kernel<T_, LN>, a);
+}
+
 // out[l] = sum over `rows` partial rows, fixed order: 32 row lanes then a serial combine.
 // Blocks past the first `nreduce` run an unrelated small job that has to happen between the row kernel and the
 // data gradient anyway and would otherwise cost a launch of its own: scaling the private rows of the weights.
@@ -548,6 +756,16 @@ cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype,
   const dim3 grid(a.T, a.t);
   const size_t smem = (size_t)a.h * sizeof(float) + 2 * 16 * 2 * sizeof(float);
   LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
+  // few rows: the cluster kernel, as long as all its CTAs are resident at once (portable cluster size 8,
+  // one chunk per thread, one CTA per SM at its register count; clusters need whole groups of SMs, hence 3/4)
+  static const int cluster_mode = [] { const char* e = getenv("CAAT_DECODE_CLUSTER"); return e ? atoi(e) : 1; }();
+  if (cluster_mode && dtype == CAAT_BF16 && a.t >= 2 && a.t <= 8 && a.h % V == 0 && a.h / V <= 512 && a.S % 4 == 0 &&
+      (a.h - a.S) % 4 == 0) {
+    const size_t csm = cluster_partials_smem(a);
+    if (csm <= 200 * 1024 && (long long)a.T * a.t <= (long long)sm_count() * 3 / 4)
+      return a.norm == 1 ? launch_partials_cluster<__nv_bfloat16, true>(a, threads, csm, st)
+                         : launch_partials_cluster<__nv_bfloat16, false>(a, threads, csm, st);
+  }
   if (dtype == CAAT_BF16) {
     if (a.norm == 1) return launch_pdl(rows_forward_partials_kernel<__nv_bfloat16, true>, grid, dim3(threads), smem, st, a);
     return launch_pdl(rows_forward_partials_kernel<__nv_bfloat16, false>, grid, dim3(threads), smem, st, a);

@@ -250,7 +250,11 @@ def test_block_forward_backward_small():
 
 @pytest.mark.parametrize("no_decode", [False, True])
 @pytest.mark.parametrize("t,T,h,ffn,S,norm", [(8, 64, 4096, 11008, 2048, 0), (4, 37, 768, 3072, 384, 1),
-                                             (8, 1, 2048, 5632, 2048, 0), (2, 5, 256, 1024, 0, 0)])
+                                             (8, 1, 2048, 5632, 2048, 0), (2, 5, 256, 1024, 0, 0),
+                                             # a handful of tokens: the cluster row kernel (LayerNorm; a shared
+                                             # slice that does not divide evenly among the ranks; three ranks)
+                                             (4, 3, 768, 3072, 384, 1), (8, 2, 4096, 11008, 1000, 0),
+                                             (3, 4, 768, 3072, 256, 0)])
 def test_few_token_forward_both_paths(no_decode, t, T, h, ffn, S, norm):
     # forward calls with at most 64 tokens take the weight-streaming path (swapped GEMM operands,
     # rank sum in the row kernel); CAAT_OPT_DECODE = 1 sends them down the large-batch path
