@@ -321,9 +321,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     // Two single-thread producers run the same schedule: warp 0 issues the A boxes (and, in the
     // leader CTA, posts the stage's expected bytes), warp kProducerB the B boxes.  Issuing a
     // stage's boxes from one thread was the bottleneck of the operand pipeline (up to four boxes
-    // per stage for M-/N-major operands); two independent instruction streams halve it.
-    if (lane == 0) {
-      const bool isA = warp == 0;
+    // per stage for M-/N-major operands); two independent instruction streams halve it, and an
+    // operand that needs several boxes per stage (M-/N-major: one per 64 rows or columns) has them
+    // issued by as many lanes of its warp, each of which follows the barriers itself.
+    const bool isA = warp == 0;
+    static_assert(BM / 64 <= 32, "one lane per box");
+    const bool wide = (isA ? p.a_mn : p.b_mn) && !(p.debug & 512);
+    if (lane == 0 || wide) {
       int stage = 0; uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
@@ -348,7 +352,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
               // completion is signalled on the LEADER's barrier; the leader expects both CTAs' bytes
               const uint32_t fb = CG == 2 ? mapa_rank(fb_local, 0) : fb_local;
               const uint32_t sa = tiles_sa + (uint32_t)stage * stage_bytes, sb = sa + a_bytes;
-              if (isA && rank == 0) {
+              if (isA && rank == 0 && lane == 0) {
                 if (p.debug & 1) mbar_arrive(fb_local); else mbar_expect_tx(fb_local, tx);
               }
               if (!(p.debug & 1) && !skip) {
@@ -358,6 +362,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
                 if (isA) {
                   if (!p.a_mn) {
                     load(sa, u.ak0 + kk * BK, m0);
+                  } else if (wide) {
+                    if (lane < BM / 64) load(sa + lane * (64 * BK * 2), u.am0 + m0 + lane * 64, u.ak0 + kk * BK);
                   } else {
 #pragma unroll
                     for (int ch = 0; ch < BM / 64; ++ch) load(sa + ch * (64 * BK * 2), u.am0 + m0 + ch * 64, u.ak0 + kk * BK);
@@ -365,6 +371,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
                 } else {
                   if (!p.b_mn) {
                     load(sb, u.bk0 + kk * BK, u.bn0 + n0);
+                  } else if (wide) {
+                    if (lane < (int)cols_cta / 64) load(sb + lane * (64 * BK * 2), u.bn0 + n0 + lane * 64, u.bk0 + kk * BK);
                   } else {
                     for (int ch = 0; ch < (int)cols_cta / 64; ++ch)
                       load(sb + ch * (64 * BK * 2), u.bn0 + n0 + ch * 64, u.bk0 + kk * BK);
@@ -377,7 +385,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           }
         }
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         // gave up: flag it, then wait (bounded) for the copies still in flight
         // (the pair's copies complete on the leader's barriers; the peer just gives them time)
         *abort_flag = 1;
@@ -488,10 +496,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols + cc), v);
           tmem_ld_wait();
           if (chan < r.M) {
+            float* dst = r.out_t + ((long long)zc * r.N + n0 + cc) * p.out_t_ld + chan;
+            const int ntok = r.N - (n0 + cc);           // tokens left from this column on (>= 1)
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-              const int tok = n0 + cc + e;
-              if (tok < r.N) r.out_t[((long long)zc * r.N + tok) * p.out_t_ld + chan] = total_k == 0 ? 0.f : __uint_as_float(v[e]);
+              if (e < ntok) *dst = total_k == 0 ? 0.f : __uint_as_float(v[e]);
+              dst += p.out_t_ld;
             }
           }
         }

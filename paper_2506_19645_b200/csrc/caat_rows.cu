@@ -497,8 +497,8 @@ inline size_t cluster_partials_smem(const RowPartArgs& a) {
   return f4 * sizeof(float4);
 }
 
-template <typename T_, bool LN>
-__global__ void __launch_bounds__(512, 1) rows_forward_partials_cluster_kernel(const RowPartArgs a) {
+template <typename T_, bool LN, int MINB>
+__global__ void __launch_bounds__(512, MINB) rows_forward_partials_cluster_kernel(const RowPartArgs a) {
   using V_ = VT<T_>;
   using raw = typename V_::raw;
   constexpr int V = V_::N;
@@ -647,13 +647,13 @@ __global__ void __launch_bounds__(512, 1) rows_forward_partials_cluster_kernel(c
   }
 }
 
-template <typename T_, bool LN>
+template <typename T_, bool LN, int MINB>
 cudaError_t launch_partials_cluster(const RowPartArgs& a, int threads, size_t smem, cudaStream_t st) {
   static bool attr_set[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (!attr_set[dev]) {
-    const cudaError_t e = cudaFuncSetAttribute(rows_forward_partials_cluster_kernel<T_, LN>,
+    const cudaError_t e = cudaFuncSetAttribute(rows_forward_partials_cluster_kernel<T_, LN, MINB>,
                                                cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
@@ -672,7 +672,7 @@ cudaError_t launch_partials_cluster(const RowPartArgs& a, int threads, size_t sm
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, rows_forward_partials_cluster_kernel<T_, LN>, a);
+  return cudaLaunchKernelEx(&cfg, rows_forward_partials_cluster_kernel<T_, LN, MINB>, a);
 }
 
 // out[l] = sum over `rows` partial rows, fixed order: 32 row lanes then a serial combine.
@@ -763,8 +763,14 @@ cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype,
       (a.h - a.S) % 4 == 0) {
     const size_t csm = cluster_partials_smem(a);
     if (csm <= 200 * 1024 && (long long)a.T * a.t <= (long long)sm_count() * 3 / 4)
-      return a.norm == 1 ? launch_partials_cluster<__nv_bfloat16, true>(a, threads, csm, st)
-                         : launch_partials_cluster<__nv_bfloat16, false>(a, threads, csm, st);
+      return a.norm == 1 ? launch_partials_cluster<__nv_bfloat16, true, 1>(a, threads, csm, st)
+                         : launch_partials_cluster<__nv_bfloat16, false, 1>(a, threads, csm, st);
+    // more rows than that: two CTAs per SM (64 registers, RMSNorm variant), a few waves.  Pays when most
+    // channels are shared, where the kernel below reads every shared plane once per rank (measured at
+    // 64 tokens of the 7B shapes: 3 % faster at p = 1, 5 % slower at p = 0.5).
+    if (a.norm != 1 && csm <= 100 * 1024 && (long long)a.S * 4 > (long long)a.h * 3 &&
+        (long long)a.T * a.t <= (long long)sm_count() * 4)
+      return launch_partials_cluster<__nv_bfloat16, false, 2>(a, threads, csm, st);
   }
   if (dtype == CAAT_BF16) {
     if (a.norm == 1) return launch_pdl(rows_forward_partials_kernel<__nv_bfloat16, true>, grid, dim3(threads), smem, st, a);
