@@ -120,6 +120,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// One lane of a converged warp (the hardware's pick).  Branching on it instead of on the lane index keeps
+// the surrounding control flow warp-uniform, so loop state and the operands of the tensor-core and
+// TMA instructions can live in uniform registers: issuing four MMAs and a commit from a divergent
+// single-lane branch cost 310 cycles per k-step, from a uniform loop 130.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.u32 %0, 1, 0, P;\n}" : "=r"(pred));
+  return pred != 0;
+}
+// Bounded wait by a whole warp with a warp-uniform result.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -401,7 +415,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only when CG == 2)
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {                              // the whole warp walks the schedule, one elected lane issues
       const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
                               ((uint32_t)(BMT >> 4) << 24);
       int stage = 0; uint32_t phase = 0;
@@ -421,7 +435,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       for (int tile = worker; tile < p.tiles_total && ok; tile += nworkers) {
         const TileCoord c = decode_tile(p, tile);
         const Region& r = p.r[c.region];
-        if (!mbar_wait(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_warp(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
         const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(p, r, c.nt, CG) >> 3) << 17);
@@ -432,18 +446,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           split_range(r.splits, u, c.split, kb, ke);
           for (int q = 0; q < u.Q && ok; ++q) {
             for (int kk = kb; kk < ke; ++kk) {
-              if (!mbar_wait(full_bar, phase, abort_flag)) { ok = false; break; }
+              if (!mbar_wait_warp(full_bar, phase, abort_flag)) { ok = false; break; }
               tc_fence_after();
+              if (elect_one()) {
 #pragma unroll
-              for (int k = 0; k < BK / UMMA_K; ++k) {
-                const uint64_t ad = ((uint64_t)a_hi << 32) | (a_lo + (uint32_t)k * a_k16);
-                const uint64_t bd = ((uint64_t)b_hi << 32) | (b_lo + (uint32_t)k * b_k16);
-                if (CG == 2) umma_bf16_pair(d_tmem, ad, bd, idesc, accumulate);
-                else umma_bf16(d_tmem, ad, bd, idesc, accumulate);
-                accumulate = 1;
+                for (int k = 0; k < BK / UMMA_K; ++k) {
+                  const uint64_t ad = ((uint64_t)a_hi << 32) | (a_lo + (uint32_t)k * a_k16);
+                  const uint64_t bd = ((uint64_t)b_hi << 32) | (b_lo + (uint32_t)k * b_k16);
+                  if (CG == 2) umma_bf16_pair(d_tmem, ad, bd, idesc, k == 0 ? accumulate : 1u);
+                  else umma_bf16(d_tmem, ad, bd, idesc, k == 0 ? accumulate : 1u);
+                }
+                // frees the stage (in both CTAs) once these MMAs have read it
+                if (CG == 2) umma_commit_pair(empty_bar); else umma_commit(empty_bar);
               }
-              // frees the stage (in both CTAs) once these MMAs have read it
-              if (CG == 2) umma_commit_pair(empty_bar); else umma_commit(empty_bar);
+              accumulate = 1;
               a_lo += stage16; b_lo += stage16; full_bar += 8u; empty_bar += 8u;
               if (++stage == p.nstages) {
                 stage = 0; phase ^= 1u;
@@ -452,13 +468,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
             }
           }
         }
-        if (ok) {                                   // accumulator complete (in both CTAs)
+        if (ok && elect_one()) {                    // accumulator complete (in both CTAs)
           if (CG == 2) umma_commit_pair(tfull0 + 8u * acc); else umma_commit(tfull0 + 8u * acc);
         }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
-      if (!ok) { *abort_flag = 1; atomicExch(p.status, 2u); }
+      if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, 2u); }
     }
   } else if (warp <= 5) {
     // ------------------------------------------------------------ epilogue (warps 2..5)
