@@ -254,7 +254,9 @@ def test_block_forward_backward_small():
                                              # a handful of tokens: the cluster row kernel (LayerNorm; a shared
                                              # slice that does not divide evenly among the ranks; three ranks)
                                              (4, 3, 768, 3072, 384, 1), (8, 2, 4096, 11008, 1000, 0),
-                                             (3, 4, 768, 3072, 256, 0)])
+                                             (3, 4, 768, 3072, 256, 0),
+                                             # shared part smaller than the cluster: most CTAs own no slice
+                                             (8, 2, 4096, 11008, 8, 0), (8, 3, 4096, 11008, 4088, 1)])
 def test_few_token_forward_both_paths(no_decode, t, T, h, ffn, S, norm):
     # forward calls with at most 64 tokens take the weight-streaming path (swapped GEMM operands,
     # rank sum in the row kernel); CAAT_OPT_DECODE = 1 sends them down the large-batch path
