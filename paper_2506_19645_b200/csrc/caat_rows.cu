@@ -647,8 +647,11 @@ __global__ void __launch_bounds__(512, MINB) rows_forward_partials_cluster_kerne
   }
 }
 
+// *launched = false (and cudaSuccess) when this device cannot place such a cluster: the caller then
+// takes the general kernel.
 template <typename T_, bool LN, int MINB>
-cudaError_t launch_partials_cluster(const RowPartArgs& a, int threads, size_t smem, cudaStream_t st) {
+cudaError_t launch_partials_cluster(const RowPartArgs& a, int threads, size_t smem, cudaStream_t st, bool* launched) {
+  *launched = false;
   static bool attr_set[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
@@ -671,7 +674,24 @@ cudaError_t launch_partials_cluster(const RowPartArgs& a, int threads, size_t sm
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  // can a cluster of t such CTAs be co-scheduled here at all?  (asked once per device, cluster size and footprint)
+  struct Seen { int dev, t, threads; size_t smem; int clusters; };
+  static Seen seen[8] = {};
+  static int nseen = 0;
+  int clusters = -1;
+  for (int q = 0; q < nseen; ++q)
+    if (seen[q].dev == dev && seen[q].t == a.t && seen[q].threads == threads && seen[q].smem == smem) clusters = seen[q].clusters;
+  if (clusters < 0) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, rows_forward_partials_cluster_kernel<T_, LN, MINB>, &cfg) != cudaSuccess) {
+      cudaGetLastError();
+      clusters = 0;
+    }
+    if (nseen < 8) seen[nseen++] = Seen{dev, a.t, threads, smem, clusters};
+  }
+  if (clusters < 1) return cudaSuccess;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  *launched = true;
   return cudaLaunchKernelEx(&cfg, rows_forward_partials_cluster_kernel<T_, LN, MINB>, a);
 }
 
@@ -762,15 +782,21 @@ cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype,
   if (cluster_mode && dtype == CAAT_BF16 && a.t >= 2 && a.t <= 8 && a.h % V == 0 && a.h / V <= 512 && a.S % 4 == 0 &&
       (a.h - a.S) % 4 == 0) {
     const size_t csm = cluster_partials_smem(a);
-    if (csm <= 200 * 1024 && (long long)a.T * a.t <= (long long)sm_count() * 3 / 4)
-      return a.norm == 1 ? launch_partials_cluster<__nv_bfloat16, true, 1>(a, threads, csm, st)
-                         : launch_partials_cluster<__nv_bfloat16, false, 1>(a, threads, csm, st);
+    bool launched = false;
+    cudaError_t e = cudaSuccess;
+    if (csm <= 200 * 1024 && (long long)a.T * a.t <= (long long)sm_count() * 3 / 4) {
+      e = a.norm == 1 ? launch_partials_cluster<__nv_bfloat16, true, 1>(a, threads, csm, st, &launched)
+                      : launch_partials_cluster<__nv_bfloat16, false, 1>(a, threads, csm, st, &launched);
+      if (launched || e != cudaSuccess) return e;
+    }
     // more rows than that: two CTAs per SM (64 registers, RMSNorm variant), a few waves.  Pays when most
     // channels are shared, where the kernel below reads every shared plane once per rank (measured at
     // 64 tokens of the 7B shapes: 3 % faster at p = 1, 5 % slower at p = 0.5).
     if (a.norm != 1 && csm <= 100 * 1024 && (long long)a.S * 4 > (long long)a.h * 3 &&
-        (long long)a.T * a.t <= (long long)sm_count() * 4)
-      return launch_partials_cluster<__nv_bfloat16, false, 2>(a, threads, csm, st);
+        (long long)a.T * a.t <= (long long)sm_count() * 4) {
+      e = launch_partials_cluster<__nv_bfloat16, false, 2>(a, threads, csm, st, &launched);
+      if (launched || e != cudaSuccess) return e;
+    }
   }
   if (dtype == CAAT_BF16) {
     if (a.norm == 1) return launch_pdl(rows_forward_partials_kernel<__nv_bfloat16, true>, grid, dim3(threads), smem, st, a);
