@@ -77,10 +77,13 @@ struct Params {
   int tiles_r0;          // tiles of region 0 (including splits)
   int tiles_total;
   unsigned int* status;
+  uint32_t spin_cap;     // polls of one mbarrier wait before the role gives up (kSpinCap; CAAT_TC_SPINCAP for the timeout test)
   int debug;             // measurement aid (env CAAT_TC_DEBUG; results are then wrong): 1 = no operand loads,
                          // 2 = no epilogue work at all, 4 = no A loads, 8 = no B loads; epilogue stops after the
                          // tensor-memory load (32) / after the staging stores (16); 64 = no slab barrier,
-                         // 128 = no TMA store
+                         // 128 = no TMA store; 512 = one lane issues all boxes of a stage; 1024 = the A boxes are
+                         // announced to the stage barrier but never issued, so the consumers' waits run out
+                         // (the timeout test: the kernel must flag it, drain and return)
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -105,8 +108,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false when the cap ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinCap; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t cap) {
+  for (uint32_t it = 0; it < cap; ++it) {
     if (mbar_try(bar, parity)) return true;
     if ((it & 1023u) == 1023u && *abort_flag) return false;
   }
@@ -130,8 +133,8 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 // Bounded wait by a whole warp with a warp-uniform result.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t cap) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, cap));
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -352,7 +355,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         const uint32_t b_tile_bytes = cols_cta * BK * 2;
         const int m0 = c.mt * BMT + (int)rank * BM, n0 = c.nt * p.BN + (int)(rank * cols_cta);
         const uint32_t tx = (uint32_t)CG * (((p.debug & 4) ? 0u : a_bytes) + ((p.debug & 8) ? 0u : b_tile_bytes));
-        const bool skip = isA ? (p.debug & 4) != 0 : (p.debug & 8) != 0;
+        const bool skip = isA ? (p.debug & (4 | 1024)) != 0 : (p.debug & 8) != 0;
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
           const CUtensorMap* map = maps[isA ? u.mapA : u.mapB];
@@ -361,7 +364,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           for (int q = 0; q < u.Q && ok; ++q) {
             const int z = isA ? c.b * u.a_zb + q * u.a_zq : c.b * u.b_zb + q * u.b_zq;
             for (int kk = kb; kk < ke; ++kk) {
-              if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+              if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag, p.spin_cap)) { ok = false; break; }
               const uint32_t fb_local = full0 + 8u * stage;
               // completion is signalled on the LEADER's barrier; the leader expects both CTAs' bytes
               const uint32_t fb = CG == 2 ? mapa_rank(fb_local, 0) : fb_local;
@@ -408,7 +411,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         int s = stage; uint32_t ph = phase;
         for (int k = 0; k < pending; ++k) {
           if (--s < 0) { s = p.nstages - 1; ph ^= 1u; }
-          for (uint32_t it = 0; it < (1u << 20); ++it)
+          for (uint32_t it = 0; it < (p.spin_cap < (1u << 20) ? p.spin_cap : (1u << 20)); ++it)
             if (rank == 0 && mbar_try(full0 + 8u * s, ph)) break;
         }
       }
@@ -435,7 +438,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       for (int tile = worker; tile < p.tiles_total && ok; tile += nworkers) {
         const TileCoord c = decode_tile(p, tile);
         const Region& r = p.r[c.region];
-        if (!mbar_wait_warp(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_warp(tempty0 + 8u * acc, acc_phase ^ 1u, abort_flag, p.spin_cap)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
         const uint32_t idesc = idesc0 | ((uint32_t)(tile_cols(p, r, c.nt, CG) >> 3) << 17);
@@ -446,7 +449,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           split_range(r.splits, u, c.split, kb, ke);
           for (int q = 0; q < u.Q && ok; ++q) {
             for (int kk = kb; kk < ke; ++kk) {
-              if (!mbar_wait_warp(full_bar, phase, abort_flag)) { ok = false; break; }
+              if (!mbar_wait_warp(full_bar, phase, abort_flag, p.spin_cap)) { ok = false; break; }
               tc_fence_after();
               if (elect_one()) {
 #pragma unroll
@@ -492,7 +495,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         split_range(r.splits, r.u[ui], c.split, kb, ke);
         total_k += (ke - kb) * r.u[ui].Q;
       }
-      if (!mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(tfull0 + 8u * acc, acc_phase, abort_flag, p.spin_cap)) { ok = false; break; }
       tc_fence_after();
       // Drain 64-byte-wide column slabs (32 bf16 / 16 fp32 columns): TMEM -> registers ->
       // swizzled staging buffer -> TMA store (coalesced; rows and columns outside the region's
@@ -734,6 +737,8 @@ cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params
   if (!p.status) return cudaErrorUnknown;
   static const int dbg = [] { const char* e = getenv("CAAT_TC_DEBUG"); return e ? atoi(e) : 0; }();
   p.debug = dbg;
+  static const uint32_t cap_env = [] { const char* e = getenv("CAAT_TC_SPINCAP"); return e ? (uint32_t)atoi(e) : 0u; }();
+  p.spin_cap = cap_env >= 1024 ? cap_env : kSpinCap;
   static const bool verbose = getenv("CAAT_TC_VERBOSE") != nullptr;
   if (verbose)
     fprintf(stderr, "[caat tc] kind=%d BN=%d cg=%d splits=%d stages=%d tiles=%d (r0 M=%d N=%d b=%d)\n", kind, p.BN, p.cg,
