@@ -566,9 +566,9 @@ def run_cuda(args):
                 continue
             try:
                 r = make_runner(synthetic.WORKLOADS[name], dev)
-                for _ in range(3):
+                for _ in range(5):
                     r.step()
-                k = max(3, min(args.steps, 10))
+                k = max(3, min(args.steps, 30))
                 sms = time_steps(r, k, False) / k
                 fl, by = paper_level_work(r.w)
                 peaks = measured_peaks()
