@@ -80,7 +80,7 @@ typedef enum {
   CAAT_OPT_DECODE = 6,          /* 0 = automatic (default: forward calls with at most 64 tokens
                                    stream the weights with swapped GEMM operands),
                                    1 = always use the large-batch forward                */
-  CAAT_OPT_BACKWARD_REDUCE = 7  /* precision of the backward rank sum on the shared channels
+  CAAT_OPT_BACKWARD_REDUCE = 7, /* precision of the backward rank sum on the shared channels
                                    (Section 4, "fp32 accumulation"); a numerics-study switch:
                                    0 = the ranks' gradients are summed in fp32 as computed (default);
                                    1 = each rank's gradient is first rounded to the run dtype (what
@@ -88,6 +88,11 @@ typedef enum {
                                    2 = rounded, and the running sum is rounded to the run dtype
                                        after every addition (accumulation in 16 bit).
                                    1 and 2 run on the plain-load row kernels.              */
+  CAAT_OPT_TP_GROUPS = 8        /* G >= 1 (default 1): this context holds t of t*G tensor-parallel ranks,
+                                   one group of t ranks per GPU (see caat_tp_*): K_r becomes K / (t*G).
+                                   Setting it also sets alpha = sqrt(t*G) (Section 4: the square root of
+                                   the number of devices); CAAT_OPT_PRIVATE_SCALE may override that
+                                   afterwards.  CAAT_ESHAPE unless t*G divides h and ffn.               */
 } caat_option;
 
 /* Creates a context for hidden size h, MLP width ffn, t ranks, synchronisation
@@ -325,13 +330,59 @@ caat_status caat_colpar_backward(const caat_ctx *ctx, caat_activation act, int n
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Real tensor parallelism over several GPUs (Section 3: the all-reduce of the shared channels is the
+ * layer's one exchange step; Appendix D: reduce-scatter + all-gather of tokens*S elements).  A layer call
+ * is split into the half before and the half after that exchange; the caller owns the collective (NCCL
+ * through its framework, or its own kernel over peer memory) and runs it, on the same stream, on the
+ * packed slab the first half leaves in the workspace:
+ *
+ *   forward :  caat_tp_forward_local   slab[i,l] = sum over this GPU's ranks m of Zt[m,i,l], l < S
+ *                                      (the private columns of Zt stay in the workspace as well)
+ *              all-reduce(slab, sum)   over the GPUs of the tensor-parallel group
+ *              caat_tp_forward_finish  private scaling, residual add, per-rank norm (Eq. 9)
+ *   backward:  caat_tp_backward_local  norm backward + residual gradient: dR, this GPU's dgamma / dbeta,
+ *                                      slab[i,l] = sum over this GPU's ranks of g[m,i,l], l < S
+ *              all-reduce(slab, sum)   -- Section 4: accumulate this sum in fp32; also all-reduce
+ *                                         dgamma / dbeta [h] fp32 (Eq. 10-11: summed over devices)
+ *              caat_tp_backward_finish dY and dW from the reduced slab and this GPU's dR
+ *
+ * The context describes this GPU's t ranks of the t*G in the group (CAAT_OPT_TP_GROUPS = G); tensors
+ * are the same as in caat_rowpar_forward / _backward with this GPU's ranks only.  The slab is
+ * [tokens, S] elements of the run dtype, row-major and dense, at byte `offset` of the workspace
+ * (caat_tp_slab; the forward and the backward slab may sit at different offsets).  Both halves of a
+ * direction must get the same workspace, untouched in between except for the slab.  Tensor-core path
+ * only (bf16, K_r and S multiples of 8): CAAT_EUNSUPPORTED otherwise.  Workspace size:
+ * caat_workspace_bytes.  With G = 1 the two halves and no collective give caat_rowpar_forward /
+ * _backward's results for more than 64 tokens (few-token calls take another route there).
+ */
+caat_status caat_tp_slab(const caat_ctx *ctx, caat_layer layer, int tokens, int backward,
+                         size_t *offset_bytes, int *rows, int *cols);
+caat_status caat_tp_forward_local(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                  const void *Y, const void *W,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
+caat_status caat_tp_forward_finish(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                   const void *R, const void *gamma, const void *beta,
+                                   void *Hn, void *X, float *rstd, float *mean,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+caat_status caat_tp_backward_local(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                   const void *dX, const void *dHn, const void *W, const void *Hn,
+                                   const float *rstd, const float *mean, const void *gamma,
+                                   void *dR, float *dgamma, float *dbeta,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+caat_status caat_tp_backward_finish(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                    const void *Y, const void *W, const void *dR,
+                                    void *dY, float *dW,
+                                    void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Analytic bytes ONE partial channel-reduce would move on a real t-device system
  * (Appendix C: each device sends and receives tokens*h*p activations per reduce;
  * Appendix D: all-reduce = reduce-scatter + all-gather, traffic cut by 100(1-p) %).
  * elem_bytes is 2 for 16-bit communication.  Host-only.  Outputs may be NULL.
  *   payload_per_rank     = tokens * S * elem_bytes
  *   payload_per_rank_p1  = tokens * h * elem_bytes          (full all-reduce)
- *   ring_wire_per_rank   = 2 (t-1) * payload / t            (rounded down)
+ *   ring_wire_per_rank   = 2 (n-1) * payload / n            (rounded down; n = t, or the number of
+ *                                                             GPUs G when CAAT_OPT_TP_GROUPS > 1)
  */
 caat_status caat_allreduce_bytes(const caat_ctx *ctx, int tokens, int elem_bytes,
                                  unsigned long long *payload_per_rank,

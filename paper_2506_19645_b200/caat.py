@@ -22,7 +22,7 @@ CAAT_ATTN_OUT, CAAT_MLP_DOWN = 0, 1
  CAAT_ETIMEOUT, CAAT_ELIMIT) = range(9)
 CAAT_NOALLOC_SCRATCH_BYTES = 32 * 1024 * 1024
 (CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM, CAAT_OPT_ROWS,
- CAAT_OPT_DECODE, CAAT_OPT_BACKWARD_REDUCE) = range(8)
+ CAAT_OPT_DECODE, CAAT_OPT_BACKWARD_REDUCE, CAAT_OPT_TP_GROUPS) = range(9)
 RMSNORM, LAYERNORM = 0, 1
 CAAT_ACT_NONE, CAAT_ACT_SILU, CAAT_ACT_SWIGLU = 0, 1, 2
 
@@ -53,6 +53,11 @@ _sigs = {
     "caat_colpar_workspace_bytes": (c_size_t, [_P, c_int, c_int, c_int]),
     "caat_colpar_forward": (c_int, [_P, c_int, c_int, c_int] + [_P] * 4 + [_P]),
     "caat_colpar_backward": (c_int, [_P, c_int, c_int, c_int] + [_P] * 6 + [_P, c_size_t, _P]),
+    "caat_tp_slab": (c_int, [_P, c_int, c_int, c_int, POINTER(c_size_t), POINTER(c_int), POINTER(c_int)]),
+    "caat_tp_forward_local": (c_int, [_P, c_int, c_int] + [_P] * 2 + [_P, c_size_t, _P]),
+    "caat_tp_forward_finish": (c_int, [_P, c_int, c_int] + [_P] * 7 + [_P, c_size_t, _P]),
+    "caat_tp_backward_local": (c_int, [_P, c_int, c_int] + [_P] * 10 + [_P, c_size_t, _P]),
+    "caat_tp_backward_finish": (c_int, [_P, c_int, c_int] + [_P] * 5 + [_P, c_size_t, _P]),
     "caat_allreduce_bytes": (c_int, [_P, c_int, c_int] + [POINTER(c_ulonglong)] * 3),
     "caat_last_device_status": (c_int, [_P, _P]),
     "caat_kernel_launches": (c_ulonglong, []),
@@ -119,6 +124,7 @@ class Context:
         self.dtype_code = _dtype_code(dtype)
         self.torch_dtype = torch.bfloat16 if self.dtype_code == CAAT_BF16 else torch.float32
         self.norm = RMSNORM
+        self.groups = 1
         _check(lib.caat_create(h, ffn, t, float(p), self.dtype_code, byref(self._h)), "caat_create")
 
     def __del__(self):
@@ -132,6 +138,8 @@ class Context:
         _check(lib.caat_set_option(self._h, opt, float(value)), "caat_set_option")
         if opt == CAAT_OPT_NORM:
             self.norm = int(value)
+        if opt == CAAT_OPT_TP_GROUPS:
+            self.groups = int(value)
         return self
 
     @property
@@ -143,7 +151,7 @@ class Context:
         return lib.caat_private_scale(self._h)
 
     def k_r(self, layer: int) -> int:
-        return (self.h if layer == CAAT_ATTN_OUT else self.ffn) // self.t
+        return (self.h if layer == CAAT_ATTN_OUT else self.ffn) // (self.t * self.groups)
 
     def workspace_bytes(self, layer: int, tokens: int, backward: bool) -> int:
         return lib.caat_workspace_bytes(self._h, layer, tokens, 1 if backward else 0)
@@ -345,6 +353,48 @@ class Context:
             _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel() if workspace is not None else 0,
             _stream())
         _check(st, "caat_colpar_backward")
+
+    # ---- real tensor parallelism: the halves of a layer call around the caller's all-reduce
+    def tp_slab(self, layer, tokens, backward, workspace):
+        """The [tokens, S] slab of `workspace` that the caller all-reduces between the two halves (a view)."""
+        off, rows, cols = c_size_t(), c_int(), c_int()
+        _check(lib.caat_tp_slab(self._h, layer, tokens, 1 if backward else 0, byref(off), byref(rows), byref(cols)),
+               "caat_tp_slab")
+        es = 2 if self.dtype_code == CAAT_BF16 else 4
+        nbytes = rows.value * cols.value * es
+        return workspace[off.value:off.value + nbytes].view(self.torch_dtype).view(rows.value, cols.value)
+
+    def tp_forward_local(self, layer, tokens, Y, W, workspace):
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        _check(lib.caat_tp_forward_local(
+            self._h, layer, tokens, _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()), "caat_tp_forward_local")
+
+    def tp_forward_finish(self, layer, tokens, R, gamma, beta, Hn, X, rstd, mean, workspace):
+        td, t, h = self.torch_dtype, self.t, self.h
+        _check(lib.caat_tp_forward_finish(
+            self._h, layer, tokens, _ptr(R, td, (t, tokens, h), "R"), _ptr(gamma, td, (h,), "gamma"),
+            _ptr(beta, td, (h,), "beta"), _ptr(Hn, td, (t, tokens, h), "Hn"), _ptr(X, td, (t, tokens, h), "X"),
+            _ptr(rstd, torch.float32, (t, tokens), "rstd"), _ptr(mean, torch.float32, (t, tokens), "mean"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()), "caat_tp_forward_finish")
+
+    def tp_backward_local(self, layer, tokens, dX, dHn, W, Hn, rstd, mean, gamma, dR, dgamma, dbeta, workspace):
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        f32 = torch.float32
+        _check(lib.caat_tp_backward_local(
+            self._h, layer, tokens, _ptr(dX, td, (t, tokens, h), "dX"), _ptr(dHn, td, (t, tokens, h), "dHn"),
+            _ptr(W, td, (t, h, k), "W"), _ptr(Hn, td, (t, tokens, h), "Hn"), _ptr(rstd, f32, (t, tokens), "rstd"),
+            _ptr(mean, f32, (t, tokens), "mean"), _ptr(gamma, td, (h,), "gamma"), _ptr(dR, td, (t, tokens, h), "dR"),
+            _ptr(dgamma, f32, (h,), "dgamma"), _ptr(dbeta, f32, (h,), "dbeta"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()), "caat_tp_backward_local")
+
+    def tp_backward_finish(self, layer, tokens, Y, W, dR, dY, dW, workspace):
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        _check(lib.caat_tp_backward_finish(
+            self._h, layer, tokens, _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"),
+            _ptr(dR, td, (t, tokens, h), "dR"), _ptr(dY, td, (t, tokens, k), "dY"),
+            _ptr(dW, torch.float32, (t, h, k), "dW"),
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()), "caat_tp_backward_finish")
 
     # ---- buffer helpers (torch.empty only; no arithmetic)
     def alloc_workspace(self, nbytes: int, device="cuda"):

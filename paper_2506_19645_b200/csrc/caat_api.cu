@@ -117,7 +117,7 @@ Scratch scratch_layout(const caat_ctx* ctx, int K_r, int tokens, int backward) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static int layer_kr(const caat_ctx* ctx, caat_layer layer) {
-  return (layer == CAAT_ATTN_OUT ? ctx->h : ctx->ffn) / ctx->t;
+  return (layer == CAAT_ATTN_OUT ? ctx->h : ctx->ffn) / (ctx->t * ctx->groups);
 }
 
 static caat_status check_common(const caat_ctx* ctx, caat_layer layer, int tokens) {
@@ -135,7 +135,9 @@ static caat_status check_common(const caat_ctx* ctx, caat_layer layer, int token
 static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void* Y, const void* W, const void* R,
                                 const void* gamma, const void* beta, void* Hn, void* X, float* rstd, float* mean,
                                 void* ws, cudaStream_t st, int compact = 0, const void* Rs = nullptr,
-                                void* Hns = nullptr) {
+                                void* Hns = nullptr, int phase = 0) {
+  // phase: 0 = the whole layer; 1 = the GEMM only (leaves the partial sums in the scratch); 2 = the row
+  // kernel only (on what the scratch holds).  1 and 2 are the halves around a caller's all-reduce.
   // compact: R / Hn are the private parts [t, T, h - S], Rs / Hns the shared part [T, S] stored once
   const Scratch L = scratch_layout(ctx, K_r, T, 0);
   char* wsb = static_cast<char*>(ws);
@@ -145,7 +147,7 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
   const size_t e = elem_size(ctx->dtype);
   cudaError_t ce;
 
-  if (T <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r)) {
+  if (phase == 0 && T <= kDecodeMaxTokens && !ctx->no_decode && tc_gemm_usable(ctx, K_r)) {
     // few tokens (decode): the weights dominate the traffic; stream them with swapped operands and
     // let the row kernel form the rank sum from fp32 per-rank partials
     float* zt = reinterpret_cast<float*>(wsb + L.zt_off);
@@ -161,7 +163,9 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
     if (ce != cudaSuccess) return cuda_fail(ce);
     return CAAT_OK;
   }
-  if (tc_gemm_usable(ctx, K_r)) {
+  if (phase == 2) {
+    // nothing to multiply
+  } else if (tc_gemm_usable(ctx, K_r)) {
     RowparShapes sh{t, T, h, K_r, S, L.S_lo, L.S_hi, L.P};
     ce = launch_tc_forward(sh, Y, W, zs, zp, st);
     if (ce != cudaSuccess) return cuda_fail(ce);
@@ -185,6 +189,7 @@ static caat_status forward_impl(const caat_ctx* ctx, int K_r, int T, const void*
       if (ce != cudaSuccess) return cuda_fail(ce);
     }
   }
+  if (phase == 1) return CAAT_OK;
   RowFwdArgs a{zs, zp, R, gamma, beta, Hn, X, rstd, mean, t, T, h, S, L.S_lo, L.S_hi, L.P,
                (float)ctx->alpha, (float)ctx->eps, ctx->norm};
   a.compact = compact; a.Rs = Rs; a.Hns = Hns;
@@ -198,7 +203,9 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
                                  const void* W, const void* Hn, const float* rstd, const float* mean,
                                  const void* gamma, void* dY, float* dW, void* dR, float* dgamma, float* dbeta,
                                  void* ws, cudaStream_t st, int compact = 0, const void* Hns = nullptr,
-                                 const void* dHns = nullptr, void* dRs = nullptr) {
+                                 const void* dHns = nullptr, void* dRs = nullptr, int phase = 0) {
+  // phase: 0 = the whole layer; 1 = the row kernel only (dR, the shared gradient slab, the norm-parameter
+  // gradients, the scaled weight rows); 2 = the two GEMMs only, on the slab as it then stands
   // compact: Hn / dHn / dR are the private parts; the shared residual gradient dRs [T, S] is at the
   // same time the shared part of dZt, so the GEMMs read it where the caller wants it
   const Scratch L = scratch_layout(ctx, K_r, T, 1);
@@ -221,8 +228,11 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
   a.reduce_mode = ctx->bwd_reduce;
   const bool prescale = tc && ctx->alpha != 1.0 && S < h;
   if (prescale) { a.w_src = W; a.w_dst = wsb + L.wt_off; a.w_Kr = K_r; }
-  ce = launch_rows_backward(a, ctx->dtype, ctx->bwd_reduce ? 1 : ctx->direct_rows, st);
-  if (ce != cudaSuccess) return cuda_fail(ce);
+  if (phase != 2) {
+    ce = launch_rows_backward(a, ctx->dtype, ctx->bwd_reduce ? 1 : ctx->direct_rows, st);
+    if (ce != cudaSuccess) return cuda_fail(ce);
+  }
+  if (phase == 1) return CAAT_OK;
 
   if (tc) {
     RowparShapes sh{t, T, h, K_r, S, L.S_lo, L.S_hi, L.P};
@@ -270,7 +280,7 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
 // [t, T, h - S] and R0s / Hn1s / Hn2s the shared part [T, S] of the stream.
 static bool block_decode_applies(const caat_ctx* ctx, int tokens) {
   return ctx && tokens >= 1 && tokens <= kDecodeMaxTokens && !ctx->no_decode &&
-         tc_gemm_usable(ctx, ctx->h / ctx->t) && tc_gemm_usable(ctx, ctx->ffn / ctx->t);
+         tc_gemm_usable(ctx, layer_kr(ctx, CAAT_ATTN_OUT)) && tc_gemm_usable(ctx, layer_kr(ctx, CAAT_MLP_DOWN));
 }
 
 static caat_status block_decode(const caat_ctx* ctx, int tokens, const void* Y_attn, const void* W_o, const void* Y_mlp,
@@ -293,7 +303,7 @@ static caat_status block_decode(const caat_ctx* ctx, int tokens, const void* Y_a
                         Hn2, Hn2s, X2, rstd2, mean2, workspace};
   for (const void* p : ptrs)
     if (p && !aligned16(p)) return CAAT_EALIGN;
-  const int ka = ctx->h / ctx->t, km = ctx->ffn / ctx->t;
+  const int ka = layer_kr(ctx, CAAT_ATTN_OUT), km = layer_kr(ctx, CAAT_MLP_DOWN);
   const Scratch L = scratch_layout(ctx, km, tokens, 0);
   if (!workspace || workspace_bytes < L.total) return CAAT_EWORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -334,6 +344,7 @@ caat_status caat_create(int h, int ffn, int t, double p, caat_dtype dtype, caat_
   c->S = (int)std::floor((double)h * p);   // Eq. A3: l < floor(h p) is shared
   c->alpha = std::sqrt((double)t);         // Section 4: private channels times sqrt(r)
   c->norm = 0; c->eps = 1e-5; c->force_simt = 0; c->direct_rows = 0; c->no_decode = 0; c->bwd_reduce = 0;
+  c->groups = 1;
   *out = c;
   return CAAT_OK;
 }
@@ -366,6 +377,14 @@ caat_status caat_set_option(caat_ctx* ctx, caat_option opt, double value) {
     case CAAT_OPT_BACKWARD_REDUCE:
       if (value != 0.0 && value != 1.0 && value != 2.0) return CAAT_EINVAL;
       ctx->bwd_reduce = (int)value; return CAAT_OK;
+    case CAAT_OPT_TP_GROUPS: {
+      if (value != std::floor(value) || value < 1.0 || value > 65536.0) return CAAT_EINVAL;
+      const int g = (int)value;
+      if (ctx->h % (ctx->t * g) != 0 || ctx->ffn % (ctx->t * g) != 0) return CAAT_ESHAPE;
+      ctx->groups = g;
+      ctx->alpha = std::sqrt((double)ctx->t * g);   // Section 4: sqrt of the number of devices; may be overridden afterwards
+      return CAAT_OK;
+    }
   }
   return CAAT_EINVAL;
 }
@@ -675,6 +694,86 @@ caat_status caat_colpar_backward(const caat_ctx* ctx, caat_activation act, int n
   return CAAT_OK;
 }
 
+// ---- real tensor parallelism: the two halves of a layer call around the caller's all-reduce ---------
+static caat_status check_tp(const caat_ctx* ctx, caat_layer layer, int tokens, const void* ws, size_t ws_bytes,
+                            int backward) {
+  caat_status s = check_common(ctx, layer, tokens);
+  if (s != CAAT_OK) return s;
+  const int K_r = layer_kr(ctx, layer);
+  if (!tc_gemm_usable(ctx, K_r)) return CAAT_EUNSUPPORTED;   // the packed [T, S] slab exists on the tensor-core path
+  if (!ws || !aligned16(ws) || ws_bytes < scratch_layout(ctx, K_r, tokens, backward).total) return CAAT_EWORKSPACE;
+  return CAAT_OK;
+}
+
+caat_status caat_tp_slab(const caat_ctx* ctx, caat_layer layer, int tokens, int backward, size_t* offset_bytes,
+                         int* rows, int* cols) {
+  caat_status s = check_common(ctx, layer, tokens);
+  if (s != CAAT_OK) return s;
+  const int K_r = layer_kr(ctx, layer);
+  if (!tc_gemm_usable(ctx, K_r)) return CAAT_EUNSUPPORTED;
+  const Scratch L = scratch_layout(ctx, K_r, tokens, backward ? 1 : 0);
+  if (L.S_hi != ctx->S) return CAAT_EUNSUPPORTED;
+  if (offset_bytes) *offset_bytes = L.zs_off;
+  if (rows) *rows = tokens;
+  if (cols) *cols = ctx->S;
+  return CAAT_OK;
+}
+
+caat_status caat_tp_forward_local(const caat_ctx* ctx, caat_layer layer, int tokens, const void* Y, const void* W,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = check_tp(ctx, layer, tokens, workspace, workspace_bytes, 0);
+  if (s != CAAT_OK) return s;
+  if (!Y || !W) return CAAT_EINVAL;
+  if (!aligned16(Y) || !aligned16(W)) return CAAT_EALIGN;
+  return forward_impl(ctx, layer_kr(ctx, layer), tokens, Y, W, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                      nullptr, workspace, static_cast<cudaStream_t>(cuda_stream), 0, nullptr, nullptr, 1);
+}
+
+caat_status caat_tp_forward_finish(const caat_ctx* ctx, caat_layer layer, int tokens, const void* R, const void* gamma,
+                                   const void* beta, void* Hn, void* X, float* rstd, float* mean, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = check_tp(ctx, layer, tokens, workspace, workspace_bytes, 0);
+  if (s != CAAT_OK) return s;
+  if (!R || !gamma || !Hn || !X || !rstd) return CAAT_EINVAL;
+  if (ctx->norm == 1 && !mean) return CAAT_EINVAL;
+  const void* ptrs[] = {R, gamma, beta, Hn, X, rstd, mean};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  return forward_impl(ctx, layer_kr(ctx, layer), tokens, nullptr, nullptr, R, gamma, beta, Hn, X, rstd, mean, workspace,
+                      static_cast<cudaStream_t>(cuda_stream), 0, nullptr, nullptr, 2);
+}
+
+caat_status caat_tp_backward_local(const caat_ctx* ctx, caat_layer layer, int tokens, const void* dX, const void* dHn,
+                                   const void* W, const void* Hn, const float* rstd, const float* mean,
+                                   const void* gamma, void* dR, float* dgamma, float* dbeta, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream) {
+  caat_status s = check_tp(ctx, layer, tokens, workspace, workspace_bytes, 1);
+  if (s != CAAT_OK) return s;
+  if (!dX || !W || !Hn || !rstd || !gamma || !dR || !dgamma) return CAAT_EINVAL;
+  if (ctx->norm == 1 && (!mean || !dbeta)) return CAAT_EINVAL;
+  const void* ptrs[] = {dX, dHn, W, Hn, rstd, mean, gamma, dR, dgamma, dbeta};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  return backward_impl(ctx, layer_kr(ctx, layer), tokens, dX, dHn, nullptr, W, Hn, rstd, mean, gamma, nullptr, nullptr,
+                       dR, dgamma, dbeta, workspace, static_cast<cudaStream_t>(cuda_stream), 0, nullptr, nullptr,
+                       nullptr, 1);
+}
+
+caat_status caat_tp_backward_finish(const caat_ctx* ctx, caat_layer layer, int tokens, const void* Y, const void* W,
+                                    const void* dR, void* dY, float* dW, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream) {
+  caat_status s = check_tp(ctx, layer, tokens, workspace, workspace_bytes, 1);
+  if (s != CAAT_OK) return s;
+  if (!Y || !W || !dR || !dY || !dW) return CAAT_EINVAL;
+  const void* ptrs[] = {Y, W, dR, dY, dW};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return CAAT_EALIGN;
+  return backward_impl(ctx, layer_kr(ctx, layer), tokens, nullptr, nullptr, Y, W, nullptr, nullptr, nullptr, nullptr, dY,
+                       dW, const_cast<void*>(dR), nullptr, nullptr, workspace, static_cast<cudaStream_t>(cuda_stream),
+                       0, nullptr, nullptr, nullptr, 2);
+}
+
+
 caat_status caat_allreduce_bytes(const caat_ctx* ctx, int tokens, int elem_bytes, unsigned long long* payload,
                                  unsigned long long* payload_p1, unsigned long long* ring_wire) {
   if (!ctx || elem_bytes < 1) return CAAT_EINVAL;
@@ -682,7 +781,9 @@ caat_status caat_allreduce_bytes(const caat_ctx* ctx, int tokens, int elem_bytes
   const unsigned long long pay = (unsigned long long)tokens * (unsigned long long)ctx->S * (unsigned long long)elem_bytes;
   if (payload) *payload = pay;
   if (payload_p1) *payload_p1 = (unsigned long long)tokens * (unsigned long long)ctx->h * (unsigned long long)elem_bytes;
-  if (ring_wire) *ring_wire = 2ull * (unsigned long long)(ctx->t - 1) * pay / (unsigned long long)ctx->t;
+  // devices in the reduce: the t simulated ranks, or the G GPUs when the context is one group of a real run
+  const unsigned long long ndev = (unsigned long long)(ctx->groups > 1 ? ctx->groups : ctx->t);
+  if (ring_wire) *ring_wire = 2ull * (ndev - 1) * pay / ndev;
   return CAAT_OK;
 }
 

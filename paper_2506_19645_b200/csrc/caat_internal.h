@@ -19,6 +19,7 @@ struct caat_ctx {
   int direct_rows; // CAAT_OPT_ROWS
   int no_decode;   // CAAT_OPT_DECODE
   int bwd_reduce;  // CAAT_OPT_BACKWARD_REDUCE
+  int groups;      // CAAT_OPT_TP_GROUPS: this context holds t of t * groups tensor-parallel ranks
 };
 
 namespace caat {
