@@ -285,6 +285,76 @@ class MlpRunner:
         return n + sum(v.numel() * v.element_size() for v in self.out.values())
 
 
+# 8-GPU all-reduce bus bandwidth at 1 GiB measured on this pool's NVSwitch machines (nominal NVLink 5:
+# 900 GB/s per direction per GPU); NCCL's convention: time = 2 (n - 1) / n * bytes / bus bandwidth.
+NVLINK_ALLREDUCE_BUSBW_GBS = 725.0
+
+
+def tp_projection(dev, name="block_7b", steps=20):
+    """What the paper's claim looks like on this hardware: ONE GPU's share of a real t-GPU run of the block (one
+    rank per GPU), timed with the library's two halves of every layer call and no collective, next to the time
+    the four all-reduces of a step (Appendix C) would take for the analytic payload at the bandwidth above, not
+    overlapped.  A projection, labelled as such: nothing here ran on more than one GPU."""
+    from paper_2506_19645_b200 import caat
+    w0 = synthetic.WORKLOADS[name]
+    G, T, h = w0.t, w0.tokens, w0.h
+    rows = []
+    for p in (1.0, 0.75, 0.5, 0.25, 0.0):
+        ctx = caat.Context(h, w0.ffn, 1, p, "bf16")
+        ctx.set_option(caat.CAAT_OPT_TP_GROUPS, G)
+        S = ctx.shared_channels
+        if S % 8:
+            continue
+        layers = []
+        for layer in (caat.CAAT_ATTN_OUT, caat.CAAT_MLP_DOWN):
+            k = ctx.k_r(layer)
+            d = synthetic.layer_inputs(1, T, h, k, "bf16", seed=layer, S=S, backward=True, device=dev)
+            mk = lambda *sh, dt=torch.bfloat16: torch.empty(*sh, dtype=dt, device=dev)
+            o = {"Hn": mk(1, T, h), "X": mk(1, T, h), "rstd": mk(1, T, dt=torch.float32), "dY": mk(1, T, k),
+                 "dW": mk(1, h, k, dt=torch.float32), "dR": mk(1, T, h), "dg": mk(h, dt=torch.float32)}
+            layers.append((layer, d, o))
+        ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, True), device=dev)
+
+        def step():
+            for layer, d, o in layers:
+                ctx.tp_forward_local(layer, T, d["Y"], d["W"], ws)
+                ctx.tp_forward_finish(layer, T, d["R"], d["gamma"], None, o["Hn"], o["X"], o["rstd"], None, ws)
+            for layer, d, o in reversed(layers):
+                ctx.tp_backward_local(layer, T, d["dX"], d["dHn"], d["W"], o["Hn"], o["rstd"], None, d["gamma"], o["dR"],
+                                      o["dg"], None, ws)
+                ctx.tp_backward_finish(layer, T, d["Y"], d["W"], o["dR"], o["dY"], o["dW"], ws)
+
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        compute_ms = e0.elapsed_time(e1) / steps
+        ring = 2.0 * (G - 1) / G
+        ar = lambda nbytes: ring * nbytes / (NVLINK_ALLREDUCE_BUSBW_GBS * 1e9) * 1e3
+        fwd_ms = 2 * ar(T * S * 2)                       # two reduces per block forward, 16-bit payload
+        bwd16_ms, bwd32_ms = 2 * ar(T * S * 2), 2 * ar(T * S * 4)
+        rows.append({"p": p, "S": S, "compute_ms_per_gpu": compute_ms, "allreduce_ms_forward": fwd_ms,
+                     "allreduce_ms_backward_16bit": bwd16_ms, "allreduce_ms_backward_fp32": bwd32_ms,
+                     "step_ms_no_overlap": compute_ms + fwd_ms + bwd32_ms})
+        del layers, ws
+        torch.cuda.empty_cache()
+    if rows:
+        base = rows[0]["step_ms_no_overlap"]
+        for r in rows:
+            r["speedup_vs_p1"] = base / r["step_ms_no_overlap"]
+    return {"workload": name, "gpus": G, "ranks_per_gpu": 1, "tokens": T,
+            "allreduce_bus_bandwidth_gbs": NVLINK_ALLREDUCE_BUSBW_GBS,
+            "note": "projection: measured one-GPU compute (two-halves calls, no collective) + analytic all-reduce "
+                    "time (2 forward 16-bit + 2 backward fp32 reduces per block, ring factor 2(n-1)/n), no overlap; "
+                    "not a multi-GPU measurement",
+            "rows": rows}
+
+
 def make_runner(w, device, compact=False):
     return MlpRunner(w, device, compact) if w.kind == "mlp" else BlockRunner(w, device, compact)
 
@@ -591,6 +661,10 @@ def run_cuda(args):
             except Exception as ex:
                 sweep.append({"workload": name, "error": str(ex)[:200]})
         result["sweep"] = sweep
+        try:
+            result["tp_projection"] = tp_projection(dev)
+        except Exception as ex:  # noqa: BLE001
+            result["tp_projection"] = {"error": str(ex)[:200]}
     if rank == 0:
         if not args.no_cpu and world == 1:
             result["cpu_baseline"] = cpu_baseline(w)
