@@ -301,7 +301,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     // wait (bounded) for this CTA's copies still in flight before its shared memory goes away
     const long long issued = (k + NS) < total ? (k + NS) : total;
     for (long long q = k + 1; q < issued; ++q)
-      for (uint32_t it = 0; it < (1u << 20); ++it)
+      for (uint32_t it = 0; it < (1u << 10); ++it)   // each poll sleeps up to the suspend hint: ~20 ms per stage at most
         if (mbar_try(bar0 + 8u * (uint32_t)(q % NS), (uint32_t)((q / NS) & 1))) break;
   }
 }
@@ -593,7 +593,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
       atomicExch(status, 5u);
       const long long issued = (k + NS) < total ? (k + NS) : total;
       for (long long q = k + 1; q < issued; ++q)
-        for (uint32_t it = 0; it < (1u << 20); ++it)
+        for (uint32_t it = 0; it < (1u << 10); ++it)   // each poll sleeps up to the suspend hint: ~20 ms per stage at most
           if (mbar_try(bar0 + 8u * (uint32_t)(q % NS), (uint32_t)((q / NS) & 1))) break;
     }
     return;
