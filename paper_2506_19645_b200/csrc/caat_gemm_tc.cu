@@ -81,7 +81,7 @@ struct Params {
   int debug;             // measurement aid (env CAAT_TC_DEBUG; results are then wrong): 1 = no operand loads,
                          // 2 = no epilogue work at all, 4 = no A loads, 8 = no B loads; epilogue stops after the
                          // tensor-memory load (32) / after the staging stores (16); 64 = no slab barrier,
-                         // 128 = no TMA store; 512 = one lane issues all boxes of a stage; 1024 = the A boxes are
+                         // 128 = no TMA store; 512 = producer lanes take no second k-step; 1024 = the A boxes are
                          // announced to the stage barrier but never issued, so the consumers' waits run out
                          // (the timeout test: the kernel must flag it, drain and return)
 };
@@ -335,16 +335,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
 
   if (warp == 0 || warp == kProducerB) {
     // ------------------------------------------------------------ TMA producers
-    // Two single-thread producers run the same schedule: warp 0 issues the A boxes (and, in the
-    // leader CTA, posts the stage's expected bytes), warp kProducerB the B boxes.  Issuing a
-    // stage's boxes from one thread was the bottleneck of the operand pipeline (up to four boxes
-    // per stage for M-/N-major operands); two independent instruction streams halve it, and an
-    // operand that needs several boxes per stage (M-/N-major: one per 64 rows or columns) has them
-    // issued by as many lanes of its warp, each of which follows the barriers itself.
+    // Two producer warps run the same schedule: warp 0 issues the A boxes (and, in the leader CTA, posts
+    // the stage's expected bytes), warp kProducerB the B boxes.
     const bool isA = warp == 0;
-    static_assert(BM / 64 <= 32, "one lane per box");
-    const bool wide = (isA ? p.a_mn : p.b_mn) && !(p.debug & 512);
-    if (lane == 0 || wide) {
+    // Lanes of the producer warp share the issue work: lane = (k-step of a group of kKI consecutive k-steps,
+    // box of the stage).  A K-major operand is one box per stage, an M-/N-major one a box per 64 rows or
+    // columns.  All active lanes run the same instructions on different stages / boxes, so the group is
+    // issued in the time of one k-step: a single lane needs ~575 cycles per k-step (240 for the wait on a
+    // barrier that is already free, 250 for the announcement and one box, 85 of loop), more than the 384-512
+    // cycles the tensor cores take for it.
+    constexpr int kKI = 2;
+    const bool multi = (isA ? p.a_mn : p.b_mn) != 0;
+    const int nbmax = multi ? (isA ? BM / 64 : (int)(p.BN / CG) / 64) : 1;      // boxes per stage, at most
+    // measured: pays for multi-box operands (dgrad / wgrad -5...-8 %) and the weight stream of the decode
+    // path (-5 %); a K-major operand of the large GEMMs gains nothing (its tiles wait for L2, not for the
+    // issue) and a ring shorter than six stages loses more to pairwise refills than it gains
+    const int nki = ((multi || p.out_transposed) && p.nstages >= 6 && !(p.debug & 512)) ? kKI : 1;
+    const int jk = lane / nbmax, box = lane - jk * nbmax;                         // this lane's k-step slot and box
+    if (jk < nki) {
       int stage = 0; uint32_t phase = 0;
       long long issued = 0;
       bool ok = true;
@@ -356,6 +364,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         const int m0 = c.mt * BMT + (int)rank * BM, n0 = c.nt * p.BN + (int)(rank * cols_cta);
         const uint32_t tx = (uint32_t)CG * (((p.debug & 4) ? 0u : a_bytes) + ((p.debug & 8) ? 0u : b_tile_bytes));
         const bool skip = isA ? (p.debug & (4 | 1024)) != 0 : (p.debug & 8) != 0;
+        const int nb = multi ? (isA ? BM / 64 : (int)cols_cta / 64) : 1;         // boxes of this tile's stages
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
           const CUtensorMap* map = maps[isA ? u.mapA : u.mapB];
@@ -363,41 +372,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           split_range(r.splits, u, c.split, kb, ke);
           for (int q = 0; q < u.Q && ok; ++q) {
             const int z = isA ? c.b * u.a_zb + q * u.a_zq : c.b * u.b_zb + q * u.b_zq;
-            for (int kk = kb; kk < ke; ++kk) {
-              if (!mbar_wait(empty0 + 8u * stage, phase ^ 1u, abort_flag, p.spin_cap)) { ok = false; break; }
-              const uint32_t fb_local = full0 + 8u * stage;
-              // completion is signalled on the LEADER's barrier; the leader expects both CTAs' bytes
-              const uint32_t fb = CG == 2 ? mapa_rank(fb_local, 0) : fb_local;
-              const uint32_t sa = tiles_sa + (uint32_t)stage * stage_bytes, sb = sa + a_bytes;
-              if (isA && rank == 0 && lane == 0) {
-                if (p.debug & 1) mbar_arrive(fb_local); else mbar_expect_tx(fb_local, tx);
-              }
-              if (!(p.debug & 1) && !skip) {
-                auto load = [&](uint32_t dst, int x, int y) {
-                  if (CG == 2) tma_load_3d_pair(dst, map, x, y, z, fb); else tma_load_3d(dst, map, x, y, z, fb);
-                };
-                if (isA) {
-                  if (!p.a_mn) {
-                    load(sa, u.ak0 + kk * BK, m0);
-                  } else if (wide) {
-                    if (lane < BM / 64) load(sa + lane * (64 * BK * 2), u.am0 + m0 + lane * 64, u.ak0 + kk * BK);
+            for (int k0 = kb; k0 < ke; k0 += nki) {
+              const int ngrp = ke - k0 < nki ? ke - k0 : nki;      // k-steps of this group
+              if (jk < ngrp) {
+                const int kk = k0 + jk;
+                int st = stage + jk; uint32_t ph = phase;
+                if (st >= p.nstages) { st -= p.nstages; ph ^= 1u; }
+                if (!mbar_wait(empty0 + 8u * st, ph ^ 1u, abort_flag, p.spin_cap)) { ok = false; break; }
+                const uint32_t fb_local = full0 + 8u * st;
+                // completion is signalled on the LEADER's barrier; the leader expects both CTAs' bytes
+                const uint32_t fb = CG == 2 ? mapa_rank(fb_local, 0) : fb_local;
+                const uint32_t sa = tiles_sa + (uint32_t)st * stage_bytes, sb = sa + a_bytes;
+                if (isA && rank == 0 && box == 0) {
+                  if (p.debug & 1) mbar_arrive(fb_local); else mbar_expect_tx(fb_local, tx);
+                }
+                if (!(p.debug & 1) && !skip && box < nb) {
+                  auto load = [&](uint32_t dst, int x, int y) {
+                    if (CG == 2) tma_load_3d_pair(dst, map, x, y, z, fb); else tma_load_3d(dst, map, x, y, z, fb);
+                  };
+                  if (isA) {
+                    if (!p.a_mn) load(sa, u.ak0 + kk * BK, m0);
+                    else load(sa + box * (64 * BK * 2), u.am0 + m0 + box * 64, u.ak0 + kk * BK);
                   } else {
-#pragma unroll
-                    for (int ch = 0; ch < BM / 64; ++ch) load(sa + ch * (64 * BK * 2), u.am0 + m0 + ch * 64, u.ak0 + kk * BK);
-                  }
-                } else {
-                  if (!p.b_mn) {
-                    load(sb, u.bk0 + kk * BK, u.bn0 + n0);
-                  } else if (wide) {
-                    if (lane < (int)cols_cta / 64) load(sb + lane * (64 * BK * 2), u.bn0 + n0 + lane * 64, u.bk0 + kk * BK);
-                  } else {
-                    for (int ch = 0; ch < (int)cols_cta / 64; ++ch)
-                      load(sb + ch * (64 * BK * 2), u.bn0 + n0 + ch * 64, u.bk0 + kk * BK);
+                    if (!p.b_mn) load(sb, u.bk0 + kk * BK, u.bn0 + n0);
+                    else load(sb + box * (64 * BK * 2), u.bn0 + n0 + box * 64, u.bk0 + kk * BK);
                   }
                 }
               }
-              ++issued;
-              if (++stage == p.nstages) { stage = 0; phase ^= 1u; }
+              issued += ngrp;
+              stage += ngrp;
+              if (stage >= p.nstages) { stage -= p.nstages; phase ^= 1u; }
             }
           }
         }
