@@ -40,6 +40,12 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// one lane of a converged warp (the hardware's pick); branching on it keeps the control flow warp-uniform
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.u32 %0, 1, 0, P;\n}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   for (uint32_t it = 0; it < kSpinCap; ++it)
     if (mbar_try(bar, parity)) return true;
@@ -103,7 +109,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
   // its arrival; a copy landing before that only drives the byte count negative for a moment, the phase
   // cannot complete before the arrival.
   int nn = 0, mm = 0, ss = 0;
-  const int issuer = ((threadIdx.y * TX + threadIdx.x) & 31) == 0 ? (int)(threadIdx.y * TX + threadIdx.x) >> 5 : 99;
+  const int issuer = __shfl_sync(0xffffffffu, (int)(threadIdx.y * TX + threadIdx.x) >> 5, 0);   // warp index, warp-uniform
   auto issue = [&]() {
     if (nn >= my_groups) return;
     const int n = nn, m = mm, s = ss;
@@ -119,6 +125,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     const uint32_t bR = CL ? bP : (uint32_t)rowsN * a.h * ES;
     const uint32_t bS = (m == 0 && has_shared) ? (uint32_t)rowsN * a.S_hi * ES : 0u;
     const long long row = (long long)m * a.T + i0;
+    if (!elect_one()) return;
     if (issuer == 0) {
       mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS));
       if (bR) bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * (CL ? a.P : a.h) * ES, bR, bar);
@@ -338,7 +345,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
   // fetch (token group nn, rank mm) into stage ss: called by every thread, one copy per issuing warp
   // (see the forward kernel)
   int nn = 0, mm = 0, ss = 0;
-  const int issuer = (tid & 31) == 0 ? tid >> 5 : 99;
+  const int issuer = __shfl_sync(0xffffffffu, tid >> 5, 0);   // warp index, warp-uniform
   auto issue = [&]() {
     if (nn >= my_groups) return;
     const int n = nn, m = mm, s = ss;
@@ -352,6 +359,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
     const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
     const uint32_t b = (uint32_t)rowsN * a.h * ES;
     const long long off = ((long long)m * a.T + i0) * a.h * ES;
+    if (!elect_one()) return;
     if constexpr (CL) {
       const uint32_t bP = (uint32_t)rowsN * a.P * ES;                       // 0 when there is no private part
       const uint32_t bS = m == 0 ? (uint32_t)rowsN * a.S_hi * ES : 0u;      // 0 when there is no shared part
