@@ -37,8 +37,9 @@ METRIC = "CAAT block tokens/s (sim. TP=t, sync p) on 1 B200"
 
 def metric_name(w):
     return METRIC.replace("block", "MLP (column- + row-parallel half)") if w.kind == "mlp" else METRIC
-SWEEP = ["block_1p1b_p100", "block_1p1b_p075", "block_1p1b_p050", "block_1p1b_p025", "block_7b",
-         "mlp_130m", "mlp_1p1b_p050", "mlp_7b"]
+# lightest first: the 7B workloads run into the power cap and leave the GPU's clocks low for what follows
+SWEEP = ["mlp_130m", "block_1p1b_p100", "block_1p1b_p075", "block_1p1b_p050", "block_1p1b_p025", "mlp_1p1b_p050",
+         "block_7b", "mlp_7b"]
 
 
 # --------------------------------------------------------------------------- peaks
