@@ -107,3 +107,32 @@ def test_allreduce_bytes_matches_closed_form(caat):
     from oracle import caat_oracle as O
     o = O.allreduce_bytes(16384, 4096, 8, 2048, 2)
     assert o["payload_per_rank"] == a["payload_per_rank"] and o["ring_wire_per_rank"] == a["ring_wire_per_rank"]
+
+
+def test_tensor_parallel_groups_and_slab(caat):
+    # CAAT_OPT_TP_GROUPS: this context holds t of t*G ranks; K_r and alpha follow; the slab is the dense [T, S] block
+    ctx = caat.Context(4096, 11008, 1, 0.5, "bf16")
+    ctx.set_option(caat.CAAT_OPT_TP_GROUPS, 8)
+    assert ctx.k_r(caat.CAAT_ATTN_OUT) == 512 and ctx.k_r(caat.CAAT_MLP_DOWN) == 1376
+    assert ctx.private_scale == pytest.approx(8 ** 0.5)
+    with pytest.raises(caat.CaatError) as e:
+        ctx.set_option(caat.CAAT_OPT_TP_GROUPS, 3)              # 3 does not divide h
+    assert e.value.status == caat.CAAT_ESHAPE
+    with pytest.raises(caat.CaatError):
+        ctx.set_option(caat.CAAT_OPT_TP_GROUPS, 0)
+    off, rows, cols = ctypes.c_size_t(), ctypes.c_int(), ctypes.c_int()
+    for backward in (0, 1):
+        st = caat.lib.caat_tp_slab(ctx._h, caat.CAAT_MLP_DOWN, 300, backward, ctypes.byref(off), ctypes.byref(rows),
+                                   ctypes.byref(cols))
+        assert st == caat.CAAT_OK and (rows.value, cols.value) == (300, 2048) and off.value % 16 == 0
+        assert off.value + 300 * 2048 * 2 <= ctx.workspace_bytes(caat.CAAT_MLP_DOWN, 300, True)
+    # analytic ring bytes count the GPUs of the group
+    ar = ctx.allreduce_bytes(300, 2)
+    assert ar["payload_per_rank"] == 300 * 2048 * 2 and ar["ring_wire_per_rank"] == 2 * 7 * ar["payload_per_rank"] // 8
+    # no packed slab off the tensor-core path: fp32, or a partition that is not a multiple of 8
+    c32 = caat.Context(256, 1024, 2, 0.5, "f32")
+    assert caat.lib.caat_tp_slab(c32._h, caat.CAAT_MLP_DOWN, 64, 0, None, None, None) == caat.CAAT_EUNSUPPORTED
+    odd = caat.Context(4096, 11008, 8, 0.5, "bf16").set_option(caat.CAAT_OPT_SHARED_CHANNELS, 100)
+    assert caat.lib.caat_tp_slab(odd._h, caat.CAAT_MLP_DOWN, 64, 0, None, None, None) == caat.CAAT_EUNSUPPORTED
+    # the halves reject a missing workspace before any launch
+    assert caat.lib.caat_tp_forward_local(ctx._h, caat.CAAT_MLP_DOWN, 300, None, None, None, 0, None) == caat.CAAT_EWORKSPACE
