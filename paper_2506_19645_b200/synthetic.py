@@ -1,8 +1,10 @@
 """Seeded synthetic inputs shaped like the paper's workloads.
 
-This module only draws random tensors and names shapes.  It holds none of the
-method's arithmetic and imports neither the CUDA binding nor the oracle, so
-both sides of a parity test can be fed from it.
+This module only draws random tensors and names shapes.  It imports neither the
+CUDA binding nor the oracle, so both sides of a parity test can be fed from it;
+the channel partition S is not computed here: callers pass the value their side
+computed (the library's ``caat_shared_channels`` or the oracle's
+``shared_channels``) to say how many leading residual channels to tie.
 
 Recipe: one ``torch.Generator`` per workload seeded with the workload's seed;
 tensors are drawn in fp32 in the fixed order ``Y_attn, W_o, Y_mlp, W_down, R,
@@ -15,7 +17,6 @@ a rank sum).
 """
 from __future__ import annotations
 
-import math
 from dataclasses import dataclass, replace
 
 import torch
@@ -34,10 +35,6 @@ class Workload:
                     # "mlp" (column-parallel gate/up + SwiGLU, then the MLP-down layer)
     backward: bool
     seed: int = 0
-
-    @property
-    def S(self) -> int:
-        return int(math.floor(float(self.h) * float(self.p)))
 
     @property
     def kr_attn(self) -> int:
@@ -116,7 +113,7 @@ def layer_inputs(t, tokens, h, k_r, dtype="bf16", seed=0, S=0, backward=False,
     return out
 
 
-def mlp_inputs(w: Workload, tied_residual=True, device="cpu", weight_std=0.02) -> dict:
+def mlp_inputs(w: Workload, S: int, tied_residual=True, device="cpu", weight_std=0.02) -> dict:
     """Inputs of a whole MLP: per-rank normalised input X [t,T,h], gate|up weights A [t, 2 ffn/t, h],
     down weights B [t, h, ffn/t], residual R, gain, and the upstream gradients of the backward."""
     td = torch_dtype(w.dtype)
@@ -131,15 +128,16 @@ def mlp_inputs(w: Workload, tied_residual=True, device="cpu", weight_std=0.02) -
         "gamma": torch.ones(h, dtype=td, device=device),
     }
     if tied_residual:
-        tie_shared_channels(out["R"], w.S)
+        tie_shared_channels(out["R"], S)
     if w.backward:
         out["dXout"] = _randn(gen, (t, T, h), 1.0, td, device)
         out["dHn"] = _randn(gen, (t, T, h), 1.0, td, device)
     return out
 
 
-def block_inputs(w: Workload, tied_residual=True, device="cpu", weight_std=0.02) -> dict:
-    """Inputs of a block (attention-out then MLP-down) in the fixed drawing order."""
+def block_inputs(w: Workload, S: int, tied_residual=True, device="cpu", weight_std=0.02) -> dict:
+    """Inputs of a block (attention-out then MLP-down) in the fixed drawing order; S = the caller's number of
+    shared channels (the leading S channels of R0 are tied across ranks)."""
     td = torch_dtype(w.dtype)
     gen = torch.Generator(device=device)
     gen.manual_seed(w.seed)
@@ -154,7 +152,7 @@ def block_inputs(w: Workload, tied_residual=True, device="cpu", weight_std=0.02)
         "gamma2": torch.ones(h, dtype=td, device=device),
     }
     if tied_residual:
-        tie_shared_channels(out["R0"], w.S)
+        tie_shared_channels(out["R0"], S)
     if w.backward:
         out["dX1"] = _randn(gen, (t, T, h), 1.0, td, device)
         out["dX2"] = _randn(gen, (t, T, h), 1.0, td, device)

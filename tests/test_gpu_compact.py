@@ -139,7 +139,7 @@ def test_compact_rejects_unaligned_partition():
 def test_compact_block_matches_oracle():
     t, T, h, ffn, S = 4, 300, 768, 3072, 384
     w = synthetic.Workload("compact_block_case", t, T, h, ffn, 0.5, "bf16", "block", True, 31)
-    d = synthetic.block_inputs(w)
+    d = synthetic.block_inputs(w, S)
     ctx = G.make_ctx(t, h, ffn, "bf16", S=S)
     td, f32, alpha = torch.bfloat16, torch.float32, ctx.private_scale
     R0s, R0p = _split(d["R0"], S)
@@ -188,7 +188,7 @@ def test_compact_block_few_tokens(no_decode, T, t, h, ffn, S):
     # few tokens: both layers' weights stream through one swapped-operand GEMM and one row kernel walks both layers of
     # a row, here on the compact stream; the large-batch path (no_decode) must give the same block
     w = synthetic.Workload("compact_decode_case", t, T, h, ffn, S / h, "bf16", "block", False, 7 + T)
-    d = synthetic.block_inputs(w)
+    d = synthetic.block_inputs(w, S)
     ctx = G.make_ctx(t, h, ffn, "bf16", S=S, no_decode=no_decode)
     td, f32, alpha = torch.bfloat16, torch.float32, ctx.private_scale
     R0s, R0p = _split(d["R0"], S)

@@ -3,11 +3,23 @@ forward + backward through the C ABI on the full token count).
 
 The fp64 oracle cannot hold a full-size problem at once, so it walks the tokens in chunks
 (tokens are independent rows in everything except dW and dgamma, which are sums over tokens
-and are accumulated across chunks).  Compared: every forward/backward activation output on a
-seeded sample of tokens (whole rows, all ranks), dgamma in full, and dW on a seeded sample of
-(rank, channel, input) entries, each a full sum over all tokens.  Saved tensors handed to the
-GPU backward are the oracle's forward results rounded to their storage types, never GPU
-outputs."""
+and are accumulated across chunks).  Compared:
+
+* every forward/backward activation output on a STRATIFIED sample of tokens (whole rows, all
+  ranks): the first and the last row of every 128-row tile of the token axis (that also
+  covers both sides of every 256-row pair-tile edge), the ragged tail after the last full
+  tile, and a few seeded random rows - at least 256 rows in all, so every row tile of every
+  GEMM and every token group of the row kernels is touched; the 130M block compares the
+  forward outputs on ALL tokens;
+* dgamma in full;
+* dW on a stratified sample of (rank, channel, input) entries, each a full sum over all
+  tokens (hence over every split-K slice): at least one entry - the two extreme corners
+  plus random ones - in every (rank, 128-channel block, 256-input block) output tile, at
+  least 4096 entries in all.
+
+Saved tensors handed to the GPU backward are the oracle's forward results rounded to their
+storage types, never GPU outputs - except in the chained case, where the GPU backward runs
+on the GPU forward's own saved tensors while the oracle keeps to its own chain."""
 import math
 
 import numpy as np
@@ -16,7 +28,7 @@ import torch
 
 from oracle import caat_oracle as O
 from paper_2506_19645_b200 import caat, synthetic
-from tests.helpers import assert_close, f64
+from tests.helpers import assert_close, f64, stratified_entries, stratified_tokens
 
 pytestmark = pytest.mark.gpu
 
@@ -28,34 +40,22 @@ def _chunks(T):
         yield a, min(T, a + CHUNK)
 
 
-def _check_block_full(name, n_tok=48, n_dw=512, seed=123):
+def _check_block_full(name, seed=123, all_forward_rows=False, chained=False):
     w = synthetic.WORKLOADS[name]
-    t, T, h, S = w.t, w.tokens, w.h, w.S
+    t, T, h = w.t, w.tokens, w.h
+    S = O.shared_channels(h, w.p)
     alpha = math.sqrt(t)
     ka, km = w.kr_attn, w.kr_mlp
-    dev = synthetic.block_inputs(w, device="cuda")
+    dev = synthetic.block_inputs(w, S, device="cuda")
     host = {k: v.cpu() for k, v in dev.items()}
     rng = np.random.default_rng(seed)
-    tok = np.sort(rng.choice(T, size=min(n_tok, T), replace=False))
-    dws = {"attn": (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, ka, n_dw)),
-           "mlp": (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, km, n_dw))}
+    tok = stratified_tokens(T, rng)
+    assert len(tok) >= 256 or len(tok) == T
+    edge = (S - 1, S)
+    dws = {"attn": stratified_entries(t, h, ka, rng, extra_rows=edge), "mlp": stratified_entries(t, h, km, rng, extra_rows=edge)}
+    assert all(len(v[0]) >= 4096 for v in dws.values())
     Wd = {"attn": f64(host["W_o"]), "mlp": f64(host["W_down"])}
     g1, g2 = f64(host["gamma1"]), f64(host["gamma2"])
-
-    # ---------------- oracle forward, chunked; keep saved tensors (rounded) and sampled rows
-    sHn1 = torch.empty((t, T, h), dtype=torch.bfloat16); sHn2 = torch.empty_like(sHn1)
-    sr1 = torch.empty((t, T), dtype=torch.float32); sr2 = torch.empty_like(sr1)
-    fwd_s = {k: [] for k in ("Hn1", "X1", "rstd1", "Hn2", "X2", "rstd2")}
-    for a, b in _chunks(T):
-        sl = slice(a, b)
-        o = O.block_forward(f64(host["Y_attn"][:, sl]), Wd["attn"], f64(host["Y_mlp"][:, sl]), Wd["mlp"],
-                            f64(host["R0"][:, sl]), g1, g2, S=S, alpha=alpha)
-        sHn1[:, sl] = torch.from_numpy(o["Hn1"]).to(torch.bfloat16); sHn2[:, sl] = torch.from_numpy(o["Hn2"]).to(torch.bfloat16)
-        sr1[:, sl] = torch.from_numpy(o["rstd1"]).float(); sr2[:, sl] = torch.from_numpy(o["rstd2"]).float()
-        loc = tok[(tok >= a) & (tok < b)] - a
-        for k in fwd_s:
-            fwd_s[k].append(o[k][:, loc])
-    fwd_s = {k: np.concatenate(v, axis=1) for k, v in fwd_s.items()}
 
     # ---------------- GPU: the bench's launch configuration (block forward, then block backward)
     ctx = caat.Context(w.h, w.ffn, t, w.p, "bf16")
@@ -70,23 +70,47 @@ def _check_block_full(name, n_tok=48, n_dw=512, seed=123):
                       out["rstd2"], None, ws)
     torch.cuda.synchronize()
     assert ctx.last_device_status() == caat.CAAT_OK
+
+    # ---------------- oracle forward, chunked; keep saved tensors (rounded) and sampled rows
+    sHn1 = torch.empty((t, T, h), dtype=torch.bfloat16); sHn2 = torch.empty_like(sHn1)
+    sr1 = torch.empty((t, T), dtype=torch.float32); sr2 = torch.empty_like(sr1)
+    fkeys = ("Hn1", "X1", "rstd1", "Hn2", "X2", "rstd2")
+    fwd_s = {k: [] for k in fkeys}
+    for a, b in _chunks(T):
+        sl = slice(a, b)
+        o = O.block_forward(f64(host["Y_attn"][:, sl]), Wd["attn"], f64(host["Y_mlp"][:, sl]), Wd["mlp"],
+                            f64(host["R0"][:, sl]), g1, g2, S=S, alpha=alpha)
+        sHn1[:, sl] = torch.from_numpy(o["Hn1"]).to(torch.bfloat16); sHn2[:, sl] = torch.from_numpy(o["Hn2"]).to(torch.bfloat16)
+        sr1[:, sl] = torch.from_numpy(o["rstd1"]).float(); sr2[:, sl] = torch.from_numpy(o["rstd2"]).float()
+        if all_forward_rows:
+            for k in fkeys:
+                assert_close(out[k][:, sl], o[k], "bf16", f"{name}:{k}[{a}:{b}]")
+        loc = tok[(tok >= a) & (tok < b)] - a
+        for k in fkeys:
+            fwd_s[k].append(o[k][:, loc])
+    fwd_s = {k: np.concatenate(v, axis=1) for k, v in fwd_s.items()}
     tk = torch.from_numpy(tok).cuda()
-    for k in fwd_s:
+    for k in fkeys:
         assert_close(out[k].index_select(1, tk), fwd_s[k], "bf16", f"{name}:{k}")
     if not w.backward:
         return
-    del out
     bo = {"dY_attn": mk(t, T, ka), "dW_o": mk(t, h, ka, dt=f32), "dY_mlp": mk(t, T, km), "dW_down": mk(t, h, km, dt=f32),
           "dR0": mk(t, T, h), "dHn1": mk(t, T, h), "dgamma1": mk(h, dt=f32), "dgamma2": mk(h, dt=f32)}
+    if chained:       # the GPU's own saved tensors; the oracle below keeps its own
+        sv = (out["Hn1"], out["rstd1"], out["Hn2"], out["rstd2"])
+    else:
+        del out
+        sv = (sHn1.cuda(), sr1.cuda(), sHn2.cuda(), sr2.cuda())
     ctx.block_backward(T, dev["dX1"], dev["dX2"], dev["dHn2"], dev["Y_attn"], dev["W_o"], dev["Y_mlp"], dev["W_down"],
-                       sHn1.cuda(), sr1.cuda(), None, sHn2.cuda(), sr2.cuda(), None, dev["gamma1"], dev["gamma2"],
+                       sv[0], sv[1], None, sv[2], sv[3], None, dev["gamma1"], dev["gamma2"],
                        bo["dY_attn"], bo["dW_o"], bo["dY_mlp"], bo["dW_down"], bo["dR0"], bo["dHn1"], bo["dgamma1"], None,
                        bo["dgamma2"], None, ws)
     torch.cuda.synchronize()
     assert ctx.last_device_status() == caat.CAAT_OK
 
     # ---------------- oracle backward, chunked (MLP-down first, then attention-out on its dR)
-    acc = {"dgamma1": np.zeros(h), "dgamma2": np.zeros(h), "dW_attn": np.zeros(n_dw), "dW_mlp": np.zeros(n_dw)}
+    acc = {"dgamma1": np.zeros(h), "dgamma2": np.zeros(h), "dW_attn": np.zeros(len(dws["attn"][0])),
+           "dW_mlp": np.zeros(len(dws["mlp"][0]))}
     bwd_s = {k: [] for k in ("dY_attn", "dY_mlp", "dR0", "dHn1")}
     for a, b in _chunks(T):
         sl = slice(a, b)
@@ -118,7 +142,12 @@ def _check_block_full(name, n_tok=48, n_dw=512, seed=123):
 
 
 def test_full_size_block_130m():
-    _check_block_full("block_130m", n_tok=96)
+    _check_block_full("block_130m", all_forward_rows=True)
+
+
+def test_full_size_block_130m_chained():
+    # forward -> backward on the library's own saved tensors (Hn, rstd as the GPU wrote them)
+    _check_block_full("block_130m", seed=77, chained=True)
 
 
 @pytest.mark.parametrize("name", ["block_1p1b_p100", "block_1p1b_p050", "block_1p1b_p025"])
@@ -138,21 +167,23 @@ def test_full_size_block_1p1b_p075_forward_sample():
 
 
 def test_full_size_block_7b():
-    _check_block_full("block_7b", n_tok=32, n_dw=384)
+    _check_block_full("block_7b")
 
 
-def _check_mlp_full(name, n_tok=32, n_dw=384, seed=321):
+def _check_mlp_full(name, seed=321):
     """Whole MLP (column-parallel gate|up + SwiGLU, then MLP-down with partial channel-reduce) at the bench's
     size and launch sequence; the oracle walks the tokens in chunks and accumulates the token sums."""
     w = synthetic.WORKLOADS[name]
-    t, T, h, S, F = w.t, w.tokens, w.h, w.S, w.kr_mlp
+    t, T, h, F = w.t, w.tokens, w.h, w.kr_mlp
+    S = O.shared_channels(h, w.p)
     alpha = math.sqrt(t)
-    dev = synthetic.mlp_inputs(w, device="cuda")
+    dev = synthetic.mlp_inputs(w, S, device="cuda")
     host = {k: v.cpu() for k, v in dev.items()}
     rng = np.random.default_rng(seed)
-    tok = np.sort(rng.choice(T, size=min(n_tok, T), replace=False))
-    iA = (rng.integers(0, t, n_dw), rng.integers(0, 2 * F, n_dw), rng.integers(0, h, n_dw))
-    iB = (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, F, n_dw))
+    tok = stratified_tokens(T, rng)
+    iA = stratified_entries(t, 2 * F, h, rng, extra_rows=(F - 1, F))          # dA [t, 2F, h]; F = the gate | up edge
+    iB = stratified_entries(t, h, F, rng, extra_rows=(S - 1, S))              # dB [t, h, F]
+    assert len(iA[0]) >= 4096 and len(iB[0]) >= 4096
     A, B, g = f64(host["A"]), f64(host["B"]), f64(host["gamma"])
     bf, f32 = torch.bfloat16, torch.float32
 
@@ -170,6 +201,7 @@ def _check_mlp_full(name, n_tok=32, n_dw=384, seed=321):
     fwd_s = {k: np.concatenate(v, axis=1) for k, v in fwd_s.items()}
 
     ctx = caat.Context(w.h, w.ffn, t, w.p, "bf16")
+    assert ctx.shared_channels == S
     mk = lambda *s, dt=bf: torch.empty(*s, dtype=dt, device="cuda")
     out = {"pre": mk(t, T, 2 * F), "Y": mk(t, T, F), "Hn": mk(t, T, h), "X": mk(t, T, h), "rstd": mk(t, T, dt=f32)}
     ws = ctx.alloc_workspace(max(ctx.workspace_bytes(caat.CAAT_MLP_DOWN, T, True),
@@ -187,7 +219,7 @@ def _check_mlp_full(name, n_tok=32, n_dw=384, seed=321):
     bo = {"dY": mk(t, T, F), "dB": mk(t, h, F, dt=f32), "dR": mk(t, T, h), "dgamma": mk(h, dt=f32), "dX": mk(t, T, h),
           "dA": mk(t, 2 * F, h, dt=f32)}
     dY_saved = torch.empty((t, T, F), dtype=bf)
-    acc = {"dgamma": np.zeros(h), "dA": np.zeros(n_dw), "dB": np.zeros(n_dw)}
+    acc = {"dgamma": np.zeros(h), "dA": np.zeros(len(iA[0])), "dB": np.zeros(len(iB[0]))}
     bwd_s = {k: [] for k in ("dX", "dR", "dY")}
     for a, b in _chunks(T):
         sl = slice(a, b)
@@ -226,21 +258,22 @@ def test_full_size_mlp(name):
     _check_mlp_full(name)
 
 
-def _check_block_full_compact(name, n_tok=32, n_dw=384, seed=456):
+def _check_block_full_compact(name, seed=456):
     """The block on the compact residual stream (shared channels stored once) at the bench's size and launch
-    sequence: chunked oracle, sampled tokens for per-token outputs, token sums accumulated over chunks."""
+    sequence: chunked oracle, stratified tokens for per-token outputs, token sums accumulated over chunks."""
     w = synthetic.WORKLOADS[name]
-    t, T, h, S = w.t, w.tokens, w.h, w.S
+    t, T, h = w.t, w.tokens, w.h
+    S = O.shared_channels(h, w.p)
     alpha = math.sqrt(t)
     ka, km = w.kr_attn, w.kr_mlp
-    dev = synthetic.block_inputs(w, device="cuda")
+    dev = synthetic.block_inputs(w, S, device="cuda")
     host = {k: v.cpu() for k, v in dev.items()}
     split = lambda x: (x[0, :, :S].contiguous(), x[:, :, S:].contiguous())
     R0s, R0p = split(host["R0"]); dH2s, dH2p = split(host["dHn2"])
     rng = np.random.default_rng(seed)
-    tok = np.sort(rng.choice(T, size=min(n_tok, T), replace=False))
-    dws = {"attn": (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, ka, n_dw)),
-           "mlp": (rng.integers(0, t, n_dw), rng.integers(0, h, n_dw), rng.integers(0, km, n_dw))}
+    tok = stratified_tokens(T, rng)
+    edge = (S - 1, S)
+    dws = {"attn": stratified_entries(t, h, ka, rng, extra_rows=edge), "mlp": stratified_entries(t, h, km, rng, extra_rows=edge)}
     Wd = {"attn": f64(host["W_o"]), "mlp": f64(host["W_down"])}
     g1, g2 = f64(host["gamma1"]), f64(host["gamma2"])
     bf, f32 = torch.bfloat16, torch.float32
@@ -265,6 +298,7 @@ def _check_block_full_compact(name, n_tok=32, n_dw=384, seed=456):
     fwd_s = {k: np.concatenate(v, axis=tdim(k)) for k, v in fwd_s.items()}
 
     ctx = caat.Context(w.h, w.ffn, t, w.p, "bf16")
+    assert ctx.shared_channels == S
     mk = lambda *s, dt=bf: torch.empty(*s, dtype=dt, device="cuda")
     out = {"Hn1s": mk(T, S), "Hn1p": mk(t, T, h - S), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=f32),
            "Hn2s": mk(T, S), "Hn2p": mk(t, T, h - S), "X2": mk(t, T, h), "rstd2": mk(t, T, dt=f32)}
@@ -290,7 +324,8 @@ def _check_block_full_compact(name, n_tok=32, n_dw=384, seed=456):
     torch.cuda.synchronize()
     assert ctx.last_device_status() == caat.CAAT_OK
 
-    acc = {"dgamma1": np.zeros(h), "dgamma2": np.zeros(h), "dW_attn": np.zeros(n_dw), "dW_mlp": np.zeros(n_dw)}
+    acc = {"dgamma1": np.zeros(h), "dgamma2": np.zeros(h), "dW_attn": np.zeros(len(dws["attn"][0])),
+           "dW_mlp": np.zeros(len(dws["mlp"][0]))}
     bkeys = ("dY_attn", "dY_mlp", "dR0s", "dR0p", "dHn1s", "dHn1p")
     bwd_s = {k: [] for k in bkeys}
     for a, b in _chunks(T):

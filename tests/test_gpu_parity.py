@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import caat_oracle as O
 from paper_2506_19645_b200 import caat, synthetic
 from tests import gpu_harness as G
 from tests.helpers import TOL, assert_close, f64
@@ -41,7 +42,7 @@ def _check_backward(ctx, layer, d, dtype, with_dHn=True):
 # ------------------------------------------------------------------ the small fp32 configuration
 def test_config1_fp32_forward():
     w = synthetic.WORKLOADS["layer_fp32_small"]
-    d = _layer_case(w.t, w.tokens, w.h, w.kr_mlp, "f32", w.S, seed=w.seed)
+    d = _layer_case(w.t, w.tokens, w.h, w.kr_mlp, "f32", O.shared_channels(w.h, w.p), seed=w.seed)
     ctx = G.make_ctx(w.t, w.h, w.ffn, "f32", p=w.p)
     assert ctx.shared_channels == 128
     _check_forward(ctx, caat.CAAT_MLP_DOWN, d, "f32")
@@ -49,7 +50,7 @@ def test_config1_fp32_forward():
 
 def test_config1_fp32_backward_and_layernorm():
     w = synthetic.WORKLOADS["layer_fp32_small"]
-    d = _layer_case(w.t, w.tokens, w.h, w.kr_mlp, "f32", w.S, seed=1, backward=True)
+    d = _layer_case(w.t, w.tokens, w.h, w.kr_mlp, "f32", O.shared_channels(w.h, w.p), seed=1, backward=True)
     for norm in (0, 1):
         ctx = G.make_ctx(w.t, w.h, w.ffn, "f32", p=w.p, norm=norm)
         d["gamma"] = (1 + 0.1 * torch.randn(w.h, generator=torch.Generator().manual_seed(3))).float()
@@ -214,9 +215,8 @@ def test_in_place_residual_update():
 
 # ------------------------------------------------------------------ block
 def test_block_forward_backward_small():
-    from oracle import caat_oracle as O
     w = synthetic.Workload("blk", 4, 150, 768, 3072, 0.5, "bf16", "block", True, 7)
-    d = synthetic.block_inputs(w)
+    d = synthetic.block_inputs(w, O.shared_channels(w.h, w.p))
     ctx = G.make_ctx(w.t, w.h, w.ffn, "bf16", p=w.p)
     t, T, h = w.t, w.tokens, w.h
     dev = {k: v.cuda() for k, v in d.items()}
@@ -272,9 +272,8 @@ def test_few_token_forward_both_paths(no_decode, t, T, h, ffn, S, norm):
 @pytest.mark.parametrize("T,p,no_decode", [(1, 1.0, False), (8, 0.5, False), (64, 0.5, False), (64, 0.5, True), (33, 0.25, False)])
 def test_block_forward_few_tokens(T, p, no_decode):
     # block forward at decode sizes: one GEMM launch for both layers + one row kernel for both
-    from oracle import caat_oracle as O
     w = synthetic.Workload("blk_dec", 8, T, 4096, 11008, p, "bf16", "block", False, 3)
-    d = synthetic.block_inputs(w)
+    d = synthetic.block_inputs(w, O.shared_channels(w.h, w.p))
     ctx = G.make_ctx(w.t, w.h, w.ffn, "bf16", p=w.p, no_decode=no_decode)
     t, h = w.t, w.h
     dev = {k: v.cuda() for k, v in d.items()}
@@ -299,5 +298,5 @@ def test_decode_7b_forward(T, p):
     w = synthetic.WORKLOADS[f"decode_7b_T{T}_p{int(p * 100):03d}"]
     ctx = G.make_ctx(w.t, w.h, w.ffn, "bf16", p=w.p)
     for layer, k in ((caat.CAAT_ATTN_OUT, w.kr_attn), (caat.CAAT_MLP_DOWN, w.kr_mlp)):
-        d = _layer_case(w.t, T, w.h, k, "bf16", w.S, seed=T)
+        d = _layer_case(w.t, T, w.h, k, "bf16", O.shared_channels(w.h, w.p), seed=T)
         _check_forward(ctx, layer, d, "bf16")
