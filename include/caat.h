@@ -34,6 +34,14 @@
  *              atomics; rank sums run m = 0..t-1).
  *   Aliasing   Hn may alias R (in-place residual update); dR may alias dHn; nothing
  *              else may overlap.
+ *   Threads    compute calls may be made from several host threads at once (each with its
+ *              own stream and its own workspace; a context is read-only while calls run
+ *              on it and must not be reconfigured with caat_set_option meanwhile).  The
+ *              library's host-side caches are filled under a lock.  Two things are
+ *              process-wide and therefore NOT per thread or per stream: the device status
+ *              word behind caat_last_device_status (a time-out on any stream of the device
+ *              sets it; the call that reads it clears it) and the caat_profile_* benchmark
+ *              aid (one recording at a time, not thread-safe).
  *   Limits     h must be a multiple of 8 (CAAT_EUNSUPPORTED otherwise); t divides
  *              h and ffn.  The tensor-core GEMM is used for CAAT_BF16 when K_r and S
  *              are multiples of 8; other shapes run a slower CUDA-core GEMM.
@@ -158,10 +166,16 @@ caat_status caat_rowpar_forward(const caat_ctx *ctx, caat_layer layer, int token
  *              caat_workspace_bytes(ctx, layer, tokens, 0) exceeds CAAT_NOALLOC_SCRATCH_BYTES
  *              (e.g. 130M shapes, t=4, h=768, p=0.5: up to 8738 tokens per call).
  *   Set-up     the first call on each device looks up the scratch array's device address
- *              (once per device, with that device current).  Make that first call before
- *              starting any CUDA stream capture on the device.
- *   Allocation the call itself performs no cudaMalloc / cudaFree and calls no allocating
- *              library routine.
+ *              (once per device, with that device current).  With CUDA's lazy module loading
+ *              that lookup is also the moment the driver loads this part of the library onto
+ *              the device and reserves the array there, so the FIRST call per device can
+ *              take device memory and can fail with CAAT_ECUDA when none is left
+ *              (caat_last_cuda_error() has the text).  Make that first call at start-up:
+ *              before the memory pool is frozen and before starting any CUDA stream capture
+ *              on the device.  The address is cached per device ordinal for the life of the
+ *              process; after a cudaDeviceReset the library must not be used again.
+ *   Allocation after that first call per device, a call performs no cudaMalloc / cudaFree and
+ *              calls no allocating library routine.
  *   Sharing    all calls on a device use the same array, which keeps whatever the last call
  *              left in it.  Nothing in it needs to start at zero (every element that is read
  *              is written earlier in the same call).  Two calls that overlap on the GPU

@@ -17,14 +17,20 @@ void* g_scratch_ptr[kMaxDevices] = {};   // device address of g_noalloc_scratch,
 
 // In host code the array's name is only a handle: the address kernels must be given is the one
 // cudaGetSymbolAddress returns for the CURRENT device.  Looked up once per device.
+// (With lazy module loading that first lookup is also what makes the driver load this file's device
+// image and reserve the array on the device: it can fail for lack of memory, and it is the reason
+// the first call per device belongs at start-up.)
 caat_status scratch_address(void** out) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CAAT_ECUDA;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return caat::cuda_fail(e);
+  if (dev < 0 || dev >= kMaxDevices) return caat::cuda_fail(cudaErrorInvalidDevice);
   std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (g_scratch_ptr[dev] == nullptr) {
     void* p = nullptr;
-    const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
-    if (e != cudaSuccess || p == nullptr) return CAAT_ECUDA;
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess) return caat::cuda_fail(e);
+    if (p == nullptr) return caat::cuda_fail(cudaErrorInvalidSymbol);
     g_scratch_ptr[dev] = p;
   }
   *out = g_scratch_ptr[dev];
