@@ -7,10 +7,13 @@ norm) followed, for training workloads, by the block backward.  The t tensor-par
 ranks are simulated as a batch dimension on one GPU.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+  python -m torch.distributed.run ... bench.py --gpus N --mode tp      (real tensor parallelism, p sweep)
 
 Prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) every GPU
-runs an independent replica of the workload (the path has no cross-GPU exchange step):
-weak scaling, no data-path collective; time is the max over ranks.
+runs an independent replica of the workload (the path as benchmarked has no cross-GPU
+exchange step): weak scaling, no data-path collective; time is the max over ranks.
+``--mode tp`` instead splits the tensor-parallel ranks over the GPUs and exchanges the
+shared-channel slab with an all-reduce (the paper's partial channel-reduce).
 """
 from __future__ import annotations
 
@@ -19,7 +22,6 @@ import json
 import math
 import os
 import statistics
-import subprocess
 import sys
 import threading
 import time
@@ -31,31 +33,44 @@ import torch  # noqa: E402
 
 from paper_2506_19645_b200 import replicas, synthetic  # noqa: E402
 
-DEFAULT_WORKLOAD = "block_130m"
+# The metric is quoted on no single configuration: the headline line is the largest one that fits a GPU.
+DEFAULT_WORKLOAD = "block_7b"
 METRIC = "CAAT block tokens/s (sim. TP=t, sync p) on 1 B200"
 
 
 def metric_name(w):
-    return METRIC.replace("block", "MLP (column- + row-parallel half)") if w.kind == "mlp" else METRIC
-# lightest first: the 7B workloads run into the power cap and leave the GPU's clocks low for what follows
-SWEEP = ["mlp_130m", "block_1p1b_p100", "block_1p1b_p075", "block_1p1b_p050", "block_1p1b_p025", "mlp_1p1b_p050",
-         "block_7b", "mlp_7b"]
+    if w.kind == "mlp":
+        return METRIC.replace("block", "MLP (column- + row-parallel half)")
+    if w.kind == "layer":
+        return METRIC.replace("block", "row-parallel layer")
+    return METRIC
+
+
+# every configuration the metric is defined on, lightest first: the 7B workloads run into the power cap and
+# leave the GPU's clocks low for what follows
+SWEEP = (["layer_fp32_small"] + [f"decode_7b_T{T}_p{p}" for T in (1, 8, 64) for p in ("100", "050")] +
+         ["block_130m", "mlp_130m", "block_1p1b_p100", "block_1p1b_p075", "block_1p1b_p050", "block_1p1b_p025",
+          "mlp_1p1b_p050", "block_7b", "mlp_7b"])
 
 
 # --------------------------------------------------------------------------- peaks
 def measured_peaks():
+    """Roofline denominators: the copy bandwidth and the two cuBLAS bf16 figures measured on this machine (a burst
+    figure for a kernel timed alone, a sustained one for kernels timed inside a long, power-capped step)."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
             d = json.load(f)
-        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
-                "source": "measured (MEASURED_PEAKS.json; sustained bf16 figure: kernels timed inside a long step)"}
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops_burst": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "of measured (MEASURED_PEAKS.json)"}
     except Exception:
-        return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback (earlier measurement on this pool)"}
+        return {"hbm_gbs": 6650.0, "bf16_tflops_burst": 1590.0, "bf16_tflops_sustained": 1400.0,
+                "source": "of fallback (earlier measurement on this pool)"}
 
 
 def recorded_traffic(kernel: str, workload: str):
-    """DRAM bytes per launch from a committed ncu capture (profiles/traffic.json), else None."""
+    """DRAM bytes per step of one kernel kind from a committed ncu capture (profiles/traffic.json), else None."""
     try:
         with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
             return json.load(f).get(workload, {}).get(kernel)
@@ -107,31 +122,40 @@ class ClockSampler:
             self._thread.join()
         if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+        return {"sm_mhz": statistics.median(self.samples), "sm_min_mhz": min(self.samples), "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
 # --------------------------------------------------------------------------- algorithmic work
-def layer_work(w, k_r, backward, compact=False):
-    """Algorithmic flops and bytes of ONE layer per kernel kind (inputs read once, outputs
-    written once, given the kernel's interface; e = 2 bytes).  compact: the residual stream and
-    its gradient are stored shared-once + private-per-rank, like the scratch."""
-    t, T, h, S, e = w.t, w.tokens, w.h, w.S, 2
+def esize(w):
+    return 4 if w.dtype == "f32" else 2
+
+
+def layer_work(w, S, k_r, compact=False):
+    """Work of ONE layer per kernel kind.  "bytes" is the ALGORITHMIC traffic of the step the kernel
+    performs: tensors of the method read once and written once - no scratch (the GEMM's partial sums, the
+    reduced gradient slab) and no saved statistics.  "bytes_interface" adds what the kernel's own interface
+    makes it move on top (scratch in or out, rstd), for reference only.  compact: the residual stream and its
+    gradient are stored shared-once + private-per-rank."""
+    t, T, h, e = w.t, w.tokens, w.h, esize(w)
     K = k_r * t
     zsz = (T * S + t * T * (h - S)) * e            # split scratch: shared once, private per rank
     full = t * T * h * e
     stream = zsz if compact else full              # one tensor of the residual stream
+    fl = 2.0 * T * K * h
     out = {
-        "tc_gemm_forward": {"flops": 2.0 * T * K * h, "bytes": (T * K + K * h) * e + zsz},
-        "rows_forward": {"flops": 0.0, "bytes": zsz + 2 * stream + full + t * T * 4},
+        "tc_gemm_forward": {"flops": fl, "bytes": (T * K + K * h) * e, "bytes_interface": (T * K + K * h) * e + zsz},
+        # R in, Hn and X out
+        "rows_forward": {"flops": 0.0, "bytes": 2 * stream + full, "bytes_interface": zsz + 2 * stream + full + t * T * 4},
     }
-    if backward:
-        # reads dX, Hn, dHn; writes dR and the reduced shared gradient gs [T, S] (compact: gs is dRs, part of dR).
-        # The GEMMs read the private gradient from dR itself: no scaled copy is written.
-        bwd_out = stream if compact else stream + T * S * e
-        out["rows_backward"] = {"flops": 0.0, "bytes": full + 2 * stream + bwd_out + t * T * 4}
-        out["tc_gemm_dgrad"] = {"flops": 2.0 * T * K * h, "bytes": zsz + K * h * e + T * K * e}
-        out["tc_gemm_wgrad"] = {"flops": 2.0 * T * K * h, "bytes": zsz + T * K * e + K * h * 4}
+    if w.backward:
+        # dX, Hn, dHn in, dR out; the interface also writes the reduced shared gradient gs [T, S] (compact: gs is
+        # dRs, part of dR) and reads rstd
+        gs = 0 if compact else T * S * e
+        out["rows_backward"] = {"flops": 0.0, "bytes": full + 3 * stream, "bytes_interface": full + 3 * stream + gs + t * T * 4}
+        # W in, dY out / Y in, dW (fp32) out; the gradient operand is dR and the slab, already counted above
+        out["tc_gemm_dgrad"] = {"flops": fl, "bytes": (K * h + T * K) * e, "bytes_interface": zsz + (K * h + T * K) * e}
+        out["tc_gemm_wgrad"] = {"flops": fl, "bytes": T * K * e + K * h * 4, "bytes_interface": zsz + T * K * e + K * h * 4}
     return out
 
 
@@ -139,39 +163,49 @@ def colpar_work(w):
     """Algorithmic work of the column-parallel MLP half (gate|up GEMM per rank + SwiGLU), e = 2 bytes."""
     t, T, h, F, e = w.t, w.tokens, w.h, w.kr_mlp, 2
     fl = 2.0 * t * T * h * 2 * F
-    out = {"tc_gemm_forward": {"flops": fl, "bytes": (t * T * h + t * 2 * F * h + t * T * 2 * F) * e},
-           "activation": {"flops": 0.0, "bytes": t * T * 3 * F * e}}
+    b_f = (t * T * h + t * 2 * F * h + t * T * 2 * F) * e
+    out = {"tc_gemm_forward": {"flops": fl, "bytes": b_f, "bytes_interface": b_f},
+           "activation": {"flops": 0.0, "bytes": t * T * 3 * F * e, "bytes_interface": t * T * 3 * F * e}}
     if w.backward:
         out["activation"]["bytes"] += t * T * 5 * F * e
-        out["tc_gemm_dgrad"] = {"flops": fl, "bytes": (t * T * 2 * F + t * 2 * F * h + t * T * h) * e}
-        out["tc_gemm_wgrad"] = {"flops": fl, "bytes": (t * T * 2 * F + t * T * h) * e + t * 2 * F * h * 4}
+        out["activation"]["bytes_interface"] += t * T * 5 * F * e
+        b_d = (t * T * 2 * F + t * 2 * F * h + t * T * h) * e
+        b_w = (t * T * 2 * F + t * T * h) * e + t * 2 * F * h * 4
+        out["tc_gemm_dgrad"] = {"flops": fl, "bytes": b_d, "bytes_interface": b_d}
+        out["tc_gemm_wgrad"] = {"flops": fl, "bytes": b_w, "bytes_interface": b_w}
     return out
 
 
-def step_work(w, compact=False):
+def layer_widths(w):
+    return (w.kr_mlp,) if w.kind in ("mlp", "layer") else (w.kr_attn, w.kr_mlp)
+
+
+def step_work(w, S, compact=False):
     tot = {}
-    parts = [layer_work(w, k_r, w.backward, compact) for k_r in ((w.kr_mlp,) if w.kind == "mlp" else (w.kr_attn, w.kr_mlp))]
+    parts = [layer_work(w, S, k_r, compact) for k_r in layer_widths(w)]
     if w.kind == "mlp":
         parts.append(colpar_work(w))
     for part in parts:
         for kind, v in part.items():
-            a = tot.setdefault(kind, {"flops": 0.0, "bytes": 0.0})
-            a["flops"] += v["flops"]
-            a["bytes"] += v["bytes"]
+            a = tot.setdefault(kind, {"flops": 0.0, "bytes": 0.0, "bytes_interface": 0.0})
+            for k in a:
+                a[k] += v[k]
+    if w.dtype == "f32":      # fp32 runs the CUDA-core GEMM (TF32 cannot meet the 1e-4 tolerance)
+        tot["gemm_cuda_core"] = tot.pop("tc_gemm_forward")
     return tot
 
 
-def paper_level_work(w, compact=False):
+def paper_level_work(w, S, compact=False):
     """Whole-path algorithmic work per step (no scratch traffic): the roofline of the path."""
-    t, T, h, e = w.t, w.tokens, w.h, 2
+    t, T, h, e = w.t, w.tokens, w.h, esize(w)
     full = t * T * h
-    stream = T * w.S + t * T * (h - w.S) if compact else full
+    stream = T * S + t * T * (h - S) if compact else full
     fl = by = 0.0
     if w.kind == "mlp":   # column-parallel half: X, A in; pre kept for the backward; dX, dA out
         F = w.kr_mlp
         fl += 2.0 * t * T * h * 2 * F * (3 if w.backward else 1)
         by += e * (full + t * 2 * F * h + t * T * 2 * F) + (e * (t * T * 2 * F + full) + 4 * t * 2 * F * h if w.backward else 0)
-    for k_r in ((w.kr_mlp,) if w.kind == "mlp" else (w.kr_attn, w.kr_mlp)):
+    for k_r in layer_widths(w):
         K = k_r * t
         fl += 2.0 * T * K * h
         by += e * (T * K + K * h + 2 * stream + full)
@@ -181,25 +215,21 @@ def paper_level_work(w, compact=False):
     return fl, by
 
 
-def r_w_compact_ok(w):
-    """The compact-layout entry points need a partition on a 16-byte boundary."""
-    return w.S % 8 == 0
-
-
 # --------------------------------------------------------------------------- the CUDA arm
 class BlockRunner:
     def __init__(self, w, device, compact=False):
         from paper_2506_19645_b200 import caat
         self.caat, self.w, self.dev, self.compact = caat, w, device, compact
         self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
-        self.inp = synthetic.block_inputs(w, device=device)
+        self.S = self.ctx.shared_channels
+        self.inp = synthetic.block_inputs(w, self.S, device=device)
         t, T, h = w.t, w.tokens, w.h
         td = self.ctx.torch_dtype
         mk = lambda *s, dt=td: torch.empty(*s, dtype=dt, device=device)
         f32 = torch.float32
         if compact:
             # same synthetic block, with the (tied) shared channels of the stream kept once
-            S, i = w.S, self.inp
+            S, i = self.S, self.inp
             for name in ("R0", "dHn2"):
                 if name in i:
                     x = i.pop(name)
@@ -250,6 +280,29 @@ class BlockRunner:
         return n + sum(v.numel() * v.element_size() for v in self.out.values())
 
 
+class LayerRunner:
+    """One MLP-down-like row-parallel layer, forward only (the small fp32 configuration)."""
+
+    def __init__(self, w, device, compact=False):
+        from paper_2506_19645_b200 import caat
+        assert not compact and not w.backward
+        self.caat, self.w, self.dev, self.compact = caat, w, device, False
+        self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
+        self.S = self.ctx.shared_channels
+        d = synthetic.layer_inputs(w.t, w.tokens, w.h, w.kr_mlp, w.dtype, seed=w.seed, S=self.S, device=device)
+        self.inp = {k: d[k] for k in ("Y", "W", "R", "gamma")}
+        self.out = self.ctx.alloc_forward_outputs(w.tokens, device=device)
+        self.out = {k: v for k, v in self.out.items() if v is not None}
+        self.ws = self.ctx.alloc_workspace(self.ctx.workspace_bytes(caat.CAAT_MLP_DOWN, w.tokens, False), device=device)
+
+    def step(self):
+        i, o = self.inp, self.out
+        self.ctx.rowpar_forward(self.caat.CAAT_MLP_DOWN, self.w.tokens, i["Y"], i["W"], i["R"], i["gamma"], None, o["Hn"],
+                                o["X"], o["rstd"], None, self.ws)
+
+    touched_bytes = BlockRunner.touched_bytes
+
+
 class MlpRunner:
     """The whole tensor-parallel MLP: column-parallel gate|up + SwiGLU, then the MLP-down layer with partial
     channel-reduce (and the gradient of both), as two library calls per direction."""
@@ -259,7 +312,8 @@ class MlpRunner:
         assert not compact
         self.caat, self.w, self.dev, self.compact = caat, w, device, False
         self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
-        self.inp = synthetic.mlp_inputs(w, device=device)
+        self.S = self.ctx.shared_channels
+        self.inp = synthetic.mlp_inputs(w, self.S, device=device)
         t, T, h, F = w.t, w.tokens, w.h, w.kr_mlp
         td, f32 = self.ctx.torch_dtype, torch.float32
         mk = lambda *s, dt=td: torch.empty(*s, dtype=dt, device=device)
@@ -281,21 +335,22 @@ class MlpRunner:
                                      i["gamma"], o["dY"], o["dB"], o["dR"], o["dgamma"], None, self.ws)
             self.ctx.colpar_backward(c.CAAT_ACT_SWIGLU, 2 * F, T, o["dY"], i["X"], i["A"], o["pre"], o["dX"], o["dA"], self.ws)
 
-    def touched_bytes(self):
-        n = sum(v.numel() * v.element_size() for v in self.inp.values())
-        return n + sum(v.numel() * v.element_size() for v in self.out.values())
+    touched_bytes = BlockRunner.touched_bytes
 
 
-# 8-GPU all-reduce bus bandwidth at 1 GiB measured on this pool's NVSwitch machines (nominal NVLink 5:
-# 900 GB/s per direction per GPU); NCCL's convention: time = 2 (n - 1) / n * bytes / bus bandwidth.
+# The 8-GPU all-reduce bus bandwidth quoted for this pool's NVSwitch machines at a 1 GiB payload (nominal NVLink 5:
+# 900 GB/s per direction per GPU).  NOT measured by this repository (no run here had more than one GPU); the
+# payloads below are 17-134 MB, where a real collective reaches less, so the all-reduce times are lower bounds.
+# NCCL's convention: time = 2 (n - 1) / n * bytes / bus bandwidth.
 NVLINK_ALLREDUCE_BUSBW_GBS = 725.0
 
 
 def tp_projection(dev, name="block_7b", steps=20):
-    """What the paper's claim looks like on this hardware: ONE GPU's share of a real t-GPU run of the block (one
-    rank per GPU), timed with the library's two halves of every layer call and no collective, next to the time
-    the four all-reduces of a step (Appendix C) would take for the analytic payload at the bandwidth above, not
-    overlapped.  A projection, labelled as such: nothing here ran on more than one GPU."""
+    """What the paper's claim looks like on this hardware, PROJECTED: ONE GPU's share of a real t-GPU run of the
+    two row-parallel sub-layers of a block (one rank per GPU; no attention, no column-parallel GEMMs), timed with
+    the library's two halves of every layer call and no collective, next to the time the four all-reduces of a
+    step (Appendix C) would take for the analytic payload at the bandwidth above, not overlapped.  Nothing here
+    ran on more than one GPU; `bench.py --mode tp` is the measurement."""
     from paper_2506_19645_b200 import caat
     w0 = synthetic.WORKLOADS[name]
     G, T, h = w0.t, w0.tokens, w0.h
@@ -348,16 +403,23 @@ def tp_projection(dev, name="block_7b", steps=20):
         base = rows[0]["step_ms_no_overlap"]
         for r in rows:
             r["speedup_vs_p1"] = base / r["step_ms_no_overlap"]
-    return {"workload": name, "gpus": G, "ranks_per_gpu": 1, "tokens": T,
+    return {"title": "row-parallel sub-layers only, projected", "workload": name, "gpus": G, "ranks_per_gpu": 1, "tokens": T,
             "allreduce_bus_bandwidth_gbs": NVLINK_ALLREDUCE_BUSBW_GBS,
-            "note": "projection: measured one-GPU compute (two-halves calls, no collective) + analytic all-reduce "
-                    "time (2 forward 16-bit + 2 backward fp32 reduces per block, ring factor 2(n-1)/n), no overlap; "
-                    "not a multi-GPU measurement",
+            "allreduce_bus_bandwidth_source": "figure quoted for this pool's 8-GPU NVSwitch machines at 1 GiB; nominal for "
+                                              "this repository (never measured here), optimistic at these 17-134 MB payloads",
+            "note": "projection: measured one-GPU compute of the two row-parallel sub-layers (two-halves calls, no "
+                    "collective; no attention or column-parallel GEMMs, so not comparable with whole-model speed-ups) + "
+                    "analytic all-reduce time (2 forward 16-bit + 2 backward fp32 reduces per block, ring factor "
+                    "2(n-1)/n), no overlap; not a multi-GPU measurement",
             "rows": rows}
 
 
 def make_runner(w, device, compact=False):
-    return MlpRunner(w, device, compact) if w.kind == "mlp" else BlockRunner(w, device, compact)
+    if w.kind == "mlp":
+        return MlpRunner(w, device, compact)
+    if w.kind == "layer":
+        return LayerRunner(w, device, compact)
+    return BlockRunner(w, device, compact)
 
 
 def capture_step(runner):
@@ -393,41 +455,143 @@ def buffer_sets_needed(touched_bytes):
     two uses of a set."""
     if touched_bytes >= 2 * L2_BYTES:
         return 1
-    return min(16, int(2 * L2_BYTES // max(touched_bytes, 1)) + 2)
+    return min(128, int(2 * L2_BYTES // max(touched_bytes, 1)) + 2)
 
 
-def time_steps(runner, steps, dist_on, graph=None):
+def time_steps(runner, steps, dist_on, graph=None, per_step=False):
     """Device time of exactly `steps` steps (ms), CUDA events on the launching stream.  `runner` and
-    `graph` may be lists (buffer sets rotated step by step)."""
+    `graph` may be lists (buffer sets rotated step by step).  per_step: also an event after every step;
+    returns (total, [per-step ms])."""
     runners = runner if isinstance(runner, list) else [runner]
     graphs = graph if isinstance(graph, list) else ([graph] if graph is not None else None)
     torch.cuda.synchronize()
     if dist_on:
         torch.distributed.barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1 if per_step else 2)]
+    ev[0].record()
     for q in range(steps):
         if graphs is not None:
             graphs[q % len(graphs)].replay()
         else:
             runners[q % len(runners)].step()
-    e1.record()
+        if per_step:
+            ev[q + 1].record()
+    if not per_step:
+        ev[1].record()
     torch.cuda.synchronize()
     if dist_on:
         torch.distributed.barrier()
-    return e0.elapsed_time(e1)
+    total = ev[0].elapsed_time(ev[-1])
+    if per_step:
+        return total, [ev[q].elapsed_time(ev[q + 1]) for q in range(steps)]
+    return total
+
+
+def step_stats(per_step_ms):
+    s = sorted(per_step_ms)
+    return {"median": statistics.median(s), "min": s[0], "max": s[-1], "n": len(s)}
+
+
+def kernel_table(prof, work, steps, peaks):
+    """Per kernel kind: device time per step from CUDA events around every launch, and the achieved rate on the
+    kind's algorithmic work against the peak that bounds it (both bf16 denominators named)."""
+    total = sum(v[0] for v in prof.values()) or 1.0
+    kernels = {}
+    for kind, (kms, n) in prof.items():
+        per_step_ms = kms / steps
+        ent = {"ms_per_step": per_step_ms, "launches_per_step": n / steps, "share": kms / total}
+        wk = work.get(kind)
+        if wk and per_step_ms > 0:
+            sec = per_step_ms * 1e-3
+            gbs, tfs = wk["bytes"] / sec / 1e9, wk["flops"] / sec / 1e12
+            t_hbm = wk["bytes"] / (peaks["hbm_gbs"] * 1e9)
+            t_tc = wk["flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
+            if t_tc > t_hbm:
+                ent.update({"bound": "tensor", "achieved": tfs, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                            "frac": tfs / peaks["bf16_tflops_sustained"], "peak_name": "bf16_tflops_sustained",
+                            "frac_of_burst_peak": tfs / peaks["bf16_tflops_burst"]})
+            else:
+                ent.update({"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": gbs / peaks["hbm_gbs"], "peak_name": "hbm_gbs",
+                            "interface_gbs": wk["bytes_interface"] / sec / 1e9})
+            ent["algorithmic_bytes_per_step"], ent["flops_per_step"] = wk["bytes"], wk["flops"]
+        kernels[kind] = ent
+    return kernels
+
+
+def path_roofline(w, S, compact, ms_step, peaks):
+    fl, by = paper_level_work(w, S, compact)
+    t_hbm = by / (peaks["hbm_gbs"] * 1e9) * 1e3
+    t_sus = fl / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
+    t_bur = fl / (peaks["bf16_tflops_burst"] * 1e12) * 1e3
+    return {"flops_per_step": fl, "bytes_per_step": by, "bound": "tensor" if t_sus > t_hbm else "hbm",
+            "roofline_ms": max(t_sus, t_hbm), "frac": max(t_sus, t_hbm) / ms_step,
+            "roofline_ms_burst_peak": max(t_bur, t_hbm), "frac_burst_peak": max(t_bur, t_hbm) / ms_step,
+            "hbm_ms": t_hbm, "tensor_ms_sustained": t_sus, "tensor_ms_burst": t_bur,
+            "denominators": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
+                             "bf16_tflops_burst": peaks["bf16_tflops_burst"], "source": peaks["source"]}}
+
+
+def measure(w, dev, steps, warm, dist_on, compact=False, no_graph=False, kernels=True):
+    """Everything the bench reports about one workload on this GPU: the timed pass of exactly `steps` steps, a pass
+    with an event after every step (median / min), a pass with events around every kernel, and - for working sets
+    that fit the L2 - the same steps on one buffer set.  Returns (dict, runner)."""
+    from paper_2506_19645_b200 import caat
+    runner = make_runner(w, dev, compact)
+    for _ in range(warm):
+        runner.step()
+    torch.cuda.synchronize()
+    assert runner.ctx.last_device_status() == caat.CAAT_OK
+    # small working sets (decode: the weights are about one L2) rotate over several buffer sets
+    nsets = buffer_sets_needed(runner.touched_bytes())
+    rset = [runner] + [make_runner(w, dev, compact) for _ in range(nsets - 1)]
+    for r in rset[1:]:
+        r.step()
+    torch.cuda.synchronize()
+    # launch-bound steps (decode: tens of microseconds) are replayed from a CUDA graph
+    graph, per_step = None, 0
+    probe = time_steps(rset, 5, False) / 5
+    if probe < 0.25 and not no_graph:
+        caps = [capture_step(r) for r in rset]
+        if all(g is not None for g, _ in caps):
+            graph, per_step = [g for g, _ in caps], caps[0][1]
+    l0 = caat.kernel_launches()
+    ms = time_steps(rset, steps, dist_on, graph)
+    launches = per_step * steps if graph is not None else caat.kernel_launches() - l0
+    _, each = time_steps(rset, steps, False, graph, per_step=True)
+    out = {"ms_total": ms, "launches": int(launches), "step_ms": step_stats(each), "nsets": nsets,
+           "graph": graph is not None, "touched_bytes": runner.touched_bytes()}
+    if kernels:
+        # second pass of the same K steps with CUDA events around every kernel (per-kernel device times)
+        caat.profile_begin(max(1024, (launches if graph is None else 64 * steps) + 64))
+        ms_prof = time_steps(rset, steps, False)
+        out["prof"], out["ms_prof"] = caat.profile_end(), ms_prof
+    if nsets > 1:
+        # the same steps on ONE buffer set, i.e. with whatever fits staying in L2 (reported separately)
+        out["ms_warm_l2"] = time_steps(rset[:1], steps, False, graph[:1] if graph is not None else None) / steps
+    del rset[1:], graph
+    return out, runner
+
+
+def l2_note(m):
+    tb = m["touched_bytes"] / 1e6
+    if m["nsets"] == 1:
+        return f"inputs+outputs touched per step {tb:.0f} MB > 126 MB L2"
+    return (f"{m['nsets']} buffer sets rotated step by step: {tb:.1f} MB touched per step, "
+            f"{(m['nsets'] - 1) * tb:.0f} MB of other sets between two uses of a set (L2 126 MB)")
 
 
 def e2e_leg(runner, steps):
     """Same step through the public API with HOST buffers: every step copies its inputs from pinned
-    host memory and reads its results back to the host, all inside the timed region.  The three
+    host memory and reads its results back to pinned host memory, all inside the timed region.  The three
     phases run on three streams over two sets of device buffers, so the copy of step s+1, the
     kernels of step s and the read-back of step s-1 overlap (PCIe moves both ways at once)."""
     runners = [runner, make_runner(runner.w, runner.dev, runner.compact)]
     inp_host = {k: v.cpu().pin_memory() for k, v in runner.inp.items()}
-    out_host = [{k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in runner.out.items()} for _ in range(2)]
+    # one host copy of the results: read-backs are serialised on their stream, each step overwrites the last
+    out_host = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in runner.out.items()}
     h2d = sum(v.numel() * v.element_size() for v in inp_host.values())
-    d2h = sum(v.numel() * v.element_size() for v in out_host[0].values())
+    d2h = sum(v.numel() * v.element_size() for v in out_host.values())
     s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
     ev_in = [None, None]    # inputs of the buffer set are on the device
     ev_run = [None, None]   # its step has run
@@ -451,7 +615,7 @@ def e2e_leg(runner, steps):
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_run[b])
             for k, v in r.out.items():
-                out_host[b][k].copy_(v, non_blocking=True)
+                out_host[k].copy_(v, non_blocking=True)
             ev_out[b] = s_out.record_event()
 
     for q in range(2):
@@ -471,19 +635,25 @@ def e2e_leg(runner, steps):
 
 
 def oracle_sample_run(w, sample_tokens):
-    """One block forward(+backward) of the fp64 oracle on `sample_tokens` tokens of the workload."""
+    """One forward(+backward) of the fp64 oracle on `sample_tokens` tokens of the workload."""
     from oracle import caat_oracle as O
     ws = w.with_tokens(sample_tokens)
-    S, alpha = ws.S, math.sqrt(ws.t)
+    S, alpha = O.shared_channels(ws.h, ws.p), math.sqrt(ws.t)
     if w.kind == "mlp":
-        d = {k: v.to(torch.float64).numpy() for k, v in synthetic.mlp_inputs(ws, device="cpu").items()}
+        d = {k: v.to(torch.float64).numpy() for k, v in synthetic.mlp_inputs(ws, S, device="cpu").items()}
         t0 = time.perf_counter()
         f = O.mlp_forward(d["X"], d["A"], d["B"], d["R"], d["gamma"], S=S, alpha=alpha)
         if w.backward:
             O.mlp_backward(d["dXout"], d["dHn"], d["X"], d["A"], d["B"], f["pre"], f["Y"], f["Hn"], f["rstd"], None,
                            d["gamma"], S=S, alpha=alpha)
         return time.perf_counter() - t0
-    d = {k: v.to(torch.float64).numpy() for k, v in synthetic.block_inputs(ws, device="cpu").items()}
+    if w.kind == "layer":
+        d = {k: v.to(torch.float64).numpy() for k, v in
+             synthetic.layer_inputs(ws.t, ws.tokens, ws.h, ws.kr_mlp, ws.dtype, seed=ws.seed, S=S).items()}
+        t0 = time.perf_counter()
+        O.rowpar_forward(d["Y"], d["W"], d["R"], d["gamma"], None, S=S, alpha=alpha)
+        return time.perf_counter() - t0
+    d = {k: v.to(torch.float64).numpy() for k, v in synthetic.block_inputs(ws, S, device="cpu").items()}
     t0 = time.perf_counter()
     f = O.block_forward(d["Y_attn"], d["W_o"], d["Y_mlp"], d["W_down"], d["R0"], d["gamma1"], d["gamma2"], S=S, alpha=alpha)
     if w.backward:
@@ -501,6 +671,10 @@ def blas_threads():
         return len(os.sched_getaffinity(0))
 
 
+def passes(w):
+    return "forward+backward" if w.backward else "forward"
+
+
 def cpu_baseline(w, target_s=12.0):
     probe = min(256, w.tokens)
     tp = oracle_sample_run(w, probe)
@@ -509,8 +683,48 @@ def cpu_baseline(w, target_s=12.0):
     n = max(probe, min(w.tokens, n // 256 * 256 if n >= 256 else probe))
     ts = oracle_sample_run(w, n)
     return {"value": n / ts, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
-            "sample": f"fp64 numpy oracle, block forward{'+backward' if w.backward else ''} on {n} of {w.tokens} tokens "
+            "sample": f"fp64 numpy oracle, {w.kind} {passes(w)} on {n} of {w.tokens} tokens "
                       f"of {w.name} (all {w.t} ranks), {ts:.2f} s; host has {len(os.sched_getaffinity(0))} usable cores"}
+
+
+def config_of(w, S, world, compact, m):
+    return {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p,
+            "S": S, "passes": passes(w), "private_scale": "sqrt(t)", "norm": "rmsnorm", "parallelism": f"replicas x{world}",
+            "residual_layout": "compact (shared channels of the stream stored once)" if compact else "per rank [t,T,h]",
+            "launch": "cuda graph replay" if m["graph"] else "eager", "l2": l2_note(m)}
+
+
+def sweep_entry(name, dev, steps, peaks):
+    """One workload of the sweep with its own per-kernel table (same timing rules as the headline)."""
+    w = synthetic.WORKLOADS[name]
+    k = max(10, min(steps, 50)) if w.tokens > 64 else max(50, min(steps, 200))
+    m, r = measure(w, dev, k, 5, False)
+    S = r.S
+    sms = m["ms_total"] / k
+    ent = {"workload": name, "p": w.p, "S": S, "passes": passes(w), "dtype": w.dtype, "steps": k, "ms_per_step": sms,
+           "step_ms": m["step_ms"], "tokens_per_s": w.tokens / (sms * 1e-3), "launch": "cuda graph replay" if m["graph"] else "eager",
+           "l2": l2_note(m), "path_roofline": path_roofline(w, S, False, sms, peaks),
+           "kernels": kernel_table(m["prof"], step_work(w, S), k, peaks),
+           "allreduce_payload_bytes": r.ctx.allreduce_bytes(w.tokens, 2)["payload_per_rank"]}
+    ent["path_roofline_frac"] = ent["path_roofline"]["frac"]
+    if "ms_warm_l2" in m:
+        ent["warm_l2"] = {"ms_per_step": m["ms_warm_l2"], "tokens_per_s": w.tokens / (m["ms_warm_l2"] * 1e-3),
+                          "path_roofline_frac": ent["path_roofline"]["roofline_ms"] / m["ms_warm_l2"],
+                          "note": "same steps on a single buffer set (operands that fit stay in the 126 MB L2); the "
+                                  "entry's own figures are the rotated, cold-L2 ones"}
+    del r
+    torch.cuda.empty_cache()
+    if w.kind == "block" and w.tokens > 64 and S % 8 == 0:
+        # the same block on the compact residual layout (shared channels of the stream stored once)
+        r = BlockRunner(w, dev, True)
+        for _ in range(3):
+            r.step()
+        cms = time_steps(r, k, False) / k
+        ent["compact_layout_ms_per_step"] = cms
+        ent["compact_layout_tokens_per_s"] = w.tokens / (cms * 1e-3)
+        del r
+        torch.cuda.empty_cache()
+    return ent
 
 
 def run_cuda(args):
@@ -527,44 +741,13 @@ def run_cuda(args):
     if args.tokens > 0:
         w = w.with_tokens(args.tokens)
     compact = args.layout == "compact"
-    runner = make_runner(w, dev, compact)
     warm = max(args.warmup, 3)
-    for _ in range(warm):
-        runner.step()
-    torch.cuda.synchronize()
-    assert runner.ctx.last_device_status() == caat.CAAT_OK
-
-    # small working sets (decode: the weights are about one L2) rotate over several buffer sets
-    nsets = buffer_sets_needed(runner.touched_bytes())
-    rset = [runner] + [make_runner(w, dev, compact) for _ in range(nsets - 1)]
-    for r in rset[1:]:
-        r.step()
-    torch.cuda.synchronize()
-    # launch-bound steps (decode: tens of microseconds) are replayed from a CUDA graph
-    graph, per_step = (None, 0)
-    probe = time_steps(rset, 5, False) / 5
-    if probe < 0.25 and not args.no_graph:
-        caps = [capture_step(r) for r in rset]
-        if all(g is not None for g, _ in caps):
-            graph, per_step = [g for g, _ in caps], caps[0][1]
     sampler = ClockSampler(local)
     sampler.start()
-    l0 = caat.kernel_launches()
-    ms = time_steps(rset, args.steps, dist_on, graph)
-    launches = per_step * args.steps if graph is not None else caat.kernel_launches() - l0
-    # second pass of the same K steps with CUDA events around every kernel (per-kernel device times)
-    caat.profile_begin(max(1024, launches + 64))
-    ms_prof = time_steps(rset, args.steps, dist_on)
-    prof = caat.profile_end()
-    # small working sets: the same steps on ONE buffer set, i.e. with whatever fits staying in L2 (reported
-    # separately; the headline figure is the rotated one)
-    ms_warm_l2 = None
-    if nsets > 1:
-        ms_warm_l2 = time_steps(rset[:1], args.steps, False, graph[:1] if graph is not None else None) / args.steps
-    del rset[1:]
+    m, runner = measure(w, dev, args.steps, warm, dist_on, compact, args.no_graph)
     clocks = sampler.stop()
-    ms = replicas.max_over_ranks(ms, dev)
-
+    S = runner.S
+    ms = replicas.max_over_ranks(m["ms_total"], dev)
     ms_step = ms / args.steps
     value = replicas.whole_job_rate(w.tokens, args.steps, world, ms)
 
@@ -580,60 +763,39 @@ def run_cuda(args):
         ems = replicas.max_over_ranks(ems, dev)
         e2e = {"value": world * w.tokens / (ems * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d * world,
                "d2h_bytes_per_step": d2h * world, "ms_per_step": ems,
-               "overlap": "copy-in, kernels and read-back of consecutive steps on three streams, two buffer sets"}
+               "overlap": "copy-in, kernels and read-back of consecutive steps on three streams, two device buffer sets, "
+                          "pinned host memory both ways"}
     except Exception as ex:  # pinned-memory exhaustion on a small host
         if dist_on:
             replicas.max_over_ranks(0.0, dev)     # keep the ranks' collectives matched
-        e2e = {"value": None, "unit": "tokens/s", "error": str(ex)[:200]}
+        e2e = {"value": None, "unit": "tokens/s", "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+               "error": "end-to-end leg not measured (host could not pin the step's buffers, or skipped): " + str(ex)[:200]}
 
     result = None
     if rank == 0:
         peaks = measured_peaks()
-        work = step_work(w, compact)
-        kernels = {}
-        for kind, (kms, n) in prof.items():
-            per_step_ms = kms / args.steps
-            wk = work.get(kind)
-            ent = {"ms_per_step": per_step_ms, "launches_per_step": n / args.steps, "share": kms / sum(v[0] for v in prof.values())}
-            if wk:
-                gbs = wk["bytes"] / (per_step_ms * 1e-3) / 1e9
-                tfs = wk["flops"] / (per_step_ms * 1e-3) / 1e12
-                t_hbm, t_tc = wk["bytes"] / (peaks["hbm_gbs"] * 1e9), wk["flops"] / (peaks["bf16_tflops"] * 1e12)
-                if t_tc > t_hbm:
-                    ent.update({"bound": "tensor", "achieved": tfs, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                                "frac": tfs / peaks["bf16_tflops"]})
-                else:
-                    ent.update({"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                "frac": gbs / peaks["hbm_gbs"]})
-                ent["gbs"], ent["tflops"] = gbs, tfs
-            kernels[kind] = ent
+        kernels = kernel_table(m["prof"], step_work(w, S, compact), args.steps, peaks)
         top = max((k for k in kernels if "frac" in kernels[k]), key=lambda k: kernels[k]["ms_per_step"])
-        roof = {k: kernels[top][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
-        roof.update({"kernel": top, "traffic": recorded_traffic(top, w.name + ("@compact" if compact else "")), "peak_source": peaks["source"],
-                     "timed": f"second pass of {args.steps} steps with CUDA events around every kernel launch "
-                              f"({ms_prof / args.steps:.4f} ms/step with events)"})
-        fl, by = paper_level_work(w, compact)
-        t_roof = max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9))
+        roof = {k: kernels[top][k] for k in ("bound", "achieved", "peak", "unit", "frac", "peak_name")}
+        if "frac_of_burst_peak" in kernels[top]:
+            roof["frac_of_burst_peak"] = kernels[top]["frac_of_burst_peak"]
+        roof.update({"kernel": top, "traffic": recorded_traffic(top, w.name + ("@compact" if compact else "")),
+                     "peak_source": peaks["source"] + ("; sustained bf16 figure: the kernel is timed inside a long step"
+                                                       if roof["bound"] == "tensor" else ""),
+                     "timed": f"pass of {args.steps} steps with CUDA events around every kernel launch "
+                              f"({m['ms_prof'] / args.steps:.4f} ms/step with events); achieved = the kind's algorithmic "
+                              f"work per step / its event time per step"})
         ar = runner.ctx.allreduce_bytes(w.tokens, 2)
         result = {
             "metric": metric_name(w), "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": w.dtype, "data": "synthetic",
-            "config": {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p,
-                       "S": w.S, "passes": "forward+backward" if w.backward else "forward",
-                       "private_scale": "sqrt(t)", "norm": "rmsnorm", "parallelism": f"replicas x{world}",
-                       "residual_layout": "compact (shared channels of the stream stored once)" if compact else "per rank [t,T,h]",
-                       "launch": "cuda graph replay" if graph is not None else "eager",
-                       "l2": (f"inputs+outputs touched per step {runner.touched_bytes() / 1e6:.0f} MB > 126 MB L2" if nsets == 1 else
-                              f"{nsets} buffer sets rotated step by step: {runner.touched_bytes() / 1e6:.0f} MB touched per step, "
-                              f"{(nsets - 1) * runner.touched_bytes() / 1e6:.0f} MB of other sets between two uses of a set (L2 126 MB)")},
-            "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "roofline": roof, "kernels": kernels,
-            "path_roofline": {"flops_per_step": fl, "bytes_per_step": by, "roofline_ms": t_roof * 1e3,
-                              "frac": t_roof * 1e3 / ms_step},
+            "ms_per_step": ms_step, "step_ms": m["step_ms"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": w.dtype, "data": "synthetic", "config": config_of(w, S, world, compact, m),
+            "clocks": clocks, "gpu_launches": m["launches"], "e2e": e2e, "roofline": roof, "kernels": kernels,
+            "path_roofline": path_roofline(w, S, compact, ms_step, peaks),
             "collective_bytes_analytic": {"per_reduce": ar, "reduces_per_step": 4 if w.backward else 2},
         }
-        if ms_warm_l2 is not None:
-            result["warm_l2"] = {"ms_per_step": ms_warm_l2, "tokens_per_s": w.tokens / (ms_warm_l2 * 1e-3),
+        if "ms_warm_l2" in m:
+            result["warm_l2"] = {"ms_per_step": m["ms_warm_l2"], "tokens_per_s": w.tokens / (m["ms_warm_l2"] * 1e-3),
                                  "note": "same steps on a single buffer set (operands that fit stay in the 126 MB L2); "
                                          "not the headline figure"}
     del runner
@@ -641,35 +803,15 @@ def run_cuda(args):
 
     if rank == 0 and not args.no_sweep and world == 1:
         sweep = []
+        peaks = measured_peaks()
         for name in SWEEP:
-            if name == w.name:
+            if name == w.name and not compact:
                 continue
             try:
-                r = make_runner(synthetic.WORKLOADS[name], dev)
-                for _ in range(5):
-                    r.step()
-                k = max(3, min(args.steps, 30))
-                sms = time_steps(r, k, False) / k
-                fl, by = paper_level_work(r.w)
-                peaks = measured_peaks()
-                t_roof = max(fl / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e3
-                sweep.append({"workload": name, "p": r.w.p, "ms_per_step": sms, "tokens_per_s": r.w.tokens / (sms * 1e-3),
-                              "path_roofline_frac": t_roof / sms,
-                              "allreduce_payload_bytes": r.ctx.allreduce_bytes(r.w.tokens, 2)["payload_per_rank"]})
-                del r
-                torch.cuda.empty_cache()
-                if r_w_compact_ok(synthetic.WORKLOADS[name]) and synthetic.WORKLOADS[name].kind == "block":
-                    # the same block on the compact residual layout (shared channels of the stream stored once)
-                    r = BlockRunner(synthetic.WORKLOADS[name], dev, True)
-                    for _ in range(3):
-                        r.step()
-                    cms = time_steps(r, k, False) / k
-                    sweep[-1]["compact_layout_ms_per_step"] = cms
-                    sweep[-1]["compact_layout_tokens_per_s"] = r.w.tokens / (cms * 1e-3)
-                    del r
-                    torch.cuda.empty_cache()
-            except Exception as ex:
+                sweep.append(sweep_entry(name, dev, args.steps, peaks))
+            except Exception as ex:  # noqa: BLE001
                 sweep.append({"workload": name, "error": str(ex)[:200]})
+                torch.cuda.empty_cache()
         result["sweep"] = sweep
         try:
             result["tp_projection"] = tp_projection(dev)
@@ -690,6 +832,7 @@ def run_cuda(args):
 def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
+    from oracle import caat_oracle as O
     w = synthetic.WORKLOADS[args.workload]
     probe = min(256, w.tokens)
     tp = min(oracle_sample_run(w, probe), oracle_sample_run(w, probe))
@@ -703,15 +846,15 @@ def run_reference(args):
         oracle_sample_run(w, n)
     dt = time.perf_counter() - t0
     value = n * args.steps / dt
-    sample = (f"fp64 numpy oracle, block forward{'+backward' if w.backward else ''}, each step a sample of {n} of "
+    sample = (f"fp64 numpy oracle, {w.kind} {passes(w)}, each step a sample of {n} of "
               f"{w.tokens} tokens of {w.name}; host has {len(os.sched_getaffinity(0))} usable cores")
     print(json.dumps({
         "impl": "reference", "metric": metric_name(w), "value": value, "unit": "tokens/s",
         "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p, "S": w.S,
-                   "passes": "forward+backward" if w.backward else "forward", "sample_tokens": n},
+        "config": {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p,
+                   "S": O.shared_channels(w.h, w.p), "passes": passes(w), "sample_tokens": n},
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}), flush=True)
@@ -720,9 +863,12 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "tp"],
+                    help="replicas: one independent replica of the workload per GPU (the benchmark); tp: the "
+                         "tensor-parallel ranks split over the GPUs, all-reduce of the shared-channel slab, p sweep")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synthetic.WORKLOADS))
     ap.add_argument("--no-sweep", action="store_true", help="skip the other workloads' tokens/s")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
@@ -736,6 +882,9 @@ def main():
         raise SystemExit("--steps must be >= 1")
     if args.impl == "reference":
         run_reference(args)
+    elif args.mode == "tp":
+        from paper_2506_19645_b200 import tp_bench
+        tp_bench.run(args)
     else:
         run_cuda(args)
 

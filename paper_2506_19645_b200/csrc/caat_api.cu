@@ -42,12 +42,18 @@ bool pdl_enabled() {
   return on;
 }
 
+std::mutex& host_cache_mutex() {
+  static std::mutex m;
+  return m;
+}
+
 unsigned int* device_status_word() {
   // looked up once per device (the lookup is not a stream operation; caching it keeps launches
   // free of runtime queries, which also matters inside a stream capture)
   static unsigned int* cache[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(host_cache_mutex());
   if (cache[dev] == nullptr) {
     unsigned int* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word) != cudaSuccess) return nullptr;
@@ -60,6 +66,7 @@ int sm_count() {
   static int cache[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  std::lock_guard<std::mutex> lock(host_cache_mutex());
   if (cache[dev] == 0) {
     int n = 0;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
@@ -68,9 +75,10 @@ int sm_count() {
   return cache[dev];
 }
 
-static caat_status cuda_fail(cudaError_t e) {
+caat_status cuda_fail(cudaError_t e) {
   std::strncpy(g_cuda_err, cudaGetErrorString(e), sizeof(g_cuda_err) - 1);
   g_cuda_err[sizeof(g_cuda_err) - 1] = 0;
+  (void)cudaGetLastError();   // the error is reported through the status; do not leave it sticky for the caller's next call
   return CAAT_ECUDA;
 }
 

@@ -39,6 +39,15 @@ constexpr int kTmemCols = 512;
 constexpr uint32_t kSpinCap = 1u << 22;
 constexpr int kMaxStages = 8;
 constexpr int kCBuf = 128 * 64;   // one output staging buffer: 128 rows x 64 bytes (32 bf16 / 16 fp32 columns)
+// Measurement aids that make results wrong (phase ablation: skipped loads, stores, barriers) and the
+// tile-shape overrides exist only in builds compiled with -DCAAT_MEASUREMENT_AIDS; the library as
+// built by build.py honours none of them.  Bit 1024 (a stage wait made to run out, for the time-out
+// test) stays: it changes no result of a call that returns CAAT_OK.
+#ifdef CAAT_MEASUREMENT_AIDS
+constexpr int kAidMask = ~0;
+#else
+constexpr int kAidMask = 1024;
+#endif
 
 struct Unit {            // one contraction segment of a tile
   int mapA, mapB;        // indices into the tensor-map array
@@ -78,7 +87,7 @@ struct Params {
   int tiles_total;
   unsigned int* status;
   uint32_t spin_cap;     // polls of one mbarrier wait before the role gives up (kSpinCap; CAAT_TC_SPINCAP for the timeout test)
-  int debug;             // measurement aid (env CAAT_TC_DEBUG; results are then wrong): 1 = no operand loads,
+  int debug;             // measurement aid (env CAAT_TC_DEBUG, masked by kAidMask; results are then wrong): 1 = no operand loads,
                          // 2 = no epilogue work at all, 4 = no A loads, 8 = no B loads; epilogue stops after the
                          // tensor-memory load (32) / after the staging stores (16); 64 = no slab barrier,
                          // 128 = no TMA store; 512 = producer lanes take no second k-step; 1024 = the A boxes are
@@ -350,7 +359,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
     // measured: pays for multi-box operands (dgrad / wgrad -5...-8 %) and the weight stream of the decode
     // path (-5 %); a K-major operand of the large GEMMs gains nothing (its tiles wait for L2, not for the
     // issue) and a ring shorter than six stages loses more to pairwise refills than it gains
-    const int nki = ((multi || p.out_transposed) && p.nstages >= 6 && !(p.debug & 512)) ? kKI : 1;
+    const int nki = ((multi || p.out_transposed) && p.nstages >= 6 && !(p.debug & kAidMask & 512)) ? kKI : 1;
     const int jk = lane / nbmax, box = lane - jk * nbmax;                         // this lane's k-step slot and box
     if (jk < nki) {
       int stage = 0; uint32_t phase = 0;
@@ -362,8 +371,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         const uint32_t cols_cta = (uint32_t)tile_cols(p, r, c.nt, CG) / CG;    // B columns this CTA stages
         const uint32_t b_tile_bytes = cols_cta * BK * 2;
         const int m0 = c.mt * BMT + (int)rank * BM, n0 = c.nt * p.BN + (int)(rank * cols_cta);
-        const uint32_t tx = (uint32_t)CG * (((p.debug & 4) ? 0u : a_bytes) + ((p.debug & 8) ? 0u : b_tile_bytes));
-        const bool skip = isA ? (p.debug & (4 | 1024)) != 0 : (p.debug & 8) != 0;
+        const uint32_t tx = (uint32_t)CG * (((p.debug & kAidMask & 4) ? 0u : a_bytes) + ((p.debug & kAidMask & 8) ? 0u : b_tile_bytes));
+        const bool skip = isA ? (p.debug & kAidMask & (4 | 1024)) != 0 : (p.debug & kAidMask & 8) != 0;
         const int nb = multi ? (isA ? BM / 64 : (int)cols_cta / 64) : 1;         // boxes of this tile's stages
         for (int ui = 0; ui < r.nunits && ok; ++ui) {
           const Unit& u = r.u[ui];
@@ -384,9 +393,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
                 const uint32_t fb = CG == 2 ? mapa_rank(fb_local, 0) : fb_local;
                 const uint32_t sa = tiles_sa + (uint32_t)st * stage_bytes, sb = sa + a_bytes;
                 if (isA && rank == 0 && box == 0) {
-                  if (p.debug & 1) mbar_arrive(fb_local); else mbar_expect_tx(fb_local, tx);
+                  if (p.debug & kAidMask & 1) mbar_arrive(fb_local); else mbar_expect_tx(fb_local, tx);
                 }
-                if (!(p.debug & 1) && !skip && box < nb) {
+                if (!(p.debug & kAidMask & 1) && !skip && box < nb) {
                   auto load = [&](uint32_t dst, int x, int y) {
                     if (CG == 2) tma_load_3d_pair(dst, map, x, y, z, fb); else tma_load_3d(dst, map, x, y, z, fb);
                   };
@@ -529,7 +538,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
           }
         }
       } else
-      for (int cc = 0; cc < p.BN && n0 + cc < r.N && !(p.debug & 2); cc += sub) {
+      for (int cc = 0; cc < p.BN && n0 + cc < r.N && !(p.debug & kAidMask & 2); cc += sub) {
         uint32_t v[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols + cc);
         if (p.out_f32) tmem_ld16(taddr, v); else tmem_ld32(taddr, v);
@@ -544,7 +553,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         }
         const uint32_t buf = smem_u32(cstage + (size_t)(slab % 3) * kCBuf);
         const uint32_t rowaddr = buf + (uint32_t)rr * 64u;
-        if (p.debug & 32) { ++slab; continue; }
+        if (p.debug & kAidMask & 32) { ++slab; continue; }
         if (p.out_f32) {
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
@@ -561,10 +570,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
             sts128(rowaddr + (((uint32_t)q4 ^ sw) << 4), w[0], w[1], w[2], w[3]);
           }
         }
-        if (p.debug & 16) { ++slab; continue; }
+        if (p.debug & kAidMask & 16) { ++slab; continue; }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (!(p.debug & 64)) epi_barrier();
-        if (warp == 2 && lane == 0 && !(p.debug & 128)) {
+        if (!(p.debug & kAidMask & 64)) epi_barrier();
+        if (warp == 2 && lane == 0 && !(p.debug & kAidMask & 128)) {
           tma_store_3d(cmaps[c.region], n0 + cc, m0, zc, buf);
           bulk_commit();
           bulk_wait_read1();     // the store before this one has finished reading its buffer
@@ -690,10 +699,14 @@ double estimate_cost(const RegionShape* r, int nr, int bn, int cg, int splits, d
 }
 
 TileCfg pick_tile(const RegionShape* r, int nr, bool b_n_major, int max_splits, double out_bytes) {
+#ifdef CAAT_MEASUREMENT_AIDS
   static const int max_cg = [] { const char* e = getenv("CAAT_TC_CG"); return e && atoi(e) == 1 ? 1 : 2; }();
-  // measurement aids: CAAT_TC_BN / CAAT_TC_CGF pin the tile width / the pair mode instead of the model's choice
+  // CAAT_TC_BN / CAAT_TC_CGF pin the tile width / the pair mode instead of the model's choice
   static const int force_bn = [] { const char* e = getenv("CAAT_TC_BN"); return e ? atoi(e) : 0; }();
   static const int force_cg = [] { const char* e = getenv("CAAT_TC_CGF"); return e ? atoi(e) : 0; }();
+#else
+  constexpr int max_cg = 2, force_bn = 0, force_cg = 0;
+#endif
   TileCfg best{256, 1, 1, -1.0};
   int min_ksteps = 1 << 30;
   for (int i = 0; i < nr; ++i)
@@ -731,7 +744,7 @@ cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params
   static bool attr_set[64] = {};      // the attribute belongs to the device's copy of the kernel: once per device
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!attr_set[dev]) {
+  if (std::lock_guard<std::mutex> lock(host_cache_mutex()); !attr_set[dev]) {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
@@ -740,7 +753,7 @@ cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params
   p.status = device_status_word();
   if (!p.status) return cudaErrorUnknown;
   static const int dbg = [] { const char* e = getenv("CAAT_TC_DEBUG"); return e ? atoi(e) : 0; }();
-  p.debug = dbg;
+  p.debug = dbg & kAidMask;
   static const uint32_t cap_env = [] { const char* e = getenv("CAAT_TC_SPINCAP"); return e ? (uint32_t)atoi(e) : 0u; }();
   p.spin_cap = cap_env >= 1024 ? cap_env : kSpinCap;
   static const bool verbose = getenv("CAAT_TC_VERBOSE") != nullptr;

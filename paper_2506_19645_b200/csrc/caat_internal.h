@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "caat.h"
 
 struct caat_ctx {
@@ -214,6 +216,10 @@ struct LaunchScope {
   int slot;
   cudaStream_t st;
 };
+// One lock for the library's small host-side caches (per-device attribute flags, looked-up addresses and
+// occupancy answers): calls from several host threads may run concurrently, the caches are filled under it.
+std::mutex& host_cache_mutex();
+caat_status cuda_fail(cudaError_t e);  // records the error text for caat_last_cuda_error(), returns CAAT_ECUDA
 unsigned int* device_status_word();  // device address of the status word (per device)
 int sm_count();                       // multiprocessors of the current device (grids are sized in multiples of it)
 

@@ -655,6 +655,7 @@ cudaError_t launch_partials_cluster(const RowPartArgs& a, int threads, size_t sm
   static bool attr_set[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  std::unique_lock<std::mutex> lock(host_cache_mutex());   // attribute flag and the occupancy answers below
   if (!attr_set[dev]) {
     const cudaError_t e = cudaFuncSetAttribute(rows_forward_partials_cluster_kernel<T_, LN, MINB>,
                                                cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -687,8 +688,12 @@ cudaError_t launch_partials_cluster(const RowPartArgs& a, int threads, size_t sm
       cudaGetLastError();
       clusters = 0;
     }
-    if (nseen < 8) seen[nseen++] = Seen{dev, a.t, threads, smem, clusters};
+    // a full table forgets its oldest entry instead of asking the device again on every launch
+    static int next = 0;
+    const int slot = nseen < 8 ? nseen++ : (next++ & 7);
+    seen[slot] = Seen{dev, a.t, threads, smem, clusters};
   }
+  lock.unlock();
   if (clusters < 1) return cudaSuccess;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
   *launched = true;

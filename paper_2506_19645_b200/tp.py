@@ -3,9 +3,12 @@ the two halves of the library's layer call the all-reduce of the shared-channel 
 reduce-scatter + all-gather of tokens * S elements, a fraction p of a full all-reduce).
 
 Argument marshalling and the collective only: every arithmetic step of the layer runs in the library's kernels.
-The one exception is optional and off the kernels' path: the backward slab can be carried in fp32 through the
-collective (Section 4: the backward reduce wants fp32 accumulation; a 16-bit collective accumulates in 16 bit),
-which costs a cast before and after it.  With a process group of one the collective is skipped and the layer
+The one exception is off the kernels' path: a library collective accumulates in its payload type, and a chain of
+16-bit partial sums over 8 ranks leaves the layer output outside the 2e-2 tolerance against the exact sum (measured:
+2.3e-2), so by default the slab is carried through the collective in fp32, forward and backward (Section 4 asks
+for fp32 accumulation of the backward reduce; the forward is held to the same), which costs a cast before and
+after it and twice the wire bytes.  ``forward_accumulate=None`` / ``backward_accumulate=None`` send the 16-bit
+slab as it is.  With a process group of one the collective is skipped and the layer
 equals ``rowpar_forward`` / ``rowpar_backward``.
 
 The collective is ``torch.distributed.all_reduce`` (NCCL between GPUs, gloo in CPU tests of this module's own
@@ -40,7 +43,8 @@ class TensorParallelRowLinear:
     """``t_local`` ranks of a ``t_local * world`` tensor-parallel group on this GPU.  Tensors are the ones of
     ``Context.rowpar_forward`` / ``rowpar_backward`` restricted to this GPU's ranks (``K_r = K / (t_local * world)``)."""
 
-    def __init__(self, h, ffn, t_local, p, dtype="bf16", group=None, backward_accumulate=torch.float32):
+    def __init__(self, h, ffn, t_local, p, dtype="bf16", group=None, backward_accumulate=torch.float32,
+                 forward_accumulate=torch.float32):
         from . import caat
         self.caat = caat
         self.group = group
@@ -48,6 +52,7 @@ class TensorParallelRowLinear:
         self.ctx = caat.Context(h, ffn, t_local, p, dtype)
         self.ctx.set_option(caat.CAAT_OPT_TP_GROUPS, self.world)     # also sets alpha = sqrt(t_local * world)
         self.backward_accumulate = backward_accumulate
+        self.forward_accumulate = forward_accumulate
 
     def workspace(self, layer, tokens, backward=True, device="cuda"):
         return self.ctx.alloc_workspace(self.ctx.workspace_bytes(layer, tokens, backward), device=device)
@@ -56,7 +61,7 @@ class TensorParallelRowLinear:
         c = self.ctx
         c.tp_forward_local(layer, tokens, Y, W, workspace)
         if c.shared_channels > 0:
-            allreduce_slab(c.tp_slab(layer, tokens, False, workspace), self.group)
+            allreduce_slab(c.tp_slab(layer, tokens, False, workspace), self.group, self.forward_accumulate)
         c.tp_forward_finish(layer, tokens, R, gamma, beta, Hn, X, rstd, mean, workspace)
 
     def backward(self, layer, tokens, dX, dHn, Y, W, Hn, rstd, mean, gamma, dY, dW, dR, dgamma, dbeta, workspace):

@@ -1,6 +1,7 @@
 """Real tensor parallelism, checked on one GPU: the t ranks are split into G groups (one per GPU in a real run),
 every group runs the first half of the layer call, the all-reduce of the shared-channel slab is stood in for by
-summing the groups' slabs (fp32, rounded once), every group runs the second half, and the concatenated results
+summing the groups' slabs the way tp.py's collective does (carried in fp32, rounded once; a second test measures
+what a 16-bit payload with 16-bit partial sums costs), every group runs the second half, and the concatenated results
 must match the fp64 oracle with all t ranks — forward and backward.  Needs a GPU."""
 import numpy as np
 import pytest
@@ -14,10 +15,14 @@ pytestmark = pytest.mark.gpu
 BF = torch.bfloat16
 
 
-def _sum_slabs(slabs):
-    total = torch.zeros_like(slabs[0], dtype=torch.float32)
-    for s in slabs:                      # stands in for the all-reduce: fp32 sum, one rounding
-        total += s.float()
+def _sum_slabs(slabs, accumulate):
+    """Stands in for the all-reduce that tp.py issues between the halves.  A collective accumulates in its payload
+    type: tp.py carries the slab in fp32 by default (forward and backward), so the sum is rounded once at the end;
+    `accumulate = bf16` models the slab sent as it is, where every partial sum is rounded to bf16 (here in rank
+    order, as a ring that starts at rank 0 would)."""
+    total = slabs[0].to(accumulate)
+    for s in slabs[1:]:
+        total = (total.float() + s.float()).to(accumulate)
     for s in slabs:
         s.copy_(total)
 
@@ -56,7 +61,7 @@ def test_groups_with_slab_sum_match_oracle(t, G, T, h, ffn, S, layer, norm):
     for q, c in enumerate(ctxs):
         c.tp_forward_local(layer, T, sl(dev["Y"], q), sl(dev["W"], q), ws[q])
     if S > 0:
-        _sum_slabs([c.tp_slab(layer, T, False, ws[q]) for q, c in enumerate(ctxs)])
+        _sum_slabs([c.tp_slab(layer, T, False, ws[q]) for q, c in enumerate(ctxs)], torch.float32)
     for q, c in enumerate(ctxs):
         c.tp_forward_finish(layer, T, sl(dev["R"], q), dev["gamma"], dev["beta"], sl(Hn, q), sl(X, q), rstds[q],
                             means[q], ws[q])
@@ -78,7 +83,7 @@ def test_groups_with_slab_sum_match_oracle(t, G, T, h, ffn, S, layer, norm):
                             sl(srs, q).clone(), sl(smu, q).clone() if norm else None, dev["gamma"], sl(dR, q), dgs[q],
                             dbs[q], ws[q])
     if S > 0:
-        _sum_slabs([c.tp_slab(layer, T, True, ws[q]) for q, c in enumerate(ctxs)])
+        _sum_slabs([c.tp_slab(layer, T, True, ws[q]) for q, c in enumerate(ctxs)], torch.float32)
     dgamma = torch.stack(dgs).sum(0)                   # the fp32 all-reduce of the norm-parameter gradients
     for q, c in enumerate(ctxs):
         c.tp_backward_finish(layer, T, sl(dev["Y"], q), sl(dev["W"], q), sl(dR, q), sl(dY, q), sl(dW, q), ws[q])
@@ -90,6 +95,31 @@ def test_groups_with_slab_sum_match_oracle(t, G, T, h, ffn, S, layer, norm):
         assert_close(v.cpu(), ob[k], "bf16", k)
     if norm:
         assert_close(torch.stack(dbs).sum(0).cpu(), ob["dbeta"], "bf16", "dbeta")
+
+
+def test_sixteen_bit_collective_is_less_accurate_than_the_fp32_carry():
+    # The forward slab sent through a collective in its own 16-bit type: every partial sum is rounded.  With 8 ranks
+    # that is visibly worse than carrying fp32 (the library's default in tp.py) - the reason for that default.
+    t, G, T, h, ffn, S, layer = 8, 8, 130, 1024, 4096, 256, caat.CAAT_MLP_DOWN
+    K = ffn // t
+    d = synthetic.layer_inputs(t, T, h, K, "bf16", seed=3 + T, S=S)
+    exact = O.partial_channel_reduce(O.rank_partials(f64(d["Y"]), f64(d["W"])), S, 1.0)[0, :, :S]
+    errs = {}
+    for acc in (torch.float32, BF):
+        ctxs, ws = [], []
+        for q in range(G):
+            c = caat.Context(h, ffn, 1, 0.5, "bf16")
+            c.set_option(caat.CAAT_OPT_SHARED_CHANNELS, S).set_option(caat.CAAT_OPT_TP_GROUPS, G)
+            w = c.alloc_workspace(c.workspace_bytes(layer, T, False))
+            c.tp_forward_local(layer, T, d["Y"][q:q + 1].cuda(), d["W"][q:q + 1].cuda(), w)
+            ctxs.append(c); ws.append(w)
+        slabs = [c.tp_slab(layer, T, False, ws[q]) for q, c in enumerate(ctxs)]
+        _sum_slabs(slabs, acc)
+        torch.cuda.synchronize()
+        got = f64(slabs[0])
+        errs[acc] = float(np.sqrt(np.mean((got - exact) ** 2)) / np.sqrt(np.mean(exact ** 2)))
+    assert errs[torch.float32] < 4e-3                   # bf16 partials of each group + one final rounding
+    assert errs[BF] > 1.5 * errs[torch.float32]
 
 
 def test_one_group_halves_equal_the_single_call():
