@@ -7,6 +7,7 @@ header changed), then the objects are linked into the shared library.
 from __future__ import annotations
 
 import os
+import shlex
 import subprocess
 import sys
 from concurrent.futures import ThreadPoolExecutor
@@ -29,7 +30,9 @@ def _headers_mtime() -> float:
 
 
 def _compile(nvcc: str, src: str, obj: str, verbose: bool) -> str:
+    # CAAT_NVCC_EXTRA: extra compiler flags, e.g. -DCAAT_MEASUREMENT_AIDS for a build with the ablation switches
     cmd = [nvcc, *ARCH, "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC", "-rdc=false",
+           *shlex.split(os.environ.get("CAAT_NVCC_EXTRA", "")),
            "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", src, "-o", obj]
     if verbose:
         cmd[1:1] = ["-Xptxas", "-v"]

@@ -47,6 +47,22 @@ std::mutex& host_cache_mutex() {
   return m;
 }
 
+LaunchLimits& launch_limits() {
+  static thread_local LaunchLimits lim;
+  return lim;
+}
+
+const LaunchLimits effective_limits() {
+  LaunchLimits lim = launch_limits();
+#ifdef CAAT_MEASUREMENT_AIDS
+  // read at every launch so that a measurement script can change them between calls
+  auto env = [](const char* name, int& v) { const char* e = getenv(name); if (e && v == 0) v = atoi(e); };
+  env("CAAT_X_GEMM_WORKERS", lim.gemm_workers); env("CAAT_X_GEMM_SMEM", lim.gemm_smem);
+  env("CAAT_X_ROWS_CTAS", lim.rows_ctas); env("CAAT_X_ROWS_PER_SM", lim.rows_per_sm); env("CAAT_X_ROWS_SMEM", lim.rows_smem);
+#endif
+  return lim;
+}
+
 unsigned int* device_status_word() {
   // looked up once per device (the lookup is not a stream operation; caching it keeps launches
   // free of runtime queries, which also matters inside a stream capture)

@@ -735,8 +735,10 @@ TileCfg pick_tile(const RegionShape* r, int nr, bool b_n_major, int max_splits, 
 }
 
 cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params& p, int kind, cudaStream_t st) {
+  const LaunchLimits lim = effective_limits();
   const int stage_bytes = BM * BK * 2 + (p.BN / p.cg) * BK * 2;
-  int nst = (227 * 1024 - 2048 - 3 * kCBuf) / stage_bytes;
+  const int budget = lim.gemm_smem > 0 && lim.gemm_smem < 227 * 1024 ? lim.gemm_smem : 227 * 1024;
+  int nst = (budget - 2048 - 3 * kCBuf) / stage_bytes;
   if (nst > kMaxStages) nst = kMaxStages;
   if (nst < 2) return cudaErrorInvalidConfiguration;
   p.nstages = nst;
@@ -760,7 +762,8 @@ cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params
   if (verbose)
     fprintf(stderr, "[caat tc] kind=%d BN=%d cg=%d splits=%d stages=%d tiles=%d (r0 M=%d N=%d b=%d)\n", kind, p.BN, p.cg,
             p.splits, nst, p.tiles_total, p.r[0].M, p.r[0].N, p.r[0].batch);
-  const int workers_max = sm_count() / p.cg;
+  int workers_max = sm_count() / p.cg;
+  if (lim.gemm_workers > 0 && lim.gemm_workers / p.cg < workers_max) workers_max = lim.gemm_workers / p.cg;
   const int workers = p.tiles_total < workers_max ? p.tiles_total : workers_max;
   if (workers < 1) return cudaSuccess;
   cudaLaunchConfig_t cfg{};

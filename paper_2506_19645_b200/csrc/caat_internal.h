@@ -207,6 +207,25 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// ---- launch limits ---------------------------------------------------------------
+// A block call runs a layer's HBM-bound row kernel beside the other layer's tensor-bound GEMMs by giving
+// each a share of the GPU: the row kernel is held to a few CTAs, the GEMM to the remaining workers.  The limits
+// are a property of the launching host thread for the duration of one launch call (0 = no limit).
+struct LaunchLimits {
+  int gemm_workers = 0;   // CTAs of a tensor-core GEMM launch, at most
+  int gemm_smem = 0;      // dynamic shared memory of a GEMM CTA, at most (bytes): fewer pipeline stages
+  int rows_ctas = 0;      // CTAs of a row-kernel launch, at most
+  int rows_per_sm = 0;    // resident row-kernel CTAs per SM the shared-memory ring is sized for
+  int rows_smem = 0;      // shared memory the row kernel's CTAs of one SM may use together (bytes)
+};
+LaunchLimits& launch_limits();                  // this host thread's current limits
+const LaunchLimits effective_limits();          // the above, or a measurement build's environment overrides
+struct ScopedLimits {
+  LaunchLimits saved;
+  explicit ScopedLimits(const LaunchLimits& l) : saved(launch_limits()) { launch_limits() = l; }
+  ~ScopedLimits() { launch_limits() = saved; }
+};
+
 // ---- bookkeeping ------------------------------------------------------------
 // Brackets one kernel launch: counts it and, while profiling is on, records a CUDA event
 // before and after it on the launching stream.

@@ -771,16 +771,19 @@ bool rows_staged_usable(int h, int t, int S_lo, int S_hi, caat_dtype dtype, bool
 cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st) {
   const RowGeom g = row_geometry(a.h, dtype);
   const int ES = (int)elem_size(dtype);
-  int per_sm = ctas_per_sm(g);
+  const LaunchLimits lim = effective_limits();
+  int per_sm = lim.rows_per_sm > 0 ? lim.rows_per_sm : ctas_per_sm(g);
+  const size_t sm_budget = lim.rows_smem > 0 && (size_t)lim.rows_smem < kSmemPerSm ? (size_t)lim.rows_smem : kSmemPerSm;
   const bool cl = a.compact != 0;
-  StageGeom sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, cl, kSmemPerSm / per_sm - 1024);
+  StageGeom sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, cl, sm_budget / per_sm - 1024);
   while (sg.nstages < 3 && per_sm > 1) {   // rows too long: fewer CTAs per SM, each with a larger ring
     --per_sm;
-    sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, cl, kSmemPerSm / per_sm - 1024);
+    sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, false, true, cl, sm_budget / per_sm - 1024);
   }
   if (sg.nstages < 2) return cudaErrorInvalidConfiguration;
   const int ngroups = (a.T + g.TY - 1) / g.TY;
   int grid = sm_count() * per_sm;
+  if (lim.rows_ctas > 0 && grid > lim.rows_ctas) grid = lim.rows_ctas;
   if (grid > ngroups) grid = ngroups;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
@@ -804,16 +807,19 @@ cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, i
   const RowGeom g = row_geometry(a.h, dtype);
   const int ES = (int)elem_size(dtype);
   const bool has_c = a.dHn != nullptr;
-  int per_sm = ctas_per_sm(g);
+  const LaunchLimits lim = effective_limits();
+  int per_sm = lim.rows_per_sm > 0 ? lim.rows_per_sm : ctas_per_sm(g);
+  const size_t sm_budget = lim.rows_smem > 0 && (size_t)lim.rows_smem < kSmemPerSm ? (size_t)lim.rows_smem : kSmemPerSm;
   const bool cl = a.compact != 0;
-  StageGeom sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, true, has_c, cl, kSmemPerSm / per_sm - 1024);
+  StageGeom sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, true, has_c, cl, sm_budget / per_sm - 1024);
   while (sg.nstages < 3 && per_sm > 1) {
     --per_sm;
-    sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, true, has_c, cl, kSmemPerSm / per_sm - 1024);
+    sg = stage_geometry(g, a.h, a.P, a.S_hi, a.t, ES, true, has_c, cl, sm_budget / per_sm - 1024);
   }
   if (sg.nstages < 2) return cudaErrorInvalidConfiguration;
   const int ngroups = (a.T + g.TY - 1) / g.TY;
   int grid = sm_count() * per_sm;
+  if (lim.rows_ctas > 0 && grid > lim.rows_ctas) grid = lim.rows_ctas;
   if (grid > ngroups) grid = ngroups;
   if (grid > max_rows) grid = max_rows;
   *rows_used = grid;

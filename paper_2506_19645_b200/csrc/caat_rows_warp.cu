@@ -639,10 +639,14 @@ int rows_warp_cpt(int h, int t, caat_dtype dtype) {
 cudaError_t launch_rows_forward_warp(const RowFwdArgs& a, caat_dtype dtype, cudaStream_t st) {
   const int cpt = rows_warp_cpt(a.h, a.t, dtype);
   const int ES = (int)elem_size(dtype);
-  const WarpGeom g = warp_geometry(a.h, a.P, a.S_hi, ES, false, true, a.compact != 0, kSmemPerSm / kCtasPerSm - 1024);
+  const LaunchLimits lim = effective_limits();
+  const int per_sm = lim.rows_per_sm > 0 && lim.rows_per_sm < kCtasPerSm ? lim.rows_per_sm : kCtasPerSm;
+  const size_t sm_budget = lim.rows_smem > 0 && (size_t)lim.rows_smem < kSmemPerSm ? (size_t)lim.rows_smem : kSmemPerSm;
+  const WarpGeom g = warp_geometry(a.h, a.P, a.S_hi, ES, false, true, a.compact != 0, sm_budget / per_sm - 1024);
   if (cpt == 0 || g.nstages < 2) return cudaErrorInvalidConfiguration;
   const int ngroups = (a.T + kW - 1) / kW;
-  int grid = sm_count() * kCtasPerSm;
+  int grid = sm_count() * per_sm;
+  if (lim.rows_ctas > 0 && grid > lim.rows_ctas) grid = lim.rows_ctas;
   if (grid > ngroups) grid = ngroups;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
@@ -664,10 +668,14 @@ cudaError_t launch_rows_backward_warp(const RowBwdArgs& a, caat_dtype dtype, int
                                       cudaStream_t st) {
   const int cpt = rows_warp_cpt(a.h, a.t, dtype);
   const int ES = (int)elem_size(dtype);
-  const WarpGeom g = warp_geometry(a.h, a.P, a.S_hi, ES, true, a.dHn != nullptr, a.compact != 0, kSmemPerSm / kCtasPerSm - 1024);
+  const LaunchLimits lim = effective_limits();
+  const int per_sm = lim.rows_per_sm > 0 && lim.rows_per_sm < kCtasPerSm ? lim.rows_per_sm : kCtasPerSm;
+  const size_t sm_budget = lim.rows_smem > 0 && (size_t)lim.rows_smem < kSmemPerSm ? (size_t)lim.rows_smem : kSmemPerSm;
+  const WarpGeom g = warp_geometry(a.h, a.P, a.S_hi, ES, true, a.dHn != nullptr, a.compact != 0, sm_budget / per_sm - 1024);
   if (cpt == 0 || g.nstages < 2) return cudaErrorInvalidConfiguration;
   const int ngroups = (a.T + kW - 1) / kW;
-  int grid = sm_count() * kCtasPerSm;
+  int grid = sm_count() * per_sm;
+  if (lim.rows_ctas > 0 && grid > lim.rows_ctas) grid = lim.rows_ctas;
   if (grid > ngroups) grid = ngroups;
   if (grid > max_rows) grid = max_rows;
   *rows_used = grid;
