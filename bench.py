@@ -869,6 +869,8 @@ def main():
     ap.add_argument("--mode", default="replicas", choices=["replicas", "tp"],
                     help="replicas: one independent replica of the workload per GPU (the benchmark); tp: the "
                          "tensor-parallel ranks split over the GPUs, all-reduce of the shared-channel slab, p sweep")
+    ap.add_argument("--tp-exchange", default="nccl", choices=["nccl", "push"],
+                    help="--mode tp: the slab exchange - a library all-reduce, or the package's own kernels over peer memory")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synthetic.WORKLOADS))
     ap.add_argument("--no-sweep", action="store_true", help="skip the other workloads' tokens/s")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")

@@ -389,6 +389,66 @@ caat_status caat_tp_backward_finish(const caat_ctx *ctx, caat_layer layer, int t
                                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * The exchange of the shared-channel slab over PEER MEMORY, in the library's own kernels (Section 3:
+ * partial channel-reduce; Appendix D: reduce-scatter + all-gather of tokens*S elements; Section 4:
+ * communicate in 16 bit, accumulate in 32 bit).  It replaces the caller's collective between the two
+ * halves of a layer call (see above) when the GPUs of the group can address each other's memory
+ * (NVLink / NVSwitch peers: plain loads and stores, no multicast load anywhere):
+ *
+ *   scatter   every GPU stores rows [q*slice, (q+1)*slice) of its slab - its ranks' partial sum -
+ *             into slot `rank` of GPU q's receive buffer (16-bit payload), then raises flag `rank`
+ *             on GPU q.  caat_tp_forward_local_push does the same from inside the forward GEMM: the
+ *             tiles of the shared columns leave the epilogue straight for their owner's slot while
+ *             the private columns' tiles are still being multiplied, and the slab is never written.
+ *   reduce    GPU q waits for all `world` flags, sums the `world` slots of its token slice in fp32 in
+ *             the fixed order 0..world-1, rounds once to the run dtype and stores the result rows
+ *             into EVERY GPU's slab (the all-gather), then raises flag `world + q` on every GPU.
+ *   wait      every GPU waits for all `world` gather flags: its slab is complete; the second half of
+ *             the layer call (caat_tp_forward_finish / caat_tp_backward_finish) follows on the stream.
+ *
+ * caat_tp_exchange runs the three phases in a row on one GPU's stream; in a job every GPU of the group
+ * calls it at the same point of its stream.  The phases are also exported one by one, which is how a
+ * single GPU can stand in for the whole group in a test (all scatters, then all reduces, then all waits).
+ *
+ *   peers->world, rank   size of the group (<= CAAT_MAX_PEERS) and this GPU's index in it
+ *   peers->recv[q]       GPU q's receive buffer, caat_tp_exchange_bytes' recv_bytes, as THIS GPU addresses it
+ *   peers->slab[q]       GPU q's slab (workspace + caat_tp_slab's offset), as this GPU addresses it
+ *   peers->flags[q]      GPU q's flag words, CAAT_TP_FLAG_BYTES, zeroed once by their owner before first use
+ *   epoch                a number every GPU of the group passes alike, larger (mod 2^32) in every new exchange
+ *                        on the same buffers; flags are compared with it and never reset
+ * slice = tokens per owner = caat_tp_exchange_bytes' slice_rows (the same on every GPU).  Every wait on a
+ * flag is bounded (about a second): when it runs out the kernel raises the device status word
+ * (caat_last_device_status returns CAAT_ETIMEOUT), skips its work and returns; nothing traps or spins on.
+ * bf16 tensor-core path only, S a multiple of 8; caat_tp_forward_local_push further needs slice_rows to be
+ * a multiple of 256 (CAAT_EUNSUPPORTED otherwise: use caat_tp_forward_local + the scatter phase).
+ * Buffers named in `peers` are owned by the callers; the library keeps no pointer after the call returns.
+ */
+#define CAAT_MAX_PEERS 8
+#define CAAT_TP_FLAG_BYTES 256
+typedef struct caat_peers {
+  int world, rank;
+  void *recv[CAAT_MAX_PEERS];
+  void *slab[CAAT_MAX_PEERS];
+  unsigned int *flags[CAAT_MAX_PEERS];
+} caat_peers;
+caat_status caat_tp_exchange_bytes(const caat_ctx *ctx, caat_layer layer, int tokens, int world,
+                                   size_t *recv_bytes, int *slice_rows);
+caat_status caat_tp_exchange_scatter(const caat_ctx *ctx, caat_layer layer, int tokens, int backward,
+                                     const caat_peers *peers, unsigned int epoch,
+                                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+caat_status caat_tp_exchange_reduce(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                    const caat_peers *peers, unsigned int epoch, void *cuda_stream);
+caat_status caat_tp_exchange_wait(const caat_ctx *ctx, const caat_peers *peers, unsigned int epoch,
+                                  void *cuda_stream);
+caat_status caat_tp_exchange(const caat_ctx *ctx, caat_layer layer, int tokens, int backward,
+                             const caat_peers *peers, unsigned int epoch,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+caat_status caat_tp_forward_local_push(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                       const void *Y, const void *W,
+                                       const caat_peers *peers, unsigned int epoch,
+                                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Analytic bytes ONE partial channel-reduce would move on a real t-device system
  * (Appendix C: each device sends and receives tokens*h*p activations per reduce;
  * Appendix D: all-reduce = reduce-scatter + all-gather, traffic cut by 100(1-p) %).
@@ -430,7 +490,8 @@ typedef enum {
   CAAT_K_TC_WGRAD = 6,       /* tcgen05 GEMM, weight gradient                       */
   CAAT_K_SPLITK_REDUCE = 7,  /* split-K reduction of the weight gradient            */
   CAAT_K_ACTIVATION = 8,     /* activation of the column-parallel half / its derivative */
-  CAAT_K_COUNT = 9
+  CAAT_K_TP_EXCHANGE = 9,    /* slab exchange over peer memory: scatter, reduce + gather, waits */
+  CAAT_K_COUNT = 10
 } caat_kernel_kind;
 caat_status caat_profile_begin(int max_launches);
 caat_status caat_profile_end(int n_kinds, double *ms_by_kind, unsigned long long *launches_by_kind);

@@ -9,7 +9,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import POINTER, byref, c_char_p, c_double, c_int, c_size_t, c_ulonglong, c_void_p
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_int, c_size_t, c_uint, c_ulonglong, c_void_p
 
 import torch
 
@@ -24,6 +24,13 @@ CAAT_NOALLOC_SCRATCH_BYTES = 32 * 1024 * 1024
 (CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM, CAAT_OPT_ROWS,
  CAAT_OPT_DECODE, CAAT_OPT_BACKWARD_REDUCE, CAAT_OPT_TP_GROUPS) = range(9)
 RMSNORM, LAYERNORM = 0, 1
+CAAT_MAX_PEERS, CAAT_TP_FLAG_BYTES = 8, 256
+
+
+class caat_peers(Structure):
+    """Mirror of the C struct: the GPUs of a slab exchange as this GPU addresses their buffers."""
+    _fields_ = [("world", c_int), ("rank", c_int), ("recv", c_void_p * CAAT_MAX_PEERS),
+                ("slab", c_void_p * CAAT_MAX_PEERS), ("flags", c_void_p * CAAT_MAX_PEERS)]
 CAAT_ACT_NONE, CAAT_ACT_SILU, CAAT_ACT_SWIGLU = 0, 1, 2
 
 if not os.path.exists(LIB_PATH):
@@ -58,6 +65,12 @@ _sigs = {
     "caat_tp_forward_finish": (c_int, [_P, c_int, c_int] + [_P] * 7 + [_P, c_size_t, _P]),
     "caat_tp_backward_local": (c_int, [_P, c_int, c_int] + [_P] * 10 + [_P, c_size_t, _P]),
     "caat_tp_backward_finish": (c_int, [_P, c_int, c_int] + [_P] * 5 + [_P, c_size_t, _P]),
+    "caat_tp_exchange_bytes": (c_int, [_P, c_int, c_int, c_int, POINTER(c_size_t), POINTER(c_int)]),
+    "caat_tp_exchange_scatter": (c_int, [_P, c_int, c_int, c_int, POINTER(caat_peers), c_uint, _P, c_size_t, _P]),
+    "caat_tp_exchange_reduce": (c_int, [_P, c_int, c_int, POINTER(caat_peers), c_uint, _P]),
+    "caat_tp_exchange_wait": (c_int, [_P, POINTER(caat_peers), c_uint, _P]),
+    "caat_tp_exchange": (c_int, [_P, c_int, c_int, c_int, POINTER(caat_peers), c_uint, _P, c_size_t, _P]),
+    "caat_tp_forward_local_push": (c_int, [_P, c_int, c_int, _P, _P, POINTER(caat_peers), c_uint, _P, c_size_t, _P]),
     "caat_allreduce_bytes": (c_int, [_P, c_int, c_int] + [POINTER(c_ulonglong)] * 3),
     "caat_last_device_status": (c_int, [_P, _P]),
     "caat_kernel_launches": (c_ulonglong, []),
@@ -396,6 +409,46 @@ class Context:
             _ptr(dW, torch.float32, (t, h, k), "dW"),
             _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()), "caat_tp_backward_finish")
 
+    # ---- the slab exchange over peer memory (the library's own kernels instead of a collective)
+    def tp_exchange_bytes(self, layer, tokens, world):
+        """(bytes of one GPU's receive buffer, tokens per owner)."""
+        n, sl = c_size_t(), c_int()
+        _check(lib.caat_tp_exchange_bytes(self._h, layer, tokens, world, byref(n), byref(sl)), "caat_tp_exchange_bytes")
+        return n.value, sl.value
+
+    @staticmethod
+    def make_peers(rank, recv_ptrs, slab_ptrs, flag_ptrs):
+        """caat_peers from device addresses (ints), one per GPU of the group, as THIS GPU addresses them."""
+        pe = caat_peers()
+        pe.world, pe.rank = len(flag_ptrs), rank
+        for q in range(pe.world):
+            pe.recv[q] = recv_ptrs[q] if recv_ptrs else None
+            pe.slab[q] = slab_ptrs[q] if slab_ptrs else None
+            pe.flags[q] = flag_ptrs[q]
+        return pe
+
+    def tp_exchange_scatter(self, layer, tokens, backward, peers, epoch, workspace):
+        _check(lib.caat_tp_exchange_scatter(self._h, layer, tokens, 1 if backward else 0, byref(peers), epoch,
+                                            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()),
+               "caat_tp_exchange_scatter")
+
+    def tp_exchange_reduce(self, layer, tokens, peers, epoch):
+        _check(lib.caat_tp_exchange_reduce(self._h, layer, tokens, byref(peers), epoch, _stream()), "caat_tp_exchange_reduce")
+
+    def tp_exchange_wait(self, peers, epoch):
+        _check(lib.caat_tp_exchange_wait(self._h, byref(peers), epoch, _stream()), "caat_tp_exchange_wait")
+
+    def tp_exchange(self, layer, tokens, backward, peers, epoch, workspace):
+        _check(lib.caat_tp_exchange(self._h, layer, tokens, 1 if backward else 0, byref(peers), epoch,
+                                    _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()),
+               "caat_tp_exchange")
+
+    def tp_forward_local_push(self, layer, tokens, Y, W, peers, epoch, workspace):
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        _check(lib.caat_tp_forward_local_push(
+            self._h, layer, tokens, _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"), byref(peers), epoch,
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()), "caat_tp_forward_local_push")
+
     # ---- buffer helpers (torch.empty only; no arithmetic)
     def alloc_workspace(self, nbytes: int, device="cuda"):
         return torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
@@ -421,7 +474,7 @@ def kernel_launches() -> int:
     return int(lib.caat_kernel_launches())
 
 
-CAAT_K_COUNT = 9
+CAAT_K_COUNT = 10
 
 
 def profile_begin(max_launches: int = 65536):

@@ -872,6 +872,7 @@ const char* caat_kernel_kind_name(int kind) {
     case CAAT_K_TC_WGRAD: return "tc_gemm_wgrad";
     case CAAT_K_SPLITK_REDUCE: return "splitk_reduce";
     case CAAT_K_ACTIVATION: return "activation";
+    case CAAT_K_TP_EXCHANGE: return "tp_exchange";
   }
   return "";
 }

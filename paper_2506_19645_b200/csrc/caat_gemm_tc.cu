@@ -83,6 +83,8 @@ struct Params {
   long long out_t_ld;    // channels per token row of out_t
   int cg;                // CTAs per tile: 1, or 2 (tcgen05 cta_group::2, clusters of two)
   int splits;            // split-K factor (only with a single unit and Q == 1)
+  int push_slice;        // > 0: tiles of region 0 (the shared columns) are stored into the peer GPUs' receive slots, the
+                         // owner of a tile being its first row / push_slice (a multiple of the tile's rows)
   int tiles_r0;          // tiles of region 0 (including splits)
   int tiles_total;
   unsigned int* status;
@@ -208,6 +210,9 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
   return d;
 }
 
+// Output maps of the peers' receive slots (the exchange of the shared-channel slab over peer memory).
+struct PeerMaps { CUtensorMap m[CAAT_MAX_PEERS]; };
+
 struct TileCoord {
   int region, b, mt, nt, split;
 };
@@ -294,7 +299,8 @@ template <int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
                const __grid_constant__ CUtensorMap map2, const __grid_constant__ CUtensorMap map3,
-               const __grid_constant__ CUtensorMap cmap0, const __grid_constant__ CUtensorMap cmap1, const Params p) {
+               const __grid_constant__ CUtensorMap cmap0, const __grid_constant__ CUtensorMap cmap1,
+               const __grid_constant__ PeerMaps pm, const Params p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   constexpr int BMT = BM * CG;                     // rows of a tile (of the pair's tile)
   const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;
@@ -516,6 +522,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
       const int n0 = c.nt * p.BN;
       const int m0 = c.mt * BMT + (int)rank * BM;
       const int zc = c.split * r.batch + c.b;
+      // where this tile's rows go: the region's own output, or - shared columns of a multi-GPU forward - the
+      // receive slot of the GPU that owns these token rows, through its own map (row 0 = the owner's first token)
+      const CUtensorMap* omap = cmaps[c.region];
+      int om0 = m0;
+      if (p.push_slice > 0 && c.region == 0) {
+        const int owner = m0 / p.push_slice;
+        omap = &pm.m[owner];
+        om0 = m0 - owner * p.push_slice;
+      }
       const int sub = p.out_f32 ? 16 : 32;
       const int rr = quarter * 32 + lane;                 // row of the tile this thread holds
       const uint32_t sw = (uint32_t)((rr >> 1) & 3);      // 64-byte swizzle: chunk ^= (row / 2) % 4
@@ -574,7 +589,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         if (!(p.debug & kAidMask & 64)) epi_barrier();
         if (warp == 2 && lane == 0 && !(p.debug & kAidMask & 128)) {
-          tma_store_3d(cmaps[c.region], n0 + cc, m0, zc, buf);
+          tma_store_3d(omap, n0 + cc, om0, zc, buf);
           bulk_commit();
           bulk_wait_read1();     // the store before this one has finished reading its buffer
         }
@@ -734,7 +749,8 @@ TileCfg pick_tile(const RegionShape* r, int nr, bool b_n_major, int max_splits, 
   return best;
 }
 
-cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params& p, int kind, cudaStream_t st) {
+cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params& p, int kind, cudaStream_t st,
+                   const PeerMaps* peer_maps = nullptr) {
   const LaunchLimits lim = effective_limits();
   const int stage_bytes = BM * BK * 2 + (p.BN / p.cg) * BK * 2;
   const int budget = lim.gemm_smem > 0 && lim.gemm_smem < 227 * 1024 ? lim.gemm_smem : 227 * 1024;
@@ -781,9 +797,11 @@ cudaError_t launch(const CUtensorMap maps[4], const CUtensorMap cmaps[2], Params
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
   LaunchScope scope(kind, st);
+  static const PeerMaps no_peers{};
+  const PeerMaps& pm = peer_maps ? *peer_maps : no_peers;
   if (p.cg == 2)
-    return cudaLaunchKernelEx(&cfg, tc_gemm_kernel<2>, maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], p);
-  return cudaLaunchKernelEx(&cfg, tc_gemm_kernel<1>, maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], p);
+    return cudaLaunchKernelEx(&cfg, tc_gemm_kernel<2>, maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], pm, p);
+  return cudaLaunchKernelEx(&cfg, tc_gemm_kernel<1>, maps[0], maps[1], maps[2], maps[3], cmaps[0], cmaps[1], pm, p);
 }
 
 void finish_tiles(Params& p) {
@@ -805,8 +823,9 @@ bool tc_gemm_usable(const caat_ctx* ctx, int K_r) {
 
 // ---- forward: zs[T,S] = sum_m Y[m] W[m][:S]^T ; zp[m][T,h-S] = Y[m] W[m][S:]^T
 cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* W, void* zs, void* zp,
-                              cudaStream_t st) {
+                              cudaStream_t st, const PushTarget* push) {
   CUtensorMap maps[4], cmaps[2];
+  PeerMaps pmaps{};
   Params p{};
   const int n_sh = s.S, n_pr = s.h - s.S;
   const int ksteps = (s.K_r + BK - 1) / BK;
@@ -839,8 +858,21 @@ cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* 
   }
   if (g == 1) cmaps[1] = cmaps[0];
   p.nregions = g;
+  if (push && n_sh > 0) {
+    // shared tiles go to the owners' receive slots: slot `rank` of GPU q is [slice, S] 16-bit elements; the map of
+    // owner q covers only the tokens q really owns, so rows past the end of a ragged last slice are clipped
+    if (push->world < 1 || push->world > CAAT_MAX_PEERS || push->slice % (BM * p.cg) != 0) return cudaErrorInvalidValue;
+    for (int q = 0; q < push->world; ++q) {
+      long long rows = (long long)s.T - (long long)q * push->slice;
+      if (rows > push->slice) rows = push->slice;
+      if (rows < 1) { pmaps.m[q] = cmaps[0]; continue; }     // owns no token: never addressed
+      __nv_bfloat16* slot = static_cast<__nv_bfloat16*>(push->recv[q]) + (size_t)push->rank * push->slice * n_sh;
+      if (!make_cmap(&pmaps.m[q], slot, n_sh, rows, 1, n_sh, (long long)push->slice * n_sh, false)) return cudaErrorInvalidValue;
+    }
+    p.push_slice = push->slice;
+  }
   finish_tiles(p);
-  return launch(maps, cmaps, p, CAAT_K_TC_FORWARD, st);
+  return launch(maps, cmaps, p, CAAT_K_TC_FORWARD, st, push && n_sh > 0 ? &pmaps : nullptr);
 }
 
 // ---- decode forward (few tokens): zt[m][i][l] = sum_k W[m][l][k] Y[m][i][k], fp32, for ALL channels.

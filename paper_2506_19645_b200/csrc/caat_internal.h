@@ -80,8 +80,12 @@ struct RowparShapes {
 };
 bool tc_gemm_usable(const caat_ctx* ctx, int K_r);
 // Zt -> (zs, zp):   zs[i,l] = sum_m sum_k Y[m,i,k] W[m,l,k] (l < S);  zp[m,i,l-S_lo] = sum_k ... (l >= S)
+// push != nullptr: the shared columns' tiles are stored into the peer GPUs' receive slots instead of zs
+// (exchange of the slab over peer memory): recv[q] is GPU q's receive buffer [world][slice][S] as this GPU
+// addresses it, the owner of token i is i / slice, slice a multiple of 256
+struct PushTarget { int world, rank, slice; void* const* recv; };
 cudaError_t launch_tc_forward(const RowparShapes& s, const void* Y, const void* W, void* zs, void* zp,
-                              cudaStream_t st);
+                              cudaStream_t st, const PushTarget* push = nullptr);
 // The private part of dZt as the backward GEMMs read it: element (m, i, l) for l >= S sits at
 // ptr[(m * T + i) * ld + col0 + (l - S)], and the gradient is alpha times the stored value.
 //   scratch copy written by the row kernel:   {zp, P, S - S_lo, 1}

@@ -31,7 +31,7 @@ P_SWEEP = (1.0, 0.75, 0.5, 0.25, 0.0)
 ATTN_OUT, MLP_DOWN = 0, 1
 
 
-def plan(workload: str, world: int, tokens: int = 0) -> dict:
+def plan(workload: str, world: int, tokens: int = 0, exchange: str = "nccl") -> dict:
     """How the workload's ranks map onto `world` GPUs: ranks per GPU, total ranks, per-rank contraction widths."""
     w = synthetic.WORKLOADS[workload]
     if tokens > 0:
@@ -40,7 +40,7 @@ def plan(workload: str, world: int, tokens: int = 0) -> dict:
     t_total = t_local * world
     if w.h % t_total or w.ffn % t_total:
         raise SystemExit(f"--mode tp: {t_total} tensor-parallel ranks do not divide h={w.h} / ffn={w.ffn}")
-    return {"workload": w.name, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "world": world, "t_local": t_local,
+    return {"workload": w.name, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "world": world, "t_local": t_local, "exchange": exchange,
             "t_total": t_total, "kr_attn": w.h // t_total, "kr_mlp": w.ffn // t_total, "backward": bool(w.backward)}
 
 
@@ -50,6 +50,7 @@ class _GpuLayers:
     def __init__(self, pl: dict, p: float, device, group=None):
         from . import caat
         self.pl, self.group = pl, group
+        self.exchange = pl.get("exchange", "nccl")
         self.lay = tp.TensorParallelRowLinear(pl["h"], pl["ffn"], pl["t_local"], p, "bf16", group)
         ctx = self.lay.ctx
         self.S = ctx.shared_channels
@@ -64,13 +65,27 @@ class _GpuLayers:
             o = {"Hn": mk(t, T, h), "X": mk(t, T, h), "rstd": mk(t, T, dt=f32), "dY": mk(t, T, k),
                  "dW": mk(t, h, k, dt=f32), "dR": mk(t, T, h), "dg": mk(h, dt=f32)}
             self.layers.append((layer, d, o))
-        self.ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, True), device=device)
         self.payload_elems = T * self.S
-        key = lambda acc: "fp32" if acc == torch.float32 else "16bit"
-        self.payload_keys = (key(self.lay.forward_accumulate), key(self.lay.backward_accumulate))
+        if self.exchange == "push":
+            # the library's own exchange over peer memory: 16-bit wire both ways, fp32 accumulation at the owner
+            self.pbs = [self.lay.peer_buffers(layer, T, device) for layer, _, _ in self.layers]
+            self.ws = self.pbs[0].workspace
+            self.payload_keys = ("16bit", "16bit")
+        else:
+            self.ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, True), device=device)
+            key = lambda acc: "fp32" if acc == torch.float32 else "16bit"
+            self.payload_keys = (key(self.lay.forward_accumulate), key(self.lay.backward_accumulate))
 
     def step(self):
         T, ws = self.pl["tokens"], self.ws
+        if self.exchange == "push":
+            for (layer, d, o), pb in zip(self.layers, self.pbs):
+                self.lay.forward_push(layer, T, d["Y"], d["W"], d["R"], d["gamma"], None, o["Hn"], o["X"], o["rstd"], None, pb)
+            if self.pl["backward"]:
+                for (layer, d, o), pb in zip(reversed(self.layers), reversed(self.pbs)):
+                    self.lay.backward_push(layer, T, d["dX"], d["dHn"], d["Y"], d["W"], o["Hn"], o["rstd"], None, d["gamma"],
+                                           o["dY"], o["dW"], o["dR"], o["dg"], None, pb)
+            return
         for layer, d, o in self.layers:
             self.lay.forward(layer, T, d["Y"], d["W"], d["R"], d["gamma"], None, o["Hn"], o["X"], o["rstd"], None, ws)
         if self.pl["backward"]:
@@ -179,7 +194,7 @@ def run(args, make_layers=_GpuLayers, backend="nccl", out=sys.stdout):
     if world > 1 and not dist.is_initialized():
         dist.init_process_group(backend, **({"device_id": device} if on_gpu else {}))
         created = True
-    pl = plan(args.workload, world, getattr(args, "tokens", 0))
+    pl = plan(args.workload, world, getattr(args, "tokens", 0), getattr(args, "tp_exchange", "nccl"))
     rows = sweep(pl, args.steps, args.warmup, device, make_layers, on_gpu)
     if rank == 0:
         head = next((r for r in rows if r["p"] == 0.5), rows[0])
@@ -191,8 +206,11 @@ def run(args, make_layers=_GpuLayers, backend="nccl", out=sys.stdout):
             "config": {"workload": pl["workload"], "tokens": pl["tokens"], "h": pl["h"], "ffn": pl["ffn"],
                        "tp_ranks": pl["t_total"], "ranks_per_gpu": pl["t_local"], "p": head["p"],
                        "parallelism": f"tp{pl['t_total']} over {world} GPUs",
-                       "exchange": "all-reduce of the packed [T, S] slab between the library's two halves of a layer call "
-                                   f"(forward payload {head['payload_forward']}, backward payload {head['payload_backward']})"},
+                       "exchange": ("the library's exchange kernels over peer memory (reduce-scatter into per-source slots, fp32 "
+                                    "sum in fixed order, all-gather by peer stores; forward GEMM pushes its shared tiles)"
+                                    if pl["exchange"] == "push" else
+                                    "all-reduce of the packed [T, S] slab between the library's two halves of a layer call") +
+                                   f" (forward payload {head['payload_forward']}, backward payload {head['payload_backward']})"},
             "p_sweep": rows,
             "model": "Appendix C with measured constants: step(p) = step(p=0) + p * exchange(p=1), exchange = the step's "
                      "all-reduces timed alone",
