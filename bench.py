@@ -217,10 +217,14 @@ def paper_level_work(w, S, compact=False):
 
 # --------------------------------------------------------------------------- the CUDA arm
 class BlockRunner:
+    overlap = False    # --overlap: the block forward runs layer 1's row kernel beside layer 2's GEMM (CAAT_OPT_BLOCK_OVERLAP)
+
     def __init__(self, w, device, compact=False):
         from paper_2506_19645_b200 import caat
         self.caat, self.w, self.dev, self.compact = caat, w, device, compact
         self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
+        if BlockRunner.overlap:
+            self.ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, 1)
         self.S = self.ctx.shared_channels
         self.inp = synthetic.block_inputs(w, self.S, device=device)
         t, T, h = w.t, w.tokens, w.h
@@ -691,7 +695,10 @@ def config_of(w, S, world, compact, m):
     return {"workload": w.name, "t": w.t, "tokens": w.tokens, "h": w.h, "ffn": w.ffn, "p": w.p,
             "S": S, "passes": passes(w), "private_scale": "sqrt(t)", "norm": "rmsnorm", "parallelism": f"replicas x{world}",
             "residual_layout": "compact (shared channels of the stream stored once)" if compact else "per rank [t,T,h]",
-            "launch": "cuda graph replay" if m["graph"] else "eager", "l2": l2_note(m)}
+            "launch": "cuda graph replay" if m["graph"] else "eager", "l2": l2_note(m),
+            "block_forward_schedule": ("row kernel of layer 1 beside the GEMM of layer 2 (two streams)"
+                                       if BlockRunner.overlap and w.kind == "block" and w.tokens > 64 and not compact
+                                       else "kernels one after the other")}
 
 
 def sweep_entry(name, dev, steps, peaks):
@@ -714,6 +721,19 @@ def sweep_entry(name, dev, steps, peaks):
                                   "entry's own figures are the rotated, cold-L2 ones"}
     del r
     torch.cuda.empty_cache()
+    if w.kind == "block" and w.tokens > 64 and not BlockRunner.overlap:
+        # the same block with the forward's side-by-side schedule (CAAT_OPT_BLOCK_OVERLAP), same steps
+        BlockRunner.overlap = True
+        try:
+            r = BlockRunner(w, dev)
+            for _ in range(3):
+                r.step()
+            oms = time_steps(r, k, False) / k
+            ent["side_by_side_forward_ms_per_step"] = oms
+            del r
+            torch.cuda.empty_cache()
+        finally:
+            BlockRunner.overlap = False
     if w.kind == "block" and w.tokens > 64 and S % 8 == 0:
         # the same block on the compact residual layout (shared channels of the stream stored once)
         r = BlockRunner(w, dev, True)
@@ -876,12 +896,16 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-graph", action="store_true", help="never replay launch-bound steps from a CUDA graph")
+    ap.add_argument("--overlap", action="store_true",
+                    help="block forward: run the first layer's row kernel beside the second layer's GEMM (two streams) "
+                         "instead of the layers' kernels one after the other")
     ap.add_argument("--layout", default="per_rank", choices=["per_rank", "compact"],
                     help="residual-stream layout: per rank [t,T,h] (the benchmark's configuration) or compact")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling on a small case)")
     args = ap.parse_args()
     if args.steps < 1:
         raise SystemExit("--steps must be >= 1")
+    BlockRunner.overlap = args.overlap
     if args.impl == "reference":
         run_reference(args)
     elif args.mode == "tp":

@@ -96,11 +96,17 @@ typedef enum {
                                    2 = rounded, and the running sum is rounded to the run dtype
                                        after every addition (accumulation in 16 bit).
                                    1 and 2 run on the plain-load row kernels.              */
-  CAAT_OPT_TP_GROUPS = 8        /* G >= 1 (default 1): this context holds t of t*G tensor-parallel ranks,
+  CAAT_OPT_TP_GROUPS = 8,       /* G >= 1 (default 1): this context holds t of t*G tensor-parallel ranks,
                                    one group of t ranks per GPU (see caat_tp_*): K_r becomes K / (t*G).
                                    Setting it also sets alpha = sqrt(t*G) (Section 4: the square root of
                                    the number of devices); CAAT_OPT_PRIVATE_SCALE may override that
                                    afterwards.  CAAT_ESHAPE unless t*G divides h and ffn.               */
+  CAAT_OPT_BLOCK_OVERLAP = 9    /* caat_block_forward: 0 (default) = the layers' kernels run one after the other on the
+                                   caller's stream; 1 = the attention-out layer's row kernel (HBM-bound) runs on a second
+                                   stream beside the MLP-down layer's GEMM (tensor-bound), which does not depend on it,
+                                   when the workspace holds both layers' scratch (caat_block_workspace_bytes).  Worth
+                                   2-3 % of a training step at the 1.1B shapes, nothing where the step is launch-bound
+                                   (130M shapes) or the GPU is at its power limit (7B shapes)                          */
 } caat_option;
 
 /* Creates a context for hidden size h, MLP width ffn, t ranks, synchronisation
@@ -116,10 +122,16 @@ int caat_shared_channels(const caat_ctx *ctx);
 /* alpha currently in effect. */
 double caat_private_scale(const caat_ctx *ctx);
 
+/* Bytes of device scratch for the block calls (caat_block_forward / _backward and the compact variants):
+ * enough for the two layers' scratch side by side, which lets the block forward overlap the first layer's row
+ * kernel with the second layer's GEMM.  A workspace of only the larger of the two layers' caat_workspace_bytes
+ * is accepted as well; the block forward then runs its kernels one after the other. */
+size_t caat_block_workspace_bytes(const caat_ctx *ctx, int tokens, int backward);
+
 /* Bytes of device scratch for `tokens` tokens of `layer`: backward = 0, what the forward
  * call needs; backward = 1, enough for the forward AND the backward call (a training step
- * runs both on one buffer; neither keeps anything in it between calls).  For the block
- * calls pass the larger of the two layers' figures (CAAT_MLP_DOWN's, when ffn >= h).
+ * runs both on one buffer; neither keeps anything in it between calls).  The block calls
+ * have their own figure, caat_block_workspace_bytes.
  * 0 on bad arguments. */
 size_t caat_workspace_bytes(const caat_ctx *ctx, caat_layer layer, int tokens, int backward);
 
@@ -219,6 +231,13 @@ caat_status caat_rowpar_backward(const caat_ctx *ctx, caat_layer layer, int toke
  * block, chained through the residual stream: R of the second layer is Hn1.
  * Tensors as in caat_rowpar_forward with K_r = h/t for Y_attn, W_o and ffn/t for
  * Y_mlp, W_down.  beta1/beta2/mean1/mean2 are NULL for RMSNorm.
+ *
+ * The second layer's GEMM does not depend on the first layer's row kernel.  With a workspace of
+ * caat_block_workspace_bytes (both layers' scratch side by side) and CAAT_OPT_BLOCK_OVERLAP set to 1, that row
+ * kernel runs on a stream of the library's own, forked from and joined back into `cuda_stream` with events
+ * inside this call (legal inside a stream capture; the library creates that stream on the first such call per
+ * device, so make one call before capturing): everything the call enqueued is ordered before whatever the caller
+ * enqueues on `cuda_stream` next.  Results do not depend on the schedule.
  */
 caat_status caat_block_forward(const caat_ctx *ctx, int tokens,
                                const void *Y_attn, const void *W_o,

@@ -22,7 +22,7 @@ CAAT_ATTN_OUT, CAAT_MLP_DOWN = 0, 1
  CAAT_ETIMEOUT, CAAT_ELIMIT) = range(9)
 CAAT_NOALLOC_SCRATCH_BYTES = 32 * 1024 * 1024
 (CAAT_OPT_NORM, CAAT_OPT_EPS, CAAT_OPT_PRIVATE_SCALE, CAAT_OPT_SHARED_CHANNELS, CAAT_OPT_GEMM, CAAT_OPT_ROWS,
- CAAT_OPT_DECODE, CAAT_OPT_BACKWARD_REDUCE, CAAT_OPT_TP_GROUPS) = range(9)
+ CAAT_OPT_DECODE, CAAT_OPT_BACKWARD_REDUCE, CAAT_OPT_TP_GROUPS, CAAT_OPT_BLOCK_OVERLAP) = range(10)
 RMSNORM, LAYERNORM = 0, 1
 CAAT_MAX_PEERS, CAAT_TP_FLAG_BYTES = 8, 256
 
@@ -46,6 +46,7 @@ _sigs = {
     "caat_shared_channels": (c_int, [_P]),
     "caat_private_scale": (c_double, [_P]),
     "caat_workspace_bytes": (c_size_t, [_P, c_int, c_int, c_int]),
+    "caat_block_workspace_bytes": (c_size_t, [_P, c_int, c_int]),
     "caat_strerror": (c_char_p, [c_int]),
     "caat_last_cuda_error": (c_char_p, []),
     "caat_rowpar_forward": (c_int, [_P, c_int, c_int] + [_P] * 9 + [_P, c_size_t, _P]),
@@ -170,8 +171,7 @@ class Context:
         return lib.caat_workspace_bytes(self._h, layer, tokens, 1 if backward else 0)
 
     def block_workspace_bytes(self, tokens: int, backward: bool) -> int:
-        return max(self.workspace_bytes(CAAT_ATTN_OUT, tokens, backward),
-                   self.workspace_bytes(CAAT_MLP_DOWN, tokens, backward))
+        return lib.caat_block_workspace_bytes(self._h, tokens, 1 if backward else 0)
 
     def allreduce_bytes(self, tokens: int, elem_bytes: int = 2) -> dict:
         a, b, c = c_ulonglong(), c_ulonglong(), c_ulonglong()

@@ -22,6 +22,7 @@ struct caat_ctx {
   int no_decode;   // CAAT_OPT_DECODE
   int bwd_reduce;  // CAAT_OPT_BACKWARD_REDUCE
   int groups;      // CAAT_OPT_TP_GROUPS: this context holds t of t * groups tensor-parallel ranks
+  int block_overlap;  // CAAT_OPT_BLOCK_OVERLAP: the block forward runs the first layer's row kernel beside the second GEMM
 };
 
 namespace caat {

@@ -300,3 +300,49 @@ def test_decode_7b_forward(T, p):
     for layer, k in ((caat.CAAT_ATTN_OUT, w.kr_attn), (caat.CAAT_MLP_DOWN, w.kr_mlp)):
         d = _layer_case(w.t, T, w.h, k, "bf16", O.shared_channels(w.h, w.p), seed=T)
         _check_forward(ctx, layer, d, "bf16")
+
+
+@pytest.mark.parametrize("t,T,h,ffn,p,norm", [(4, 1500, 768, 3072, 0.5, 0), (8, 700, 2048, 5632, 0.25, 1), (8, 300, 4096, 11008, 1.0, 0)])
+def test_block_forward_side_by_side_schedule_equals_the_serial_one(t, T, h, ffn, p, norm):
+    # the block forward that runs the first layer's row kernel beside the second layer's GEMM (second stream,
+    # plain-load row kernel, a GEMM with one pipeline stage less) against the same call with the overlap switched
+    # off, and against a workspace too small for two scratch regions (which must fall back to the serial schedule)
+    w = synthetic.Workload("blk_ovl", t, T, h, ffn, p, "bf16", "block", False, 11)
+    S = O.shared_channels(h, p)
+    d = synthetic.block_inputs(w, S)
+    g = torch.Generator().manual_seed(5)
+    for k in ("gamma1", "gamma2"):
+        d[k] = (1 + 0.1 * torch.randn(h, generator=g)).to(torch.bfloat16)
+    b1 = (0.1 * torch.randn(h, generator=g)).to(torch.bfloat16).cuda() if norm else None
+    b2 = (0.1 * torch.randn(h, generator=g)).to(torch.bfloat16).cuda() if norm else None
+    dev = {k: v.cuda() for k, v in d.items()}
+    mk = lambda *s, dt=torch.bfloat16: torch.empty(*s, dtype=dt, device="cuda")
+    outs = []
+    for overlap, small_ws in ((1, False), (0, False), (1, True)):
+        ctx = G.make_ctx(t, h, ffn, "bf16", p=p, norm=norm)
+        assert ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, overlap) is ctx
+        nbytes = ctx.block_workspace_bytes(T, False)
+        one = max(ctx.workspace_bytes(caat.CAAT_ATTN_OUT, T, False), ctx.workspace_bytes(caat.CAAT_MLP_DOWN, T, False))
+        assert nbytes > one
+        ws = ctx.alloc_workspace(one if small_ws else nbytes)
+        o = {"Hn1": mk(t, T, h), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=torch.float32), "Hn2": mk(t, T, h), "X2": mk(t, T, h),
+             "rstd2": mk(t, T, dt=torch.float32)}
+        m1 = mk(t, T, dt=torch.float32) if norm else None
+        m2 = mk(t, T, dt=torch.float32) if norm else None
+        launches = caat.kernel_launches()
+        ctx.block_forward(T, dev["Y_attn"], dev["W_o"], dev["Y_mlp"], dev["W_down"], dev["R0"], dev["gamma1"], b1,
+                          dev["gamma2"], b2, o["Hn1"], o["X1"], o["rstd1"], m1, o["Hn2"], o["X2"], o["rstd2"], m2, ws)
+        torch.cuda.synchronize()
+        assert caat.kernel_launches() - launches == 4
+        assert ctx.last_device_status() == caat.CAAT_OK
+        outs.append(o)
+    fo = O.block_forward(f64(d["Y_attn"]), f64(d["W_o"]), f64(d["Y_mlp"]), f64(d["W_down"]), f64(d["R0"]), f64(d["gamma1"]),
+                         f64(d["gamma2"]), f64(b1.cpu()) if norm else None, f64(b2.cpu()) if norm else None, S=S,
+                         alpha=math.sqrt(t), norm=norm)
+    for k in outs[0]:
+        assert_close(outs[0][k], fo[k], "bf16", f"side by side: {k}")
+        assert torch.equal(outs[1][k], outs[2][k]), f"serial schedule, two workspace sizes: {k}"
+        if k.startswith("Hn"):        # sums and one rounding per element: the same on every row-kernel variant
+            assert torch.equal(outs[0][k], outs[1][k]), f"side by side against serial: {k}"
+        else:                         # the row statistics are reduced in another order by the plain-load kernel
+            assert_close(outs[0][k], f64(outs[1][k]), "bf16", f"side by side against serial: {k}", scale=0.5)
