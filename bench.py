@@ -217,14 +217,14 @@ def paper_level_work(w, S, compact=False):
 
 # --------------------------------------------------------------------------- the CUDA arm
 class BlockRunner:
-    overlap = False    # --overlap: the block forward runs layer 1's row kernel beside layer 2's GEMM (CAAT_OPT_BLOCK_OVERLAP)
+    overlap = True     # --no-overlap: the block forward's kernels one after the other (CAAT_OPT_BLOCK_OVERLAP = 0)
 
     def __init__(self, w, device, compact=False):
         from paper_2506_19645_b200 import caat
         self.caat, self.w, self.dev, self.compact = caat, w, device, compact
         self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
-        if BlockRunner.overlap:
-            self.ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, 1)
+        if not BlockRunner.overlap:
+            self.ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, 0)
         self.S = self.ctx.shared_channels
         self.inp = synthetic.block_inputs(w, self.S, device=device)
         t, T, h = w.t, w.tokens, w.h
@@ -721,19 +721,19 @@ def sweep_entry(name, dev, steps, peaks):
                                   "entry's own figures are the rotated, cold-L2 ones"}
     del r
     torch.cuda.empty_cache()
-    if w.kind == "block" and w.tokens > 64 and not BlockRunner.overlap:
-        # the same block with the forward's side-by-side schedule (CAAT_OPT_BLOCK_OVERLAP), same steps
-        BlockRunner.overlap = True
+    if w.kind == "block" and w.tokens > 64 and BlockRunner.overlap:
+        # the same block with the forward's kernels one after the other (CAAT_OPT_BLOCK_OVERLAP = 0), same steps
+        BlockRunner.overlap = False
         try:
             r = BlockRunner(w, dev)
             for _ in range(3):
                 r.step()
             oms = time_steps(r, k, False) / k
-            ent["side_by_side_forward_ms_per_step"] = oms
+            ent["serial_forward_ms_per_step"] = oms
             del r
             torch.cuda.empty_cache()
         finally:
-            BlockRunner.overlap = False
+            BlockRunner.overlap = True
     if w.kind == "block" and w.tokens > 64 and S % 8 == 0:
         # the same block on the compact residual layout (shared channels of the stream stored once)
         r = BlockRunner(w, dev, True)
@@ -896,16 +896,16 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU oracle baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-graph", action="store_true", help="never replay launch-bound steps from a CUDA graph")
-    ap.add_argument("--overlap", action="store_true",
-                    help="block forward: run the first layer's row kernel beside the second layer's GEMM (two streams) "
-                         "instead of the layers' kernels one after the other")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="block forward: run the layers' kernels one after the other instead of the first layer's row "
+                         "kernel beside the second layer's GEMM (the library's default, two streams)")
     ap.add_argument("--layout", default="per_rank", choices=["per_rank", "compact"],
                     help="residual-stream layout: per rank [t,T,h] (the benchmark's configuration) or compact")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling on a small case)")
     args = ap.parse_args()
     if args.steps < 1:
         raise SystemExit("--steps must be >= 1")
-    BlockRunner.overlap = args.overlap
+    BlockRunner.overlap = not args.no_overlap
     if args.impl == "reference":
         run_reference(args)
     elif args.mode == "tp":

@@ -390,7 +390,7 @@ caat_status caat_create(int h, int ffn, int t, double p, caat_dtype dtype, caat_
   c->alpha = std::sqrt((double)t);         // Section 4: private channels times sqrt(r)
   c->norm = 0; c->eps = 1e-5; c->force_simt = 0; c->direct_rows = 0; c->no_decode = 0; c->bwd_reduce = 0;
   c->groups = 1;
-  c->block_overlap = 0;
+  c->block_overlap = 1;
   *out = c;
   return CAAT_OK;
 }
@@ -518,8 +518,8 @@ size_t caat_block_workspace_bytes(const caat_ctx* ctx, int tokens, int backward)
 // The GEMM's CTAs fill every SM's shared memory, so the row kernel that shares the SMs with it is the plain-load
 // variant (registers only); the GEMM gives up one pipeline stage, which leaves the row kernel's loads some L1.
 // Measured: the pair alone gains 13-19 % (7B shapes: 1.74 ms one after the other, 1.41-1.51 ms side by side), a whole
-// training step 2.5 % at the 1.1B shapes and nothing at the 130M shapes (launch-bound) or the 7B shapes (the GPU runs
-// into its power limit there: with both kernels active the clock drops and the step takes as long).  Off by default.
+// training step 2-4 % at the 130M and 1.1B shapes and 1-2 % at the 7B shapes (the GPU runs into its power limit there:
+// with both kernels active the clock drops, which eats most of the gain).
 static caat_status block_forward_overlapped(const caat_ctx* ctx, int tokens, const void* Y_attn, const void* W_o,
                                             const void* Y_mlp, const void* W_down, const void* R0, const void* gamma1,
                                             const void* beta1, const void* gamma2, const void* beta2, void* Hn1, void* X1,

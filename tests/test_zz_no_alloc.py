@@ -12,6 +12,8 @@ leaves the device's free memory and the framework's allocation count where they 
 
 Collected last on purpose (file name), so a run that stops at the first failure has already run
 every other test.  Passes alone in a fresh process and after the other tests."""
+import gc
+
 import pytest
 import torch
 
@@ -85,12 +87,19 @@ def test_noalloc_call_allocates_nothing():
         out = ctx.alloc_forward_outputs(T)
         _noalloc(ctx, layer, d, T, out)       # the first call per device may load the module: not measured
         torch.cuda.synchronize()
-        free0, _ = torch.cuda.mem_get_info()
-        alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
-        _noalloc(ctx, layer, d, T, out)
-        free1, _ = torch.cuda.mem_get_info()
-        assert free1 == free0, f"T={T}: free device memory moved by {free0 - free1} bytes across the call"
-        assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+        gc.collect()                          # leftovers of earlier tests must not be released in the middle of the check
+        gc.disable()
+        try:
+            free0, _ = torch.cuda.mem_get_info()
+            count0 = torch.cuda.memory_stats()["allocation.all.allocated"]
+            alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+            _noalloc(ctx, layer, d, T, out)
+            free1, _ = torch.cuda.mem_get_info()
+            assert free1 == free0, f"T={T}: free device memory moved by {free0 - free1} bytes across the call"
+            assert torch.cuda.memory_stats()["allocation.all.allocated"] == count0     # no request to the framework's allocator
+            assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+        finally:
+            gc.enable()
 
 
 def test_noalloc_rejects_sizes_beyond_its_scratch():
