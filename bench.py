@@ -217,14 +217,14 @@ def paper_level_work(w, S, compact=False):
 
 # --------------------------------------------------------------------------- the CUDA arm
 class BlockRunner:
-    overlap = True     # --no-overlap: the block forward's kernels one after the other (CAAT_OPT_BLOCK_OVERLAP = 0)
+    overlap = None     # --overlap / --no-overlap force CAAT_OPT_BLOCK_OVERLAP to 1 / 0; None: the library's own choice
 
     def __init__(self, w, device, compact=False):
         from paper_2506_19645_b200 import caat
         self.caat, self.w, self.dev, self.compact = caat, w, device, compact
         self.ctx = caat.Context(w.h, w.ffn, w.t, w.p, w.dtype)
-        if not BlockRunner.overlap:
-            self.ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, 0)
+        if BlockRunner.overlap is not None:
+            self.ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, 1 if BlockRunner.overlap else 0)
         self.S = self.ctx.shared_channels
         self.inp = synthetic.block_inputs(w, self.S, device=device)
         t, T, h = w.t, w.tokens, w.h
@@ -696,9 +696,9 @@ def config_of(w, S, world, compact, m):
             "S": S, "passes": passes(w), "private_scale": "sqrt(t)", "norm": "rmsnorm", "parallelism": f"replicas x{world}",
             "residual_layout": "compact (shared channels of the stream stored once)" if compact else "per rank [t,T,h]",
             "launch": "cuda graph replay" if m["graph"] else "eager", "l2": l2_note(m),
-            "block_forward_schedule": ("row kernel of layer 1 beside the GEMM of layer 2 (two streams)"
-                                       if BlockRunner.overlap and w.kind == "block" and w.tokens > 64 and not compact
-                                       else "kernels one after the other")}
+            "block_forward_schedule": {None: "library's choice by shape (side by side unless the GEMM is much the longer kernel)",
+                                       True: "row kernel of layer 1 beside the GEMM of layer 2 (two streams)",
+                                       False: "kernels one after the other"}[BlockRunner.overlap]}
 
 
 def sweep_entry(name, dev, steps, peaks):
@@ -721,19 +721,21 @@ def sweep_entry(name, dev, steps, peaks):
                                   "entry's own figures are the rotated, cold-L2 ones"}
     del r
     torch.cuda.empty_cache()
-    if w.kind == "block" and w.tokens > 64 and BlockRunner.overlap:
-        # the same block with the forward's kernels one after the other (CAAT_OPT_BLOCK_OVERLAP = 0), same steps
-        BlockRunner.overlap = False
-        try:
-            r = BlockRunner(w, dev)
-            for _ in range(3):
-                r.step()
-            oms = time_steps(r, k, False) / k
-            ent["serial_forward_ms_per_step"] = oms
-            del r
-            torch.cuda.empty_cache()
-        finally:
-            BlockRunner.overlap = True
+    if w.kind == "block" and w.tokens > 64 and BlockRunner.overlap is None:
+        # the same block with the forward's schedule forced either way (CAAT_OPT_BLOCK_OVERLAP = 0 / 1), same steps.
+        # The kernel table above comes from the library's own schedule: where two kernels share the GPU their event
+        # times include each other's slow-down, so the serial pass's table is printed as well.
+        for flag, key in ((False, "serial_forward"), (True, "side_by_side_forward")):
+            BlockRunner.overlap = flag
+            try:
+                m2, r2 = measure(w, dev, k, 3, False, kernels=not flag)
+                ent[key + "_ms_per_step"] = m2["ms_total"] / k
+                if not flag:
+                    ent["kernels_serial_forward"] = kernel_table(m2["prof"], step_work(w, S), k, peaks)
+                del r2
+                torch.cuda.empty_cache()
+            finally:
+                BlockRunner.overlap = None
     if w.kind == "block" and w.tokens > 64 and S % 8 == 0:
         # the same block on the compact residual layout (shared channels of the stream stored once)
         r = BlockRunner(w, dev, True)
@@ -897,15 +899,17 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-graph", action="store_true", help="never replay launch-bound steps from a CUDA graph")
     ap.add_argument("--no-overlap", action="store_true",
-                    help="block forward: run the layers' kernels one after the other instead of the first layer's row "
-                         "kernel beside the second layer's GEMM (the library's default, two streams)")
+                    help="block forward: run the layers' kernels one after the other (CAAT_OPT_BLOCK_OVERLAP = 0)")
+    ap.add_argument("--overlap", action="store_true",
+                    help="block forward: run the first layer's row kernel beside the second layer's GEMM on two streams "
+                         "(CAAT_OPT_BLOCK_OVERLAP = 1); default: the library chooses by shape")
     ap.add_argument("--layout", default="per_rank", choices=["per_rank", "compact"],
                     help="residual-stream layout: per rank [t,T,h] (the benchmark's configuration) or compact")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling on a small case)")
     args = ap.parse_args()
     if args.steps < 1:
         raise SystemExit("--steps must be >= 1")
-    BlockRunner.overlap = not args.no_overlap
+    BlockRunner.overlap = True if args.overlap else (False if args.no_overlap else None)
     if args.impl == "reference":
         run_reference(args)
     elif args.mode == "tp":

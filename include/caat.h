@@ -101,11 +101,13 @@ typedef enum {
                                    Setting it also sets alpha = sqrt(t*G) (Section 4: the square root of
                                    the number of devices); CAAT_OPT_PRIVATE_SCALE may override that
                                    afterwards.  CAAT_ESHAPE unless t*G divides h and ffn.               */
-  CAAT_OPT_BLOCK_OVERLAP = 9    /* caat_block_forward: 1 (default) = the attention-out layer's row kernel (HBM-bound) runs on a
-                                   second stream beside the MLP-down layer's GEMM (tensor-bound), which does not depend
-                                   on it, when the workspace holds both layers' scratch (caat_block_workspace_bytes);
-                                   0 = the layers' kernels run one after the other on the caller's stream.  Worth 2-4 %
-                                   of a training step at the 130M / 1.1B shapes, 1-2 % at the 7B shapes (power limit)   */
+  CAAT_OPT_BLOCK_OVERLAP = 9    /* caat_block_forward: 1 = the attention-out layer's row kernel (HBM-bound) runs on a second
+                                   stream beside the MLP-down layer's GEMM (tensor-bound), which does not depend on it,
+                                   when the workspace holds both layers' scratch (caat_block_workspace_bytes); 0 = the
+                                   layers' kernels run one after the other on the caller's stream; 2 (default) = 1
+                                   unless that GEMM is much the longer of the two kernels (ffn / t large, e.g. the 7B
+                                   shapes, where the GPU is at its power limit and running both at once gains nothing).
+                                   Worth 2-4 % of a training step at the 130M / 1.1B shapes                             */
 } caat_option;
 
 /* Creates a context for hidden size h, MLP width ffn, t ranks, synchronisation
@@ -232,7 +234,7 @@ caat_status caat_rowpar_backward(const caat_ctx *ctx, caat_layer layer, int toke
  * Y_mlp, W_down.  beta1/beta2/mean1/mean2 are NULL for RMSNorm.
  *
  * The second layer's GEMM does not depend on the first layer's row kernel.  With a workspace of
- * caat_block_workspace_bytes (both layers' scratch side by side) and CAAT_OPT_BLOCK_OVERLAP on (the default), that row
+ * caat_block_workspace_bytes (both layers' scratch side by side) and CAAT_OPT_BLOCK_OVERLAP on (or chosen automatically), that row
  * kernel runs on a stream of the library's own, forked from and joined back into `cuda_stream` with events
  * inside this call (legal inside a stream capture; the library creates that stream on the first such call per
  * device, so make one call before capturing): everything the call enqueued is ordered before whatever the caller

@@ -390,7 +390,7 @@ caat_status caat_create(int h, int ffn, int t, double p, caat_dtype dtype, caat_
   c->alpha = std::sqrt((double)t);         // Section 4: private channels times sqrt(r)
   c->norm = 0; c->eps = 1e-5; c->force_simt = 0; c->direct_rows = 0; c->no_decode = 0; c->bwd_reduce = 0;
   c->groups = 1;
-  c->block_overlap = 1;
+  c->block_overlap = 2;
   *out = c;
   return CAAT_OK;
 }
@@ -424,7 +424,7 @@ caat_status caat_set_option(caat_ctx* ctx, caat_option opt, double value) {
       if (value != 0.0 && value != 1.0 && value != 2.0) return CAAT_EINVAL;
       ctx->bwd_reduce = (int)value; return CAAT_OK;
     case CAAT_OPT_BLOCK_OVERLAP:
-      if (value != 0.0 && value != 1.0) return CAAT_EINVAL;
+      if (value != 0.0 && value != 1.0 && value != 2.0) return CAAT_EINVAL;
       ctx->block_overlap = (int)value; return CAAT_OK;
     case CAAT_OPT_TP_GROUPS: {
       if (value != std::floor(value) || value < 1.0 || value > 65536.0) return CAAT_EINVAL;
@@ -519,7 +519,15 @@ size_t caat_block_workspace_bytes(const caat_ctx* ctx, int tokens, int backward)
 // variant (registers only); the GEMM gives up one pipeline stage, which leaves the row kernel's loads some L1.
 // Measured: the pair alone gains 13-19 % (7B shapes: 1.74 ms one after the other, 1.41-1.51 ms side by side), a whole
 // training step 2-4 % at the 130M and 1.1B shapes and 1-2 % at the 7B shapes (the GPU runs into its power limit there:
-// with both kernels active the clock drops, which eats most of the gain).
+// with both kernels active the clock drops, which eats the gain).  Hence the automatic choice below: side by side
+// unless the GEMM is the much longer of the two.
+static bool overlap_pays(const caat_ctx* ctx) {
+  if (ctx->block_overlap != 2) return ctx->block_overlap == 1;
+  // time of the MLP-down GEMM at the tensor rate over the time of a row kernel at the HBM rate (tokens cancel):
+  // (2 K h / 1.4e15) / (3 t h e / 6.4e12).  1.1 at the 1.1B shapes, 1.2 at 130M, 2.1 at 7B.
+  const double ratio = (2.0 * ctx->ffn / ctx->groups / 1.4e15) / (3.0 * ctx->t * elem_size(ctx->dtype) / 6.4e12);
+  return ratio <= 1.5;
+}
 static caat_status block_forward_overlapped(const caat_ctx* ctx, int tokens, const void* Y_attn, const void* W_o,
                                             const void* Y_mlp, const void* W_down, const void* R0, const void* gamma1,
                                             const void* beta1, const void* gamma2, const void* beta2, void* Hn1, void* X1,
@@ -566,7 +574,7 @@ caat_status caat_block_forward(const caat_ctx* ctx, int tokens, const void* Y_at
   if (block_decode_applies(ctx, tokens))
     return block_decode(ctx, tokens, Y_attn, W_o, Y_mlp, W_down, R0, gamma1, beta1, gamma2, beta2, Hn1, X1, rstd1, mean1,
                         Hn2, X2, rstd2, mean2, workspace, workspace_bytes, cuda_stream, 0, nullptr, nullptr, nullptr);
-  if (ctx && ctx->block_overlap && !ctx->direct_rows && check_common(ctx, CAAT_MLP_DOWN, tokens) == CAAT_OK &&
+  if (ctx && overlap_pays(ctx) && !ctx->direct_rows && check_common(ctx, CAAT_MLP_DOWN, tokens) == CAAT_OK &&
       tc_gemm_usable(ctx, layer_kr(ctx, CAAT_ATTN_OUT)) && tc_gemm_usable(ctx, layer_kr(ctx, CAAT_MLP_DOWN)) &&
       Y_attn && W_o && Y_mlp && W_down && R0 && gamma1 && gamma2 && Hn1 && X1 && rstd1 && Hn2 && X2 && rstd2 &&
       (ctx->norm == 0 || (mean1 && mean2)) && Hn1 != R0 && workspace &&
