@@ -346,3 +346,36 @@ def test_block_forward_side_by_side_schedule_equals_the_serial_one(t, T, h, ffn,
             assert torch.equal(outs[0][k], outs[1][k]), f"side by side against serial: {k}"
         else:                         # the row statistics are reduced in another order by the plain-load kernel
             assert_close(outs[0][k], f64(outs[1][k]), "bf16", f"side by side against serial: {k}", scale=0.5)
+
+
+def test_side_by_side_block_forward_inside_a_stream_capture():
+    # the fork onto the library's own stream and the join back are events recorded and waited on inside the call,
+    # which a stream capture turns into graph edges: the captured call replays to the same results as the eager one
+    t, T, h, ffn, p = 4, 1500, 768, 3072, 0.5
+    w = synthetic.Workload("blk_graph", t, T, h, ffn, p, "bf16", "block", False, 13)
+    dev = {k: v.cuda() for k, v in synthetic.block_inputs(w, O.shared_channels(h, p)).items()}
+    ctx = G.make_ctx(t, h, ffn, "bf16", p=p)
+    ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, 1)
+    ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, False))
+    mk = lambda *s, dt=torch.bfloat16: torch.empty(*s, dtype=dt, device="cuda")
+    outs = [{"Hn1": mk(t, T, h), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=torch.float32), "Hn2": mk(t, T, h), "X2": mk(t, T, h),
+             "rstd2": mk(t, T, dt=torch.float32)} for _ in range(2)]
+
+    def call(o):
+        ctx.block_forward(T, dev["Y_attn"], dev["W_o"], dev["Y_mlp"], dev["W_down"], dev["R0"], dev["gamma1"], None,
+                          dev["gamma2"], None, o["Hn1"], o["X1"], o["rstd1"], None, o["Hn2"], o["X2"], o["rstd2"], None, ws)
+
+    call(outs[0])                                   # eager; also creates the library's stream before any capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        call(outs[1])
+    for v in outs[1].values():
+        v.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+    for k in outs[0]:
+        assert torch.equal(outs[0][k], outs[1][k]), k
