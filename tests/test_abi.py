@@ -136,3 +136,47 @@ def test_tensor_parallel_groups_and_slab(caat):
     assert caat.lib.caat_tp_slab(odd._h, caat.CAAT_MLP_DOWN, 64, 0, None, None, None) == caat.CAAT_EUNSUPPORTED
     # the halves reject a missing workspace before any launch
     assert caat.lib.caat_tp_forward_local(ctx._h, caat.CAAT_MLP_DOWN, 300, None, None, None, 0, None) == caat.CAAT_EWORKSPACE
+
+
+def test_block_workspace_and_schedule_option(caat):
+    # the block calls' scratch: both layers' forward regions side by side, never less than one layer's full need
+    ctx = caat.Context(2048, 5632, 8, 0.5, "bf16")
+    A, M = caat.CAAT_ATTN_OUT, caat.CAAT_MLP_DOWN
+    for T in (300, 16384):
+        for backward in (False, True):
+            one = max(ctx.workspace_bytes(A, T, backward), ctx.workspace_bytes(M, T, backward))
+            both = ctx.block_workspace_bytes(T, backward)
+            assert both >= one
+            assert both >= ctx.workspace_bytes(A, T, False) + ctx.workspace_bytes(M, T, False)
+    assert caat.lib.caat_block_workspace_bytes(None, 16, 0) == 0
+    assert caat.lib.caat_block_workspace_bytes(ctx._h, 0, 0) == 0
+    for v in (0, 1, 2):
+        ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, v)
+    with pytest.raises(caat.CaatError) as e:
+        ctx.set_option(caat.CAAT_OPT_BLOCK_OVERLAP, 3)
+    assert e.value.status == caat.CAAT_EINVAL
+
+
+def test_exchange_geometry_and_argument_errors(caat):
+    # the slab exchange over peer memory: slices of tokens per owner, receive-buffer size, arguments checked on the host
+    ctx = caat.Context(4096, 11008, 1, 0.5, "bf16")
+    ctx.set_option(caat.CAAT_OPT_TP_GROUPS, 8)
+    M = caat.CAAT_MLP_DOWN
+    assert ctx.tp_exchange_bytes(M, 16384, 8) == (8 * 2048 * 2048 * 2, 2048)       # [world][slice][S] 16-bit
+    assert ctx.tp_exchange_bytes(M, 1000, 4)[1] == 256                              # ceil(1000/4) = 250 -> 8-row units
+    assert ctx.tp_exchange_bytes(M, 4097, 2)[1] == 2304                             # 2049 -> whole 256-row pair tiles
+    assert ctx.tp_exchange_bytes(M, 130, 8)[1] == 24
+    n = ctypes.c_size_t()
+    assert caat.lib.caat_tp_exchange_bytes(ctx._h, M, 64, 9, ctypes.byref(n), None) == caat.CAAT_EINVAL      # > CAAT_MAX_PEERS
+    assert caat.lib.caat_tp_exchange_bytes(ctx._h, M, 0, 2, ctypes.byref(n), None) == caat.CAAT_ESHAPE
+    c32 = caat.Context(256, 1024, 2, 0.5, "f32")
+    assert caat.lib.caat_tp_exchange_bytes(c32._h, M, 64, 2, ctypes.byref(n), None) == caat.CAAT_EUNSUPPORTED
+    pe = caat.caat_peers()
+    pe.world, pe.rank = 2, 2                                                        # rank outside the group
+    assert caat.lib.caat_tp_exchange_wait(ctx._h, ctypes.byref(pe), 1, None) == caat.CAAT_EINVAL
+    pe.rank = 0                                                                     # no flag words given
+    assert caat.lib.caat_tp_exchange_wait(ctx._h, ctypes.byref(pe), 1, None) == caat.CAAT_EINVAL
+    pe.flags[0] = pe.flags[1] = 0x1008                                              # not 16-byte aligned
+    assert caat.lib.caat_tp_exchange_wait(ctx._h, ctypes.byref(pe), 1, None) == caat.CAAT_EALIGN
+    assert caat.lib.caat_tp_exchange_reduce(ctx._h, M, 64, None, 1, None) == caat.CAAT_EINVAL
+    assert ctypes.sizeof(caat.caat_peers) == 8 + 3 * 8 * caat.CAAT_MAX_PEERS         # the C struct's layout
