@@ -806,12 +806,16 @@ cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype,
   // more rows than two CTAs of 512 threads per SM can hold at once (64 registers per thread): two chunks per thread in
   // CTAs of 256, four of which fit an SM, keep every row's CTA resident in one wave (7B shapes, 64 tokens: -3.6 %)
   if (threads > 256 && (long long)a.T * a.t > 2LL * sm_count()) threads = 256;
-  if (dtype == CAAT_BF16) {
-    if (a.norm == 1) return launch_pdl(rows_forward_partials_kernel<__nv_bfloat16, true>, grid, dim3(threads), smem, st, a);
-    return launch_pdl(rows_forward_partials_kernel<__nv_bfloat16, false>, grid, dim3(threads), smem, st, a);
-  }
-  if (a.norm == 1) return launch_pdl(rows_forward_partials_kernel<float, true>, grid, dim3(threads), smem, st, a);
-  return launch_pdl(rows_forward_partials_kernel<float, false>, grid, dim3(threads), smem, st, a);
+  auto go = [&](auto kernel) -> cudaError_t {
+    if (smem > 48 * 1024) {   // long rows: more dynamic shared memory than a kernel gets without asking
+      const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    return launch_pdl(kernel, grid, dim3(threads), smem, st, a);
+  };
+  if (dtype == CAAT_BF16)
+    return a.norm == 1 ? go(rows_forward_partials_kernel<__nv_bfloat16, true>) : go(rows_forward_partials_kernel<__nv_bfloat16, false>);
+  return a.norm == 1 ? go(rows_forward_partials_kernel<float, true>) : go(rows_forward_partials_kernel<float, false>);
 }
 
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype) {

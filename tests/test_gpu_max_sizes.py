@@ -91,3 +91,27 @@ def test_rowpar_beyond_2_31_elements():
         del dY2, dR2
     assert_close((parts_W[0] + parts_W[1]).cpu(), f64(dW.cpu()), "f32", "dW halves")
     assert_close((parts_g[0] + parts_g[1]).cpu(), f64(dg.cpu()), "f32", "dgamma halves")
+
+
+@pytest.mark.parametrize("T,norm", [(3, 0), (40, 1)])
+def test_longest_rows_with_few_tokens(T, norm):
+    # h = 16384, the longest row the library takes (2048 16-byte chunks): the few-token row kernels keep a whole
+    # row in shared memory as fp32, 64 KB here - more than a kernel gets without asking for it
+    from paper_2506_19645_b200 import synthetic
+    t, h, ffn, S = 2, 16384, 16384, 8192
+    ctx = caat.Context(h, ffn, t, 0.5, "bf16")
+    ctx.set_option(caat.CAAT_OPT_NORM, norm)
+    layer, k = caat.CAAT_MLP_DOWN, ffn // t
+    d = synthetic.layer_inputs(t, T, h, k, "bf16", seed=T, S=S)
+    dev = {n: v.cuda() for n, v in d.items()}
+    out = ctx.alloc_forward_outputs(T)
+    mean = torch.empty((t, T), dtype=torch.float32, device="cuda") if norm else None
+    ws = ctx.alloc_workspace(ctx.workspace_bytes(layer, T, False))
+    ctx.rowpar_forward(layer, T, dev["Y"], dev["W"], dev["R"], dev["gamma"], dev["beta"] if norm else None, out["Hn"], out["X"],
+                       out["rstd"], mean, ws)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == caat.CAAT_OK
+    fo = O.rowpar_forward(f64(d["Y"]), f64(d["W"]), f64(d["R"]), f64(d["gamma"]), f64(d["beta"]) if norm else None, S=S,
+                          alpha=ctx.private_scale, norm=norm)
+    for name in ("Hn", "X", "rstd"):
+        assert_close(out[name].cpu(), fo[name], "bf16", name)
