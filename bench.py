@@ -418,6 +418,55 @@ def tp_projection(dev, name="block_7b", steps=20):
             "rows": rows}
 
 
+def library_gemm_yardstick(w, dev, secs=1.0):
+    """Context for the GEMM fractions, NOT part of the path: the vendor library's batched GEMM (torch.bmm) on the
+    workload's own shapes - t products [T, K_r] x [K_r, h] and their two gradient products per layer - each run back to
+    back for about `secs` seconds, i.e. under the same power cap as the step.  The peak the fractions are quoted
+    against comes from an 8192^3 product; the layer's shards are shorter in the contraction and write more output per
+    flop, and this says how much of the gap the shapes themselves account for."""
+    t, T, h = w.t, w.tokens, w.h
+    out = {}
+    bf = torch.bfloat16
+
+    def sustained(fn, flops):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        n, t0 = 0, time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        while True:
+            for _ in range(5):
+                fn()
+            n += 5
+            if time.perf_counter() - t0 > secs:
+                break
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / n
+        return ms, flops / (ms * 1e-3) / 1e12
+
+    tot = {"forward": [0.0, 0.0], "dgrad": [0.0, 0.0], "wgrad": [0.0, 0.0]}
+    for K in layer_widths(w):
+        Y = torch.randn(t, T, K, device=dev, dtype=bf)
+        W = torch.randn(t, h, K, device=dev, dtype=bf) * 0.02
+        Gd = torch.randn(t, T, h, device=dev, dtype=bf)
+        Z, dY, dW = torch.empty(t, T, h, device=dev, dtype=bf), torch.empty_like(Y), torch.empty_like(W)
+        fl = 2.0 * t * T * K * h
+        for kind, fn in (("forward", lambda: torch.bmm(Y, W.transpose(1, 2), out=Z)), ("dgrad", lambda: torch.bmm(Gd, W, out=dY)),
+                         ("wgrad", lambda: torch.bmm(Gd.transpose(1, 2), Y, out=dW))):
+            ms, _ = sustained(fn, fl)
+            tot[kind][0] += ms
+            tot[kind][1] += fl
+        del Y, W, Gd, Z, dY, dW
+        torch.cuda.empty_cache()
+    for kind, (ms, fl) in tot.items():
+        out[kind] = {"ms_per_step": ms, "tflops": fl / (ms * 1e-3) / 1e12}
+    out["note"] = ("vendor-library batched GEMM (torch.bmm, bf16) on this workload's per-rank shapes, both layers, each "
+                   f"product looped for about {secs:g} s; a yardstick for the shapes, not a step of the path")
+    return out
+
+
 def make_runner(w, device, compact=False):
     if w.kind == "mlp":
         return MlpRunner(w, device, compact)
@@ -822,6 +871,17 @@ def run_cuda(args):
                                          "not the headline figure"}
     del runner
     torch.cuda.empty_cache()
+
+    if rank == 0 and world == 1 and not args.no_sweep and w.kind == "block" and w.backward and w.dtype == "bf16":
+        try:
+            result["library_gemm_same_shapes"] = library_gemm_yardstick(w, dev)
+            for kind, v in result["library_gemm_same_shapes"].items():
+                k = "tc_gemm_" + kind
+                if isinstance(v, dict) and k in result["kernels"] and "achieved" in result["kernels"][k]:
+                    result["kernels"][k]["vs_library_gemm_same_shapes"] = result["kernels"][k]["achieved"] / v["tflops"]
+        except Exception as ex:  # noqa: BLE001
+            result["library_gemm_same_shapes"] = {"error": str(ex)[:200]}
+            torch.cuda.empty_cache()
 
     if rank == 0 and not args.no_sweep and world == 1:
         sweep = []
