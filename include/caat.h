@@ -420,6 +420,8 @@ caat_status caat_tp_backward_finish(const caat_ctx *ctx, caat_layer layer, int t
  *             on GPU q.  caat_tp_forward_local_push does the same from inside the forward GEMM: the
  *             tiles of the shared columns leave the epilogue straight for their owner's slot while
  *             the private columns' tiles are still being multiplied, and the slab is never written.
+ *             caat_tp_backward_local_push is the backward's counterpart: the row kernel that forms the
+ *             reduced shared gradient stores each token's row into its owner's slot instead of the slab.
  *   reduce    GPU q waits for all `world` flags, sums the `world` slots of its token slice in fp32 in
  *             the fixed order 0..world-1, rounds once to the run dtype and stores the result rows
  *             into EVERY GPU's slab (the all-gather), then raises flag `world + q` on every GPU.
@@ -467,6 +469,14 @@ caat_status caat_tp_forward_local_push(const caat_ctx *ctx, caat_layer layer, in
                                        const void *Y, const void *W,
                                        const caat_peers *peers, unsigned int epoch,
                                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+/* caat_tp_backward_local (same tensors) with the scatter phase folded into the row kernel; follow it with
+ * caat_tp_exchange_reduce and caat_tp_exchange_wait, then caat_tp_backward_finish.  Any slice_rows. */
+caat_status caat_tp_backward_local_push(const caat_ctx *ctx, caat_layer layer, int tokens,
+                                        const void *dX, const void *dHn, const void *W, const void *Hn,
+                                        const float *rstd, const float *mean, const void *gamma,
+                                        void *dR, float *dgamma, float *dbeta,
+                                        const caat_peers *peers, unsigned int epoch,
+                                        void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Analytic bytes ONE partial channel-reduce would move on a real t-device system

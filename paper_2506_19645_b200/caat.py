@@ -72,6 +72,7 @@ _sigs = {
     "caat_tp_exchange_wait": (c_int, [_P, POINTER(caat_peers), c_uint, _P]),
     "caat_tp_exchange": (c_int, [_P, c_int, c_int, c_int, POINTER(caat_peers), c_uint, _P, c_size_t, _P]),
     "caat_tp_forward_local_push": (c_int, [_P, c_int, c_int, _P, _P, POINTER(caat_peers), c_uint, _P, c_size_t, _P]),
+    "caat_tp_backward_local_push": (c_int, [_P, c_int, c_int] + [_P] * 10 + [POINTER(caat_peers), c_uint, _P, c_size_t, _P]),
     "caat_allreduce_bytes": (c_int, [_P, c_int, c_int] + [POINTER(c_ulonglong)] * 3),
     "caat_last_device_status": (c_int, [_P, _P]),
     "caat_kernel_launches": (c_ulonglong, []),
@@ -448,6 +449,17 @@ class Context:
         _check(lib.caat_tp_forward_local_push(
             self._h, layer, tokens, _ptr(Y, td, (t, tokens, k), "Y"), _ptr(W, td, (t, h, k), "W"), byref(peers), epoch,
             _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()), "caat_tp_forward_local_push")
+
+    def tp_backward_local_push(self, layer, tokens, dX, dHn, W, Hn, rstd, mean, gamma, dR, dgamma, dbeta, peers, epoch,
+                               workspace):
+        td, t, h, k = self.torch_dtype, self.t, self.h, self.k_r(layer)
+        f32 = torch.float32
+        _check(lib.caat_tp_backward_local_push(
+            self._h, layer, tokens, _ptr(dX, td, (t, tokens, h), "dX"), _ptr(dHn, td, (t, tokens, h), "dHn"),
+            _ptr(W, td, (t, h, k), "W"), _ptr(Hn, td, (t, tokens, h), "Hn"), _ptr(rstd, f32, (t, tokens), "rstd"),
+            _ptr(mean, f32, (t, tokens), "mean"), _ptr(gamma, td, (h,), "gamma"), _ptr(dR, td, (t, tokens, h), "dR"),
+            _ptr(dgamma, f32, (h,), "dgamma"), _ptr(dbeta, f32, (h,), "dbeta"), byref(peers), epoch,
+            _ptr(workspace, torch.uint8, None, "workspace"), workspace.numel(), _stream()), "caat_tp_backward_local_push")
 
     # ---- buffer helpers (torch.empty only; no arithmetic)
     def alloc_workspace(self, nbytes: int, device="cuda"):

@@ -248,7 +248,8 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
                                  const void* W, const void* Hn, const float* rstd, const float* mean,
                                  const void* gamma, void* dY, float* dW, void* dR, float* dgamma, float* dbeta,
                                  void* ws, cudaStream_t st, int compact = 0, const void* Hns = nullptr,
-                                 const void* dHns = nullptr, void* dRs = nullptr, int phase = 0) {
+                                 const void* dHns = nullptr, void* dRs = nullptr, int phase = 0,
+                                 const PushTarget* push = nullptr) {
   // phase: 0 = the whole layer; 1 = the row kernel only (dR, the shared gradient slab, the norm-parameter
   // gradients, the scaled weight rows); 2 = the two GEMMs only, on the slab as it then stands
   // compact: Hn / dHn / dR are the private parts; the shared residual gradient dRs [T, S] is at the
@@ -271,6 +272,10 @@ static caat_status backward_impl(const caat_ctx* ctx, int K_r, int T, const void
                dgamma, dbeta, t, T, h, S, L.S_lo, L.S_hi, L.P, (float)ctx->alpha, ctx->norm};
   a.compact = compact; a.Hns = Hns; a.dHns = dHns;
   a.reduce_mode = ctx->bwd_reduce;
+  if (push) {   // the reduced shared gradient goes straight to the owners' receive slots (multi-GPU exchange)
+    a.gs_slice = push->slice; a.gs_rank = push->rank;
+    for (int q = 0; q < push->world && q < CAAT_MAX_PEERS; ++q) a.gs_recv[q] = push->recv[q];
+  }
   const bool prescale = tc && ctx->alpha != 1.0 && S < h;
   if (prescale) { a.w_src = W; a.w_dst = wsb + L.wt_off; a.w_Kr = K_r; }
   if (phase != 2) {
@@ -886,6 +891,28 @@ caat_status caat_tp_backward_local(const caat_ctx* ctx, caat_layer layer, int to
                        dR, dgamma, dbeta, workspace, static_cast<cudaStream_t>(cuda_stream), 0, nullptr, nullptr,
                        nullptr, 1);
 }
+
+}  // extern "C"
+
+namespace caat {
+caat_status tp_backward_local_push_impl(const caat_ctx* ctx, caat_layer layer, int tokens, const void* dX, const void* dHn,
+                                        const void* W, const void* Hn, const float* rstd, const float* mean,
+                                        const void* gamma, void* dR, float* dgamma, float* dbeta, void* workspace,
+                                        size_t workspace_bytes, cudaStream_t st, const PushTarget& push) {
+  caat_status s = check_tp(ctx, layer, tokens, workspace, workspace_bytes, 1);
+  if (s != CAAT_OK) return s;
+  if (!dX || !W || !Hn || !rstd || !gamma || !dR || !dgamma) return CAAT_EINVAL;
+  if (ctx->norm == 1 && (!mean || !dbeta)) return CAAT_EINVAL;
+  if (ctx->bwd_reduce != 0) return CAAT_EUNSUPPORTED;      // the numerics-study modes run on kernels without this path
+  const void* ptrs[] = {dX, dHn, W, Hn, rstd, mean, gamma, dR, dgamma, dbeta};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return CAAT_EALIGN;
+  return backward_impl(ctx, layer_kr(ctx, layer), tokens, dX, dHn, nullptr, W, Hn, rstd, mean, gamma, nullptr, nullptr, dR,
+                       dgamma, dbeta, workspace, st, 0, nullptr, nullptr, nullptr, 1, &push);
+}
+}  // namespace caat
+
+extern "C" {
 
 caat_status caat_tp_backward_finish(const caat_ctx* ctx, caat_layer layer, int tokens, const void* Y, const void* W,
                                     const void* dR, void* dY, float* dW, void* workspace, size_t workspace_bytes,

@@ -169,7 +169,21 @@ struct RowBwdArgs {
   const void* w_src;
   void* w_dst;
   int w_Kr;
+  // exchange of the gradient slab over peer memory: gs_slice > 0 sends row i of the reduced shared gradient to slot
+  // gs_rank of GPU i / gs_slice (gs_recv[q] = that GPU's receive buffer [world][gs_slice][S]) instead of to gs
+  int gs_slice, gs_rank;
+  void* gs_recv[CAAT_MAX_PEERS];
 };
+#ifdef __CUDACC__
+// where row i of the reduced shared gradient goes (S_hi == S whenever the slab is exchanged)
+__device__ __forceinline__ char* gs_row(const RowBwdArgs& a, long long i, int ES) {
+  if (a.gs_slice > 0) {
+    const int q = (int)(i / a.gs_slice);
+    return static_cast<char*>(a.gs_recv[q]) + (((long long)a.gs_rank * a.gs_slice + (i - (long long)q * a.gs_slice)) * a.S_hi) * ES;
+  }
+  return static_cast<char*>(a.gs) + i * a.S_hi * ES;
+}
+#endif
 cudaError_t launch_rows_backward(const RowBwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st);
 cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,
                                         cudaStream_t st);
@@ -211,6 +225,13 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.numAttrs = pdl_enabled() ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+
+// first half of the backward (row kernel, norm-gradient reduction) with the gradient slab's rows sent to the
+// owners' receive slots
+caat_status tp_backward_local_push_impl(const caat_ctx* ctx, caat_layer layer, int tokens, const void* dX, const void* dHn,
+                                        const void* W, const void* Hn, const float* rstd, const float* mean,
+                                        const void* gamma, void* dR, float* dgamma, float* dbeta, void* workspace,
+                                        size_t workspace_bytes, cudaStream_t st, const PushTarget& push);
 
 // ---- launch limits ---------------------------------------------------------------
 // A block call runs a layer's HBM-bound row kernel beside the other layer's tensor-bound GEMMs by giving

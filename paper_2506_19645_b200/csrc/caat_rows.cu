@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(512, CPT == 1 ? 2 : 1) rows_backward_kernel(co
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
       if (act[j] && cls[j] != 1)
-        stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, V_::pack(gsum[j]));
+        stg<raw>(gs_row(a, i, ES) + (long long)col[j] * ES, V_::pack(gsum[j]));
   }
 
   // Partial norm-parameter gradients of this CTA: one row of [h] per CTA.  With several

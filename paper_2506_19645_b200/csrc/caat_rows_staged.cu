@@ -580,7 +580,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
 #pragma unroll
     for (int j = 0; j < CPT; ++j)
       if (act[j] && cls[j] != 1)
-        stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, pack2(gsum[j]));
+        stg<raw>(gs_row(a, i, ES) + (long long)col[j] * ES, pack2(gsum[j]));
     // park the next group's statistics; the last barrier of this group separates these writes
     // from the reads of group n-1's buffer, the barrier below from the reads of group n+1
 #pragma unroll

@@ -509,7 +509,7 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
 #pragma unroll
       for (int j = 0; j < CPT; ++j)
         if (valid && colok[j] && cls[j] != 1)
-          stg<raw>(static_cast<char*>(a.gs) + (i * a.S_hi + col[j]) * ES, pack2(gsum[j]));
+          stg<raw>(gs_row(a, i, ES) + (long long)col[j] * ES, pack2(gsum[j]));
     }
   }
 

@@ -275,4 +275,23 @@ caat_status caat_tp_forward_local_push(const caat_ctx* ctx, caat_layer layer, in
   return e == cudaSuccess ? CAAT_OK : cuda_fail(e);
 }
 
+caat_status caat_tp_backward_local_push(const caat_ctx* ctx, caat_layer layer, int tokens, const void* dX,
+                                        const void* dHn, const void* W, const void* Hn, const float* rstd,
+                                        const float* mean, const void* gamma, void* dR, float* dgamma, float* dbeta,
+                                        const caat_peers* peers, unsigned int epoch, void* workspace,
+                                        size_t workspace_bytes, void* cuda_stream) {
+  Peers pr{};
+  caat_status s = check_peers(ctx, peers, &pr, true, false);
+  if (s != CAAT_OK) return s;
+  if (tokens < 1) return CAAT_ESHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const PushTarget pt{peers->world, peers->rank, slice_rows(tokens, peers->world), pr.recv};
+  s = tp_backward_local_push_impl(ctx, layer, tokens, dX, dHn, W, Hn, rstd, mean, gamma, dR, dgamma, dbeta, workspace,
+                                  workspace_bytes, st, pt);
+  if (s != CAAT_OK) return s;
+  LaunchScope scope(CAAT_K_TP_EXCHANGE, st);
+  const cudaError_t e = launch_pdl(tp_signal_kernel, dim3(1), dim3(32), 0, st, pr, peers->world, peers->rank, epoch);
+  return e == cudaSuccess ? CAAT_OK : cuda_fail(e);
+}
+
 }  // extern "C"

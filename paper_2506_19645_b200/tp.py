@@ -142,9 +142,14 @@ class TensorParallelRowLinear:
 
     def backward_push(self, layer, tokens, dX, dHn, Y, W, Hn, rstd, mean, gamma, dY, dW, dR, dgamma, dbeta, pb: PeerBuffers):
         c = self.ctx
-        c.tp_backward_local(layer, tokens, dX, dHn, W, Hn, rstd, mean, gamma, dR, dgamma, dbeta, pb.workspace)
-        if c.shared_channels > 0:
-            c.tp_exchange(layer, tokens, True, pb.peers(True), pb.next_epoch(), pb.workspace)
+        if c.shared_channels > 0:     # the row kernel sends each token's reduced gradient row to its owner's slot
+            pe, epoch = pb.peers(True), pb.next_epoch()
+            c.tp_backward_local_push(layer, tokens, dX, dHn, W, Hn, rstd, mean, gamma, dR, dgamma, dbeta, pe, epoch,
+                                     pb.workspace)
+            c.tp_exchange_reduce(layer, tokens, pe, epoch)
+            c.tp_exchange_wait(pe, epoch)
+        else:
+            c.tp_backward_local(layer, tokens, dX, dHn, W, Hn, rstd, mean, gamma, dR, dgamma, dbeta, pb.workspace)
         allreduce_slab(dgamma, self.group)          # fp32 [h], a few KB: the library collective
         if dbeta is not None:
             allreduce_slab(dbeta, self.group)

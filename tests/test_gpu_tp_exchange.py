@@ -230,3 +230,47 @@ def test_wrapper_with_its_own_exchange_in_a_group_of_one(T):
         for k in ref:
             assert torch.equal(ref[k], got[k]), k
     assert pb.epoch == 4
+
+
+@pytest.mark.parametrize("t,G,T,h,ffn,S,layer,norm", [
+    (8, 4, 300, 1024, 4096, 512, caat.CAAT_ATTN_OUT, 0),      # warp-per-token row kernel, ragged slices of 80 tokens
+    (8, 8, 130, 2048, 8192, 1024, caat.CAAT_MLP_DOWN, 1),     # staged row kernel, LayerNorm, owners without tokens
+    (4, 2, 700, 768, 3072, 768, caat.CAAT_MLP_DOWN, 0),       # p = 1
+])
+def test_backward_row_kernel_sending_the_slab_rows_equals_row_kernel_plus_scatter(t, G, T, h, ffn, S, layer, norm):
+    tl = t // G
+    K = (h if layer == caat.CAAT_ATTN_OUT else ffn) // t
+    d = synthetic.layer_inputs(t, T, h, K, "bf16", seed=9 + T, S=S, backward=True)
+    fo = O.rowpar_forward(f64(d["Y"]), f64(d["W"]), f64(d["R"]), f64(d["gamma"]), f64(d["beta"]) if norm else None, S=S,
+                          alpha=float(np.sqrt(t)), norm=norm)
+    sHn, srs = to_dtype(fo["Hn"], BF).cuda(), to_dtype(fo["rstd"], F32).cuda()
+    smu = to_dtype(fo["mean"], F32).cuda() if norm else None
+    dev = {k: v.cuda() for k, v in d.items()}
+    sl = lambda x, q: x[q * tl:(q + 1) * tl]
+    mk = lambda *s, dt=BF: torch.empty(*s, dtype=dt, device="cuda")
+    results = []
+    for fused in (False, True):
+        groups = [Group(tl, G, h, ffn, S, layer, T, norm) for _ in range(G)]
+        peers, slabs = make_peers(groups, layer, T, True)
+        dY, dW, dR = mk(t, T, K), mk(t, h, K, dt=F32), mk(t, T, h)
+        dgs = [mk(h, dt=F32) for _ in range(G)]
+        dbs = [mk(h, dt=F32) if norm else None for _ in range(G)]
+        for q, (g, pe) in enumerate(zip(groups, peers)):
+            args = (layer, T, sl(dev["dX"], q), sl(dev["dHn"], q), sl(dev["W"], q), sl(sHn, q), sl(srs, q).clone(),
+                    sl(smu, q).clone() if norm else None, dev["gamma"], sl(dR, q), dgs[q], dbs[q])
+            if fused:
+                g.ctx.tp_backward_local_push(*args, pe, 3, g.ws)
+            else:
+                g.ctx.tp_backward_local(*args, g.ws)
+        exchange(groups, peers, layer, T, True, epoch=3, scatter=not fused)
+        for q, g in enumerate(groups):
+            g.ctx.tp_backward_finish(layer, T, sl(dev["Y"], q), sl(dev["W"], q), sl(dR, q), sl(dY, q), sl(dW, q), g.ws)
+        torch.cuda.synchronize()
+        assert all(g.ctx.last_device_status() == caat.CAAT_OK for g in groups)
+        results.append((slabs[0].clone(), dY, dW, dR, torch.stack(dgs).sum(0)))
+    for a, b, name in zip(results[0], results[1], ("slab", "dY", "dW", "dR", "dgamma")):
+        assert torch.equal(a, b), name
+    ob = O.rowpar_backward(f64(d["dX"]), f64(d["dHn"]), f64(d["Y"]), f64(d["W"]), f64(sHn.cpu()), f64(srs.cpu()),
+                           f64(smu.cpu()) if norm else None, f64(d["gamma"]), S=S, alpha=float(np.sqrt(t)), norm=norm)
+    assert_close(results[1][1].cpu(), ob["dY"], "bf16", "dY (fused) against the oracle")
+    assert_close(results[1][2].cpu(), ob["dW"], "bf16", "dW (fused) against the oracle")
