@@ -150,20 +150,9 @@ def test_full_size_block_130m_chained():
     _check_block_full("block_130m", seed=77, chained=True)
 
 
-@pytest.mark.parametrize("name", ["block_1p1b_p100", "block_1p1b_p050", "block_1p1b_p025"])
+@pytest.mark.parametrize("name", ["block_1p1b_p100", "block_1p1b_p075", "block_1p1b_p050", "block_1p1b_p025"])
 def test_full_size_block_1p1b(name):
     _check_block_full(name)
-
-
-def test_full_size_block_1p1b_p075_forward_sample():
-    # p = 0.75 at full size: forward only (the backward reduce at this S is covered at reduced T)
-    w = synthetic.WORKLOADS["block_1p1b_p075"]
-    fw = synthetic.Workload("block_1p1b_p075_fwd", w.t, w.tokens, w.h, w.ffn, w.p, w.dtype, w.kind, False, w.seed)
-    synthetic.WORKLOADS[fw.name] = fw
-    try:
-        _check_block_full(fw.name)
-    finally:
-        del synthetic.WORKLOADS[fw.name]
 
 
 def test_full_size_block_7b():
