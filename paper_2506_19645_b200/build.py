@@ -17,7 +17,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libcaat.so")
-SOURCES = ["caat_api.cu", "caat_rows.cu", "caat_rows_staged.cu", "caat_rows_warp.cu", "caat_gemm_simt.cu",
+SOURCES = ["caat_api.cu", "caat_rows.cu", "caat_rows_staged.cu", "caat_rows_lean.cu", "caat_rows_warp.cu", "caat_gemm_simt.cu",
            "caat_gemm_tc.cu", "caat_static.cu", "caat_colpar.cu", "caat_tp_push.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 

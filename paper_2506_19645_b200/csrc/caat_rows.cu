@@ -783,7 +783,11 @@ cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype,
   LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
   // few rows: the cluster kernel, as long as all its CTAs are resident at once (portable cluster size 8,
   // one chunk per thread, one CTA per SM at its register count; clusters need whole groups of SMs, hence 3/4)
+#ifdef CAAT_MEASUREMENT_AIDS
   static const int cluster_mode = [] { const char* e = getenv("CAAT_DECODE_CLUSTER"); return e ? atoi(e) : 1; }();
+#else
+  constexpr int cluster_mode = 1;
+#endif
   if (cluster_mode && dtype == CAAT_BF16 && a.t >= 2 && a.t <= 8 && a.h % V == 0 && a.h / V <= 512 && a.S % 4 == 0 &&
       (a.h - a.S) % 4 == 0) {
     const size_t csm = cluster_partials_smem(a);
@@ -824,9 +828,13 @@ int rows_backward_partial_rows(int h, int T, caat_dtype dtype) {
   return ngroups < kMaxPartialRows ? ngroups : kMaxPartialRows;
 }
 
-static int rows_mode_override(int direct) {   // CAAT_ROWS_MODE = 0/1/2 overrides the context option (experiments)
+static int rows_mode_override(int direct) {   // measurement builds: CAAT_ROWS_MODE = 0/1/2 overrides the context option
+#ifdef CAAT_MEASUREMENT_AIDS
   static const int env = [] { const char* e = getenv("CAAT_ROWS_MODE"); return e ? atoi(e) : -1; }();
   return env >= 0 ? env : direct;
+#else
+  return direct;
+#endif
 }
 
 cudaError_t launch_rows_forward(const RowFwdArgs& a, caat_dtype dtype, int direct, cudaStream_t st) {

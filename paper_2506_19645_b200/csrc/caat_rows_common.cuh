@@ -156,7 +156,11 @@ inline RowGeom row_geometry(int h, caat_dtype dtype) {
   // Two chunks per thread whenever the row is long enough: the per-rank overhead (barrier
   // wait, row reduction, pointer updates) is paid once per thread, and 256 threads with up
   // to 128 registers leave room for two CTAs per SM without spills.
+#ifdef CAAT_MEASUREMENT_AIDS
   static const int thr = [] { const char* e = getenv("CAAT_ROWS_CPT1_MAX"); return e ? atoi(e) : 128; }();
+#else
+  constexpr int thr = 128;
+#endif
   g.CPT = chunks <= thr ? 1 : 2;   // short rows: one chunk per thread keeps every lane busy and more warps resident
   int tx = round_up((chunks + g.CPT - 1) / g.CPT, 32);
   while (tx > 512) {

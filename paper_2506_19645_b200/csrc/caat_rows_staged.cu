@@ -13,71 +13,15 @@
 // CTAs are persistent (token groups strided by the grid).  Every mbarrier wait is bounded:
 // on a timeout the CTA sets the library's status word, drains its copies in flight and
 // returns.
-#include "caat_rows_common.cuh"
+#include "caat_rows_bulk.cuh"
 
 namespace caat {
 namespace {
 
 using namespace rows;
 
-constexpr uint32_t kSpinCap = 1u << 18;
-constexpr uint32_t kSuspendHintNs = 20000u;   // the waiting warp sleeps in hardware instead of spinning
-constexpr int kMaxStages = 8;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
-      : "memory");
-  return ok != 0;
-}
-// one lane of a converged warp (the hardware's pick); branching on it keeps the control flow warp-uniform
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.u32 %0, 1, 0, P;\n}" : "=r"(pred));
-  return pred != 0;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kSpinCap; ++it)
-    if (mbar_try(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-
-template <typename raw>
-__device__ __forceinline__ raw lds(const uint8_t* p) { return *reinterpret_cast<const raw*>(p); }
-
-struct StageGeom {
-  int nstages;
-  uint32_t off_a, off_b, off_c;  // byte offsets of the three row buffers inside a stage
-  uint32_t off_d, off_e;         // compact layout: the shared rows of the stream (and of its gradient)
-  uint32_t stage_bytes;
-  uint32_t ring_off, bar_off, red_off, stat_off, acc_off;
-  uint32_t zero_off;             // 16 zero bytes inside every stage (read by chunks past the row end)
-  uint32_t keep_off;             // compact backward: [TY, S] shared rows of the stream, kept for all ranks of a token group
-  size_t smem;
-};
-
 // ------------------------------------------------------------------ forward
 // stage buffers: a = R rows [TY, h], b = zp rows [TY, P], c = zs rows [TY, S_hi] (rank 0 only)
-// resident CTAs per SM the launch bounds ask for: one chunk per thread in small CTAs leaves ~85
-// registers per thread at three CTAs, two chunks per thread 128 registers at two CTAs
-template <int CPT, int MAXT>
-struct MinBlocks { static constexpr int value = MAXT <= 256 ? (CPT == 1 ? 3 : 2) : (CPT == 1 ? 2 : 1); };
-
 // compact layout (CL): a = private residual rows [TY, P], d = shared residual rows [TY, S] (rank 0 only)
 template <typename T_, int CPT, bool LN, int MAXT, bool CL>
 __global__ void __launch_bounds__(MAXT, MinBlocks<CPT, MAXT>::value)
@@ -656,54 +600,6 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
 }
 
 // ------------------------------------------------------------------ host side
-StageGeom stage_geometry(const RowGeom& g, int h, int P, int S_hi, int t, int ES, bool backward, bool has_c,
-                         bool compact, size_t budget) {
-  StageGeom sg{};
-  const uint32_t rowA = (uint32_t)g.TY * h * ES;
-  const uint32_t rowP = (uint32_t)g.TY * P * ES, rowS = (uint32_t)g.TY * S_hi * ES;
-  if (backward && compact) {          // dX | Hnp | dHnp | Hns | dHns   (P + S_hi = h)
-    sg.off_a = 0; sg.off_b = rowA; sg.off_c = rowA + rowP;
-    sg.off_d = has_c ? rowA + 2 * rowP : rowA + rowP;
-    sg.off_e = sg.off_d + rowS;
-    sg.stage_bytes = sg.off_d + (has_c ? 2 : 1) * rowS;
-  } else if (backward) {
-    sg.off_a = 0; sg.off_b = rowA; sg.off_c = 2 * rowA;
-    sg.stage_bytes = (has_c ? 3 : 2) * rowA;
-  } else if (compact) {               // Rp | zp | zs | Rs
-    sg.off_a = 0; sg.off_b = rowP; sg.off_c = 2 * rowP; sg.off_d = 2 * rowP + rowS;
-    sg.stage_bytes = 2 * rowP + 2 * rowS;
-  } else {
-    sg.off_a = 0; sg.off_b = rowA; sg.off_c = rowA + rowP;
-    sg.stage_bytes = rowA + rowP + rowS;
-  }
-  sg.zero_off = sg.stage_bytes;
-  sg.stage_bytes = (sg.stage_bytes + 16u + 127u) & ~127u;
-  // fixed part: barriers + abort flag, reduction scratch, row statistics
-  size_t off = 0;
-  sg.bar_off = (uint32_t)off; off += 8 * kMaxStages + 16;
-  off = align_up(off, 16);
-  sg.red_off = (uint32_t)off; off += (size_t)2 * g.TY * 16 * 2 * sizeof(float);
-  sg.stat_off = (uint32_t)off; off += backward ? (size_t)2 * 2 * t * g.TY * sizeof(float) : 0;
-  off = align_up(off, 128);
-  sg.keep_off = (uint32_t)off; off += (backward && compact) ? (size_t)rowS : 0;
-  off = align_up(off, 128);
-  sg.ring_off = (uint32_t)off;
-  sg.acc_off = sg.ring_off;
-  const size_t acc = (backward && g.TY > 1) ? (size_t)g.TY * g.TX * g.CPT * (16 / ES) * sizeof(float) : 0;
-  int ns = (int)((budget - off) / sg.stage_bytes);
-  if (ns > kMaxStages) ns = kMaxStages;
-  sg.nstages = ns;
-  size_t ring = (size_t)(ns > 0 ? ns : 0) * sg.stage_bytes;
-  if (ring < acc) ring = acc;
-  sg.smem = off + ring;
-  return sg;
-}
-
-template <typename K>
-cudaError_t set_smem(K kernel, size_t bytes) {
-  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-}
-
 template <typename T_, bool LN, bool CL>
 cudaError_t launch_fwd_staged_t(const RowFwdArgs& a, const RowGeom& g, const StageGeom& sg, int grid, int ngroups,
                                 unsigned int* status, cudaStream_t st) {
@@ -748,18 +644,19 @@ cudaError_t launch_bwd_staged_t(const RowBwdArgs& a, const RowGeom& g, const Sta
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-constexpr size_t kSmemPerSm = 227 * 1024;
-
-// resident CTAs per SM the register budget allows (64 registers per thread when CPT == 1)
-int ctas_per_sm(const RowGeom& g) {
-  const int threads = g.TX * g.TY;
-  if (g.CPT != 1) return threads <= 256 ? 2 : 1;   // 128 registers per thread
-  if (threads > 256) return 2;                      // 64 registers per thread
-  int n = 65536 / (threads * 80);                   // 80 registers per thread
-  return n < 1 ? 1 : (n > 6 ? 6 : n);
-}
-
 }  // namespace
+
+// the lean kernels take over wherever they apply (a measurement build can keep the general kernels:
+// CAAT_ROWS_LEAN bit 0 = forward, bit 1 = backward)
+static bool rows_lean_enabled(int dir) {
+#ifdef CAAT_MEASUREMENT_AIDS
+  static const int on = [] { const char* e = getenv("CAAT_ROWS_LEAN"); return e ? atoi(e) : 3; }();
+  return (on >> dir) & 1;
+#else
+  (void)dir;
+  return true;
+#endif
+}
 
 bool rows_staged_usable(int h, int t, int S_lo, int S_hi, caat_dtype dtype, bool backward) {
   const RowGeom g = row_geometry(h, dtype);
@@ -787,6 +684,8 @@ cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cu
   if (grid > ngroups) grid = ngroups;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
+  if (rows_lean_enabled(0) && rows_lean_usable(a.compact, a.h, a.T, a.S, a.S_lo, a.S_hi, dtype))
+    return launch_rows_forward_lean(a, dtype, g, sg, grid, ngroups, status, st);
   if (cl) {
     if (dtype == CAAT_BF16)
       return a.norm == 1 ? launch_fwd_staged_t<__nv_bfloat16, true, true>(a, g, sg, grid, ngroups, status, st)
@@ -825,6 +724,8 @@ cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, i
   *rows_used = grid;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
+  if (rows_lean_enabled(1) && rows_lean_usable(a.compact, a.h, a.T, a.S, a.S_lo, a.S_hi, dtype))
+    return launch_rows_backward_lean(a, dtype, g, sg, grid, ngroups, status, st);
   if (cl) {
     if (dtype == CAAT_BF16)
       return a.norm == 1 ? launch_bwd_staged_t<__nv_bfloat16, true, true>(a, g, sg, grid, ngroups, status, st)

@@ -118,6 +118,25 @@ def test_both_row_kernel_variants(direct_rows, t, T, h, ffn, S, norm, dtype):
     _check_backward(ctx, caat.CAAT_ATTN_OUT, d, dtype)
 
 
+@pytest.mark.parametrize("with_dHn", [True, False])
+@pytest.mark.parametrize("t,T,h,S,norm,dtype", [
+    (4, 333, 4096, 2056, 0, "bf16"),   # two chunks per thread, the partition inside a warp: lanes of both classes
+    (4, 100, 4096, 1024, 1, "bf16"),   # LayerNorm; warps with one shared + one private chunk and with two private ones
+    (2, 50, 8192, 6144, 0, "bf16"),    # rows of 512 threads; warps with two shared chunks and with one of each
+    (4, 75, 2304, 1152, 1, "bf16"),    # 288 chunks on 2 x 160 threads: chunks past the row end
+    (4, 131, 1024, 512, 0, "f32"),     # fp32, two token rows per CTA, odd token count
+    (8, 131, 512, 256, 1, "f32"),      # fp32, one chunk per thread, LayerNorm
+    (4, 257, 2048, 0, 0, "bf16"),      # no shared channels
+    (4, 257, 2048, 2048, 1, "bf16")])  # no private channels
+def test_row_kernels_with_the_partition_on_a_chunk_boundary(t, T, h, S, norm, dtype, with_dHn):
+    # S a multiple of 8 and the per-rank layout: the staged family's lean kernels, whose loop body is compiled once
+    # per warp-uniform pattern of shared / private chunks plus a general one
+    ctx = G.make_ctx(t, h, h, dtype, S=S, norm=norm, direct_rows=2)
+    d = _layer_case(t, T, h, ctx.k_r(caat.CAAT_ATTN_OUT), dtype, S, seed=T + S, backward=True, tied=with_dHn)
+    _check_forward(ctx, caat.CAAT_ATTN_OUT, d, dtype)
+    _check_backward(ctx, caat.CAAT_ATTN_OUT, d, dtype, with_dHn=with_dHn)
+
+
 # ------------------------------------------------------------------ partition: bit-exact
 @pytest.mark.parametrize("S", [0, 1, 7, 8, 9, 127, 128, 129, 255, 256, 257, 504, 511, 512])
 def test_partition_bit_exact_integer_inputs(S):
