@@ -125,10 +125,8 @@ inline int ctas_per_sm(const RowGeom& g) {
 
 }  // namespace rows
 
-// lean variant of the staged kernels (per-rank layout, partition on a chunk boundary); same ring and grid
+// lean variant of the staged backward kernel (per-rank layout, partition on a chunk boundary); same ring and grid
 bool rows_lean_usable(int compact, int h, int T, int S, int S_lo, int S_hi, caat_dtype dtype);
-cudaError_t launch_rows_forward_lean(const RowFwdArgs& a, caat_dtype dtype, const rows::RowGeom& g, const rows::StageGeom& sg,
-                                     int grid, int ngroups, unsigned int* status, cudaStream_t st);
 cudaError_t launch_rows_backward_lean(const RowBwdArgs& a, caat_dtype dtype, const rows::RowGeom& g, const rows::StageGeom& sg,
                                       int grid, int ngroups, unsigned int* status, cudaStream_t st);
 

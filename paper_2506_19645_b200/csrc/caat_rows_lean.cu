@@ -1,18 +1,26 @@
-// Row kernels, lean variant of the bulk-copy staged kernels: per-rank residual layout, partition on a chunk boundary.
+// Backward row kernel, lean variant of the bulk-copy staged kernel: per-rank residual layout, partition on a chunk
+// boundary.
 //
 // Inside a long training step the GPU runs at its power cap (SM clocks near two thirds of the maximum) and every
-// instruction the row kernels do not execute is energy the step gets back.  These kernels do the staged kernels' work
-// with fewer instructions per 16-byte chunk:
+// instruction the row kernels do not execute is energy the step gets back.  This kernel does the staged backward
+// kernel's work with a quarter fewer instructions per 16-byte chunk (about 300 instead of 400 per rank for a thread's
+// two chunks at h = 4096), most of them saved by needing fewer registers than the 128 a thread may have:
 //   * the loop body exists once per WARP-UNIFORM pattern of chunk classes (NSH = how many of the thread's chunks are
 //     shared channels, the rest private; -1 = classes differ between lanes or a chunk lies past the row end), so the
-//     common patterns carry no class branches;
+//     common patterns carry no class branches and no rank sum for private chunks;
+//   * whether the stream's own gradient is given is a template parameter;
 //   * only the three warps that issue bulk copies keep the producer's counters;
-//   * outputs are addressed as a per-rank base pointer plus one 32-bit offset per chunk;
+//   * outputs are addressed as a per-rank base pointer plus one 32-bit offset per chunk, stored by predicated
+//     instructions instead of branches;
+//   * the next token group's row statistics go from global to shared memory by asynchronous copies, not through
+//     registers;
 //   * the row reduction's barrier also carries the "a wait ran out" vote (barrier with OR reduction), and its second
 //     stage reads the warps' partial sums as vectors.
 // Warps of one CTA may run different instances of the body; they meet at the same CTA barrier (barrier 0) the same
 // number of times, and every instance is entered by whole warps.
-// Shared-memory ring, stage layout, bounded waits and the status word are those of the staged kernels.
+// Shared-memory ring, stage layout, bounded waits and the status word are those of the staged kernels.  (The same
+// treatment of the forward kernel saves a fifth of its instructions and 3 % of its time when it runs alone, but
+// nothing inside a training step, so the forward stays on the staged kernel.)
 #include "caat_rows_bulk.cuh"
 
 namespace caat {
@@ -59,6 +67,20 @@ __device__ __forceinline__ int row_sum(float (&v)[NV], float* red, int& par, int
   return bad;
 }
 
+__device__ __forceinline__ void cp_async4(float* dst_shared, const float* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst_shared)), "l"(src) : "memory");
+}
+
+// 16-byte global store under a predicate held as an integer (nonzero = store): a predicated instruction, no branch
+template <typename raw>
+__device__ __forceinline__ void stg_if(uint32_t on, char* p, const raw& v) {
+  static_assert(sizeof(raw) == 16, "one 16-byte chunk");
+  const uint4 u = *reinterpret_cast<const uint4*>(&v);
+  asm volatile("{\n .reg .pred p;\n setp.ne.u32 p, %5, 0;\n @p st.global.v4.b32 [%0], {%1, %2, %3, %4};\n}"
+               ::"l"(p), "r"(u.x), "r"(u.y), "r"(u.z), "r"(u.w), "r"(on)
+               : "memory");
+}
+
 // chunk pattern of this warp: the number of shared chunks when every lane has the same classes and all chunks lie
 // inside the row, else -1
 template <int CPT>
@@ -70,208 +92,10 @@ __device__ __forceinline__ int warp_pattern(const int (&cls)[CPT]) {
   return __all_sync(0xffffffffu, code == first) ? first : -1;
 }
 
-// ------------------------------------------------------------------ forward
-// stage buffers: a = R rows [TY, h], b = zp rows [TY, P], c = zs rows [TY, S] (fetched with rank 0 only)
-template <typename T_, int CPT, bool LN, int MAXT>
-__global__ void __launch_bounds__(MAXT, MinBlocks<CPT, MAXT>::value)
-rows_forward_lean(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
-  using V_ = VT<T_>;
-  using raw = typename V_::raw;
-  constexpr int V = V_::N;
-  constexpr int ES = sizeof(T_);
-  constexpr int H2 = V / 2;
-  extern __shared__ __align__(128) uint8_t smem[];
-  const uint32_t ring32 = smem_u32(smem + sg.ring_off);
-  const uint32_t bar0 = smem_u32(smem + sg.bar_off);
-  float* red = reinterpret_cast<float*>(smem + sg.red_off);
-  const int TX = blockDim.x, TY = blockDim.y;
-  const int tid = threadIdx.y * TX + threadIdx.x;
-  const int lane = tid & 31;
-  const int wid = __shfl_sync(0xffffffffu, tid >> 5, 0);             // warp of the CTA, warp-uniform
-  const int wx = __shfl_sync(0xffffffffu, (int)threadIdx.x >> 5, 0);  // warp of the token row
-  const int warps_x = TX >> 5;
-  const int NS = sg.nstages;
-  const int t = a.t;
-  const float inv_h = 1.0f / (float)a.h;
-
-  const int my_groups = blockIdx.x < ngroups ? (ngroups - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-  const long long total = (long long)my_groups * t;
-
-  // producer: the next (token group, rank) to fetch, kept by the issuing warps (0: R, 1: zp, 2: zs); the stage it
-  // goes to is the one the consumers have just finished with
-  int pn = 0, pm = 0;
-  auto fetch = [&](uint32_t stage, uint32_t bar) {
-    if (pn >= my_groups) return;
-    const int n = pn, m = pm;
-    if (++pm == t) { pm = 0; ++pn; }
-    const long long i0 = (blockIdx.x + (long long)n * gridDim.x) * TY;
-    const int rowsN = (int)((a.T - i0) < TY ? (a.T - i0) : TY);
-    const uint32_t bR = (uint32_t)rowsN * a.h * ES;
-    const uint32_t bP = (uint32_t)rowsN * a.P * ES;                       // 0 without private channels (P = h - S)
-    const uint32_t bS = m == 0 ? (uint32_t)rowsN * a.S * ES : 0u;         // 0 without shared channels
-    const long long row = (long long)m * a.T + i0;
-    if (!elect_one()) return;
-    if (wid == 0) {
-      mbar_expect_tx(bar, bR + bP + bS);
-      bulk_g2s(stage + sg.off_a, static_cast<const char*>(a.R) + row * a.h * ES, bR, bar);
-    } else if (wid == 1) {
-      if (bP) bulk_g2s(stage + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
-    } else {
-      if (bS) bulk_g2s(stage + sg.off_c, static_cast<const char*>(a.zs) + i0 * a.S * ES, bS, bar);
-    }
-  };
-
-  if (tid == 0) {
-    for (int s = 0; s < NS; ++s) mbar_init(bar0 + 8u * s, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (tid < NS)   // the zero slot of every stage (no copy ever lands there)
-    *reinterpret_cast<uint4*>(smem + sg.ring_off + (size_t)tid * sg.stage_bytes + sg.zero_off) = make_uint4(0u, 0u, 0u, 0u);
-  __syncthreads();
-  pdl_wait();   // from here on global memory is touched
-  if (wid < 3)
-    for (int q = 0; q < NS; ++q) fetch(ring32 + (uint32_t)q * sg.stage_bytes, bar0 + 8u * q);
-
-  // per-thread constants: class of each chunk (0 shared, 1 private, 3 past the row end) and its byte offsets
-  // inside a stage; chunks past the row end read the zero slot
-  int col[CPT], cls[CPT];
-  uint32_t oA[CPT], oB[CPT];
-  float2 gam[CPT][H2], bet[LN ? CPT : 1][H2];
-#pragma unroll
-  for (int j = 0; j < CPT; ++j) {
-    col[j] = (threadIdx.x + j * TX) * V;
-    cls[j] = col[j] >= a.h ? 3 : (col[j] < a.S ? 0 : 1);
-#pragma unroll
-    for (int q = 0; q < H2; ++q) { gam[j][q] = f2(0.f); if constexpr (LN) bet[j][q] = f2(0.f); }
-    oA[j] = oB[j] = sg.zero_off;
-    if (cls[j] != 3) {
-      unpack2(ldg<raw>(static_cast<const char*>(a.gamma) + (long long)col[j] * ES), gam[j]);
-      if constexpr (LN) {
-        if (a.beta) unpack2(ldg<raw>(static_cast<const char*>(a.beta) + (long long)col[j] * ES), bet[j]);
-      }
-      oA[j] = sg.off_a + ((uint32_t)threadIdx.y * a.h + col[j]) * ES;
-      oB[j] = cls[j] == 0 ? sg.off_c + ((uint32_t)threadIdx.y * a.S + col[j]) * ES          // its zs chunk
-                          : sg.off_b + ((uint32_t)threadIdx.y * a.P + (uint32_t)(col[j] - a.S)) * ES;   // its zp chunk
-    }
-  }
-  const float2 alpha2 = f2(a.alpha);
-  const long long rank_h = (long long)a.T * a.h * ES;
-  const int pattern = warp_pattern<CPT>(cls);
-
-  long long k = 0;
-  bool dead = false;
-  auto body = [&](auto tag) {
-    constexpr int NSH = decltype(tag)::value;
-    auto shared_chunk = [&](int j) { if constexpr (NSH >= 0) return j < NSH; else return cls[j] == 0; };
-    uint32_t sb = ring32;   // consumer's stage (shared address), its index and phase parity
-    int cs = 0, par = 0;
-    uint32_t cph = 0;
-    for (int n = 0; n < my_groups; ++n) {
-      const long long i = (blockIdx.x + (long long)n * gridDim.x) * TY + threadIdx.y;
-      const bool valid = i < a.T;
-      bool act[CPT];
-      uint32_t off[CPT];      // of the chunk inside one rank's [T, h] plane
-      float2 zs[CPT][H2];     // shared part of the layer output, read once per token
-#pragma unroll
-      for (int j = 0; j < CPT; ++j) {
-        act[j] = valid && (NSH >= 0 || cls[j] != 3);
-        off[j] = (uint32_t)((i * a.h + col[j]) * ES);
-#pragma unroll
-        for (int q = 0; q < H2; ++q) zs[j][q] = f2(0.f);
-      }
-      char* hn_m = static_cast<char*>(a.Hn);
-      char* x_m = static_cast<char*>(a.X);
-      float* rstd_m = a.rstd + i;
-      float* mean_m = (LN && a.mean) ? a.mean + i : nullptr;
-
-      for (int m = 0; m < t; ++m, ++k) {
-        const int failed = mbar_wait(bar0 + 8u * cs, cph) ? 0 : 1;
-        float2 hn[CPT][H2];
-        float2 acc = f2(0.f);
-#pragma unroll
-        for (int j = 0; j < CPT; ++j) {
-          float2 r[H2];
-          unpack2(lds32<raw>(sb + oA[j]), r);
-          if (shared_chunk(j)) {
-            if (m == 0) unpack2(lds32<raw>(sb + oB[j]), zs[j]);
-#pragma unroll
-            for (int q = 0; q < H2; ++q) hn[j][q] = add2(zs[j][q], r[q]);
-          } else {
-            float2 zp[H2];
-            unpack2(lds32<raw>(sb + oB[j]), zp);
-#pragma unroll
-            for (int q = 0; q < H2; ++q) hn[j][q] = fma2(alpha2, zp[q], r[q]);
-          }
-          if (act[j]) stg<raw>(hn_m + off[j], pack2(hn[j]));
-#pragma unroll
-          for (int q = 0; q < H2; ++q) acc = LN ? add2(acc, hn[j][q]) : fma2(hn[j][q], hn[j][q], acc);
-        }
-        float st[1] = {acc.x + acc.y};
-        if (row_sum<1>(st, red, par, warps_x, wx, lane, failed)) { dead = true; return; }   // barrier: stage fully read
-        if (wid < 3) fetch(sb, bar0 + 8u * cs);
-        sb += sg.stage_bytes;
-        if (++cs == NS) { cs = 0; cph ^= 1u; sb = ring32; }
-        float mu = 0.f, rs;
-        if (LN) {
-          mu = st[0] * inv_h;
-          float2 sq2 = f2(0.f);
-#pragma unroll
-          for (int j = 0; j < CPT; ++j) {
-            if (NSH < 0 && cls[j] == 3) continue;
-#pragma unroll
-            for (int q = 0; q < H2; ++q) {
-              const float2 d = add2(hn[j][q], f2(-mu));
-              sq2 = fma2(d, d, sq2);
-            }
-          }
-          float sq[1] = {sq2.x + sq2.y};
-          row_sum<1>(sq, red, par, warps_x, wx, lane, 0);
-          rs = rsqrtf(fmaf(sq[0], inv_h, a.eps));
-        } else {
-          rs = rsqrtf(fmaf(st[0], inv_h, a.eps));
-        }
-        const float2 rs2 = f2(rs);
-#pragma unroll
-        for (int j = 0; j < CPT; ++j) {
-          float2 x[H2];
-#pragma unroll
-          for (int q = 0; q < H2; ++q) {
-            const float2 sc = mul2(rs2, gam[j][q]);
-            if constexpr (LN) x[q] = fma2(add2(hn[j][q], f2(-mu)), sc, bet[j][q]);
-            else x[q] = mul2(hn[j][q], sc);
-          }
-          if (act[j]) stg<raw>(x_m + off[j], pack2(x));
-        }
-        if (valid && threadIdx.x == 0) {
-          *rstd_m = rs;
-          if (LN && mean_m) *mean_m = mu;
-        }
-        hn_m += rank_h;
-        x_m += rank_h;
-        rstd_m += a.T;
-        if (LN && mean_m) mean_m += a.T;
-      }
-    }
-  };
-  if (pattern == 0) body(Int<0>{});
-  else if (pattern == CPT) body(Int<CPT>{});
-  else if (CPT == 2 && pattern == 1) body(Int<(CPT == 2 ? 1 : 0)>{});
-  else body(Int<-1>{});
-
-  if (dead && tid == 0) {
-    atomicExch(status, 4u);
-    // wait (bounded) for this CTA's copies still in flight before its shared memory goes away
-    const long long issued = (k + NS) < total ? (k + NS) : total;
-    for (long long q = k + 1; q < issued; ++q)
-      for (uint32_t it = 0; it < (1u << 10); ++it)   // each poll sleeps up to the suspend hint: ~20 ms per stage at most
-        if (mbar_try(bar0 + 8u * (uint32_t)(q % NS), (uint32_t)((q / NS) & 1))) break;
-  }
-}
-
 // ------------------------------------------------------------------ backward
 // stage buffers: a = dX rows, b = Hn rows, c = dHn rows (when given), each [TY, h]
-template <typename T_, int CPT, bool LN, int MAXT>
+// DH: the gradient arriving at the stored stream (dHn) is given
+template <typename T_, int CPT, bool LN, int MAXT, bool DH>
 __global__ void __launch_bounds__(MAXT, MinBlocks<CPT, MAXT>::value)
 rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned int* status) {
   using V_ = VT<T_>;
@@ -293,13 +117,14 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
   const int NS = sg.nstages;
   const int t = a.t;
   const float inv_h = 1.0f / (float)a.h;
-  const bool has_dh = a.dHn != nullptr;
+  constexpr bool has_dh = DH;
   const int nstat = t * TY;
 
   const int my_groups = blockIdx.x < ngroups ? (ngroups - blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
   const long long total = (long long)my_groups * t;
 
-  // producer (issuing warps 0: dX, 1: Hn, 2: dHn), see the forward kernel
+  // producer: the next (token group, rank) to fetch, kept by the issuing warps (0: dX, 1: Hn, 2: dHn); the stage it
+  // goes to is the one the consumers have just finished with
   int pn = 0, pm = 0;
   auto fetch = [&](uint32_t stage, uint32_t bar) {
     if (pn >= my_groups) return;
@@ -353,7 +178,6 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
   const uint32_t off_hc = sg.off_c - sg.off_b;   // from a chunk of the stream to the same chunk of its gradient
   const float2 alpha2 = f2(a.alpha);
   const long long rank_h = (long long)a.T * a.h * ES;
-  const long long rank_p = (long long)a.T * a.P * ES;
   const int pattern = warp_pattern<CPT>(cls);
   __syncthreads();   // stats of group 0 visible
 
@@ -366,31 +190,29 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
     int cs = 0, par = 0;
     uint32_t cph = 0;
     for (int n = 0; n < my_groups; ++n) {
-      const long long i = (blockIdx.x + (long long)n * gridDim.x) * TY + threadIdx.y;
+      const int i = (blockIdx.x + n * gridDim.x) * TY + threadIdx.y;   // < T + TY
       const bool valid = i < a.T;
       const float* st_cur = stat + (size_t)(n & 1) * 2 * nstat + threadIdx.y;
       float* st_nxt = stat + (size_t)((n + 1) & 1) * 2 * nstat;
-      // prefetch the next group's row statistics into registers; they are parked in shared memory at the end of
-      // this group (a whole group of work hides the latency)
-      float pre_r[2] = {0.f, 0.f}, pre_m[2] = {0.f, 0.f};
-      {
-        const long long g2 = blockIdx.x + (long long)(n + 1) * gridDim.x;
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int q = tid + u * nthr;
-          if (q < nstat && n + 1 < my_groups) {
-            const int m2 = q / TY, ty2 = q % TY;
-            const long long i2 = g2 * TY + ty2;
-            if (i2 < a.T) {
-              pre_r[u] = a.rstd[(long long)m2 * a.T + i2];
-              if (LN) pre_m[u] = a.mean[(long long)m2 * a.T + i2];
-            }
+      // the next group's row statistics go straight from global to shared memory (4-byte asynchronous copies into the
+      // buffer nobody reads during this group); they are awaited before the barrier that ends the group
+      if (n + 1 < my_groups) {
+        const int g2 = blockIdx.x + (n + 1) * gridDim.x;
+        for (int q = tid; q < nstat; q += nthr) {
+          const int m2 = q / TY, ty2 = q % TY;
+          const int i2 = g2 * TY + ty2;
+          if (i2 < a.T) {
+            cp_async4(st_nxt + q, a.rstd + (long long)m2 * a.T + i2);
+            if (LN) cp_async4(st_nxt + nstat + q, a.mean + (long long)m2 * a.T + i2);
+          } else {
+            st_nxt[q] = 0.f;
+            if (LN) st_nxt[nstat + q] = 0.f;
           }
         }
       }
       bool act[CPT];
       uint32_t aX[CPT], aH[CPT];   // stage-relative addresses of the dX and stream chunks; the zero slot when inactive
-      uint32_t off[CPT], offz[CPT];   // of the chunk inside one rank's [T, h] plane of dR, [T, P] plane of zp
+      uint32_t off[CPT];   // of the chunk inside one rank's [T, h] plane of dR
       float2 gsum[CPT][H2];
 #pragma unroll
       for (int j = 0; j < CPT; ++j) {
@@ -398,16 +220,14 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
         const uint32_t oX = ((uint32_t)threadIdx.y * a.h + col[j]) * ES;
         aX[j] = act[j] ? sg.off_a + oX : sg.zero_off;
         aH[j] = act[j] ? sg.off_b + oX : sg.zero_off;
-        off[j] = (uint32_t)((i * a.h + col[j]) * ES);
-        offz[j] = (uint32_t)((i * a.P + (col[j] - a.S)) * ES);
+        off[j] = (uint32_t)(((long long)i * a.h + col[j]) * ES);
 #pragma unroll
         for (int q = 0; q < H2; ++q) gsum[j][q] = f2(0.f);
       }
       const uint32_t hc = valid ? off_hc : 0u;
       char* dr_m = static_cast<char*>(a.dR);
-      char* zp_m = static_cast<char*>(a.zp);
 
-      for (int m = 0; m < t; ++m, ++k) {
+      for (int m = 0; m < t; ++m) {
         const int failed = mbar_wait(bar0 + 8u * cs, cph) ? 0 : 1;
         const float rs_c = st_cur[m * TY];
         const float mu_c = LN ? st_cur[nstat + m * TY] : 0.f;
@@ -421,8 +241,7 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
           float2 dx[H2], hn[H2];
           unpack2(lds32<raw>(sb + aX[j]), dx);
           unpack2(lds32<raw>(sb + aH[j]), hn);
-          const uint32_t hcj = (NSH >= 0 || cls[j] != 3) ? hc : 0u;
-          rdh[j] = has_dh ? lds32<raw>(sb + aH[j] + hcj) : zero_raw<raw>();
+          if constexpr (DH) rdh[j] = lds32<raw>(sb + aH[j] + ((NSH >= 0 || cls[j] != 3) ? hc : 0u));
 #pragma unroll
           for (int q = 0; q < H2; ++q) {
             xh[j][q] = LN ? mul2(add2(hn[q], f2(-mu_c)), rs2) : mul2(hn[q], rs2);
@@ -436,7 +255,11 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
         float sacc[LN ? 2 : 1];
         if (LN) { sacc[0] = s1.x + s1.y; sacc[LN ? 1 : 0] = s2.x + s2.y; }
         else sacc[0] = s2.x + s2.y;
-        if (row_sum<LN ? 2 : 1>(sacc, red, par, warps_x, wx, lane, failed)) { dead = true; return; }   // barrier: stage fully read
+        if (row_sum<LN ? 2 : 1>(sacc, red, par, warps_x, wx, lane, failed)) {   // barrier: stage fully read
+          k = (long long)n * t + m;
+          dead = true;
+          return;
+        }
         if (wid < 3) fetch(sb, bar0 + 8u * cs);
         sb += sg.stage_bytes;
         if (++cs == NS) { cs = 0; cph ^= 1u; sb = ring32; }
@@ -446,43 +269,31 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
 #pragma unroll
         for (int j = 0; j < CPT; ++j) {
           float2 gg[H2], dh[H2];
-          unpack2(rdh[j], dh);
+          if constexpr (DH) unpack2(rdh[j], dh);
 #pragma unroll
           for (int q = 0; q < H2; ++q) {
             float2 tt = fma2(xh[j][q], nc2, dxh[j][q]);
             if (LN) tt = add2(tt, nc1);
-            gg[q] = fma2(rs2, tt, dh[q]);
+            gg[q] = DH ? fma2(rs2, tt, dh[q]) : mul2(rs2, tt);
           }
-          if (act[j]) stg<raw>(dr_m + off[j], pack2(gg));
+          stg_if<raw>(act[j] ? 1u : 0u, dr_m + off[j], pack2(gg));
           if (shared_chunk(j)) {
 #pragma unroll
             for (int q = 0; q < H2; ++q) gsum[j][q] = add2(gsum[j][q], gg[q]);   // fp32 rank sum, m ascending
-          } else if (zp_m) {
+          } else if (a.zp) {   // the scaled private copy, for a GEMM that does not read dR in place
             float2 zp[H2];
 #pragma unroll
             for (int q = 0; q < H2; ++q) zp[q] = mul2(alpha2, gg[q]);           // private gradient carries alpha
-            if (act[j]) stg<raw>(zp_m + offz[j], pack2(zp));
+            if (act[j])
+              stg<raw>(static_cast<char*>(a.zp) + (((long long)m * a.T + i) * a.P + (col[j] - a.S)) * ES, pack2(zp));
           }
         }
         dr_m += rank_h;
-        if (zp_m) zp_m += rank_p;
       }
 #pragma unroll
       for (int j = 0; j < CPT; ++j)
-        if (act[j] && shared_chunk(j)) stg<raw>(gs_row(a, i, ES) + (long long)col[j] * ES, pack2(gsum[j]));
-      // park the next group's statistics; the last barrier of this group separates these writes from the reads of
-      // group n-1's buffer, the barrier below from the reads of group n+1
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int q = tid + u * nthr;
-        if (q < nstat) { st_nxt[q] = pre_r[u]; if (LN) st_nxt[nstat + q] = pre_m[u]; }
-      }
-      for (int q = tid + 2 * nthr; q < nstat && n + 1 < my_groups; q += nthr) {   // t * TY > 2 * threads: rare
-        const int m2 = q / TY, ty2 = q % TY;
-        const long long i2 = (blockIdx.x + (long long)(n + 1) * gridDim.x) * TY + ty2;
-        st_nxt[q] = i2 < a.T ? a.rstd[(long long)m2 * a.T + i2] : 0.f;
-        if (LN) st_nxt[nstat + q] = i2 < a.T ? a.mean[(long long)m2 * a.T + i2] : 0.f;
-      }
+        if (act[j] && shared_chunk(j)) stg<raw>(gs_row(a, (long long)i, ES) + (long long)col[j] * ES, pack2(gsum[j]));
+      asm volatile("cp.async.wait_all;" ::: "memory");   // this thread's copies of the next group's statistics have landed
       __syncthreads();
     }
   };
@@ -552,28 +363,6 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
 
 // ------------------------------------------------------------------ host side
 template <typename T_, bool LN>
-cudaError_t launch_fwd_lean_t(const RowFwdArgs& a, const RowGeom& g, const StageGeom& sg, int grid, int ngroups,
-                              unsigned int* status, cudaStream_t st) {
-  const dim3 block(g.TX, g.TY);
-  cudaError_t e = cudaSuccess;
-  LaunchScope scope(CAAT_K_ROWS_FORWARD, st);
-  const int threads = g.TX * g.TY;
-#define CAAT_LAUNCH(CPT_, MAXT_)                                                                                        \
-  do {                                                                                                                  \
-    e = set_smem(rows_forward_lean<T_, CPT_, LN, MAXT_>, sg.smem);                                                      \
-    if (e == cudaSuccess)                                                                                               \
-      e = launch_pdl(rows_forward_lean<T_, CPT_, LN, MAXT_>, dim3(grid), block, sg.smem, st, a, sg, ngroups, status);   \
-  } while (0)
-  if (g.CPT == 1 && threads <= 256) CAAT_LAUNCH(1, 256);
-  else if (g.CPT == 1) CAAT_LAUNCH(1, 512);
-  else if (g.CPT == 2 && threads <= 256) CAAT_LAUNCH(2, 256);
-  else if (g.CPT == 2) CAAT_LAUNCH(2, 512);
-  else return cudaErrorInvalidValue;
-#undef CAAT_LAUNCH
-  return e != cudaSuccess ? e : cudaGetLastError();
-}
-
-template <typename T_, bool LN>
 cudaError_t launch_bwd_lean_t(const RowBwdArgs& a, const RowGeom& g, const StageGeom& sg, int grid, int ngroups,
                               unsigned int* status, cudaStream_t st) {
   const dim3 block(g.TX, g.TY);
@@ -582,9 +371,17 @@ cudaError_t launch_bwd_lean_t(const RowBwdArgs& a, const RowGeom& g, const Stage
   const int threads = g.TX * g.TY;
 #define CAAT_LAUNCH(CPT_, MAXT_)                                                                                        \
   do {                                                                                                                  \
-    e = set_smem(rows_backward_lean<T_, CPT_, LN, MAXT_>, sg.smem);                                                     \
-    if (e == cudaSuccess)                                                                                               \
-      e = launch_pdl(rows_backward_lean<T_, CPT_, LN, MAXT_>, dim3(grid), block, sg.smem, st, a, sg, ngroups, status);  \
+    if (a.dHn) {                                                                                                        \
+      e = set_smem(rows_backward_lean<T_, CPT_, LN, MAXT_, true>, sg.smem);                                             \
+      if (e == cudaSuccess)                                                                                             \
+        e = launch_pdl(rows_backward_lean<T_, CPT_, LN, MAXT_, true>, dim3(grid), block, sg.smem, st, a, sg, ngroups,   \
+                       status);                                                                                         \
+    } else {                                                                                                            \
+      e = set_smem(rows_backward_lean<T_, CPT_, LN, MAXT_, false>, sg.smem);                                            \
+      if (e == cudaSuccess)                                                                                             \
+        e = launch_pdl(rows_backward_lean<T_, CPT_, LN, MAXT_, false>, dim3(grid), block, sg.smem, st, a, sg, ngroups,  \
+                       status);                                                                                         \
+    }                                                                                                                   \
   } while (0)
   if (g.CPT == 1 && threads <= 256) CAAT_LAUNCH(1, 256);
   else if (g.CPT == 1) CAAT_LAUNCH(1, 512);
@@ -604,15 +401,6 @@ bool rows_lean_usable(int compact, int h, int T, int S, int S_lo, int S_hi, caat
   const RowGeom g = row_geometry(h, dtype);
   return !compact && S_lo == S && S_hi == S && (long long)T * h * (long long)elem_size(dtype) < (1LL << 32) &&
          g.CPT <= 2 && g.TX * g.TY >= 96;
-}
-
-cudaError_t launch_rows_forward_lean(const RowFwdArgs& a, caat_dtype dtype, const RowGeom& g, const StageGeom& sg, int grid,
-                                     int ngroups, unsigned int* status, cudaStream_t st) {
-  if (dtype == CAAT_BF16)
-    return a.norm == 1 ? launch_fwd_lean_t<__nv_bfloat16, true>(a, g, sg, grid, ngroups, status, st)
-                       : launch_fwd_lean_t<__nv_bfloat16, false>(a, g, sg, grid, ngroups, status, st);
-  return a.norm == 1 ? launch_fwd_lean_t<float, true>(a, g, sg, grid, ngroups, status, st)
-                     : launch_fwd_lean_t<float, false>(a, g, sg, grid, ngroups, status, st);
 }
 
 cudaError_t launch_rows_backward_lean(const RowBwdArgs& a, caat_dtype dtype, const RowGeom& g, const StageGeom& sg, int grid,

@@ -646,14 +646,13 @@ cudaError_t launch_bwd_staged_t(const RowBwdArgs& a, const RowGeom& g, const Sta
 
 }  // namespace
 
-// the lean kernels take over wherever they apply (a measurement build can keep the general kernels:
-// CAAT_ROWS_LEAN bit 0 = forward, bit 1 = backward)
-static bool rows_lean_enabled(int dir) {
+// the lean backward kernel takes over wherever it applies (a measurement build can keep the general kernel:
+// CAAT_ROWS_LEAN=0)
+static bool rows_lean_enabled() {
 #ifdef CAAT_MEASUREMENT_AIDS
-  static const int on = [] { const char* e = getenv("CAAT_ROWS_LEAN"); return e ? atoi(e) : 3; }();
-  return (on >> dir) & 1;
+  static const bool on = [] { const char* e = getenv("CAAT_ROWS_LEAN"); return !(e && atoi(e) == 0); }();
+  return on;
 #else
-  (void)dir;
   return true;
 #endif
 }
@@ -684,8 +683,6 @@ cudaError_t launch_rows_forward_staged(const RowFwdArgs& a, caat_dtype dtype, cu
   if (grid > ngroups) grid = ngroups;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
-  if (rows_lean_enabled(0) && rows_lean_usable(a.compact, a.h, a.T, a.S, a.S_lo, a.S_hi, dtype))
-    return launch_rows_forward_lean(a, dtype, g, sg, grid, ngroups, status, st);
   if (cl) {
     if (dtype == CAAT_BF16)
       return a.norm == 1 ? launch_fwd_staged_t<__nv_bfloat16, true, true>(a, g, sg, grid, ngroups, status, st)
@@ -724,7 +721,7 @@ cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, i
   *rows_used = grid;
   unsigned int* status = device_status_word();
   if (!status) return cudaErrorUnknown;
-  if (rows_lean_enabled(1) && rows_lean_usable(a.compact, a.h, a.T, a.S, a.S_lo, a.S_hi, dtype))
+  if (rows_lean_enabled() && rows_lean_usable(a.compact, a.h, a.T, a.S, a.S_lo, a.S_hi, dtype))
     return launch_rows_backward_lean(a, dtype, g, sg, grid, ngroups, status, st);
   if (cl) {
     if (dtype == CAAT_BF16)

@@ -129,8 +129,9 @@ def test_both_row_kernel_variants(direct_rows, t, T, h, ffn, S, norm, dtype):
     (4, 257, 2048, 0, 0, "bf16"),      # no shared channels
     (4, 257, 2048, 2048, 1, "bf16")])  # no private channels
 def test_row_kernels_with_the_partition_on_a_chunk_boundary(t, T, h, S, norm, dtype, with_dHn):
-    # S a multiple of 8 and the per-rank layout: the staged family's lean kernels, whose loop body is compiled once
-    # per warp-uniform pattern of shared / private chunks plus a general one
+    # S a multiple of 8 and the per-rank layout: the backward runs the staged family's lean kernel, whose loop body is
+    # compiled once per warp-uniform pattern of shared / private chunks plus a general one (the forward runs the
+    # staged kernel on the same shapes)
     ctx = G.make_ctx(t, h, h, dtype, S=S, norm=norm, direct_rows=2)
     d = _layer_case(t, T, h, ctx.k_r(caat.CAAT_ATTN_OUT), dtype, S, seed=T + S, backward=True, tied=with_dHn)
     _check_forward(ctx, caat.CAAT_ATTN_OUT, d, dtype)
