@@ -190,6 +190,13 @@ cudaError_t launch_rows_backward_staged(const RowBwdArgs& a, caat_dtype dtype, i
 cudaError_t launch_rows_backward_warp(const RowBwdArgs& a, caat_dtype dtype, int max_rows, int* rows_used,
                                       cudaStream_t st);
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype);
+// Wait limit of the bulk-copy row kernels and the switch of their time-out test, read once per process from the
+// environment: CAAT_ROWS_SPINCAP (polls of one mbarrier wait, default 2^18; each poll may sleep up to 20 us in
+// hardware) and CAAT_ROWS_STALL=1 (every stage announces 16 bytes that never arrive, so the first wait runs out:
+// the kernels must raise the status word, let their copies land and return).  Neither changes a result of a call
+// that returns CAAT_OK.
+struct RowsHooks { uint32_t spin_cap; int stall; };
+RowsHooks rows_hooks();
 
 // ---- activation of the column-parallel half (streaming kernels) ---------------
 // gated: pre has 2 * width_out columns [gate | up], Y = silu(gate) * up; else Y = silu(pre)

@@ -822,6 +822,16 @@ cudaError_t launch_rows_forward_partials(const RowPartArgs& a, caat_dtype dtype,
   return a.norm == 1 ? go(rows_forward_partials_kernel<float, true>) : go(rows_forward_partials_kernel<float, false>);
 }
 
+RowsHooks rows_hooks() {
+  static const RowsHooks hooks = [] {
+    RowsHooks k{1u << 18, 0};
+    if (const char* e = getenv("CAAT_ROWS_SPINCAP")) { const int v = atoi(e); if (v >= 16) k.spin_cap = (uint32_t)v; }
+    if (const char* e = getenv("CAAT_ROWS_STALL")) k.stall = atoi(e) == 1 ? 1 : 0;
+    return k;
+  }();
+  return hooks;
+}
+
 int rows_backward_partial_rows(int h, int T, caat_dtype dtype) {
   const RowGeom g = row_geometry(h, dtype);
   const int ngroups = (T + g.TY - 1) / g.TY;

@@ -7,7 +7,6 @@
 namespace caat {
 namespace rows {
 
-constexpr uint32_t kSpinCap = 1u << 18;
 constexpr uint32_t kSuspendHintNs = 20000u;   // the waiting warp sleeps in hardware instead of spinning
 constexpr int kMaxStages = 8;
 
@@ -33,8 +32,8 @@ __device__ __forceinline__ bool elect_one() {
   asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.u32 %0, 1, 0, P;\n}" : "=r"(pred));
   return pred != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kSpinCap; ++it)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t cap) {
+  for (uint32_t it = 0; it < cap; ++it)
     if (mbar_try(bar, parity)) return true;
   return false;
 }
@@ -56,6 +55,8 @@ struct StageGeom {
   uint32_t zero_off;             // 16 zero bytes inside every stage (read by chunks past the row end)
   uint32_t keep_off;             // compact backward: [TY, S] shared rows of the stream, kept for all ranks of a token group
   size_t smem;
+  uint32_t spin_cap;             // polls of one mbarrier wait before the CTA gives up (rows_hooks)
+  uint32_t stall_bytes;          // time-out test: bytes every stage announces on top of its copies (0 otherwise)
 };
 
 // resident CTAs per SM the launch bounds ask for: one chunk per thread in small CTAs leaves ~85
@@ -103,6 +104,9 @@ inline StageGeom stage_geometry(const RowGeom& g, int h, int P, int S_hi, int t,
   size_t ring = (size_t)(ns > 0 ? ns : 0) * sg.stage_bytes;
   if (ring < acc) ring = acc;
   sg.smem = off + ring;
+  const RowsHooks hooks = rows_hooks();
+  sg.spin_cap = hooks.spin_cap;
+  sg.stall_bytes = hooks.stall ? 16u : 0u;
   return sg;
 }
 

@@ -136,7 +136,7 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
     const long long off = ((long long)m * a.T + i0) * a.h * ES;
     if (!elect_one()) return;
     if (wid == 0) {
-      mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
+      mbar_expect_tx(bar, (has_dh ? 3 * b : 2 * b) + sg.stall_bytes);
       bulk_g2s(stage + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
     } else if (wid == 1) {
       bulk_g2s(stage + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
@@ -224,17 +224,17 @@ rows_backward_lean(const RowBwdArgs a, const StageGeom sg, int ngroups, unsigned
 #pragma unroll
         for (int q = 0; q < H2; ++q) gsum[j][q] = f2(0.f);
       }
-      const uint32_t hc = valid ? off_hc : 0u;
+      [[maybe_unused]] const uint32_t hc = valid ? off_hc : 0u;
       char* dr_m = static_cast<char*>(a.dR);
 
       for (int m = 0; m < t; ++m) {
-        const int failed = mbar_wait(bar0 + 8u * cs, cph) ? 0 : 1;
+        const int failed = mbar_wait(bar0 + 8u * cs, cph, sg.spin_cap) ? 0 : 1;
         const float rs_c = st_cur[m * TY];
         const float mu_c = LN ? st_cur[nstat + m * TY] : 0.f;
         const float2 rs2 = f2(rs_c);
 
         float2 xh[CPT][H2], dxh[CPT][H2];
-        raw rdh[CPT];     // stream-gradient chunk, kept packed across the barrier (it is needed only after it)
+        [[maybe_unused]] raw rdh[CPT];   // stream-gradient chunk, kept packed across the barrier (needed only after it)
         float2 s1 = f2(0.f), s2 = f2(0.f);
 #pragma unroll
         for (int j = 0; j < CPT; ++j) {

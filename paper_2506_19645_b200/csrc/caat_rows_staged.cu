@@ -71,7 +71,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     const long long row = (long long)m * a.T + i0;
     if (!elect_one()) return;
     if (issuer == 0) {
-      mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS));
+      mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS) + sg.stall_bytes);
       if (bR) bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * (CL ? a.P : a.h) * ES, bR, bar);
     } else if (issuer == 1) {
       if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
@@ -155,7 +155,7 @@ rows_forward_staged(const RowFwdArgs a, const StageGeom sg, int ngroups, unsigne
     float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
 
     for (int m = 0; m < a.t; ++m, ++k) {
-      if (!mbar_wait(bar0 + 8u * cs, cph)) *abort_flag = 1;
+      if (!mbar_wait(bar0 + 8u * cs, cph, sg.spin_cap)) *abort_flag = 1;
 
       float2 hn[CPT][H2];
       float2 acc = f2(0.f);
@@ -309,7 +309,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
       const uint32_t bS = m == 0 ? (uint32_t)rowsN * a.S_hi * ES : 0u;      // 0 when there is no shared part
       const long long offp = ((long long)m * a.T + i0) * a.P * ES, offs = i0 * a.S_hi * ES;
       if (issuer == 0) {
-        mbar_expect_tx(bar, b + (has_dh ? 2 : 1) * (bP + bS));
+        mbar_expect_tx(bar, b + (has_dh ? 2 : 1) * (bP + bS) + sg.stall_bytes);
         bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
       } else if (issuer == 1) {
         if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + offp, bP, bar);
@@ -322,7 +322,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
       }
     } else {
       if (issuer == 0) {
-        mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
+        mbar_expect_tx(bar, (has_dh ? 3 * b : 2 * b) + sg.stall_bytes);
         bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
       } else if (issuer == 1) {
         bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
@@ -431,7 +431,7 @@ rows_backward_staged(const RowBwdArgs a, const StageGeom sg, int ngroups, unsign
     }
 
     for (int m = 0; m < a.t; ++m, ++k) {
-      if (!mbar_wait(bar0 + 8u * cs, cph)) *abort_flag = 1;
+      if (!mbar_wait(bar0 + 8u * cs, cph, sg.spin_cap)) *abort_flag = 1;
       const float rs_c = st_cur[m * TY + threadIdx.y];
       const float mu_c = LN ? st_cur[nstat + m * TY + threadIdx.y] : 0.f;
       const float2 rs2 = f2(rs_c);

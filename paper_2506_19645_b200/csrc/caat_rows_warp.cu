@@ -17,7 +17,6 @@ using namespace rows;
 constexpr int kW = 4;                    // consumer warps = tokens per group
 constexpr int kThreads = (kW + 1) * 32;  // + one producer warp
 constexpr int kMaxStages = 8;
-constexpr uint32_t kSpinCap = 1u << 18;
 constexpr uint32_t kSuspendHintNs = 20000u;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -39,8 +38,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinCap; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t cap) {
+  for (uint32_t it = 0; it < cap; ++it) {
     if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
   }
@@ -54,6 +53,23 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 template <typename raw>
 __device__ __forceinline__ raw lds(const uint8_t* p) { return *reinterpret_cast<const raw*>(p); }
 
+// A consumer warp whose wait for a stage ran out: it raises the abort flag and the status word (the producer may have
+// issued everything and left already, so nobody else would), then gives the copies that may still be in flight into
+// this CTA's ring a bounded time to land - stage by stage from the one it waited for - before it leaves the loop.
+__device__ __forceinline__ void consumer_gave_up(unsigned int* status, unsigned int code, volatile int* abort_flag,
+                                                 uint32_t full0, int s, uint32_t ph, int NS, int lane) {
+  if (lane == 0) {
+    *abort_flag = 1;
+    atomicExch(status, code);
+    for (int k = 0; k < NS; ++k) {
+      for (uint32_t it = 0; it < (1u << 10); ++it)   // each poll sleeps up to the suspend hint: ~20 ms per stage at most
+        if (mbar_try(full0 + 8u * s, ph)) break;
+      if (++s == NS) { s = 0; ph ^= 1u; }
+    }
+  }
+  __syncwarp();
+}
+
 struct WarpGeom {
   int nstages;
   uint32_t off_a, off_b, off_c, off_d, off_e, stage_bytes;   // d, e: compact layout only
@@ -61,6 +77,8 @@ struct WarpGeom {
   uint32_t keep_off;   // compact backward: [kW, S] shared rows of the stream, parked for all ranks of a token
   uint32_t bar_off, ring_off;
   size_t smem;
+  uint32_t spin_cap;     // polls of one mbarrier wait before the role gives up (rows_hooks)
+  uint32_t stall_bytes;  // time-out test: bytes every stage announces on top of its copies (0 otherwise)
 };
 
 // ------------------------------------------------------------------ forward
@@ -103,13 +121,13 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
         const long long i0 = (blockIdx.x + (long long)n * gridDim.x) * kW;
         const int rowsN = (int)((a.T - i0) < kW ? (a.T - i0) : kW);
         for (int m = 0; m < a.t; ++m) {
-          if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, abort_flag, sg.spin_cap)) { ok = false; break; }
           const uint32_t bar = full0 + 8u * s;
           const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
           const uint32_t bP = has_priv ? (uint32_t)rowsN * a.P * ES : 0u;
           const uint32_t bR = CL ? bP : (uint32_t)rowsN * a.h * ES;
           const uint32_t bS = (m == 0 && has_shared) ? (uint32_t)rowsN * a.S_hi * ES : 0u;
-          mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS));
+          mbar_expect_tx(bar, bR + bP + (CL ? 2 * bS : bS) + sg.stall_bytes);
           const long long row = (long long)m * a.T + i0;
           if (bR) bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.R) + row * (CL ? a.P : a.h) * ES, bR, bar);
           if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.zp) + row * a.P * ES, bP, bar);
@@ -181,7 +199,11 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
     float* rstd_p = a.rstd + i;
     float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
     for (int m = 0; m < a.t; ++m) {
-      if (!mbar_wait(full0 + 8u * s, ph, abort_flag)) { dead = true; break; }
+      if (!mbar_wait(full0 + 8u * s, ph, abort_flag, sg.spin_cap)) {
+        consumer_gave_up(status, 8u, abort_flag, full0, s, ph, NS, lane);
+        dead = true;
+        break;
+      }
       float2 hn[CPT][H2];
       float2 acc = f2(0.f);
 #pragma unroll
@@ -330,14 +352,14 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
         const int rowsN = (int)((a.T - i0) < kW ? (a.T - i0) : kW);
         const uint32_t b = (uint32_t)rowsN * a.h * ES;
         for (int m = 0; m < a.t; ++m) {
-          if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, abort_flag, sg.spin_cap)) { ok = false; break; }
           const uint32_t bar = full0 + 8u * s;
           const uint32_t dst = smem_u32(ring + (size_t)s * sg.stage_bytes);
           const long long off = ((long long)m * a.T + i0) * a.h * ES;
           if constexpr (CL) {
             const uint32_t bP = (uint32_t)rowsN * a.P * ES;                       // 0 when there is no private part
             const uint32_t bS = m == 0 ? (uint32_t)rowsN * a.S_hi * ES : 0u;      // 0 when there is no shared part
-            mbar_expect_tx(bar, b + (has_dh ? 2 : 1) * (bP + bS));
+            mbar_expect_tx(bar, b + (has_dh ? 2 : 1) * (bP + bS) + sg.stall_bytes);
             const long long offp = ((long long)m * a.T + i0) * a.P * ES, offs = i0 * a.S_hi * ES;
             bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
             if (bP) bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + offp, bP, bar);
@@ -345,7 +367,7 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
             if (bS) bulk_g2s(dst + sg.off_d, static_cast<const char*>(a.Hns) + offs, bS, bar);
             if (bS && has_dh) bulk_g2s(dst + sg.off_e, static_cast<const char*>(a.dHns) + offs, bS, bar);
           } else {
-            mbar_expect_tx(bar, has_dh ? 3 * b : 2 * b);
+            mbar_expect_tx(bar, (has_dh ? 3 * b : 2 * b) + sg.stall_bytes);
             bulk_g2s(dst + sg.off_a, static_cast<const char*>(a.dX) + off, b, bar);
             bulk_g2s(dst + sg.off_b, static_cast<const char*>(a.Hn) + off, b, bar);
             if (has_dh) bulk_g2s(dst + sg.off_c, static_cast<const char*>(a.dHn) + off, b, bar);
@@ -410,7 +432,11 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
       char* pdR = CL ? static_cast<char*>(a.dR) + (i * a.P - a.S_lo) * ES : static_cast<char*>(a.dR) + i * a.h * ES;
       char* pZ = static_cast<char*>(a.zp) + (i * a.P - a.S_lo) * ES;
       for (int m = 0; m < a.t; ++m) {
-        if (!mbar_wait(full0 + 8u * s, ph, abort_flag)) { dead = true; break; }
+        if (!mbar_wait(full0 + 8u * s, ph, abort_flag, sg.spin_cap)) {
+          consumer_gave_up(status, 9u, abort_flag, full0, s, ph, NS, lane);
+          dead = true;
+          break;
+        }
         const float rs = __shfl_sync(0xffffffffu, rs_lane, m);
         const float mu = LN ? __shfl_sync(0xffffffffu, mu_lane, m) : 0.f;
         const float2 rs2 = f2(rs);
@@ -573,6 +599,9 @@ WarpGeom warp_geometry(int h, int P, int S_hi, int ES, bool backward, bool has_c
   const size_t acc = backward ? (size_t)kW * h * sizeof(float) : 0;
   if (ring < acc) ring = acc;
   g.smem = g.ring_off + ring;
+  const RowsHooks hooks = rows_hooks();
+  g.spin_cap = hooks.spin_cap;
+  g.stall_bytes = hooks.stall ? 16u : 0u;
   return g;
 }
 
