@@ -495,7 +495,11 @@ caat_status caat_allreduce_bytes(const caat_ctx *ctx, int tokens, int elem_bytes
 
 /* Synchronises `cuda_stream` and reports CAAT_ETIMEOUT if a kernel launched
  * through this library gave up on a bounded wait since the last call of this
- * function, CAAT_ECUDA if the stream is in error, else CAAT_OK. */
+ * function, CAAT_ECUDA if the stream is in error, else CAAT_OK.
+ * The wait limits can be shortened, and a wait made to run out, from the environment
+ * (read once per process; for tests of this path, no effect on a call that returns
+ * CAAT_OK): CAAT_TC_SPINCAP / CAAT_TC_DEBUG=1024 (tensor-core GEMM), CAAT_ROWS_SPINCAP /
+ * CAAT_ROWS_STALL=1 (bulk-copy row kernels), CAAT_TP_POLLCAP (exchange kernels). */
 caat_status caat_last_device_status(const caat_ctx *ctx, void *cuda_stream);
 
 /* Number of kernels launched through this library by the calling process since it
