@@ -430,7 +430,8 @@ __global__ void __launch_bounds__(512) rows_forward_partials_kernel(const RowPar
         hn[e] = (shared_chunk ? z[e] : a.alpha * z[e]) + r[e];
         st[0] = LN ? st[0] + hn[e] : fmaf(hn[e], hn[e], st[0]);
       }
-      if (layer > 0) __syncwarp();
+      // (a thread reads and writes only its own chunks of hrow: no ordering between threads is needed, and a
+      // warp-wide sync here would deadlock rows whose chunk count is not a multiple of 32)
 #pragma unroll
       for (int e = 0; e < V; ++e) hrow[c + e] = hn[e];
       if (a.compact) {      // every rank's CTA forms the same shared values; rank 0's writes them

@@ -199,7 +199,7 @@ rows_forward_warp(const RowFwdArgs a, const WarpGeom sg, int ngroups, unsigned i
     float* rstd_p = a.rstd + i;
     float* mean_p = (LN && a.mean) ? a.mean + i : nullptr;
     for (int m = 0; m < a.t; ++m) {
-      if (!mbar_wait(full0 + 8u * s, ph, abort_flag, sg.spin_cap)) {
+      if (!__all_sync(0xffffffffu, mbar_wait(full0 + 8u * s, ph, abort_flag, sg.spin_cap))) {   // warp-uniform verdict
         consumer_gave_up(status, 8u, abort_flag, full0, s, ph, NS, lane);
         dead = true;
         break;
@@ -432,7 +432,7 @@ rows_backward_warp(const RowBwdArgs a, const WarpGeom sg, int ngroups, unsigned 
       char* pdR = CL ? static_cast<char*>(a.dR) + (i * a.P - a.S_lo) * ES : static_cast<char*>(a.dR) + i * a.h * ES;
       char* pZ = static_cast<char*>(a.zp) + (i * a.P - a.S_lo) * ES;
       for (int m = 0; m < a.t; ++m) {
-        if (!mbar_wait(full0 + 8u * s, ph, abort_flag, sg.spin_cap)) {
+        if (!__all_sync(0xffffffffu, mbar_wait(full0 + 8u * s, ph, abort_flag, sg.spin_cap))) {   // warp-uniform verdict
           consumer_gave_up(status, 9u, abort_flag, full0, s, ph, NS, lane);
           dead = true;
           break;

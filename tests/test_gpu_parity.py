@@ -311,6 +311,42 @@ def test_block_forward_few_tokens(T, p, no_decode):
         assert_close(g, fo[name], "bf16", name)
 
 
+@pytest.mark.timeout(180)
+@pytest.mark.parametrize("t,T,h,ffn,p,norm", [
+    (1, 28, 128, 256, 1.0, 0),      # a single rank (no cluster of ranks): 16 chunks per row, half a warp
+    (16, 20, 896, 1792, 0.5, 1),    # more ranks than a cluster holds; 112 chunks per row: 3 1/2 warps
+    (4, 23, 160, 320, 0.95, 0),     # the cluster kernel on a row of 20 chunks, slices of 5, 5, 5, 4 chunks
+    (2, 64, 96, 192, 0.5, 1)])      # 12 chunks per row
+def test_block_forward_few_tokens_with_rows_that_do_not_fill_their_warps(t, T, h, ffn, p, norm):
+    # two layers in one row-kernel launch, rows whose 16-byte chunks are no multiple of 32: lanes without a chunk skip
+    # the chunk loop, so nothing inside it may synchronise the warp (a sync there deadlocked the second layer)
+    w = synthetic.Workload("blk_dec_small", t, T, h, ffn, p, "bf16", "block", False, 5)
+    S = O.shared_channels(h, p) // 8 * 8
+    d = synthetic.block_inputs(w, S)
+    g = torch.Generator().manual_seed(8)
+    b1 = (0.1 * torch.randn(h, generator=g)).to(torch.bfloat16).cuda() if norm else None
+    b2 = (0.1 * torch.randn(h, generator=g)).to(torch.bfloat16).cuda() if norm else None
+    ctx = G.make_ctx(t, h, ffn, "bf16", S=S, norm=norm)
+    dev = {k: v.cuda() for k, v in d.items()}
+    mk = lambda *s, dt=torch.bfloat16: torch.empty(*s, dtype=dt, device="cuda")
+    o = {"Hn1": mk(t, T, h), "X1": mk(t, T, h), "rstd1": mk(t, T, dt=torch.float32), "Hn2": mk(t, T, h), "X2": mk(t, T, h),
+         "rstd2": mk(t, T, dt=torch.float32)}
+    m1 = mk(t, T, dt=torch.float32) if norm else None
+    m2 = mk(t, T, dt=torch.float32) if norm else None
+    ws = ctx.alloc_workspace(ctx.block_workspace_bytes(T, False))
+    launches = caat.kernel_launches()
+    ctx.block_forward(T, dev["Y_attn"], dev["W_o"], dev["Y_mlp"], dev["W_down"], dev["R0"], dev["gamma1"], b1,
+                      dev["gamma2"], b2, o["Hn1"], o["X1"], o["rstd1"], m1, o["Hn2"], o["X2"], o["rstd2"], m2, ws)
+    torch.cuda.synchronize()
+    assert caat.kernel_launches() - launches == 2          # the weight-streaming GEMM and one row kernel for both layers
+    assert ctx.last_device_status() == caat.CAAT_OK
+    fo = O.block_forward(f64(d["Y_attn"]), f64(d["W_o"]), f64(d["Y_mlp"]), f64(d["W_down"]), f64(d["R0"]), f64(d["gamma1"]),
+                         f64(d["gamma2"]), f64(b1.cpu()) if norm else None, f64(b2.cpu()) if norm else None, S=S,
+                         alpha=math.sqrt(t), norm=norm)
+    for k in o:
+        assert_close(o[k], fo[k], "bf16", k)
+
+
 # ------------------------------------------------------------------ decode shapes (forward only)
 @pytest.mark.parametrize("T", [1, 8, 64])
 @pytest.mark.parametrize("p", [1.0, 0.5])
