@@ -42,8 +42,8 @@
  *              word behind caat_last_device_status (a time-out on any stream of the device
  *              sets it; the call that reads it clears it) and the caat_profile_* benchmark
  *              aid (one recording at a time, not thread-safe).
- *   Limits     h must be a multiple of 8 (CAAT_EUNSUPPORTED otherwise); t divides
- *              h and ffn.  The tensor-core GEMM is used for CAAT_BF16 when K_r and S
+ *   Limits     h must be a multiple of 8 and at most 16384 (bf16) or 8192 (fp32) channels,
+ *              t * tokens at most 2e9 (CAAT_EUNSUPPORTED otherwise); t divides h and ffn.  The tensor-core GEMM is used for CAAT_BF16 when K_r and S
  *              are multiples of 8; other shapes run a slower CUDA-core GEMM.
  */
 #ifndef CAAT_H_
