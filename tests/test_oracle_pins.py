@@ -587,6 +587,27 @@ def test_allreduce_bytes_closed_forms():
     assert O.allreduce_bytes(1, 4096, 8, 4096, 2)["norm_grad_sync_bytes"] == 4096 * 4
 
 
+def test_collective_byte_counts_are_the_sizes_of_the_tensors_the_method_exchanges():
+    # Not the formulas again: the payload is the storage size of the slab the forward really sums over the ranks (the
+    # shared columns of one rank's partial output), and the norm-parameter synchronisation (Eq. 10-11, Section 4) is
+    # the storage size of the fp32 gradient of gamma that the backward really produces.
+    t, T, h, K, S = 4, 37, 96, 8, 40
+    rng = np.random.default_rng(3)
+    Y, W = rng.standard_normal((t, T, K)), rng.standard_normal((t, h, K))
+    R, gamma = rng.standard_normal((t, T, h)), 1 + 0.1 * rng.standard_normal(h)
+    f = O.rowpar_forward(Y, W, R, gamma, None, S=S, alpha=2.0)
+    slab = f["Zt"][0][:, :S]                                           # what one rank contributes to the reduce
+    b = O.rowpar_backward(rng.standard_normal((t, T, h)), None, Y, W, f["Hn"], f["rstd"], None, gamma, S=S, alpha=2.0)
+    for e, dt in ((2, np.float16), (4, np.float32)):
+        a = O.allreduce_bytes(T, h, t, S, e)
+        assert a["payload_per_rank"] == slab.astype(dt).nbytes
+        assert a["payload_per_rank_p1"] == f["Zt"][0].astype(dt).nbytes
+        assert a["norm_grad_sync_bytes"] == b["dgamma"].astype(np.float32).nbytes
+    # the private scale acts on exactly the columns the reduce leaves out: alpha times the rank's own partial there
+    assert np.array_equal(f["Z"][1][:, S:], 2.0 * f["Zt"][1][:, S:])
+    assert np.allclose(f["Z"][1][:, :S], f["Zt"][:, :, :S].sum(0))
+
+
 def test_speedup_model_closed_form():
     # Appendix C: (T(1) - T(p)) / T(1) = (1 - p) / (1 + (12 h + 2 s) / (C r)).
     for h, s, r, C, p in [(4096, 2048, 8, 3000.0, 0.5), (768, 1024, 16, 500.0, 0.25), (2048, 2048, 4, 8000.0, 0.75)]:
